@@ -1,0 +1,218 @@
+"""CPU oracle for MVUE N:M gradient pruning and the products that consume it.
+
+TEST INFRASTRUCTURE ONLY: a plain, slow statement of what the method computes,
+written from the paper.  Only the tests, the smoke check and the benchmark's
+CPU-baseline leg may import this package; the CUDA library never does, and the
+two share no code.
+
+`mvue_oracle.c` holds the arithmetic (binary32, fixed order, no fused
+multiply-add); this module compiles it with gcc on first use and exposes it
+through ctypes with numpy arrays.  `theory.py` holds the binary64 closed forms
+of the paper (probabilities, marginals, variances) that pin the sampler.
+`philox_py.py` is an independent big-integer restatement of the generator.
+"""
+from __future__ import annotations
+
+import ctypes
+import os
+import subprocess
+from pathlib import Path
+
+import numpy as np
+
+_HERE = Path(__file__).resolve().parent
+_SRC = _HERE / "mvue_oracle.c"
+_LIB = _HERE / "_build" / "libmvue_oracle.so"
+
+_CFLAGS = ["-O2", "-ffp-contract=off", "-fno-fast-math", "-std=c11", "-fPIC", "-shared", "-fopenmp"]
+
+
+def build(force: bool = False) -> Path:
+    """Compile the C oracle (gcc, no fast-math, no FMA contraction)."""
+    if force or not _LIB.exists() or _LIB.stat().st_mtime < _SRC.stat().st_mtime:
+        _LIB.parent.mkdir(exist_ok=True)
+        tmp = _LIB.with_suffix(f".{os.getpid()}.tmp")
+        subprocess.run(["gcc", *_CFLAGS, str(_SRC), "-o", str(tmp), "-lm"], check=True)
+        os.replace(tmp, _LIB)
+    return _LIB
+
+
+_lib = None
+
+
+def lib() -> ctypes.CDLL:
+    global _lib
+    if _lib is None:
+        L = ctypes.CDLL(str(build()))
+        u32p = ctypes.POINTER(ctypes.c_uint32)
+        L.oracle_philox4x32_10.argtypes = [u32p, u32p, u32p]
+        L.oracle_philox4x32_10.restype = None
+        L.oracle_block_word.argtypes = [ctypes.c_uint64, ctypes.c_uint64]
+        L.oracle_block_word.restype = ctypes.c_uint32
+        L.oracle_uniform24.argtypes = [ctypes.c_uint32]
+        L.oracle_uniform24.restype = ctypes.c_float
+        L.oracle_bf16_rne.argtypes = [ctypes.c_float]
+        L.oracle_bf16_rne.restype = ctypes.c_uint16
+        L.oracle_bf16_to_f32.argtypes = [ctypes.c_uint16]
+        L.oracle_bf16_to_f32.restype = ctypes.c_float
+        L.oracle_mvue_1of2.argtypes = [ctypes.c_float, ctypes.c_float, ctypes.c_uint32,
+                                       ctypes.POINTER(ctypes.c_float)]
+        L.oracle_mvue_1of2.restype = ctypes.c_int
+        L.oracle_mvue_2of4.argtypes = [ctypes.POINTER(ctypes.c_float), ctypes.c_uint32,
+                                       ctypes.POINTER(ctypes.c_int), ctypes.POINTER(ctypes.c_float)]
+        L.oracle_mvue_2of4.restype = None
+        L.oracle_prune.argtypes = [ctypes.c_void_p, ctypes.c_int, ctypes.c_int64, ctypes.c_int64,
+                                   ctypes.c_int64, ctypes.c_int, ctypes.c_int, ctypes.c_int,
+                                   ctypes.c_uint64, ctypes.c_int64, ctypes.c_int64,
+                                   ctypes.c_void_p, ctypes.c_void_p, ctypes.c_int]
+        L.oracle_prune.restype = ctypes.c_int
+        L.oracle_unpack.argtypes = [ctypes.c_void_p, ctypes.c_void_p, ctypes.c_int64, ctypes.c_int64,
+                                    ctypes.c_void_p]
+        L.oracle_unpack.restype = None
+        L.oracle_gemm.argtypes = [ctypes.c_void_p, ctypes.c_int64, ctypes.c_int64, ctypes.c_void_p,
+                                  ctypes.c_int64, ctypes.c_int64, ctypes.c_void_p, ctypes.c_int64,
+                                  ctypes.c_void_p, ctypes.c_int]
+        L.oracle_gemm.restype = None
+        L.oracle_gemm_entry.argtypes = [ctypes.c_void_p, ctypes.c_int64, ctypes.c_void_p,
+                                        ctypes.c_int64, ctypes.c_int64]
+        L.oracle_gemm_entry.restype = ctypes.c_double
+        L.oracle_sweep_2of4.argtypes = [ctypes.POINTER(ctypes.c_float), ctypes.POINTER(ctypes.c_uint64),
+                                        ctypes.POINTER(ctypes.c_double), ctypes.POINTER(ctypes.c_double)]
+        L.oracle_sweep_2of4.restype = None
+        L.oracle_sweep_1of2.argtypes = [ctypes.c_float, ctypes.c_float, ctypes.POINTER(ctypes.c_uint64),
+                                        ctypes.POINTER(ctypes.c_double), ctypes.POINTER(ctypes.c_double)]
+        L.oracle_sweep_1of2.restype = None
+        _lib = L
+    return _lib
+
+
+def host_threads() -> int:
+    return len(os.sched_getaffinity(0))
+
+
+# --------------------------------------------------------------------------
+# thin numpy wrappers
+# --------------------------------------------------------------------------
+def philox4x32_10(ctr, key):
+    c = (ctypes.c_uint32 * 4)(*[int(x) & 0xFFFFFFFF for x in ctr])
+    k = (ctypes.c_uint32 * 2)(*[int(x) & 0xFFFFFFFF for x in key])
+    o = (ctypes.c_uint32 * 4)()
+    lib().oracle_philox4x32_10(c, k, o)
+    return tuple(int(x) for x in o)
+
+
+def block_word(seed: int, q: int) -> int:
+    return int(lib().oracle_block_word(seed & (2**64 - 1), q))
+
+
+def uniform24(word: int) -> float:
+    return float(lib().oracle_uniform24(word & 0xFFFFFFFF))
+
+
+def bf16_rne(x: np.ndarray) -> np.ndarray:
+    """binary32 array -> bf16 bit patterns (uint16), element by element."""
+    x = np.ascontiguousarray(x, dtype=np.float32)
+    f = lib().oracle_bf16_rne
+    return np.fromiter((f(float(v)) for v in x.ravel()), dtype=np.uint16, count=x.size).reshape(x.shape)
+
+
+def bf16_to_f32(h: np.ndarray) -> np.ndarray:
+    h = np.ascontiguousarray(h, dtype=np.uint16)
+    return (h.astype(np.uint32) << 16).view(np.float32)
+
+
+def mvue_1of2(a1: float, a2: float, word: int):
+    kept = ctypes.c_float()
+    idx = lib().oracle_mvue_1of2(a1, a2, word & 0xFFFFFFFF, ctypes.byref(kept))
+    return int(idx), float(kept.value)
+
+
+def mvue_2of4(a, word: int):
+    arr = (ctypes.c_float * 4)(*[float(x) for x in a])
+    idx = (ctypes.c_int * 2)()
+    val = (ctypes.c_float * 2)()
+    lib().oracle_mvue_2of4(arr, word & 0xFFFFFFFF, idx, val)
+    return (int(idx[0]), int(idx[1])), (float(val[0]), float(val[1]))
+
+
+def packed_shapes(rows: int, cols: int, axis: int):
+    mrows, k = (rows, cols) if axis == 1 else (cols, rows)
+    return (mrows, k // 2), (mrows, k // 8)
+
+
+def prune(g: np.ndarray, n: int, m: int, axis: int, seed: int, *, k_total: int | None = None,
+          k_offset: int = 0, threads: int = 1):
+    """MVUE n:m prune + pack of a 2-D array (float32, or uint16 holding bf16 bits).
+
+    Returns (values uint16 [Mrows, K/2], meta uint8 [Mrows, K/8]) in canonical form.
+    """
+    assert g.ndim == 2 and g.dtype in (np.float32, np.uint16)
+    g = np.ascontiguousarray(g)
+    rows, cols = g.shape
+    vshape, mshape = packed_shapes(rows, cols, axis)
+    k = cols if axis == 1 else rows
+    values = np.zeros(vshape, dtype=np.uint16)
+    meta = np.zeros(mshape, dtype=np.uint8)
+    rc = lib().oracle_prune(g.ctypes.data, int(g.dtype == np.uint16), rows, cols, cols, n, m, axis,
+                            seed & (2**64 - 1), k if k_total is None else k_total, k_offset,
+                            values.ctypes.data, meta.ctypes.data, max(1, threads))
+    if rc != 0:
+        raise ValueError("oracle_prune: unsupported N:M or shape")
+    return values, meta
+
+
+def unpack(values: np.ndarray, meta: np.ndarray) -> np.ndarray:
+    """Canonical packed operand -> dense float32 A[Mrows, K]."""
+    values = np.ascontiguousarray(values, dtype=np.uint16)
+    meta = np.ascontiguousarray(meta, dtype=np.uint8)
+    mrows, kh = values.shape
+    dense = np.empty((mrows, 2 * kh), dtype=np.float32)
+    lib().oracle_unpack(values.ctypes.data, meta.ctypes.data, mrows, 2 * kh, dense.ctypes.data)
+    return dense
+
+
+def gemm(A: np.ndarray, B: np.ndarray, E: np.ndarray | None = None, threads: int = 1) -> np.ndarray:
+    """C = A @ B (* E), A float32 [M,K], B / E uint16 bf16 bits [K,N] / [M,N]; float64 result."""
+    A = np.ascontiguousarray(A, dtype=np.float32)
+    B = np.ascontiguousarray(B, dtype=np.uint16)
+    M, K = A.shape
+    assert B.shape[0] == K
+    N = B.shape[1]
+    C = np.empty((M, N), dtype=np.float64)
+    if E is not None:
+        E = np.ascontiguousarray(E, dtype=np.uint16)
+        assert E.shape == (M, N)
+    lib().oracle_gemm(A.ctypes.data, M, K, B.ctypes.data, N, N,
+                      None if E is None else E.ctypes.data, N, C.ctypes.data, max(1, threads))
+    return C
+
+
+def gemm_entry(A_row: np.ndarray, B: np.ndarray, j: int) -> float:
+    A_row = np.ascontiguousarray(A_row, dtype=np.float32)
+    B = np.ascontiguousarray(B, dtype=np.uint16)
+    return float(lib().oracle_gemm_entry(A_row.ctypes.data, A_row.size, B.ctypes.data, B.shape[1], j))
+
+
+PAIRS = ((0, 1), (0, 2), (0, 3), (1, 2), (1, 3), (2, 3))
+
+
+def sweep_2of4(a):
+    """Frequencies of the six outcomes, mean of theta(a) and block variance over all 2^24 eps."""
+    arr = (ctypes.c_float * 4)(*[float(x) for x in a])
+    counts = (ctypes.c_uint64 * 6)()
+    sums = (ctypes.c_double * 4)()
+    sq = ctypes.c_double()
+    lib().oracle_sweep_2of4(arr, counts, sums, ctypes.byref(sq))
+    n = float(1 << 24)
+    return (np.array([c for c in counts], dtype=np.float64) / n,
+            np.array([s for s in sums]) / n, sq.value / n)
+
+
+def sweep_1of2(a1: float, a2: float):
+    counts = (ctypes.c_uint64 * 2)()
+    sums = (ctypes.c_double * 2)()
+    sq = ctypes.c_double()
+    lib().oracle_sweep_1of2(a1, a2, counts, sums, ctypes.byref(sq))
+    n = float(1 << 24)
+    return (np.array([c for c in counts], dtype=np.float64) / n,
+            np.array([s for s in sums]) / n, sq.value / n)

@@ -1,0 +1,387 @@
+/*
+ * CPU oracle for minimum-variance unbiased (MVUE) N:M pruning of a neural
+ * gradient and for the matrix products that consume the pruned operand.
+ *
+ * TEST INFRASTRUCTURE ONLY.  This file is the slow, plain statement of what
+ * the method computes.  It shares no code with the CUDA library and must never
+ * be linked into, imported by, or called from the product path.
+ *
+ * Every floating-point step of the selection is IEEE binary32, round to
+ * nearest even, evaluated in exactly the order written.  Build with
+ * -ffp-contract=off so the compiler never fuses a multiply with an add, and
+ * without any fast-math option.
+ *
+ * Notation follows the paper: a block a = [a_1..a_M], theta(a) the pruned
+ * block, p_i the probability that element i survives, p_ij the probability
+ * that the pair (i, j) survives (indices refer to the block sorted by
+ * magnitude, a_1 <= a_2 <= a_3 <= a_4).
+ *
+ * Parity pins (see tests): Philox against two independent implementations;
+ * the 1:2 sampler against the closed form of Sec. 4.1; the 2:4 sampler against
+ * the pair table of App. A.2 and the optimal marginals of Sec. 4.2 by an
+ * exhaustive sweep over every value of the 24-bit uniform; bf16 rounding
+ * against a library cast; the product against a library fp64 matmul.
+ */
+#include <math.h>
+#include <stddef.h>
+#include <stdint.h>
+#include <string.h>
+
+/* ------------------------------------------------------------------------
+ * Counter-based random numbers: Philox4x32 with ten rounds (Salmon, Moraes,
+ * Dror, Shaw, "Parallel random numbers: as easy as 1, 2, 3", SC'11).
+ * The paper only asks for i.i.d. eps ~ U[0,1] (App. "Pruning Overhead",
+ * Part 1); a counter-based generator keyed by (seed, block index) makes every
+ * block's draw a pure function of its position.
+ * ---------------------------------------------------------------------- */
+void oracle_philox4x32_10(const uint32_t ctr[4], const uint32_t key[2], uint32_t out[4])
+{
+    const uint64_t mult0 = 0xD2511F53u;    /* multiplies counter word 0 */
+    const uint64_t mult1 = 0xCD9E8D57u;    /* multiplies counter word 2 */
+    const uint32_t bump0 = 0x9E3779B9u;    /* added to key word 0 after each round */
+    const uint32_t bump1 = 0xBB67AE85u;    /* added to key word 1 after each round */
+    uint32_t c0 = ctr[0], c1 = ctr[1], c2 = ctr[2], c3 = ctr[3];
+    uint32_t k0 = key[0], k1 = key[1];
+    for (int round = 0; round < 10; ++round) {
+        uint64_t prod0 = mult0 * (uint64_t)c0;
+        uint64_t prod1 = mult1 * (uint64_t)c2;
+        uint32_t hi0 = (uint32_t)(prod0 >> 32), lo0 = (uint32_t)prod0;
+        uint32_t hi1 = (uint32_t)(prod1 >> 32), lo1 = (uint32_t)prod1;
+        uint32_t n0 = hi1 ^ c1 ^ k0;
+        uint32_t n1 = lo1;
+        uint32_t n2 = hi0 ^ c3 ^ k1;
+        uint32_t n3 = lo0;
+        c0 = n0; c1 = n1; c2 = n2; c3 = n3;
+        k0 += bump0;
+        k1 += bump1;
+    }
+    out[0] = c0; out[1] = c1; out[2] = c2; out[3] = c3;
+}
+
+/* The 32-bit word that drives block number q (q counts blocks of the whole
+ * operand, row by row): one generator call serves four consecutive blocks. */
+uint32_t oracle_block_word(uint64_t seed, uint64_t q)
+{
+    uint64_t call = q >> 2;
+    uint32_t ctr[4] = { (uint32_t)call, (uint32_t)(call >> 32), 0u, 0u };
+    uint32_t key[2] = { (uint32_t)seed, (uint32_t)(seed >> 32) };
+    uint32_t out[4];
+    oracle_philox4x32_10(ctr, key, out);
+    return out[q & 3u];
+}
+
+/* eps in [0,1): the top 24 bits of the word, exactly representable. */
+float oracle_uniform24(uint32_t word)
+{
+    return (float)(word >> 8) * 5.9604644775390625e-08f;   /* 2^-24 */
+}
+
+/* ------------------------------------------------------------------------
+ * bf16 storage: round a binary32 value to the nearest bfloat16, ties to even,
+ * by integer arithmetic on the bit pattern.  Inputs are finite.
+ * ---------------------------------------------------------------------- */
+uint16_t oracle_bf16_rne(float x)
+{
+    uint32_t bits;
+    memcpy(&bits, &x, 4);
+    uint32_t lsb = (bits >> 16) & 1u;
+    bits += 0x7FFFu + lsb;
+    return (uint16_t)(bits >> 16);
+}
+
+float oracle_bf16_to_f32(uint16_t h)
+{
+    uint32_t bits = (uint32_t)h << 16;
+    float x;
+    memcpy(&x, &bits, 4);
+    return x;
+}
+
+/* ------------------------------------------------------------------------
+ * MVUE 1:2 (Sec. 4.1, the estimator that closes that section; derivation in
+ * App. A.1): keep a_1 with probability |a_1| / (|a_1| + |a_2|), else a_2; the
+ * survivor becomes sign(a_i) (|a_1| + |a_2|).  The draw is the threshold test
+ * eps < p_1 (App. "Pruning Overhead", Part 1) written without the division:
+ * eps (|a_1|+|a_2|) < |a_1|.
+ * Zero rules (the paper leaves 0/0 open): a zero is never preferred to a
+ * non-zero; an all-zero block keeps element 0 with value +0.
+ * Returns the kept index (0 or 1); *kept receives the new value.
+ * ---------------------------------------------------------------------- */
+int oracle_mvue_1of2(float a1, float a2, uint32_t word, float *kept)
+{
+    float m1 = fabsf(a1), m2 = fabsf(a2);
+    float S = m1 + m2;
+    int idx;
+    if (m1 == 0.0f && m2 == 0.0f) { *kept = 0.0f; return 0; }
+    if (m2 == 0.0f) idx = 0;
+    else if (m1 == 0.0f) idx = 1;
+    else {
+        float eps = oracle_uniform24(word);
+        float t = eps * S;
+        idx = (t < m1) ? 0 : 1;
+    }
+    *kept = copysignf(S, idx == 0 ? a1 : a2);
+    return idx;
+}
+
+/* ------------------------------------------------------------------------
+ * MVUE 2:4 (optimal marginals: Sec. 4.2; joint law over pairs: App. A.2).
+ *
+ * 1. Sort the magnitudes ascending, ties by original position:
+ *      s_1 <= s_2 <= s_3 <= s_4, original indices i_1..i_4.
+ * 2. Case 3 (s_4 >= s_1+s_2+s_3): the dominant element survives with
+ *    probability one and keeps its value (a_i / p_i with p_i = 1); one of the
+ *    other three survives with probability s_k / (s_1+s_2+s_3) and becomes
+ *    sign(a) (s_1+s_2+s_3).
+ *    Case 1 (s_4 <= 2 s_1 + s_3) and case 2 (otherwise): the pair (i, j)
+ *    survives with the probability p_ij of the appendix table; both survivors
+ *    become a_i / p_i with p_i = 2 s_i / sum, i.e. sign(a_i) sum / 2.
+ * 3. The pair is drawn by walking the cumulative table in the fixed order
+ *    13, 14, 23, 24, 34 with eps scaled by the table's common denominator, so
+ *    no division appears.  A numerator that rounding pushes below zero is
+ *    clamped to zero.
+ * Zero rules: an element of magnitude zero survives only if fewer than two
+ * non-zeros exist, and then with value +0 (lowest free positions).
+ *
+ * idx[0] < idx[1] are the surviving original positions, val[] their new
+ * values in that order.
+ * ---------------------------------------------------------------------- */
+static float clamp0(float x) { return x < 0.0f ? 0.0f : x; }
+
+void oracle_mvue_2of4(const float a[4], uint32_t word, int idx[2], float val[2])
+{
+    float s[4];
+    int   pos[4];
+    /* insertion sort on (magnitude, position); strict '<' keeps ties stable */
+    for (int i = 0; i < 4; ++i) {
+        float m = fabsf(a[i]);
+        int j = i;
+        while (j > 0 && m < s[j - 1]) { s[j] = s[j - 1]; pos[j] = pos[j - 1]; --j; }
+        s[j] = m; pos[j] = i;
+    }
+    const float s1 = s[0], s2 = s[1], s3 = s[2], s4 = s[3];
+    const float S3 = (s1 + s2) + s3;
+    const float S  = S3 + s4;
+    const float eps = oracle_uniform24(word);
+
+    int   ka, kb;          /* sorted ranks (0..3) of the two survivors */
+    float va, vb;          /* their new values */
+
+    if (s4 == 0.0f) {                       /* nothing to keep */
+        idx[0] = 0; idx[1] = 1; val[0] = 0.0f; val[1] = 0.0f;
+        return;
+    }
+    if (s4 >= S3) {                         /* case 3 */
+        kb = 3; vb = a[pos[3]];
+        if (S3 == 0.0f) {                   /* a single non-zero in the block */
+            int other = (pos[3] == 0) ? 1 : 0;
+            if (other < pos[3]) { idx[0] = other; idx[1] = pos[3]; val[0] = 0.0f; val[1] = vb; }
+            else                { idx[0] = pos[3]; idx[1] = other; val[0] = vb; val[1] = 0.0f; }
+            return;
+        }
+        float t = eps * S3;
+        if (t < s1) ka = 0;
+        else if (t < s1 + s2) ka = 1;
+        else ka = 2;
+        va = copysignf(S3, a[pos[ka]]);
+    } else {
+        float w13, w14, w23, w24, denom;
+        if (s4 <= (s1 + s1) + s3) {         /* case 1: numerators over 2 * sum */
+            w13 = clamp0(((s1 + s1) + s3) - s4);
+            w14 = clamp0(((s1 + s1) - s3) + s4);
+            w23 = clamp0(((s2 + s2) + s3) - s4);
+            w24 = clamp0(((s2 + s2) - s3) + s4);
+            denom = S + S;
+        } else {                            /* case 2: numerators over sum */
+            w13 = 0.0f;
+            w14 = s1 + s1;
+            w23 = clamp0(S3 - s4);
+            w24 = clamp0((s2 - s1) + (s4 - s3));
+            denom = S;
+        }
+        float t = eps * denom;
+        float c = w13;
+        if (t < c) { ka = 0; kb = 2; }
+        else {
+            c = c + w14;
+            if (t < c) { ka = 0; kb = 3; }
+            else {
+                c = c + w23;
+                if (t < c) { ka = 1; kb = 2; }
+                else {
+                    c = c + w24;
+                    if (t < c) { ka = 1; kb = 3; }
+                    else       { ka = 2; kb = 3; }
+                }
+            }
+        }
+        float half = 0.5f * S;
+        va = copysignf(half, a[pos[ka]]);
+        vb = copysignf(half, a[pos[kb]]);
+    }
+    if (pos[ka] < pos[kb]) { idx[0] = pos[ka]; idx[1] = pos[kb]; val[0] = va; val[1] = vb; }
+    else                   { idx[0] = pos[kb]; idx[1] = pos[ka]; val[0] = vb; val[1] = va; }
+}
+
+/* ------------------------------------------------------------------------
+ * Tensor-wide prune and pack.
+ *
+ * g is a row-major [rows x cols] matrix with leading dimension ld, fp32
+ * (is_bf16 = 0) or bf16 bit patterns (is_bf16 = 1; widened exactly).
+ * The sparse operand is A[Mrows x K] with K the reduction axis of the GEMM
+ * that will consume it: axis = 1 -> A = g (blocks along a row of g),
+ * axis = 0 -> A = g^T (blocks run down a column of g).
+ * Blocks are M contiguous elements along K (Sec. 1; Sec. 4).
+ *
+ * Block numbering: row r of A owns k_total/M consecutive numbers; k_offset is
+ * the global K position of this tensor's first element (0 unless the K axis
+ * is sharded), so a shard draws the same words as the whole tensor would.
+ *
+ * Output (canonical packed form):
+ *   values[Mrows x K/2]  bf16, the survivors in ascending position;
+ *   meta  [Mrows x K/8]  bytes; each nibble = idx0 | idx1 << 2 for one group
+ *                        of four, low nibble = even group.
+ * A 1:2 result is written as a valid 2:4 pattern: the pair (4j, 4j+1) gives
+ * idx0 in {0,1}, the pair (4j+2, 4j+3) gives idx1 in {2,3}.
+ * Returns 0, or -1 for an unsupported shape.
+ * ---------------------------------------------------------------------- */
+static float load_elem(const void *g, int is_bf16, int64_t off)
+{
+    if (is_bf16) return oracle_bf16_to_f32(((const uint16_t *)g)[off]);
+    return ((const float *)g)[off];
+}
+
+int oracle_prune(const void *g, int is_bf16, int64_t rows, int64_t cols, int64_t ld,
+                 int n, int m, int axis, uint64_t seed, int64_t k_total, int64_t k_offset,
+                 uint16_t *values, uint8_t *meta, int threads)
+{
+    const int64_t Mrows = axis == 1 ? rows : cols;
+    const int64_t K     = axis == 1 ? cols : rows;
+    if (!((n == 1 && m == 2) || (n == 2 && m == 4))) return -1;
+    if (K % 8 != 0 || k_total % 8 != 0 || k_offset % 8 != 0 || k_offset + K > k_total) return -1;
+    (void)threads;
+#pragma omp parallel for num_threads(threads) schedule(static)
+    for (int64_t r = 0; r < Mrows; ++r) {
+        for (int64_t j = 0; j < K / 4; ++j) {           /* j: group of four along K */
+            float a[4];
+            for (int e = 0; e < 4; ++e) {
+                int64_t k = 4 * j + e;
+                int64_t off = axis == 1 ? r * ld + k : k * ld + r;
+                a[e] = load_elem(g, is_bf16, off);
+            }
+            int idx[2]; float val[2];
+            if (m == 4) {
+                uint64_t q = (uint64_t)r * (uint64_t)(k_total / 4) + (uint64_t)(k_offset / 4 + j);
+                oracle_mvue_2of4(a, oracle_block_word(seed, q), idx, val);
+            } else {
+                for (int half = 0; half < 2; ++half) {
+                    uint64_t q = (uint64_t)r * (uint64_t)(k_total / 2)
+                               + (uint64_t)(k_offset / 2 + 2 * j + half);
+                    idx[half] = 2 * half + oracle_mvue_1of2(a[2 * half], a[2 * half + 1],
+                                                            oracle_block_word(seed, q), &val[half]);
+                }
+            }
+            values[r * (K / 2) + 2 * j]     = oracle_bf16_rne(val[0]);
+            values[r * (K / 2) + 2 * j + 1] = oracle_bf16_rne(val[1]);
+            uint8_t nib = (uint8_t)(idx[0] | (idx[1] << 2));
+            uint8_t *byte = &meta[r * (K / 8) + j / 2];
+            if (j % 2 == 0) *byte = (uint8_t)((*byte & 0xF0u) | nib);
+            else            *byte = (uint8_t)((*byte & 0x0Fu) | (nib << 4));
+        }
+    }
+    return 0;
+}
+
+/* Expand the canonical packed form back to a dense fp32 A[Mrows x K]. */
+void oracle_unpack(const uint16_t *values, const uint8_t *meta, int64_t Mrows, int64_t K,
+                   float *dense)
+{
+    for (int64_t r = 0; r < Mrows; ++r) {
+        for (int64_t j = 0; j < K / 4; ++j) {
+            uint8_t byte = meta[r * (K / 8) + j / 2];
+            uint8_t nib = (j % 2 == 0) ? (byte & 0x0Fu) : (byte >> 4);
+            float *out = &dense[r * K + 4 * j];
+            out[0] = out[1] = out[2] = out[3] = 0.0f;
+            /* written in this order so that a malformed nibble with equal
+             * indices still yields a defined result (second value wins) */
+            out[nib & 3u]        = oracle_bf16_to_f32(values[r * (K / 2) + 2 * j]);
+            out[(nib >> 2) & 3u] = oracle_bf16_to_f32(values[r * (K / 2) + 2 * j + 1]);
+        }
+    }
+}
+
+/* ------------------------------------------------------------------------
+ * Matrix product that consumes the pruned operand (Sec. 1: the update
+ * dC/dW_l = g_l h_{l-1}^T and the backward product W^T g).
+ *   C[M x N] = A[M x K] . B[K x N]  (+ elementwise * E[M x N] if E != NULL)
+ * A is the dense expansion of the packed operand (fp32), B and E hold bf16 bit
+ * patterns, row-major with leading dimensions ldb / lde.  Plain triple loop,
+ * accumulated in binary64.  Update: A = theta(g)^T, B = h.  Backward:
+ * A = theta(g), B = W, E = f'(z).
+ * ---------------------------------------------------------------------- */
+void oracle_gemm(const float *A, int64_t M, int64_t K, const uint16_t *B, int64_t N, int64_t ldb,
+                 const uint16_t *E, int64_t lde, double *C, int threads)
+{
+    (void)threads;
+#pragma omp parallel for num_threads(threads) schedule(static)
+    for (int64_t i = 0; i < M; ++i) {
+        for (int64_t j = 0; j < N; ++j) {
+            double acc = 0.0;
+            for (int64_t k = 0; k < K; ++k)
+                acc += (double)A[i * K + k] * (double)oracle_bf16_to_f32(B[k * ldb + j]);
+            if (E) acc *= (double)oracle_bf16_to_f32(E[i * lde + j]);
+            C[i * N + j] = acc;
+        }
+    }
+}
+
+/* One output entry of the same product, for sampled checks at sizes where the
+ * full triple loop is too slow. */
+double oracle_gemm_entry(const float *A_row, int64_t K, const uint16_t *B, int64_t ldb, int64_t j)
+{
+    double acc = 0.0;
+    for (int64_t k = 0; k < K; ++k)
+        acc += (double)A_row[k] * (double)oracle_bf16_to_f32(B[k * ldb + j]);
+    return acc;
+}
+
+/* ------------------------------------------------------------------------
+ * Exhaustive sweep helper for the pins: run the block sampler for every one
+ * of the 2^24 values eps can take and count how often each outcome occurs.
+ * 2:4: counts[6] over the position pairs (0,1),(0,2),(0,3),(1,2),(1,3),(2,3)
+ * of the ORIGINAL block; sum_val[4] accumulates theta(a) per position;
+ * sum_sq accumulates |theta(a) - a|^2.  1:2: counts[0..1], sum_val[0..1].
+ * ---------------------------------------------------------------------- */
+void oracle_sweep_2of4(const float a[4], uint64_t counts[6], double sum_val[4], double *sum_sq)
+{
+    static const int pair_id[4][4] = { { -1, 0, 1, 2 }, { 0, -1, 3, 4 }, { 1, 3, -1, 5 }, { 2, 4, 5, -1 } };
+    for (int i = 0; i < 6; ++i) counts[i] = 0;
+    for (int i = 0; i < 4; ++i) sum_val[i] = 0.0;
+    *sum_sq = 0.0;
+    for (uint32_t n = 0; n < (1u << 24); ++n) {
+        int idx[2]; float val[2];
+        oracle_mvue_2of4(a, n << 8, idx, val);
+        counts[pair_id[idx[0]][idx[1]]] += 1;
+        double th[4] = { 0, 0, 0, 0 };
+        th[idx[0]] = val[0]; th[idx[1]] = val[1];
+        for (int i = 0; i < 4; ++i) {
+            sum_val[i] += th[i];
+            double d = th[i] - (double)a[i];
+            *sum_sq += d * d;
+        }
+    }
+}
+
+void oracle_sweep_1of2(float a1, float a2, uint64_t counts[2], double sum_val[2], double *sum_sq)
+{
+    counts[0] = counts[1] = 0; sum_val[0] = sum_val[1] = 0.0; *sum_sq = 0.0;
+    for (uint32_t n = 0; n < (1u << 24); ++n) {
+        float kept;
+        int idx = oracle_mvue_1of2(a1, a2, n << 8, &kept);
+        counts[idx] += 1;
+        double th[2] = { 0, 0 };
+        th[idx] = kept;
+        sum_val[0] += th[0]; sum_val[1] += th[1];
+        *sum_sq += (th[0] - (double)a1) * (th[0] - (double)a1) + (th[1] - (double)a2) * (th[1] - (double)a2);
+    }
+}
