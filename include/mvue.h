@@ -1,0 +1,125 @@
+/*
+ * mvue.h -- C ABI of the B200 (sm_100a) library for minimum-variance unbiased
+ * (MVUE) N:M pruning of neural gradients and the 2:4-sparse matrix products that
+ * consume the pruned gradient.
+ *
+ * Method: Chmiel, Hubara, Banner, Soudry, "Minimum Variance Unbiased N:M
+ * Sparsity for the Neural Gradients" (arXiv 2203.10991).  Citations below name
+ * the paper's sections, equations and appendices.
+ *
+ * General rules for every call
+ *  - All tensor pointers are DEVICE pointers unless an argument says "host".
+ *    The caller owns every buffer; the library never allocates or frees device
+ *    memory and keeps no device state.
+ *  - `stream` is a cudaStream_t passed as void* (NULL = the legacy default
+ *    stream).  Calls enqueue work on that stream and return without waiting.
+ *  - The return value is an mvue_status.  Argument errors are detected on the
+ *    host before anything is launched; nothing is written in that case.
+ *    Nothing throws, aborts or traps across this boundary.
+ *  - Matrices are row-major; leading dimensions are in ELEMENTS.
+ *  - The device must be compute capability 10.x; otherwise MVUE_ERR_ARCH.
+ *  - Inputs must be finite with |x| <= 2^125; other values give unspecified
+ *    results but never an out-of-bounds access.
+ */
+#ifndef MVUE_H_
+#define MVUE_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#if defined(__GNUC__)
+#define MVUE_API __attribute__((visibility("default")))
+#else
+#define MVUE_API
+#endif
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef enum {
+    MVUE_OK = 0,
+    MVUE_ERR_NULL = -1,           /* a required pointer is NULL */
+    MVUE_ERR_NM = -2,             /* only (N,M) = (1,2) and (2,4) exist */
+    MVUE_ERR_SHAPE = -3,          /* non-positive / non-multiple extents, ld < cols, bad axis or K shard */
+    MVUE_ERR_ALIGN = -4,          /* base pointer or leading dimension not 16-byte aligned */
+    MVUE_ERR_DTYPE = -5,
+    MVUE_ERR_LAYOUT = -6,
+    MVUE_ERR_WORKSPACE = -7,      /* workspace NULL or smaller than mvue_gemm_workspace_bytes */
+    MVUE_ERR_ARCH = -8,           /* current device is not sm_100 */
+    MVUE_ERR_CUDA = -9,           /* a CUDA runtime/driver call failed; text in mvue_last_cuda_error() */
+    MVUE_ERR_DEVICE_TIMEOUT = -10 /* only ever written to a device status word: a bounded wait expired */
+} mvue_status;
+
+typedef enum { MVUE_F32 = 0, MVUE_BF16 = 1 } mvue_dtype;
+
+/* Packed operand layouts.
+ * MVUE_LAYOUT_CANONICAL: for the sparse operand A[Mrows x K] (K = pruned axis)
+ *   values: bf16 [Mrows x K/2] row-major -- the two survivors of each group of
+ *           four consecutive k, in ascending k;
+ *   meta:   bytes [Mrows x K/8] row-major -- one nibble per group,
+ *           idx0 | idx1 << 2 with idx0 < idx1 the survivors' positions in the
+ *           group, low nibble = even group.  (The 2-bit-per-survivor encoding
+ *           of 2:4 sparse tensor cores.)
+ *   This is also what the GEMM entry points consume. */
+typedef enum { MVUE_LAYOUT_CANONICAL = 0 } mvue_layout;
+
+/* Bytes of the packed outputs of mvue_prune for a [rows x cols] input.
+ * values_bytes / meta_bytes are HOST pointers (either may be NULL). */
+MVUE_API int mvue_packed_sizes(int64_t rows, int64_t cols, int n, int m, int axis, int layout,
+                      size_t* values_bytes, size_t* meta_bytes);
+
+/* MVUE N:M prune + pack of a neural gradient g in one pass.
+ *
+ * What it computes.  Each block of M elements that are contiguous along the
+ * reduction axis K of the GEMM that will consume g is replaced by an unbiased,
+ * minimum-variance N:M-sparse block theta(a), E[theta(a)] = a:
+ *   (1,2): Sec. 4.1, closing equation (derivation App. A.1): a_1 survives with
+ *          probability |a_1|/(|a_1|+|a_2|), else a_2; the survivor becomes
+ *          sign(a_i)(|a_1|+|a_2|).
+ *   (2,4): Sec. 4.2 (optimal survival probabilities p_i, survivors a_i/p_i) with
+ *          the joint law over pairs of App. A.2 (three cases on the sorted
+ *          magnitudes), drawn by walking the cumulative pair table in the order
+ *          13, 14, 23, 24, 34.
+ * The draw is the threshold test eps < p of App. "Pruning Overhead" (Part 1)
+ * with eps = (w >> 8) * 2^-24, w the 32-bit word of block number q:
+ *   w = Philox4x32-10(counter = (lo32(q>>2), hi32(q>>2), 0, 0),
+ *                     key = (lo32(seed), hi32(seed)))[q & 3],
+ *   q = r * (k_total / M) + (k_offset / M + j) for block j of row r of A.
+ * All selection arithmetic is IEEE binary32 in a fixed order without fused
+ * multiply-add; survivors are rounded once to bf16 (nearest even).  Zeros: an
+ * element of magnitude zero survives only when fewer than N non-zeros exist,
+ * with value +0, in the lowest free position.  A (1,2) result is emitted as a
+ * valid 2:4 pattern (pair 0 -> position 0/1, pair 1 -> position 2/3).
+ * The same (g, n, m, axis, seed, k_total, k_offset) always gives the same bits.
+ *
+ * Arguments.
+ *   g        [rows x cols], leading dimension ld, dtype MVUE_F32 or MVUE_BF16.
+ *   axis     1: A = g      (Mrows = rows, K = cols; blocks along a row of g;
+ *                            the backward product's operand),
+ *            0: A = g^T    (Mrows = cols, K = rows; blocks down a column of g;
+ *                            the update product's operand).
+ *   k_total  K of the whole (unsharded) operand, k_offset the global k of this
+ *            tensor's first element; pass K and 0 unless K is sharded.
+ *   values, meta   outputs in `layout`, sizes from mvue_packed_sizes.
+ * Preconditions (else MVUE_ERR_SHAPE / MVUE_ERR_ALIGN): K, k_total and k_offset
+ * multiples of 16; Mrows a multiple of 8; ld >= cols; g, values, meta and
+ * ld * sizeof(element) 16-byte aligned. */
+MVUE_API int mvue_prune(const void* g, int dtype, int64_t rows, int64_t cols, int64_t ld, int n, int m,
+               int axis, uint64_t seed, int64_t k_total, int64_t k_offset, void* values,
+               void* meta, int layout, void* stream);
+
+/* Expand a packed operand back to dense bf16 A[Mrows x K] (row-major, ld = K).
+ * A checking aid: the inverse of the pack step, no arithmetic. */
+MVUE_API int mvue_unpack(const void* values, const void* meta, int layout, int64_t mrows, int64_t K,
+                void* dense_bf16, void* stream);
+
+MVUE_API const char* mvue_status_string(int status);
+/* Text of the last CUDA error seen by the calling thread ("" if none). */
+MVUE_API const char* mvue_last_cuda_error(void);
+MVUE_API int mvue_version(void);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* MVUE_H_ */

@@ -1,0 +1,103 @@
+"""Python binding of the C ABI in include/mvue.h: argument marshalling only.
+
+Tensors are torch CUDA tensors used purely as device memory; every function passes
+raw pointers, sizes and the current CUDA stream to the library.  There is no
+fallback: if the library is missing or a call fails, an exception is raised.
+"""
+from __future__ import annotations
+
+import ctypes
+from pathlib import Path
+
+import torch
+
+_LIB_PATH = Path(__file__).resolve().parent / "libmvue_b200.so"
+_lib = None
+
+MVUE_F32, MVUE_BF16 = 0, 1
+MVUE_LAYOUT_CANONICAL = 0
+
+EXPORTS = ("mvue_version", "mvue_status_string", "mvue_last_cuda_error", "mvue_packed_sizes",
+           "mvue_prune", "mvue_unpack")
+
+
+class MvueError(RuntimeError):
+    def __init__(self, status: int, what: str):
+        L = lib()
+        msg = L.mvue_status_string(status).decode()
+        cuda = L.mvue_last_cuda_error().decode()
+        super().__init__(f"{what}: {msg} [{status}]" + (f" -- {cuda}" if status == -9 and cuda else ""))
+        self.status = status
+
+
+def lib() -> ctypes.CDLL:
+    """Load libmvue_b200.so (built by `python -m paper_2203_10991_b200.build`)."""
+    global _lib
+    if _lib is None:
+        if not _LIB_PATH.exists():
+            raise RuntimeError(f"{_LIB_PATH} is missing: build it with "
+                               "`python -m paper_2203_10991_b200.build` (there is no CPU fallback)")
+        L = ctypes.CDLL(str(_LIB_PATH))
+        i64, u64, vp, ci = ctypes.c_int64, ctypes.c_uint64, ctypes.c_void_p, ctypes.c_int
+        szp = ctypes.POINTER(ctypes.c_size_t)
+        L.mvue_version.restype = ci
+        L.mvue_status_string.argtypes = [ci]
+        L.mvue_status_string.restype = ctypes.c_char_p
+        L.mvue_last_cuda_error.restype = ctypes.c_char_p
+        L.mvue_packed_sizes.argtypes = [i64, i64, ci, ci, ci, ci, szp, szp]
+        L.mvue_prune.argtypes = [vp, ci, i64, i64, i64, ci, ci, ci, u64, i64, i64, vp, vp, ci, vp]
+        L.mvue_unpack.argtypes = [vp, vp, ci, i64, i64, vp, vp]
+        _lib = L
+    return _lib
+
+
+def _check(status: int, what: str):
+    if status != 0:
+        raise MvueError(status, what)
+
+
+def _stream_ptr() -> int:
+    return torch.cuda.current_stream().cuda_stream
+
+
+def _dtype_code(t: torch.Tensor) -> int:
+    if t.dtype == torch.float32:
+        return MVUE_F32
+    if t.dtype == torch.bfloat16:
+        return MVUE_BF16
+    raise TypeError(f"unsupported dtype {t.dtype}")
+
+
+def mvue_packed_sizes(rows: int, cols: int, n: int, m: int, axis: int, layout: int = MVUE_LAYOUT_CANONICAL):
+    vb, mb = ctypes.c_size_t(), ctypes.c_size_t()
+    _check(lib().mvue_packed_sizes(rows, cols, n, m, axis, layout, ctypes.byref(vb), ctypes.byref(mb)),
+           "mvue_packed_sizes")
+    return vb.value, mb.value
+
+
+def mvue_prune(g: torch.Tensor, n: int, m: int, axis: int, seed: int, *, k_total: int | None = None,
+               k_offset: int = 0, values: torch.Tensor | None = None, meta: torch.Tensor | None = None,
+               layout: int = MVUE_LAYOUT_CANONICAL):
+    """MVUE n:m prune + pack of a 2-D CUDA tensor g (fp32 or bf16, unit column stride).
+
+    Returns (values bf16 [Mrows, K/2], meta uint8 [Mrows, K/8]).
+    """
+    assert g.is_cuda and g.dim() == 2 and g.stride(1) == 1
+    rows, cols = g.shape
+    mrows, k = (rows, cols) if axis == 1 else (cols, rows)
+    if values is None or meta is None:
+        mvue_packed_sizes(rows, cols, n, m, axis, layout)          # validates before allocating
+        values = torch.empty((mrows, k // 2), dtype=torch.bfloat16, device=g.device)
+        meta = torch.empty((mrows, k // 8), dtype=torch.uint8, device=g.device)
+    _check(lib().mvue_prune(g.data_ptr(), _dtype_code(g), rows, cols, g.stride(0), n, m, axis,
+                            seed & (2**64 - 1), k if k_total is None else k_total, k_offset,
+                            values.data_ptr(), meta.data_ptr(), layout, _stream_ptr()), "mvue_prune")
+    return values, meta
+
+
+def mvue_unpack(values: torch.Tensor, meta: torch.Tensor, layout: int = MVUE_LAYOUT_CANONICAL) -> torch.Tensor:
+    mrows, kh = values.shape
+    dense = torch.empty((mrows, 2 * kh), dtype=torch.bfloat16, device=values.device)
+    _check(lib().mvue_unpack(values.data_ptr(), meta.data_ptr(), layout, mrows, 2 * kh, dense.data_ptr(),
+                             _stream_ptr()), "mvue_unpack")
+    return dense

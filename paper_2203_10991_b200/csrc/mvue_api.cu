@@ -1,0 +1,122 @@
+// C ABI of the library: argument validation on the host, then one launch on the
+// caller's stream.  No allocation, no synchronisation, no exceptions.
+#include <cuda_runtime.h>
+
+#include <cstdio>
+#include <cstring>
+#include <mutex>
+
+#include "../../include/mvue.h"
+#include "mvue_internal.h"
+
+namespace mvue {
+
+static thread_local char g_cuda_error[256] = "";
+
+void set_cuda_error(cudaError_t e, const char* where) {
+    std::snprintf(g_cuda_error, sizeof(g_cuda_error), "%s: %s (%s)", where, cudaGetErrorName(e),
+                  cudaGetErrorString(e));
+}
+
+int current_device_info(DeviceInfo* info) {
+    static std::mutex mu;
+    static DeviceInfo cache[64];
+    static bool known[64] = {};
+    int dev = 0;
+    cudaError_t e = cudaGetDevice(&dev);
+    if (e != cudaSuccess) { set_cuda_error(e, "cudaGetDevice"); return MVUE_ERR_CUDA; }
+    if (dev < 0 || dev >= 64) return MVUE_ERR_ARCH;
+    std::lock_guard<std::mutex> lock(mu);
+    if (!known[dev]) {
+        DeviceInfo d;
+        e = cudaDeviceGetAttribute(&d.cc_major, cudaDevAttrComputeCapabilityMajor, dev);
+        if (e == cudaSuccess) e = cudaDeviceGetAttribute(&d.sm_count, cudaDevAttrMultiProcessorCount, dev);
+        if (e != cudaSuccess) { set_cuda_error(e, "cudaDeviceGetAttribute"); return MVUE_ERR_CUDA; }
+        cache[dev] = d;
+        known[dev] = true;
+    }
+    *info = cache[dev];
+    return info->cc_major == 10 ? MVUE_OK : MVUE_ERR_ARCH;
+}
+
+static bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
+
+static int check_nm(int n, int m) {
+    return ((n == 1 && m == 2) || (n == 2 && m == 4)) ? MVUE_OK : MVUE_ERR_NM;
+}
+
+}  // namespace mvue
+
+using namespace mvue;
+
+extern "C" {
+
+int mvue_version(void) { return 100; }
+
+const char* mvue_status_string(int status) {
+    switch (status) {
+        case MVUE_OK: return "ok";
+        case MVUE_ERR_NULL: return "null pointer";
+        case MVUE_ERR_NM: return "unsupported N:M (only 1:2 and 2:4)";
+        case MVUE_ERR_SHAPE: return "bad shape, axis, leading dimension or K shard";
+        case MVUE_ERR_ALIGN: return "pointer or leading dimension not 16-byte aligned";
+        case MVUE_ERR_DTYPE: return "unsupported dtype";
+        case MVUE_ERR_LAYOUT: return "unsupported layout";
+        case MVUE_ERR_WORKSPACE: return "workspace missing or too small";
+        case MVUE_ERR_ARCH: return "device is not compute capability 10.x";
+        case MVUE_ERR_CUDA: return "CUDA call failed (see mvue_last_cuda_error)";
+        case MVUE_ERR_DEVICE_TIMEOUT: return "a bounded device-side wait expired";
+        default: return "unknown status";
+    }
+}
+
+const char* mvue_last_cuda_error(void) { return g_cuda_error; }
+
+int mvue_packed_sizes(int64_t rows, int64_t cols, int n, int m, int axis, int layout,
+                      size_t* values_bytes, size_t* meta_bytes) {
+    if (int s = check_nm(n, m)) return s;
+    if (layout != MVUE_LAYOUT_CANONICAL) return MVUE_ERR_LAYOUT;
+    if (axis != 0 && axis != 1) return MVUE_ERR_SHAPE;
+    if (rows <= 0 || cols <= 0) return MVUE_ERR_SHAPE;
+    const int64_t mrows = axis == 1 ? rows : cols;
+    const int64_t K = axis == 1 ? cols : rows;
+    if (K % 16 != 0 || mrows % 8 != 0) return MVUE_ERR_SHAPE;
+    if (values_bytes) *values_bytes = (size_t)mrows * (size_t)(K / 2) * 2;
+    if (meta_bytes) *meta_bytes = (size_t)mrows * (size_t)(K / 8);
+    return MVUE_OK;
+}
+
+int mvue_prune(const void* g, int dtype, int64_t rows, int64_t cols, int64_t ld, int n, int m,
+               int axis, uint64_t seed, int64_t k_total, int64_t k_offset, void* values,
+               void* meta, int layout, void* stream) {
+    if (!g || !values || !meta) return MVUE_ERR_NULL;
+    if (dtype != MVUE_F32 && dtype != MVUE_BF16) return MVUE_ERR_DTYPE;
+    if (int s = mvue_packed_sizes(rows, cols, n, m, axis, layout, nullptr, nullptr)) return s;
+    const int64_t K = axis == 1 ? cols : rows;
+    if (ld < cols) return MVUE_ERR_SHAPE;
+    if (k_total % 16 != 0 || k_offset % 16 != 0 || k_offset < 0 || k_offset + K > k_total) return MVUE_ERR_SHAPE;
+    const int64_t esz = dtype == MVUE_BF16 ? 2 : 4;
+    if (!aligned16(g) || !aligned16(values) || !aligned16(meta) || (ld * esz) % 16 != 0) return MVUE_ERR_ALIGN;
+    DeviceInfo dev;
+    if (int s = current_device_info(&dev)) return s;
+    PruneArgs a{g, dtype == MVUE_BF16, rows, cols, ld, m, axis, seed, k_total, k_offset, values, meta, dev.sm_count};
+    cudaError_t e = launch_prune(a, reinterpret_cast<cudaStream_t>(stream));
+    if (e != cudaSuccess) { set_cuda_error(e, "mvue_prune launch"); return MVUE_ERR_CUDA; }
+    return MVUE_OK;
+}
+
+int mvue_unpack(const void* values, const void* meta, int layout, int64_t mrows, int64_t K,
+                void* dense_bf16, void* stream) {
+    if (!values || !meta || !dense_bf16) return MVUE_ERR_NULL;
+    if (layout != MVUE_LAYOUT_CANONICAL) return MVUE_ERR_LAYOUT;
+    if (mrows <= 0 || K <= 0 || K % 16 != 0) return MVUE_ERR_SHAPE;
+    if (!aligned16(values) || !aligned16(meta) || !aligned16(dense_bf16)) return MVUE_ERR_ALIGN;
+    DeviceInfo dev;
+    if (int s = current_device_info(&dev)) return s;
+    cudaError_t e = launch_unpack(values, meta, mrows, K, dense_bf16, dev.sm_count,
+                                  reinterpret_cast<cudaStream_t>(stream));
+    if (e != cudaSuccess) { set_cuda_error(e, "mvue_unpack launch"); return MVUE_ERR_CUDA; }
+    return MVUE_OK;
+}
+
+}  // extern "C"

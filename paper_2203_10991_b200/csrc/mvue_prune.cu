@@ -1,0 +1,194 @@
+// MVUE N:M prune + pack kernels (memory-bound: one pass over g, packed bf16
+// survivors and 2-bit position metadata written in the same pass).
+//
+// Work unit: 16 consecutive elements along the pruned axis K.  For 2:4 that is
+// four blocks sharing one generator call; for 1:2 it is eight pairs using two.
+//   axis 1 (K contiguous in memory): one thread owns one unit = 32 contiguous
+//           bytes of bf16 (64 of fp32); a warp reads 1 KiB (2 KiB) contiguous.
+//   axis 0 (K runs down the rows of g): one thread owns a strip of 16 rows by
+//           16 bytes of columns; a warp reads 512 contiguous bytes per row.
+#include <cuda_runtime.h>
+
+#include "mvue_device.cuh"
+#include "mvue_internal.h"
+
+namespace mvue {
+namespace {
+
+__device__ __forceinline__ uint4 ldg128(const void* p) {
+    return __ldg(reinterpret_cast<const uint4*>(p));
+}
+
+// 16 elements (as binary32 bit patterns, order = position along K) -> 8 packed
+// bf16 survivors (uint4) + 4 nibbles (uint16).
+template <int M, bool kBf16>
+__device__ __forceinline__ void prune_unit(const uint32_t (&b)[16], uint64_t unit_index,
+                                           const RoundKeys& rk, uint4* out_values,
+                                           uint16_t* out_meta) {
+    uint32_t v[4];                                   // 8 survivors, two bf16 per word
+    uint32_t meta = 0;
+    if (M == 4) {
+        const uint4 w = philox4x32_10(unit_index, rk);
+        const uint32_t words[4] = {w.x, w.y, w.z, w.w};
+#pragma unroll
+        for (int j = 0; j < 4; ++j) {
+            uint32_t nib, v0, v1;
+            mvue_2of4<kBf16>(b[4 * j], b[4 * j + 1], b[4 * j + 2], b[4 * j + 3], words[j], &nib, &v0, &v1);
+            v[j] = pack_bf16x2(v0, v1);
+            meta |= nib << (4 * j);
+        }
+    } else {
+        const uint4 wa = philox4x32_10(2 * unit_index, rk);
+        const uint4 wb = philox4x32_10(2 * unit_index + 1, rk);
+        const uint32_t words[8] = {wa.x, wa.y, wa.z, wa.w, wb.x, wb.y, wb.z, wb.w};
+#pragma unroll
+        for (int j = 0; j < 4; ++j) {
+            uint32_t v0, v1;
+            const uint32_t i0 = mvue_1of2(b[4 * j], b[4 * j + 1], words[2 * j], &v0);
+            const uint32_t i1 = mvue_1of2(b[4 * j + 2], b[4 * j + 3], words[2 * j + 1], &v1);
+            v[j] = pack_bf16x2(v0, v1);
+            meta |= (i0 | ((2u + i1) << 2)) << (4 * j);
+        }
+    }
+    *out_values = make_uint4(v[0], v[1], v[2], v[3]);
+    *out_meta = (uint16_t)meta;
+}
+
+// ---- axis 1 ---------------------------------------------------------------
+// slot = r * units_per_row + c.  kLinear: the tensor is contiguous and unsharded,
+// so the input offset and the generator call number are linear in the slot.
+template <int M, bool kBf16, bool kLinear>
+__global__ void __launch_bounds__(256)
+prune_axis1_kernel(const void* __restrict__ g, int64_t n_slots, int64_t units_per_row, int64_t ld,
+                   int64_t units_per_row_total, int64_t unit_offset, RoundKeys rk,
+                   uint4* __restrict__ values, uint16_t* __restrict__ meta) {
+    const int64_t stride = (int64_t)gridDim.x * blockDim.x;
+    for (int64_t slot = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; slot < n_slots; slot += stride) {
+        int64_t elem_off;
+        uint64_t unit;
+        if (kLinear) {
+            elem_off = slot * 16;
+            unit = (uint64_t)slot;
+        } else {
+            const int64_t r = slot / units_per_row;
+            const int64_t c = slot - r * units_per_row;
+            elem_off = r * ld + c * 16;
+            unit = (uint64_t)r * (uint64_t)units_per_row_total + (uint64_t)(unit_offset + c);
+        }
+        uint32_t b[16];
+        if (kBf16) {
+            const char* p = reinterpret_cast<const char*>(g) + elem_off * 2;
+            const uint4 x = ldg128(p), y = ldg128(p + 16);
+            const uint32_t raw[8] = {x.x, x.y, x.z, x.w, y.x, y.y, y.z, y.w};
+#pragma unroll
+            for (int i = 0; i < 8; ++i) {
+                b[2 * i] = raw[i] << 16;
+                b[2 * i + 1] = raw[i] & 0xFFFF0000u;
+            }
+        } else {
+            const char* p = reinterpret_cast<const char*>(g) + elem_off * 4;
+#pragma unroll
+            for (int i = 0; i < 4; ++i) {
+                const uint4 x = ldg128(p + 16 * i);
+                b[4 * i] = x.x; b[4 * i + 1] = x.y; b[4 * i + 2] = x.z; b[4 * i + 3] = x.w;
+            }
+        }
+        prune_unit<M, kBf16>(b, unit, rk, &values[slot], &meta[slot]);
+    }
+}
+
+// ---- axis 0 ---------------------------------------------------------------
+// g is [K x C] row-major; A = g^T.  Thread (strip, chunk) owns rows
+// [16 strip, 16 strip + 16) and the 16-byte column chunk `chunk`.
+template <int M, bool kBf16>
+__global__ void __launch_bounds__(128)
+prune_axis0_kernel(const void* __restrict__ g, int64_t n_strips, int64_t n_chunks, int64_t ld,
+                   int64_t units_per_row_total, int64_t unit_offset, RoundKeys rk,
+                   uint4* __restrict__ values, uint16_t* __restrict__ meta) {
+    constexpr int CW = kBf16 ? 8 : 4;                 // columns per 16-byte chunk
+    const int64_t chunk = (int64_t)blockIdx.y * 32 + (threadIdx.x & 31);
+    const int64_t strip = (int64_t)blockIdx.x * (blockDim.x >> 5) + (threadIdx.x >> 5);
+    if (chunk >= n_chunks || strip >= n_strips) return;
+    const char* p = reinterpret_cast<const char*>(g) + ((strip * 16) * ld) * (kBf16 ? 2 : 4) + chunk * 16;
+    uint4 raw[16];
+#pragma unroll
+    for (int i = 0; i < 16; ++i) raw[i] = ldg128(p + i * ld * (kBf16 ? 2 : 4));
+#pragma unroll
+    for (int e = 0; e < CW; ++e) {
+        uint32_t b[16];
+#pragma unroll
+        for (int i = 0; i < 16; ++i) {
+            const uint32_t w = kBf16 ? (&raw[i].x)[e >> 1] : (&raw[i].x)[e];
+            b[i] = kBf16 ? ((e & 1) ? (w & 0xFFFF0000u) : (w << 16)) : w;
+        }
+        const int64_t r = chunk * CW + e;             // row of A
+        const uint64_t unit = (uint64_t)r * (uint64_t)units_per_row_total + (uint64_t)(unit_offset + strip);
+        const int64_t slot = r * n_strips + strip;
+        prune_unit<M, kBf16>(b, unit, rk, &values[slot], &meta[slot]);
+    }
+}
+
+// ---- unpack ---------------------------------------------------------------
+// One thread expands one metadata byte (two groups = 8 dense elements = 16 bytes).
+__global__ void __launch_bounds__(256)
+unpack_kernel(const uint32_t* __restrict__ values, const uint8_t* __restrict__ meta, int64_t n_bytes,
+              uint4* __restrict__ dense) {
+    const int64_t stride = (int64_t)gridDim.x * blockDim.x;
+    for (int64_t i = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; i < n_bytes; i += stride) {
+        const uint32_t mb = meta[i];
+        const uint32_t va = values[2 * i], vb = values[2 * i + 1];
+        uint16_t out[8] = {0, 0, 0, 0, 0, 0, 0, 0};
+        out[mb & 3u] = (uint16_t)va;
+        out[(mb >> 2) & 3u] = (uint16_t)(va >> 16);
+        out[4 + ((mb >> 4) & 3u)] = (uint16_t)vb;
+        out[4 + ((mb >> 6) & 3u)] = (uint16_t)(vb >> 16);
+        dense[i] = make_uint4(out[0] | ((uint32_t)out[1] << 16), out[2] | ((uint32_t)out[3] << 16),
+                              out[4] | ((uint32_t)out[5] << 16), out[6] | ((uint32_t)out[7] << 16));
+    }
+}
+
+template <int M, bool kBf16>
+cudaError_t launch_prune_t(const PruneArgs& a, cudaStream_t stream) {
+    const RoundKeys rk = make_round_keys(a.seed);
+    const int64_t upr_total = a.k_total / 16, uoff = a.k_offset / 16;
+    uint4* values = reinterpret_cast<uint4*>(a.values);
+    uint16_t* meta = reinterpret_cast<uint16_t*>(a.meta);
+    if (a.axis == 1) {
+        const int64_t upr = a.cols / 16;
+        const int64_t n_slots = a.rows * upr;
+        const bool linear = (a.ld == a.cols) && (a.k_total == a.cols) && (a.k_offset == 0);
+        const int64_t want = (n_slots + 255) / 256;
+        const int grid = (int)(want < (int64_t)a.sm_count * 64 ? want : (int64_t)a.sm_count * 64);
+        if (linear)
+            prune_axis1_kernel<M, kBf16, true><<<grid, 256, 0, stream>>>(a.g, n_slots, upr, a.ld, upr_total, uoff, rk, values, meta);
+        else
+            prune_axis1_kernel<M, kBf16, false><<<grid, 256, 0, stream>>>(a.g, n_slots, upr, a.ld, upr_total, uoff, rk, values, meta);
+    } else {
+        constexpr int CW = kBf16 ? 8 : 4;
+        const int64_t n_strips = a.rows / 16;
+        const int64_t n_chunks = a.cols / CW;
+        dim3 grid((unsigned)((n_strips + 3) / 4), (unsigned)((n_chunks + 31) / 32));
+        prune_axis0_kernel<M, kBf16><<<grid, 128, 0, stream>>>(a.g, n_strips, n_chunks, a.ld, upr_total, uoff, rk, values, meta);
+    }
+    return cudaGetLastError();
+}
+
+}  // namespace
+
+cudaError_t launch_prune(const PruneArgs& a, cudaStream_t stream) {
+    if (a.m == 4) return a.is_bf16 ? launch_prune_t<4, true>(a, stream) : launch_prune_t<4, false>(a, stream);
+    return a.is_bf16 ? launch_prune_t<2, true>(a, stream) : launch_prune_t<2, false>(a, stream);
+}
+
+cudaError_t launch_unpack(const void* values, const void* meta, int64_t mrows, int64_t K, void* dense,
+                          int sm_count, cudaStream_t stream) {
+    const int64_t n_bytes = mrows * (K / 8);
+    const int64_t want = (n_bytes + 255) / 256;
+    const int grid = (int)(want < (int64_t)sm_count * 32 ? want : (int64_t)sm_count * 32);
+    unpack_kernel<<<grid, 256, 0, stream>>>(reinterpret_cast<const uint32_t*>(values),
+                                            reinterpret_cast<const uint8_t*>(meta), n_bytes,
+                                            reinterpret_cast<uint4*>(dense));
+    return cudaGetLastError();
+}
+
+}  // namespace mvue
