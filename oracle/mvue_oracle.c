@@ -102,24 +102,19 @@ float oracle_bf16_to_f32(uint16_t h)
  * App. A.1): keep a_1 with probability |a_1| / (|a_1| + |a_2|), else a_2; the
  * survivor becomes sign(a_i) (|a_1| + |a_2|).  The draw is the threshold test
  * eps < p_1 (App. "Pruning Overhead", Part 1) written without the division:
- * eps (|a_1|+|a_2|) < |a_1|.
- * Zero rules (the paper leaves 0/0 open): a zero is never preferred to a
- * non-zero; an all-zero block keeps element 0 with value +0.
+ * eps (|a_1|+|a_2|) < |a_1|, with eps = n / 2^24, n the top 24 bits of the
+ * block's random word, evaluated as n * ((|a_1|+|a_2|) * 2^-24).
+ * Zero rule (the paper leaves 0/0 open): a_2 = 0 always keeps a_1, so a zero
+ * is never preferred to a non-zero; an all-zero block keeps a_1 (a signed zero).
  * Returns the kept index (0 or 1); *kept receives the new value.
  * ---------------------------------------------------------------------- */
 int oracle_mvue_1of2(float a1, float a2, uint32_t word, float *kept)
 {
     float m1 = fabsf(a1), m2 = fabsf(a2);
     float S = m1 + m2;
-    int idx;
-    if (m1 == 0.0f && m2 == 0.0f) { *kept = 0.0f; return 0; }
-    if (m2 == 0.0f) idx = 0;
-    else if (m1 == 0.0f) idx = 1;
-    else {
-        float eps = oracle_uniform24(word);
-        float t = eps * S;
-        idx = (t < m1) ? 0 : 1;
-    }
+    float scale = S * 5.9604644775390625e-08f;            /* S * 2^-24, exact */
+    float t = (float)(word >> 8) * scale;                 /* eps * S */
+    int idx = (t < m1 || m2 == 0.0f) ? 0 : 1;
     *kept = copysignf(S, idx == 0 ? a1 : a2);
     return idx;
 }
@@ -128,26 +123,38 @@ int oracle_mvue_1of2(float a1, float a2, uint32_t word, float *kept)
  * MVUE 2:4 (optimal marginals: Sec. 4.2; joint law over pairs: App. A.2).
  *
  * 1. Sort the magnitudes ascending, ties by original position:
- *      s_1 <= s_2 <= s_3 <= s_4, original indices i_1..i_4.
- * 2. Case 3 (s_4 >= s_1+s_2+s_3): the dominant element survives with
- *    probability one and keeps its value (a_i / p_i with p_i = 1); one of the
- *    other three survives with probability s_k / (s_1+s_2+s_3) and becomes
- *    sign(a) (s_1+s_2+s_3).
- *    Case 1 (s_4 <= 2 s_1 + s_3) and case 2 (otherwise): the pair (i, j)
- *    survives with the probability p_ij of the appendix table; both survivors
- *    become a_i / p_i with p_i = 2 s_i / sum, i.e. sign(a_i) sum / 2.
- * 3. The pair is drawn by walking the cumulative table in the fixed order
- *    13, 14, 23, 24, 34 with eps scaled by the table's common denominator, so
- *    no division appears.  A numerator that rounding pushes below zero is
- *    clamped to zero.
- * Zero rules: an element of magnitude zero survives only if fewer than two
- * non-zeros exist, and then with value +0 (lowest free positions).
+ *      s_1 <= s_2 <= s_3 <= s_4  at original positions i_1..i_4.
+ * 2. The appendix gives, for each of its three cases, the probability p_ij
+ *    that the pair of ranks (i, j) survives.  The pair is drawn by walking the
+ *    table in the fixed order 13, 14, 23, 24, 34: the first pair whose
+ *    cumulative probability exceeds eps wins.  No division is needed: with
+ *    d = s_4 - s_3 every case has the SAME cumulative numerators over the
+ *    denominator D,
+ *         C_13 = 2 s_1 - d                        (only case 1 has p_13 > 0)
+ *         C_14 = 4 s_1
+ *         C_23 = 4 s_1 + (2 s_2 - d) + min(2 s_1 - d, 0)
+ *         C_24 = 4 (s_1 + s_2)
+ *      case 1 (s_4 <= 2 s_1 + s_3):  D = 2 sum; the four numerators of the
+ *              table are C_13, C_14 - C_13, C_23 - C_14, C_24 - C_23.
+ *      case 2 (2 s_1 + s_3 <= s_4 <= s_1+s_2+s_3):  D = 2 sum; C_13 <= 0 is
+ *              never hit (p_13 = 0) and C_23 = 2 (3 s_1 + s_2 - d)
+ *              = 2 (2 s_1 + (s_1+s_2+s_3-s_4)), the table's p_14 + p_23.
+ *      case 3 (s_4 >= s_1+s_2+s_3):  D = 4 (s_1+s_2+s_3); C_13 <= 0 and
+ *              C_23 <= C_14 are never hit, leaving s_1 and s_1 + s_2 over
+ *              s_1+s_2+s_3 for the partner of the dominant element.
+ *    D = 2 (S3 + min(s_4, S3)) with S3 = s_1+s_2+s_3 covers all three.
+ *    In case 3 the larger survivor is the dominant element whatever rounding
+ *    does to C_23.
+ * 3. Survivors become a_i / p_i (Sec. 4.2): sign(a_i) D/4 for every survivor
+ *    with p_i < 1 (sum/2 in cases 1-2, S3 in case 3), and the dominant
+ *    element of case 3 keeps its value: max(s_4, D/4).
+ * Zero rule: an element of magnitude zero has zero-width intervals in the
+ * walk, so it survives only if fewer than two non-zeros exist (pair 34 of the
+ * (magnitude, position) order), as a signed zero.
  *
  * idx[0] < idx[1] are the surviving original positions, val[] their new
  * values in that order.
  * ---------------------------------------------------------------------- */
-static float clamp0(float x) { return x < 0.0f ? 0.0f : x; }
-
 void oracle_mvue_2of4(const float a[4], uint32_t word, int idx[2], float val[2])
 {
     float s[4];
@@ -160,65 +167,30 @@ void oracle_mvue_2of4(const float a[4], uint32_t word, int idx[2], float val[2])
         s[j] = m; pos[j] = i;
     }
     const float s1 = s[0], s2 = s[1], s3 = s[2], s4 = s[3];
-    const float S3 = (s1 + s2) + s3;
-    const float S  = S3 + s4;
-    const float eps = oracle_uniform24(word);
+    const float S12 = s1 + s2;
+    const float S3  = S12 + s3;
+    const float d   = s4 - s3;
+    const float x   = (s1 + s1) - d;                       /* 2 s_1 - d */
+    const float y   = (s2 + s2) - d;                       /* 2 s_2 - d */
+    const float C13 = x;
+    const float C14 = 4.0f * s1;
+    const float C23 = (C14 + y) + (x < 0.0f ? x : 0.0f);
+    const float C24 = 4.0f * S12;
+    const float Dh  = S3 + (s4 < S3 ? s4 : S3);            /* D / 2 */
+    const float scale = Dh * 1.1920928955078125e-07f;      /* D * 2^-24, exact */
+    const float t = (float)(word >> 8) * scale;            /* eps * D */
 
-    int   ka, kb;          /* sorted ranks (0..3) of the two survivors */
-    float va, vb;          /* their new values */
+    int ka, kb;                                            /* sorted ranks (0..3) of the survivors */
+    if      (t < C13) { ka = 0; kb = 2; }
+    else if (t < C14) { ka = 0; kb = 3; }
+    else if (t < C23) { ka = 1; kb = 2; }
+    else if (t < C24) { ka = 1; kb = 3; }
+    else              { ka = 2; kb = 3; }
+    if (s4 >= S3) kb = 3;                                  /* case 3: the dominant element always survives */
 
-    if (s4 == 0.0f) {                       /* nothing to keep */
-        idx[0] = 0; idx[1] = 1; val[0] = 0.0f; val[1] = 0.0f;
-        return;
-    }
-    if (s4 >= S3) {                         /* case 3 */
-        kb = 3; vb = a[pos[3]];
-        if (S3 == 0.0f) {                   /* a single non-zero in the block */
-            int other = (pos[3] == 0) ? 1 : 0;
-            if (other < pos[3]) { idx[0] = other; idx[1] = pos[3]; val[0] = 0.0f; val[1] = vb; }
-            else                { idx[0] = pos[3]; idx[1] = other; val[0] = vb; val[1] = 0.0f; }
-            return;
-        }
-        float t = eps * S3;
-        if (t < s1) ka = 0;
-        else if (t < s1 + s2) ka = 1;
-        else ka = 2;
-        va = copysignf(S3, a[pos[ka]]);
-    } else {
-        float w13, w14, w23, w24, denom;
-        if (s4 <= (s1 + s1) + s3) {         /* case 1: numerators over 2 * sum */
-            w13 = clamp0(((s1 + s1) + s3) - s4);
-            w14 = clamp0(((s1 + s1) - s3) + s4);
-            w23 = clamp0(((s2 + s2) + s3) - s4);
-            w24 = clamp0(((s2 + s2) - s3) + s4);
-            denom = S + S;
-        } else {                            /* case 2: numerators over sum */
-            w13 = 0.0f;
-            w14 = s1 + s1;
-            w23 = clamp0(S3 - s4);
-            w24 = clamp0((s2 - s1) + (s4 - s3));
-            denom = S;
-        }
-        float t = eps * denom;
-        float c = w13;
-        if (t < c) { ka = 0; kb = 2; }
-        else {
-            c = c + w14;
-            if (t < c) { ka = 0; kb = 3; }
-            else {
-                c = c + w23;
-                if (t < c) { ka = 1; kb = 2; }
-                else {
-                    c = c + w24;
-                    if (t < c) { ka = 1; kb = 3; }
-                    else       { ka = 2; kb = 3; }
-                }
-            }
-        }
-        float half = 0.5f * S;
-        va = copysignf(half, a[pos[ka]]);
-        vb = copysignf(half, a[pos[kb]]);
-    }
+    const float quarter_D = 0.5f * Dh;
+    const float va = copysignf(quarter_D, a[pos[ka]]);
+    const float vb = copysignf(s4 > quarter_D ? s4 : quarter_D, a[pos[kb]]);
     if (pos[ka] < pos[kb]) { idx[0] = pos[ka]; idx[1] = pos[kb]; val[0] = va; val[1] = vb; }
     else                   { idx[0] = pos[kb]; idx[1] = pos[ka]; val[0] = vb; val[1] = va; }
 }

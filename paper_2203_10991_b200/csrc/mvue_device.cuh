@@ -2,9 +2,14 @@
 // the 1:2 and 2:4 block estimators and small packing helpers.
 //
 // Every floating-point step that decides a mask or a kept value is written with
-// the explicit round-to-nearest intrinsics (__fadd_rn, __fmul_rn, ...) so that the
-// compiler can neither fuse a multiply with an add nor reorder a sum: the result
-// is a pure function of the inputs and the seed, bit for bit.
+// the explicit round-to-nearest intrinsics (__fadd_rn, __fmul_rn, __fmaf_rn with an
+// exact power-of-two product) so that the compiler can neither fuse nor reorder:
+// the result is a pure function of the inputs and the seed, bit for bit.
+//
+// The prune is bound by the integer/logic pipe, not by memory, unless the
+// selection is written tightly; the bf16 paths below therefore keep compares,
+// selects and bit operations to a minimum and push what they can onto the
+// floating-point and multiply pipes.
 #pragma once
 #include <cstdint>
 #include <cuda_bf16.h>
@@ -50,153 +55,138 @@ __device__ __forceinline__ uint4 philox4x32_10(uint64_t call, const RoundKeys& r
     return make_uint4(c0, c1, c2, c3);
 }
 
-// eps in [0,1): top 24 bits of the word, exact in binary32.
-__device__ __forceinline__ float uniform24(uint32_t word) {
-    return __fmul_rn(__uint2float_rn(word >> 8), 5.9604644775390625e-08f);
+// The top 24 bits of a word as a float (exact): eps * 2^24.
+__device__ __forceinline__ float top24(uint32_t word) {
+    return __uint2float_rn(__umulhi(word, 1u << 24));   // high product = word >> 8, on the multiply pipe
 }
 
-// ---------------------------------------------------------------------------
-// MVUE 1:2 (Sec. 4.1): keep a_1 iff eps (|a_1|+|a_2|) < |a_1|; the survivor
-// becomes sign(a_i)(|a_1|+|a_2|).  b1, b2 are the binary32 bit patterns.
-// Returns the kept index; *kept_bits receives the new value's bit pattern.
-// A zero is never preferred to a non-zero; an all-zero block keeps index 0, +0.
-// ---------------------------------------------------------------------------
-__device__ __forceinline__ uint32_t mvue_1of2(uint32_t b1, uint32_t b2, uint32_t word,
-                                              uint32_t* kept_bits) {
-    const float m1 = __uint_as_float(b1 & 0x7FFFFFFFu);
-    const float m2 = __uint_as_float(b2 & 0x7FFFFFFFu);
-    const float S = __fadd_rn(m1, m2);
-    const float t = __fmul_rn(uniform24(word), S);
-    const uint32_t idx = (m2 != 0.0f && !(t < m1)) ? 1u : 0u;
-    const uint32_t sign = (idx ? b2 : b1) & 0x80000000u;
-    const uint32_t sbits = __float_as_uint(S);
-    *kept_bits = sbits ? (sbits | sign) : 0u;
-    return idx;
+// Two binary32 values -> one word of two bf16 (round to nearest even), lo first.
+__device__ __forceinline__ uint32_t pack_bf16x2(float lo, float hi) {
+    __nv_bfloat162 p = __floats2bfloat162_rn(lo, hi);
+    return *reinterpret_cast<uint32_t*>(&p);
 }
 
-// ---------------------------------------------------------------------------
-// MVUE 2:4 (marginals: Sec. 4.2; joint law: App. A.2).
+// ===========================================================================
+// MVUE 1:2 (Sec. 4.1): keep a_1 iff eps (|a_1|+|a_2|) < |a_1| (or a_2 = 0); the
+// survivor becomes sign(a_i)(|a_1|+|a_2|).
+// ===========================================================================
+// f0, f1: the pair as binary32.  Returns true when a_1 (f0) is kept; *kept
+// receives the new value.
+__device__ __forceinline__ bool mvue_1of2(float f0, float f1, uint32_t word, float* kept) {
+    const float m0 = fabsf(f0), m1 = fabsf(f1);
+    const float S = __fadd_rn(m0, m1);
+    const float t = __fmul_rn(top24(word), __fmul_rn(S, 5.9604644775390625e-08f));
+    const bool keep0 = (t < m0) || (m1 == 0.0f);
+    const uint32_t src = __float_as_uint(keep0 ? f0 : f1);
+    *kept = __uint_as_float(__float_as_uint(S) | (src & 0x80000000u));
+    return keep0;
+}
+
+// ===========================================================================
+// MVUE 2:4 (marginals: Sec. 4.2; joint law over pairs: App. A.2).
 //
-// Sorted magnitudes s1 <= s2 <= s3 <= s4 (ties by position).  All three cases of
-// the appendix are evaluated as one cumulative table over the pairs 13, 14, 23,
-// 24 (else 34) with numerators w and common denominator D:
-//   case 3 (s4 >= s1+s2+s3): w = (0, s1, 0, s2),                         D = s1+s2+s3
-//   case 1 (s4 <= 2 s1 + s3): w = (2s1+s3-s4, 2s1-s3+s4, 2s2+s3-s4, 2s2-s3+s4), D = 2 sum
-//   case 2 (otherwise):       w = (0, 2s1, s1+s2+s3-s4, s2-s1+s4-s3),    D = sum
-// and the pair is the first whose cumulative numerator exceeds eps * D.
-// Kept values: case 3 -> dominant unchanged, the other sign * (s1+s2+s3);
-// cases 1, 2 -> both sign * sum / 2.
-//
-// Key: a 64-bit (or, when the low two magnitude bits are known to be zero, a
-// 32-bit) integer whose order is (magnitude, position).
-// ---------------------------------------------------------------------------
-template <typename KeyT>
-__device__ __forceinline__ void cswap(KeyT& a, KeyT& b) {
-    const KeyT lo = a < b ? a : b;
-    const KeyT hi = a < b ? b : a;
-    a = lo;
-    b = hi;
-}
-
-template <bool kLowBitsFree>
-struct SortKey;
-
-template <>
-struct SortKey<true> {   // magnitudes widened from bf16: the low 16 bits are zero
-    using T = uint32_t;
-    static __device__ __forceinline__ T make(uint32_t mag_bits, uint32_t pos) { return mag_bits | pos; }
-    static __device__ __forceinline__ float mag(T k) { return __uint_as_float(k & ~3u); }
-    static __device__ __forceinline__ uint32_t pos(T k) { return k & 3u; }
+// With the magnitudes sorted, s1 <= s2 <= s3 <= s4 (ties by position), d = s4-s3,
+// the cumulative numerators of the appendix's pair table in the order 13, 14, 23,
+// 24 are, for all three of its cases and over the common denominator D,
+//     C13 = 2 s1 - d,  C14 = 4 s1,  C23 = 4 s1 + (2 s2 - d) + min(2 s1 - d, 0),
+//     C24 = 4 (s1 + s2),  D = 2 (S3 + min(s4, S3)),  S3 = s1 + s2 + s3,
+// and the pair is the first with eps D < C (else 34).  When s4 >= S3 the larger
+// survivor is always the dominant element.  Survivors become sign(a) D/4, the
+// dominant element of the capped case keeps max(s4, D/4) = s4.
+// ===========================================================================
+struct Pick24 {
+    uint32_t ia, ib;     // original positions of the smaller / larger survivor
+    float va, vb;        // their new magnitudes
 };
 
-template <>
-struct SortKey<false> {  // arbitrary binary32 magnitudes
-    using T = uint64_t;
-    static __device__ __forceinline__ T make(uint32_t mag_bits, uint32_t pos) {
-        return ((uint64_t)mag_bits << 2) | pos;
-    }
-    static __device__ __forceinline__ float mag(T k) { return __uint_as_float((uint32_t)(k >> 2)); }
-    static __device__ __forceinline__ uint32_t pos(T k) { return (uint32_t)k & 3u; }
-};
-
-// b0..b3: binary32 bit patterns of the block.  Outputs: nibble idx0 | idx1 << 2
-// (idx0 < idx1) and the two new values' bit patterns in that order.
-template <bool kLowBitsFree>
-__device__ __forceinline__ void mvue_2of4(uint32_t b0, uint32_t b1, uint32_t b2, uint32_t b3,
-                                          uint32_t word, uint32_t* nibble, uint32_t* v0_bits,
-                                          uint32_t* v1_bits) {
-    using SK = SortKey<kLowBitsFree>;
-    typename SK::T k1 = SK::make(b0 & 0x7FFFFFFFu, 0u);
-    typename SK::T k2 = SK::make(b1 & 0x7FFFFFFFu, 1u);
-    typename SK::T k3 = SK::make(b2 & 0x7FFFFFFFu, 2u);
-    typename SK::T k4 = SK::make(b3 & 0x7FFFFFFFu, 3u);
-    cswap(k1, k2); cswap(k3, k4); cswap(k1, k3); cswap(k2, k4); cswap(k2, k3);
-
-    const float s1 = SK::mag(k1), s2 = SK::mag(k2), s3 = SK::mag(k3), s4 = SK::mag(k4);
+// k1..k4: sort keys ascending; KEY_MAG(k) its magnitude, KEY_POS(k) its position.
+template <typename KeyT, typename MagF, typename PosF>
+__device__ __forceinline__ Pick24 pick_2of4(KeyT k1, KeyT k2, KeyT k3, KeyT k4, uint32_t word,
+                                            MagF mag, PosF pos) {
+    const float s1 = mag(k1), s2 = mag(k2), s3 = mag(k3), s4 = mag(k4);
     const float S12 = __fadd_rn(s1, s2);
     const float S3 = __fadd_rn(S12, s3);
-    const float S = __fadd_rn(S3, s4);
+    const float d = __fsub_rn(s4, s3);
+    const float x = __fmaf_rn(2.0f, s1, -d);            // 2 s1 is exact: one rounding, as (s1+s1)-d
+    const float y = __fmaf_rn(2.0f, s2, -d);
+    const float C14 = __fmul_rn(4.0f, s1);
+    const float C23 = __fadd_rn(__fadd_rn(C14, y), fminf(x, 0.0f));
+    const float C24 = __fmul_rn(4.0f, S12);
+    const float Dh = __fadd_rn(S3, fminf(s4, S3));
+    const float t = __fmul_rn(top24(word), __fmul_rn(Dh, 1.1920928955078125e-07f));
 
-    const float two_s1 = __fadd_rn(s1, s1);
-    const float two_s2 = __fadd_rn(s2, s2);
-    const bool capped = s4 >= S3;                               // case 3
-    const bool tight = s4 <= __fadd_rn(two_s1, s3);             // case 1 (when not capped)
+    const bool p1 = t < x;
+    const bool p12 = p1 || (t < C14);
+    const bool p3 = t < C23;
+    const bool p34 = p3 || (t < C24);
+    const bool capped = s4 >= S3;
+    const KeyT key_a = p12 ? k1 : (p34 ? k2 : k3);
+    const bool b_is_third = !capped && (p1 || (!p12 && p3));
+    const KeyT key_b = b_is_third ? k3 : k4;
 
-    // case 1 numerators
-    const float a13 = fmaxf(0.0f, __fsub_rn(__fadd_rn(two_s1, s3), s4));
-    const float a14 = fmaxf(0.0f, __fadd_rn(__fsub_rn(two_s1, s3), s4));
-    const float a23 = fmaxf(0.0f, __fsub_rn(__fadd_rn(two_s2, s3), s4));
-    const float a24 = fmaxf(0.0f, __fadd_rn(__fsub_rn(two_s2, s3), s4));
-    // case 2 numerators
-    const float c23 = fmaxf(0.0f, __fsub_rn(S3, s4));
-    const float c24 = fmaxf(0.0f, __fadd_rn(__fsub_rn(s2, s1), __fsub_rn(s4, s3)));
-
-    const float w13 = (tight && !capped) ? a13 : 0.0f;
-    const float w14 = capped ? s1 : (tight ? a14 : two_s1);
-    const float w23 = capped ? 0.0f : (tight ? a23 : c23);
-    const float w24 = capped ? s2 : (tight ? a24 : c24);
-    const float D = capped ? S3 : (tight ? __fadd_rn(S, S) : S);
-
-    const float t = __fmul_rn(uniform24(word), D);
-    const float c1 = w13;
-    const float c2 = __fadd_rn(c1, w14);
-    const float c3 = __fadd_rn(c2, w23);
-    const float c4 = __fadd_rn(c3, w24);
-    // index of the first cumulative numerator above t: 0..3 -> pairs 13,14,23,24; 4 -> pair 34
-    const uint32_t pair = (uint32_t)!(t < c1) + (uint32_t)!(t < c2) + (uint32_t)!(t < c3) + (uint32_t)!(t < c4);
-
-    const uint32_t ka = pair >> 1;                              // rank of the smaller survivor: 0,0,1,1,2
-    const bool b_is_top = (pair & 1u) | (pair >> 2);            // larger survivor is rank 3 (else rank 2)
-    const typename SK::T key_a = ka == 0 ? k1 : (ka == 1 ? k2 : k3);
-    const typename SK::T key_b = b_is_top ? k4 : k3;
-    uint32_t ia = SK::pos(key_a), ib = SK::pos(key_b);
-
-    const float half = __fmul_rn(0.5f, S);
-    uint32_t va = __float_as_uint(capped ? S3 : half);
-    uint32_t vb = __float_as_uint(capped ? s4 : half);
-    // signs of the original elements at positions ia, ib
-    const uint32_t sa = ia == 0 ? b0 : (ia == 1 ? b1 : (ia == 2 ? b2 : b3));
-    const uint32_t sb = ib == 0 ? b0 : (ib == 1 ? b1 : (ib == 2 ? b2 : b3));
-    va |= sa & 0x80000000u;
-    vb |= sb & 0x80000000u;
-
-    if (S3 == 0.0f) {            // at most one non-zero: a zero fills the lowest free position with +0
-        ia = (ib == 0u) ? 1u : 0u;
-        va = 0u;
-    }
-    if (s4 == 0.0f) {            // all zero
-        ia = 0u; ib = 1u; va = 0u; vb = 0u;
-    }
-    const bool a_first = ia < ib;
-    *nibble = a_first ? (ia | (ib << 2)) : (ib | (ia << 2));
-    *v0_bits = a_first ? va : vb;
-    *v1_bits = a_first ? vb : va;
+    Pick24 r;
+    r.ia = pos(key_a);
+    r.ib = pos(key_b);
+    r.va = __fmul_rn(0.5f, Dh);
+    r.vb = fmaxf(s4, r.va);
+    return r;
 }
 
-// Two binary32 values -> one 32-bit word of two bf16 (round to nearest even), lo first.
-__device__ __forceinline__ uint32_t pack_bf16x2(uint32_t lo_bits, uint32_t hi_bits) {
-    __nv_bfloat162 p = __floats2bfloat162_rn(__uint_as_float(lo_bits), __uint_as_float(hi_bits));
-    return *reinterpret_cast<uint32_t*>(&p);
+// ---- bf16 source: x01 = a0 | a1 << 16, x23 = a2 | a3 << 16 ------------------
+// The sort key of an element is its widened magnitude with the position in the
+// two lowest mantissa bits (zero in a widened bf16): as a positive float its
+// order is (magnitude, position).  The first comparator layer takes absolute
+// values, which strips the sign for free.
+// Outputs: `out` = the two survivors as bf16 (lower position in the low half),
+// and the group's nibble idx0 | idx1 << 2.
+__device__ __forceinline__ void mvue_2of4_bf16(uint32_t x01, uint32_t x23, uint32_t word,
+                                               uint32_t* out, uint32_t* nibble) {
+    const float f0 = __uint_as_float(__byte_perm(x01, 0u, 0x1054));
+    const float f1 = __uint_as_float(__byte_perm(x01, 1u, 0x3254));
+    const float f2 = __uint_as_float(__byte_perm(x23, 2u, 0x1054));
+    const float f3 = __uint_as_float(__byte_perm(x23, 3u, 0x3254));
+    const float lo01 = fminf(fabsf(f0), fabsf(f1)), hi01 = fmaxf(fabsf(f0), fabsf(f1));
+    const float lo23 = fminf(fabsf(f2), fabsf(f3)), hi23 = fmaxf(fabsf(f2), fabsf(f3));
+    const float k1 = fminf(lo01, lo23), mid_a = fmaxf(lo01, lo23);
+    const float mid_b = fminf(hi01, hi23), k4 = fmaxf(hi01, hi23);
+    const float k2 = fminf(mid_a, mid_b), k3 = fmaxf(mid_a, mid_b);
+
+    const Pick24 r = pick_2of4(
+        k1, k2, k3, k4, word,
+        [](float k) { return __uint_as_float(__float_as_uint(k) & 0xFFFF0000u); },
+        [](float k) { return __float_as_uint(k) & 3u; });
+
+    // byte 2 i + 1 of {x01, x23} carries the sign of element i in its top bit
+    const uint32_t sel = (r.ia << 5) | (r.ib << 13) | 0x1010u;
+    const uint32_t signs = __byte_perm(x01, x23, sel) & 0x80008000u;
+    const uint32_t ab = pack_bf16x2(r.va, r.vb) | signs;        // a low, b high
+    const bool swap = r.ia > r.ib;
+    *out = swap ? __byte_perm(ab, 0u, 0x1032) : ab;
+    *nibble = swap ? (r.ib | (r.ia << 2)) : (r.ia | (r.ib << 2));
+}
+
+// ---- binary32 source ---------------------------------------------------------
+// 64-bit keys (magnitude bits << 2 | position); b0..b3 are the raw bit patterns.
+__device__ __forceinline__ void mvue_2of4_f32(uint32_t b0, uint32_t b1, uint32_t b2, uint32_t b3,
+                                              uint32_t word, uint32_t* out, uint32_t* nibble) {
+    auto make = [](uint32_t b, uint32_t p) { return ((uint64_t)(b & 0x7FFFFFFFu) << 2) | p; };
+    auto cswap = [](uint64_t& a, uint64_t& b) {
+        const uint64_t lo = a < b ? a : b, hi = a < b ? b : a;
+        a = lo; b = hi;
+    };
+    uint64_t k1 = make(b0, 0u), k2 = make(b1, 1u), k3 = make(b2, 2u), k4 = make(b3, 3u);
+    cswap(k1, k2); cswap(k3, k4); cswap(k1, k3); cswap(k2, k4); cswap(k2, k3);
+    const Pick24 r = pick_2of4(
+        k1, k2, k3, k4, word,
+        [](uint64_t k) { return __uint_as_float((uint32_t)(k >> 2)); },
+        [](uint64_t k) { return (uint32_t)k & 3u; });
+    const uint32_t sa = (r.ia == 0 ? b0 : (r.ia == 1 ? b1 : (r.ia == 2 ? b2 : b3))) & 0x80000000u;
+    const uint32_t sb = (r.ib == 0 ? b0 : (r.ib == 1 ? b1 : (r.ib == 2 ? b2 : b3))) & 0x80000000u;
+    const float va = __uint_as_float(__float_as_uint(r.va) | sa);
+    const float vb = __uint_as_float(__float_as_uint(r.vb) | sb);
+    const bool swap = r.ia > r.ib;
+    *out = swap ? pack_bf16x2(vb, va) : pack_bf16x2(va, vb);
+    *nibble = swap ? (r.ib | (r.ia << 2)) : (r.ia | (r.ib << 2));
 }
 
 }  // namespace mvue

