@@ -142,7 +142,8 @@ int oracle_mvue_1of2(float a1, float a2, uint32_t word, float *kept)
  *      case 3 (s_4 >= s_1+s_2+s_3):  D = 4 (s_1+s_2+s_3); C_13 <= 0 and
  *              C_23 <= C_14 are never hit, leaving s_1 and s_1 + s_2 over
  *              s_1+s_2+s_3 for the partner of the dominant element.
- *    D = 2 (S3 + min(s_4, S3)) with S3 = s_1+s_2+s_3 covers all three.
+ *    D = 2 (2 S3 + min(s_4 - S3, 0)) with S3 = s_1+s_2+s_3 covers all three
+ *    (sum + sum in cases 1-2, 4 S3 in case 3).
  *    In case 3 the larger survivor is the dominant element whatever rounding
  *    does to C_23.
  * 3. Survivors become a_i / p_i (Sec. 4.2): sign(a_i) D/4 for every survivor
@@ -176,7 +177,8 @@ void oracle_mvue_2of4(const float a[4], uint32_t word, int idx[2], float val[2])
     const float C14 = 4.0f * s1;
     const float C23 = (C14 + y) + (x < 0.0f ? x : 0.0f);
     const float C24 = 4.0f * S12;
-    const float Dh  = S3 + (s4 < S3 ? s4 : S3);            /* D / 2 */
+    const float e   = s4 - S3;                             /* >= 0: case 3 */
+    const float Dh  = (S3 + S3) + (e < 0.0f ? e : 0.0f);   /* D / 2 */
     const float scale = Dh * 1.1920928955078125e-07f;      /* D * 2^-24, exact */
     const float t = (float)(word >> 8) * scale;            /* eps * D */
 
@@ -186,7 +188,7 @@ void oracle_mvue_2of4(const float a[4], uint32_t word, int idx[2], float val[2])
     else if (t < C23) { ka = 1; kb = 2; }
     else if (t < C24) { ka = 1; kb = 3; }
     else              { ka = 2; kb = 3; }
-    if (s4 >= S3) kb = 3;                                  /* case 3: the dominant element always survives */
+    if (e >= 0.0f) kb = 3;                                 /* case 3: the dominant element always survives */
 
     const float quarter_D = 0.5f * Dh;
     const float va = copysignf(quarter_D, a[pos[ka]]);

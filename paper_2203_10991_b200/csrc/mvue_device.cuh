@@ -82,6 +82,26 @@ __device__ __forceinline__ bool mvue_1of2(float f0, float f1, uint32_t word, flo
     return keep0;
 }
 
+// Two adjacent bf16 pairs (one group of four): x0 = a0 | a1 << 16, x1 = a2 | a3 << 16.
+// Outputs the group's two survivors as bf16 (pair 0 in the low half) and its nibble
+// (pair 0 -> position 0/1, pair 1 -> position 2/3).
+__device__ __forceinline__ void mvue_1of2x2_bf16(uint32_t x0, uint32_t x1, uint32_t word0,
+                                                 uint32_t word1, uint32_t* out, uint32_t* nibble) {
+    const float a0 = __uint_as_float(x0 << 16), a1 = __uint_as_float(x0 & 0xFFFF0000u);
+    const float b0 = __uint_as_float(x1 << 16), b1 = __uint_as_float(x1 & 0xFFFF0000u);
+    const float SA = __fadd_rn(fabsf(a0), fabsf(a1));
+    const float SB = __fadd_rn(fabsf(b0), fabsf(b1));
+    const float tA = __fmul_rn(top24(word0), __fmul_rn(SA, 5.9604644775390625e-08f));
+    const float tB = __fmul_rn(top24(word1), __fmul_rn(SB, 5.9604644775390625e-08f));
+    const bool keepA = (tA < fabsf(a0)) || (fabsf(a1) == 0.0f);
+    const bool keepB = (tB < fabsf(b0)) || (fabsf(b1) == 0.0f);
+    // byte 1 <- high byte of the survivor of pair 0, byte 3 <- high byte of the survivor of pair 1
+    const uint32_t sel = (keepA ? 0x0010u : 0x0030u) | (keepB ? 0x5000u : 0x7000u);
+    const uint32_t signs = __byte_perm(x0, x1, sel) & 0x80008000u;
+    *out = pack_bf16x2(SA, SB) | signs;
+    *nibble = (keepA ? 0u : 1u) | (keepB ? 8u : 12u);
+}
+
 // ===========================================================================
 // MVUE 2:4 (marginals: Sec. 4.2; joint law over pairs: App. A.2).
 //
@@ -89,20 +109,21 @@ __device__ __forceinline__ bool mvue_1of2(float f0, float f1, uint32_t word, flo
 // the cumulative numerators of the appendix's pair table in the order 13, 14, 23,
 // 24 are, for all three of its cases and over the common denominator D,
 //     C13 = 2 s1 - d,  C14 = 4 s1,  C23 = 4 s1 + (2 s2 - d) + min(2 s1 - d, 0),
-//     C24 = 4 (s1 + s2),  D = 2 (S3 + min(s4, S3)),  S3 = s1 + s2 + s3,
+//     C24 = 4 (s1 + s2),  D = 2 (2 S3 + min(s4 - S3, 0)),  S3 = s1 + s2 + s3,
 // and the pair is the first with eps D < C (else 34).  When s4 >= S3 the larger
 // survivor is always the dominant element.  Survivors become sign(a) D/4, the
 // dominant element of the capped case keeps max(s4, D/4) = s4.
 // ===========================================================================
+template <typename KeyT>
 struct Pick24 {
-    uint32_t ia, ib;     // original positions of the smaller / larger survivor
+    KeyT key_a, key_b;   // sort keys of the smaller / larger survivor
     float va, vb;        // their new magnitudes
 };
 
 // k1..k4: sort keys ascending; KEY_MAG(k) its magnitude, KEY_POS(k) its position.
-template <typename KeyT, typename MagF, typename PosF>
-__device__ __forceinline__ Pick24 pick_2of4(KeyT k1, KeyT k2, KeyT k3, KeyT k4, uint32_t word,
-                                            MagF mag, PosF pos) {
+template <typename KeyT, typename MagF>
+__device__ __forceinline__ Pick24<KeyT> pick_2of4(KeyT k1, KeyT k2, KeyT k3, KeyT k4, uint32_t word,
+                                                  MagF mag) {
     const float s1 = mag(k1), s2 = mag(k2), s3 = mag(k3), s4 = mag(k4);
     const float S12 = __fadd_rn(s1, s2);
     const float S3 = __fadd_rn(S12, s3);
@@ -110,59 +131,66 @@ __device__ __forceinline__ Pick24 pick_2of4(KeyT k1, KeyT k2, KeyT k3, KeyT k4, 
     const float x = __fmaf_rn(2.0f, s1, -d);            // 2 s1 is exact: one rounding, as (s1+s1)-d
     const float y = __fmaf_rn(2.0f, s2, -d);
     const float C14 = __fmul_rn(4.0f, s1);
-    const float C23 = __fadd_rn(__fadd_rn(C14, y), fminf(x, 0.0f));
+    // min(v, 0) = (v - |v|) / 2 exactly: keeps the minimum off the compare/select pipe
+    const float C23 = __fmaf_rn(0.5f, __fsub_rn(x, fabsf(x)), __fadd_rn(C14, y));
     const float C24 = __fmul_rn(4.0f, S12);
-    const float Dh = __fadd_rn(S3, fminf(s4, S3));
+    const float e = __fsub_rn(s4, S3);                  // >= 0: the dominant element is capped at p = 1
+    const float Dh = __fmaf_rn(0.5f, __fsub_rn(e, fabsf(e)), __fadd_rn(S3, S3));
     const float t = __fmul_rn(top24(word), __fmul_rn(Dh, 1.1920928955078125e-07f));
 
     const bool p1 = t < x;
     const bool p12 = p1 || (t < C14);
     const bool p3 = t < C23;
     const bool p34 = p3 || (t < C24);
-    const bool capped = s4 >= S3;
+    const bool capped = e >= 0.0f;
     const KeyT key_a = p12 ? k1 : (p34 ? k2 : k3);
     const bool b_is_third = !capped && (p1 || (!p12 && p3));
     const KeyT key_b = b_is_third ? k3 : k4;
 
-    Pick24 r;
-    r.ia = pos(key_a);
-    r.ib = pos(key_b);
+    Pick24<KeyT> r;
+    r.key_a = key_a;
+    r.key_b = key_b;
     r.va = __fmul_rn(0.5f, Dh);
     r.vb = fmaxf(s4, r.va);
     return r;
 }
 
 // ---- bf16 source: x01 = a0 | a1 << 16, x23 = a2 | a3 << 16 ------------------
-// The sort key of an element is its widened magnitude with the position in the
-// two lowest mantissa bits (zero in a widened bf16): as a positive float its
-// order is (magnitude, position).  The first comparator layer takes absolute
-// values, which strips the sign for free.
+// The sort key of an element is one byte permute of its source word:
+//   bits 31..16  the bf16 itself (widened to binary32 it is the element),
+//   bits 15..14  its position in the block, bits 13..8 zero,
+//   bits  7..0   a copy of the bf16's high byte (bit 7 = its sign).
+// The first comparator layer takes absolute values, which strips bit 31 for free;
+// as positive floats the keys then order by (magnitude, position), and the
+// survivors' keys still carry position and sign, so nothing is looked up again.
 // Outputs: `out` = the two survivors as bf16 (lower position in the low half),
-// and the group's nibble idx0 | idx1 << 2.
+// `nibble` = idx0 | idx1 << 2.
 __device__ __forceinline__ void mvue_2of4_bf16(uint32_t x01, uint32_t x23, uint32_t word,
                                                uint32_t* out, uint32_t* nibble) {
-    const float f0 = __uint_as_float(__byte_perm(x01, 0u, 0x1054));
-    const float f1 = __uint_as_float(__byte_perm(x01, 1u, 0x3254));
-    const float f2 = __uint_as_float(__byte_perm(x23, 2u, 0x1054));
-    const float f3 = __uint_as_float(__byte_perm(x23, 3u, 0x3254));
+    const float f0 = __uint_as_float(__byte_perm(x01, 0x00u, 0x1041));
+    const float f1 = __uint_as_float(__byte_perm(x01, 0x40u, 0x3243));
+    const float f2 = __uint_as_float(__byte_perm(x23, 0x80u, 0x1041));
+    const float f3 = __uint_as_float(__byte_perm(x23, 0xC0u, 0x3243));
     const float lo01 = fminf(fabsf(f0), fabsf(f1)), hi01 = fmaxf(fabsf(f0), fabsf(f1));
     const float lo23 = fminf(fabsf(f2), fabsf(f3)), hi23 = fmaxf(fabsf(f2), fabsf(f3));
     const float k1 = fminf(lo01, lo23), mid_a = fmaxf(lo01, lo23);
     const float mid_b = fminf(hi01, hi23), k4 = fmaxf(hi01, hi23);
     const float k2 = fminf(mid_a, mid_b), k3 = fmaxf(mid_a, mid_b);
 
-    const Pick24 r = pick_2of4(
+    const Pick24<float> r = pick_2of4(
         k1, k2, k3, k4, word,
-        [](float k) { return __uint_as_float(__float_as_uint(k) & 0xFFFF0000u); },
-        [](float k) { return __float_as_uint(k) & 3u; });
+        [](float k) { return __uint_as_float(__float_as_uint(k) & 0xFFFF0000u); });
 
-    // byte 2 i + 1 of {x01, x23} carries the sign of element i in its top bit
-    const uint32_t sel = (r.ia << 5) | (r.ib << 13) | 0x1010u;
-    const uint32_t signs = __byte_perm(x01, x23, sel) & 0x80008000u;
-    const uint32_t ab = pack_bf16x2(r.va, r.vb) | signs;        // a low, b high
-    const bool swap = r.ia > r.ib;
-    *out = swap ? __byte_perm(ab, 0u, 0x1032) : ab;
-    *nibble = swap ? (r.ib | (r.ia << 2)) : (r.ia | (r.ib << 2));
+    const uint32_t ua = __float_as_uint(r.key_a), ub = __float_as_uint(r.key_b);
+    const uint32_t signs = __byte_perm(ua, ub, 0x4000) & 0x80008000u;   // byte 1 <- a's sign byte, byte 3 <- b's
+    const uint32_t ab = pack_bf16x2(r.va, r.vb) | signs;                // a low, b high
+    const uint32_t pa = ua << 16, pb = ub << 16;                        // position in the top two bits
+    const bool swap = pa > pb;
+    *out = __byte_perm(ab, 0u, swap ? 0x1032u : 0x3210u);
+    // (p >> 30) and (p >> 28) as high products: bits 29..28 of p are zero, so p >> 28 = position << 2
+    const uint32_t nib_ab = __umulhi(pa, 4u) + __umulhi(pb, 16u);
+    const uint32_t nib_ba = __umulhi(pb, 4u) + __umulhi(pa, 16u);
+    *nibble = swap ? nib_ba : nib_ab;
 }
 
 // ---- binary32 source ---------------------------------------------------------
@@ -176,17 +204,17 @@ __device__ __forceinline__ void mvue_2of4_f32(uint32_t b0, uint32_t b1, uint32_t
     };
     uint64_t k1 = make(b0, 0u), k2 = make(b1, 1u), k3 = make(b2, 2u), k4 = make(b3, 3u);
     cswap(k1, k2); cswap(k3, k4); cswap(k1, k3); cswap(k2, k4); cswap(k2, k3);
-    const Pick24 r = pick_2of4(
+    const Pick24<uint64_t> r = pick_2of4(
         k1, k2, k3, k4, word,
-        [](uint64_t k) { return __uint_as_float((uint32_t)(k >> 2)); },
-        [](uint64_t k) { return (uint32_t)k & 3u; });
-    const uint32_t sa = (r.ia == 0 ? b0 : (r.ia == 1 ? b1 : (r.ia == 2 ? b2 : b3))) & 0x80000000u;
-    const uint32_t sb = (r.ib == 0 ? b0 : (r.ib == 1 ? b1 : (r.ib == 2 ? b2 : b3))) & 0x80000000u;
+        [](uint64_t k) { return __uint_as_float((uint32_t)(k >> 2)); });
+    const uint32_t ia = (uint32_t)r.key_a & 3u, ib = (uint32_t)r.key_b & 3u;
+    const uint32_t sa = (ia == 0 ? b0 : (ia == 1 ? b1 : (ia == 2 ? b2 : b3))) & 0x80000000u;
+    const uint32_t sb = (ib == 0 ? b0 : (ib == 1 ? b1 : (ib == 2 ? b2 : b3))) & 0x80000000u;
     const float va = __uint_as_float(__float_as_uint(r.va) | sa);
     const float vb = __uint_as_float(__float_as_uint(r.vb) | sb);
-    const bool swap = r.ia > r.ib;
+    const bool swap = ia > ib;
     *out = swap ? pack_bf16x2(vb, va) : pack_bf16x2(va, vb);
-    *nibble = swap ? (r.ib | (r.ia << 2)) : (r.ia | (r.ib << 2));
+    *nibble = swap ? (ib | (ia << 2)) : (ia | (ib << 2));
 }
 
 }  // namespace mvue

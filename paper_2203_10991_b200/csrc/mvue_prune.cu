@@ -33,7 +33,7 @@ __device__ __forceinline__ void prune_unit_bf16(const uint32_t (&raw)[8], uint64
         for (int j = 0; j < 4; ++j) {
             uint32_t nib;
             mvue_2of4_bf16(raw[2 * j], raw[2 * j + 1], words[j], &v[j], &nib);
-            meta |= nib << (4 * j);
+            meta += nib << (4 * j);
         }
     } else {
         const uint4 wa = philox4x32_10(2 * unit_index, rk);
@@ -41,12 +41,9 @@ __device__ __forceinline__ void prune_unit_bf16(const uint32_t (&raw)[8], uint64
         const uint32_t words[8] = {wa.x, wa.y, wa.z, wa.w, wb.x, wb.y, wb.z, wb.w};
 #pragma unroll
         for (int j = 0; j < 4; ++j) {
-            float v0, v1;
-            const uint32_t x0 = raw[2 * j], x1 = raw[2 * j + 1];
-            const bool k0 = mvue_1of2(__uint_as_float(x0 << 16), __uint_as_float(x0 & 0xFFFF0000u), words[2 * j], &v0);
-            const bool k1 = mvue_1of2(__uint_as_float(x1 << 16), __uint_as_float(x1 & 0xFFFF0000u), words[2 * j + 1], &v1);
-            v[j] = pack_bf16x2(v0, v1);
-            meta |= (k0 ? 0u : (1u << (4 * j))) | (k1 ? (8u << (4 * j)) : (12u << (4 * j)));
+            uint32_t nib;
+            mvue_1of2x2_bf16(raw[2 * j], raw[2 * j + 1], words[2 * j], words[2 * j + 1], &v[j], &nib);
+            meta += nib << (4 * j);
         }
     }
     *out_values = make_uint4(v[0], v[1], v[2], v[3]);
@@ -90,127 +87,146 @@ __device__ __forceinline__ void prune_unit_f32(const uint32_t (&b)[16], uint64_t
 // slot = r * units_per_row + c.  kLinear: the tensor is contiguous and unsharded,
 // so the input offset and the generator call number are linear in the slot.
 template <int M, bool kBf16, bool kLinear>
-__global__ void __launch_bounds__(256)
+__global__ void __launch_bounds__(256, kBf16 ? 6 : 4)
 prune_axis1_kernel(const void* __restrict__ g, int64_t n_slots, int64_t units_per_row, int64_t ld,
                    int64_t units_per_row_total, int64_t unit_offset, RoundKeys rk,
                    uint4* __restrict__ values, uint16_t* __restrict__ meta) {
-    const int64_t stride = (int64_t)gridDim.x * blockDim.x;
-    for (int64_t slot = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; slot < n_slots; slot += stride) {
-        int64_t elem_off;
-        uint64_t unit;
-        if (kLinear) {
-            elem_off = slot * 16;
-            unit = (uint64_t)slot;
-        } else {
-            const int64_t r = slot / units_per_row;
-            const int64_t c = slot - r * units_per_row;
-            elem_off = r * ld + c * 16;
-            unit = (uint64_t)r * (uint64_t)units_per_row_total + (uint64_t)(unit_offset + c);
-        }
-        uint4 v;
-        uint32_t mt;
-        if (kBf16) {
-            const char* p = reinterpret_cast<const char*>(g) + elem_off * 2;
-            const uint4 x = ldg128(p), y = ldg128(p + 16);
-            const uint32_t raw[8] = {x.x, x.y, x.z, x.w, y.x, y.y, y.z, y.w};
-            prune_unit_bf16<M>(raw, unit, rk, &v, &mt);
-        } else {
-            const char* p = reinterpret_cast<const char*>(g) + elem_off * 4;
-            uint32_t b[16];
+    constexpr int U = 1;                              // units per thread per trip, loads issued first
+    constexpr int LW = kBf16 ? 2 : 4;                 // 16-byte loads per unit
+    const int64_t trip = (int64_t)blockDim.x * U;
+    for (int64_t base = (int64_t)blockIdx.x * trip; base < n_slots; base += (int64_t)gridDim.x * trip) {
+        uint4 in[U][LW];
+        uint64_t unit[U];
 #pragma unroll
-            for (int i = 0; i < 4; ++i) {
-                const uint4 x = ldg128(p + 16 * i);
-                b[4 * i] = x.x; b[4 * i + 1] = x.y; b[4 * i + 2] = x.z; b[4 * i + 3] = x.w;
+        for (int u = 0; u < U; ++u) {
+            const int64_t slot = base + (int64_t)u * blockDim.x + threadIdx.x;
+            if (slot < n_slots) {
+                int64_t elem_off;
+                if (kLinear) {
+                    elem_off = slot * 16;
+                    unit[u] = (uint64_t)slot;
+                } else {
+                    const int64_t r = slot / units_per_row;
+                    const int64_t c = slot - r * units_per_row;
+                    elem_off = r * ld + c * 16;
+                    unit[u] = (uint64_t)r * (uint64_t)units_per_row_total + (uint64_t)(unit_offset + c);
+                }
+                const char* p = reinterpret_cast<const char*>(g) + elem_off * (kBf16 ? 2 : 4);
+#pragma unroll
+                for (int i = 0; i < LW; ++i) in[u][i] = ldg128(p + 16 * i);
             }
-            prune_unit_f32<M>(b, unit, rk, &v, &mt);
         }
-        values[slot] = v;
-        meta[slot] = (uint16_t)mt;
+#pragma unroll
+        for (int u = 0; u < U; ++u) {
+            const int64_t slot = base + (int64_t)u * blockDim.x + threadIdx.x;
+            if (slot < n_slots) {
+                uint4 v;
+                uint32_t mt;
+                if (kBf16) {
+                    const uint32_t raw[8] = {in[u][0].x, in[u][0].y, in[u][0].z, in[u][0].w,
+                                             in[u][1].x, in[u][1].y, in[u][1].z, in[u][1].w};
+                    prune_unit_bf16<M>(raw, unit[u], rk, &v, &mt);
+                } else {
+                    uint32_t b[16];
+#pragma unroll
+                    for (int i = 0; i < 4; ++i) {
+                        b[4 * i] = (&in[u][i].x)[0]; b[4 * i + 1] = (&in[u][i].x)[1];
+                        b[4 * i + 2] = (&in[u][i].x)[2]; b[4 * i + 3] = (&in[u][i].x)[3];
+                    }
+                    prune_unit_f32<M>(b, unit[u], rk, &v, &mt);
+                }
+                values[slot] = v;
+                meta[slot] = (uint16_t)mt;
+            }
+        }
     }
 }
 
 // ---- axis 0 ---------------------------------------------------------------
 // g is [K x C] row-major; A = g^T.  A thread block owns a tile of 256 rows (16
-// strips of 16) by 8 column chunks of 16 bytes; thread (strip, chunk) loads its
-// 16 x 16-byte strip with coalesced row reads, prunes each column, and stages
-// the packed outputs in shared memory (values: per column 16 slots of 16 bytes,
-// slot index XOR chunk to avoid bank conflicts; metadata: per column 16 x 2
-// bytes) so that the tile leaves as contiguous runs of 256 / 32 bytes per
-// column of g.
+// strips of 16, one warp per strip) by 64 columns (two per lane).  Each lane reads
+// its two columns of every row of the strip (a warp reads one 128-byte line of
+// bf16, two of binary32, per row), prunes both columns, and stages the packed
+// outputs in shared memory (values: per column 16 slots of 16 bytes, slot index
+// XOR lane to avoid bank conflicts; metadata: per column 16 x 2 bytes) so that
+// the tile leaves as contiguous runs of 256 / 32 bytes per column of g.
 constexpr int kTileStrips = 16;
-constexpr int kTileChunks = 8;
+constexpr int kTileCols = 64;
 constexpr int kMetaPitch = 36;                       // bytes per staged metadata row
 
 template <int M, bool kBf16>
-__global__ void __launch_bounds__(kTileStrips * kTileChunks)
-prune_axis0_kernel(const void* __restrict__ g, int64_t n_strips, int64_t n_chunks, int64_t ld,
+__global__ void __launch_bounds__(kTileStrips * 32, kBf16 ? 3 : 2)
+prune_axis0_kernel(const void* __restrict__ g, int64_t n_strips, int64_t n_cols, int64_t ld,
                    int64_t units_per_row_total, int64_t unit_offset, RoundKeys rk,
                    uint4* __restrict__ values, uint16_t* __restrict__ meta) {
-    constexpr int CW = kBf16 ? 8 : 4;                // columns per 16-byte chunk
-    constexpr int TC = CW * kTileChunks;             // columns per tile
     constexpr int ES = kBf16 ? 2 : 4;
-    __shared__ uint4 s_val[TC * kTileStrips];
-    __shared__ __align__(16) unsigned char s_meta[TC * kMetaPitch];
+    constexpr int NT = kTileStrips * 32;
+    __shared__ uint4 s_val[kTileCols * kTileStrips];
+    __shared__ __align__(16) unsigned char s_meta[kTileCols * kMetaPitch];
 
     const int tid = threadIdx.x;
-    const int chunk_l = tid & (kTileChunks - 1);
-    const int strip_l = tid >> 3;
+    const int lane = tid & 31;
+    const int strip_l = tid >> 5;
     const int64_t strip0 = (int64_t)blockIdx.x * kTileStrips;
-    const int64_t chunk0 = (int64_t)blockIdx.y * kTileChunks;
+    const int64_t col0 = (int64_t)blockIdx.y * kTileCols;
     const int64_t strip = strip0 + strip_l;
-    const int64_t chunk = chunk0 + chunk_l;
+    const int64_t col = col0 + 2 * lane;             // this lane's first column (n_cols is even)
 
-    if (strip < n_strips && chunk < n_chunks) {
-        const char* p = reinterpret_cast<const char*>(g) + ((strip * 16) * ld) * ES + chunk * 16;
-        uint4 rows[16];
+    if (strip < n_strips && col < n_cols) {
+        const char* p = reinterpret_cast<const char*>(g) + ((strip * 16) * ld + col) * ES;
+        uint32_t w[16][kBf16 ? 1 : 2];
 #pragma unroll
-        for (int i = 0; i < 16; ++i) rows[i] = ldg128(p + (int64_t)i * ld * ES);
+        for (int i = 0; i < 16; ++i) {
+            if (kBf16) {
+                w[i][0] = __ldg(reinterpret_cast<const uint32_t*>(p + (int64_t)i * ld * ES));
+            } else {
+                const uint2 t = __ldg(reinterpret_cast<const uint2*>(p + (int64_t)i * ld * ES));
+                w[i][0] = t.x;
+                w[i][kBf16 ? 0 : 1] = t.y;
+            }
+        }
         const uint64_t unit_base = (uint64_t)(unit_offset + strip);
 #pragma unroll
-        for (int e = 0; e < CW; ++e) {
-            const int col_l = chunk_l * CW + e;      // column inside the tile = row of A
-            const uint64_t unit = (uint64_t)(chunk * CW + e) * (uint64_t)units_per_row_total + unit_base;
+        for (int e = 0; e < 2; ++e) {
+            const int col_l = 2 * lane + e;          // column inside the tile = row of A
+            const uint64_t unit = (uint64_t)(col + e) * (uint64_t)units_per_row_total + unit_base;
             uint4 v;
             uint32_t mt;
             if (kBf16) {
                 uint32_t raw[8];
 #pragma unroll
-                for (int j = 0; j < 8; ++j) {
-                    const uint32_t w0 = (&rows[2 * j].x)[e >> 1], w1 = (&rows[2 * j + 1].x)[e >> 1];
-                    raw[j] = __byte_perm(w0, w1, (e & 1) ? 0x7632 : 0x5410);
-                }
+                for (int j = 0; j < 8; ++j)
+                    raw[j] = __byte_perm(w[2 * j][0], w[2 * j + 1][0], e ? 0x7632 : 0x5410);
                 prune_unit_bf16<M>(raw, unit, rk, &v, &mt);
             } else {
                 uint32_t b[16];
 #pragma unroll
-                for (int i = 0; i < 16; ++i) b[i] = (&rows[i].x)[e];
+                for (int i = 0; i < 16; ++i) b[i] = w[i][kBf16 ? 0 : e];
                 prune_unit_f32<M>(b, unit, rk, &v, &mt);
             }
-            s_val[col_l * kTileStrips + (strip_l ^ chunk_l)] = v;
+            s_val[col_l * kTileStrips + (strip_l ^ (lane & 15))] = v;
             *reinterpret_cast<uint16_t*>(&s_meta[col_l * kMetaPitch + strip_l * 2]) = (uint16_t)mt;
         }
     }
     __syncthreads();
 
     const int64_t strips_here = n_strips - strip0 < kTileStrips ? n_strips - strip0 : kTileStrips;
-    // values: TC columns x 16 slots of 16 bytes; 16 consecutive threads write one column's run
+    // values: 64 columns x 16 slots of 16 bytes; 16 consecutive threads write one column's run
 #pragma unroll
-    for (int it = 0; it < TC * kTileStrips / (kTileStrips * kTileChunks); ++it) {
-        const int idx = it * (kTileStrips * kTileChunks) + tid;
+    for (int it = 0; it < kTileCols * kTileStrips / NT; ++it) {
+        const int idx = it * NT + tid;
         const int col_l = idx >> 4, j = idx & 15;
-        const int64_t col = chunk0 * CW + col_l;
-        if (j < strips_here && col < n_chunks * CW)
-            values[col * n_strips + strip0 + j] = s_val[col_l * kTileStrips + (j ^ (col_l / CW))];
+        const int64_t c = col0 + col_l;
+        if (j < strips_here && c < n_cols)
+            values[c * n_strips + strip0 + j] = s_val[col_l * kTileStrips + (j ^ ((col_l >> 1) & 15))];
     }
-    // metadata: TC columns x 32 bytes; 8 consecutive threads write one column's run as words
-#pragma unroll
-    for (int it = 0; it < TC * 8 / (kTileStrips * kTileChunks); ++it) {
-        const int idx = it * (kTileStrips * kTileChunks) + tid;
-        const int col_l = idx >> 3, wd = idx & 7;
-        const int64_t col = chunk0 * CW + col_l;
-        if (col < n_chunks * CW) {
+    // metadata: 64 columns x 32 bytes; 8 consecutive threads write one column's run as words
+    {
+        const int col_l = tid >> 3, wd = tid & 7;
+        const int64_t c = col0 + col_l;
+        if (c < n_cols) {
             const uint32_t word = *reinterpret_cast<const uint32_t*>(&s_meta[col_l * kMetaPitch + wd * 4]);
-            uint16_t* dst = meta + col * n_strips + strip0 + 2 * wd;
+            uint16_t* dst = meta + c * n_strips + strip0 + 2 * wd;
             const bool word_ok = (reinterpret_cast<uintptr_t>(dst) & 3u) == 0;   // odd K/16 misaligns rows
             if (2 * wd + 1 < strips_here && word_ok) {
                 *reinterpret_cast<uint32_t*>(dst) = word;
@@ -252,18 +268,16 @@ cudaError_t launch_prune_t(const PruneArgs& a, cudaStream_t stream) {
         const int64_t n_slots = a.rows * upr;
         const bool linear = (a.ld == a.cols) && (a.k_total == a.cols) && (a.k_offset == 0);
         const int64_t want = (n_slots + 255) / 256;
-        const int grid = (int)(want < (int64_t)a.sm_count * 64 ? want : (int64_t)a.sm_count * 64);
+        const int grid = (int)(want < (int64_t)a.sm_count * 48 ? want : (int64_t)a.sm_count * 48);
         if (linear)
             prune_axis1_kernel<M, kBf16, true><<<grid, 256, 0, stream>>>(a.g, n_slots, upr, a.ld, upr_total, uoff, rk, values, meta);
         else
             prune_axis1_kernel<M, kBf16, false><<<grid, 256, 0, stream>>>(a.g, n_slots, upr, a.ld, upr_total, uoff, rk, values, meta);
     } else {
-        constexpr int CW = kBf16 ? 8 : 4;
         const int64_t n_strips = a.rows / 16;
-        const int64_t n_chunks = a.cols / CW;
         dim3 grid((unsigned)((n_strips + kTileStrips - 1) / kTileStrips),
-                  (unsigned)((n_chunks + kTileChunks - 1) / kTileChunks));
-        prune_axis0_kernel<M, kBf16><<<grid, kTileStrips * kTileChunks, 0, stream>>>(a.g, n_strips, n_chunks, a.ld, upr_total, uoff, rk, values, meta);
+                  (unsigned)((a.cols + kTileCols - 1) / kTileCols));
+        prune_axis0_kernel<M, kBf16><<<grid, kTileStrips * 32, 0, stream>>>(a.g, n_strips, a.cols, a.ld, upr_total, uoff, rk, values, meta);
     }
     return cudaGetLastError();
 }
