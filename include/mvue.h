@@ -114,6 +114,44 @@ MVUE_API int mvue_prune(const void* g, int dtype, int64_t rows, int64_t cols, in
 MVUE_API int mvue_unpack(const void* values, const void* meta, int layout, int64_t mrows, int64_t K,
                 void* dense_bf16, void* stream);
 
+/* Update product with the pruned gradient as the 2:4-sparse operand
+ * (Sec. 1, update equation dC/dW_l = g_l h_{l-1}^T):
+ *   dW[out x in] (+)= theta(g)^T[out x T] . h[T x in]
+ * values/meta: packed theta(g)^T (mvue_prune with axis 0 on g[T x out]);
+ * h: bf16 [T x in], ld ldh; dW: MVUE_F32 or MVUE_BF16 [out x in], ld lddW;
+ * accumulate != 0 adds into dW (MVUE_F32 only).  bf16 x bf16 products, fp32
+ * accumulation on the sparse tensor cores.
+ * workspace: mvue_gemm_workspace_bytes(0, out, in, T) bytes (may be 0, then
+ * NULL is accepted), 16-byte aligned, contents scratch: small outputs with a long
+ * reduction are split along K and summed in a second, deterministic pass.  dev_status: optional device int, receives
+ * MVUE_ERR_DEVICE_TIMEOUT if a bounded pipeline wait expires (then dW is
+ * unspecified); otherwise left untouched.
+ * Preconditions: T a multiple of 64; out, in multiples of 8; pointers and
+ * leading dimensions (in bytes) 16-byte aligned; act_grad needs a bf16 or
+ * MVUE_F32 output without accumulate. */
+MVUE_API int mvue_sparse_update_gemm(const void* values, const void* meta, int layout, int64_t out,
+                            int64_t T, const void* h, int64_t in, int64_t ldh, void* dW,
+                            int dW_dtype, int64_t lddW, int accumulate, void* workspace,
+                            size_t workspace_bytes, int* dev_status, void* stream);
+
+/* Backward product with the pruned gradient as the 2:4-sparse operand
+ * (Sec. 1, backward equation g_l = Diag(f'(z_l)) W_{l+1}^T g_{l+1}, written for
+ * a batch of T rows):
+ *   dh[T x in] = (theta(g)[T x out] . W[out x in]) (* act_grad[T x in])
+ * values/meta: packed theta(g) (mvue_prune with axis 1 on g[T x out]);
+ * W: bf16 [out x in]; act_grad: optional bf16 [T x in] (f'(z)), ld = lddh,
+ * multiplied elementwise in the epilogue, or NULL; dh: MVUE_F32 or MVUE_BF16.
+ * Workspace, dev_status and preconditions as above with K = out. */
+MVUE_API int mvue_sparse_backward_gemm(const void* values, const void* meta, int layout, int64_t T,
+                              int64_t out, const void* W, int64_t in, int64_t ldW,
+                              const void* act_grad, void* dh, int dh_dtype, int64_t lddh,
+                              void* workspace, size_t workspace_bytes, int* dev_status,
+                              void* stream);
+
+/* Scratch bytes the product C[M x N] = A[M x K] . B[K x N] needs
+ * (which: 0 update, 1 backward).  bytes is a HOST pointer. */
+MVUE_API int mvue_gemm_workspace_bytes(int which, int64_t M, int64_t N, int64_t K, size_t* bytes);
+
 MVUE_API const char* mvue_status_string(int status);
 /* Text of the last CUDA error seen by the calling thread ("" if none). */
 MVUE_API const char* mvue_last_cuda_error(void);

@@ -18,7 +18,8 @@ MVUE_F32, MVUE_BF16 = 0, 1
 MVUE_LAYOUT_CANONICAL = 0
 
 EXPORTS = ("mvue_version", "mvue_status_string", "mvue_last_cuda_error", "mvue_packed_sizes",
-           "mvue_prune", "mvue_unpack")
+           "mvue_prune", "mvue_unpack", "mvue_sparse_update_gemm", "mvue_sparse_backward_gemm",
+           "mvue_gemm_workspace_bytes")
 
 
 class MvueError(RuntimeError):
@@ -47,6 +48,11 @@ def lib() -> ctypes.CDLL:
         L.mvue_packed_sizes.argtypes = [i64, i64, ci, ci, ci, ci, szp, szp]
         L.mvue_prune.argtypes = [vp, ci, i64, i64, i64, ci, ci, ci, u64, i64, i64, vp, vp, ci, vp]
         L.mvue_unpack.argtypes = [vp, vp, ci, i64, i64, vp, vp]
+        L.mvue_sparse_update_gemm.argtypes = [vp, vp, ci, i64, i64, vp, i64, i64, vp, ci, i64, ci, vp,
+                                              ctypes.c_size_t, vp, vp]
+        L.mvue_sparse_backward_gemm.argtypes = [vp, vp, ci, i64, i64, vp, i64, i64, vp, vp, ci, i64, vp,
+                                                ctypes.c_size_t, vp, vp]
+        L.mvue_gemm_workspace_bytes.argtypes = [ci, i64, i64, i64, szp]
         _lib = L
     return _lib
 
@@ -101,3 +107,60 @@ def mvue_unpack(values: torch.Tensor, meta: torch.Tensor, layout: int = MVUE_LAY
     _check(lib().mvue_unpack(values.data_ptr(), meta.data_ptr(), layout, mrows, 2 * kh, dense.data_ptr(),
                              _stream_ptr()), "mvue_unpack")
     return dense
+
+
+def mvue_gemm_workspace_bytes(which: int, M: int, N: int, K: int) -> int:
+    b = ctypes.c_size_t()
+    _check(lib().mvue_gemm_workspace_bytes(which, M, N, K, ctypes.byref(b)), "mvue_gemm_workspace_bytes")
+    return b.value
+
+
+def _workspace(which, M, N, K, device, workspace):
+    need = mvue_gemm_workspace_bytes(which, M, N, K)
+    if need == 0:
+        return None, 0
+    if workspace is None or workspace.numel() * workspace.element_size() < need:
+        workspace = torch.empty(need, dtype=torch.uint8, device=device)
+    return workspace, workspace.numel() * workspace.element_size()
+
+
+def mvue_sparse_update_gemm(values: torch.Tensor, meta: torch.Tensor, h: torch.Tensor, *,
+                            out: torch.Tensor | None = None, out_dtype=torch.float32, accumulate: bool = False,
+                            workspace: torch.Tensor | None = None, dev_status: torch.Tensor | None = None,
+                            layout: int = MVUE_LAYOUT_CANONICAL) -> torch.Tensor:
+    """dW[out, in] (+)= theta(g)^T . h with the packed operand of mvue_prune(g, axis=0)."""
+    n_out, half_t = values.shape
+    T, n_in = h.shape
+    assert h.dtype == torch.bfloat16 and h.stride(1) == 1 and 2 * half_t == T
+    if out is None:
+        out = torch.empty((n_out, n_in), dtype=out_dtype, device=h.device)
+    ws, ws_bytes = _workspace(0, n_out, n_in, T, h.device, workspace)
+    _check(lib().mvue_sparse_update_gemm(values.data_ptr(), meta.data_ptr(), layout, n_out, T, h.data_ptr(), n_in,
+                                         h.stride(0), out.data_ptr(), _dtype_code(out), out.stride(0),
+                                         int(accumulate), None if ws is None else ws.data_ptr(), ws_bytes,
+                                         None if dev_status is None else dev_status.data_ptr(), _stream_ptr()),
+           "mvue_sparse_update_gemm")
+    return out
+
+
+def mvue_sparse_backward_gemm(values: torch.Tensor, meta: torch.Tensor, W: torch.Tensor, *,
+                              act_grad: torch.Tensor | None = None, out: torch.Tensor | None = None,
+                              out_dtype=torch.bfloat16, workspace: torch.Tensor | None = None,
+                              dev_status: torch.Tensor | None = None,
+                              layout: int = MVUE_LAYOUT_CANONICAL) -> torch.Tensor:
+    """dh[T, in] = (theta(g) . W) (* act_grad) with the packed operand of mvue_prune(g, axis=1)."""
+    T, half_o = values.shape
+    n_out, n_in = W.shape
+    assert W.dtype == torch.bfloat16 and W.stride(1) == 1 and 2 * half_o == n_out
+    if out is None:
+        out = torch.empty((T, n_in), dtype=out_dtype, device=W.device)
+    if act_grad is not None:
+        assert act_grad.dtype == torch.bfloat16 and act_grad.shape == out.shape and act_grad.stride(0) == out.stride(0)
+    ws, ws_bytes = _workspace(1, T, n_in, n_out, W.device, workspace)
+    _check(lib().mvue_sparse_backward_gemm(values.data_ptr(), meta.data_ptr(), layout, T, n_out, W.data_ptr(), n_in,
+                                           W.stride(0), None if act_grad is None else act_grad.data_ptr(),
+                                           out.data_ptr(), _dtype_code(out), out.stride(0),
+                                           None if ws is None else ws.data_ptr(), ws_bytes,
+                                           None if dev_status is None else dev_status.data_ptr(), _stream_ptr()),
+           "mvue_sparse_backward_gemm")
+    return out

@@ -45,6 +45,30 @@ static int check_nm(int n, int m) {
     return ((n == 1 && m == 2) || (n == 2 && m == 4)) ? MVUE_OK : MVUE_ERR_NM;
 }
 
+static int run_gemm(const void* values, const void* meta, int layout, int64_t M, int64_t N, int64_t K,
+                    const void* B, int64_t ldb, const void* scale, void* C, int c_dtype, int64_t ldc,
+                    int accumulate, void* workspace, size_t workspace_bytes, int* dev_status, void* stream) {
+    if (!values || !meta || !B || !C) return MVUE_ERR_NULL;
+    if (layout != MVUE_LAYOUT_CANONICAL) return MVUE_ERR_LAYOUT;
+    if (c_dtype != MVUE_F32 && c_dtype != MVUE_BF16) return MVUE_ERR_DTYPE;
+    if (accumulate && c_dtype != MVUE_F32) return MVUE_ERR_DTYPE;
+    if (accumulate && scale) return MVUE_ERR_DTYPE;
+    if (M <= 0 || N <= 0 || K <= 0 || K % 64 != 0 || M % 8 != 0 || N % 8 != 0) return MVUE_ERR_SHAPE;
+    if (ldb < N || ldc < N) return MVUE_ERR_SHAPE;
+    if (M > 0x7FFFFFFF || N > 0x7FFFFFFF || K > 0x7FFFFFFF) return MVUE_ERR_SHAPE;
+    const int64_t c_esz = c_dtype == MVUE_BF16 ? 2 : 4;
+    if (!aligned16(values) || !aligned16(meta) || !aligned16(B) || !aligned16(C) || (ldb * 2) % 16 != 0 ||
+        (ldc * c_esz) % 16 != 0 || (scale && (!aligned16(scale) || (ldc * 2) % 16 != 0)))
+        return MVUE_ERR_ALIGN;
+    DeviceInfo dev;
+    if (int s = current_device_info(&dev)) return s;
+    const size_t need = gemm_workspace_bytes(M, N, K, dev.sm_count);
+    if (need > 0 && (!workspace || workspace_bytes < need || !aligned16(workspace))) return MVUE_ERR_WORKSPACE;
+    SparseGemmArgs a{values, meta, M, N, K, B, ldb, C, ldc, c_dtype == MVUE_BF16, accumulate, scale,
+                     workspace, dev_status, dev.sm_count};
+    return launch_sparse_gemm(a, reinterpret_cast<cudaStream_t>(stream));
+}
+
 }  // namespace mvue
 
 using namespace mvue;
@@ -117,6 +141,32 @@ int mvue_unpack(const void* values, const void* meta, int layout, int64_t mrows,
                                   reinterpret_cast<cudaStream_t>(stream));
     if (e != cudaSuccess) { set_cuda_error(e, "mvue_unpack launch"); return MVUE_ERR_CUDA; }
     return MVUE_OK;
+}
+
+int mvue_gemm_workspace_bytes(int which, int64_t M, int64_t N, int64_t K, size_t* bytes) {
+    if (!bytes) return MVUE_ERR_NULL;
+    if (which != 0 && which != 1) return MVUE_ERR_SHAPE;
+    if (M <= 0 || N <= 0 || K <= 0 || K % 64 != 0) return MVUE_ERR_SHAPE;
+    DeviceInfo dev;
+    if (int s = current_device_info(&dev)) return s;
+    *bytes = gemm_workspace_bytes(M, N, K, dev.sm_count);
+    return MVUE_OK;
+}
+
+int mvue_sparse_update_gemm(const void* values, const void* meta, int layout, int64_t out, int64_t T,
+                            const void* h, int64_t in, int64_t ldh, void* dW, int dW_dtype, int64_t lddW,
+                            int accumulate, void* workspace, size_t workspace_bytes, int* dev_status,
+                            void* stream) {
+    return run_gemm(values, meta, layout, out, in, T, h, ldh, nullptr, dW, dW_dtype, lddW, accumulate,
+                    workspace, workspace_bytes, dev_status, stream);
+}
+
+int mvue_sparse_backward_gemm(const void* values, const void* meta, int layout, int64_t T, int64_t out,
+                              const void* W, int64_t in, int64_t ldW, const void* act_grad, void* dh,
+                              int dh_dtype, int64_t lddh, void* workspace, size_t workspace_bytes,
+                              int* dev_status, void* stream) {
+    return run_gemm(values, meta, layout, T, in, out, W, ldW, act_grad, dh, dh_dtype, lddh, 0, workspace,
+                    workspace_bytes, dev_status, stream);
 }
 
 }  // extern "C"

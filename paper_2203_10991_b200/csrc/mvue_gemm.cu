@@ -1,0 +1,500 @@
+// 2:4-sparse GEMM on the 5th-generation tensor cores (tcgen05.mma.sp), sm_100a.
+//
+//   C[M x N] = A[M x K] . B[K x N]
+// A is the MVUE-pruned gradient in packed form: bf16 survivors [M x K/2] (K-major)
+// plus one nibble of positions per group of four, [M x K/8] bytes.  B is dense
+// bf16, row-major [K x N] (N contiguous): the activations h for the update
+// product g^T h, the weights W for the backward product g W (Sec. 1 of the paper).
+//
+// One thread block computes one 128 x 256 output tile over a range of K:
+//   warp 0      TMA producer: per 64-deep K step, the packed A tile (128 x 32 bf16,
+//               64-byte swizzle) and four 64 x 64 boxes of B (128-byte swizzle)
+//   warp 1      MMA issuer: copies the step's metadata from shared to tensor
+//               memory (tcgen05.cp), issues two tcgen05.mma.sp (K = 32 each) with the
+//               fp32 accumulator in tensor memory, commits to the step's "empty"
+//               barrier
+//   warp 2      allocates / frees tensor memory
+//   warps 4-7   stage the metadata: read the nibbles of their rows, rearrange them
+//               into the lane/column order the tensor core expects, write them to
+//               shared memory; afterwards they are the epilogue (tcgen05.ld ->
+//               registers -> global), one quarter of the lanes each.
+// Every wait on an mbarrier is bounded; when a bound expires the block records
+// MVUE_ERR_DEVICE_TIMEOUT in the caller's status word and drains.
+#include <cuda.h>
+#include <cuda_bf16.h>
+#include <cuda_runtime.h>
+#include <cudaTypedefs.h>
+
+#include <cstdint>
+#include <mutex>
+
+#include "../../include/mvue.h"
+#include "mvue_internal.h"
+
+namespace mvue {
+namespace {
+
+constexpr int BM = 128;
+constexpr int BN = 256;
+constexpr int BK = 64;                     // logical K per pipeline step (two MMAs of K = 32)
+constexpr int kStages = 5;
+constexpr int kABytes = BM * (BK / 2) * 2; // 8 KiB: 128 rows x 64 bytes of survivors
+constexpr int kBBoxBytes = 64 * BK * 2;    // 8 KiB: 64 k-rows x 128 bytes
+constexpr int kBBytes = (BN / 64) * kBBoxBytes;
+constexpr int kEBytes = BM * 16;           // 2 KiB: 16 bytes per tensor-memory lane
+constexpr int kStageBytes = kABytes + kBBytes + kEBytes;
+constexpr int kSmemBytes = kStages * kStageBytes + 1024 /*alignment slack*/ + 256 /*barriers*/;
+constexpr int kThreads = 256;
+constexpr uint32_t kTmemCols = 512;
+constexpr uint32_t kTmemECol = 256;        // metadata columns start after the accumulator
+constexpr uint32_t kSpinLimit = 1u << 22;  // bounded waits: ~4M polls with back-off
+
+__device__ __forceinline__ uint32_t smem_u32(const void* p) {
+    return static_cast<uint32_t>(__cvta_generic_to_shared(p));
+}
+__device__ __forceinline__ void mbar_init(uint32_t bar, uint32_t count) {
+    asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(bar), "r"(count));
+}
+__device__ __forceinline__ void mbar_expect_tx(uint32_t bar, uint32_t bytes) {
+    asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "r"(bytes) : "memory");
+}
+__device__ __forceinline__ void mbar_arrive(uint32_t bar) {
+    asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(bar) : "memory");
+}
+__device__ __forceinline__ bool mbar_try_wait(uint32_t bar, uint32_t parity) {
+    uint32_t ok;
+    asm volatile(
+        "{\n\t.reg .pred p;\n\t"
+        "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
+        "selp.u32 %0, 1, 0, p;\n\t}"
+        : "=r"(ok) : "r"(bar), "r"(parity) : "memory");
+    return ok != 0;
+}
+// Bounded wait.  Returns false (and raises the block's abort flag) when the bound expires
+// or another role has already given up.
+__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile int* abort_flag) {
+    for (uint32_t spin = 0; spin < kSpinLimit; ++spin) {
+        if (mbar_try_wait(bar, parity)) return true;
+        if (*abort_flag) return false;
+        if (spin > 64) __nanosleep(spin > 4096 ? 256 : 32);
+    }
+    *abort_flag = 1;
+    return false;
+}
+__device__ __forceinline__ void tma_load_2d(uint32_t dst, const CUtensorMap* map, int x, int y, uint32_t bar) {
+    asm volatile(
+        "cp.async.bulk.tensor.2d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3}], [%4];"
+        ::"r"(dst), "l"(map), "r"(x), "r"(y), "r"(bar) : "memory");
+}
+__device__ __forceinline__ void tmem_alloc(uint32_t dst_smem, uint32_t cols) {
+    asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(dst_smem), "r"(cols) : "memory");
+}
+__device__ __forceinline__ void tmem_relinquish() {
+    asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+}
+__device__ __forceinline__ void tmem_dealloc(uint32_t addr, uint32_t cols) {
+    asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(addr), "r"(cols) : "memory");
+}
+__device__ __forceinline__ void tc_fence_before() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
+__device__ __forceinline__ void tc_fence_after() { asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory"); }
+__device__ __forceinline__ void tc_commit(uint32_t bar) {
+    asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(bar) : "memory");
+}
+__device__ __forceinline__ void tc_copy_128x128b(uint32_t tmem_addr, uint64_t smem_desc) {
+    asm volatile("tcgen05.cp.cta_group::1.128x128b [%0], %1;" ::"r"(tmem_addr), "l"(smem_desc) : "memory");
+}
+__device__ __forceinline__ void tc_mma_sp_bf16(uint32_t tmem_d, uint64_t a_desc, uint64_t b_desc,
+                                               uint32_t tmem_meta, uint32_t idesc, uint32_t accumulate) {
+    const uint32_t zero = 0u;                 // no output lane is disabled
+    asm volatile(
+        "{\n\t.reg .pred p;\n\t"
+        "setp.ne.b32 p, %5, 0;\n\t"
+        "tcgen05.mma.sp.cta_group::1.kind::f16 [%0], %1, %2, [%3], %4, {%6, %6, %6, %6}, p;\n\t}"
+        ::"r"(tmem_d), "l"(a_desc), "l"(b_desc), "r"(tmem_meta), "r"(idesc), "r"(accumulate), "r"(zero) : "memory");
+}
+__device__ __forceinline__ void tmem_ld_32x32b_x32(uint32_t taddr, uint32_t (&v)[32]) {
+    asm volatile(
+        "tcgen05.ld.sync.aligned.32x32b.x32.b32 "
+        "{%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15, "
+        "%16, %17, %18, %19, %20, %21, %22, %23, %24, %25, %26, %27, %28, %29, %30, %31}, [%32];"
+        : "=r"(v[0]), "=r"(v[1]), "=r"(v[2]), "=r"(v[3]), "=r"(v[4]), "=r"(v[5]), "=r"(v[6]), "=r"(v[7]),
+          "=r"(v[8]), "=r"(v[9]), "=r"(v[10]), "=r"(v[11]), "=r"(v[12]), "=r"(v[13]), "=r"(v[14]), "=r"(v[15]),
+          "=r"(v[16]), "=r"(v[17]), "=r"(v[18]), "=r"(v[19]), "=r"(v[20]), "=r"(v[21]), "=r"(v[22]), "=r"(v[23]),
+          "=r"(v[24]), "=r"(v[25]), "=r"(v[26]), "=r"(v[27]), "=r"(v[28]), "=r"(v[29]), "=r"(v[30]), "=r"(v[31])
+        : "r"(taddr) : "memory");
+}
+__device__ __forceinline__ void tmem_ld_wait() { asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory"); }
+
+// Shared-memory matrix descriptor (64 bits): start address, leading / stride byte offsets
+// (all >> 4), descriptor version 1, swizzle mode in the top three bits.
+__device__ __forceinline__ uint64_t make_smem_desc(uint32_t addr, uint32_t lbo_bytes, uint32_t sbo_bytes,
+                                                   uint32_t swizzle_code) {
+    return (uint64_t)((addr >> 4) & 0x3FFFu) | ((uint64_t)((lbo_bytes >> 4) & 0x3FFFu) << 16) |
+           ((uint64_t)((sbo_bytes >> 4) & 0x3FFFu) << 32) | (1ull << 46) | ((uint64_t)swizzle_code << 61);
+}
+constexpr uint32_t kSwizzleNone = 0, kSwizzle128B = 2, kSwizzle64B = 4;
+
+// Instruction descriptor of tcgen05.mma.sp.kind::f16: sparse, fp32 accumulate, bf16 x bf16,
+// A K-major, B N-major, N = 256, M = 128.
+constexpr uint32_t kInstrDesc = (1u << 2) /*sparse*/ | (1u << 4) /*D = f32*/ | (1u << 7) /*A = bf16*/ |
+                                (1u << 10) /*B = bf16*/ | (0u << 15) /*A K-major*/ | (1u << 16) /*B N-major*/ |
+                                ((uint32_t)(BN >> 3) << 17) | ((uint32_t)(BM >> 4) << 24);
+
+struct GemmParams {
+    const uint8_t* meta;      // canonical nibbles [M x K/8]
+    int64_t M, N, K;
+    int64_t k_steps_per_split;
+    float* partial;           // split-K workspace [splits x M x N] (splits > 1) else unused
+    void* C;                  // output when splits == 1
+    int64_t ldc;
+    const __nv_bfloat16* scale;  // optional elementwise multiplier [M x N], ld = ldc (splits == 1 path)
+    int c_is_bf16;
+    int accumulate;
+    int splits;
+    int* dev_status;
+};
+
+__global__ void __launch_bounds__(kThreads, 1)
+sparse_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ CUtensorMap map_b,
+                   const GemmParams p) {
+    extern __shared__ uint8_t smem_raw[];
+    const uint32_t smem_base = (smem_u32(smem_raw) + 1023u) & ~1023u;
+    uint8_t* smem_gen = smem_raw + (smem_base - smem_u32(smem_raw));
+    const uint32_t bar_base = smem_base + kStages * kStageBytes;
+    // barriers: full[kStages], empty[kStages], acc_done; then the tensor-memory base word and the abort flag
+    auto full_bar = [&](int s) { return bar_base + 8u * s; };
+    auto empty_bar = [&](int s) { return bar_base + 8u * (kStages + s); };
+    const uint32_t acc_bar = bar_base + 8u * (2 * kStages);
+    uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(smem_gen + kStages * kStageBytes + 8 * (2 * kStages + 1));
+    volatile int* abort_flag = reinterpret_cast<volatile int*>(tmem_slot + 1);
+
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const int64_t m0 = (int64_t)blockIdx.y * BM;
+    const int64_t n0 = (int64_t)blockIdx.x * BN;
+    const int split = blockIdx.z;
+    const int64_t total_steps = p.K / BK;
+    const int64_t step_begin = (int64_t)split * p.k_steps_per_split;
+    int64_t step_end = step_begin + p.k_steps_per_split;
+    if (step_end > total_steps) step_end = total_steps;
+    const int64_t n_steps = step_end > step_begin ? step_end - step_begin : 0;
+
+    if (threadIdx.x == 0) {
+        for (int s = 0; s < kStages; ++s) {
+            mbar_init(full_bar(s), 1 + 4);   // TMA thread (with byte count) + one arrival per metadata warp
+            mbar_init(empty_bar(s), 1);      // tcgen05.commit
+        }
+        mbar_init(acc_bar, 1);
+        *abort_flag = 0;
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    }
+    // the upper 8 bytes of every metadata lane slot are never used: clear them once
+    for (int i = threadIdx.x; i < kStages * BM; i += kThreads) {
+        const int s = i / BM, l = i % BM;
+        *reinterpret_cast<uint2*>(smem_gen + s * kStageBytes + kABytes + kBBytes + l * 16 + 8) = make_uint2(0u, 0u);
+    }
+    if (warp == 2) {
+        tmem_alloc(smem_u32(tmem_slot), kTmemCols);
+        tmem_relinquish();
+    }
+    asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+    tc_fence_before();
+    __syncthreads();
+    tc_fence_after();
+    const uint32_t tmem_base = *tmem_slot;
+
+    if (warp == 0) {
+        // ------------------------------------------------------------ TMA producer
+        if (lane == 0) {
+            for (int64_t i = 0; i < n_steps; ++i) {
+                const int s = (int)(i % kStages);
+                const uint32_t use = (uint32_t)(i / kStages);
+                if (use > 0 && !mbar_wait(empty_bar(s), (use - 1) & 1u, abort_flag)) break;
+                const uint32_t a_dst = smem_base + s * kStageBytes;
+                const uint32_t b_dst = a_dst + kABytes;
+                const int k = (int)((step_begin + i) * BK);
+                mbar_expect_tx(full_bar(s), kABytes + kBBytes);
+                tma_load_2d(a_dst, &map_a, k / 2, (int)m0, full_bar(s));
+#pragma unroll
+                for (int j = 0; j < BN / 64; ++j)
+                    tma_load_2d(b_dst + j * kBBoxBytes, &map_b, (int)n0 + 64 * j, k, full_bar(s));
+            }
+        }
+    } else if (warp == 1) {
+        // ------------------------------------------------------------ MMA issuer
+        if (lane == 0) {
+            bool ok = true;
+            for (int64_t i = 0; i < n_steps && ok; ++i) {
+                const int s = (int)(i % kStages);
+                const uint32_t use = (uint32_t)(i / kStages);
+                ok = mbar_wait(full_bar(s), use & 1u, abort_flag);
+                if (!ok) break;
+                tc_fence_after();
+                const uint32_t a_addr = smem_base + s * kStageBytes;
+                const uint32_t b_addr = a_addr + kABytes;
+                const uint32_t e_addr = b_addr + kBBytes;
+                const uint32_t tmem_e = tmem_base + kTmemECol + 4u * s;
+                // metadata: 128 lanes x 16 bytes, rows contiguous (8-row core matrices 128 bytes apart)
+                tc_copy_128x128b(tmem_e, make_smem_desc(e_addr, 16, 128, kSwizzleNone));
+#pragma unroll
+                for (int kb = 0; kb < BK / 32; ++kb) {
+                    // A: K-major, 64-byte swizzle, 8-row groups 512 bytes apart; 32 bytes per K = 32 block
+                    const uint64_t a_desc = make_smem_desc(a_addr + kb * 32, 16, 512, kSwizzle64B);
+                    // B: N-major, 128-byte swizzle; 64-column blocks kBBoxBytes apart (leading),
+                    //    8-row groups 1024 bytes apart (stride); 32 k-rows per block = 4096 bytes
+                    const uint64_t b_desc = make_smem_desc(b_addr + kb * 4096, kBBoxBytes, 1024, kSwizzle128B);
+                    tc_mma_sp_bf16(tmem_base, a_desc, b_desc, tmem_e, kInstrDesc | (uint32_t)kb,
+                                   (i > 0 || kb > 0) ? 1u : 0u);
+                }
+                tc_commit(empty_bar(s));     // frees the stage (and its metadata columns) when the MMAs retire
+            }
+            tc_commit(acc_bar);              // accumulator complete
+        }
+    } else if (warp >= 4) {
+        // ------------------------------------------------------------ metadata staging
+        const int L = threadIdx.x - 128;                 // tensor-memory lane 0..127
+        const int j = L & 7, h = (L >> 3) & 1, G = L >> 4;
+        const int64_t r0 = m0 + 16 * G + j, r1 = r0 + 8; // the two rows that share this lane
+        const int64_t pitch = p.K / 8;
+        const uint8_t* row0 = p.meta + (r0 < p.M ? r0 : 0) * pitch + (step_begin * BK) / 8;
+        const uint8_t* row1 = p.meta + (r1 < p.M ? r1 : 0) * pitch + (step_begin * BK) / 8;
+        constexpr int PD = 4;                            // prefetch distance in steps
+        uint2 q0[PD], q1[PD];
+#pragma unroll
+        for (int d = 0; d < PD; ++d) {
+            if (d < n_steps) {
+                q0[d] = __ldg(reinterpret_cast<const uint2*>(row0 + 8 * d));
+                q1[d] = __ldg(reinterpret_cast<const uint2*>(row1 + 8 * d));
+            }
+        }
+        bool ok = true;
+        for (int64_t i0 = 0; i0 < n_steps && ok; i0 += PD) {
+#pragma unroll
+            for (int d = 0; d < PD; ++d) {
+                const int64_t i = i0 + d;
+                if (i >= n_steps || !ok) break;
+                const int s = (int)(i % kStages);
+                const uint32_t use = (uint32_t)(i / kStages);
+                if (use > 0) ok = mbar_wait(empty_bar(s), (use - 1) & 1u, abort_flag);
+                if (!ok) break;
+                // 16 bits = four nibbles = 16 logical k; x: k 0..31 of the step, y: k 32..63
+                uint2 a = q0[d], b = q1[d];
+                if (r0 >= p.M) a = make_uint2(0x44444444u, 0x44444444u);
+                if (r1 >= p.M) b = make_uint2(0x44444444u, 0x44444444u);
+                const uint32_t sel = h ? 0x7632u : 0x5410u;      // {row1 half h : row0 half h}
+                const uint2 w = make_uint2(__byte_perm(a.x, b.x, sel), __byte_perm(a.y, b.y, sel));
+                *reinterpret_cast<uint2*>(smem_gen + s * kStageBytes + kABytes + kBBytes + L * 16) = w;
+                if (i + PD < n_steps) {
+                    q0[d] = __ldg(reinterpret_cast<const uint2*>(row0 + 8 * (i + PD)));
+                    q1[d] = __ldg(reinterpret_cast<const uint2*>(row1 + 8 * (i + PD)));
+                }
+                asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+                __syncwarp();
+                if (lane == 0) mbar_arrive(full_bar(s));
+            }
+        }
+        // ------------------------------------------------------------ epilogue
+        const int q = warp - 4;                                  // lanes 32 q .. 32 q + 31
+        const bool acc_ok = n_steps > 0 ? (ok && mbar_wait(acc_bar, 0, abort_flag)) : ok;
+        tc_fence_after();
+        const int64_t row = m0 + 32 * q + lane;
+        if (acc_ok) {
+#pragma unroll 1
+            for (int c = 0; c < BN; c += 32) {
+                uint32_t v[32];
+                if (n_steps > 0) {
+                    tmem_ld_32x32b_x32(tmem_base + ((uint32_t)(32 * q) << 16) + (uint32_t)c, v);
+                    tmem_ld_wait();
+                } else {
+#pragma unroll
+                    for (int e = 0; e < 32; ++e) v[e] = 0u;
+                }
+                if (row < p.M) {
+                    const int64_t col0 = n0 + c;
+                    if (p.splits > 1) {
+                        float* dst = p.partial + ((int64_t)split * p.M + row) * p.N + col0;
+#pragma unroll
+                        for (int e = 0; e < 32; e += 4)
+                            if (col0 + e < p.N)
+                                *reinterpret_cast<uint4*>(dst + e) = make_uint4(v[e], v[e + 1], v[e + 2], v[e + 3]);
+                    } else {
+#pragma unroll
+                        for (int e = 0; e < 32; e += 8) {
+                            if (col0 + e >= p.N) break;
+                            float f[8];
+#pragma unroll
+                            for (int t = 0; t < 8; ++t) f[t] = __uint_as_float(v[e + t]);
+                            if (p.scale) {
+                                const uint4 sc = *reinterpret_cast<const uint4*>(p.scale + row * p.ldc + col0 + e);
+                                const uint32_t sw[4] = {sc.x, sc.y, sc.z, sc.w};
+#pragma unroll
+                                for (int t = 0; t < 4; ++t) {
+                                    f[2 * t] *= __uint_as_float(sw[t] << 16);
+                                    f[2 * t + 1] *= __uint_as_float(sw[t] & 0xFFFF0000u);
+                                }
+                            }
+                            if (p.c_is_bf16) {
+                                __nv_bfloat16* dst = reinterpret_cast<__nv_bfloat16*>(p.C) + row * p.ldc + col0 + e;
+                                uint32_t o[4];
+#pragma unroll
+                                for (int t = 0; t < 4; ++t) {
+                                    __nv_bfloat162 pr = __floats2bfloat162_rn(f[2 * t], f[2 * t + 1]);
+                                    o[t] = *reinterpret_cast<uint32_t*>(&pr);
+                                }
+                                *reinterpret_cast<uint4*>(dst) = make_uint4(o[0], o[1], o[2], o[3]);
+                            } else {
+                                float* dst = reinterpret_cast<float*>(p.C) + row * p.ldc + col0 + e;
+                                if (p.accumulate) {
+                                    const float4 c0 = *reinterpret_cast<const float4*>(dst);
+                                    const float4 c1 = *reinterpret_cast<const float4*>(dst + 4);
+                                    f[0] += c0.x; f[1] += c0.y; f[2] += c0.z; f[3] += c0.w;
+                                    f[4] += c1.x; f[5] += c1.y; f[6] += c1.z; f[7] += c1.w;
+                                }
+                                *reinterpret_cast<float4*>(dst) = make_float4(f[0], f[1], f[2], f[3]);
+                                *reinterpret_cast<float4*>(dst + 4) = make_float4(f[4], f[5], f[6], f[7]);
+                            }
+                        }
+                    }
+                }
+            }
+        }
+    }
+
+    tc_fence_before();
+    __syncthreads();
+    if (*abort_flag) {
+        // give copies that may still be in flight a bounded chance to land before the block exits
+        if (threadIdx.x == 0) {
+            for (int s = 0; s < kStages; ++s)
+                for (uint32_t spin = 0; spin < 4096 && !mbar_try_wait(full_bar(s), 0) && !mbar_try_wait(full_bar(s), 1); ++spin)
+                    __nanosleep(64);
+            if (p.dev_status) *p.dev_status = MVUE_ERR_DEVICE_TIMEOUT;
+        }
+        __syncthreads();
+    }
+    if (warp == 2) {
+        tc_fence_after();
+        tmem_dealloc(tmem_base, kTmemCols);
+    }
+}
+
+// Second pass of split-K: sums the partial tiles in a fixed order (deterministic) and applies the
+// same epilogue as the single-pass path.
+__global__ void __launch_bounds__(256)
+splitk_reduce_kernel(const float* __restrict__ partial, int splits, int64_t M, int64_t N, void* C, int64_t ldc,
+                     const __nv_bfloat16* __restrict__ scale, int c_is_bf16, int accumulate) {
+    const int64_t n4 = N / 4;
+    const int64_t total = M * n4;
+    for (int64_t i = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; i < total; i += (int64_t)gridDim.x * blockDim.x) {
+        const int64_t r = i / n4, c = (i - r * n4) * 4;
+        float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
+        for (int s = 0; s < splits; ++s) {
+            const float4 v = *reinterpret_cast<const float4*>(partial + ((int64_t)s * M + r) * N + c);
+            acc.x += v.x; acc.y += v.y; acc.z += v.z; acc.w += v.w;
+        }
+        if (scale) {
+            const uint2 sc = *reinterpret_cast<const uint2*>(scale + r * ldc + c);
+            acc.x *= __uint_as_float(sc.x << 16); acc.y *= __uint_as_float(sc.x & 0xFFFF0000u);
+            acc.z *= __uint_as_float(sc.y << 16); acc.w *= __uint_as_float(sc.y & 0xFFFF0000u);
+        }
+        if (c_is_bf16) {
+            __nv_bfloat162 lo = __floats2bfloat162_rn(acc.x, acc.y), hi = __floats2bfloat162_rn(acc.z, acc.w);
+            *reinterpret_cast<uint2*>(reinterpret_cast<__nv_bfloat16*>(C) + r * ldc + c) =
+                make_uint2(*reinterpret_cast<uint32_t*>(&lo), *reinterpret_cast<uint32_t*>(&hi));
+        } else {
+            float* dst = reinterpret_cast<float*>(C) + r * ldc + c;
+            if (accumulate) {
+                const float4 o = *reinterpret_cast<const float4*>(dst);
+                acc.x += o.x; acc.y += o.y; acc.z += o.z; acc.w += o.w;
+            }
+            *reinterpret_cast<float4*>(dst) = acc;
+        }
+    }
+}
+
+// ---- host side ----------------------------------------------------------------
+PFN_cuTensorMapEncodeTiled_v12000 encode_fn() {
+    static PFN_cuTensorMapEncodeTiled_v12000 fn = nullptr;
+    static std::once_flag once;
+    std::call_once(once, [] {
+        void* ptr = nullptr;
+        cudaDriverEntryPointQueryResult qres;
+        if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &ptr, cudaEnableDefault, &qres) == cudaSuccess &&
+            qres == cudaDriverEntryPointSuccess)
+            fn = reinterpret_cast<PFN_cuTensorMapEncodeTiled_v12000>(ptr);
+    });
+    return fn;
+}
+
+bool make_map_2d(CUtensorMap* map, const void* base, uint64_t inner, uint64_t outer, uint64_t pitch_bytes,
+                 uint32_t box_inner, uint32_t box_outer, CUtensorMapSwizzle swizzle) {
+    auto fn = encode_fn();
+    if (!fn) return false;
+    const cuuint64_t dims[2] = {inner, outer};
+    const cuuint64_t strides[1] = {pitch_bytes};
+    const cuuint32_t box[2] = {box_inner, box_outer};
+    const cuuint32_t estr[2] = {1, 1};
+    return fn(map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void*>(base), dims, strides, box, estr,
+              CU_TENSOR_MAP_INTERLEAVE_NONE, swizzle, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+              CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+}
+
+}  // namespace
+
+int gemm_split_count(int64_t M, int64_t N, int64_t K, int sm_count) {
+    const int64_t tiles = ((M + BM - 1) / BM) * ((N + BN - 1) / BN);
+    const int64_t steps = K / BK;
+    if (tiles >= sm_count || steps < 16) return 1;
+    int64_t splits = sm_count / tiles;
+    if (splits > steps / 8) splits = steps / 8;      // at least 8 steps (K = 512) per split
+    if (splits > 64) splits = 64;
+    return (int)(splits < 1 ? 1 : splits);
+}
+
+size_t gemm_workspace_bytes(int64_t M, int64_t N, int64_t K, int sm_count) {
+    const int splits = gemm_split_count(M, N, K, sm_count);
+    return splits > 1 ? (size_t)splits * (size_t)M * (size_t)N * sizeof(float) : 0;
+}
+
+int launch_sparse_gemm(const SparseGemmArgs& a, cudaStream_t stream) {
+    CUtensorMap map_a, map_b;
+    if (!make_map_2d(&map_a, a.values, (uint64_t)(a.K / 2), (uint64_t)a.M, (uint64_t)(a.K / 2) * 2, BK / 2, BM,
+                     CU_TENSOR_MAP_SWIZZLE_64B) ||
+        !make_map_2d(&map_b, a.B, (uint64_t)a.N, (uint64_t)a.K, (uint64_t)a.ldb * 2, 64, BK,
+                     CU_TENSOR_MAP_SWIZZLE_128B)) {
+        set_cuda_error(cudaErrorUnknown, "cuTensorMapEncodeTiled");
+        return MVUE_ERR_CUDA;
+    }
+    static std::once_flag once;
+    static cudaError_t attr_err = cudaSuccess;
+    std::call_once(once, [] {
+        attr_err = cudaFuncSetAttribute(sparse_gemm_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemBytes);
+    });
+    if (attr_err != cudaSuccess) { set_cuda_error(attr_err, "cudaFuncSetAttribute"); return MVUE_ERR_CUDA; }
+
+    const int splits = gemm_split_count(a.M, a.N, a.K, a.sm_count);
+    const int64_t steps = a.K / BK;
+    GemmParams p;
+    p.meta = reinterpret_cast<const uint8_t*>(a.meta);
+    p.M = a.M; p.N = a.N; p.K = a.K;
+    p.k_steps_per_split = (steps + splits - 1) / splits;
+    p.partial = reinterpret_cast<float*>(a.workspace);
+    p.C = a.C; p.ldc = a.ldc;
+    p.scale = reinterpret_cast<const __nv_bfloat16*>(a.scale);
+    p.c_is_bf16 = a.c_is_bf16; p.accumulate = a.accumulate; p.splits = splits;
+    p.dev_status = a.dev_status;
+    dim3 grid((unsigned)((a.N + BN - 1) / BN), (unsigned)((a.M + BM - 1) / BM), (unsigned)splits);
+    sparse_gemm_kernel<<<grid, kThreads, kSmemBytes, stream>>>(map_a, map_b, p);
+    cudaError_t e = cudaGetLastError();
+    if (e == cudaSuccess && splits > 1) {
+        const int64_t total = a.M * (a.N / 4);
+        const int64_t want = (total + 255) / 256;
+        const int blocks = (int)(want < (int64_t)a.sm_count * 8 ? want : (int64_t)a.sm_count * 8);
+        splitk_reduce_kernel<<<blocks, 256, 0, stream>>>(p.partial, splits, a.M, a.N, a.C, a.ldc, p.scale,
+                                                         a.c_is_bf16, a.accumulate);
+        e = cudaGetLastError();
+    }
+    if (e != cudaSuccess) { set_cuda_error(e, "sparse GEMM launch"); return MVUE_ERR_CUDA; }
+    return MVUE_OK;
+}
+
+}  // namespace mvue

@@ -24,6 +24,25 @@ cudaError_t launch_prune(const PruneArgs& a, cudaStream_t stream);
 cudaError_t launch_unpack(const void* values, const void* meta, int64_t mrows, int64_t K, void* dense,
                           int sm_count, cudaStream_t stream);
 
+struct SparseGemmArgs {
+    const void* values;   // packed survivors [M x K/2] bf16
+    const void* meta;     // canonical nibbles [M x K/8]
+    int64_t M, N, K;
+    const void* B;        // dense bf16 [K x N], leading dimension ldb
+    int64_t ldb;
+    void* C;              // [M x N] fp32 or bf16, leading dimension ldc
+    int64_t ldc;
+    int c_is_bf16;
+    int accumulate;
+    const void* scale;    // optional bf16 [M x N] (ld = ldc) multiplied into the result, or nullptr
+    void* workspace;
+    int* dev_status;
+    int sm_count;
+};
+int launch_sparse_gemm(const SparseGemmArgs& a, cudaStream_t stream);     // returns an mvue_status
+int gemm_split_count(int64_t M, int64_t N, int64_t K, int sm_count);
+size_t gemm_workspace_bytes(int64_t M, int64_t N, int64_t K, int sm_count);
+
 // Per-device facts, looked up once.
 struct DeviceInfo {
     int cc_major = 0;

@@ -1,0 +1,157 @@
+"""Parity of the 2:4-sparse tensor-core products with the CPU oracle (fp64 plain-loop product of the
+oracle's own packed operand): relative Frobenius error <= 1e-2 for bf16 inputs with fp32
+accumulation (the kernel is in fact exact to ~1e-6: bf16 products are exact in fp32)."""
+import numpy as np
+import pytest
+import torch
+
+import oracle
+from paper_2203_10991_b200 import binding, workloads
+
+pytestmark = pytest.mark.gpu
+TOL = 1e-2          # the stated bar
+TIGHT = 2e-5        # what fp32 accumulation of exact products actually gives at these K
+
+
+def to_dev(a: np.ndarray) -> torch.Tensor:
+    return torch.from_numpy(a.view(np.int16)).cuda().view(torch.bfloat16)
+
+
+def rel_fro(got, want):
+    return np.linalg.norm(got - want) / max(np.linalg.norm(want), 1e-300)
+
+
+def pack_canonical(A: np.ndarray):
+    """Test-side packer for a hand-made 2:4 matrix (at most two non-zeros per group of four)."""
+    M, K = A.shape
+    vals = np.zeros((M, K // 2), dtype=np.float32)
+    meta = np.zeros((M, K // 8), dtype=np.uint8)
+    for r in range(M):
+        for j in range(K // 4):
+            nz = [i for i in range(4) if A[r, 4 * j + i] != 0]
+            assert len(nz) <= 2
+            idx = sorted(nz + [i for i in range(4) if i not in nz][:2 - len(nz)])
+            vals[r, 2 * j], vals[r, 2 * j + 1] = A[r, 4 * j + idx[0]], A[r, 4 * j + idx[1]]
+            meta[r, j // 2] |= (idx[0] | (idx[1] << 2)) << (4 * (j % 2))
+    return workloads.to_bf16_bits(vals), meta
+
+
+def test_one_hot_probes_fix_every_layout():
+    # a single non-zero in A and in B: any mistake in the operand layouts, the metadata placement or
+    # the output mapping moves or loses the single product
+    M, N, K = 256, 512, 192
+    rng = np.random.Generator(np.random.PCG64(3))
+    for _ in range(24):
+        m, n, k = int(rng.integers(0, M)), int(rng.integers(0, N)), int(rng.integers(0, K))
+        A = np.zeros((M, K), dtype=np.float32)
+        B = np.zeros((K, N), dtype=np.float32)
+        A[m, k] = 2.0
+        B[k, n] = -3.0
+        vals, meta = pack_canonical(A)
+        assert np.array_equal(oracle.unpack(vals, meta), A)
+        out = binding.mvue_sparse_update_gemm(to_dev(vals), torch.from_numpy(meta).cuda(),
+                                              to_dev(workloads.to_bf16_bits(B)))
+        got = out.cpu().numpy()
+        want = np.zeros((M, N), dtype=np.float32)
+        want[m, n] = -6.0
+        assert np.array_equal(got, want), (m, n, k, np.argwhere(got != 0)[:4])
+
+
+@pytest.mark.parametrize("T,n_out,n_in", [(64, 8, 8), (512, 256, 256), (640, 136, 264), (2048, 384, 520),
+                                          (8192, 768, 3072), (16384, 256, 2304)])
+@pytest.mark.parametrize("n,m", [(2, 4), (1, 2)])
+def test_update_gemm_matches_oracle(T, n_out, n_in, n, m):
+    g = workloads.gradient((T, n_out), "student_t", seed=T + n_out, dtype="bf16")
+    h = workloads.normal_bf16((T, n_in), seed=7)
+    vals, meta = binding.mvue_prune(to_dev(g), n, m, 0, seed=11)
+    st = torch.zeros(1, dtype=torch.int32, device="cuda")
+    dW = binding.mvue_sparse_update_gemm(vals, meta, to_dev(h), dev_status=st)
+    torch.cuda.synchronize()
+    assert int(st.item()) == 0
+    v_ref, m_ref = oracle.prune(g, n, m, axis=0, seed=11, threads=oracle.host_threads())
+    A = oracle.unpack(v_ref, m_ref)
+    if T * n_out * n_in <= 2 ** 31:
+        want = oracle.gemm(A, h, threads=oracle.host_threads())
+        err = rel_fro(dW.double().cpu().numpy(), want)
+        assert err <= TOL and err <= TIGHT, err
+    else:
+        # too large for the plain loops: whole rows and columns, plus a seeded sample of entries
+        got = dW.double().cpu().numpy()
+        rng = np.random.Generator(np.random.PCG64(5))
+        rows = [0, n_out - 1] + [int(x) for x in rng.integers(0, n_out, 6)]
+        want_rows = oracle.gemm(A[rows], h, threads=oracle.host_threads())
+        assert rel_fro(got[rows], want_rows) <= TIGHT
+        for _ in range(200):
+            i, j = int(rng.integers(0, n_out)), int(rng.integers(0, n_in))
+            w = oracle.gemm_entry(A[i], h, j)
+            assert abs(got[i, j] - w) <= 1e-4 * (abs(w) + np.abs(A[i]).sum() * 1e-3)
+
+
+@pytest.mark.parametrize("T,n_out,n_in", [(256, 512, 128), (1000 // 8 * 8, 768, 3072), (8192, 3072, 768)])
+@pytest.mark.parametrize("with_act", [False, True])
+@pytest.mark.parametrize("out_dtype", [torch.float32, torch.bfloat16])
+def test_backward_gemm_matches_oracle(T, n_out, n_in, with_act, out_dtype):
+    g = workloads.gradient((T, n_out), "student_t", seed=3, dtype="bf16")
+    W = workloads.normal_bf16((n_out, n_in), seed=4, std=0.02)
+    act = workloads.normal_bf16((T, n_in), seed=5) if with_act else None
+    vals, meta = binding.mvue_prune(to_dev(g), 2, 4, 1, seed=21)
+    dh = binding.mvue_sparse_backward_gemm(vals, meta, to_dev(W), act_grad=None if act is None else to_dev(act),
+                                           out_dtype=out_dtype)
+    v_ref, m_ref = oracle.prune(g, 2, 4, axis=1, seed=21, threads=oracle.host_threads())
+    A = oracle.unpack(v_ref, m_ref)
+    rows = np.arange(T) if T * n_out * n_in <= 2 ** 30 else np.random.Generator(np.random.PCG64(1)).integers(0, T, 64)
+    want = oracle.gemm(A[rows], W, None if act is None else act[rows], threads=oracle.host_threads())
+    err = rel_fro(dh.double().cpu().numpy()[rows], want)
+    assert err <= TOL
+    assert err <= (TIGHT if out_dtype == torch.float32 else 4e-3), err
+
+
+def test_accumulate_and_preallocated_output():
+    T, n_out, n_in = 1024, 256, 512
+    g = workloads.gradient((T, n_out), "relu_lognormal", seed=1, dtype="bf16")
+    h = workloads.normal_bf16((T, n_in), seed=2)
+    vals, meta = binding.mvue_prune(to_dev(g), 2, 4, 0, seed=1)
+    once = binding.mvue_sparse_update_gemm(vals, meta, to_dev(h))
+    acc = torch.full((n_out, n_in), 1.5, dtype=torch.float32, device="cuda")
+    binding.mvue_sparse_update_gemm(vals, meta, to_dev(h), out=acc, accumulate=True)
+    assert torch.allclose(acc, once + 1.5, rtol=1e-6, atol=1e-6)
+    # a strided output view
+    big = torch.zeros((n_out, n_in + 64), dtype=torch.float32, device="cuda")
+    binding.mvue_sparse_update_gemm(vals, meta, to_dev(h), out=big[:, :n_in])
+    assert torch.equal(big[:, :n_in], once) and float(big[:, n_in:].abs().sum()) == 0.0
+
+
+def test_split_k_is_deterministic_and_equal_to_unsplit_sum():
+    # 2 x 1 tiles with K = 32768: the reduction is split; two runs give the same bits
+    T, n_out, n_in = 32768, 256, 256
+    g = workloads.gradient((T, n_out), "student_t", seed=9, dtype="bf16")
+    h = workloads.normal_bf16((T, n_in), seed=8)
+    assert binding.mvue_gemm_workspace_bytes(0, n_out, n_in, T) > 0
+    vals, meta = binding.mvue_prune(to_dev(g), 2, 4, 0, seed=2)
+    a = binding.mvue_sparse_update_gemm(vals, meta, to_dev(h))
+    b = binding.mvue_sparse_update_gemm(vals, meta, to_dev(h))
+    assert torch.equal(a, b)
+    v_ref, m_ref = oracle.prune(g, 2, 4, axis=0, seed=2, threads=oracle.host_threads())
+    want = oracle.gemm(oracle.unpack(v_ref, m_ref), h, threads=oracle.host_threads())
+    assert rel_fro(a.double().cpu().numpy(), want) <= TIGHT
+
+
+def test_gemm_argument_checks():
+    vals = torch.zeros((64, 64), dtype=torch.bfloat16, device="cuda")
+    meta = torch.zeros((64, 16), dtype=torch.uint8, device="cuda")
+    h = torch.zeros((128, 64), dtype=torch.bfloat16, device="cuda")
+    L = binding.lib()
+    args = lambda **kw: None
+    # K = 96 is not a multiple of 64
+    assert L.mvue_sparse_update_gemm(vals.data_ptr(), meta.data_ptr(), 0, 64, 96, h.data_ptr(), 64, 64,
+                                     h.data_ptr(), 0, 64, 0, None, 0, None, None) == -3
+    assert L.mvue_sparse_update_gemm(None, meta.data_ptr(), 0, 64, 128, h.data_ptr(), 64, 64,
+                                     h.data_ptr(), 0, 64, 0, None, 0, None, None) == -1
+    # accumulate into bf16 is refused
+    assert L.mvue_sparse_update_gemm(vals.data_ptr(), meta.data_ptr(), 0, 64, 128, h.data_ptr(), 64, 64,
+                                     h.data_ptr(), 1, 64, 1, None, 0, None, None) == -5
+    # a reduction that needs split-K refuses a missing workspace
+    big_k = 1 << 16
+    if binding.mvue_gemm_workspace_bytes(0, 64, 64, big_k) > 0:
+        assert L.mvue_sparse_update_gemm(vals.data_ptr(), meta.data_ptr(), 0, 64, big_k, h.data_ptr(), 64, 64,
+                                         h.data_ptr(), 0, 64, 0, None, 0, None, None) == -7
