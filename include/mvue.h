@@ -61,8 +61,16 @@ typedef enum { MVUE_F32 = 0, MVUE_BF16 = 1 } mvue_dtype;
  *           idx0 | idx1 << 2 with idx0 < idx1 the survivors' positions in the
  *           group, low nibble = even group.  (The 2-bit-per-survivor encoding
  *           of 2:4 sparse tensor cores.)
- *   This is also what the GEMM entry points consume. */
-typedef enum { MVUE_LAYOUT_CANONICAL = 0 } mvue_layout;
+ * MVUE_LAYOUT_TC: same values; the metadata in the order the sparse tensor cores
+ *   read it, so that the GEMMs move it with one bulk copy per K block and no
+ *   rearrangement: blocks of 128 rows x 128 k (2048 bytes; row-block major, rows
+ *   padded to a multiple of 128), inside a block 128 "lanes" of 16 bytes,
+ *   lane = r%8 + 8*((k/16)%2) + 16*((r%128)/16); the 32-bit word (k%128)/32 of a
+ *   lane holds the 16-bit nibble string of k%32 in [0,16) or [16,32) for row r
+ *   (low half, (r/8)%2 = 0) and row r+8 (high half).  Needs K a multiple of 128.
+ *   This is what the GEMM entry points consume; canonical is the interchange
+ *   and checking form (mvue_unpack reads both). */
+typedef enum { MVUE_LAYOUT_CANONICAL = 0, MVUE_LAYOUT_TC = 1 } mvue_layout;
 
 /* Bytes of the packed outputs of mvue_prune for a [rows x cols] input.
  * values_bytes / meta_bytes are HOST pointers (either may be NULL). */

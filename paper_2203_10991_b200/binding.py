@@ -16,6 +16,7 @@ _lib = None
 
 MVUE_F32, MVUE_BF16 = 0, 1
 MVUE_LAYOUT_CANONICAL = 0
+MVUE_LAYOUT_TC = 1
 
 EXPORTS = ("mvue_version", "mvue_status_string", "mvue_last_cuda_error", "mvue_packed_sizes",
            "mvue_prune", "mvue_unpack", "mvue_sparse_update_gemm", "mvue_sparse_backward_gemm",
@@ -92,9 +93,9 @@ def mvue_prune(g: torch.Tensor, n: int, m: int, axis: int, seed: int, *, k_total
     rows, cols = g.shape
     mrows, k = (rows, cols) if axis == 1 else (cols, rows)
     if values is None or meta is None:
-        mvue_packed_sizes(rows, cols, n, m, axis, layout)          # validates before allocating
+        _, meta_bytes = mvue_packed_sizes(rows, cols, n, m, axis, layout)   # validates before allocating
         values = torch.empty((mrows, k // 2), dtype=torch.bfloat16, device=g.device)
-        meta = torch.empty((mrows, k // 8), dtype=torch.uint8, device=g.device)
+        meta = torch.empty((meta_bytes // (k // 8), k // 8), dtype=torch.uint8, device=g.device)
     _check(lib().mvue_prune(g.data_ptr(), _dtype_code(g), rows, cols, g.stride(0), n, m, axis,
                             seed & (2**64 - 1), k if k_total is None else k_total, k_offset,
                             values.data_ptr(), meta.data_ptr(), layout, _stream_ptr()), "mvue_prune")
@@ -127,8 +128,8 @@ def _workspace(which, M, N, K, device, workspace):
 def mvue_sparse_update_gemm(values: torch.Tensor, meta: torch.Tensor, h: torch.Tensor, *,
                             out: torch.Tensor | None = None, out_dtype=torch.float32, accumulate: bool = False,
                             workspace: torch.Tensor | None = None, dev_status: torch.Tensor | None = None,
-                            layout: int = MVUE_LAYOUT_CANONICAL) -> torch.Tensor:
-    """dW[out, in] (+)= theta(g)^T . h with the packed operand of mvue_prune(g, axis=0)."""
+                            layout: int = MVUE_LAYOUT_TC) -> torch.Tensor:
+    """dW[out, in] (+)= theta(g)^T . h with the packed operand of mvue_prune(g, axis=0, layout=MVUE_LAYOUT_TC)."""
     n_out, half_t = values.shape
     T, n_in = h.shape
     assert h.dtype == torch.bfloat16 and h.stride(1) == 1 and 2 * half_t == T
@@ -147,8 +148,8 @@ def mvue_sparse_backward_gemm(values: torch.Tensor, meta: torch.Tensor, W: torch
                               act_grad: torch.Tensor | None = None, out: torch.Tensor | None = None,
                               out_dtype=torch.bfloat16, workspace: torch.Tensor | None = None,
                               dev_status: torch.Tensor | None = None,
-                              layout: int = MVUE_LAYOUT_CANONICAL) -> torch.Tensor:
-    """dh[T, in] = (theta(g) . W) (* act_grad) with the packed operand of mvue_prune(g, axis=1)."""
+                              layout: int = MVUE_LAYOUT_TC) -> torch.Tensor:
+    """dh[T, in] = (theta(g) . W) (* act_grad) with the packed operand of mvue_prune(g, axis=1, layout=MVUE_LAYOUT_TC)."""
     T, half_o = values.shape
     n_out, n_in = W.shape
     assert W.dtype == torch.bfloat16 and W.stride(1) == 1 and 2 * half_o == n_out

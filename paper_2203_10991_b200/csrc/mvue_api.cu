@@ -49,11 +49,11 @@ static int run_gemm(const void* values, const void* meta, int layout, int64_t M,
                     const void* B, int64_t ldb, const void* scale, void* C, int c_dtype, int64_t ldc,
                     int accumulate, void* workspace, size_t workspace_bytes, int* dev_status, void* stream) {
     if (!values || !meta || !B || !C) return MVUE_ERR_NULL;
-    if (layout != MVUE_LAYOUT_CANONICAL) return MVUE_ERR_LAYOUT;
+    if (layout != MVUE_LAYOUT_TC) return MVUE_ERR_LAYOUT;
     if (c_dtype != MVUE_F32 && c_dtype != MVUE_BF16) return MVUE_ERR_DTYPE;
     if (accumulate && c_dtype != MVUE_F32) return MVUE_ERR_DTYPE;
     if (accumulate && scale) return MVUE_ERR_DTYPE;
-    if (M <= 0 || N <= 0 || K <= 0 || K % 64 != 0 || M % 8 != 0 || N % 8 != 0) return MVUE_ERR_SHAPE;
+    if (M <= 0 || N <= 0 || K <= 0 || K % 128 != 0 || M % 8 != 0 || N % 8 != 0) return MVUE_ERR_SHAPE;
     if (ldb < N || ldc < N) return MVUE_ERR_SHAPE;
     if (M > 0x7FFFFFFF || N > 0x7FFFFFFF || K > 0x7FFFFFFF) return MVUE_ERR_SHAPE;
     const int64_t c_esz = c_dtype == MVUE_BF16 ? 2 : 4;
@@ -99,14 +99,16 @@ const char* mvue_last_cuda_error(void) { return g_cuda_error; }
 int mvue_packed_sizes(int64_t rows, int64_t cols, int n, int m, int axis, int layout,
                       size_t* values_bytes, size_t* meta_bytes) {
     if (int s = check_nm(n, m)) return s;
-    if (layout != MVUE_LAYOUT_CANONICAL) return MVUE_ERR_LAYOUT;
+    if (layout != MVUE_LAYOUT_CANONICAL && layout != MVUE_LAYOUT_TC) return MVUE_ERR_LAYOUT;
     if (axis != 0 && axis != 1) return MVUE_ERR_SHAPE;
     if (rows <= 0 || cols <= 0) return MVUE_ERR_SHAPE;
     const int64_t mrows = axis == 1 ? rows : cols;
     const int64_t K = axis == 1 ? cols : rows;
     if (K % 16 != 0 || mrows % 8 != 0) return MVUE_ERR_SHAPE;
+    if (layout == MVUE_LAYOUT_TC && K % 128 != 0) return MVUE_ERR_SHAPE;
+    const int64_t meta_rows = layout == MVUE_LAYOUT_TC ? (mrows + 127) / 128 * 128 : mrows;
     if (values_bytes) *values_bytes = (size_t)mrows * (size_t)(K / 2) * 2;
-    if (meta_bytes) *meta_bytes = (size_t)mrows * (size_t)(K / 8);
+    if (meta_bytes) *meta_bytes = (size_t)meta_rows * (size_t)(K / 8);
     return MVUE_OK;
 }
 
@@ -123,7 +125,9 @@ int mvue_prune(const void* g, int dtype, int64_t rows, int64_t cols, int64_t ld,
     if (!aligned16(g) || !aligned16(values) || !aligned16(meta) || (ld * esz) % 16 != 0) return MVUE_ERR_ALIGN;
     DeviceInfo dev;
     if (int s = current_device_info(&dev)) return s;
-    PruneArgs a{g, dtype == MVUE_BF16, rows, cols, ld, m, axis, seed, k_total, k_offset, values, meta, dev.sm_count};
+    if (layout == MVUE_LAYOUT_TC && (k_total != K || k_offset != 0)) return MVUE_ERR_LAYOUT;   // shards pack canonically
+    PruneArgs a{g, dtype == MVUE_BF16, rows, cols, ld, m, axis, seed, k_total, k_offset, values, meta, dev.sm_count,
+                layout == MVUE_LAYOUT_TC};
     cudaError_t e = launch_prune(a, reinterpret_cast<cudaStream_t>(stream));
     if (e != cudaSuccess) { set_cuda_error(e, "mvue_prune launch"); return MVUE_ERR_CUDA; }
     return MVUE_OK;
@@ -132,12 +136,13 @@ int mvue_prune(const void* g, int dtype, int64_t rows, int64_t cols, int64_t ld,
 int mvue_unpack(const void* values, const void* meta, int layout, int64_t mrows, int64_t K,
                 void* dense_bf16, void* stream) {
     if (!values || !meta || !dense_bf16) return MVUE_ERR_NULL;
-    if (layout != MVUE_LAYOUT_CANONICAL) return MVUE_ERR_LAYOUT;
+    if (layout != MVUE_LAYOUT_CANONICAL && layout != MVUE_LAYOUT_TC) return MVUE_ERR_LAYOUT;
     if (mrows <= 0 || K <= 0 || K % 16 != 0) return MVUE_ERR_SHAPE;
+    if (layout == MVUE_LAYOUT_TC && K % 128 != 0) return MVUE_ERR_SHAPE;
     if (!aligned16(values) || !aligned16(meta) || !aligned16(dense_bf16)) return MVUE_ERR_ALIGN;
     DeviceInfo dev;
     if (int s = current_device_info(&dev)) return s;
-    cudaError_t e = launch_unpack(values, meta, mrows, K, dense_bf16, dev.sm_count,
+    cudaError_t e = launch_unpack(values, meta, layout == MVUE_LAYOUT_TC, mrows, K, dense_bf16, dev.sm_count,
                                   reinterpret_cast<cudaStream_t>(stream));
     if (e != cudaSuccess) { set_cuda_error(e, "mvue_unpack launch"); return MVUE_ERR_CUDA; }
     return MVUE_OK;
@@ -146,7 +151,7 @@ int mvue_unpack(const void* values, const void* meta, int layout, int64_t mrows,
 int mvue_gemm_workspace_bytes(int which, int64_t M, int64_t N, int64_t K, size_t* bytes) {
     if (!bytes) return MVUE_ERR_NULL;
     if (which != 0 && which != 1) return MVUE_ERR_SHAPE;
-    if (M <= 0 || N <= 0 || K <= 0 || K % 64 != 0) return MVUE_ERR_SHAPE;
+    if (M <= 0 || N <= 0 || K <= 0 || K % 128 != 0) return MVUE_ERR_SHAPE;
     DeviceInfo dev;
     if (int s = current_device_info(&dev)) return s;
     *bytes = gemm_workspace_bytes(M, N, K, dev.sm_count);

@@ -1,23 +1,24 @@
 // 2:4-sparse GEMM on the 5th-generation tensor cores (tcgen05.mma.sp), sm_100a.
 //
 //   C[M x N] = A[M x K] . B[K x N]
-// A is the MVUE-pruned gradient in packed form: bf16 survivors [M x K/2] (K-major)
-// plus one nibble of positions per group of four, [M x K/8] bytes.  B is dense
-// bf16, row-major [K x N] (N contiguous): the activations h for the update
-// product g^T h, the weights W for the backward product g W (Sec. 1 of the paper).
+// A is the MVUE-pruned gradient in packed form: bf16 survivors [M x K/2] (K-major) plus
+// the position nibbles in tensor-core order (MVUE_LAYOUT_TC).  B is dense bf16, row-major
+// [K x N] (N contiguous): the activations h for the update product g^T h, the weights W
+// for the backward product g W (Sec. 1 of the paper).
 //
-// One thread block computes one 128 x 256 output tile over a range of K:
-//   warp 0      TMA producer: per 64-deep K step, the packed A tile (128 x 32 bf16,
-//               64-byte swizzle) and four 64 x 64 boxes of B (128-byte swizzle)
-//   warp 1      MMA issuer: copies the step's metadata from shared to tensor
-//               memory (tcgen05.cp), issues two tcgen05.mma.sp (K = 32 each) with the
-//               fp32 accumulator in tensor memory, commits to the step's "empty"
-//               barrier
+// A cluster of two thread blocks computes one 256 x 256 output tile over a range of K with
+// tcgen05.mma.sp.cta_group::2: block r of the pair loads its own 128 rows of A (and their
+// metadata) and its own 128 columns of B, the leader (r = 0) issues the MMAs for both, and
+// each block keeps the fp32 accumulator of its 128 rows in its own tensor memory.  Per block
+// and 128-deep K step that is 50 KiB of TMA traffic for 16.8 MFLOP, three times less L2
+// traffic per flop than a single-SM 128 x 256 tile.
+//   warp 0      TMA producer: A tile (128 x 64 bf16, 128-byte swizzle), two 64 x 128 boxes
+//               of B (128-byte swizzle), one 2 KiB metadata block; all complete on the
+//               leader's "full" barrier of the stage
+//   warp 1      (leader) per stage: tcgen05.cp of the metadata into tensor memory, four
+//               tcgen05.mma.sp of K = 32, commit to both blocks' "empty" barrier
 //   warp 2      allocates / frees tensor memory
-//   warps 4-7   stage the metadata: read the nibbles of their rows, rearrange them
-//               into the lane/column order the tensor core expects, write them to
-//               shared memory; afterwards they are the epilogue (tcgen05.ld ->
-//               registers -> global), one quarter of the lanes each.
+//   warps 4-7   epilogue: tcgen05.ld -> registers -> global, one quarter of the lanes each
 // Every wait on an mbarrier is bounded; when a bound expires the block records
 // MVUE_ERR_DEVICE_TIMEOUT in the caller's status word and drains.
 #include <cuda.h>
@@ -34,13 +35,13 @@
 namespace mvue {
 namespace {
 
-constexpr int BM = 128;
+constexpr int BM = 128;                    // rows of A per thread block (256 per pair)
 constexpr int BN = 256;
-constexpr int BK = 64;                     // logical K per pipeline step (two MMAs of K = 32)
-constexpr int kStages = 5;
-constexpr int kABytes = BM * (BK / 2) * 2; // 8 KiB: 128 rows x 64 bytes of survivors
-constexpr int kBBoxBytes = 64 * BK * 2;    // 8 KiB: 64 k-rows x 128 bytes
-constexpr int kBBytes = (BN / 64) * kBBoxBytes;
+constexpr int BK = 128;                    // logical K per pipeline stage (four MMAs of K = 32)
+constexpr int kStages = 4;
+constexpr int kABytes = BM * (BK / 2) * 2; // 16 KiB: 128 rows x 128 bytes of survivors
+constexpr int kBBoxBytes = 64 * BK * 2;    // 16 KiB: 128 k-rows x 128 bytes (64 columns)
+constexpr int kBBytes = (BN / 2 / 64) * kBBoxBytes;   // this block's 128 columns
 constexpr int kEBytes = BM * 16;           // 2 KiB: 16 bytes per tensor-memory lane
 constexpr int kStageBytes = kABytes + kBBytes + kEBytes;
 constexpr int kSmemBytes = kStages * kStageBytes + 1024 /*alignment slack*/ + 256 /*barriers*/;
@@ -54,12 +55,6 @@ __device__ __forceinline__ uint32_t smem_u32(const void* p) {
 }
 __device__ __forceinline__ void mbar_init(uint32_t bar, uint32_t count) {
     asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(bar), "r"(count));
-}
-__device__ __forceinline__ void mbar_expect_tx(uint32_t bar, uint32_t bytes) {
-    asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "r"(bytes) : "memory");
-}
-__device__ __forceinline__ void mbar_arrive(uint32_t bar) {
-    asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(bar) : "memory");
 }
 __device__ __forceinline__ bool mbar_try_wait(uint32_t bar, uint32_t parity) {
     uint32_t ok;
@@ -81,37 +76,8 @@ __device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatil
     *abort_flag = 1;
     return false;
 }
-__device__ __forceinline__ void tma_load_2d(uint32_t dst, const CUtensorMap* map, int x, int y, uint32_t bar) {
-    asm volatile(
-        "cp.async.bulk.tensor.2d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3}], [%4];"
-        ::"r"(dst), "l"(map), "r"(x), "r"(y), "r"(bar) : "memory");
-}
-__device__ __forceinline__ void tmem_alloc(uint32_t dst_smem, uint32_t cols) {
-    asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(dst_smem), "r"(cols) : "memory");
-}
-__device__ __forceinline__ void tmem_relinquish() {
-    asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
-}
-__device__ __forceinline__ void tmem_dealloc(uint32_t addr, uint32_t cols) {
-    asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(addr), "r"(cols) : "memory");
-}
 __device__ __forceinline__ void tc_fence_before() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
 __device__ __forceinline__ void tc_fence_after() { asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory"); }
-__device__ __forceinline__ void tc_commit(uint32_t bar) {
-    asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(bar) : "memory");
-}
-__device__ __forceinline__ void tc_copy_128x128b(uint32_t tmem_addr, uint64_t smem_desc) {
-    asm volatile("tcgen05.cp.cta_group::1.128x128b [%0], %1;" ::"r"(tmem_addr), "l"(smem_desc) : "memory");
-}
-__device__ __forceinline__ void tc_mma_sp_bf16(uint32_t tmem_d, uint64_t a_desc, uint64_t b_desc,
-                                               uint32_t tmem_meta, uint32_t idesc, uint32_t accumulate) {
-    const uint32_t zero = 0u;                 // no output lane is disabled
-    asm volatile(
-        "{\n\t.reg .pred p;\n\t"
-        "setp.ne.b32 p, %5, 0;\n\t"
-        "tcgen05.mma.sp.cta_group::1.kind::f16 [%0], %1, %2, [%3], %4, {%6, %6, %6, %6}, p;\n\t}"
-        ::"r"(tmem_d), "l"(a_desc), "l"(b_desc), "r"(tmem_meta), "r"(idesc), "r"(accumulate), "r"(zero) : "memory");
-}
 __device__ __forceinline__ void tmem_ld_32x32b_x32(uint32_t taddr, uint32_t (&v)[32]) {
     asm volatile(
         "tcgen05.ld.sync.aligned.32x32b.x32.b32 "
@@ -132,16 +98,15 @@ __device__ __forceinline__ uint64_t make_smem_desc(uint32_t addr, uint32_t lbo_b
     return (uint64_t)((addr >> 4) & 0x3FFFu) | ((uint64_t)((lbo_bytes >> 4) & 0x3FFFu) << 16) |
            ((uint64_t)((sbo_bytes >> 4) & 0x3FFFu) << 32) | (1ull << 46) | ((uint64_t)swizzle_code << 61);
 }
-constexpr uint32_t kSwizzleNone = 0, kSwizzle128B = 2, kSwizzle64B = 4;
+constexpr uint32_t kSwizzleNone = 0, kSwizzle128B = 2;
 
-// Instruction descriptor of tcgen05.mma.sp.kind::f16: sparse, fp32 accumulate, bf16 x bf16,
-// A K-major, B N-major, N = 256, M = 128.
-constexpr uint32_t kInstrDesc = (1u << 2) /*sparse*/ | (1u << 4) /*D = f32*/ | (1u << 7) /*A = bf16*/ |
-                                (1u << 10) /*B = bf16*/ | (0u << 15) /*A K-major*/ | (1u << 16) /*B N-major*/ |
-                                ((uint32_t)(BN >> 3) << 17) | ((uint32_t)(BM >> 4) << 24);
+// Instruction descriptor of tcgen05.mma.sp.cta_group::2.kind::f16: sparse, fp32 accumulate,
+// bf16 x bf16, A K-major, B N-major, N = 256, M = 256 (128 rows in each block of the pair).
+constexpr uint32_t kInstrDesc2 = (1u << 2) /*sparse*/ | (1u << 4) /*D = f32*/ | (1u << 7) /*A = bf16*/ |
+                                 (1u << 10) /*B = bf16*/ | (0u << 15) /*A K-major*/ | (1u << 16) /*B N-major*/ |
+                                 ((uint32_t)(BN >> 3) << 17) | ((uint32_t)((2 * BM) >> 4) << 24);
 
 struct GemmParams {
-    const uint8_t* meta;      // canonical nibbles [M x K/8]
     int64_t M, N, K;
     int64_t k_steps_per_split;
     float* partial;           // split-K workspace [splits x M x N] (splits > 1) else unused
@@ -154,23 +119,130 @@ struct GemmParams {
     int* dev_status;
 };
 
-__global__ void __launch_bounds__(kThreads, 1)
-sparse_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ CUtensorMap map_b,
-                   const GemmParams p) {
+// Epilogue of one thread: its accumulator row (32 columns at a time from tensor memory) goes to the
+// split-K workspace, or through the optional elementwise scale / accumulate / bf16 conversion to C.
+__device__ __forceinline__ void epilogue_rows(const GemmParams& p, int split, int64_t row, int64_t n0,
+                                              uint32_t tmem_rows, bool have_acc) {
+#pragma unroll 1
+    for (int c = 0; c < BN; c += 32) {
+        uint32_t v[32];
+        if (have_acc) {
+            tmem_ld_32x32b_x32(tmem_rows + (uint32_t)c, v);
+            tmem_ld_wait();
+        } else {
+#pragma unroll
+            for (int e = 0; e < 32; ++e) v[e] = 0u;
+        }
+        if (row < p.M) {
+            const int64_t col0 = n0 + c;
+            if (p.splits > 1) {
+                float* dst = p.partial + ((int64_t)split * p.M + row) * p.N + col0;
+#pragma unroll
+                for (int e = 0; e < 32; e += 4)
+                    if (col0 + e < p.N)
+                        *reinterpret_cast<uint4*>(dst + e) = make_uint4(v[e], v[e + 1], v[e + 2], v[e + 3]);
+            } else {
+#pragma unroll
+                for (int e = 0; e < 32; e += 8) {
+                    if (col0 + e >= p.N) break;
+                    float f[8];
+#pragma unroll
+                    for (int t = 0; t < 8; ++t) f[t] = __uint_as_float(v[e + t]);
+                    if (p.scale) {
+                        const uint4 sc = *reinterpret_cast<const uint4*>(p.scale + row * p.ldc + col0 + e);
+                        const uint32_t sw[4] = {sc.x, sc.y, sc.z, sc.w};
+#pragma unroll
+                        for (int t = 0; t < 4; ++t) {
+                            f[2 * t] *= __uint_as_float(sw[t] << 16);
+                            f[2 * t + 1] *= __uint_as_float(sw[t] & 0xFFFF0000u);
+                        }
+                    }
+                    if (p.c_is_bf16) {
+                        __nv_bfloat16* dst = reinterpret_cast<__nv_bfloat16*>(p.C) + row * p.ldc + col0 + e;
+                        uint32_t o[4];
+#pragma unroll
+                        for (int t = 0; t < 4; ++t) {
+                            __nv_bfloat162 pr = __floats2bfloat162_rn(f[2 * t], f[2 * t + 1]);
+                            o[t] = *reinterpret_cast<uint32_t*>(&pr);
+                        }
+                        *reinterpret_cast<uint4*>(dst) = make_uint4(o[0], o[1], o[2], o[3]);
+                    } else {
+                        float* dst = reinterpret_cast<float*>(p.C) + row * p.ldc + col0 + e;
+                        if (p.accumulate) {
+                            const float4 c0 = *reinterpret_cast<const float4*>(dst);
+                            const float4 c1 = *reinterpret_cast<const float4*>(dst + 4);
+                            f[0] += c0.x; f[1] += c0.y; f[2] += c0.z; f[3] += c0.w;
+                            f[4] += c1.x; f[5] += c1.y; f[6] += c1.z; f[7] += c1.w;
+                        }
+                        *reinterpret_cast<float4*>(dst) = make_float4(f[0], f[1], f[2], f[3]);
+                        *reinterpret_cast<float4*>(dst + 4) = make_float4(f[4], f[5], f[6], f[7]);
+                    }
+                }
+            }
+        }
+    }
+}
+
+__device__ __forceinline__ uint32_t cluster_ctarank() {
+    uint32_t r;
+    asm volatile("mov.u32 %0, %%cluster_ctarank;" : "=r"(r));
+    return r;
+}
+__device__ __forceinline__ uint32_t map_to_cta(uint32_t smem_addr, uint32_t rank) {
+    uint32_t out;
+    asm volatile("mapa.shared::cluster.u32 %0, %1, %2;" : "=r"(out) : "r"(smem_addr), "r"(rank));
+    return out;
+}
+__device__ __forceinline__ void cluster_sync() {
+    asm volatile("barrier.cluster.arrive.release.aligned;\n\tbarrier.cluster.wait.acquire.aligned;" ::: "memory");
+}
+__device__ __forceinline__ void mbar_expect_tx_cluster(uint32_t cluster_bar, uint32_t bytes) {
+    asm volatile("mbarrier.arrive.expect_tx.release.cluster.shared::cluster.b64 _, [%0], %1;"
+                 ::"r"(cluster_bar), "r"(bytes) : "memory");
+}
+// TMA load whose completion bytes are counted on a barrier of the pair's leader.
+__device__ __forceinline__ void tma_load_2d_pair(uint32_t dst, const CUtensorMap* map, int x, int y,
+                                                 uint32_t leader_bar) {
+    asm volatile(
+        "cp.async.bulk.tensor.2d.cta_group::2.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3}], [%4];"
+        ::"r"(dst), "l"(map), "r"(x), "r"(y), "r"(leader_bar) : "memory");
+}
+__device__ __forceinline__ void tc_commit_pair(uint32_t bar) {      // arrives on `bar` in both blocks
+    const uint16_t mask = 3;
+    asm volatile("tcgen05.commit.cta_group::2.mbarrier::arrive::one.shared::cluster.multicast::cluster.b64 [%0], %1;"
+                 ::"r"(bar), "h"(mask) : "memory");
+}
+__device__ __forceinline__ void tc_copy_128x128b_pair(uint32_t tmem_addr, uint64_t smem_desc) {
+    asm volatile("tcgen05.cp.cta_group::2.128x128b [%0], %1;" ::"r"(tmem_addr), "l"(smem_desc) : "memory");
+}
+__device__ __forceinline__ void tc_mma_sp_bf16_pair(uint32_t tmem_d, uint64_t a_desc, uint64_t b_desc,
+                                                    uint32_t tmem_meta, uint32_t idesc, uint32_t accumulate) {
+    const uint32_t zero = 0u;
+    asm volatile(
+        "{\n\t.reg .pred p;\n\t"
+        "setp.ne.b32 p, %5, 0;\n\t"
+        "tcgen05.mma.sp.cta_group::2.kind::f16 [%0], %1, %2, [%3], %4, {%6, %6, %6, %6, %6, %6, %6, %6}, p;\n\t}"
+        ::"r"(tmem_d), "l"(a_desc), "l"(b_desc), "r"(tmem_meta), "r"(idesc), "r"(accumulate), "r"(zero) : "memory");
+}
+
+__global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(kThreads, 1)
+sparse_gemm_pair_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ CUtensorMap map_b,
+                        const __grid_constant__ CUtensorMap map_e, const GemmParams p) {
     extern __shared__ uint8_t smem_raw[];
     const uint32_t smem_base = (smem_u32(smem_raw) + 1023u) & ~1023u;
     uint8_t* smem_gen = smem_raw + (smem_base - smem_u32(smem_raw));
     const uint32_t bar_base = smem_base + kStages * kStageBytes;
-    // barriers: full[kStages], empty[kStages], acc_done; then the tensor-memory base word and the abort flag
-    auto full_bar = [&](int s) { return bar_base + 8u * s; };
+    auto full_bar = [&](int s) { return bar_base + 8u * s; };                 // used in the leader only
     auto empty_bar = [&](int s) { return bar_base + 8u * (kStages + s); };
     const uint32_t acc_bar = bar_base + 8u * (2 * kStages);
     uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(smem_gen + kStages * kStageBytes + 8 * (2 * kStages + 1));
     volatile int* abort_flag = reinterpret_cast<volatile int*>(tmem_slot + 1);
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-    const int64_t m0 = (int64_t)blockIdx.y * BM;
-    const int64_t n0 = (int64_t)blockIdx.x * BN;
+    const uint32_t rank = cluster_ctarank();
+    const int64_t m_block = (int64_t)(blockIdx.x >> 1) * 2 + rank;                  // 128-row block of A
+    const int64_t m0 = m_block * BM;
+    const int64_t n0 = (int64_t)blockIdx.y * BN;                                    // the pair's columns
     const int split = blockIdx.z;
     const int64_t total_steps = p.K / BK;
     const int64_t step_begin = (int64_t)split * p.k_steps_per_split;
@@ -180,48 +252,53 @@ sparse_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_const
 
     if (threadIdx.x == 0) {
         for (int s = 0; s < kStages; ++s) {
-            mbar_init(full_bar(s), 1 + 4);   // TMA thread (with byte count) + one arrival per metadata warp
-            mbar_init(empty_bar(s), 1);      // tcgen05.commit
+            mbar_init(full_bar(s), 2);       // one arrival (with byte count) per block of the pair
+            mbar_init(empty_bar(s), 1);      // the leader's tcgen05.commit
         }
         mbar_init(acc_bar, 1);
         *abort_flag = 0;
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     }
-    // the upper 8 bytes of every metadata lane slot are never used: clear them once
-    for (int i = threadIdx.x; i < kStages * BM; i += kThreads) {
-        const int s = i / BM, l = i % BM;
-        *reinterpret_cast<uint2*>(smem_gen + s * kStageBytes + kABytes + kBBytes + l * 16 + 8) = make_uint2(0u, 0u);
-    }
     if (warp == 2) {
-        tmem_alloc(smem_u32(tmem_slot), kTmemCols);
-        tmem_relinquish();
+        asm volatile("tcgen05.alloc.cta_group::2.sync.aligned.shared::cta.b32 [%0], %1;"
+                     ::"r"(smem_u32(tmem_slot)), "r"(kTmemCols) : "memory");
+        asm volatile("tcgen05.relinquish_alloc_permit.cta_group::2.sync.aligned;" ::: "memory");
     }
-    asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
     tc_fence_before();
     __syncthreads();
+    cluster_sync();                          // the peer's barriers exist before anyone signals them
     tc_fence_after();
     const uint32_t tmem_base = *tmem_slot;
 
     if (warp == 0) {
-        // ------------------------------------------------------------ TMA producer
+        // ------------------------------------------------------------ TMA producer (both blocks)
         if (lane == 0) {
+            const bool rows_exist = m0 < p.M;            // a pair may hang over the last row block
             for (int64_t i = 0; i < n_steps; ++i) {
                 const int s = (int)(i % kStages);
                 const uint32_t use = (uint32_t)(i / kStages);
                 if (use > 0 && !mbar_wait(empty_bar(s), (use - 1) & 1u, abort_flag)) break;
                 const uint32_t a_dst = smem_base + s * kStageBytes;
                 const uint32_t b_dst = a_dst + kABytes;
-                const int k = (int)((step_begin + i) * BK);
-                mbar_expect_tx(full_bar(s), kABytes + kBBytes);
-                tma_load_2d(a_dst, &map_a, k / 2, (int)m0, full_bar(s));
+                const uint32_t e_dst = b_dst + kBBytes;
+                const int64_t step = step_begin + i;
+                const int k = (int)(step * BK);
+                const uint32_t leader_full = map_to_cta(full_bar(s), 0);
+                mbar_expect_tx_cluster(leader_full, kStageBytes);
+                // rows past M read as zeros (out-of-range boxes are zero-filled); the metadata of a row
+                // block that does not exist is taken from block 0 -- any valid pattern is harmless there
+                tma_load_2d_pair(a_dst, &map_a, k / 2, (int)m0, leader_full);
 #pragma unroll
-                for (int j = 0; j < BN / 64; ++j)
-                    tma_load_2d(b_dst + j * kBBoxBytes, &map_b, (int)n0 + 64 * j, k, full_bar(s));
+                for (int j = 0; j < BN / 2 / 64; ++j)
+                    tma_load_2d_pair(b_dst + j * kBBoxBytes, &map_b, (int)n0 + (int)rank * (BN / 2) + 64 * j, k,
+                                     leader_full);
+                const int64_t e_block = (rows_exist ? m_block : 0) * total_steps + step;
+                tma_load_2d_pair(e_dst, &map_e, 0, (int)(e_block * 8), leader_full);
             }
         }
     } else if (warp == 1) {
-        // ------------------------------------------------------------ MMA issuer
-        if (lane == 0) {
+        // ------------------------------------------------------------ MMA issuer (leader only)
+        if (rank == 0 && lane == 0) {
             bool ok = true;
             for (int64_t i = 0; i < n_steps && ok; ++i) {
                 const int s = (int)(i % kStages);
@@ -234,146 +311,44 @@ sparse_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_const
                 const uint32_t e_addr = b_addr + kBBytes;
                 const uint32_t tmem_e = tmem_base + kTmemECol + 4u * s;
                 // metadata: 128 lanes x 16 bytes, rows contiguous (8-row core matrices 128 bytes apart)
-                tc_copy_128x128b(tmem_e, make_smem_desc(e_addr, 16, 128, kSwizzleNone));
+                tc_copy_128x128b_pair(tmem_e, make_smem_desc(e_addr, 16, 128, kSwizzleNone));
 #pragma unroll
                 for (int kb = 0; kb < BK / 32; ++kb) {
-                    // A: K-major, 64-byte swizzle, 8-row groups 512 bytes apart; 32 bytes per K = 32 block
-                    const uint64_t a_desc = make_smem_desc(a_addr + kb * 32, 16, 512, kSwizzle64B);
-                    // B: N-major, 128-byte swizzle; 64-column blocks kBBoxBytes apart (leading),
-                    //    8-row groups 1024 bytes apart (stride); 32 k-rows per block = 4096 bytes
+                    // A: K-major, 128-byte swizzle, 8-row groups 1024 bytes apart; 32 bytes per K = 32 block
+                    const uint64_t a_desc = make_smem_desc(a_addr + kb * 32, 16, 1024, kSwizzle128B);
+                    // B: N-major, 128-byte swizzle; 64-column blocks kBBoxBytes apart (leading), 8-row
+                    //    groups 1024 bytes apart (stride); 32 k-rows per K = 32 block = 4096 bytes
                     const uint64_t b_desc = make_smem_desc(b_addr + kb * 4096, kBBoxBytes, 1024, kSwizzle128B);
-                    tc_mma_sp_bf16(tmem_base, a_desc, b_desc, tmem_e, kInstrDesc | (uint32_t)kb,
-                                   (i > 0 || kb > 0) ? 1u : 0u);
+                    // metadata of K block kb: column pair (kb & ~1) of the stage's four, selector kb & 1
+                    tc_mma_sp_bf16_pair(tmem_base, a_desc, b_desc, tmem_e + (uint32_t)(kb & ~1),
+                                        kInstrDesc2 | (uint32_t)(kb & 1), (i > 0 || kb > 0) ? 1u : 0u);
                 }
-                tc_commit(empty_bar(s));     // frees the stage (and its metadata columns) when the MMAs retire
+                tc_commit_pair(empty_bar(s));    // frees the stage in both blocks when the MMAs retire
             }
-            tc_commit(acc_bar);              // accumulator complete
+            tc_commit_pair(acc_bar);             // accumulators complete
         }
     } else if (warp >= 4) {
-        // ------------------------------------------------------------ metadata staging
-        const int L = threadIdx.x - 128;                 // tensor-memory lane 0..127
-        const int j = L & 7, h = (L >> 3) & 1, G = L >> 4;
-        const int64_t r0 = m0 + 16 * G + j, r1 = r0 + 8; // the two rows that share this lane
-        const int64_t pitch = p.K / 8;
-        const uint8_t* row0 = p.meta + (r0 < p.M ? r0 : 0) * pitch + (step_begin * BK) / 8;
-        const uint8_t* row1 = p.meta + (r1 < p.M ? r1 : 0) * pitch + (step_begin * BK) / 8;
-        constexpr int PD = 4;                            // prefetch distance in steps
-        uint2 q0[PD], q1[PD];
-#pragma unroll
-        for (int d = 0; d < PD; ++d) {
-            if (d < n_steps) {
-                q0[d] = __ldg(reinterpret_cast<const uint2*>(row0 + 8 * d));
-                q1[d] = __ldg(reinterpret_cast<const uint2*>(row1 + 8 * d));
-            }
-        }
-        bool ok = true;
-        for (int64_t i0 = 0; i0 < n_steps && ok; i0 += PD) {
-#pragma unroll
-            for (int d = 0; d < PD; ++d) {
-                const int64_t i = i0 + d;
-                if (i >= n_steps || !ok) break;
-                const int s = (int)(i % kStages);
-                const uint32_t use = (uint32_t)(i / kStages);
-                if (use > 0) ok = mbar_wait(empty_bar(s), (use - 1) & 1u, abort_flag);
-                if (!ok) break;
-                // 16 bits = four nibbles = 16 logical k; x: k 0..31 of the step, y: k 32..63
-                uint2 a = q0[d], b = q1[d];
-                if (r0 >= p.M) a = make_uint2(0x44444444u, 0x44444444u);
-                if (r1 >= p.M) b = make_uint2(0x44444444u, 0x44444444u);
-                const uint32_t sel = h ? 0x7632u : 0x5410u;      // {row1 half h : row0 half h}
-                const uint2 w = make_uint2(__byte_perm(a.x, b.x, sel), __byte_perm(a.y, b.y, sel));
-                *reinterpret_cast<uint2*>(smem_gen + s * kStageBytes + kABytes + kBBytes + L * 16) = w;
-                if (i + PD < n_steps) {
-                    q0[d] = __ldg(reinterpret_cast<const uint2*>(row0 + 8 * (i + PD)));
-                    q1[d] = __ldg(reinterpret_cast<const uint2*>(row1 + 8 * (i + PD)));
-                }
-                asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
-                __syncwarp();
-                if (lane == 0) mbar_arrive(full_bar(s));
-            }
-        }
-        // ------------------------------------------------------------ epilogue
+        // ------------------------------------------------------------ epilogue (both blocks, own rows)
         const int q = warp - 4;                                  // lanes 32 q .. 32 q + 31
-        const bool acc_ok = n_steps > 0 ? (ok && mbar_wait(acc_bar, 0, abort_flag)) : ok;
+        const bool acc_ok = n_steps > 0 ? mbar_wait(acc_bar, 0, abort_flag) : true;
         tc_fence_after();
         const int64_t row = m0 + 32 * q + lane;
-        if (acc_ok) {
-#pragma unroll 1
-            for (int c = 0; c < BN; c += 32) {
-                uint32_t v[32];
-                if (n_steps > 0) {
-                    tmem_ld_32x32b_x32(tmem_base + ((uint32_t)(32 * q) << 16) + (uint32_t)c, v);
-                    tmem_ld_wait();
-                } else {
-#pragma unroll
-                    for (int e = 0; e < 32; ++e) v[e] = 0u;
-                }
-                if (row < p.M) {
-                    const int64_t col0 = n0 + c;
-                    if (p.splits > 1) {
-                        float* dst = p.partial + ((int64_t)split * p.M + row) * p.N + col0;
-#pragma unroll
-                        for (int e = 0; e < 32; e += 4)
-                            if (col0 + e < p.N)
-                                *reinterpret_cast<uint4*>(dst + e) = make_uint4(v[e], v[e + 1], v[e + 2], v[e + 3]);
-                    } else {
-#pragma unroll
-                        for (int e = 0; e < 32; e += 8) {
-                            if (col0 + e >= p.N) break;
-                            float f[8];
-#pragma unroll
-                            for (int t = 0; t < 8; ++t) f[t] = __uint_as_float(v[e + t]);
-                            if (p.scale) {
-                                const uint4 sc = *reinterpret_cast<const uint4*>(p.scale + row * p.ldc + col0 + e);
-                                const uint32_t sw[4] = {sc.x, sc.y, sc.z, sc.w};
-#pragma unroll
-                                for (int t = 0; t < 4; ++t) {
-                                    f[2 * t] *= __uint_as_float(sw[t] << 16);
-                                    f[2 * t + 1] *= __uint_as_float(sw[t] & 0xFFFF0000u);
-                                }
-                            }
-                            if (p.c_is_bf16) {
-                                __nv_bfloat16* dst = reinterpret_cast<__nv_bfloat16*>(p.C) + row * p.ldc + col0 + e;
-                                uint32_t o[4];
-#pragma unroll
-                                for (int t = 0; t < 4; ++t) {
-                                    __nv_bfloat162 pr = __floats2bfloat162_rn(f[2 * t], f[2 * t + 1]);
-                                    o[t] = *reinterpret_cast<uint32_t*>(&pr);
-                                }
-                                *reinterpret_cast<uint4*>(dst) = make_uint4(o[0], o[1], o[2], o[3]);
-                            } else {
-                                float* dst = reinterpret_cast<float*>(p.C) + row * p.ldc + col0 + e;
-                                if (p.accumulate) {
-                                    const float4 c0 = *reinterpret_cast<const float4*>(dst);
-                                    const float4 c1 = *reinterpret_cast<const float4*>(dst + 4);
-                                    f[0] += c0.x; f[1] += c0.y; f[2] += c0.z; f[3] += c0.w;
-                                    f[4] += c1.x; f[5] += c1.y; f[6] += c1.z; f[7] += c1.w;
-                                }
-                                *reinterpret_cast<float4*>(dst) = make_float4(f[0], f[1], f[2], f[3]);
-                                *reinterpret_cast<float4*>(dst + 4) = make_float4(f[4], f[5], f[6], f[7]);
-                            }
-                        }
-                    }
-                }
-            }
-        }
+        if (acc_ok) epilogue_rows(p, split, row, n0, tmem_base + ((uint32_t)(32 * q) << 16), n_steps > 0);
     }
 
     tc_fence_before();
     __syncthreads();
-    if (*abort_flag) {
-        // give copies that may still be in flight a bounded chance to land before the block exits
-        if (threadIdx.x == 0) {
-            for (int s = 0; s < kStages; ++s)
-                for (uint32_t spin = 0; spin < 4096 && !mbar_try_wait(full_bar(s), 0) && !mbar_try_wait(full_bar(s), 1); ++spin)
-                    __nanosleep(64);
-            if (p.dev_status) *p.dev_status = MVUE_ERR_DEVICE_TIMEOUT;
-        }
-        __syncthreads();
+    if (*abort_flag && threadIdx.x == 0) {
+        // give copies that may still be in flight a bounded chance to land before the pair exits
+        for (int s = 0; s < kStages; ++s)
+            for (uint32_t spin = 0; spin < 4096 && !mbar_try_wait(full_bar(s), 0) && !mbar_try_wait(full_bar(s), 1); ++spin)
+                __nanosleep(64);
+        if (p.dev_status) *p.dev_status = MVUE_ERR_DEVICE_TIMEOUT;
     }
+    cluster_sync();                          // neither block leaves while the other may still touch it
     if (warp == 2) {
         tc_fence_after();
-        tmem_dealloc(tmem_base, kTmemCols);
+        asm volatile("tcgen05.dealloc.cta_group::2.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"(kTmemCols) : "memory");
     }
 }
 
@@ -425,27 +400,27 @@ PFN_cuTensorMapEncodeTiled_v12000 encode_fn() {
     return fn;
 }
 
-bool make_map_2d(CUtensorMap* map, const void* base, uint64_t inner, uint64_t outer, uint64_t pitch_bytes,
-                 uint32_t box_inner, uint32_t box_outer, CUtensorMapSwizzle swizzle) {
+bool make_map_2d(CUtensorMap* map, CUtensorMapDataType dtype, const void* base, uint64_t inner, uint64_t outer,
+                 uint64_t pitch_bytes, uint32_t box_inner, uint32_t box_outer, CUtensorMapSwizzle swizzle) {
     auto fn = encode_fn();
     if (!fn) return false;
     const cuuint64_t dims[2] = {inner, outer};
     const cuuint64_t strides[1] = {pitch_bytes};
     const cuuint32_t box[2] = {box_inner, box_outer};
     const cuuint32_t estr[2] = {1, 1};
-    return fn(map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void*>(base), dims, strides, box, estr,
-              CU_TENSOR_MAP_INTERLEAVE_NONE, swizzle, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
-              CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+    return fn(map, dtype, 2, const_cast<void*>(base), dims, strides, box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE,
+              swizzle, CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
 }
 
 }  // namespace
 
 int gemm_split_count(int64_t M, int64_t N, int64_t K, int sm_count) {
-    const int64_t tiles = ((M + BM - 1) / BM) * ((N + BN - 1) / BN);
+    // thread blocks one split launches: two per 256 x 256 tile
+    const int64_t blocks = 2 * ((M + 2 * BM - 1) / (2 * BM)) * ((N + BN - 1) / BN);
     const int64_t steps = K / BK;
-    if (tiles >= sm_count || steps < 16) return 1;
-    int64_t splits = sm_count / tiles;
-    if (splits > steps / 8) splits = steps / 8;      // at least 8 steps (K = 512) per split
+    if (blocks >= sm_count || steps < 8) return 1;
+    int64_t splits = sm_count / blocks;
+    if (splits > steps / 4) splits = steps / 4;      // at least 4 stages (K = 512) per split
     if (splits > 64) splits = 64;
     return (int)(splits < 1 ? 1 : splits);
 }
@@ -456,25 +431,29 @@ size_t gemm_workspace_bytes(int64_t M, int64_t N, int64_t K, int sm_count) {
 }
 
 int launch_sparse_gemm(const SparseGemmArgs& a, cudaStream_t stream) {
-    CUtensorMap map_a, map_b;
-    if (!make_map_2d(&map_a, a.values, (uint64_t)(a.K / 2), (uint64_t)a.M, (uint64_t)(a.K / 2) * 2, BK / 2, BM,
-                     CU_TENSOR_MAP_SWIZZLE_64B) ||
-        !make_map_2d(&map_b, a.B, (uint64_t)a.N, (uint64_t)a.K, (uint64_t)a.ldb * 2, 64, BK,
-                     CU_TENSOR_MAP_SWIZZLE_128B)) {
+    CUtensorMap map_a, map_b, map_e;
+    const uint64_t e_blocks = (uint64_t)((a.M + BM - 1) / BM) * (uint64_t)(a.K / BK);
+    if (!make_map_2d(&map_a, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, a.values, (uint64_t)(a.K / 2), (uint64_t)a.M,
+                     (uint64_t)(a.K / 2) * 2, BK / 2, BM, CU_TENSOR_MAP_SWIZZLE_128B) ||
+        !make_map_2d(&map_b, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, a.B, (uint64_t)a.N, (uint64_t)a.K,
+                     (uint64_t)a.ldb * 2, 64, BK, CU_TENSOR_MAP_SWIZZLE_128B) ||
+        // metadata blocks of 2 KiB seen as 8 rows of 256 bytes
+        !make_map_2d(&map_e, CU_TENSOR_MAP_DATA_TYPE_UINT8, a.meta, 256, e_blocks * 8, 256, 256, 8,
+                     CU_TENSOR_MAP_SWIZZLE_NONE)) {
         set_cuda_error(cudaErrorUnknown, "cuTensorMapEncodeTiled");
         return MVUE_ERR_CUDA;
     }
     static std::once_flag once;
     static cudaError_t attr_err = cudaSuccess;
     std::call_once(once, [] {
-        attr_err = cudaFuncSetAttribute(sparse_gemm_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemBytes);
+        attr_err = cudaFuncSetAttribute(sparse_gemm_pair_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                        kSmemBytes);
     });
     if (attr_err != cudaSuccess) { set_cuda_error(attr_err, "cudaFuncSetAttribute"); return MVUE_ERR_CUDA; }
 
     const int splits = gemm_split_count(a.M, a.N, a.K, a.sm_count);
     const int64_t steps = a.K / BK;
     GemmParams p;
-    p.meta = reinterpret_cast<const uint8_t*>(a.meta);
     p.M = a.M; p.N = a.N; p.K = a.K;
     p.k_steps_per_split = (steps + splits - 1) / splits;
     p.partial = reinterpret_cast<float*>(a.workspace);
@@ -482,8 +461,8 @@ int launch_sparse_gemm(const SparseGemmArgs& a, cudaStream_t stream) {
     p.scale = reinterpret_cast<const __nv_bfloat16*>(a.scale);
     p.c_is_bf16 = a.c_is_bf16; p.accumulate = a.accumulate; p.splits = splits;
     p.dev_status = a.dev_status;
-    dim3 grid((unsigned)((a.N + BN - 1) / BN), (unsigned)((a.M + BM - 1) / BM), (unsigned)splits);
-    sparse_gemm_kernel<<<grid, kThreads, kSmemBytes, stream>>>(map_a, map_b, p);
+    dim3 grid((unsigned)(2 * ((a.M + 2 * BM - 1) / (2 * BM))), (unsigned)((a.N + BN - 1) / BN), (unsigned)splits);
+    sparse_gemm_pair_kernel<<<grid, kThreads, kSmemBytes, stream>>>(map_a, map_b, map_e, p);
     cudaError_t e = cudaGetLastError();
     if (e == cudaSuccess && splits > 1) {
         const int64_t total = a.M * (a.N / 4);

@@ -18,15 +18,16 @@ struct PruneArgs {
     void* values;
     void* meta;
     int sm_count;
+    bool tc_layout;      // metadata in tensor-core order instead of canonical rows
 };
 
 cudaError_t launch_prune(const PruneArgs& a, cudaStream_t stream);
-cudaError_t launch_unpack(const void* values, const void* meta, int64_t mrows, int64_t K, void* dense,
-                          int sm_count, cudaStream_t stream);
+cudaError_t launch_unpack(const void* values, const void* meta, bool tc_layout, int64_t mrows, int64_t K,
+                          void* dense, int sm_count, cudaStream_t stream);
 
 struct SparseGemmArgs {
     const void* values;   // packed survivors [M x K/2] bf16
-    const void* meta;     // canonical nibbles [M x K/8]
+    const void* meta;     // position nibbles in tensor-core order (MVUE_LAYOUT_TC)
     int64_t M, N, K;
     const void* B;        // dense bf16 [K x N], leading dimension ldb
     int64_t ldb;

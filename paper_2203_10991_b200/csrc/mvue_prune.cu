@@ -15,6 +15,16 @@
 namespace mvue {
 namespace {
 
+// Byte offset of the 16-bit metadata word of (row r of A, strip = k / 16) in the tensor-core order:
+// blocks of 128 rows x 128 k (2 KiB, row-block major), inside a block 128 lanes of 16 bytes with
+// lane = r % 8 + 8 * (strip % 2) + 16 * (r % 128 / 16), word = strip % 8 / 2, half-word = r / 8 % 2.
+// This is the arrangement tcgen05.cp.128x128b moves verbatim into tensor memory for four MMAs.
+__device__ __forceinline__ int64_t tc_meta_offset(int64_t r, int64_t strip, int64_t kblocks) {
+    const int rl = (int)(r & 127), st = (int)(strip & 7);
+    const int lane = (rl & 7) + 8 * (st & 1) + 16 * (rl >> 4);
+    return ((r >> 7) * kblocks + (strip >> 3)) * 2048 + lane * 16 + (st >> 1) * 4 + ((rl >> 3) & 1) * 2;
+}
+
 __device__ __forceinline__ uint4 ldg128(const void* p) {
     return __ldg(reinterpret_cast<const uint4*>(p));
 }
@@ -86,10 +96,10 @@ __device__ __forceinline__ void prune_unit_f32(const uint32_t (&b)[16], uint64_t
 // ---- axis 1 ---------------------------------------------------------------
 // slot = r * units_per_row + c.  kLinear: the tensor is contiguous and unsharded,
 // so the input offset and the generator call number are linear in the slot.
-template <int M, bool kBf16, bool kLinear>
+template <int M, bool kBf16, bool kLinear, bool kTC>
 __global__ void __launch_bounds__(256, kBf16 ? 6 : 4)
 prune_axis1_kernel(const void* __restrict__ g, int64_t n_slots, int64_t units_per_row, int64_t ld,
-                   int64_t units_per_row_total, int64_t unit_offset, RoundKeys rk,
+                   int64_t units_per_row_total, int64_t unit_offset, int64_t pad_rows, RoundKeys rk,
                    uint4* __restrict__ values, uint16_t* __restrict__ meta) {
     constexpr int U = 1;                              // units per thread per trip, loads issued first
     constexpr int LW = kBf16 ? 2 : 4;                 // 16-byte loads per unit
@@ -97,19 +107,25 @@ prune_axis1_kernel(const void* __restrict__ g, int64_t n_slots, int64_t units_pe
     for (int64_t base = (int64_t)blockIdx.x * trip; base < n_slots; base += (int64_t)gridDim.x * trip) {
         uint4 in[U][LW];
         uint64_t unit[U];
+        int64_t meta_off[U];
 #pragma unroll
         for (int u = 0; u < U; ++u) {
             const int64_t slot = base + (int64_t)u * blockDim.x + threadIdx.x;
             if (slot < n_slots) {
                 int64_t elem_off;
-                if (kLinear) {
+                if (kLinear && !kTC) {
                     elem_off = slot * 16;
                     unit[u] = (uint64_t)slot;
                 } else {
-                    const int64_t r = slot / units_per_row;
+                    int64_t r;
+                    if (n_slots < (1ll << 32))
+                        r = (int64_t)((uint32_t)slot / (uint32_t)units_per_row);
+                    else
+                        r = slot / units_per_row;
                     const int64_t c = slot - r * units_per_row;
                     elem_off = r * ld + c * 16;
                     unit[u] = (uint64_t)r * (uint64_t)units_per_row_total + (uint64_t)(unit_offset + c);
+                    if (kTC) meta_off[u] = tc_meta_offset(r, c, units_per_row >> 3);
                 }
                 const char* p = reinterpret_cast<const char*>(g) + elem_off * (kBf16 ? 2 : 4);
 #pragma unroll
@@ -136,8 +152,21 @@ prune_axis1_kernel(const void* __restrict__ g, int64_t n_slots, int64_t units_pe
                     prune_unit_f32<M>(b, unit[u], rk, &v, &mt);
                 }
                 values[slot] = v;
-                meta[slot] = (uint16_t)mt;
+                if (kTC)
+                    *reinterpret_cast<uint16_t*>(reinterpret_cast<char*>(meta) + meta_off[u]) = (uint16_t)mt;
+                else
+                    meta[slot] = (uint16_t)mt;
             }
+        }
+    }
+    if (kTC) {
+        // rows that pad the operand to a multiple of 128: a valid pattern (positions 0, 1), never used
+        const int64_t rows = n_slots / units_per_row;
+        const int64_t n_pad = pad_rows * units_per_row;
+        for (int64_t i = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; i < n_pad;
+             i += (int64_t)gridDim.x * blockDim.x) {
+            const int64_t r = rows + i / units_per_row, c = i % units_per_row;
+            *reinterpret_cast<uint16_t*>(reinterpret_cast<char*>(meta) + tc_meta_offset(r, c, units_per_row >> 3)) = 0x4444;
         }
     }
 }
@@ -154,7 +183,7 @@ constexpr int kTileStrips = 16;
 constexpr int kTileCols = 64;
 constexpr int kMetaPitch = 36;                       // bytes per staged metadata row
 
-template <int M, bool kBf16>
+template <int M, bool kBf16, bool kTC>
 __global__ void __launch_bounds__(kTileStrips * 32, kBf16 ? 3 : 2)
 prune_axis0_kernel(const void* __restrict__ g, int64_t n_strips, int64_t n_cols, int64_t ld,
                    int64_t units_per_row_total, int64_t unit_offset, RoundKeys rk,
@@ -162,7 +191,7 @@ prune_axis0_kernel(const void* __restrict__ g, int64_t n_strips, int64_t n_cols,
     constexpr int ES = kBf16 ? 2 : 4;
     constexpr int NT = kTileStrips * 32;
     __shared__ uint4 s_val[kTileCols * kTileStrips];
-    __shared__ __align__(16) unsigned char s_meta[kTileCols * kMetaPitch];
+    __shared__ __align__(16) unsigned char s_meta[kTileCols * kMetaPitch];   // >= 2048 bytes
 
     const int tid = threadIdx.x;
     const int lane = tid & 31;
@@ -171,6 +200,10 @@ prune_axis0_kernel(const void* __restrict__ g, int64_t n_strips, int64_t n_cols,
     const int64_t col0 = (int64_t)blockIdx.y * kTileCols;
     const int64_t strip = strip0 + strip_l;
     const int64_t col = col0 + 2 * lane;             // this lane's first column (n_cols is even)
+    if (kTC) {                                       // padding rows of A keep a valid pattern
+        for (int i = tid; i < 2048 / 4; i += NT) reinterpret_cast<uint32_t*>(s_meta)[i] = 0x44444444u;
+        __syncthreads();
+    }
 
     if (strip < n_strips && col < n_cols) {
         const char* p = reinterpret_cast<const char*>(g) + ((strip * 16) * ld + col) * ES;
@@ -205,7 +238,14 @@ prune_axis0_kernel(const void* __restrict__ g, int64_t n_strips, int64_t n_cols,
                 prune_unit_f32<M>(b, unit, rk, &v, &mt);
             }
             s_val[col_l * kTileStrips + (strip_l ^ (lane & 15))] = v;
-            *reinterpret_cast<uint16_t*>(&s_meta[col_l * kMetaPitch + strip_l * 2]) = (uint16_t)mt;
+            if (kTC) {
+                // staged as [k-block 0/1][lane of this 64-row quarter x2][16 bytes], ready to leave as 1 KiB runs
+                const int tc_lane = (col_l & 7) + 8 * (strip_l & 1) + 16 * (col_l >> 4);
+                const int off = (strip_l >> 3) * 1024 + tc_lane * 16 + ((strip_l & 7) >> 1) * 4 + ((col_l >> 3) & 1) * 2;
+                *reinterpret_cast<uint16_t*>(&s_meta[off]) = (uint16_t)mt;
+            } else {
+                *reinterpret_cast<uint16_t*>(&s_meta[col_l * kMetaPitch + strip_l * 2]) = (uint16_t)mt;
+            }
         }
     }
     __syncthreads();
@@ -220,8 +260,18 @@ prune_axis0_kernel(const void* __restrict__ g, int64_t n_strips, int64_t n_cols,
         if (j < strips_here && c < n_cols)
             values[c * n_strips + strip0 + j] = s_val[col_l * kTileStrips + (j ^ ((col_l >> 1) & 15))];
     }
-    // metadata: 64 columns x 32 bytes; 8 consecutive threads write one column's run as words
-    {
+    if (kTC) {
+        // metadata: per 128-k block one contiguous 1 KiB run (64 rows x 16 bytes of lanes)
+        if (tid < 128) {
+            const int kb = tid >> 6;
+            if (8 * kb < strips_here) {
+                const int64_t block = (col0 >> 7) * (n_strips >> 3) + (strip0 >> 3) + kb;
+                char* dst = reinterpret_cast<char*>(meta) + block * 2048 + ((col0 & 64) ? 1024 : 0) + (tid & 63) * 16;
+                *reinterpret_cast<uint4*>(dst) = *reinterpret_cast<const uint4*>(&s_meta[kb * 1024 + (tid & 63) * 16]);
+            }
+        }
+    } else {
+        // metadata: 64 columns x 32 bytes; 8 consecutive threads write one column's run as words
         const int col_l = tid >> 3, wd = tid & 7;
         const int64_t c = col0 + col_l;
         if (c < n_cols) {
@@ -239,25 +289,41 @@ prune_axis0_kernel(const void* __restrict__ g, int64_t n_strips, int64_t n_cols,
 }
 
 // ---- unpack ---------------------------------------------------------------
-// One thread expands one metadata byte (two groups = 8 dense elements = 16 bytes).
+// One thread expands one unit: a 16-bit metadata word (four groups) and its 8 survivors
+// become 16 dense elements (32 bytes).
+template <bool kTC>
 __global__ void __launch_bounds__(256)
-unpack_kernel(const uint32_t* __restrict__ values, const uint8_t* __restrict__ meta, int64_t n_bytes,
-              uint4* __restrict__ dense) {
+unpack_kernel(const uint4* __restrict__ values, const uint16_t* __restrict__ meta, int64_t n_units,
+              int64_t units_per_row, uint4* __restrict__ dense) {
     const int64_t stride = (int64_t)gridDim.x * blockDim.x;
-    for (int64_t i = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; i < n_bytes; i += stride) {
-        const uint32_t mb = meta[i];
-        const uint32_t va = values[2 * i], vb = values[2 * i + 1];
-        uint16_t out[8] = {0, 0, 0, 0, 0, 0, 0, 0};
-        out[mb & 3u] = (uint16_t)va;
-        out[(mb >> 2) & 3u] = (uint16_t)(va >> 16);
-        out[4 + ((mb >> 4) & 3u)] = (uint16_t)vb;
-        out[4 + ((mb >> 6) & 3u)] = (uint16_t)(vb >> 16);
-        dense[i] = make_uint4(out[0] | ((uint32_t)out[1] << 16), out[2] | ((uint32_t)out[3] << 16),
-                              out[4] | ((uint32_t)out[5] << 16), out[6] | ((uint32_t)out[7] << 16));
+    for (int64_t i = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; i < n_units; i += stride) {
+        uint32_t mw;
+        if (kTC) {
+            const int64_t r = i / units_per_row, c = i - r * units_per_row;
+            mw = *reinterpret_cast<const uint16_t*>(reinterpret_cast<const char*>(meta) +
+                                                    tc_meta_offset(r, c, units_per_row >> 3));
+        } else {
+            mw = meta[i];
+        }
+        const uint4 v = values[i];
+        const uint32_t vw[4] = {v.x, v.y, v.z, v.w};
+        uint32_t out[8];
+#pragma unroll
+        for (int j = 0; j < 4; ++j) {
+            const uint32_t i0 = (mw >> (4 * j)) & 3u, i1 = (mw >> (4 * j + 2)) & 3u;
+            const uint32_t lo = vw[j] & 0xFFFFu, hi = vw[j] >> 16;
+            uint32_t e[4] = {0u, 0u, 0u, 0u};
+#pragma unroll
+            for (int t = 0; t < 4; ++t) e[t] = (i1 == (uint32_t)t) ? hi : ((i0 == (uint32_t)t) ? lo : 0u);
+            out[2 * j] = e[0] | (e[1] << 16);
+            out[2 * j + 1] = e[2] | (e[3] << 16);
+        }
+        dense[2 * i] = make_uint4(out[0], out[1], out[2], out[3]);
+        dense[2 * i + 1] = make_uint4(out[4], out[5], out[6], out[7]);
     }
 }
 
-template <int M, bool kBf16>
+template <int M, bool kBf16, bool kTC>
 cudaError_t launch_prune_t(const PruneArgs& a, cudaStream_t stream) {
     const RoundKeys rk = make_round_keys(a.seed);
     const int64_t upr_total = a.k_total / 16, uoff = a.k_offset / 16;
@@ -269,15 +335,18 @@ cudaError_t launch_prune_t(const PruneArgs& a, cudaStream_t stream) {
         const bool linear = (a.ld == a.cols) && (a.k_total == a.cols) && (a.k_offset == 0);
         const int64_t want = (n_slots + 255) / 256;
         const int grid = (int)(want < (int64_t)a.sm_count * 48 ? want : (int64_t)a.sm_count * 48);
+        const int64_t pad_rows = kTC ? ((a.rows + 127) / 128) * 128 - a.rows : 0;
         if (linear)
-            prune_axis1_kernel<M, kBf16, true><<<grid, 256, 0, stream>>>(a.g, n_slots, upr, a.ld, upr_total, uoff, rk, values, meta);
+            prune_axis1_kernel<M, kBf16, true, kTC><<<grid, 256, 0, stream>>>(a.g, n_slots, upr, a.ld, upr_total, uoff, pad_rows, rk, values, meta);
         else
-            prune_axis1_kernel<M, kBf16, false><<<grid, 256, 0, stream>>>(a.g, n_slots, upr, a.ld, upr_total, uoff, rk, values, meta);
+            prune_axis1_kernel<M, kBf16, false, kTC><<<grid, 256, 0, stream>>>(a.g, n_slots, upr, a.ld, upr_total, uoff, pad_rows, rk, values, meta);
     } else {
         const int64_t n_strips = a.rows / 16;
+        // in tensor-core order the rows of A are padded to 128: cover the padding with (load-free) tiles
+        const int64_t cover_cols = kTC ? ((a.cols + 127) / 128) * 128 : a.cols;
         dim3 grid((unsigned)((n_strips + kTileStrips - 1) / kTileStrips),
-                  (unsigned)((a.cols + kTileCols - 1) / kTileCols));
-        prune_axis0_kernel<M, kBf16><<<grid, kTileStrips * 32, 0, stream>>>(a.g, n_strips, a.cols, a.ld, upr_total, uoff, rk, values, meta);
+                  (unsigned)((cover_cols + kTileCols - 1) / kTileCols));
+        prune_axis0_kernel<M, kBf16, kTC><<<grid, kTileStrips * 32, 0, stream>>>(a.g, n_strips, a.cols, a.ld, upr_total, uoff, rk, values, meta);
     }
     return cudaGetLastError();
 }
@@ -285,18 +354,27 @@ cudaError_t launch_prune_t(const PruneArgs& a, cudaStream_t stream) {
 }  // namespace
 
 cudaError_t launch_prune(const PruneArgs& a, cudaStream_t stream) {
-    if (a.m == 4) return a.is_bf16 ? launch_prune_t<4, true>(a, stream) : launch_prune_t<4, false>(a, stream);
-    return a.is_bf16 ? launch_prune_t<2, true>(a, stream) : launch_prune_t<2, false>(a, stream);
+    if (a.tc_layout) {
+        if (a.m == 4) return a.is_bf16 ? launch_prune_t<4, true, true>(a, stream) : launch_prune_t<4, false, true>(a, stream);
+        return a.is_bf16 ? launch_prune_t<2, true, true>(a, stream) : launch_prune_t<2, false, true>(a, stream);
+    }
+    if (a.m == 4) return a.is_bf16 ? launch_prune_t<4, true, false>(a, stream) : launch_prune_t<4, false, false>(a, stream);
+    return a.is_bf16 ? launch_prune_t<2, true, false>(a, stream) : launch_prune_t<2, false, false>(a, stream);
 }
 
-cudaError_t launch_unpack(const void* values, const void* meta, int64_t mrows, int64_t K, void* dense,
-                          int sm_count, cudaStream_t stream) {
-    const int64_t n_bytes = mrows * (K / 8);
-    const int64_t want = (n_bytes + 255) / 256;
+cudaError_t launch_unpack(const void* values, const void* meta, bool tc_layout, int64_t mrows, int64_t K,
+                          void* dense, int sm_count, cudaStream_t stream) {
+    const int64_t n_units = mrows * (K / 16);
+    const int64_t want = (n_units + 255) / 256;
     const int grid = (int)(want < (int64_t)sm_count * 32 ? want : (int64_t)sm_count * 32);
-    unpack_kernel<<<grid, 256, 0, stream>>>(reinterpret_cast<const uint32_t*>(values),
-                                            reinterpret_cast<const uint8_t*>(meta), n_bytes,
-                                            reinterpret_cast<uint4*>(dense));
+    if (tc_layout)
+        unpack_kernel<true><<<grid, 256, 0, stream>>>(reinterpret_cast<const uint4*>(values),
+                                                      reinterpret_cast<const uint16_t*>(meta), n_units, K / 16,
+                                                      reinterpret_cast<uint4*>(dense));
+    else
+        unpack_kernel<false><<<grid, 256, 0, stream>>>(reinterpret_cast<const uint4*>(values),
+                                                       reinterpret_cast<const uint16_t*>(meta), n_units, K / 16,
+                                                       reinterpret_cast<uint4*>(dense));
     return cudaGetLastError();
 }
 

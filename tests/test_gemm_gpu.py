@@ -7,6 +7,9 @@ import torch
 
 import oracle
 from paper_2203_10991_b200 import binding, workloads
+from tests.helpers import layouts
+
+TC = binding.MVUE_LAYOUT_TC
 
 pytestmark = pytest.mark.gpu
 TOL = 1e-2          # the stated bar
@@ -39,7 +42,7 @@ def pack_canonical(A: np.ndarray):
 def test_one_hot_probes_fix_every_layout():
     # a single non-zero in A and in B: any mistake in the operand layouts, the metadata placement or
     # the output mapping moves or loses the single product
-    M, N, K = 256, 512, 192
+    M, N, K = 256, 512, 384
     rng = np.random.Generator(np.random.PCG64(3))
     for _ in range(24):
         m, n, k = int(rng.integers(0, M)), int(rng.integers(0, N)), int(rng.integers(0, K))
@@ -49,7 +52,7 @@ def test_one_hot_probes_fix_every_layout():
         B[k, n] = -3.0
         vals, meta = pack_canonical(A)
         assert np.array_equal(oracle.unpack(vals, meta), A)
-        out = binding.mvue_sparse_update_gemm(to_dev(vals), torch.from_numpy(meta).cuda(),
+        out = binding.mvue_sparse_update_gemm(to_dev(vals), torch.from_numpy(layouts.canonical_to_tc(meta)).cuda(),
                                               to_dev(workloads.to_bf16_bits(B)))
         got = out.cpu().numpy()
         want = np.zeros((M, N), dtype=np.float32)
@@ -57,13 +60,13 @@ def test_one_hot_probes_fix_every_layout():
         assert np.array_equal(got, want), (m, n, k, np.argwhere(got != 0)[:4])
 
 
-@pytest.mark.parametrize("T,n_out,n_in", [(64, 8, 8), (512, 256, 256), (640, 136, 264), (2048, 384, 520),
+@pytest.mark.parametrize("T,n_out,n_in", [(128, 8, 8), (512, 256, 256), (640, 136, 264), (2048, 384, 520),
                                           (8192, 768, 3072), (16384, 256, 2304)])
 @pytest.mark.parametrize("n,m", [(2, 4), (1, 2)])
 def test_update_gemm_matches_oracle(T, n_out, n_in, n, m):
     g = workloads.gradient((T, n_out), "student_t", seed=T + n_out, dtype="bf16")
     h = workloads.normal_bf16((T, n_in), seed=7)
-    vals, meta = binding.mvue_prune(to_dev(g), n, m, 0, seed=11)
+    vals, meta = binding.mvue_prune(to_dev(g), n, m, 0, seed=11, layout=TC)
     st = torch.zeros(1, dtype=torch.int32, device="cuda")
     dW = binding.mvue_sparse_update_gemm(vals, meta, to_dev(h), dev_status=st)
     torch.cuda.synchronize()
@@ -87,14 +90,14 @@ def test_update_gemm_matches_oracle(T, n_out, n_in, n, m):
             assert abs(got[i, j] - w) <= 1e-4 * (abs(w) + np.abs(A[i]).sum() * 1e-3)
 
 
-@pytest.mark.parametrize("T,n_out,n_in", [(256, 512, 128), (1000 // 8 * 8, 768, 3072), (8192, 3072, 768)])
+@pytest.mark.parametrize("T,n_out,n_in", [(256, 512, 128), (1000, 768, 3072), (8192, 3072, 768)])
 @pytest.mark.parametrize("with_act", [False, True])
 @pytest.mark.parametrize("out_dtype", [torch.float32, torch.bfloat16])
 def test_backward_gemm_matches_oracle(T, n_out, n_in, with_act, out_dtype):
     g = workloads.gradient((T, n_out), "student_t", seed=3, dtype="bf16")
     W = workloads.normal_bf16((n_out, n_in), seed=4, std=0.02)
     act = workloads.normal_bf16((T, n_in), seed=5) if with_act else None
-    vals, meta = binding.mvue_prune(to_dev(g), 2, 4, 1, seed=21)
+    vals, meta = binding.mvue_prune(to_dev(g), 2, 4, 1, seed=21, layout=TC)
     dh = binding.mvue_sparse_backward_gemm(vals, meta, to_dev(W), act_grad=None if act is None else to_dev(act),
                                            out_dtype=out_dtype)
     v_ref, m_ref = oracle.prune(g, 2, 4, axis=1, seed=21, threads=oracle.host_threads())
@@ -110,7 +113,7 @@ def test_accumulate_and_preallocated_output():
     T, n_out, n_in = 1024, 256, 512
     g = workloads.gradient((T, n_out), "relu_lognormal", seed=1, dtype="bf16")
     h = workloads.normal_bf16((T, n_in), seed=2)
-    vals, meta = binding.mvue_prune(to_dev(g), 2, 4, 0, seed=1)
+    vals, meta = binding.mvue_prune(to_dev(g), 2, 4, 0, seed=1, layout=TC)
     once = binding.mvue_sparse_update_gemm(vals, meta, to_dev(h))
     acc = torch.full((n_out, n_in), 1.5, dtype=torch.float32, device="cuda")
     binding.mvue_sparse_update_gemm(vals, meta, to_dev(h), out=acc, accumulate=True)
@@ -127,7 +130,7 @@ def test_split_k_is_deterministic_and_equal_to_unsplit_sum():
     g = workloads.gradient((T, n_out), "student_t", seed=9, dtype="bf16")
     h = workloads.normal_bf16((T, n_in), seed=8)
     assert binding.mvue_gemm_workspace_bytes(0, n_out, n_in, T) > 0
-    vals, meta = binding.mvue_prune(to_dev(g), 2, 4, 0, seed=2)
+    vals, meta = binding.mvue_prune(to_dev(g), 2, 4, 0, seed=2, layout=TC)
     a = binding.mvue_sparse_update_gemm(vals, meta, to_dev(h))
     b = binding.mvue_sparse_update_gemm(vals, meta, to_dev(h))
     assert torch.equal(a, b)
@@ -141,17 +144,19 @@ def test_gemm_argument_checks():
     meta = torch.zeros((64, 16), dtype=torch.uint8, device="cuda")
     h = torch.zeros((128, 64), dtype=torch.bfloat16, device="cuda")
     L = binding.lib()
-    args = lambda **kw: None
-    # K = 96 is not a multiple of 64
-    assert L.mvue_sparse_update_gemm(vals.data_ptr(), meta.data_ptr(), 0, 64, 96, h.data_ptr(), 64, 64,
+    # K = 192 is not a multiple of 128
+    assert L.mvue_sparse_update_gemm(vals.data_ptr(), meta.data_ptr(), TC, 64, 192, h.data_ptr(), 64, 64,
                                      h.data_ptr(), 0, 64, 0, None, 0, None, None) == -3
-    assert L.mvue_sparse_update_gemm(None, meta.data_ptr(), 0, 64, 128, h.data_ptr(), 64, 64,
+    assert L.mvue_sparse_update_gemm(None, meta.data_ptr(), TC, 64, 128, h.data_ptr(), 64, 64,
                                      h.data_ptr(), 0, 64, 0, None, 0, None, None) == -1
-    # accumulate into bf16 is refused
+    # the products read the tensor-core metadata order only
     assert L.mvue_sparse_update_gemm(vals.data_ptr(), meta.data_ptr(), 0, 64, 128, h.data_ptr(), 64, 64,
+                                     h.data_ptr(), 0, 64, 0, None, 0, None, None) == -6
+    # accumulate into bf16 is refused
+    assert L.mvue_sparse_update_gemm(vals.data_ptr(), meta.data_ptr(), TC, 64, 128, h.data_ptr(), 64, 64,
                                      h.data_ptr(), 1, 64, 1, None, 0, None, None) == -5
     # a reduction that needs split-K refuses a missing workspace
     big_k = 1 << 16
     if binding.mvue_gemm_workspace_bytes(0, 64, 64, big_k) > 0:
-        assert L.mvue_sparse_update_gemm(vals.data_ptr(), meta.data_ptr(), 0, 64, big_k, h.data_ptr(), 64, 64,
+        assert L.mvue_sparse_update_gemm(vals.data_ptr(), meta.data_ptr(), TC, 64, big_k, h.data_ptr(), 64, 64,
                                          h.data_ptr(), 0, 64, 0, None, 0, None, None) == -7

@@ -6,6 +6,7 @@ import torch
 
 import oracle
 from paper_2203_10991_b200 import binding, workloads
+from tests.helpers import layouts
 
 pytestmark = pytest.mark.gpu
 
@@ -157,3 +158,29 @@ def test_full_size_configs_sampled(name, n, m):
     # properties that hold at any size
     lo2, hi2 = m_gpu & 3, (m_gpu >> 2) & 3
     assert (lo2 < hi2).all() and ((m_gpu >> 4) & 3 < (m_gpu >> 6) & 3).all()
+
+
+@pytest.mark.parametrize("n,m", MODES)
+@pytest.mark.parametrize("axis", [0, 1])
+@pytest.mark.parametrize("shape", [(128, 128), (384, 200), (1024, 136), (2048, 1000), (4096, 1024)])
+@pytest.mark.parametrize("dtype", ["bf16", "f32"])
+def test_tensor_core_metadata_order(n, m, axis, shape, dtype):
+    """layout = MVUE_LAYOUT_TC: same survivors, metadata bit-identical to the oracle's once carried into
+    the tensor-core order (padding rows hold a valid pattern), and mvue_unpack reads it back."""
+    rows, cols = shape
+    if axis == 1:
+        cols = (cols + 127) // 128 * 128
+    else:
+        rows, cols = (rows + 127) // 128 * 128, (cols + 7) // 8 * 8
+    g = workloads.gradient((rows, cols), "relu_lognormal", seed=rows ^ cols, dtype=dtype)
+    values, meta = binding.mvue_prune(to_dev(g), n, m, axis, 31, layout=binding.MVUE_LAYOUT_TC)
+    dense = binding.mvue_unpack(values, meta, layout=binding.MVUE_LAYOUT_TC)
+    torch.cuda.synchronize()
+    v_ref, m_ref = oracle.prune(g, n, m, axis=axis, seed=31, threads=oracle.host_threads())
+    assert np.array_equal(values.view(torch.int16).cpu().numpy().view(np.uint16), v_ref)
+    got = meta.cpu().numpy().reshape(-1)
+    want = layouts.canonical_to_tc(m_ref)
+    assert got.shape == want.shape
+    assert np.array_equal(got, want)
+    assert np.array_equal(layouts.tc_to_canonical(got, *m_ref.shape[:1], m_ref.shape[1] * 8), m_ref)
+    assert np.array_equal(dense.float().cpu().numpy(), oracle.unpack(v_ref, m_ref))
