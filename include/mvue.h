@@ -160,6 +160,34 @@ MVUE_API int mvue_sparse_backward_gemm(const void* values, const void* meta, int
  * (which: 0 update, 1 backward).  bytes is a HOST pointer. */
 MVUE_API int mvue_gemm_workspace_bytes(int which, int64_t M, int64_t N, int64_t K, size_t* bytes);
 
+/* The update product for callers that cannot allocate device memory.
+ * (The paper has no counterpart; this is a convenience of this library.)
+ *
+ * Who needs it: code that runs where cudaMalloc is off limits -- a plugin inside a host
+ * application that owns the allocator and hands out only input and output buffers, a
+ * real-time or certified loop in which allocation calls are forbidden after start-up, a
+ * callback running where the CUDA allocator may not be entered.  Such a caller cannot
+ * supply the split-K workspace that mvue_sparse_update_gemm asks for on small outputs
+ * with a long reduction.
+ *
+ * Same result and same arguments as mvue_sparse_update_gemm, minus the workspace: the
+ * scratch is a fixed 8 MiB (MVUE_NOALLOC_SCRATCH_BYTES) array inside the library's device
+ * image.  Every GPU on which the library is loaded holds those bytes until the process
+ * exits.  The call itself allocates nothing, on the host side or the device side.
+ *  - A problem whose mvue_gemm_workspace_bytes(0, out, in, T) exceeds the array is refused
+ *    with MVUE_ERR_WORKSPACE; nothing is launched.
+ *  - The first call on each device looks up the array's device address (that device must
+ *    be current, as for every call).  Make that first call outside any stream capture.
+ *  - All calls on a device share the one array, and it keeps whatever the last call left.
+ *    The kernel overwrites every scratch element it later reads, so nothing has to be
+ *    cleared in between; but two calls that overlap on the GPU (different streams) race
+ *    on it.  Keep calls to this entry point on one stream, or order them with events. */
+#define MVUE_NOALLOC_SCRATCH_BYTES (8u << 20)
+MVUE_API int mvue_sparse_update_gemm_noalloc(const void* values, const void* meta, int layout,
+                                             int64_t out, int64_t T, const void* h, int64_t in,
+                                             int64_t ldh, void* dW, int dW_dtype, int64_t lddW,
+                                             int accumulate, int* dev_status, void* stream);
+
 MVUE_API const char* mvue_status_string(int status);
 /* Text of the last CUDA error seen by the calling thread ("" if none). */
 MVUE_API const char* mvue_last_cuda_error(void);

@@ -20,7 +20,7 @@ MVUE_LAYOUT_TC = 1
 
 EXPORTS = ("mvue_version", "mvue_status_string", "mvue_last_cuda_error", "mvue_packed_sizes",
            "mvue_prune", "mvue_unpack", "mvue_sparse_update_gemm", "mvue_sparse_backward_gemm",
-           "mvue_gemm_workspace_bytes")
+           "mvue_gemm_workspace_bytes", "mvue_sparse_update_gemm_noalloc")
 
 
 class MvueError(RuntimeError):
@@ -54,6 +54,7 @@ def lib() -> ctypes.CDLL:
         L.mvue_sparse_backward_gemm.argtypes = [vp, vp, ci, i64, i64, vp, i64, i64, vp, vp, ci, i64, vp,
                                                 ctypes.c_size_t, vp, vp]
         L.mvue_gemm_workspace_bytes.argtypes = [ci, i64, i64, i64, szp]
+        L.mvue_sparse_update_gemm_noalloc.argtypes = [vp, vp, ci, i64, i64, vp, i64, i64, vp, ci, i64, ci, vp, vp]
         _lib = L
     return _lib
 
@@ -164,4 +165,20 @@ def mvue_sparse_backward_gemm(values: torch.Tensor, meta: torch.Tensor, W: torch
                                            None if ws is None else ws.data_ptr(), ws_bytes,
                                            None if dev_status is None else dev_status.data_ptr(), _stream_ptr()),
            "mvue_sparse_backward_gemm")
+    return out
+
+
+def mvue_sparse_update_gemm_noalloc(values: torch.Tensor, meta: torch.Tensor, h: torch.Tensor, out: torch.Tensor, *,
+                                    accumulate: bool = False, dev_status: torch.Tensor | None = None,
+                                    layout: int = MVUE_LAYOUT_TC) -> torch.Tensor:
+    """The update product for callers that may not allocate: the caller passes every buffer, including
+    `out`, and the split-K scratch is the fixed array inside the library (8 MiB per GPU).  Nothing is
+    allocated here either.  Raises MvueError(-7) when the problem needs more scratch than that."""
+    n_out, half_t = values.shape
+    T, n_in = h.shape
+    _check(lib().mvue_sparse_update_gemm_noalloc(values.data_ptr(), meta.data_ptr(), layout, n_out, T, h.data_ptr(),
+                                                 n_in, h.stride(0), out.data_ptr(), _dtype_code(out), out.stride(0),
+                                                 int(accumulate),
+                                                 None if dev_status is None else dev_status.data_ptr(),
+                                                 _stream_ptr()), "mvue_sparse_update_gemm_noalloc")
     return out

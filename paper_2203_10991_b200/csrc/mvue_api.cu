@@ -174,4 +174,19 @@ int mvue_sparse_backward_gemm(const void* values, const void* meta, int layout, 
                     workspace_bytes, dev_status, stream);
 }
 
+int mvue_sparse_update_gemm_noalloc(const void* values, const void* meta, int layout, int64_t out, int64_t T,
+                                    const void* h, int64_t in, int64_t ldh, void* dW, int dW_dtype,
+                                    int64_t lddW, int accumulate, int* dev_status, void* stream) {
+    if (out <= 0 || in <= 0 || T <= 0 || T % 128 != 0) return MVUE_ERR_SHAPE;
+    DeviceInfo dev;
+    if (int s = current_device_info(&dev)) return s;
+    const size_t need = gemm_workspace_bytes(out, in, T, dev.sm_count);
+    if (need > kStaticScratchBytes) return MVUE_ERR_WORKSPACE;     // beyond what the library carries
+    void* scratch = nullptr;
+    size_t scratch_bytes = 0;
+    if (int s = static_scratch(&scratch, &scratch_bytes)) return s;
+    return run_gemm(values, meta, layout, out, in, T, h, ldh, nullptr, dW, dW_dtype, lddW, accumulate,
+                    scratch, scratch_bytes, dev_status, stream);
+}
+
 }  // extern "C"

@@ -430,6 +430,31 @@ size_t gemm_workspace_bytes(int64_t M, int64_t N, int64_t K, int sm_count) {
     return splits > 1 ? (size_t)splits * (size_t)M * (size_t)N * sizeof(float) : 0;
 }
 
+// ---- library-owned split-K scratch --------------------------------------------------
+// Scratch for callers that have no way to allocate device memory.  It lives in the library's
+// device image: every GPU that loads the library carries these bytes until the process exits.
+// The name below is only a host-side handle; the device address is looked up once per device.
+__device__ __align__(256) static unsigned char g_static_scratch[kStaticScratchBytes];
+
+int static_scratch(void** ptr, size_t* bytes) {
+    static std::mutex mu;
+    static void* addr[64] = {};
+    int dev = 0;
+    cudaError_t e = cudaGetDevice(&dev);
+    if (e != cudaSuccess) { set_cuda_error(e, "cudaGetDevice"); return MVUE_ERR_CUDA; }
+    if (dev < 0 || dev >= 64) return MVUE_ERR_ARCH;
+    std::lock_guard<std::mutex> lock(mu);
+    if (!addr[dev]) {
+        void* q = nullptr;
+        e = cudaGetSymbolAddress(&q, g_static_scratch);      // the current device's copy of the array
+        if (e != cudaSuccess || !q) { set_cuda_error(e, "cudaGetSymbolAddress"); return MVUE_ERR_CUDA; }
+        addr[dev] = q;
+    }
+    *ptr = addr[dev];
+    *bytes = kStaticScratchBytes;
+    return MVUE_OK;
+}
+
 int launch_sparse_gemm(const SparseGemmArgs& a, cudaStream_t stream) {
     CUtensorMap map_a, map_b, map_e;
     const uint64_t e_blocks = (uint64_t)((a.M + BM - 1) / BM) * (uint64_t)(a.K / BK);

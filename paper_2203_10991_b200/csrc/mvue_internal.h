@@ -44,6 +44,10 @@ int launch_sparse_gemm(const SparseGemmArgs& a, cudaStream_t stream);     // ret
 int gemm_split_count(int64_t M, int64_t N, int64_t K, int sm_count);
 size_t gemm_workspace_bytes(int64_t M, int64_t N, int64_t K, int sm_count);
 
+// Split-K scratch that the library itself carries (see mvue_sparse_update_gemm_noalloc).
+constexpr size_t kStaticScratchBytes = 8u << 20;
+int static_scratch(void** ptr, size_t* bytes);   // returns an mvue_status; device address for the current device
+
 // Per-device facts, looked up once.
 struct DeviceInfo {
     int cc_major = 0;
