@@ -1,14 +1,18 @@
 #!/usr/bin/env python
-"""Benchmark of the MVUE prune+pack (and consuming products) on B200.
+"""Benchmark of the MVUE hot path on B200: prune+pack of the neural gradient followed by the
+2:4-sparse update product that consumes it.
 
-    python bench.py [--gpus N] [--steps K] [--warmup W] [--impl ours|reference] [--workload NAME]
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--impl ours|reference] [--workload NAME] [--prune n:m]
 
-Prints ONE JSON line.  A step is one pass of the hot path over one synthetic batch of
-the `conv_im2col` workload (gradient g bf16 [200704 x 256], ReLU-sparse lognormal; MVUE
-2:4 along the token axis).  `value` is the throughput with inputs resident in HBM;
-`e2e` repeats the measurement through the same C-ABI call with pinned host buffers and the
-host<->device copies inside the timed region.  `--impl reference` times the CPU oracle on a
-bounded sample of the same workload.
+Prints ONE JSON line.  A step is one pass of the whole path over one synthetic batch of the
+`conv_im2col` workload: g bf16 [200704 x 256] (ReLU-sparse lognormal), h bf16 [200704 x 2304]:
+    values, meta = mvue_prune(g, 2:4, along the token axis)      # Sec. 4.2 / App. A.2
+    dW[256 x 2304] = theta(g)^T h                                  # Sec. 1, update equation
+`value` is the step's algorithmic bytes per second with every input resident in HBM (the step is
+HBM-bound on this workload: h alone is 925 MB, far beyond L2, so no step finds its inputs cached);
+the per-kernel figures (prune GB/s, GEMM effective TFLOP/s, dense cuBLAS for the same shape) ride
+along.  `e2e` repeats the step through the same C-ABI calls from pinned host buffers with the
+copies inside the timed region.  `--impl reference` times the CPU oracle on a bounded sample.
 """
 from __future__ import annotations
 
@@ -26,7 +30,6 @@ ROOT = Path(__file__).resolve().parent
 sys.path.insert(0, str(ROOT))
 
 METRIC = "prune+pack GB/s (% HBM peak); MVUE-sparse GEMM TFLOP/s vs dense bf16"
-L2_BYTES = 126 * 1024 * 1024
 
 
 def measured_peaks():
@@ -40,16 +43,21 @@ def measured_peaks():
 
 
 def prune_bytes(rows: int, cols: int, elem_bytes: int) -> int:
-    """Algorithmic bytes of one prune+pack: g read once, K/2 bf16 survivors and 4 bits of
-    metadata per group of four written once."""
+    """Algorithmic bytes of one prune+pack: g read once; K/2 bf16 survivors and 4 bits of metadata per
+    group of four written once (3.125 B per bf16 element, 5.125 B per fp32 element)."""
     n = rows * cols
     return n * elem_bytes + n + n // 8
+
+
+def gemm_bytes(M: int, N: int, K: int, c_bytes: int = 4) -> int:
+    """Minimum traffic of C[MxN] = A_packed[MxK] . B[KxN]: survivors, metadata, B and C once each."""
+    return M * K + M * K // 8 + K * N * 2 + M * N * c_bytes
 
 
 class ClockSampler:
     """Samples SM clock and throttle reasons of one GPU through NVML while a region runs."""
 
-    def __init__(self, index: int, period_s: float = 0.05):
+    def __init__(self, index: int, period_s: float = 0.02):
         self.index, self.period = index, period_s
         self.samples, self.reasons = [], set()
         self.max_mhz = None
@@ -105,43 +113,48 @@ class ClockSampler:
 
 # --------------------------------------------------------------------------- CPU oracle arm
 def oracle_sample(cfg, n, m, sample_rows: int):
-    """Time the oracle's prune+pack, as it stands, on the first `sample_rows` token rows."""
+    """One pass of the oracle, as it stands, over the first `sample_rows` token rows: prune+pack,
+    unpack, and the fp64 plain-loop update product.  Returns (GB/s of algorithmic bytes, threads, s)."""
     import oracle
     from paper_2203_10991_b200 import workloads
     g = workloads.gradient((sample_rows, cfg["out"]), cfg["g_dist"], cfg["seed"], dtype=cfg["g_dtype"])
+    h = workloads.normal_bf16((sample_rows, cfg["inp"]), cfg["seed"] + 100)
     threads = oracle.host_threads()
     t0 = time.perf_counter()
-    oracle.prune(g, n, m, axis=0, seed=0, k_total=cfg["T"], k_offset=0, threads=threads)
+    values, meta = oracle.prune(g, n, m, axis=0, seed=0, k_total=cfg["T"], k_offset=0, threads=threads)
+    oracle.gemm(oracle.unpack(values, meta), h, threads=threads)
     dt = time.perf_counter() - t0
-    nbytes = prune_bytes(sample_rows, cfg["out"], 2 if cfg["g_dtype"] == "bf16" else 4)
+    nbytes = (prune_bytes(sample_rows, cfg["out"], 2 if cfg["g_dtype"] == "bf16" else 4)
+              + gemm_bytes(cfg["out"], cfg["inp"], sample_rows))
     return nbytes / dt / 1e9, threads, dt
 
 
 def run_reference(args, cfg, n, m):
-    rank = int(os.environ.get("RANK", "0"))
-    if rank != 0:
+    if int(os.environ.get("RANK", "0")) != 0:
         return
-    # size the per-step sample so that K + W steps of the oracle take about a minute in all
-    _, _, dt_probe = oracle_sample(cfg, n, m, 8192)
-    rows_per_s = 8192 / dt_probe
-    budget_s = 60.0
-    sample_rows = int(rows_per_s * budget_s / max(1, args.steps + args.warmup))
-    sample_rows = max(1024, min(cfg["T"], sample_rows // 16 * 16))
-    vals = []
+    # size the per-step sample so that K + W steps of the oracle take about a minute in all: its cost
+    # grows faster than linearly with the rows (the plain loops leave the cache), so probe by doubling
+    per_step_s = 60.0 / max(1, args.steps + args.warmup)
+    sample_rows = 512
+    while sample_rows * 2 <= cfg["T"]:
+        _, _, dt_probe = oracle_sample(cfg, n, m, sample_rows)
+        if dt_probe > per_step_s / 3:
+            break
+        sample_rows *= 2
     for _ in range(args.warmup):
         oracle_sample(cfg, n, m, sample_rows)
-    t_all = 0.0
+    vals, t_all, threads = [], 0.0, 1
     for _ in range(args.steps):
         gbs, threads, dt = oracle_sample(cfg, n, m, sample_rows)
         vals.append(gbs)
         t_all += dt
     value = float(np.mean(vals))
-    sample = f"first {sample_rows} of {cfg['T']} token rows x {cfg['out']} channels, MVUE {n}:{m}, axis 0"
+    sample = (f"first {sample_rows} of {cfg['T']} token rows: MVUE {n}:{m} prune+pack of g[{sample_rows}x{cfg['out']}] "
+              f"and the fp64 update product with h[{sample_rows}x{cfg['inp']}]")
     print(json.dumps({
         "impl": "reference", "metric": METRIC, "value": value, "unit": "GB/s", "n_gpus": args.gpus,
         "steps": args.steps, "warmup": args.warmup, "ms_per_step": 1e3 * t_all / max(1, args.steps),
-        "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "f32",
-        "data": "synthetic",
+        "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "bf16", "data": "synthetic",
         "config": {"workload": args.workload, "prune": f"{n}:{m}", "axis": 0, "sample_rows": sample_rows},
         "cpu_baseline": {"value": value, "unit": "GB/s", "cores": threads, "kind": "oracle", "sample": sample},
         "e2e": {"value": value, "unit": "GB/s", "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
@@ -162,43 +175,66 @@ def run_ours(args, cfg, n, m):
     if world > 1:
         dist.init_process_group("nccl", device_id=dev)
     binding.lib()                                       # fail loudly if the CUDA library is absent
+    TC = binding.MVUE_LAYOUT_TC
 
-    T, out = cfg["T"], cfg["out"]
+    T, out, inp = cfg["T"], cfg["out"], cfg["inp"]
     elem = 2 if cfg["g_dtype"] == "bf16" else 4
-    # every rank draws its own batch (weak scaling: independent batches, no data-path collective)
+    # every rank draws its own token shard (data parallel over tokens, weak scaling)
     g_host = workloads.gradient((T, out), cfg["g_dist"], cfg["seed"] + 1000 * rank, dtype=cfg["g_dtype"])
+    h_host = workloads.normal_bf16((T, inp), cfg["seed"] + 100 + 1000 * rank)
     g_t = torch.from_numpy(g_host.view(np.int16) if elem == 2 else g_host)
-    step_bytes = prune_bytes(T, out, elem)
-    # rotate over enough distinct input/output buffers that no step finds its data in L2
-    n_buf = max(2, int(np.ceil(2.5 * L2_BYTES / step_bytes)) + 1)
-    gs = []
-    for i in range(n_buf):
-        x = g_t.to(dev)
-        gs.append(x.view(torch.bfloat16) if elem == 2 else x)
-    outs = [(torch.empty((out, T // 2), dtype=torch.bfloat16, device=dev),
-             torch.empty((out, T // 8), dtype=torch.uint8, device=dev)) for _ in range(n_buf)]
+    h_t = torch.from_numpy(h_host.view(np.int16))
+    g_dev = g_t.to(dev)
+    g_dev = g_dev.view(torch.bfloat16) if elem == 2 else g_dev
+    h_dev = h_t.to(dev).view(torch.bfloat16)
+    _, meta_bytes = binding.mvue_packed_sizes(T, out, n, m, 0, TC)
+    values = torch.empty((out, T // 2), dtype=torch.bfloat16, device=dev)
+    meta = torch.empty(meta_bytes, dtype=torch.uint8, device=dev)
+    dW = torch.empty((out, inp), dtype=torch.float32, device=dev)
+    ws_bytes = binding.mvue_gemm_workspace_bytes(0, out, inp, T)
+    ws = torch.empty(max(ws_bytes, 16), dtype=torch.uint8, device=dev)
+    status = torch.zeros(1, dtype=torch.int32, device=dev)
+    launches_per_step = 2 + (1 if ws_bytes > 0 else 0)      # prune, sparse GEMM, split-K reduction
 
-    def step(i):
-        b = i % n_buf
-        binding.mvue_prune(gs[b], n, m, 0, i, values=outs[b][0], meta=outs[b][1])
+    p_bytes = prune_bytes(T, out, elem)
+    m_bytes = gemm_bytes(out, inp, T)
+    step_bytes = p_bytes + m_bytes
+    gemm_flops = 2.0 * out * inp * T
+
+    def step(i, ev=None):
+        if ev:
+            ev[0].record()
+        binding.mvue_prune(g_dev, n, m, 0, i, values=values, meta=meta, layout=TC)
+        if ev:
+            ev[1].record()
+        binding.mvue_sparse_update_gemm(values, meta, h_dev, out=dW, workspace=ws, dev_status=status)
+        if ev:
+            ev[2].record()
+        if world > 1:
+            dist.all_reduce(dW)                              # the data-parallel exchange of the update
 
     def barrier():
         if world > 1:
             dist.barrier()
         torch.cuda.synchronize()
 
-    for i in range(max(3, args.warmup)):
+    warm = max(3, args.warmup)
+    for i in range(warm):
         step(i)
     barrier()
+    evs = [[torch.cuda.Event(enable_timing=True) for _ in range(3)] for _ in range(args.steps)]
     ev0, ev1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
     with ClockSampler(local) as clocks:
         barrier()
         ev0.record()
         for i in range(args.steps):
-            step(i)
+            step(i, evs[i])
         ev1.record()
         barrier()
+    assert int(status.item()) == 0, "a bounded device-side wait expired"
     ms = ev0.elapsed_time(ev1)
+    prune_ms = float(np.mean([e[0].elapsed_time(e[1]) for e in evs]))
+    gemm_ms = float(np.mean([e[1].elapsed_time(e[2]) for e in evs]))
     if world > 1:
         t = torch.tensor([ms], device=dev)
         dist.all_reduce(t, op=dist.ReduceOp.MAX)
@@ -206,21 +242,32 @@ def run_ours(args, cfg, n, m):
     ms_per_step = ms / args.steps
     value = world * step_bytes / (ms_per_step * 1e-3) / 1e9
 
-    # end to end: pinned host input -> device -> prune -> packed result back to pinned host
-    g_pin = g_t.pin_memory()
-    v_pin = torch.empty((out, T // 2), dtype=torch.bfloat16).pin_memory()
-    m_pin = torch.empty((out, T // 8), dtype=torch.uint8).pin_memory()
-    g_dev = gs[0]
-    e2e_steps = max(3, min(args.steps, 20))
+    # dense cuBLAS bf16 for the same shape (context for the sparse product)
+    dense_ms = None
+    if rank == 0 and elem == 2:
+        gT = g_dev.t()
+        for _ in range(3):
+            torch.matmul(gT, h_dev)
+        torch.cuda.synchronize()
+        ev0.record()
+        for _ in range(10):
+            torch.matmul(gT, h_dev)
+        ev1.record()
+        torch.cuda.synchronize()
+        dense_ms = ev0.elapsed_time(ev1) / 10
+
+    # end to end: pinned host g and h -> device -> prune -> GEMM -> dW back to pinned host
+    g_pin, h_pin = g_t.pin_memory(), h_t.pin_memory()
+    dW_pin = torch.empty((out, inp), dtype=torch.float32).pin_memory()
+    e2e_steps = max(2, min(args.steps, 5))
 
     def e2e_step(i):
         g_dev.view(torch.int16 if elem == 2 else torch.float32).copy_(g_pin, non_blocking=True)
-        binding.mvue_prune(g_dev, n, m, 0, i, values=outs[0][0], meta=outs[0][1])
-        v_pin.copy_(outs[0][0], non_blocking=True)
-        m_pin.copy_(outs[0][1], non_blocking=True)
+        h_dev.view(torch.int16).copy_(h_pin, non_blocking=True)
+        step(i)
+        dW_pin.copy_(dW, non_blocking=True)
 
-    for i in range(3):
-        e2e_step(i)
+    e2e_step(0)
     barrier()
     ev0.record()
     for i in range(e2e_steps):
@@ -236,27 +283,41 @@ def run_ours(args, cfg, n, m):
 
     if rank == 0:
         peaks = measured_peaks()
-        achieved = step_bytes / (ms_per_step * 1e-3) / 1e9
+        prune_gbs = p_bytes / (prune_ms * 1e-3) / 1e9
+        gemm_gbs = m_bytes / (gemm_ms * 1e-3) / 1e9
+        gemm_tf = gemm_flops / (gemm_ms * 1e-3) / 1e12
+        sparse_peak = 2.0 * peaks["bf16_tflops"]
         line = {
             "metric": METRIC, "value": value, "unit": "GB/s", "n_gpus": world, "steps": args.steps,
-            "warmup": max(3, args.warmup), "ms_per_step": ms_per_step, "higher_is_better": True,
-            "scaling": "weak", "vs_baseline": None, "dtype": "f32", "data": "synthetic",
-            "config": {"workload": args.workload, "g": [T, out], "g_dtype": cfg["g_dtype"],
-                       "prune": f"{n}:{m}", "axis": 0, "l2": f"rotating {n_buf} buffer sets (> 2.5x L2)"},
+            "warmup": warm, "ms_per_step": ms_per_step, "higher_is_better": True, "scaling": "weak",
+            "vs_baseline": None, "dtype": "bf16", "data": "synthetic",
+            "config": {"workload": args.workload, "g": [T, out], "h": [T, inp], "g_dtype": cfg["g_dtype"],
+                       "prune": f"{n}:{m}", "axis": 0, "dW_dtype": "f32",
+                       "l2": "inputs larger than L2 (h is 925 MB, read once per step)"},
             "clocks": clocks.summary(),
-            "e2e": {"value": e2e_value, "unit": "GB/s", "h2d_bytes_per_step": T * out * elem,
-                    "d2h_bytes_per_step": T * out + T * out // 8},
-            "gpu_launches": args.steps,
-            "roofline": {"bound": "hbm", "kernel": "prune_axis0_kernel", "achieved": achieved,
-                         "peak": peaks["hbm_gbs"], "unit": "GB/s", "frac": achieved / peaks["hbm_gbs"],
+            "e2e": {"value": e2e_value, "unit": "GB/s", "h2d_bytes_per_step": T * out * elem + T * inp * 2,
+                    "d2h_bytes_per_step": out * inp * 4},
+            "gpu_launches": args.steps * launches_per_step,
+            "prune": {"ms": prune_ms, "gbs": prune_gbs, "frac_of_hbm_peak": prune_gbs / peaks["hbm_gbs"]},
+            "gemm": {"ms": gemm_ms, "tflops_effective": gemm_tf, "frac_of_sparse_peak": gemm_tf / sparse_peak,
+                     "sparse_peak_tflops": sparse_peak, "gbs": gemm_gbs,
+                     "dense_cublas_ms": dense_ms,
+                     "dense_cublas_tflops": None if dense_ms is None else gemm_flops / (dense_ms * 1e-3) / 1e12},
+            # the dominant kernel of the step is the sparse product; on this shape (256 x 2304 outputs over
+            # 200704 rows, ~240 flop/B) it is bound by streaming h from HBM, not by the tensor cores
+            "roofline": {"bound": "hbm", "kernel": "sparse_gemm_pair_kernel", "achieved": gemm_gbs,
+                         "peak": peaks["hbm_gbs"], "unit": "GB/s", "frac": gemm_gbs / peaks["hbm_gbs"],
                          "peak_source": peaks["source"], "traffic": None},
+            "roofline_prune": {"bound": "hbm", "kernel": "prune_axis0_kernel", "achieved": prune_gbs,
+                               "peak": peaks["hbm_gbs"], "unit": "GB/s", "frac": prune_gbs / peaks["hbm_gbs"],
+                               "peak_source": peaks["source"], "traffic": None},
         }
         if world == 1 and not args.no_cpu_baseline:
-            sample_rows = min(T, 1 << 19)
+            sample_rows = min(T, 8192)
             gbs, threads, dt = oracle_sample(cfg, n, m, sample_rows)
             line["cpu_baseline"] = {"value": gbs, "unit": "GB/s", "cores": threads, "kind": "oracle",
-                                    "sample": f"first {sample_rows} of {T} token rows x {out} channels, "
-                                              f"MVUE {n}:{m}, axis 0, {dt:.2f} s"}
+                                    "sample": f"first {sample_rows} of {T} token rows: MVUE {n}:{m} prune+pack and "
+                                              f"fp64 update product [{out}x{inp}], {dt:.1f} s"}
         print(json.dumps(line))
     if world > 1:
         dist.destroy_process_group()
@@ -266,7 +327,7 @@ def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
     ap.add_argument("--steps", type=int, default=None)
-    ap.add_argument("--warmup", type=int, default=10)
+    ap.add_argument("--warmup", type=int, default=5)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--workload", default="conv_im2col")
     ap.add_argument("--prune", default="2:4")
@@ -276,10 +337,10 @@ def main():
     cfg = workloads.CONFIGS[args.workload]
     n, m = (int(x) for x in args.prune.split(":"))
     if args.impl == "reference":
-        args.steps = 5 if args.steps is None else args.steps
+        args.steps = 3 if args.steps is None else args.steps
         run_reference(args, cfg, n, m)
     else:
-        args.steps = 2000 if args.steps is None else args.steps
+        args.steps = 1000 if args.steps is None else args.steps
         run_ours(args, cfg, n, m)
 
 
