@@ -196,9 +196,8 @@ __device__ __forceinline__ uint32_t map_to_cta(uint32_t smem_addr, uint32_t rank
 __device__ __forceinline__ void cluster_sync() {
     asm volatile("barrier.cluster.arrive.release.aligned;\n\tbarrier.cluster.wait.acquire.aligned;" ::: "memory");
 }
-__device__ __forceinline__ void mbar_expect_tx_cluster(uint32_t cluster_bar, uint32_t bytes) {
-    asm volatile("mbarrier.arrive.expect_tx.release.cluster.shared::cluster.b64 _, [%0], %1;"
-                 ::"r"(cluster_bar), "r"(bytes) : "memory");
+__device__ __forceinline__ void mbar_expect_tx(uint32_t bar, uint32_t bytes) {
+    asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "r"(bytes) : "memory");
 }
 // TMA load whose completion bytes are counted on a barrier of the pair's leader.
 __device__ __forceinline__ void tma_load_2d_pair(uint32_t dst, const CUtensorMap* map, int x, int y,
@@ -252,7 +251,7 @@ sparse_gemm_pair_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_
 
     if (threadIdx.x == 0) {
         for (int s = 0; s < kStages; ++s) {
-            mbar_init(full_bar(s), 2);       // one arrival (with byte count) per block of the pair
+            mbar_init(full_bar(s), 1);       // the leader's producer arrives once, expecting both blocks' bytes
             mbar_init(empty_bar(s), 1);      // the leader's tcgen05.commit
         }
         mbar_init(acc_bar, 1);
@@ -284,7 +283,9 @@ sparse_gemm_pair_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_
                 const int64_t step = step_begin + i;
                 const int k = (int)(step * BK);
                 const uint32_t leader_full = map_to_cta(full_bar(s), 0);
-                mbar_expect_tx_cluster(leader_full, kStageBytes);
+                // only the leader arrives, and locally: a cluster-scope release from the peer on every stage
+                // would wait out the copies already in flight and serialise the pipeline
+                if (rank == 0) mbar_expect_tx(full_bar(s), 2 * kStageBytes);
                 // rows past M read as zeros (out-of-range boxes are zero-filled); the metadata of a row
                 // block that does not exist is taken from block 0 -- any valid pattern is harmless there
                 tma_load_2d_pair(a_dst, &map_a, k / 2, (int)m0, leader_full);
