@@ -312,8 +312,10 @@ def run_ours(args, cfg, n, m):
                                "peak": peaks["hbm_gbs"], "unit": "GB/s", "frac": prune_gbs / peaks["hbm_gbs"],
                                "peak_source": peaks["source"], "traffic": None},
         }
+        if world == 1 and not args.no_extra:
+            line["ffn_large"] = tensor_bound_case(n, m, peaks)
         if world == 1 and not args.no_cpu_baseline:
-            sample_rows = min(T, 8192)
+            sample_rows = min(T, 32768)
             gbs, threads, dt = oracle_sample(cfg, n, m, sample_rows)
             line["cpu_baseline"] = {"value": gbs, "unit": "GB/s", "cores": threads, "kind": "oracle",
                                     "sample": f"first {sample_rows} of {T} token rows: MVUE {n}:{m} prune+pack and "
@@ -321,6 +323,50 @@ def run_ours(args, cfg, n, m):
         print(json.dumps(line))
     if world > 1:
         dist.destroy_process_group()
+
+
+def tensor_bound_case(n, m, peaks):
+    """The large FFN layer (tokens 16384, 4096 -> 14336): the shape on which the sparse product is bound by
+    the tensor cores, timed kernel by kernel next to dense cuBLAS.  Rides along in the JSON line."""
+    import torch
+    from paper_2203_10991_b200 import binding, workloads
+    cfg = workloads.CONFIGS["ffn_large"]
+    T, out, inp = cfg["T"], cfg["out"], cfg["inp"]
+    TC = binding.MVUE_LAYOUT_TC
+    g = torch.from_numpy(workloads.gradient((T, out), cfg["g_dist"], cfg["seed"], dtype="bf16").view(np.int16))
+    g = g.cuda().view(torch.bfloat16)
+    h = torch.from_numpy(workloads.normal_bf16((T, inp), cfg["seed"] + 100).view(np.int16)).cuda().view(torch.bfloat16)
+    values, meta = binding.mvue_prune(g, n, m, 0, 0, layout=TC)
+    dW = torch.empty((out, inp), dtype=torch.float32, device="cuda")
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+
+    def timed(fn, iters):
+        for _ in range(3):
+            fn()
+        torch.cuda.synchronize()
+        e0.record()
+        for _ in range(iters):
+            fn()
+        e1.record()
+        torch.cuda.synchronize()
+        return e0.elapsed_time(e1) / iters
+
+    prune_ms = timed(lambda: binding.mvue_prune(g, n, m, 0, 1, values=values, meta=meta, layout=TC), 20)
+    gemm_ms = timed(lambda: binding.mvue_sparse_update_gemm(values, meta, h, out=dW), 30)
+    gT = g.t()
+    dense_ms = timed(lambda: torch.matmul(gT, h), 30)
+    flops = 2.0 * out * inp * T
+    tf = flops / (gemm_ms * 1e-3) / 1e12
+    pgbs = prune_bytes(T, out, 2) / (prune_ms * 1e-3) / 1e9
+    return {"g": [T, out], "h": [T, inp], "prune": f"{n}:{m}",
+            "prune_ms": prune_ms, "prune_gbs": pgbs, "prune_frac_of_hbm_peak": pgbs / peaks["hbm_gbs"],
+            "gemm_ms": gemm_ms, "gemm_tflops_effective": tf,
+            "gemm_frac_of_sparse_peak_burst": tf / (2 * peaks["bf16_tflops"]),
+            "gemm_frac_of_sparse_peak_sustained": tf / (2 * peaks["bf16_tflops_sustained"]),
+            "dense_cublas_ms": dense_ms, "dense_cublas_tflops": flops / (dense_ms * 1e-3) / 1e12,
+            "roofline": {"bound": "tensor", "kernel": "sparse_gemm_pair_kernel", "achieved": tf,
+                         "peak": 2 * peaks["bf16_tflops"], "unit": "TFLOP/s", "frac": tf / (2 * peaks["bf16_tflops"]),
+                         "peak_source": peaks["source"] + " dense bf16 burst x 2 (2:4 sparse)", "traffic": None}}
 
 
 def main():
@@ -332,6 +378,7 @@ def main():
     ap.add_argument("--workload", default="conv_im2col")
     ap.add_argument("--prune", default="2:4")
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--no-extra", action="store_true", help="skip the tensor-bound ffn_large case")
     args = ap.parse_args()
     from paper_2203_10991_b200 import workloads
     cfg = workloads.CONFIGS[args.workload]
