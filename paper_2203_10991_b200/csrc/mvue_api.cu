@@ -125,7 +125,6 @@ int mvue_prune(const void* g, int dtype, int64_t rows, int64_t cols, int64_t ld,
     if (!aligned16(g) || !aligned16(values) || !aligned16(meta) || (ld * esz) % 16 != 0) return MVUE_ERR_ALIGN;
     DeviceInfo dev;
     if (int s = current_device_info(&dev)) return s;
-    if (layout == MVUE_LAYOUT_TC && (k_total != K || k_offset != 0)) return MVUE_ERR_LAYOUT;   // shards pack canonically
     PruneArgs a{g, dtype == MVUE_BF16, rows, cols, ld, m, axis, seed, k_total, k_offset, values, meta, dev.sm_count,
                 layout == MVUE_LAYOUT_TC};
     cudaError_t e = launch_prune(a, reinterpret_cast<cudaStream_t>(stream));

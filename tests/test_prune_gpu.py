@@ -184,3 +184,20 @@ def test_tensor_core_metadata_order(n, m, axis, shape, dtype):
     assert np.array_equal(got, want)
     assert np.array_equal(layouts.tc_to_canonical(got, *m_ref.shape[:1], m_ref.shape[1] * 8), m_ref)
     assert np.array_equal(dense.float().cpu().numpy(), oracle.unpack(v_ref, m_ref))
+
+
+@pytest.mark.parametrize("axis", [0, 1])
+def test_k_shards_in_tensor_core_order(axis):
+    """A token shard pruned with the global block numbering: same survivors and masks as the slice of the
+    unsharded run, metadata laid out for the shard's own K."""
+    g = workloads.gradient((512, 384), "student_t", seed=6, dtype="bf16")
+    K = g.shape[1] if axis == 1 else g.shape[0]
+    v_all, m_all = oracle.prune(g, 2, 4, axis=axis, seed=55, threads=oracle.host_threads())
+    for lo, hi in [(0, 128), (128, K)]:
+        part = np.ascontiguousarray(g[:, lo:hi] if axis == 1 else g[lo:hi])
+        values, meta = binding.mvue_prune(to_dev(part), 2, 4, axis, 55, k_total=K, k_offset=lo,
+                                          layout=binding.MVUE_LAYOUT_TC)
+        torch.cuda.synchronize()
+        assert np.array_equal(values.view(torch.int16).cpu().numpy().view(np.uint16), v_all[:, lo // 2:hi // 2])
+        want = layouts.canonical_to_tc(np.ascontiguousarray(m_all[:, lo // 8:hi // 8]))
+        assert np.array_equal(meta.cpu().numpy().reshape(-1), want)
