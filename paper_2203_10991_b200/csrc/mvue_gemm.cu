@@ -46,6 +46,7 @@ constexpr int kEBytes = BM * 16;           // 2 KiB: 16 bytes per tensor-memory 
 constexpr int kStageBytes = kABytes + kBBytes + kEBytes;
 constexpr int kSmemBytes = kStages * kStageBytes + 1024 /*alignment slack*/ + 256 /*barriers*/;
 constexpr int kThreads = 256;
+constexpr int kBandTiles = 8;              // row tiles per band of the tile order
 constexpr uint32_t kTmemCols = 512;
 constexpr uint32_t kTmemECol = 256;        // metadata columns start after the accumulator
 constexpr uint32_t kSpinLimit = 1u << 22;  // bounded waits: ~4M polls with back-off
@@ -174,8 +175,14 @@ __device__ __forceinline__ void epilogue_rows(const GemmParams& p, int split, in
                             f[0] += c0.x; f[1] += c0.y; f[2] += c0.z; f[3] += c0.w;
                             f[4] += c1.x; f[5] += c1.y; f[6] += c1.z; f[7] += c1.w;
                         }
-                        *reinterpret_cast<float4*>(dst) = make_float4(f[0], f[1], f[2], f[3]);
-                        *reinterpret_cast<float4*>(dst + 4) = make_float4(f[4], f[5], f[6], f[7]);
+                        if ((reinterpret_cast<uintptr_t>(dst) & 31u) == 0) {     // one full 32-byte sector per store
+                            asm volatile("st.global.v8.f32 [%0], {%1, %2, %3, %4, %5, %6, %7, %8};"
+                                         ::"l"(dst), "f"(f[0]), "f"(f[1]), "f"(f[2]), "f"(f[3]), "f"(f[4]), "f"(f[5]),
+                                           "f"(f[6]), "f"(f[7]) : "memory");
+                        } else {
+                            *reinterpret_cast<float4*>(dst) = make_float4(f[0], f[1], f[2], f[3]);
+                            *reinterpret_cast<float4*>(dst + 4) = make_float4(f[4], f[5], f[6], f[7]);
+                        }
                     }
                 }
             }
@@ -239,9 +246,17 @@ sparse_gemm_pair_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const uint32_t rank = cluster_ctarank();
-    const int64_t m_block = (int64_t)(blockIdx.x >> 1) * 2 + rank;                  // 128-row block of A
+    // Tile order: bands of kBandTiles row tiles, row tile fastest inside a band, so that the pairs running
+    // at the same time cover a compact block of the output and share their A and B tiles in L2.
+    const int64_t tiles_m = (p.M + 2 * BM - 1) / (2 * BM), tiles_n = (p.N + BN - 1) / BN;
+    const int64_t pair_id = blockIdx.x >> 1;
+    const int64_t band = pair_id / (kBandTiles * tiles_n);
+    const int64_t band_h = tiles_m - band * kBandTiles < kBandTiles ? tiles_m - band * kBandTiles : kBandTiles;
+    const int64_t in_band = pair_id - band * kBandTiles * tiles_n;
+    const int64_t tile_m = band * kBandTiles + in_band % band_h, tile_n = in_band / band_h;
+    const int64_t m_block = tile_m * 2 + rank;                                      // 128-row block of A
     const int64_t m0 = m_block * BM;
-    const int64_t n0 = (int64_t)blockIdx.y * BN;                                    // the pair's columns
+    const int64_t n0 = tile_n * BN;                                                 // the pair's columns
     const int split = blockIdx.z;
     const int64_t total_steps = p.K / BK;
     const int64_t step_begin = (int64_t)split * p.k_steps_per_split;
@@ -487,7 +502,7 @@ int launch_sparse_gemm(const SparseGemmArgs& a, cudaStream_t stream) {
     p.scale = reinterpret_cast<const __nv_bfloat16*>(a.scale);
     p.c_is_bf16 = a.c_is_bf16; p.accumulate = a.accumulate; p.splits = splits;
     p.dev_status = a.dev_status;
-    dim3 grid((unsigned)(2 * ((a.M + 2 * BM - 1) / (2 * BM))), (unsigned)((a.N + BN - 1) / BN), (unsigned)splits);
+    dim3 grid((unsigned)(2 * ((a.M + 2 * BM - 1) / (2 * BM)) * ((a.N + BN - 1) / BN)), 1u, (unsigned)splits);
     sparse_gemm_pair_kernel<<<grid, kThreads, kSmemBytes, stream>>>(map_a, map_b, map_e, p);
     cudaError_t e = cudaGetLastError();
     if (e == cudaSuccess && splits > 1) {
