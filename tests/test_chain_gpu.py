@@ -1,0 +1,47 @@
+"""The MLP-stack chain (prune along out -> sparse backward product with f'(z) -> prune along tokens -> sparse
+update product, layer after layer) against the same chain run with the oracle."""
+import numpy as np
+import pytest
+import torch
+
+import oracle
+from paper_2203_10991_b200 import chain, workloads
+
+pytestmark = pytest.mark.gpu
+
+
+def to_dev(a):
+    return torch.from_numpy(a.view(np.int16)).cuda().view(torch.bfloat16)
+
+
+def test_three_layer_chain_matches_oracle_chain():
+    T, dims = 512, [256, 384, 128, 256]          # layer i maps dims[i+1] <- dims[i] going up; we walk down
+    rng_seed = 5
+    layers_np = []
+    for i in range(3):                           # top layer first: out = dims[3-i], in = dims[2-i]
+        out_f, in_f = dims[3 - i], dims[2 - i]
+        layers_np.append({"W": workloads.normal_bf16((out_f, in_f), seed=10 + i, std=in_f ** -0.5),
+                          "h": workloads.normal_bf16((T, in_f), seed=20 + i),
+                          "act_grad": workloads.normal_bf16((T, in_f), seed=30 + i) if i < 2 else None})
+    g_top = workloads.gradient((T, dims[3]), "student_t", seed=rng_seed, dtype="bf16")
+
+    layers_dev = [{k: (None if v is None else to_dev(v)) for k, v in L.items()} for L in layers_np]
+    grads = chain.backward_update(to_dev(g_top), layers_dev, base_seed=3)
+    torch.cuda.synchronize()
+
+    # oracle chain; the propagated gradient is rounded to bf16 exactly where the GPU chain stores it
+    g = g_top
+    th = oracle.host_threads()
+    for i, L in enumerate(layers_np):
+        s_upd, s_bwd = chain.layer_seeds(3, i)
+        v, mt = oracle.prune(g, 2, 4, axis=0, seed=s_upd, threads=th)
+        want = oracle.gemm(oracle.unpack(v, mt), L["h"], threads=th)
+        got = grads[i].double().cpu().numpy()
+        err = np.linalg.norm(got - want) / np.linalg.norm(want)
+        # layer 0 sees identical inputs; lower layers inherit bf16 roundings of g that may differ by one ulp
+        # where the fp32 and fp64 sums straddle a rounding boundary
+        assert err <= (2e-5 if i == 0 else 1e-2), (i, err)
+        if L["act_grad"] is not None:
+            v, mt = oracle.prune(g, 2, 4, axis=1, seed=s_bwd, threads=th)
+            dh = oracle.gemm(oracle.unpack(v, mt), L["W"], L["act_grad"], threads=th)
+            g = workloads.to_bf16_bits(dh.astype(np.float32))
