@@ -7,10 +7,15 @@
 //           bytes of bf16 (64 of fp32); a warp reads 1 KiB (2 KiB) contiguous.
 //   axis 0 (K runs down the rows of g): one thread owns a strip of 16 rows by
 //           16 bytes of columns; a warp reads 512 contiguous bytes per row.
+#include <cuda.h>
 #include <cuda_runtime.h>
+
+#include <cstring>
+#include <mutex>
 
 #include "mvue_device.cuh"
 #include "mvue_internal.h"
+#include "mvue_tma.h"
 
 namespace mvue {
 namespace {
@@ -183,13 +188,30 @@ constexpr int kTileStrips = 16;
 constexpr int kTileCols = 64;
 constexpr int kMetaPitch = 36;                       // bytes per staged metadata row
 
-template <int M, bool kBf16, bool kTC>
+constexpr int kTileInBytes = kTileStrips * 16 * kTileCols * 2;   // the bf16 input tile: 256 rows x 128 bytes
+
+__device__ __forceinline__ uint32_t smem_addr(const void* p) {
+    return static_cast<uint32_t>(__cvta_generic_to_shared(p));
+}
+
+// Plain-load path of one lane's strip (16 rows x 2 bf16 columns) into the shared tile; kept out of line so
+// that the TMA-fed kernel carries none of its address arithmetic.  Used only if the copy failed to land.
+__device__ __noinline__ void fill_strip_bf16(const char* p, int64_t ld, unsigned char* dst, int pitch) {
+#pragma unroll 1
+    for (int i = 0; i < 16; ++i)
+        *reinterpret_cast<uint32_t*>(dst + i * pitch) = __ldg(reinterpret_cast<const uint32_t*>(p + (int64_t)i * ld * 2));
+}
+
+// kTma (bf16 only): the 256 x 64 input tile arrives by one TMA box copy into dynamic shared memory, so
+// the lanes read their words with compile-time offsets and no address arithmetic.
+template <int M, bool kBf16, bool kTC, bool kTma>
 __global__ void __launch_bounds__(kTileStrips * 32, kBf16 ? 3 : 2)
-prune_axis0_kernel(const void* __restrict__ g, int64_t n_strips, int64_t n_cols, int64_t ld,
-                   int64_t units_per_row_total, int64_t unit_offset, RoundKeys rk,
+prune_axis0_kernel(const __grid_constant__ CUtensorMap map_g, const void* __restrict__ g, int64_t n_strips,
+                   int64_t n_cols, int64_t ld, int64_t units_per_row_total, int64_t unit_offset, RoundKeys rk,
                    uint4* __restrict__ values, uint16_t* __restrict__ meta) {
     constexpr int ES = kBf16 ? 2 : 4;
     constexpr int NT = kTileStrips * 32;
+    extern __shared__ __align__(128) unsigned char s_in[];        // kTma: input tile, then one mbarrier
     __shared__ uint4 s_val[kTileCols * kTileStrips];
     __shared__ __align__(16) unsigned char s_meta[kTileCols * kMetaPitch];   // >= 2048 bytes
 
@@ -200,14 +222,39 @@ prune_axis0_kernel(const void* __restrict__ g, int64_t n_strips, int64_t n_cols,
     const int64_t col0 = (int64_t)blockIdx.y * kTileCols;
     const int64_t strip = strip0 + strip_l;
     const int64_t col = col0 + 2 * lane;             // this lane's first column (n_cols is even)
+    const bool tile_has_input = col0 < n_cols;
+    const uint32_t bar = smem_addr(s_in + kTileInBytes);
+    if (kTma && tid == 0 && tile_has_input) {
+        asm volatile("mbarrier.init.shared::cta.b64 [%0], 1;" ::"r"(bar));
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+        asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "r"(kTileInBytes) : "memory");
+        asm volatile(
+            "cp.async.bulk.tensor.2d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3}], [%4];"
+            ::"r"(smem_addr(s_in)), "l"(&map_g), "r"((int)col0), "r"((int)(strip0 * 16)), "r"(bar) : "memory");
+    }
     if (kTC) {                                       // padding rows of A keep a valid pattern
         for (int i = tid; i < 2048 / 4; i += NT) reinterpret_cast<uint32_t*>(s_meta)[i] = 0x44444444u;
-        __syncthreads();
     }
+    if (kTC || kTma) __syncthreads();
 
     if (strip < n_strips && col < n_cols) {
         const char* p = reinterpret_cast<const char*>(g) + ((strip * 16) * ld + col) * ES;
         uint32_t w[16][kBf16 ? 1 : 2];
+        bool landed = false;
+        if (kTma) {                                  // bounded wait; if it ever expired the plain loads below take over
+            for (uint32_t spin = 0; spin < (1u << 20) && !landed; ++spin) {
+                uint32_t ok;
+                asm volatile("{\n\t.reg .pred p;\n\tmbarrier.try_wait.parity.shared::cta.b64 p, [%1], 0;\n\t"
+                             "selp.u32 %0, 1, 0, p;\n\t}" : "=r"(ok) : "r"(bar) : "memory");
+                landed = ok != 0;
+            }
+        }
+        if (kTma) {
+            unsigned char* src = s_in + strip_l * 16 * (kTileCols * 2) + lane * 4;
+            if (!landed) fill_strip_bf16(p, ld, src, kTileCols * 2);
+#pragma unroll
+            for (int i = 0; i < 16; ++i) w[i][0] = *reinterpret_cast<const uint32_t*>(src + i * (kTileCols * 2));
+        } else
 #pragma unroll
         for (int i = 0; i < 16; ++i) {
             if (kBf16) {
@@ -346,7 +393,25 @@ cudaError_t launch_prune_t(const PruneArgs& a, cudaStream_t stream) {
         const int64_t cover_cols = kTC ? ((a.cols + 127) / 128) * 128 : a.cols;
         dim3 grid((unsigned)((n_strips + kTileStrips - 1) / kTileStrips),
                   (unsigned)((cover_cols + kTileCols - 1) / kTileCols));
-        prune_axis0_kernel<M, kBf16, kTC><<<grid, kTileStrips * 32, 0, stream>>>(a.g, n_strips, a.cols, a.ld, upr_total, uoff, rk, values, meta);
+        CUtensorMap map_g;
+        memset(&map_g, 0, sizeof(map_g));
+        if (kBf16) {
+            if (!make_map_2d(&map_g, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, a.g, (uint64_t)a.cols, (uint64_t)a.rows,
+                             (uint64_t)a.ld * 2, kTileCols, kTileStrips * 16, CU_TENSOR_MAP_SWIZZLE_NONE))
+                return cudaErrorInvalidValue;
+            static std::once_flag once;
+            static cudaError_t attr_err = cudaSuccess;
+            std::call_once(once, [] {
+                attr_err = cudaFuncSetAttribute(prune_axis0_kernel<M, true, kTC, true>,
+                                                cudaFuncAttributeMaxDynamicSharedMemorySize, kTileInBytes + 16);
+            });
+            if (attr_err != cudaSuccess) return attr_err;
+            prune_axis0_kernel<M, true, kTC, true><<<grid, kTileStrips * 32, kTileInBytes + 16, stream>>>(
+                map_g, a.g, n_strips, a.cols, a.ld, upr_total, uoff, rk, values, meta);
+        } else {
+            prune_axis0_kernel<M, false, kTC, false><<<grid, kTileStrips * 32, 0, stream>>>(
+                map_g, a.g, n_strips, a.cols, a.ld, upr_total, uoff, rk, values, meta);
+        }
     }
     return cudaGetLastError();
 }
