@@ -156,8 +156,26 @@ MVUE_API int mvue_sparse_backward_gemm(const void* values, const void* meta, int
                               void* workspace, size_t workspace_bytes, int* dev_status,
                               void* stream);
 
+/* Prune fused into the update product (Sec. 4.1 / 4.2 + App. A.2 applied to g along the
+ * token axis, then the update equation of Sec. 1) in ONE kernel:
+ *   dW[out x in] (+)= theta(g)^T h,   g bf16 [T x out] (ld ldg), h bf16 [T x in]
+ * g is read from memory once and the packed operand is never written.  The random words
+ * are those of mvue_prune(g, n, m, axis 0, seed), so the result equals mvue_prune followed by
+ * mvue_sparse_update_gemm with the same seed (up to fp32 summation order across K splits).
+ * Every 128 x 256 output tile re-prunes its rows of g: the prune work grows with in / 256,
+ * and the prune is bound by instruction issue, so for wide layers the separate calls are
+ * faster; this entry point pays off only for in <= 256 or when memory for the packed
+ * operand is not available.
+ * dtype must be MVUE_BF16 (else MVUE_ERR_DTYPE).  workspace: mvue_gemm_workspace_bytes(2, out,
+ * in, T) bytes.  Other arguments, preconditions and errors as mvue_sparse_update_gemm. */
+MVUE_API int mvue_fused_update_gemm(const void* g, int dtype, int64_t T, int64_t out, int64_t ldg, int n,
+                                    int m, uint64_t seed, const void* h, int64_t in, int64_t ldh,
+                                    void* dW, int dW_dtype, int64_t lddW, int accumulate,
+                                    void* workspace, size_t workspace_bytes, int* dev_status,
+                                    void* stream);
+
 /* Scratch bytes the product C[M x N] = A[M x K] . B[K x N] needs
- * (which: 0 update, 1 backward).  bytes is a HOST pointer. */
+ * (which: 0 update, 1 backward, 2 fused update).  bytes is a HOST pointer. */
 MVUE_API int mvue_gemm_workspace_bytes(int which, int64_t M, int64_t N, int64_t K, size_t* bytes);
 
 /* The update product for callers that cannot allocate device memory.

@@ -20,7 +20,7 @@ MVUE_LAYOUT_TC = 1
 
 EXPORTS = ("mvue_version", "mvue_status_string", "mvue_last_cuda_error", "mvue_packed_sizes",
            "mvue_prune", "mvue_unpack", "mvue_sparse_update_gemm", "mvue_sparse_backward_gemm",
-           "mvue_gemm_workspace_bytes", "mvue_sparse_update_gemm_noalloc")
+           "mvue_gemm_workspace_bytes", "mvue_sparse_update_gemm_noalloc", "mvue_fused_update_gemm")
 
 
 class MvueError(RuntimeError):
@@ -54,6 +54,8 @@ def lib() -> ctypes.CDLL:
         L.mvue_sparse_backward_gemm.argtypes = [vp, vp, ci, i64, i64, vp, i64, i64, vp, vp, ci, i64, vp,
                                                 ctypes.c_size_t, vp, vp]
         L.mvue_gemm_workspace_bytes.argtypes = [ci, i64, i64, i64, szp]
+        L.mvue_fused_update_gemm.argtypes = [vp, ci, i64, i64, i64, ci, ci, u64, vp, i64, i64, vp, ci, i64, ci, vp,
+                                             ctypes.c_size_t, vp, vp]
         L.mvue_sparse_update_gemm_noalloc.argtypes = [vp, vp, ci, i64, i64, vp, i64, i64, vp, ci, i64, ci, vp, vp]
         _lib = L
     return _lib
@@ -181,4 +183,23 @@ def mvue_sparse_update_gemm_noalloc(values: torch.Tensor, meta: torch.Tensor, h:
                                                  int(accumulate),
                                                  None if dev_status is None else dev_status.data_ptr(),
                                                  _stream_ptr()), "mvue_sparse_update_gemm_noalloc")
+    return out
+
+
+def mvue_fused_update_gemm(g: torch.Tensor, h: torch.Tensor, n: int, m: int, seed: int, *,
+                           out: torch.Tensor | None = None, out_dtype=torch.float32, accumulate: bool = False,
+                           workspace: torch.Tensor | None = None,
+                           dev_status: torch.Tensor | None = None) -> torch.Tensor:
+    """dW[out, in] (+)= theta(g)^T . h in one kernel: g bf16 [T, out] is pruned along the tokens on the fly."""
+    T, n_out = g.shape
+    T2, n_in = h.shape
+    assert T == T2 and g.stride(1) == 1 and h.stride(1) == 1
+    if out is None:
+        out = torch.empty((n_out, n_in), dtype=out_dtype, device=h.device)
+    ws, ws_bytes = _workspace(2, n_out, n_in, T, h.device, workspace)
+    _check(lib().mvue_fused_update_gemm(g.data_ptr(), _dtype_code(g), T, n_out, g.stride(0), n, m, seed & (2**64 - 1),
+                                        h.data_ptr(), n_in, h.stride(0), out.data_ptr(), _dtype_code(out),
+                                        out.stride(0), int(accumulate), None if ws is None else ws.data_ptr(), ws_bytes,
+                                        None if dev_status is None else dev_status.data_ptr(), _stream_ptr()),
+           "mvue_fused_update_gemm")
     return out

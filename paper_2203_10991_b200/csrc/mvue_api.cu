@@ -149,11 +149,11 @@ int mvue_unpack(const void* values, const void* meta, int layout, int64_t mrows,
 
 int mvue_gemm_workspace_bytes(int which, int64_t M, int64_t N, int64_t K, size_t* bytes) {
     if (!bytes) return MVUE_ERR_NULL;
-    if (which != 0 && which != 1) return MVUE_ERR_SHAPE;
+    if (which != 0 && which != 1 && which != 2) return MVUE_ERR_SHAPE;
     if (M <= 0 || N <= 0 || K <= 0 || K % 128 != 0) return MVUE_ERR_SHAPE;
     DeviceInfo dev;
     if (int s = current_device_info(&dev)) return s;
-    *bytes = gemm_workspace_bytes(M, N, K, dev.sm_count);
+    *bytes = which == 2 ? fused_workspace_bytes(M, N, K, dev.sm_count) : gemm_workspace_bytes(M, N, K, dev.sm_count);
     return MVUE_OK;
 }
 
@@ -171,6 +171,32 @@ int mvue_sparse_backward_gemm(const void* values, const void* meta, int layout, 
                               int* dev_status, void* stream) {
     return run_gemm(values, meta, layout, T, in, out, W, ldW, act_grad, dh, dh_dtype, lddh, 0, workspace,
                     workspace_bytes, dev_status, stream);
+}
+
+int mvue_fused_update_gemm(const void* g, int dtype, int64_t T, int64_t out, int64_t ldg, int n, int m,
+                           uint64_t seed, const void* h, int64_t in, int64_t ldh, void* dW, int dW_dtype,
+                           int64_t lddW, int accumulate, void* workspace, size_t workspace_bytes,
+                           int* dev_status, void* stream) {
+    if (!g || !h || !dW) return MVUE_ERR_NULL;
+    if (int s = check_nm(n, m)) return s;
+    if (dtype != MVUE_BF16) return MVUE_ERR_DTYPE;                 // the fused path takes bf16 gradients only
+    if (dW_dtype != MVUE_F32 && dW_dtype != MVUE_BF16) return MVUE_ERR_DTYPE;
+    if (accumulate && dW_dtype != MVUE_F32) return MVUE_ERR_DTYPE;
+    if (T <= 0 || out <= 0 || in <= 0 || T % 128 != 0 || out % 8 != 0 || in % 8 != 0) return MVUE_ERR_SHAPE;
+    if (ldg < out || ldh < in || lddW < in) return MVUE_ERR_SHAPE;
+    if (T > 0x7FFFFFFF || out > 0x7FFFFFFF || in > 0x7FFFFFFF) return MVUE_ERR_SHAPE;
+    const int64_t c_esz = dW_dtype == MVUE_BF16 ? 2 : 4;
+    if (!aligned16(g) || !aligned16(h) || !aligned16(dW) || (ldg * 2) % 16 != 0 || (ldh * 2) % 16 != 0 ||
+        (lddW * c_esz) % 16 != 0)
+        return MVUE_ERR_ALIGN;
+    DeviceInfo dev;
+    if (int s = current_device_info(&dev)) return s;
+    const size_t need = fused_workspace_bytes(out, in, T, dev.sm_count);
+    if (need > 0 && (!workspace || workspace_bytes < need || !aligned16(workspace))) return MVUE_ERR_WORKSPACE;
+    FusedArgs f{g, ldg, m, seed,
+                SparseGemmArgs{nullptr, nullptr, out, in, T, h, ldh, dW, lddW, dW_dtype == MVUE_BF16, accumulate,
+                               nullptr, workspace, dev_status, dev.sm_count}};
+    return launch_fused_update(f, reinterpret_cast<cudaStream_t>(stream));
 }
 
 int mvue_sparse_update_gemm_noalloc(const void* values, const void* meta, int layout, int64_t out, int64_t T,

@@ -217,4 +217,35 @@ __device__ __forceinline__ void mvue_2of4_f32(uint32_t b0, uint32_t b1, uint32_t
     *nibble = swap ? (ib | (ia << 2)) : (ia | (ib << 2));
 }
 
+// One work unit of bf16 input: raw[8] = 16 elements along K, two per word.
+template <int M>
+__device__ __forceinline__ void prune_unit_bf16(const uint32_t (&raw)[8], uint64_t unit_index,
+                                                const RoundKeys& rk, uint4* out_values,
+                                                uint32_t* out_meta) {
+    uint32_t v[4];                                   // 8 survivors, two bf16 per word
+    uint32_t meta = 0;
+    if (M == 4) {
+        const uint4 w = philox4x32_10(unit_index, rk);
+        const uint32_t words[4] = {w.x, w.y, w.z, w.w};
+#pragma unroll
+        for (int j = 0; j < 4; ++j) {
+            uint32_t nib;
+            mvue_2of4_bf16(raw[2 * j], raw[2 * j + 1], words[j], &v[j], &nib);
+            meta += nib << (4 * j);
+        }
+    } else {
+        const uint4 wa = philox4x32_10(2 * unit_index, rk);
+        const uint4 wb = philox4x32_10(2 * unit_index + 1, rk);
+        const uint32_t words[8] = {wa.x, wa.y, wa.z, wa.w, wb.x, wb.y, wb.z, wb.w};
+#pragma unroll
+        for (int j = 0; j < 4; ++j) {
+            uint32_t nib;
+            mvue_1of2x2_bf16(raw[2 * j], raw[2 * j + 1], words[2 * j], words[2 * j + 1], &v[j], &nib);
+            meta += nib << (4 * j);
+        }
+    }
+    *out_values = make_uint4(v[0], v[1], v[2], v[3]);
+    *out_meta = meta;
+}
+
 }  // namespace mvue

@@ -29,6 +29,7 @@
 #include <mutex>
 
 #include "../../include/mvue.h"
+#include "mvue_device.cuh"
 #include "mvue_internal.h"
 #include "mvue_tma.h"
 
@@ -190,6 +191,38 @@ __device__ __forceinline__ void epilogue_rows(const GemmParams& p, int split, in
     }
 }
 
+__device__ __forceinline__ void mbar_arrive(uint32_t bar) {
+    asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(bar) : "memory");
+}
+__device__ __forceinline__ void tma_load_2d(uint32_t dst, const CUtensorMap* map, int x, int y, uint32_t bar) {
+    asm volatile(
+        "cp.async.bulk.tensor.2d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3}], [%4];"
+        ::"r"(dst), "l"(map), "r"(x), "r"(y), "r"(bar) : "memory");
+}
+__device__ __forceinline__ void tmem_alloc(uint32_t dst_smem, uint32_t cols) {
+    asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(dst_smem), "r"(cols) : "memory");
+}
+__device__ __forceinline__ void tmem_relinquish() {
+    asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+}
+__device__ __forceinline__ void tmem_dealloc(uint32_t addr, uint32_t cols) {
+    asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(addr), "r"(cols) : "memory");
+}
+__device__ __forceinline__ void tc_commit(uint32_t bar) {
+    asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(bar) : "memory");
+}
+__device__ __forceinline__ void tc_copy_128x128b(uint32_t tmem_addr, uint64_t smem_desc) {
+    asm volatile("tcgen05.cp.cta_group::1.128x128b [%0], %1;" ::"r"(tmem_addr), "l"(smem_desc) : "memory");
+}
+__device__ __forceinline__ void tc_mma_sp_bf16(uint32_t tmem_d, uint64_t a_desc, uint64_t b_desc,
+                                               uint32_t tmem_meta, uint32_t idesc, uint32_t accumulate) {
+    const uint32_t zero = 0u;                 // no output lane is disabled
+    asm volatile(
+        "{\n\t.reg .pred p;\n\t"
+        "setp.ne.b32 p, %5, 0;\n\t"
+        "tcgen05.mma.sp.cta_group::1.kind::f16 [%0], %1, %2, [%3], %4, {%6, %6, %6, %6}, p;\n\t}"
+        ::"r"(tmem_d), "l"(a_desc), "l"(b_desc), "r"(tmem_meta), "r"(idesc), "r"(accumulate), "r"(zero) : "memory");
+}
 __device__ __forceinline__ uint32_t cluster_ctarank() {
     uint32_t r;
     asm volatile("mov.u32 %0, %%cluster_ctarank;" : "=r"(r));
@@ -368,6 +401,191 @@ sparse_gemm_pair_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_
     }
 }
 
+// =============================================================================
+// Prune fused into the update product: dW[out x in] = theta(g)^T h with g read once and the
+// packed operand never written to memory.  One thread block per 128 x 256 output tile
+// (tcgen05.mma.sp.cta_group::1, M = 128), two stages of K = 128:
+//   warp 0      TMA producer of the B tile only (four 64-column boxes of h)
+//   warp 1      tcgen05.cp of the stage's metadata, four MMAs, commit
+//   warp 2      tensor-memory allocation
+//   warps 4-7   epilogue
+//   warps 8-15  prune: warp w owns the 16-token strip w of the stage, lane l the four columns
+//               4l..4l+3 of g (= rows of A); each (column, strip) is one prune unit and yields 8
+//               survivors -- one 16-byte chunk of the A tile, written at its 128-byte-swizzled
+//               place -- and one 16-bit metadata word, written at its tensor-core lane / word.
+// The random words are those of mvue_prune for the same seed (block number over the whole
+// operand), so the result equals mvue_prune followed by mvue_sparse_update_gemm.
+// Every block that shares a row tile re-prunes it: the prune work grows with in / 256.
+// =============================================================================
+constexpr int kFStages = 2;
+constexpr int kFBBytes = (BN / 64) * kBBoxBytes;                 // 64 KiB: all 256 columns
+constexpr int kFStageBytes = kABytes + kFBBytes + kEBytes;       // 82 KiB
+constexpr int kFSmemBytes = kFStages * kFStageBytes + 1024 + 256;
+constexpr int kFThreads = 512;
+constexpr int kFPruneWarps = 8;
+constexpr uint32_t kInstrDesc1 = (1u << 2) | (1u << 4) | (1u << 7) | (1u << 10) | (0u << 15) | (1u << 16) |
+                                 ((uint32_t)(BN >> 3) << 17) | ((uint32_t)(BM >> 4) << 24);
+
+struct FusedParams {
+    const uint32_t* g;        // bf16 [T x out], two elements per word
+    int64_t ldg_words;        // leading dimension of g in 32-bit words
+    RoundKeys rk;
+    GemmParams gemm;          // M = out, N = in, K = T
+};
+
+template <int NM>
+__global__ void __launch_bounds__(kFThreads, 1)
+fused_update_kernel(const __grid_constant__ CUtensorMap map_b, const FusedParams fp) {
+    const GemmParams& p = fp.gemm;
+    extern __shared__ uint8_t smem_raw[];
+    const uint32_t smem_base = (smem_u32(smem_raw) + 1023u) & ~1023u;
+    uint8_t* smem_gen = smem_raw + (smem_base - smem_u32(smem_raw));
+    const uint32_t bar_base = smem_base + kFStages * kFStageBytes;
+    auto full_bar = [&](int s) { return bar_base + 8u * s; };
+    auto empty_bar = [&](int s) { return bar_base + 8u * (kFStages + s); };
+    const uint32_t acc_bar = bar_base + 8u * (2 * kFStages);
+    uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(smem_gen + kFStages * kFStageBytes + 8 * (2 * kFStages + 1));
+    volatile int* abort_flag = reinterpret_cast<volatile int*>(tmem_slot + 1);
+
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const int64_t m0 = (int64_t)blockIdx.y * BM;
+    const int64_t n0 = (int64_t)blockIdx.x * BN;
+    const int split = blockIdx.z;
+    const int64_t total_steps = p.K / BK;
+    const int64_t step_begin = (int64_t)split * p.k_steps_per_split;
+    int64_t step_end = step_begin + p.k_steps_per_split;
+    if (step_end > total_steps) step_end = total_steps;
+    const int64_t n_steps = step_end > step_begin ? step_end - step_begin : 0;
+
+    if (threadIdx.x == 0) {
+        for (int s = 0; s < kFStages; ++s) {
+            mbar_init(full_bar(s), 1 + kFPruneWarps);   // B bytes + one arrival per prune warp
+            mbar_init(empty_bar(s), 1);
+        }
+        mbar_init(acc_bar, 1);
+        *abort_flag = 0;
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    }
+    if (warp == 2) {
+        tmem_alloc(smem_u32(tmem_slot), kTmemCols);
+        tmem_relinquish();
+    }
+    tc_fence_before();
+    __syncthreads();
+    tc_fence_after();
+    const uint32_t tmem_base = *tmem_slot;
+
+    if (warp == 0) {
+        if (lane == 0) {
+            for (int64_t i = 0; i < n_steps; ++i) {
+                const int s = (int)(i % kFStages);
+                const uint32_t use = (uint32_t)(i / kFStages);
+                if (use > 0 && !mbar_wait(empty_bar(s), (use - 1) & 1u, abort_flag)) break;
+                const uint32_t b_dst = smem_base + s * kFStageBytes + kABytes;
+                const int k = (int)((step_begin + i) * BK);
+                mbar_expect_tx(full_bar(s), kFBBytes);
+#pragma unroll
+                for (int j = 0; j < BN / 64; ++j)
+                    tma_load_2d(b_dst + j * kBBoxBytes, &map_b, (int)n0 + 64 * j, k, full_bar(s));
+            }
+        }
+    } else if (warp == 1) {
+        if (lane == 0) {
+            bool ok = true;
+            for (int64_t i = 0; i < n_steps && ok; ++i) {
+                const int s = (int)(i % kFStages);
+                const uint32_t use = (uint32_t)(i / kFStages);
+                ok = mbar_wait(full_bar(s), use & 1u, abort_flag);
+                if (!ok) break;
+                tc_fence_after();
+                const uint32_t a_addr = smem_base + s * kFStageBytes;
+                const uint32_t b_addr = a_addr + kABytes;
+                const uint32_t e_addr = b_addr + kFBBytes;
+                const uint32_t tmem_e = tmem_base + kTmemECol + 4u * s;
+                tc_copy_128x128b(tmem_e, make_smem_desc(e_addr, 16, 128, kSwizzleNone));
+#pragma unroll
+                for (int kb = 0; kb < BK / 32; ++kb) {
+                    const uint64_t a_desc = make_smem_desc(a_addr + kb * 32, 16, 1024, kSwizzle128B);
+                    const uint64_t b_desc = make_smem_desc(b_addr + kb * 4096, kBBoxBytes, 1024, kSwizzle128B);
+                    tc_mma_sp_bf16(tmem_base, a_desc, b_desc, tmem_e + (uint32_t)(kb & ~1),
+                                   kInstrDesc1 | (uint32_t)(kb & 1), (i > 0 || kb > 0) ? 1u : 0u);
+                }
+                tc_commit(empty_bar(s));
+            }
+            tc_commit(acc_bar);
+        }
+    } else if (warp >= 4 && warp < 8) {
+        const int q = warp - 4;
+        const bool acc_ok = n_steps > 0 ? mbar_wait(acc_bar, 0, abort_flag) : true;
+        tc_fence_after();
+        const int64_t row = m0 + 32 * q + lane;
+        if (acc_ok) epilogue_rows(p, split, row, n0, tmem_base + ((uint32_t)(32 * q) << 16), n_steps > 0);
+    } else if (warp >= 8) {
+        // ------------------------------------------------------------ prune warps
+        const int strip_l = warp - 8;                               // 16-token strip of the stage
+        const int64_t col = m0 + 4 * lane;                          // first of this lane's four columns of g
+        const bool cols_exist = col < p.M;                          // out is a multiple of 8: all four or none
+        const int64_t units_per_row = p.K / 16;
+        bool ok = true;
+        for (int64_t i = 0; i < n_steps && ok; ++i) {
+            const int s = (int)(i % kFStages);
+            const uint32_t use = (uint32_t)(i / kFStages);
+            const int64_t k0 = (step_begin + i) * BK + 16 * strip_l;        // first token of the strip
+            uint2 w[16];
+            if (cols_exist) {
+                const uint32_t* src = fp.g + k0 * fp.ldg_words + (col >> 1);
+#pragma unroll
+                for (int r = 0; r < 16; ++r) w[r] = __ldg(reinterpret_cast<const uint2*>(src + r * fp.ldg_words));
+            }
+            if (use > 0) ok = mbar_wait(empty_bar(s), (use - 1) & 1u, abort_flag);
+            if (!ok) break;
+            uint8_t* a_tile = smem_gen + s * kFStageBytes;
+            uint8_t* e_tile = a_tile + kABytes + kFBBytes;
+#pragma unroll
+            for (int e = 0; e < 4; ++e) {
+                const int m_l = 4 * lane + e;                              // row of the A tile
+                uint4 v = make_uint4(0u, 0u, 0u, 0u);
+                uint32_t mt = 0x4444u;
+                if (cols_exist) {
+                    uint32_t raw[8];
+#pragma unroll
+                    for (int j = 0; j < 8; ++j) {
+                        const uint32_t lo = (e < 2) ? w[2 * j].x : w[2 * j].y;
+                        const uint32_t hi = (e < 2) ? w[2 * j + 1].x : w[2 * j + 1].y;
+                        raw[j] = __byte_perm(lo, hi, (e & 1) ? 0x7632 : 0x5410);
+                    }
+                    const uint64_t unit = (uint64_t)(col + e) * (uint64_t)units_per_row + (uint64_t)(k0 >> 4);
+                    prune_unit_bf16<NM>(raw, unit, fp.rk, &v, &mt);
+                }
+                // A tile: row m_l is 128 bytes; the strip's 8 survivors are chunk strip_l, swizzled by the row
+                *reinterpret_cast<uint4*>(a_tile + m_l * 128 + ((strip_l ^ (m_l & 7)) << 4)) = v;
+                // metadata: lane / word / half-word of the tensor-core order
+                const int tc_lane = (m_l & 7) + 8 * (strip_l & 1) + 16 * (m_l >> 4);
+                *reinterpret_cast<uint16_t*>(e_tile + tc_lane * 16 + (strip_l >> 1) * 4 + ((m_l >> 3) & 1) * 2) = (uint16_t)mt;
+            }
+            asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+            __syncwarp();
+            if (lane == 0) mbar_arrive(full_bar(s));
+        }
+    }
+
+    tc_fence_before();
+    __syncthreads();
+    if (*abort_flag) {
+        if (threadIdx.x == 0) {
+            for (int s = 0; s < kFStages; ++s)
+                for (uint32_t spin = 0; spin < 4096 && !mbar_try_wait(full_bar(s), 0) && !mbar_try_wait(full_bar(s), 1); ++spin)
+                    __nanosleep(64);
+            if (p.dev_status) *p.dev_status = MVUE_ERR_DEVICE_TIMEOUT;
+        }
+        __syncthreads();
+    }
+    if (warp == 2) {
+        tc_fence_after();
+        tmem_dealloc(tmem_base, kTmemCols);
+    }
+}
+
 // Second pass of split-K: sums the partial tiles in a fixed order (deterministic) and applies the
 // same epilogue as the single-pass path.
 __global__ void __launch_bounds__(256)
@@ -443,6 +661,71 @@ int static_scratch(void** ptr, size_t* bytes) {
     }
     *ptr = addr[dev];
     *bytes = kStaticScratchBytes;
+    return MVUE_OK;
+}
+
+int fused_split_count(int64_t M, int64_t N, int64_t K, int sm_count) {
+    const int64_t blocks = ((M + BM - 1) / BM) * ((N + BN - 1) / BN);
+    const int64_t steps = K / BK;
+    if (blocks >= sm_count || steps < 8) return 1;
+    int64_t splits = sm_count / blocks;
+    if (splits > steps / 4) splits = steps / 4;
+    if (splits > 64) splits = 64;
+    return (int)(splits < 1 ? 1 : splits);
+}
+
+size_t fused_workspace_bytes(int64_t M, int64_t N, int64_t K, int sm_count) {
+    const int splits = fused_split_count(M, N, K, sm_count);
+    return splits > 1 ? (size_t)splits * (size_t)M * (size_t)N * sizeof(float) : 0;
+}
+
+int launch_fused_update(const FusedArgs& f, cudaStream_t stream) {
+    const SparseGemmArgs& a = f.gemm;
+    CUtensorMap map_b;
+    if (!make_map_2d(&map_b, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, a.B, (uint64_t)a.N, (uint64_t)a.K,
+                     (uint64_t)a.ldb * 2, 64, BK, CU_TENSOR_MAP_SWIZZLE_128B)) {
+        set_cuda_error(cudaErrorUnknown, "cuTensorMapEncodeTiled");
+        return MVUE_ERR_CUDA;
+    }
+    static std::once_flag once;
+    static cudaError_t attr_err = cudaSuccess;
+    std::call_once(once, [] {
+        attr_err = cudaFuncSetAttribute(fused_update_kernel<4>, cudaFuncAttributeMaxDynamicSharedMemorySize, kFSmemBytes);
+        if (attr_err == cudaSuccess)
+            attr_err = cudaFuncSetAttribute(fused_update_kernel<2>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                            kFSmemBytes);
+    });
+    if (attr_err != cudaSuccess) { set_cuda_error(attr_err, "cudaFuncSetAttribute"); return MVUE_ERR_CUDA; }
+
+    const int splits = fused_split_count(a.M, a.N, a.K, a.sm_count);
+    const int64_t steps = a.K / BK;
+    FusedParams fp;
+    fp.g = reinterpret_cast<const uint32_t*>(f.g);
+    fp.ldg_words = f.ldg / 2;
+    fp.rk = make_round_keys(f.seed);
+    GemmParams& p = fp.gemm;
+    p.M = a.M; p.N = a.N; p.K = a.K;
+    p.k_steps_per_split = (steps + splits - 1) / splits;
+    p.partial = reinterpret_cast<float*>(a.workspace);
+    p.C = a.C; p.ldc = a.ldc;
+    p.scale = nullptr;
+    p.c_is_bf16 = a.c_is_bf16; p.accumulate = a.accumulate; p.splits = splits;
+    p.dev_status = a.dev_status;
+    dim3 grid((unsigned)((a.N + BN - 1) / BN), (unsigned)((a.M + BM - 1) / BM), (unsigned)splits);
+    if (f.m == 4)
+        fused_update_kernel<4><<<grid, kFThreads, kFSmemBytes, stream>>>(map_b, fp);
+    else
+        fused_update_kernel<2><<<grid, kFThreads, kFSmemBytes, stream>>>(map_b, fp);
+    cudaError_t e = cudaGetLastError();
+    if (e == cudaSuccess && splits > 1) {
+        const int64_t total = a.M * (a.N / 4);
+        const int64_t want = (total + 255) / 256;
+        const int blocks = (int)(want < (int64_t)a.sm_count * 8 ? want : (int64_t)a.sm_count * 8);
+        splitk_reduce_kernel<<<blocks, 256, 0, stream>>>(p.partial, splits, a.M, a.N, a.C, a.ldc, nullptr,
+                                                         a.c_is_bf16, a.accumulate);
+        e = cudaGetLastError();
+    }
+    if (e != cudaSuccess) { set_cuda_error(e, "fused update launch"); return MVUE_ERR_CUDA; }
     return MVUE_OK;
 }
 

@@ -44,6 +44,16 @@ int launch_sparse_gemm(const SparseGemmArgs& a, cudaStream_t stream);     // ret
 int gemm_split_count(int64_t M, int64_t N, int64_t K, int sm_count);
 size_t gemm_workspace_bytes(int64_t M, int64_t N, int64_t K, int sm_count);
 
+struct FusedArgs {
+    const void* g;        // dense bf16 gradient [T x out]
+    int64_t ldg;          // leading dimension in elements
+    int m;                // 2 or 4
+    uint64_t seed;
+    SparseGemmArgs gemm;  // M = out, N = in, K = T; values / meta unused
+};
+int launch_fused_update(const FusedArgs& f, cudaStream_t stream);         // returns an mvue_status
+size_t fused_workspace_bytes(int64_t M, int64_t N, int64_t K, int sm_count);
+
 // Split-K scratch that the library itself carries (see mvue_sparse_update_gemm_noalloc).
 constexpr size_t kStaticScratchBytes = 8u << 20;
 int static_scratch(void** ptr, size_t* bytes);   // returns an mvue_status; device address for the current device
