@@ -102,6 +102,26 @@ __device__ __forceinline__ void mvue_1of2x2_bf16(uint32_t x0, uint32_t x1, uint3
     *nibble = (keepA ? 0u : 1u) | (keepB ? 8u : 12u);
 }
 
+// The same for a group whose four elements are the half kHigh of four row words (K runs down the rows).
+template <bool kHigh>
+__device__ __forceinline__ void mvue_1of2x2_bf16_rows(uint32_t w0, uint32_t w1, uint32_t w2, uint32_t w3,
+                                                      uint32_t word0, uint32_t word1, uint32_t* out,
+                                                      uint32_t* nibble) {
+    auto widen = [](uint32_t w) { return __uint_as_float(kHigh ? (w & 0xFFFF0000u) : (w << 16)); };
+    const float a0 = widen(w0), a1 = widen(w1), b0 = widen(w2), b1 = widen(w3);
+    const float SA = __fadd_rn(fabsf(a0), fabsf(a1));
+    const float SB = __fadd_rn(fabsf(b0), fabsf(b1));
+    const float tA = __fmul_rn(top24(word0), __fmul_rn(SA, 5.9604644775390625e-08f));
+    const float tB = __fmul_rn(top24(word1), __fmul_rn(SB, 5.9604644775390625e-08f));
+    const bool keepA = (tA < fabsf(a0)) || (fabsf(a1) == 0.0f);
+    const bool keepB = (tB < fabsf(b0)) || (fabsf(b1) == 0.0f);
+    const uint32_t srcA = keepA ? w0 : w1, srcB = keepB ? w2 : w3;
+    // byte 1 <- high byte of pair 0's survivor, byte 3 <- high byte of pair 1's survivor
+    const uint32_t signs = __byte_perm(srcA, srcB, kHigh ? 0x7030u : 0x5010u) & 0x80008000u;
+    *out = pack_bf16x2(SA, SB) | signs;
+    *nibble = (keepA ? 0u : 1u) | (keepB ? 8u : 12u);
+}
+
 // ===========================================================================
 // MVUE 2:4 (marginals: Sec. 4.2; joint law over pairs: App. A.2).
 //
@@ -165,12 +185,15 @@ __device__ __forceinline__ Pick24<KeyT> pick_2of4(KeyT k1, KeyT k2, KeyT k3, Key
 // survivors' keys still carry position and sign, so nothing is looked up again.
 // Outputs: `out` = the two survivors as bf16 (lower position in the low half),
 // `nibble` = idx0 | idx1 << 2.
-__device__ __forceinline__ void mvue_2of4_bf16(uint32_t x01, uint32_t x23, uint32_t word,
+// The four elements are the halves (kH* = false: low, true: high) of the words w0..w3: adjacent pairs of two
+// words when K is contiguous (w0 = w1, w2 = w3), or the same half of four row words when K runs down the rows.
+template <bool kH0, bool kH1, bool kH2, bool kH3>
+__device__ __forceinline__ void mvue_2of4_bf16(uint32_t w0, uint32_t w1, uint32_t w2, uint32_t w3, uint32_t word,
                                                uint32_t* out, uint32_t* nibble) {
-    const float f0 = __uint_as_float(__byte_perm(x01, 0x00u, 0x1041));
-    const float f1 = __uint_as_float(__byte_perm(x01, 0x40u, 0x3243));
-    const float f2 = __uint_as_float(__byte_perm(x23, 0x80u, 0x1041));
-    const float f3 = __uint_as_float(__byte_perm(x23, 0xC0u, 0x3243));
+    const float f0 = __uint_as_float(__byte_perm(w0, 0x00u, kH0 ? 0x3243 : 0x1041));
+    const float f1 = __uint_as_float(__byte_perm(w1, 0x40u, kH1 ? 0x3243 : 0x1041));
+    const float f2 = __uint_as_float(__byte_perm(w2, 0x80u, kH2 ? 0x3243 : 0x1041));
+    const float f3 = __uint_as_float(__byte_perm(w3, 0xC0u, kH3 ? 0x3243 : 0x1041));
     const float lo01 = fminf(fabsf(f0), fabsf(f1)), hi01 = fmaxf(fabsf(f0), fabsf(f1));
     const float lo23 = fminf(fabsf(f2), fabsf(f3)), hi23 = fmaxf(fabsf(f2), fabsf(f3));
     const float k1 = fminf(lo01, lo23), mid_a = fmaxf(lo01, lo23);
@@ -230,7 +253,8 @@ __device__ __forceinline__ void prune_unit_bf16(const uint32_t (&raw)[8], uint64
 #pragma unroll
         for (int j = 0; j < 4; ++j) {
             uint32_t nib;
-            mvue_2of4_bf16(raw[2 * j], raw[2 * j + 1], words[j], &v[j], &nib);
+            mvue_2of4_bf16<false, true, false, true>(raw[2 * j], raw[2 * j], raw[2 * j + 1], raw[2 * j + 1], words[j],
+                                                     &v[j], &nib);
             meta += nib << (4 * j);
         }
     } else {
@@ -241,6 +265,38 @@ __device__ __forceinline__ void prune_unit_bf16(const uint32_t (&raw)[8], uint64
         for (int j = 0; j < 4; ++j) {
             uint32_t nib;
             mvue_1of2x2_bf16(raw[2 * j], raw[2 * j + 1], words[2 * j], words[2 * j + 1], &v[j], &nib);
+            meta += nib << (4 * j);
+        }
+    }
+    *out_values = make_uint4(v[0], v[1], v[2], v[3]);
+    *out_meta = meta;
+}
+
+// One work unit whose 16 elements are the half kHigh of 16 row words (K runs down the rows of g).
+template <int M, bool kHigh>
+__device__ __forceinline__ void prune_unit_bf16_rows(const uint32_t (&w)[16], uint64_t unit_index,
+                                                     const RoundKeys& rk, uint4* out_values, uint32_t* out_meta) {
+    uint32_t v[4];
+    uint32_t meta = 0;
+    if (M == 4) {
+        const uint4 r = philox4x32_10(unit_index, rk);
+        const uint32_t words[4] = {r.x, r.y, r.z, r.w};
+#pragma unroll
+        for (int j = 0; j < 4; ++j) {
+            uint32_t nib;
+            mvue_2of4_bf16<kHigh, kHigh, kHigh, kHigh>(w[4 * j], w[4 * j + 1], w[4 * j + 2], w[4 * j + 3], words[j],
+                                                       &v[j], &nib);
+            meta += nib << (4 * j);
+        }
+    } else {
+        const uint4 ra = philox4x32_10(2 * unit_index, rk);
+        const uint4 rb = philox4x32_10(2 * unit_index + 1, rk);
+        const uint32_t words[8] = {ra.x, ra.y, ra.z, ra.w, rb.x, rb.y, rb.z, rb.w};
+#pragma unroll
+        for (int j = 0; j < 4; ++j) {
+            uint32_t nib;
+            mvue_1of2x2_bf16_rows<kHigh>(w[4 * j], w[4 * j + 1], w[4 * j + 2], w[4 * j + 3], words[2 * j],
+                                         words[2 * j + 1], &v[j], &nib);
             meta += nib << (4 * j);
         }
     }

@@ -547,15 +547,12 @@ fused_update_kernel(const __grid_constant__ CUtensorMap map_b, const FusedParams
                 uint4 v = make_uint4(0u, 0u, 0u, 0u);
                 uint32_t mt = 0x4444u;
                 if (cols_exist) {
-                    uint32_t raw[8];
+                    uint32_t rw[16];
 #pragma unroll
-                    for (int j = 0; j < 8; ++j) {
-                        const uint32_t lo = (e < 2) ? w[2 * j].x : w[2 * j].y;
-                        const uint32_t hi = (e < 2) ? w[2 * j + 1].x : w[2 * j + 1].y;
-                        raw[j] = __byte_perm(lo, hi, (e & 1) ? 0x7632 : 0x5410);
-                    }
+                    for (int r = 0; r < 16; ++r) rw[r] = (e < 2) ? w[r].x : w[r].y;
                     const uint64_t unit = (uint64_t)(col + e) * (uint64_t)units_per_row + (uint64_t)(k0 >> 4);
-                    prune_unit_bf16<NM>(raw, unit, fp.rk, &v, &mt);
+                    if (e & 1) prune_unit_bf16_rows<NM, true>(rw, unit, fp.rk, &v, &mt);
+                    else       prune_unit_bf16_rows<NM, false>(rw, unit, fp.rk, &v, &mt);
                 }
                 // A tile: row m_l is 128 bytes; the strip's 8 survivors are chunk strip_l, swizzled by the row
                 *reinterpret_cast<uint4*>(a_tile + m_l * 128 + ((strip_l ^ (m_l & 7)) << 4)) = v;

@@ -242,11 +242,11 @@ prune_axis0_kernel(const __grid_constant__ CUtensorMap map_g, const void* __rest
             uint4 v;
             uint32_t mt;
             if (kBf16) {
-                uint32_t raw[8];
+                uint32_t rw[16];
 #pragma unroll
-                for (int j = 0; j < 8; ++j)
-                    raw[j] = __byte_perm(w[2 * j][0], w[2 * j + 1][0], e ? 0x7632 : 0x5410);
-                prune_unit_bf16<M>(raw, unit, rk, &v, &mt);
+                for (int i = 0; i < 16; ++i) rw[i] = w[i][0];
+                if (e == 0) prune_unit_bf16_rows<M, false>(rw, unit, rk, &v, &mt);
+                else        prune_unit_bf16_rows<M, true>(rw, unit, rk, &v, &mt);
             } else {
                 uint32_t b[16];
 #pragma unroll
