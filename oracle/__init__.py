@@ -61,10 +61,12 @@ def lib() -> ctypes.CDLL:
         L.oracle_mvue_2of4.argtypes = [ctypes.POINTER(ctypes.c_float), ctypes.c_uint32,
                                        ctypes.POINTER(ctypes.c_int), ctypes.POINTER(ctypes.c_float)]
         L.oracle_mvue_2of4.restype = None
+        L.oracle_mvue_2of4_systematic.argtypes = L.oracle_mvue_2of4.argtypes
+        L.oracle_mvue_2of4_systematic.restype = None
         L.oracle_prune.argtypes = [ctypes.c_void_p, ctypes.c_int, ctypes.c_int64, ctypes.c_int64,
                                    ctypes.c_int64, ctypes.c_int, ctypes.c_int, ctypes.c_int,
                                    ctypes.c_uint64, ctypes.c_int64, ctypes.c_int64,
-                                   ctypes.c_void_p, ctypes.c_void_p, ctypes.c_int]
+                                   ctypes.c_void_p, ctypes.c_void_p, ctypes.c_int, ctypes.c_int]
         L.oracle_prune.restype = ctypes.c_int
         L.oracle_unpack.argtypes = [ctypes.c_void_p, ctypes.c_void_p, ctypes.c_int64, ctypes.c_int64,
                                     ctypes.c_void_p]
@@ -76,7 +78,7 @@ def lib() -> ctypes.CDLL:
         L.oracle_gemm_entry.argtypes = [ctypes.c_void_p, ctypes.c_int64, ctypes.c_void_p,
                                         ctypes.c_int64, ctypes.c_int64]
         L.oracle_gemm_entry.restype = ctypes.c_double
-        L.oracle_sweep_2of4.argtypes = [ctypes.POINTER(ctypes.c_float), ctypes.POINTER(ctypes.c_uint64),
+        L.oracle_sweep_2of4.argtypes = [ctypes.POINTER(ctypes.c_float), ctypes.c_int, ctypes.POINTER(ctypes.c_uint64),
                                         ctypes.POINTER(ctypes.c_double), ctypes.POINTER(ctypes.c_double)]
         L.oracle_sweep_2of4.restype = None
         L.oracle_sweep_1of2.argtypes = [ctypes.c_float, ctypes.c_float, ctypes.POINTER(ctypes.c_uint64),
@@ -127,11 +129,15 @@ def mvue_1of2(a1: float, a2: float, word: int):
     return int(idx), float(kept.value)
 
 
-def mvue_2of4(a, word: int):
+JOINT_TABLE, JOINT_SYSTEMATIC = 0, 1      # 2:4 law over pairs: App. A.2 table / systematic sampling
+
+
+def mvue_2of4(a, word: int, joint: int = JOINT_TABLE):
     arr = (ctypes.c_float * 4)(*[float(x) for x in a])
     idx = (ctypes.c_int * 2)()
     val = (ctypes.c_float * 2)()
-    lib().oracle_mvue_2of4(arr, word & 0xFFFFFFFF, idx, val)
+    fn = lib().oracle_mvue_2of4 if joint == JOINT_TABLE else lib().oracle_mvue_2of4_systematic
+    fn(arr, word & 0xFFFFFFFF, idx, val)
     return (int(idx[0]), int(idx[1])), (float(val[0]), float(val[1]))
 
 
@@ -141,8 +147,9 @@ def packed_shapes(rows: int, cols: int, axis: int):
 
 
 def prune(g: np.ndarray, n: int, m: int, axis: int, seed: int, *, k_total: int | None = None,
-          k_offset: int = 0, threads: int = 1):
+          k_offset: int = 0, threads: int = 1, joint: int = JOINT_TABLE):
     """MVUE n:m prune + pack of a 2-D array (float32, or uint16 holding bf16 bits).
+    joint: the 2:4 law over pairs (JOINT_TABLE: App. A.2; JOINT_SYSTEMATIC); ignored for 1:2.
 
     Returns (values uint16 [Mrows, K/2], meta uint8 [Mrows, K/8]) in canonical form.
     """
@@ -155,7 +162,7 @@ def prune(g: np.ndarray, n: int, m: int, axis: int, seed: int, *, k_total: int |
     meta = np.zeros(mshape, dtype=np.uint8)
     rc = lib().oracle_prune(g.ctypes.data, int(g.dtype == np.uint16), rows, cols, cols, n, m, axis,
                             seed & (2**64 - 1), k if k_total is None else k_total, k_offset,
-                            values.ctypes.data, meta.ctypes.data, max(1, threads))
+                            values.ctypes.data, meta.ctypes.data, max(1, threads), int(joint))
     if rc != 0:
         raise ValueError("oracle_prune: unsupported N:M or shape")
     return values, meta
@@ -196,13 +203,13 @@ def gemm_entry(A_row: np.ndarray, B: np.ndarray, j: int) -> float:
 PAIRS = ((0, 1), (0, 2), (0, 3), (1, 2), (1, 3), (2, 3))
 
 
-def sweep_2of4(a):
+def sweep_2of4(a, joint: int = JOINT_TABLE):
     """Frequencies of the six outcomes, mean of theta(a) and block variance over all 2^24 eps."""
     arr = (ctypes.c_float * 4)(*[float(x) for x in a])
     counts = (ctypes.c_uint64 * 6)()
     sums = (ctypes.c_double * 4)()
     sq = ctypes.c_double()
-    lib().oracle_sweep_2of4(arr, counts, sums, ctypes.byref(sq))
+    lib().oracle_sweep_2of4(arr, int(joint), counts, sums, ctypes.byref(sq))
     n = float(1 << 24)
     return (np.array([c for c in counts], dtype=np.float64) / n,
             np.array([s for s in sums]) / n, sq.value / n)

@@ -19,7 +19,9 @@
  * Parity pins (see tests): Philox against two independent implementations;
  * the 1:2 sampler against the closed form of Sec. 4.1; the 2:4 sampler against
  * the pair table of App. A.2 and the optimal marginals of Sec. 4.2 by an
- * exhaustive sweep over every value of the 24-bit uniform; bf16 rounding
+ * exhaustive sweep over every value of the 24-bit uniform; the second 2:4 law
+ * (systematic sampling) against the same optimal marginals, mean and minimal
+ * variance by the same sweep, and against its interval-overlap law; bf16 rounding
  * against a library cast; the product against a library fp64 matmul.
  */
 #include <math.h>
@@ -198,6 +200,84 @@ void oracle_mvue_2of4(const float a[4], uint32_t word, int idx[2], float val[2])
 }
 
 /* ------------------------------------------------------------------------
+ * MVUE 2:4 with a second joint law: systematic sampling.
+ *
+ * Sec. 4.2 shows that the block variance (its variance equation) is a function
+ * of the marginals p_i alone, and that a 2:4 estimator is optimal exactly when
+ * its marginals satisfy one of the two optimality criteria of that section
+ * (all p_i = 2 a_i / sum, or one p_i = 1 and the rest a_k / sum of the rest).
+ * App. A.2 is ONE joint law over pairs with those marginals.  This function
+ * draws the pair from another law with the SAME marginals and the same kept
+ * values a_i / p_i, hence the same expectation and the same (minimal)
+ * variance, that needs no sort:
+ *
+ * 1. Work in the block's own order.  m_k = |a_k|, R_k = the sum of the other
+ *    three magnitudes, and the weight e_k = min(m_k, R_k): an element heavier
+ *    than the rest together is clipped to their sum (at most one element is
+ *    clipped).  D = e_0+e_1+e_2+e_3, H = D/2; then e_k / H is exactly the
+ *    optimal p_k of Sec. 4.2 in both of its cases (unclipped: H = sum/2;
+ *    clipped element i: H = R_i, p_i = 1, p_k = m_k / R_i).
+ * 2. Lay the weights end to end: element k owns [c_k, c_{k+1}) with c_0 = 0,
+ *    c_1 = e_0, c_2 = c_1 + e_1, c_3 = c_2 + e_2.  Draw t = eps H in [0, H) and
+ *    keep the owner of t and the owner of t + H.  Every interval is at most H
+ *    long, so the two owners differ and element k is kept with probability
+ *    e_k / H.
+ * 3. A survivor becomes sign(a_k) max(m_k, H): H = m_k / p_k when p_k < 1, and
+ *    the clipped element (p = 1, m_k >= H) keeps its value.
+ *
+ * Arithmetic (binary32, in the order written):
+ *    q01 = (m0 + m1) + tiny,  q23 = (m2 + m3) + tiny,   tiny = 2^-149
+ *    R0 = m1 + q23, R1 = m0 + q23, R2 = q01 + m3, R3 = q01 + m2
+ *    eps = n / 2^23, n = the top 23 bits of the block's word;
+ *    Hs = D 2^-24, H = D/2, t2 = (2^23 + n) Hs  (one rounding; H <= t2 < D), t = t2 - H
+ *    (exact, since H <= t2 <= 2H): the two points are exactly H apart and 0 <= t < H
+ *    i  = #{k in 1,2 : c_k <= t}
+ *    j  = max(i + 1, #{k in 1,2,3 : c_k <= t2})
+ * so that i < j are two valid positions for every input and every rounding.
+ * Where a prefix sum is inexact a boundary sits one unit in the last place off
+ * its exact position; the one or two draws (of 2^23) that fall into such a gap
+ * resolve through the max above, which moves each survival probability by at
+ * most 2^-22, the resolution of eps itself.
+ * Zero rule: an element of magnitude zero owns an empty interval and is never
+ * drawn.  tiny (the smallest positive binary32 number) leaves every R_k that is
+ * a normal number unchanged and gives a lone non-zero element a non-empty
+ * interval: then D = tiny, H and t round to zero, i is the number of zeros
+ * before it (at most 2) and j = i + 1 or 3, so the non-zero survives with its own
+ * value and a zero is kept beside it as a signed zero; an all-zero block keeps
+ * positions 2 and 3.
+ *
+ * idx[0] < idx[1] are the surviving positions, val[] their new values.
+ * ---------------------------------------------------------------------- */
+void oracle_mvue_2of4_systematic(const float a[4], uint32_t word, int idx[2], float val[2])
+{
+    const float tiny = 1.401298464324817e-45f;             /* 2^-149 */
+    const float m0 = fabsf(a[0]), m1 = fabsf(a[1]), m2 = fabsf(a[2]), m3 = fabsf(a[3]);
+    const float q01 = (m0 + m1) + tiny;
+    const float q23 = (m2 + m3) + tiny;
+    const float R0 = m1 + q23, R1 = m0 + q23, R2 = q01 + m3, R3 = q01 + m2;
+    const float e0 = m0 < R0 ? m0 : R0;
+    const float e1 = m1 < R1 ? m1 : R1;
+    const float e2 = m2 < R2 ? m2 : R2;
+    const float e3 = m3 < R3 ? m3 : R3;
+    const float c1 = e0;
+    const float c2 = c1 + e1;
+    const float c3 = c2 + e2;
+    const float D  = c3 + e3;
+    const float Hs = D * 5.9604644775390625e-08f;          /* D 2^-24 */
+    const float H  = 0.5f * D;
+    const float n2 = (float)((word >> 9) + (1u << 23));    /* 2^23 + n: 24 bits, exact */
+    const float t2 = n2 * Hs;
+    const float t  = t2 - H;
+    int i = (c1 <= t) + (c2 <= t);
+    int j = (c1 <= t2) + (c2 <= t2) + (c3 <= t2);
+    if (j < i + 1) j = i + 1;
+    const float m[4] = { m0, m1, m2, m3 };
+    idx[0] = i; idx[1] = j;
+    val[0] = copysignf(m[i] > H ? m[i] : H, a[i]);
+    val[1] = copysignf(m[j] > H ? m[j] : H, a[j]);
+}
+
+/* ------------------------------------------------------------------------
  * Tensor-wide prune and pack.
  *
  * g is a row-major [rows x cols] matrix with leading dimension ld, fp32
@@ -217,6 +297,8 @@ void oracle_mvue_2of4(const float a[4], uint32_t word, int idx[2], float val[2])
  *                        of four, low nibble = even group.
  * A 1:2 result is written as a valid 2:4 pattern: the pair (4j, 4j+1) gives
  * idx0 in {0,1}, the pair (4j+2, 4j+3) gives idx1 in {2,3}.
+ * joint selects the 2:4 law over pairs: 0 = the pair table of App. A.2,
+ * 1 = systematic sampling (above); 1:2 has a single law and ignores it.
  * Returns 0, or -1 for an unsupported shape.
  * ---------------------------------------------------------------------- */
 static float load_elem(const void *g, int is_bf16, int64_t off)
@@ -227,7 +309,7 @@ static float load_elem(const void *g, int is_bf16, int64_t off)
 
 int oracle_prune(const void *g, int is_bf16, int64_t rows, int64_t cols, int64_t ld,
                  int n, int m, int axis, uint64_t seed, int64_t k_total, int64_t k_offset,
-                 uint16_t *values, uint8_t *meta, int threads)
+                 uint16_t *values, uint8_t *meta, int threads, int joint)
 {
     const int64_t Mrows = axis == 1 ? rows : cols;
     const int64_t K     = axis == 1 ? cols : rows;
@@ -246,7 +328,8 @@ int oracle_prune(const void *g, int is_bf16, int64_t rows, int64_t cols, int64_t
             int idx[2]; float val[2];
             if (m == 4) {
                 uint64_t q = (uint64_t)r * (uint64_t)(k_total / 4) + (uint64_t)(k_offset / 4 + j);
-                oracle_mvue_2of4(a, oracle_block_word(seed, q), idx, val);
+                if (joint == 0) oracle_mvue_2of4(a, oracle_block_word(seed, q), idx, val);
+                else            oracle_mvue_2of4_systematic(a, oracle_block_word(seed, q), idx, val);
             } else {
                 for (int half = 0; half < 2; ++half) {
                     uint64_t q = (uint64_t)r * (uint64_t)(k_total / 2)
@@ -323,10 +406,11 @@ double oracle_gemm_entry(const float *A_row, int64_t K, const uint16_t *B, int64
  * Exhaustive sweep helper for the pins: run the block sampler for every one
  * of the 2^24 values eps can take and count how often each outcome occurs.
  * 2:4: counts[6] over the position pairs (0,1),(0,2),(0,3),(1,2),(1,3),(2,3)
- * of the ORIGINAL block; sum_val[4] accumulates theta(a) per position;
+ * of the ORIGINAL block (joint: 0 = App. A.2 table, 1 = systematic sampling, which reads
+ * 23 of the 24 bits, so every outcome is counted twice); sum_val[4] accumulates theta(a) per position;
  * sum_sq accumulates |theta(a) - a|^2.  1:2: counts[0..1], sum_val[0..1].
  * ---------------------------------------------------------------------- */
-void oracle_sweep_2of4(const float a[4], uint64_t counts[6], double sum_val[4], double *sum_sq)
+void oracle_sweep_2of4(const float a[4], int joint, uint64_t counts[6], double sum_val[4], double *sum_sq)
 {
     static const int pair_id[4][4] = { { -1, 0, 1, 2 }, { 0, -1, 3, 4 }, { 1, 3, -1, 5 }, { 2, 4, 5, -1 } };
     for (int i = 0; i < 6; ++i) counts[i] = 0;
@@ -334,7 +418,8 @@ void oracle_sweep_2of4(const float a[4], uint64_t counts[6], double sum_val[4], 
     *sum_sq = 0.0;
     for (uint32_t n = 0; n < (1u << 24); ++n) {
         int idx[2]; float val[2];
-        oracle_mvue_2of4(a, n << 8, idx, val);
+        if (joint == 0) oracle_mvue_2of4(a, n << 8, idx, val);
+        else            oracle_mvue_2of4_systematic(a, n << 8, idx, val);
         counts[pair_id[idx[0]][idx[1]]] += 1;
         double th[4] = { 0, 0, 0, 0 };
         th[idx[0]] = val[0]; th[idx[1]] = val[1];

@@ -103,6 +103,24 @@ def outcome_law24(a):
     return law
 
 
+def systematic_law24(a):
+    """Law of the six position pairs when the pair is drawn by systematic sampling from the
+    optimal marginals of Sec. 4.2: element k owns an interval of length H p_k (in block
+    order), t is uniform on [0, H) and the owners of t and t + H survive.  Computed as the
+    measure of {t : t in I_i, t + H in I_j}, i.e. |I_i  intersect  (I_j - H)| / H, in
+    binary64 from marginals24, with no reference to how the sampler walks its thresholds.
+    Needs at least two non-zeros.  Returns {(i, j): prob}, 0-based, i < j."""
+    m = np.abs(np.asarray(a, dtype=np.float64))
+    p = marginals24(m)
+    edges = np.concatenate([[0.0], np.cumsum(p)])          # in units of H: total length 2
+    law = {pr: 0.0 for pr in itertools.combinations(range(4), 2)}
+    for i, j in law:
+        lo = max(edges[i], edges[j] - 1.0)
+        hi = min(edges[i + 1], edges[j + 1] - 1.0)
+        law[(i, j)] = max(0.0, hi - lo)
+    return law
+
+
 # ------------------------------------------- 1:2 comparison estimators -------
 def estimator12(name: str, a1: float, a2: float):
     """Table 2's 1:2 pruners as a list of (probability, [theta_1, theta_2])."""

@@ -15,13 +15,13 @@ def _slice():
     return np.ascontiguousarray(g[:16, :16])
 
 
-@pytest.mark.parametrize("n,m", [(1, 2), (2, 4)])
-def test_mean_and_mask_frequencies_over_seeds(n, m):
+@pytest.mark.parametrize("n,m,joint", [(1, 2, 0), (2, 4, 0), (2, 4, 1)])
+def test_mean_and_mask_frequencies_over_seeds(n, m, joint):
     g = _slice()
     acc = np.zeros((16, 16))
     nib_counts = np.zeros((16, 4, 16))                    # [A row, group, nibble value]
     for seed in range(N_SEEDS):
-        values, meta = oracle.prune(g, n, m, axis=0, seed=seed)       # A = g^T: [16, 16]
+        values, meta = oracle.prune(g, n, m, axis=0, seed=seed, joint=joint)       # A = g^T: [16, 16]
         acc += oracle.unpack(values, meta)
         nibs = np.stack([meta & 0xF, meta >> 4], axis=2).reshape(16, 4)
         for r in range(16):
@@ -34,7 +34,8 @@ def test_mean_and_mask_frequencies_over_seeds(n, m):
             blk = A[r, 4 * j:4 * j + 4]
             if m == 4:
                 p = theory.marginals24(blk)
-                law = theory.outcome_law24(blk) if np.count_nonzero(blk) >= 2 else None
+                law_of = theory.outcome_law24 if joint == oracle.JOINT_TABLE else theory.systematic_law24
+                law = law_of(blk) if np.count_nonzero(blk) >= 2 else None
             else:
                 p = np.zeros(4)
                 for h in range(2):

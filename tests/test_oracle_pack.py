@@ -27,11 +27,11 @@ def test_bf16_rne_matches_library_cast():
     assert np.array_equal(oracle.bf16_rne(f[fin]), allb[fin])
 
 
-@pytest.mark.parametrize("n,m", [(1, 2), (2, 4)])
+@pytest.mark.parametrize("n,m,joint", [(1, 2, 0), (2, 4, 0), (2, 4, 1)])
 @pytest.mark.parametrize("dist", ["relu_normal", "relu_lognormal", "student_t"])
-def test_packed_form_properties(n, m, dist):
+def test_packed_form_properties(n, m, joint, dist):
     g = workloads.gradient((48, 64), dist, seed=9, dtype="bf16")
-    values, meta = oracle.prune(g, n, m, axis=1, seed=5)
+    values, meta = oracle.prune(g, n, m, axis=1, seed=5, joint=joint)
     assert values.shape == (48, 32) and meta.shape == (48, 8)
     lo, hi = meta & 3, (meta >> 2) & 3
     lo2, hi2 = (meta >> 4) & 3, (meta >> 6) & 3
@@ -62,15 +62,16 @@ def test_prune_agrees_with_per_block_calls_and_numbering():
     # tensor-wide loop == block sampler driven by word(seed, q), q = r * (K/M) + j
     g = workloads.gradient((8, 32), "student_t", seed=4, dtype="f32")
     seed = 0xDEADBEEFCAFE
-    values, meta = oracle.prune(g, 2, 4, axis=1, seed=seed)
-    for r in range(8):
-        for j in range(8):
-            q = r * 8 + j
-            (i0, i1), (v0, v1) = oracle.mvue_2of4(g[r, 4 * j:4 * j + 4], philox_py.block_word(seed, q))
-            nib = (meta[r, j // 2] >> (4 * (j % 2))) & 0xF
-            assert nib == (i0 | (i1 << 2))
-            assert values[r, 2 * j] == oracle.bf16_rne(np.float32(v0))
-            assert values[r, 2 * j + 1] == oracle.bf16_rne(np.float32(v1))
+    for joint in (oracle.JOINT_TABLE, oracle.JOINT_SYSTEMATIC):
+        values, meta = oracle.prune(g, 2, 4, axis=1, seed=seed, joint=joint)
+        for r in range(8):
+            for j in range(8):
+                q = r * 8 + j
+                (i0, i1), (v0, v1) = oracle.mvue_2of4(g[r, 4 * j:4 * j + 4], philox_py.block_word(seed, q), joint)
+                nib = (meta[r, j // 2] >> (4 * (j % 2))) & 0xF
+                assert nib == (i0 | (i1 << 2))
+                assert values[r, 2 * j] == oracle.bf16_rne(np.float32(v0))
+                assert values[r, 2 * j + 1] == oracle.bf16_rne(np.float32(v1))
     values, meta = oracle.prune(g, 1, 2, axis=1, seed=seed)
     for r in range(8):
         for j2 in range(16):
@@ -83,22 +84,22 @@ def test_prune_agrees_with_per_block_calls_and_numbering():
             assert values[r, j2] == oracle.bf16_rne(np.float32(kept))
 
 
-@pytest.mark.parametrize("n,m", [(1, 2), (2, 4)])
-def test_axis0_is_the_transpose_view(n, m):
+@pytest.mark.parametrize("n,m,joint", [(1, 2, 0), (2, 4, 0), (2, 4, 1)])
+def test_axis0_is_the_transpose_view(n, m, joint):
     # blocks down the rows of g == blocks along the rows of g^T, same block numbers
     g = workloads.gradient((64, 24), "relu_normal", seed=1, dtype="bf16")
-    v0, m0 = oracle.prune(g, n, m, axis=0, seed=3)
-    v1, m1 = oracle.prune(np.ascontiguousarray(g.T), n, m, axis=1, seed=3)
+    v0, m0 = oracle.prune(g, n, m, axis=0, seed=3, joint=joint)
+    v1, m1 = oracle.prune(np.ascontiguousarray(g.T), n, m, axis=1, seed=3, joint=joint)
     assert np.array_equal(v0, v1) and np.array_equal(m0, m1)
     assert v0.shape == (24, 32) and m0.shape == (24, 8)
 
 
-@pytest.mark.parametrize("n,m", [(1, 2), (2, 4)])
-def test_k_shards_reproduce_the_unsharded_masks(n, m):
+@pytest.mark.parametrize("n,m,joint", [(1, 2, 0), (2, 4, 0), (2, 4, 1)])
+def test_k_shards_reproduce_the_unsharded_masks(n, m, joint):
     g = workloads.gradient((96, 16), "student_t", seed=2, dtype="bf16")
-    v, mt = oracle.prune(g, n, m, axis=0, seed=8)
+    v, mt = oracle.prune(g, n, m, axis=0, seed=8, joint=joint)
     for lo, hi in [(0, 32), (32, 96)]:
-        vs, ms = oracle.prune(g[lo:hi], n, m, axis=0, seed=8, k_total=96, k_offset=lo)
+        vs, ms = oracle.prune(g[lo:hi], n, m, axis=0, seed=8, k_total=96, k_offset=lo, joint=joint)
         assert np.array_equal(vs, v[:, lo // 2:hi // 2]) and np.array_equal(ms, mt[:, lo // 8:hi // 8])
 
 
@@ -107,8 +108,12 @@ def test_threads_do_not_change_the_result_and_seed_does():
     a = oracle.prune(g, 2, 4, axis=1, seed=1, threads=1)
     b = oracle.prune(g, 2, 4, axis=1, seed=1, threads=4)
     c = oracle.prune(g, 2, 4, axis=1, seed=2, threads=1)
+    d = oracle.prune(g, 2, 4, axis=1, seed=1, threads=1, joint=oracle.JOINT_SYSTEMATIC)
+    e = oracle.prune(g, 1, 2, axis=1, seed=1), oracle.prune(g, 1, 2, axis=1, seed=1, joint=oracle.JOINT_SYSTEMATIC)
     assert np.array_equal(a[0], b[0]) and np.array_equal(a[1], b[1])
     assert not np.array_equal(a[1], c[1])
+    assert not np.array_equal(a[1], d[1])                      # the two 2:4 laws draw different pairs
+    assert np.array_equal(e[0][0], e[1][0]) and np.array_equal(e[0][1], e[1][1])   # 1:2 has one law
 
 
 def test_unsupported_modes_are_rejected():
