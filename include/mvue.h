@@ -48,10 +48,23 @@ typedef enum {
     MVUE_ERR_WORKSPACE = -7,      /* workspace NULL or smaller than mvue_gemm_workspace_bytes */
     MVUE_ERR_ARCH = -8,           /* current device is not sm_100 */
     MVUE_ERR_CUDA = -9,           /* a CUDA runtime/driver call failed; text in mvue_last_cuda_error() */
-    MVUE_ERR_DEVICE_TIMEOUT = -10 /* only ever written to a device status word: a bounded wait expired */
+    MVUE_ERR_DEVICE_TIMEOUT = -10,/* only ever written to a device status word: a bounded wait expired */
+    MVUE_ERR_JOINT = -11          /* unknown mvue_joint */
 } mvue_status;
 
 typedef enum { MVUE_F32 = 0, MVUE_BF16 = 1 } mvue_dtype;
+
+/* The joint law over pairs from which a 2:4 block's two survivors are drawn.  Sec. 4.2 fixes
+ * only the marginals p_i (the block variance is a function of them alone); both laws below have
+ * exactly those marginals and the kept values a_i / p_i, hence E[theta(a)] = a and the same,
+ * minimal, variance.  They draw different pairs for the same seed.
+ * MVUE_JOINT_TABLE:      the pair table of App. A.2 (sorts the block by magnitude).
+ * MVUE_JOINT_SYSTEMATIC: systematic sampling in the block's own order, no sort: element k owns an
+ *   interval of length e_k = min(|a_k|, sum of the other three) of [0, D), D = sum e_k; the owners
+ *   of t and t + D/2 survive, t = eps D/2 (eps: the top 23 bits of the block's random word);
+ *   a survivor becomes sign(a_k) max(|a_k|, D/2).  About a fifth fewer instructions per block.
+ * 1:2 has a single law (Sec. 4.1) and ignores the choice. */
+typedef enum { MVUE_JOINT_TABLE = 0, MVUE_JOINT_SYSTEMATIC = 1 } mvue_joint;
 
 /* Packed operand layouts.
  * MVUE_LAYOUT_CANONICAL: for the sparse operand A[Mrows x K] (K = pruned axis)
@@ -116,6 +129,13 @@ MVUE_API int mvue_packed_sizes(int64_t rows, int64_t cols, int n, int m, int axi
 MVUE_API int mvue_prune(const void* g, int dtype, int64_t rows, int64_t cols, int64_t ld, int n, int m,
                int axis, uint64_t seed, int64_t k_total, int64_t k_offset, void* values,
                void* meta, int layout, void* stream);
+
+/* mvue_prune with the 2:4 joint law chosen by the caller (an mvue_joint; mvue_prune itself uses
+ * MVUE_JOINT_TABLE).  Everything else -- block numbering, random words, packed layouts, arguments,
+ * preconditions, errors -- is as for mvue_prune; an unknown joint gives MVUE_ERR_JOINT. */
+MVUE_API int mvue_prune_joint(const void* g, int dtype, int64_t rows, int64_t cols, int64_t ld, int n, int m,
+                     int axis, uint64_t seed, int64_t k_total, int64_t k_offset, void* values,
+                     void* meta, int layout, int joint, void* stream);
 
 /* Expand a packed operand back to dense bf16 A[Mrows x K] (row-major, ld = K).
  * A checking aid: the inverse of the pack step, no arithmetic. */

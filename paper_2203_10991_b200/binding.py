@@ -17,9 +17,10 @@ _lib = None
 MVUE_F32, MVUE_BF16 = 0, 1
 MVUE_LAYOUT_CANONICAL = 0
 MVUE_LAYOUT_TC = 1
+MVUE_JOINT_TABLE, MVUE_JOINT_SYSTEMATIC = 0, 1
 
 EXPORTS = ("mvue_version", "mvue_status_string", "mvue_last_cuda_error", "mvue_packed_sizes",
-           "mvue_prune", "mvue_unpack", "mvue_sparse_update_gemm", "mvue_sparse_backward_gemm",
+           "mvue_prune", "mvue_prune_joint", "mvue_unpack", "mvue_sparse_update_gemm", "mvue_sparse_backward_gemm",
            "mvue_gemm_workspace_bytes", "mvue_sparse_update_gemm_noalloc", "mvue_fused_update_gemm")
 
 
@@ -48,6 +49,7 @@ def lib() -> ctypes.CDLL:
         L.mvue_last_cuda_error.restype = ctypes.c_char_p
         L.mvue_packed_sizes.argtypes = [i64, i64, ci, ci, ci, ci, szp, szp]
         L.mvue_prune.argtypes = [vp, ci, i64, i64, i64, ci, ci, ci, u64, i64, i64, vp, vp, ci, vp]
+        L.mvue_prune_joint.argtypes = [vp, ci, i64, i64, i64, ci, ci, ci, u64, i64, i64, vp, vp, ci, ci, vp]
         L.mvue_unpack.argtypes = [vp, vp, ci, i64, i64, vp, vp]
         L.mvue_sparse_update_gemm.argtypes = [vp, vp, ci, i64, i64, vp, i64, i64, vp, ci, i64, ci, vp,
                                               ctypes.c_size_t, vp, vp]
@@ -87,9 +89,10 @@ def mvue_packed_sizes(rows: int, cols: int, n: int, m: int, axis: int, layout: i
 
 def mvue_prune(g: torch.Tensor, n: int, m: int, axis: int, seed: int, *, k_total: int | None = None,
                k_offset: int = 0, values: torch.Tensor | None = None, meta: torch.Tensor | None = None,
-               layout: int = MVUE_LAYOUT_CANONICAL):
+               layout: int = MVUE_LAYOUT_CANONICAL, joint: int | None = None):
     """MVUE n:m prune + pack of a 2-D CUDA tensor g (fp32 or bf16, unit column stride).
 
+    joint: None calls mvue_prune (App. A.2 pair table); an mvue_joint value calls mvue_prune_joint.
     Returns (values bf16 [Mrows, K/2], meta uint8 [Mrows, K/8]).
     """
     assert g.is_cuda and g.dim() == 2 and g.stride(1) == 1
@@ -99,9 +102,15 @@ def mvue_prune(g: torch.Tensor, n: int, m: int, axis: int, seed: int, *, k_total
         _, meta_bytes = mvue_packed_sizes(rows, cols, n, m, axis, layout)   # validates before allocating
         values = torch.empty((mrows, k // 2), dtype=torch.bfloat16, device=g.device)
         meta = torch.empty((meta_bytes // (k // 8), k // 8), dtype=torch.uint8, device=g.device)
-    _check(lib().mvue_prune(g.data_ptr(), _dtype_code(g), rows, cols, g.stride(0), n, m, axis,
-                            seed & (2**64 - 1), k if k_total is None else k_total, k_offset,
-                            values.data_ptr(), meta.data_ptr(), layout, _stream_ptr()), "mvue_prune")
+    if joint is None:
+        _check(lib().mvue_prune(g.data_ptr(), _dtype_code(g), rows, cols, g.stride(0), n, m, axis,
+                                seed & (2**64 - 1), k if k_total is None else k_total, k_offset,
+                                values.data_ptr(), meta.data_ptr(), layout, _stream_ptr()), "mvue_prune")
+    else:
+        _check(lib().mvue_prune_joint(g.data_ptr(), _dtype_code(g), rows, cols, g.stride(0), n, m, axis,
+                                      seed & (2**64 - 1), k if k_total is None else k_total, k_offset,
+                                      values.data_ptr(), meta.data_ptr(), layout, int(joint), _stream_ptr()),
+               "mvue_prune_joint")
     return values, meta
 
 

@@ -90,6 +90,7 @@ const char* mvue_status_string(int status) {
         case MVUE_ERR_ARCH: return "device is not compute capability 10.x";
         case MVUE_ERR_CUDA: return "CUDA call failed (see mvue_last_cuda_error)";
         case MVUE_ERR_DEVICE_TIMEOUT: return "a bounded device-side wait expired";
+        case MVUE_ERR_JOINT: return "unknown joint law (only the App. A.2 table and systematic sampling)";
         default: return "unknown status";
     }
 }
@@ -115,7 +116,15 @@ int mvue_packed_sizes(int64_t rows, int64_t cols, int n, int m, int axis, int la
 int mvue_prune(const void* g, int dtype, int64_t rows, int64_t cols, int64_t ld, int n, int m,
                int axis, uint64_t seed, int64_t k_total, int64_t k_offset, void* values,
                void* meta, int layout, void* stream) {
+    return mvue_prune_joint(g, dtype, rows, cols, ld, n, m, axis, seed, k_total, k_offset, values, meta, layout,
+                            MVUE_JOINT_TABLE, stream);
+}
+
+int mvue_prune_joint(const void* g, int dtype, int64_t rows, int64_t cols, int64_t ld, int n, int m,
+                     int axis, uint64_t seed, int64_t k_total, int64_t k_offset, void* values,
+                     void* meta, int layout, int joint, void* stream) {
     if (!g || !values || !meta) return MVUE_ERR_NULL;
+    if (joint != MVUE_JOINT_TABLE && joint != MVUE_JOINT_SYSTEMATIC) return MVUE_ERR_JOINT;
     if (dtype != MVUE_F32 && dtype != MVUE_BF16) return MVUE_ERR_DTYPE;
     if (int s = mvue_packed_sizes(rows, cols, n, m, axis, layout, nullptr, nullptr)) return s;
     const int64_t K = axis == 1 ? cols : rows;
@@ -126,7 +135,7 @@ int mvue_prune(const void* g, int dtype, int64_t rows, int64_t cols, int64_t ld,
     DeviceInfo dev;
     if (int s = current_device_info(&dev)) return s;
     PruneArgs a{g, dtype == MVUE_BF16, rows, cols, ld, m, axis, seed, k_total, k_offset, values, meta, dev.sm_count,
-                layout == MVUE_LAYOUT_TC};
+                layout == MVUE_LAYOUT_TC, joint};
     cudaError_t e = launch_prune(a, reinterpret_cast<cudaStream_t>(stream));
     if (e != cudaSuccess) { set_cuda_error(e, "mvue_prune launch"); return MVUE_ERR_CUDA; }
     return MVUE_OK;

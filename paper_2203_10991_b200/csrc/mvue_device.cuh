@@ -240,8 +240,80 @@ __device__ __forceinline__ void mvue_2of4_f32(uint32_t b0, uint32_t b1, uint32_t
     *nibble = swap ? (ib | (ia << 2)) : (ia | (ib << 2));
 }
 
+// ===========================================================================
+// MVUE 2:4, second joint law: systematic sampling (marginals: Sec. 4.2).
+//
+// Sec. 4.2's block variance depends on the marginals p_i alone, and App. A.2 is one
+// joint law with the optimal ones.  This law has the same marginals and kept values
+// (so the same mean and the same minimal variance) and needs no sort: in the block's
+// own order, element k gets the weight e_k = min(|a_k|, R_k), R_k = sum of the other
+// three magnitudes (an element heavier than the rest together is clipped to their
+// sum), owns [c_k, c_k + e_k) of [0, D), D = sum e_k, H = D/2; the owners of t and
+// t + H survive, t = eps H.  e_k / H is exactly the optimal p_k in both cases of
+// Sec. 4.2, and a survivor becomes sign(a_k) max(|a_k|, H) = a_k / p_k.
+//   R_k carries + 2^-149 so that a lone non-zero owns a non-empty interval;
+//   t2 = (2^23 + n)(D 2^-24), n = top 23 bits of the word; t = t2 - H is exact;
+//   i = #{c_1, c_2 <= t},  j = max(i + 1, #{c_1, c_2, c_3 <= t2}).
+// Counting is done on "less than": li = #{t < c_1, t < c_2} = 2 - i and
+// lj = min(#{t2 < c_k}, li) = 3 - j; x < c is the sign bit of x - c (the difference
+// of two finite floats is never rounded across zero).
+// ===========================================================================
+struct Pick24Sys {
+    uint32_t li, lj;     // i = 2 - li, j = 3 - lj
+    float H;
+};
+
+__device__ __forceinline__ Pick24Sys pick_2of4_sys(float m0, float m1, float m2, float m3, uint32_t word) {
+    const float tiny = __uint_as_float(1u);                                   // 2^-149
+    const float q01 = __fadd_rn(__fadd_rn(m0, m1), tiny), q23 = __fadd_rn(__fadd_rn(m2, m3), tiny);
+    const float R0 = __fadd_rn(m1, q23), R1 = __fadd_rn(m0, q23);
+    const float R2 = __fadd_rn(q01, m3), R3 = __fadd_rn(q01, m2);
+    const float c1 = fminf(m0, R0), e1 = fminf(m1, R1), e2 = fminf(m2, R2), e3 = fminf(m3, R3);
+    const float c2 = __fadd_rn(c1, e1), c3 = __fadd_rn(c2, e2), D = __fadd_rn(c3, e3);
+    const float Hs = __fmul_rn(D, 5.9604644775390625e-08f);                   // D 2^-24
+    Pick24Sys r;
+    r.H = __fmul_rn(0.5f, D);
+    // 2^23 + n as a float: its bit pattern is 0x4B000000 + n
+    const float n2 = __uint_as_float(__umulhi(word, 1u << 23) + 0x4B000000u);
+    const float t2 = __fmul_rn(n2, Hs), t = __fsub_rn(t2, r.H);
+    auto below = [](float x, float c) { return __umulhi(__float_as_uint(__fsub_rn(x, c)), 2u); };   // x < c ? 1 : 0
+    r.li = below(t, c1) + below(t, c2);
+    r.lj = min(below(t2, c1) + below(t2, c2) + below(t2, c3), r.li);
+    return r;
+}
+
+// bf16 source: x01 = a0 | a1 << 16, x23 = a2 | a3 << 16.  The two survivors are gathered by one byte
+// permute (selector bytes 2i, 2i+1, 2j, 2j+1); bf16 rounding is monotone, so the rounded max(|a|, H)
+// is the larger of the element's own bits and the rounded H, taken on both halves at once as
+// signed 16-bit integers (with equal sign bits the larger magnitude is the larger integer).
+__device__ __forceinline__ void mvue_2of4_sys_bf16(uint32_t x01, uint32_t x23, uint32_t word, uint32_t* out,
+                                                   uint32_t* nibble) {
+    const Pick24Sys r = pick_2of4_sys(fabsf(__uint_as_float(x01 << 16)), fabsf(__uint_as_float(x01 & 0xFFFF0000u)),
+                                      fabsf(__uint_as_float(x23 << 16)), fabsf(__uint_as_float(x23 & 0xFFFF0000u)),
+                                      word);
+    const uint32_t sel = 0x7654u - 0x22u * r.li - 0x2200u * r.lj;
+    const uint32_t raw = __byte_perm(x01, x23, sel);
+    const uint32_t hs = pack_bf16x2(r.H, r.H) | (raw & 0x80008000u);
+    *out = __vmaxs2(raw, hs);
+    *nibble = 14u - r.li - 4u * r.lj;                                         // i | j << 2
+}
+
+// binary32 source: b0..b3 are the raw bit patterns.
+__device__ __forceinline__ void mvue_2of4_sys_f32(uint32_t b0, uint32_t b1, uint32_t b2, uint32_t b3,
+                                                  uint32_t word, uint32_t* out, uint32_t* nibble) {
+    const Pick24Sys r = pick_2of4_sys(fabsf(__uint_as_float(b0)), fabsf(__uint_as_float(b1)),
+                                      fabsf(__uint_as_float(b2)), fabsf(__uint_as_float(b3)), word);
+    const uint32_t bi = r.li == 2u ? b0 : (r.li == 1u ? b1 : b2);            // i = 2 - li in {0, 1, 2}
+    const uint32_t bj = r.lj == 2u ? b1 : (r.lj == 1u ? b2 : b3);            // j = 3 - lj in {1, 2, 3}
+    const float vi = __uint_as_float(__float_as_uint(fmaxf(fabsf(__uint_as_float(bi)), r.H)) | (bi & 0x80000000u));
+    const float vj = __uint_as_float(__float_as_uint(fmaxf(fabsf(__uint_as_float(bj)), r.H)) | (bj & 0x80000000u));
+    *out = pack_bf16x2(vi, vj);
+    *nibble = 14u - r.li - 4u * r.lj;
+}
+
 // One work unit of bf16 input: raw[8] = 16 elements along K, two per word.
-template <int M>
+// kJoint selects the 2:4 law over pairs (0: App. A.2 table, 1: systematic sampling); 1:2 has one law.
+template <int M, int kJoint = 0>
 __device__ __forceinline__ void prune_unit_bf16(const uint32_t (&raw)[8], uint64_t unit_index,
                                                 const RoundKeys& rk, uint4* out_values,
                                                 uint32_t* out_meta) {
@@ -253,8 +325,11 @@ __device__ __forceinline__ void prune_unit_bf16(const uint32_t (&raw)[8], uint64
 #pragma unroll
         for (int j = 0; j < 4; ++j) {
             uint32_t nib;
-            mvue_2of4_bf16<false, true, false, true>(raw[2 * j], raw[2 * j], raw[2 * j + 1], raw[2 * j + 1], words[j],
-                                                     &v[j], &nib);
+            if (kJoint == 0)
+                mvue_2of4_bf16<false, true, false, true>(raw[2 * j], raw[2 * j], raw[2 * j + 1], raw[2 * j + 1],
+                                                         words[j], &v[j], &nib);
+            else
+                mvue_2of4_sys_bf16(raw[2 * j], raw[2 * j + 1], words[j], &v[j], &nib);
             meta += nib << (4 * j);
         }
     } else {
@@ -273,7 +348,7 @@ __device__ __forceinline__ void prune_unit_bf16(const uint32_t (&raw)[8], uint64
 }
 
 // One work unit whose 16 elements are the half kHigh of 16 row words (K runs down the rows of g).
-template <int M, bool kHigh>
+template <int M, bool kHigh, int kJoint = 0>
 __device__ __forceinline__ void prune_unit_bf16_rows(const uint32_t (&w)[16], uint64_t unit_index,
                                                      const RoundKeys& rk, uint4* out_values, uint32_t* out_meta) {
     uint32_t v[4];
@@ -284,8 +359,14 @@ __device__ __forceinline__ void prune_unit_bf16_rows(const uint32_t (&w)[16], ui
 #pragma unroll
         for (int j = 0; j < 4; ++j) {
             uint32_t nib;
-            mvue_2of4_bf16<kHigh, kHigh, kHigh, kHigh>(w[4 * j], w[4 * j + 1], w[4 * j + 2], w[4 * j + 3], words[j],
-                                                       &v[j], &nib);
+            if (kJoint == 0) {
+                mvue_2of4_bf16<kHigh, kHigh, kHigh, kHigh>(w[4 * j], w[4 * j + 1], w[4 * j + 2], w[4 * j + 3],
+                                                           words[j], &v[j], &nib);
+            } else {   // the halves of two row words side by side: a0 | a1 << 16, a2 | a3 << 16
+                const uint32_t x01 = __byte_perm(w[4 * j], w[4 * j + 1], kHigh ? 0x7632u : 0x5410u);
+                const uint32_t x23 = __byte_perm(w[4 * j + 2], w[4 * j + 3], kHigh ? 0x7632u : 0x5410u);
+                mvue_2of4_sys_bf16(x01, x23, words[j], &v[j], &nib);
+            }
             meta += nib << (4 * j);
         }
     } else {

@@ -19,6 +19,7 @@ struct PruneArgs {
     void* meta;
     int sm_count;
     bool tc_layout;      // metadata in tensor-core order instead of canonical rows
+    int joint;           // 2:4 law over pairs: 0 = App. A.2 table, 1 = systematic sampling
 };
 
 cudaError_t launch_prune(const PruneArgs& a, cudaStream_t stream);

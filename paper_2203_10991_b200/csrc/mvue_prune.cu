@@ -35,7 +35,7 @@ __device__ __forceinline__ uint4 ldg128(const void* p) {
 }
 
 // One work unit of binary32 input: b[16] = bit patterns of 16 elements along K.
-template <int M>
+template <int M, int kJoint = 0>
 __device__ __forceinline__ void prune_unit_f32(const uint32_t (&b)[16], uint64_t unit_index,
                                                const RoundKeys& rk, uint4* out_values,
                                                uint32_t* out_meta) {
@@ -47,7 +47,8 @@ __device__ __forceinline__ void prune_unit_f32(const uint32_t (&b)[16], uint64_t
 #pragma unroll
         for (int j = 0; j < 4; ++j) {
             uint32_t nib;
-            mvue_2of4_f32(b[4 * j], b[4 * j + 1], b[4 * j + 2], b[4 * j + 3], words[j], &v[j], &nib);
+            if (kJoint == 0) mvue_2of4_f32(b[4 * j], b[4 * j + 1], b[4 * j + 2], b[4 * j + 3], words[j], &v[j], &nib);
+            else             mvue_2of4_sys_f32(b[4 * j], b[4 * j + 1], b[4 * j + 2], b[4 * j + 3], words[j], &v[j], &nib);
             meta |= nib << (4 * j);
         }
     } else {
@@ -70,7 +71,7 @@ __device__ __forceinline__ void prune_unit_f32(const uint32_t (&b)[16], uint64_t
 // ---- axis 1 ---------------------------------------------------------------
 // slot = r * units_per_row + c.  kLinear: the tensor is contiguous and unsharded,
 // so the input offset and the generator call number are linear in the slot.
-template <int M, bool kBf16, bool kLinear, bool kTC>
+template <int M, bool kBf16, bool kLinear, bool kTC, int kJoint>
 __global__ void __launch_bounds__(256, kBf16 ? 6 : 4)
 prune_axis1_kernel(const void* __restrict__ g, int64_t n_slots, int64_t units_per_row, int64_t ld,
                    int64_t units_per_row_total, int64_t unit_offset, int64_t pad_rows, RoundKeys rk,
@@ -115,7 +116,7 @@ prune_axis1_kernel(const void* __restrict__ g, int64_t n_slots, int64_t units_pe
                 if (kBf16) {
                     const uint32_t raw[8] = {in[u][0].x, in[u][0].y, in[u][0].z, in[u][0].w,
                                              in[u][1].x, in[u][1].y, in[u][1].z, in[u][1].w};
-                    prune_unit_bf16<M>(raw, unit[u], rk, &v, &mt);
+                    prune_unit_bf16<M, kJoint>(raw, unit[u], rk, &v, &mt);
                 } else {
                     uint32_t b[16];
 #pragma unroll
@@ -123,7 +124,7 @@ prune_axis1_kernel(const void* __restrict__ g, int64_t n_slots, int64_t units_pe
                         b[4 * i] = (&in[u][i].x)[0]; b[4 * i + 1] = (&in[u][i].x)[1];
                         b[4 * i + 2] = (&in[u][i].x)[2]; b[4 * i + 3] = (&in[u][i].x)[3];
                     }
-                    prune_unit_f32<M>(b, unit[u], rk, &v, &mt);
+                    prune_unit_f32<M, kJoint>(b, unit[u], rk, &v, &mt);
                 }
                 values[slot] = v;
                 if (kTC)
@@ -173,7 +174,7 @@ __device__ __noinline__ void fill_strip_bf16(const char* p, int64_t ld, unsigned
 
 // kTma (bf16 only): the 256 x 64 input tile arrives by one TMA box copy into dynamic shared memory, so
 // the lanes read their words with compile-time offsets and no address arithmetic.
-template <int M, bool kBf16, bool kTC, bool kTma>
+template <int M, bool kBf16, bool kTC, bool kTma, int kJoint>
 __global__ void __launch_bounds__(kTileStrips * 32, kBf16 ? 3 : 2)
 prune_axis0_kernel(const __grid_constant__ CUtensorMap map_g, const void* __restrict__ g, int64_t n_strips,
                    int64_t n_cols, int64_t ld, int64_t units_per_row_total, int64_t unit_offset, RoundKeys rk,
@@ -245,13 +246,13 @@ prune_axis0_kernel(const __grid_constant__ CUtensorMap map_g, const void* __rest
                 uint32_t rw[16];
 #pragma unroll
                 for (int i = 0; i < 16; ++i) rw[i] = w[i][0];
-                if (e == 0) prune_unit_bf16_rows<M, false>(rw, unit, rk, &v, &mt);
-                else        prune_unit_bf16_rows<M, true>(rw, unit, rk, &v, &mt);
+                if (e == 0) prune_unit_bf16_rows<M, false, kJoint>(rw, unit, rk, &v, &mt);
+                else        prune_unit_bf16_rows<M, true, kJoint>(rw, unit, rk, &v, &mt);
             } else {
                 uint32_t b[16];
 #pragma unroll
                 for (int i = 0; i < 16; ++i) b[i] = w[i][kBf16 ? 0 : e];
-                prune_unit_f32<M>(b, unit, rk, &v, &mt);
+                prune_unit_f32<M, kJoint>(b, unit, rk, &v, &mt);
             }
             s_val[col_l * kTileStrips + (strip_l ^ (lane & 15))] = v;
             if (kTC) {
@@ -339,7 +340,7 @@ unpack_kernel(const uint4* __restrict__ values, const uint16_t* __restrict__ met
     }
 }
 
-template <int M, bool kBf16, bool kTC>
+template <int M, bool kBf16, bool kTC, int kJoint>
 cudaError_t launch_prune_t(const PruneArgs& a, cudaStream_t stream) {
     const RoundKeys rk = make_round_keys(a.seed);
     const int64_t upr_total = a.k_total / 16, uoff = a.k_offset / 16;
@@ -353,9 +354,9 @@ cudaError_t launch_prune_t(const PruneArgs& a, cudaStream_t stream) {
         const int grid = (int)(want < (int64_t)a.sm_count * 48 ? want : (int64_t)a.sm_count * 48);
         const int64_t pad_rows = kTC ? ((a.rows + 127) / 128) * 128 - a.rows : 0;
         if (linear)
-            prune_axis1_kernel<M, kBf16, true, kTC><<<grid, 256, 0, stream>>>(a.g, n_slots, upr, a.ld, upr_total, uoff, pad_rows, rk, values, meta);
+            prune_axis1_kernel<M, kBf16, true, kTC, kJoint><<<grid, 256, 0, stream>>>(a.g, n_slots, upr, a.ld, upr_total, uoff, pad_rows, rk, values, meta);
         else
-            prune_axis1_kernel<M, kBf16, false, kTC><<<grid, 256, 0, stream>>>(a.g, n_slots, upr, a.ld, upr_total, uoff, pad_rows, rk, values, meta);
+            prune_axis1_kernel<M, kBf16, false, kTC, kJoint><<<grid, 256, 0, stream>>>(a.g, n_slots, upr, a.ld, upr_total, uoff, pad_rows, rk, values, meta);
     } else {
         const int64_t n_strips = a.rows / 16;
         // in tensor-core order the rows of A are padded to 128: cover the padding with (load-free) tiles
@@ -371,29 +372,32 @@ cudaError_t launch_prune_t(const PruneArgs& a, cudaStream_t stream) {
             static std::once_flag once;
             static cudaError_t attr_err = cudaSuccess;
             std::call_once(once, [] {
-                attr_err = cudaFuncSetAttribute(prune_axis0_kernel<M, true, kTC, true>,
+                attr_err = cudaFuncSetAttribute(prune_axis0_kernel<M, true, kTC, true, kJoint>,
                                                 cudaFuncAttributeMaxDynamicSharedMemorySize, kTileInBytes + 16);
             });
             if (attr_err != cudaSuccess) return attr_err;
-            prune_axis0_kernel<M, true, kTC, true><<<grid, kTileStrips * 32, kTileInBytes + 16, stream>>>(
+            prune_axis0_kernel<M, true, kTC, true, kJoint><<<grid, kTileStrips * 32, kTileInBytes + 16, stream>>>(
                 map_g, a.g, n_strips, a.cols, a.ld, upr_total, uoff, rk, values, meta);
         } else {
-            prune_axis0_kernel<M, false, kTC, false><<<grid, kTileStrips * 32, 0, stream>>>(
+            prune_axis0_kernel<M, false, kTC, false, kJoint><<<grid, kTileStrips * 32, 0, stream>>>(
                 map_g, a.g, n_strips, a.cols, a.ld, upr_total, uoff, rk, values, meta);
         }
     }
     return cudaGetLastError();
 }
 
+template <int M, int kJoint>
+cudaError_t launch_prune_m(const PruneArgs& a, cudaStream_t stream) {
+    if (a.tc_layout)
+        return a.is_bf16 ? launch_prune_t<M, true, true, kJoint>(a, stream) : launch_prune_t<M, false, true, kJoint>(a, stream);
+    return a.is_bf16 ? launch_prune_t<M, true, false, kJoint>(a, stream) : launch_prune_t<M, false, false, kJoint>(a, stream);
+}
+
 }  // namespace
 
 cudaError_t launch_prune(const PruneArgs& a, cudaStream_t stream) {
-    if (a.tc_layout) {
-        if (a.m == 4) return a.is_bf16 ? launch_prune_t<4, true, true>(a, stream) : launch_prune_t<4, false, true>(a, stream);
-        return a.is_bf16 ? launch_prune_t<2, true, true>(a, stream) : launch_prune_t<2, false, true>(a, stream);
-    }
-    if (a.m == 4) return a.is_bf16 ? launch_prune_t<4, true, false>(a, stream) : launch_prune_t<4, false, false>(a, stream);
-    return a.is_bf16 ? launch_prune_t<2, true, false>(a, stream) : launch_prune_t<2, false, false>(a, stream);
+    if (a.m == 2) return launch_prune_m<2, 0>(a, stream);
+    return a.joint == 1 ? launch_prune_m<4, 1>(a, stream) : launch_prune_m<4, 0>(a, stream);
 }
 
 cudaError_t launch_unpack(const void* values, const void* meta, bool tc_layout, int64_t mrows, int64_t K,
