@@ -5,8 +5,9 @@
 // four blocks sharing one generator call; for 1:2 it is eight pairs using two.
 //   axis 1 (K contiguous in memory): one thread owns one unit = 32 contiguous
 //           bytes of bf16 (64 of fp32); a warp reads 1 KiB (2 KiB) contiguous.
-//   axis 0 (K runs down the rows of g): one thread owns a strip of 16 rows by
-//           16 bytes of columns; a warp reads 512 contiguous bytes per row.
+//   axis 0 (K runs down the rows of g): bf16 tiles arrive by TMA and are handed to
+//           the lanes transposed (one lane = 16 rows of one column); binary32 is read
+//           with plain loads, one lane owning a strip of 16 rows by two columns.
 #include <cuda.h>
 #include <cuda_runtime.h>
 
@@ -158,30 +159,18 @@ constexpr int kTileStrips = 16;
 constexpr int kTileCols = 64;
 constexpr int kMetaPitch = 36;                       // bytes per staged metadata row
 
-constexpr int kTileInBytes = kTileStrips * 16 * kTileCols * 2;   // the bf16 input tile: 256 rows x 128 bytes
-
 __device__ __forceinline__ uint32_t smem_addr(const void* p) {
     return static_cast<uint32_t>(__cvta_generic_to_shared(p));
 }
 
-// Plain-load path of one lane's strip (16 rows x 2 bf16 columns) into the shared tile; kept out of line so
-// that the TMA-fed kernel carries none of its address arithmetic.  Used only if the copy failed to land.
-__device__ __noinline__ void fill_strip_bf16(const char* p, int64_t ld, unsigned char* dst, int pitch) {
-#pragma unroll 1
-    for (int i = 0; i < 16; ++i)
-        *reinterpret_cast<uint32_t*>(dst + i * pitch) = __ldg(reinterpret_cast<const uint32_t*>(p + (int64_t)i * ld * 2));
-}
-
-// kTma (bf16 only): the 256 x 64 input tile arrives by one TMA box copy into dynamic shared memory, so
-// the lanes read their words with compile-time offsets and no address arithmetic.
-template <int M, bool kBf16, bool kTC, bool kTma, int kJoint>
+// (Used for binary32 input; bf16 input takes prune_axis0_bf16_kernel below.)
+template <int M, bool kBf16, bool kTC, int kJoint>
 __global__ void __launch_bounds__(kTileStrips * 32, kBf16 ? 3 : 2)
-prune_axis0_kernel(const __grid_constant__ CUtensorMap map_g, const void* __restrict__ g, int64_t n_strips,
-                   int64_t n_cols, int64_t ld, int64_t units_per_row_total, int64_t unit_offset, RoundKeys rk,
+prune_axis0_kernel(const void* __restrict__ g, int64_t n_strips, int64_t n_cols, int64_t ld,
+                   int64_t units_per_row_total, int64_t unit_offset, RoundKeys rk,
                    uint4* __restrict__ values, uint16_t* __restrict__ meta) {
     constexpr int ES = kBf16 ? 2 : 4;
     constexpr int NT = kTileStrips * 32;
-    extern __shared__ __align__(128) unsigned char s_in[];        // kTma: input tile, then one mbarrier
     __shared__ uint4 s_val[kTileCols * kTileStrips];
     __shared__ __align__(16) unsigned char s_meta[kTileCols * kMetaPitch];   // >= 2048 bytes
 
@@ -192,39 +181,14 @@ prune_axis0_kernel(const __grid_constant__ CUtensorMap map_g, const void* __rest
     const int64_t col0 = (int64_t)blockIdx.y * kTileCols;
     const int64_t strip = strip0 + strip_l;
     const int64_t col = col0 + 2 * lane;             // this lane's first column (n_cols is even)
-    const bool tile_has_input = col0 < n_cols;
-    const uint32_t bar = smem_addr(s_in + kTileInBytes);
-    if (kTma && tid == 0 && tile_has_input) {
-        asm volatile("mbarrier.init.shared::cta.b64 [%0], 1;" ::"r"(bar));
-        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
-        asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "r"(kTileInBytes) : "memory");
-        asm volatile(
-            "cp.async.bulk.tensor.2d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3}], [%4];"
-            ::"r"(smem_addr(s_in)), "l"(&map_g), "r"((int)col0), "r"((int)(strip0 * 16)), "r"(bar) : "memory");
-    }
     if (kTC) {                                       // padding rows of A keep a valid pattern
         for (int i = tid; i < 2048 / 4; i += NT) reinterpret_cast<uint32_t*>(s_meta)[i] = 0x44444444u;
     }
-    if (kTC || kTma) __syncthreads();
+    if (kTC) __syncthreads();
 
     if (strip < n_strips && col < n_cols) {
         const char* p = reinterpret_cast<const char*>(g) + ((strip * 16) * ld + col) * ES;
         uint32_t w[16][kBf16 ? 1 : 2];
-        bool landed = false;
-        if (kTma) {                                  // bounded wait; if it ever expired the plain loads below take over
-            for (uint32_t spin = 0; spin < (1u << 20) && !landed; ++spin) {
-                uint32_t ok;
-                asm volatile("{\n\t.reg .pred p;\n\tmbarrier.try_wait.parity.shared::cta.b64 p, [%1], 0;\n\t"
-                             "selp.u32 %0, 1, 0, p;\n\t}" : "=r"(ok) : "r"(bar) : "memory");
-                landed = ok != 0;
-            }
-        }
-        if (kTma) {
-            unsigned char* src = s_in + strip_l * 16 * (kTileCols * 2) + lane * 4;
-            if (!landed) fill_strip_bf16(p, ld, src, kTileCols * 2);
-#pragma unroll
-            for (int i = 0; i < 16; ++i) w[i][0] = *reinterpret_cast<const uint32_t*>(src + i * (kTileCols * 2));
-        } else
 #pragma unroll
         for (int i = 0; i < 16; ++i) {
             if (kBf16) {
@@ -305,6 +269,117 @@ prune_axis0_kernel(const __grid_constant__ CUtensorMap map_g, const void* __rest
     }
 }
 
+// ---- axis 0, bf16 -----------------------------------------------------------
+// A thread block owns a tile of kStrips strips of 16 rows of g by 64 columns, one warp per strip.  The tile
+// arrives by ONE TMA box copy through the 4-D view of make_map_strips, which lays it out so that two
+// transposing 8x8 matrix loads hand a lane the 16 consecutive rows of one column as eight words of two bf16
+// -- exactly the form a unit has when K is contiguous -- with no bank conflict, no byte shuffles and no
+// address arithmetic per element.  A warp covers 4 strips x 8 columns per step (lane = 4 (column % 8) +
+// strip % 4) and takes two steps whose columns are 8 apart, so in the tensor-core order the two 16-bit nibble
+// strings of a lane share one 32-bit word.  Packed survivors go straight from registers to memory: the four
+// lanes of a column write 64 contiguous bytes.  Small tiles (4 strips, 128 threads, 12 blocks per SM) keep
+// the copy of one block hidden behind the arithmetic of the others.
+constexpr int kA0Cols = 64;
+template <int kStrips> struct A0 {                               // kStrips: strips of 16 rows per tile (8 or 16)
+    static constexpr int kRows = 16 * kStrips, kThreads = 32 * kStrips;
+    static constexpr int kTileBytes = kRows * kA0Cols * 2;
+    static constexpr int kSmemBytes = kTileBytes + 1024 + 16;     // alignment slack + one mbarrier
+};
+
+// Plain-load replacement of the box copy (same shared-memory arrangement), used only if the copy never landed.
+template <int kStrips>
+__device__ __noinline__ void fill_tile_bf16(const char* g, int64_t ld, int64_t n_rows, int64_t n_cols, int64_t row0,
+                                            int64_t col0, unsigned char* tile) {
+    for (int i = threadIdx.x; i < A0<kStrips>::kRows * 8; i += A0<kStrips>::kThreads) {   // 16-byte chunks
+        const int line = i >> 3, chunk = i & 7;
+        const int k8 = line / (2 * kStrips), strip = (line >> 1) % kStrips, k2 = line & 1;
+        const int64_t r = row0 + 16 * strip + 2 * k8 + k2, c = col0 + 8 * chunk;
+        uint4 v = make_uint4(0u, 0u, 0u, 0u);
+        if (r < n_rows && c < n_cols) v = ldg128(g + (r * ld + c) * 2);     // n_cols is a multiple of 8
+        *reinterpret_cast<uint4*>(tile + line * 128 + ((chunk ^ (line & 7)) << 4)) = v;
+    }
+}
+
+template <int M, bool kTC, int kJoint, int kStrips>
+__global__ void __launch_bounds__(32 * kStrips, 1536 / (32 * kStrips))
+prune_axis0_bf16_kernel(const __grid_constant__ CUtensorMap map_g, const void* __restrict__ g, int64_t n_strips,
+                        int64_t n_cols, int64_t ld, int64_t units_per_row_total, int64_t unit_offset, RoundKeys rk,
+                        uint4* __restrict__ values, uint16_t* __restrict__ meta) {
+    constexpr int kTileBytes = A0<kStrips>::kTileBytes;
+    constexpr int kQuads = kStrips / 4;                                      // groups of 4 strips per tile
+    extern __shared__ unsigned char s_raw[];
+    const uint32_t tile = (smem_addr(s_raw) + 1023u) & ~1023u;              // the 128-byte swizzle needs 1 KiB alignment
+    const uint32_t bar = tile + kTileBytes;
+    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+    const int64_t strip0 = (int64_t)blockIdx.x * kStrips;
+    const int64_t col0 = (int64_t)blockIdx.y * kA0Cols;
+    const bool has_input = col0 < n_cols;                                    // false only for tiles that pad A's rows
+
+    if (has_input) {
+        if (tid == 0) {
+            asm volatile("mbarrier.init.shared::cta.b64 [%0], 1;" ::"r"(bar));
+            asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+            asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "r"(kTileBytes) : "memory");
+            asm volatile(
+                "cp.async.bulk.tensor.4d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3, %4, %5}], [%6];"
+                ::"r"(tile), "l"(&map_g), "r"((int)col0), "r"(0), "r"((int)strip0), "r"(0), "r"(bar) : "memory");
+        }
+        __syncthreads();
+        bool landed = false;
+        for (uint32_t spin = 0; spin < (1u << 20) && !landed; ++spin) {      // bounded wait
+            uint32_t ok;
+            asm volatile("{\n\t.reg .pred p;\n\tmbarrier.try_wait.parity.shared::cta.b64 p, [%1], 0;\n\t"
+                         "selp.u32 %0, 1, 0, p;\n\t}" : "=r"(ok) : "r"(bar) : "memory");
+            landed = ok != 0;
+        }
+        if (__syncthreads_or(!landed)) {
+            fill_tile_bf16<kStrips>(reinterpret_cast<const char*>(g), ld, n_strips * 16, n_cols, strip0 * 16, col0,
+                                    s_raw + (tile - smem_addr(s_raw)));
+            __syncthreads();
+        }
+    }
+
+    // this lane's units: strip = strip0 + 4 (warp % kQuads) + lane % 4,
+    //                    column = col0 + 8 (2 (warp / kQuads) + step) + lane / 4
+    const int quad = warp % kQuads, cpair = warp / kQuads, p = lane & 3;
+    const int64_t strip = strip0 + 4 * quad + p;
+    const bool strip_ok = strip < n_strips;
+    // address this lane supplies to the matrix loads: matrix lane / 8 (= k8, +4 for the second load), line lane % 8
+    const uint32_t ld_base = tile + (uint32_t)(((lane >> 3) * (2 * kStrips) + 8 * quad + (lane & 7)) * 128);
+    uint32_t meta_pair = 0;
+#pragma unroll
+    for (int step = 0; step < 2; ++step) {
+        const int cb = 2 * cpair + step;                                     // 8-column block inside the tile
+        const int64_t c = col0 + 8 * cb + (lane >> 2);
+        uint32_t mt = 0x4444u;                                               // rows that pad A keep a valid pattern
+        if (has_input) {
+            const uint32_t addr = ld_base + (uint32_t)((cb ^ (lane & 7)) << 4);
+            uint32_t raw[8];
+            asm volatile("ldmatrix.sync.aligned.m8n8.x4.trans.shared.b16 {%0, %1, %2, %3}, [%4];"
+                         : "=r"(raw[0]), "=r"(raw[1]), "=r"(raw[2]), "=r"(raw[3]) : "r"(addr));
+            asm volatile("ldmatrix.sync.aligned.m8n8.x4.trans.shared.b16 {%0, %1, %2, %3}, [%4];"
+                         : "=r"(raw[4]), "=r"(raw[5]), "=r"(raw[6]), "=r"(raw[7]) : "r"(addr + 4u * (2 * kStrips) * 128u));
+            if (strip_ok && c < n_cols) {
+                const uint64_t unit = (uint64_t)c * (uint64_t)units_per_row_total + (uint64_t)(unit_offset + strip);
+                uint4 v;
+                prune_unit_bf16<M, kJoint>(raw, unit, rk, &v, &mt);
+                values[c * n_strips + strip] = v;
+                if (!kTC) meta[c * n_strips + strip] = (uint16_t)mt;
+            }
+        }
+        meta_pair |= mt << (16 * step);
+    }
+    if (kTC && strip_ok) {
+        // rows c and c + 8 share the 32-bit word (k % 128) / 32 of lane c % 8 + 8 (strip % 2) + 16 (c % 128 / 16)
+        const int64_t c = col0 + 16 * cpair + (lane >> 2);
+        const int rl = (int)(c & 127);
+        const int tc_lane = (rl & 7) + 8 * (p & 1) + 16 * (rl >> 4);
+        const int64_t block = (c >> 7) * (n_strips >> 3) + (strip >> 3);
+        const int word = 2 * ((int)(strip >> 2) & 1) + (p >> 1);
+        *reinterpret_cast<uint32_t*>(reinterpret_cast<char*>(meta) + block * 2048 + tc_lane * 16 + word * 4) = meta_pair;
+    }
+}
+
 // ---- unpack ---------------------------------------------------------------
 // One thread expands one unit: a 16-bit metadata word (four groups) and its 8 survivors
 // become 16 dense elements (32 bytes).
@@ -363,24 +438,25 @@ cudaError_t launch_prune_t(const PruneArgs& a, cudaStream_t stream) {
         const int64_t cover_cols = kTC ? ((a.cols + 127) / 128) * 128 : a.cols;
         dim3 grid((unsigned)((n_strips + kTileStrips - 1) / kTileStrips),
                   (unsigned)((cover_cols + kTileCols - 1) / kTileCols));
-        CUtensorMap map_g;
-        memset(&map_g, 0, sizeof(map_g));
         if (kBf16) {
-            if (!make_map_2d(&map_g, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, a.g, (uint64_t)a.cols, (uint64_t)a.rows,
-                             (uint64_t)a.ld * 2, kTileCols, kTileStrips * 16, CU_TENSOR_MAP_SWIZZLE_NONE))
+            CUtensorMap map_g;
+            memset(&map_g, 0, sizeof(map_g));
+            constexpr int kS = 4;                                            // strips per tile
+            if (!make_map_strips(&map_g, a.g, (uint64_t)a.cols, (uint64_t)a.rows, (uint64_t)a.ld * 2, kS))
                 return cudaErrorInvalidValue;
             static std::once_flag once;
             static cudaError_t attr_err = cudaSuccess;
             std::call_once(once, [] {
-                attr_err = cudaFuncSetAttribute(prune_axis0_kernel<M, true, kTC, true, kJoint>,
-                                                cudaFuncAttributeMaxDynamicSharedMemorySize, kTileInBytes + 16);
+                attr_err = cudaFuncSetAttribute(prune_axis0_bf16_kernel<M, kTC, kJoint, kS>,
+                                                cudaFuncAttributeMaxDynamicSharedMemorySize, A0<kS>::kSmemBytes);
             });
             if (attr_err != cudaSuccess) return attr_err;
-            prune_axis0_kernel<M, true, kTC, true, kJoint><<<grid, kTileStrips * 32, kTileInBytes + 16, stream>>>(
+            dim3 grid_b((unsigned)((n_strips + kS - 1) / kS), (unsigned)((cover_cols + kA0Cols - 1) / kA0Cols));
+            prune_axis0_bf16_kernel<M, kTC, kJoint, kS><<<grid_b, A0<kS>::kThreads, A0<kS>::kSmemBytes, stream>>>(
                 map_g, a.g, n_strips, a.cols, a.ld, upr_total, uoff, rk, values, meta);
         } else {
-            prune_axis0_kernel<M, false, kTC, false, kJoint><<<grid, kTileStrips * 32, 0, stream>>>(
-                map_g, a.g, n_strips, a.cols, a.ld, upr_total, uoff, rk, values, meta);
+            prune_axis0_kernel<M, false, kTC, kJoint><<<grid, kTileStrips * 32, 0, stream>>>(
+                a.g, n_strips, a.cols, a.ld, upr_total, uoff, rk, values, meta);
         }
     }
     return cudaGetLastError();
