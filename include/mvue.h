@@ -125,7 +125,8 @@ MVUE_API int mvue_packed_sizes(int64_t rows, int64_t cols, int n, int m, int axi
  *   values, meta   outputs in `layout`, sizes from mvue_packed_sizes.
  * Preconditions (else MVUE_ERR_SHAPE / MVUE_ERR_ALIGN): K, k_total and k_offset
  * multiples of 16; Mrows a multiple of 8; ld >= cols; g, values, meta and
- * ld * sizeof(element) 16-byte aligned. */
+ * ld * sizeof(element) 16-byte aligned; K <= 65535 * 256 for axis 1, Mrows <=
+ * 65535 * 64 for axis 0. */
 MVUE_API int mvue_prune(const void* g, int dtype, int64_t rows, int64_t cols, int64_t ld, int n, int m,
                int axis, uint64_t seed, int64_t k_total, int64_t k_offset, void* values,
                void* meta, int layout, void* stream);

@@ -129,6 +129,8 @@ int mvue_prune_joint(const void* g, int dtype, int64_t rows, int64_t cols, int64
     if (int s = mvue_packed_sizes(rows, cols, n, m, axis, layout, nullptr, nullptr)) return s;
     const int64_t K = axis == 1 ? cols : rows;
     if (ld < cols) return MVUE_ERR_SHAPE;
+    // launch-grid limits: 65535 blocks of 256 k (axis 1) or of 64 rows of A (axis 0) in the second grid dimension
+    if (axis == 1 ? K > 65535ll * 256 : cols > 65535ll * 64) return MVUE_ERR_SHAPE;
     if (k_total % 16 != 0 || k_offset % 16 != 0 || k_offset < 0 || k_offset + K > k_total) return MVUE_ERR_SHAPE;
     const int64_t esz = dtype == MVUE_BF16 ? 2 : 4;
     if (!aligned16(g) || !aligned16(values) || !aligned16(meta) || (ld * esz) % 16 != 0) return MVUE_ERR_ALIGN;

@@ -70,81 +70,53 @@ __device__ __forceinline__ void prune_unit_f32(const uint32_t (&b)[16], uint64_t
 }
 
 // ---- axis 1 ---------------------------------------------------------------
-// slot = r * units_per_row + c.  kLinear: the tensor is contiguous and unsharded,
-// so the input offset and the generator call number are linear in the slot.
-template <int M, bool kBf16, bool kLinear, bool kTC, int kJoint>
-__global__ void __launch_bounds__(256, kBf16 ? 6 : 4)
-prune_axis1_kernel(const void* __restrict__ g, int64_t n_slots, int64_t units_per_row, int64_t ld,
-                   int64_t units_per_row_total, int64_t unit_offset, int64_t pad_rows, RoundKeys rk,
+// K is contiguous: a unit is 32 contiguous bytes of bf16 (64 of binary32).  A thread block owns 16 rows of A
+// by 16 units; thread = (row % 8, unit) and handles rows r and r + 8 of its unit, whose 16-bit nibble strings
+// share one 32-bit word in the tensor-core order.  A warp reads full 128-byte lines (8 rows x 4 units) and no
+// index needs a division.
+constexpr int kA1Units = 16;                          // units per block along K
+
+template <int M, bool kBf16, bool kTC, int kJoint>
+__global__ void __launch_bounds__(8 * kA1Units, kBf16 ? 12 : 8)
+prune_axis1_kernel(const void* __restrict__ g, int64_t n_rows, int units_per_row, int64_t ld,
+                   int64_t units_per_row_total, int64_t unit_offset, RoundKeys rk,
                    uint4* __restrict__ values, uint16_t* __restrict__ meta) {
-    constexpr int U = 1;                              // units per thread per trip, loads issued first
     constexpr int LW = kBf16 ? 2 : 4;                 // 16-byte loads per unit
-    const int64_t trip = (int64_t)blockDim.x * U;
-    for (int64_t base = (int64_t)blockIdx.x * trip; base < n_slots; base += (int64_t)gridDim.x * trip) {
-        uint4 in[U][LW];
-        uint64_t unit[U];
-        int64_t meta_off[U];
+    const int j = threadIdx.x & 7;
+    const int c = blockIdx.y * kA1Units + (threadIdx.x >> 3);
+    if (c >= units_per_row) return;
+    const int64_t r0 = (int64_t)blockIdx.x * 16 + j;
+    uint32_t meta_pair = 0;
 #pragma unroll
-        for (int u = 0; u < U; ++u) {
-            const int64_t slot = base + (int64_t)u * blockDim.x + threadIdx.x;
-            if (slot < n_slots) {
-                int64_t elem_off;
-                if (kLinear && !kTC) {
-                    elem_off = slot * 16;
-                    unit[u] = (uint64_t)slot;
-                } else {
-                    int64_t r;
-                    if (n_slots < (1ll << 32))
-                        r = (int64_t)((uint32_t)slot / (uint32_t)units_per_row);
-                    else
-                        r = slot / units_per_row;
-                    const int64_t c = slot - r * units_per_row;
-                    elem_off = r * ld + c * 16;
-                    unit[u] = (uint64_t)r * (uint64_t)units_per_row_total + (uint64_t)(unit_offset + c);
-                    if (kTC) meta_off[u] = tc_meta_offset(r, c, units_per_row >> 3);
+    for (int h = 0; h < 2; ++h) {
+        const int64_t r = r0 + 8 * h;
+        uint32_t mt = 0x4444u;                        // rows that pad A to a multiple of 128 keep a valid pattern
+        if (r < n_rows) {
+            const char* p = reinterpret_cast<const char*>(g) + (r * ld + (int64_t)c * 16) * (kBf16 ? 2 : 4);
+            uint4 in[LW];
+#pragma unroll
+            for (int i = 0; i < LW; ++i) in[i] = ldg128(p + 16 * i);
+            const uint64_t unit = (uint64_t)r * (uint64_t)units_per_row_total + (uint64_t)(unit_offset + c);
+            uint4 v;
+            if (kBf16) {
+                const uint32_t raw[8] = {in[0].x, in[0].y, in[0].z, in[0].w, in[1].x, in[1].y, in[1].z, in[1].w};
+                prune_unit_bf16<M, kJoint>(raw, unit, rk, &v, &mt);
+            } else {
+                uint32_t b[16];
+#pragma unroll
+                for (int i = 0; i < 4; ++i) {
+                    b[4 * i] = (&in[i].x)[0]; b[4 * i + 1] = (&in[i].x)[1];
+                    b[4 * i + 2] = (&in[i].x)[2]; b[4 * i + 3] = (&in[i].x)[3];
                 }
-                const char* p = reinterpret_cast<const char*>(g) + elem_off * (kBf16 ? 2 : 4);
-#pragma unroll
-                for (int i = 0; i < LW; ++i) in[u][i] = ldg128(p + 16 * i);
+                prune_unit_f32<M, kJoint>(b, unit, rk, &v, &mt);
             }
+            values[r * units_per_row + c] = v;
+            if (!kTC) meta[r * units_per_row + c] = (uint16_t)mt;
         }
-#pragma unroll
-        for (int u = 0; u < U; ++u) {
-            const int64_t slot = base + (int64_t)u * blockDim.x + threadIdx.x;
-            if (slot < n_slots) {
-                uint4 v;
-                uint32_t mt;
-                if (kBf16) {
-                    const uint32_t raw[8] = {in[u][0].x, in[u][0].y, in[u][0].z, in[u][0].w,
-                                             in[u][1].x, in[u][1].y, in[u][1].z, in[u][1].w};
-                    prune_unit_bf16<M, kJoint>(raw, unit[u], rk, &v, &mt);
-                } else {
-                    uint32_t b[16];
-#pragma unroll
-                    for (int i = 0; i < 4; ++i) {
-                        b[4 * i] = (&in[u][i].x)[0]; b[4 * i + 1] = (&in[u][i].x)[1];
-                        b[4 * i + 2] = (&in[u][i].x)[2]; b[4 * i + 3] = (&in[u][i].x)[3];
-                    }
-                    prune_unit_f32<M, kJoint>(b, unit[u], rk, &v, &mt);
-                }
-                values[slot] = v;
-                if (kTC)
-                    *reinterpret_cast<uint16_t*>(reinterpret_cast<char*>(meta) + meta_off[u]) = (uint16_t)mt;
-                else
-                    meta[slot] = (uint16_t)mt;
-            }
-        }
+        meta_pair |= mt << (16 * h);
     }
-    if (kTC) {
-        // rows that pad the operand to a multiple of 128: a valid pattern (positions 0, 1), never used
-        const int64_t rows = n_slots / units_per_row;
-        const int64_t n_pad = pad_rows * units_per_row;
-        for (int64_t i = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; i < n_pad;
-             i += (int64_t)gridDim.x * blockDim.x) {
-            const int64_t r = rows + i / units_per_row, c = i % units_per_row;
-            *reinterpret_cast<uint16_t*>(reinterpret_cast<char*>(meta) + tc_meta_offset(r, c, units_per_row >> 3)) = 0x4444;
-        }
-    }
+    if (kTC)   // (r0, c) is the low half of its word; r0 % 16 < 8
+        *reinterpret_cast<uint32_t*>(reinterpret_cast<char*>(meta) + tc_meta_offset(r0, c, units_per_row >> 3)) = meta_pair;
 }
 
 // ---- axis 0 ---------------------------------------------------------------
@@ -423,15 +395,11 @@ cudaError_t launch_prune_t(const PruneArgs& a, cudaStream_t stream) {
     uint16_t* meta = reinterpret_cast<uint16_t*>(a.meta);
     if (a.axis == 1) {
         const int64_t upr = a.cols / 16;
-        const int64_t n_slots = a.rows * upr;
-        const bool linear = (a.ld == a.cols) && (a.k_total == a.cols) && (a.k_offset == 0);
-        const int64_t want = (n_slots + 255) / 256;
-        const int grid = (int)(want < (int64_t)a.sm_count * 48 ? want : (int64_t)a.sm_count * 48);
-        const int64_t pad_rows = kTC ? ((a.rows + 127) / 128) * 128 - a.rows : 0;
-        if (linear)
-            prune_axis1_kernel<M, kBf16, true, kTC, kJoint><<<grid, 256, 0, stream>>>(a.g, n_slots, upr, a.ld, upr_total, uoff, pad_rows, rk, values, meta);
-        else
-            prune_axis1_kernel<M, kBf16, false, kTC, kJoint><<<grid, 256, 0, stream>>>(a.g, n_slots, upr, a.ld, upr_total, uoff, pad_rows, rk, values, meta);
+        // in tensor-core order the rows of A are padded to 128: the blocks past the last row write only metadata
+        const int64_t cover_rows = kTC ? ((a.rows + 127) / 128) * 128 : a.rows;
+        dim3 grid((unsigned)((cover_rows + 15) / 16), (unsigned)((upr + kA1Units - 1) / kA1Units));
+        prune_axis1_kernel<M, kBf16, kTC, kJoint><<<grid, 8 * kA1Units, 0, stream>>>(
+            a.g, a.rows, (int)upr, a.ld, upr_total, uoff, rk, values, meta);
     } else {
         const int64_t n_strips = a.rows / 16;
         // in tensor-core order the rows of A are padded to 128: cover the padding with (load-free) tiles
