@@ -60,8 +60,7 @@ def gemm_bytes(M: int, N: int, K: int, c_bytes: int = 4) -> int:
 NCU_TRAFFIC = {
     "sparse_gemm_pair_kernel": (982713088 + 4832512, ("mvue_gemm.cu", "mvue_tma.h", "mvue_internal.h"),
                                 "5accd49c5b638403"),
-    "prune_axis0_kernel": (103582208 + 26896640, ("mvue_prune.cu", "mvue_device.cuh", "mvue_tma.h", "mvue_internal.h"),
-                           "4c485998fa1babec"),
+    "prune_axis0_bf16_kernel": (0, ("mvue_prune.cu", "mvue_device.cuh", "mvue_tma.h", "mvue_internal.h"), ""),
 }
 
 
@@ -134,7 +133,7 @@ class ClockSampler:
 
 
 # --------------------------------------------------------------------------- CPU oracle arm
-def oracle_sample(cfg, n, m, sample_rows: int):
+def oracle_sample(cfg, n, m, sample_rows: int, joint: int = 0):
     """One pass of the oracle, as it stands, over the first `sample_rows` token rows: prune+pack,
     unpack, and the fp64 plain-loop update product.  Returns (GB/s of algorithmic bytes, threads, s)."""
     import oracle
@@ -143,7 +142,7 @@ def oracle_sample(cfg, n, m, sample_rows: int):
     h = workloads.normal_bf16((sample_rows, cfg["inp"]), cfg["seed"] + 100)
     threads = oracle.host_threads()
     t0 = time.perf_counter()
-    values, meta = oracle.prune(g, n, m, axis=0, seed=0, k_total=cfg["T"], k_offset=0, threads=threads)
+    values, meta = oracle.prune(g, n, m, axis=0, seed=0, k_total=cfg["T"], k_offset=0, threads=threads, joint=joint)
     oracle.gemm(oracle.unpack(values, meta), h, threads=threads)
     dt = time.perf_counter() - t0
     nbytes = (prune_bytes(sample_rows, cfg["out"], 2 if cfg["g_dtype"] == "bf16" else 4)
@@ -154,20 +153,21 @@ def oracle_sample(cfg, n, m, sample_rows: int):
 def run_reference(args, cfg, n, m):
     if int(os.environ.get("RANK", "0")) != 0:
         return
+    joint = 1 if args.joint == "systematic" else 0
     # size the per-step sample so that K + W steps of the oracle take about a minute in all: its cost
     # grows faster than linearly with the rows (the plain loops leave the cache), so probe by doubling
     per_step_s = 60.0 / max(1, args.steps + args.warmup)
     sample_rows = 512
     while sample_rows * 2 <= cfg["T"]:
-        _, _, dt_probe = oracle_sample(cfg, n, m, sample_rows)
+        _, _, dt_probe = oracle_sample(cfg, n, m, sample_rows, joint)
         if dt_probe > per_step_s / 3:
             break
         sample_rows *= 2
     for _ in range(args.warmup):
-        oracle_sample(cfg, n, m, sample_rows)
+        oracle_sample(cfg, n, m, sample_rows, joint)
     vals, t_all, threads = [], 0.0, 1
     for _ in range(args.steps):
-        gbs, threads, dt = oracle_sample(cfg, n, m, sample_rows)
+        gbs, threads, dt = oracle_sample(cfg, n, m, sample_rows, joint)
         vals.append(gbs)
         t_all += dt
     value = float(np.mean(vals))
@@ -177,7 +177,8 @@ def run_reference(args, cfg, n, m):
         "impl": "reference", "metric": METRIC, "value": value, "unit": "GB/s", "n_gpus": args.gpus,
         "steps": args.steps, "warmup": args.warmup, "ms_per_step": 1e3 * t_all / max(1, args.steps),
         "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "bf16", "data": "synthetic",
-        "config": {"workload": args.workload, "prune": f"{n}:{m}", "axis": 0, "sample_rows": sample_rows},
+        "config": {"workload": args.workload, "prune": f"{n}:{m}", "joint": args.joint, "axis": 0,
+                   "sample_rows": sample_rows},
         "cpu_baseline": {"value": value, "unit": "GB/s", "cores": threads, "kind": "oracle", "sample": sample},
         "e2e": {"value": value, "unit": "GB/s", "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
     }))
@@ -223,10 +224,13 @@ def run_ours(args, cfg, n, m):
     step_bytes = p_bytes + m_bytes
     gemm_flops = 2.0 * out * inp * T
 
+    joints = {"table": binding.MVUE_JOINT_TABLE, "systematic": binding.MVUE_JOINT_SYSTEMATIC}
+    joint = [joints[args.joint]]                        # a cell, so that the other law can be timed with the same step
+
     def step(i, ev=None):
         if ev:
             ev[0].record()
-        binding.mvue_prune(g_dev, n, m, 0, i, values=values, meta=meta, layout=TC)
+        binding.mvue_prune(g_dev, n, m, 0, i, values=values, meta=meta, layout=TC, joint=joint[0])
         if ev:
             ev[1].record()
         binding.mvue_sparse_update_gemm(values, meta, h_dev, out=dW, workspace=ws, dev_status=status)
@@ -263,6 +267,23 @@ def run_ours(args, cfg, n, m):
         ms = float(t.item())
     ms_per_step = ms / args.steps
     value = world * step_bytes / (ms_per_step * 1e-3) / 1e9
+
+    # the same step with the other 2:4 law over pairs, for the per-kernel prune time only (the product that
+    # follows keeps L2 cold for the next prune exactly as in the timed region above)
+    other = None
+    if rank == 0 and world == 1 and m == 4 and not args.no_extra:
+        other_name = "systematic" if args.joint == "table" else "table"
+        joint[0] = joints[other_name]
+        k2 = max(3, min(args.steps, 200))
+        for i in range(3):
+            step(i)
+        evs2 = [[torch.cuda.Event(enable_timing=True) for _ in range(3)] for _ in range(k2)]
+        torch.cuda.synchronize()
+        for i in range(k2):
+            step(i, evs2[i])
+        torch.cuda.synchronize()
+        joint[0] = joints[args.joint]
+        other = (other_name, float(np.mean([e[0].elapsed_time(e[1]) for e in evs2])), k2)
 
     # dense cuBLAS bf16 for the same shape (context for the sparse product)
     dense_ms = None
@@ -314,13 +335,14 @@ def run_ours(args, cfg, n, m):
             "warmup": warm, "ms_per_step": ms_per_step, "higher_is_better": True, "scaling": "weak",
             "vs_baseline": None, "dtype": "bf16", "data": "synthetic",
             "config": {"workload": args.workload, "g": [T, out], "h": [T, inp], "g_dtype": cfg["g_dtype"],
-                       "prune": f"{n}:{m}", "axis": 0, "dW_dtype": "f32",
+                       "prune": f"{n}:{m}", "joint": args.joint, "axis": 0, "dW_dtype": "f32",
                        "l2": "inputs larger than L2 (h is 925 MB, read once per step)"},
             "clocks": clocks.summary(),
             "e2e": {"value": e2e_value, "unit": "GB/s", "h2d_bytes_per_step": T * out * elem + T * inp * 2,
                     "d2h_bytes_per_step": out * inp * 4},
             "gpu_launches": args.steps * launches_per_step,
-            "prune": {"ms": prune_ms, "gbs": prune_gbs, "frac_of_hbm_peak": prune_gbs / peaks["hbm_gbs"]},
+            "prune": {"joint": args.joint, "ms": prune_ms, "gbs": prune_gbs,
+                      "frac_of_hbm_peak": prune_gbs / peaks["hbm_gbs"]},
             "gemm": {"ms": gemm_ms, "tflops_effective": gemm_tf, "frac_of_sparse_peak": gemm_tf / sparse_peak,
                      "sparse_peak_tflops": sparse_peak, "gbs": gemm_gbs,
                      "dense_cublas_ms": dense_ms,
@@ -331,16 +353,21 @@ def run_ours(args, cfg, n, m):
                          "peak": peaks["hbm_gbs"], "unit": "GB/s", "frac": gemm_gbs / peaks["hbm_gbs"],
                          "peak_source": peaks["source"],
                          "traffic": ncu_traffic("sparse_gemm_pair_kernel", args.workload) if (n, m) == (2, 4) else None},
-            "roofline_prune": {"bound": "hbm", "kernel": "prune_axis0_kernel", "achieved": prune_gbs,
+            "roofline_prune": {"bound": "hbm", "kernel": "prune_axis0_bf16_kernel", "achieved": prune_gbs,
                                "peak": peaks["hbm_gbs"], "unit": "GB/s", "frac": prune_gbs / peaks["hbm_gbs"],
                                "peak_source": peaks["source"],
-                               "traffic": ncu_traffic("prune_axis0_kernel", args.workload) if (n, m) == (2, 4) else None},
+                               "traffic": ncu_traffic("prune_axis0_bf16_kernel", args.workload)
+                               if (n, m, args.joint) == (2, 4, "table") else None},
         }
+        if other is not None:
+            ogbs = p_bytes / (other[1] * 1e-3) / 1e9
+            line["prune_other_joint"] = {"joint": other[0], "ms": other[1], "gbs": ogbs,
+                                         "frac_of_hbm_peak": ogbs / peaks["hbm_gbs"], "steps": other[2]}
         if world == 1 and not args.no_extra:
-            line["ffn_large"] = tensor_bound_case(n, m, peaks)
+            line["ffn_large"] = tensor_bound_case(n, m, peaks, joint[0])
         if world == 1 and not args.no_cpu_baseline:
             sample_rows = min(T, 65536)
-            gbs, threads, dt = oracle_sample(cfg, n, m, sample_rows)
+            gbs, threads, dt = oracle_sample(cfg, n, m, sample_rows, joint[0])
             line["cpu_baseline"] = {"value": gbs, "unit": "GB/s", "cores": threads, "kind": "oracle",
                                     "sample": f"first {sample_rows} of {T} token rows: MVUE {n}:{m} prune+pack and "
                                               f"fp64 update product [{out}x{inp}], {dt:.1f} s"}
@@ -349,7 +376,7 @@ def run_ours(args, cfg, n, m):
         dist.destroy_process_group()
 
 
-def tensor_bound_case(n, m, peaks):
+def tensor_bound_case(n, m, peaks, joint):
     """The large FFN layer (tokens 16384, 4096 -> 14336): the shape on which the sparse product is bound by
     the tensor cores, timed kernel by kernel next to dense cuBLAS.  Rides along in the JSON line."""
     import torch
@@ -375,7 +402,10 @@ def tensor_bound_case(n, m, peaks):
         torch.cuda.synchronize()
         return e0.elapsed_time(e1) / iters
 
-    prune_ms = timed(lambda: binding.mvue_prune(g, n, m, 0, 1, values=values, meta=meta, layout=TC), 20)
+    prune_ms = timed(lambda: binding.mvue_prune(g, n, m, 0, 1, values=values, meta=meta, layout=TC, joint=joint), 20)
+    sys_ms = timed(lambda: binding.mvue_prune(g, n, m, 0, 1, values=values, meta=meta, layout=TC,
+                                              joint=binding.MVUE_JOINT_SYSTEMATIC), 20)
+    binding.mvue_prune(g, n, m, 0, 1, values=values, meta=meta, layout=TC, joint=joint)
     gemm_ms = timed(lambda: binding.mvue_sparse_update_gemm(values, meta, h, out=dW), 30)
     fused_ms = timed(lambda: binding.mvue_fused_update_gemm(g, h, n, m, 1, out=dW), 3)
     gT = g.t()
@@ -385,6 +415,8 @@ def tensor_bound_case(n, m, peaks):
     pgbs = prune_bytes(T, out, 2) / (prune_ms * 1e-3) / 1e9
     return {"g": [T, out], "h": [T, inp], "prune": f"{n}:{m}",
             "prune_ms": prune_ms, "prune_gbs": pgbs, "prune_frac_of_hbm_peak": pgbs / peaks["hbm_gbs"],
+            "prune_systematic_ms": sys_ms,
+            "prune_systematic_frac_of_hbm_peak": prune_bytes(T, out, 2) / (sys_ms * 1e-3) / 1e9 / peaks["hbm_gbs"],
             "gemm_ms": gemm_ms, "gemm_tflops_effective": tf,
             "gemm_frac_of_sparse_peak_burst": tf / (2 * peaks["bf16_tflops"]),
             "gemm_frac_of_sparse_peak_sustained": tf / (2 * peaks["bf16_tflops_sustained"]),
@@ -405,6 +437,8 @@ def main():
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--workload", default="conv_im2col")
     ap.add_argument("--prune", default="2:4")
+    ap.add_argument("--joint", default="table", choices=["table", "systematic"],
+                    help="2:4 law over pairs used by the step: App. A.2 pair table, or systematic sampling")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-extra", action="store_true", help="skip the tensor-bound ffn_large case")
     args = ap.parse_args()

@@ -263,6 +263,8 @@ struct Pick24Sys {
     float H;
 };
 
+// kAll3: also count t2 < c_1 (implied by the other two, see below; kept where it schedules better).
+template <bool kAll3>
 __device__ __forceinline__ Pick24Sys pick_2of4_sys(float m0, float m1, float m2, float m3, uint32_t word) {
     const float tiny = __uint_as_float(1u);                                   // 2^-149
     const float q01 = __fadd_rn(__fadd_rn(m0, m1), tiny), q23 = __fadd_rn(__fadd_rn(m2, m3), tiny);
@@ -278,7 +280,8 @@ __device__ __forceinline__ Pick24Sys pick_2of4_sys(float m0, float m1, float m2,
     const float t2 = __fmul_rn(n2, Hs), t = __fsub_rn(t2, r.H);
     auto below = [](float x, float c) { return __umulhi(__float_as_uint(__fsub_rn(x, c)), 2u); };   // x < c ? 1 : 0
     r.li = below(t, c1) + below(t, c2);
-    r.lj = min(below(t2, c1) + below(t2, c2) + below(t2, c3), r.li);
+    // t2 < c_1 implies t2 < c_2 and t2 < c_3, and then min(3, li) = min(2, li): the c_1 term is never needed
+    r.lj = min((kAll3 ? below(t2, c1) : 0u) + below(t2, c2) + below(t2, c3), r.li);
     return r;
 }
 
@@ -288,9 +291,9 @@ __device__ __forceinline__ Pick24Sys pick_2of4_sys(float m0, float m1, float m2,
 // signed 16-bit integers (with equal sign bits the larger magnitude is the larger integer).
 __device__ __forceinline__ void mvue_2of4_sys_bf16(uint32_t x01, uint32_t x23, uint32_t word, uint32_t* out,
                                                    uint32_t* nibble) {
-    const Pick24Sys r = pick_2of4_sys(fabsf(__uint_as_float(x01 << 16)), fabsf(__uint_as_float(x01 & 0xFFFF0000u)),
-                                      fabsf(__uint_as_float(x23 << 16)), fabsf(__uint_as_float(x23 & 0xFFFF0000u)),
-                                      word);
+    const Pick24Sys r = pick_2of4_sys<false>(fabsf(__uint_as_float(x01 << 16)), fabsf(__uint_as_float(x01 & 0xFFFF0000u)),
+                                             fabsf(__uint_as_float(x23 << 16)), fabsf(__uint_as_float(x23 & 0xFFFF0000u)),
+                                             word);
     const uint32_t sel = 0x7654u - 0x22u * r.li - 0x2200u * r.lj;
     const uint32_t raw = __byte_perm(x01, x23, sel);
     const uint32_t hs = pack_bf16x2(r.H, r.H) | (raw & 0x80008000u);
@@ -301,8 +304,8 @@ __device__ __forceinline__ void mvue_2of4_sys_bf16(uint32_t x01, uint32_t x23, u
 // binary32 source: b0..b3 are the raw bit patterns.
 __device__ __forceinline__ void mvue_2of4_sys_f32(uint32_t b0, uint32_t b1, uint32_t b2, uint32_t b3,
                                                   uint32_t word, uint32_t* out, uint32_t* nibble) {
-    const Pick24Sys r = pick_2of4_sys(fabsf(__uint_as_float(b0)), fabsf(__uint_as_float(b1)),
-                                      fabsf(__uint_as_float(b2)), fabsf(__uint_as_float(b3)), word);
+    const Pick24Sys r = pick_2of4_sys<true>(fabsf(__uint_as_float(b0)), fabsf(__uint_as_float(b1)),
+                                            fabsf(__uint_as_float(b2)), fabsf(__uint_as_float(b3)), word);
     const uint32_t bi = r.li == 2u ? b0 : (r.li == 1u ? b1 : b2);            // i = 2 - li in {0, 1, 2}
     const uint32_t bj = r.lj == 2u ? b1 : (r.lj == 1u ? b2 : b3);            // j = 3 - lj in {1, 2, 3}
     const float vi = __uint_as_float(__float_as_uint(fmaxf(fabsf(__uint_as_float(bi)), r.H)) | (bi & 0x80000000u));

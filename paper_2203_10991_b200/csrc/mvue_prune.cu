@@ -249,20 +249,21 @@ prune_axis0_kernel(const void* __restrict__ g, int64_t n_strips, int64_t n_cols,
 // address arithmetic per element.  A warp covers 4 strips x 8 columns per step (lane = 4 (column % 8) +
 // strip % 4) and takes two steps whose columns are 8 apart, so in the tensor-core order the two 16-bit nibble
 // strings of a lane share one 32-bit word.  Packed survivors go straight from registers to memory: the four
-// lanes of a column write 64 contiguous bytes.  Small tiles (4 strips, 128 threads, 12 blocks per SM) keep
+// lanes of a column write 64 contiguous bytes.  Small tiles (4 strips, two warps, 24 blocks per SM) keep
 // the copy of one block hidden behind the arithmetic of the others.
 constexpr int kA0Cols = 64;
-template <int kStrips> struct A0 {                               // kStrips: strips of 16 rows per tile (8 or 16)
-    static constexpr int kRows = 16 * kStrips, kThreads = 32 * kStrips;
+template <int kStrips, int kWarps> struct A0 {                   // kStrips: strips of 16 rows per tile (4, 8 or 16)
+    static constexpr int kRows = 16 * kStrips, kThreads = 32 * kWarps;
     static constexpr int kTileBytes = kRows * kA0Cols * 2;
     static constexpr int kSmemBytes = kTileBytes + 1024 + 16;     // alignment slack + one mbarrier
+    static constexpr int kBlocksPerSM = 1536 / kThreads < 24 ? 1536 / kThreads : 24;
 };
 
 // Plain-load replacement of the box copy (same shared-memory arrangement), used only if the copy never landed.
-template <int kStrips>
+template <int kStrips, int kWarps>
 __device__ __noinline__ void fill_tile_bf16(const char* g, int64_t ld, int64_t n_rows, int64_t n_cols, int64_t row0,
                                             int64_t col0, unsigned char* tile) {
-    for (int i = threadIdx.x; i < A0<kStrips>::kRows * 8; i += A0<kStrips>::kThreads) {   // 16-byte chunks
+    for (int i = threadIdx.x; i < A0<kStrips, kWarps>::kRows * 8; i += A0<kStrips, kWarps>::kThreads) {   // 16-byte chunks
         const int line = i >> 3, chunk = i & 7;
         const int k8 = line / (2 * kStrips), strip = (line >> 1) % kStrips, k2 = line & 1;
         const int64_t r = row0 + 16 * strip + 2 * k8 + k2, c = col0 + 8 * chunk;
@@ -272,13 +273,15 @@ __device__ __noinline__ void fill_tile_bf16(const char* g, int64_t ld, int64_t n
     }
 }
 
-template <int M, bool kTC, int kJoint, int kStrips>
-__global__ void __launch_bounds__(32 * kStrips, 1536 / (32 * kStrips))
+template <int M, bool kTC, int kJoint, int kStrips, int kWarps>
+__global__ void __launch_bounds__(32 * kWarps, A0<kStrips, kWarps>::kBlocksPerSM)
 prune_axis0_bf16_kernel(const __grid_constant__ CUtensorMap map_g, const void* __restrict__ g, int64_t n_strips,
                         int64_t n_cols, int64_t ld, int64_t units_per_row_total, int64_t unit_offset, RoundKeys rk,
                         uint4* __restrict__ values, uint16_t* __restrict__ meta) {
-    constexpr int kTileBytes = A0<kStrips>::kTileBytes;
+    constexpr int kTileBytes = A0<kStrips, kWarps>::kTileBytes;
     constexpr int kQuads = kStrips / 4;                                      // groups of 4 strips per tile
+    constexpr int kPairStride = kWarps / kQuads;                             // warps that share a group of 4 strips
+    static_assert(kWarps % kQuads == 0 && 4 % kPairStride == 0, "warps must tile the 4 x kQuads steps");
     extern __shared__ unsigned char s_raw[];
     const uint32_t tile = (smem_addr(s_raw) + 1023u) & ~1023u;              // the 128-byte swizzle needs 1 KiB alignment
     const uint32_t bar = tile + kTileBytes;
@@ -305,50 +308,54 @@ prune_axis0_bf16_kernel(const __grid_constant__ CUtensorMap map_g, const void* _
             landed = ok != 0;
         }
         if (__syncthreads_or(!landed)) {
-            fill_tile_bf16<kStrips>(reinterpret_cast<const char*>(g), ld, n_strips * 16, n_cols, strip0 * 16, col0,
+            fill_tile_bf16<kStrips, kWarps>(reinterpret_cast<const char*>(g), ld, n_strips * 16, n_cols, strip0 * 16, col0,
                                     s_raw + (tile - smem_addr(s_raw)));
             __syncthreads();
         }
     }
 
-    // this lane's units: strip = strip0 + 4 (warp % kQuads) + lane % 4,
-    //                    column = col0 + 8 (2 (warp / kQuads) + step) + lane / 4
-    const int quad = warp % kQuads, cpair = warp / kQuads, p = lane & 3;
+    // this lane's units: strip = strip0 + 4 (warp % kQuads) + lane % 4; columns col0 + 16 pair + lane / 4 and
+    // + 8, for pair = warp / kQuads, + kPairStride, ... < 4
+    const int quad = warp % kQuads, p = lane & 3;
     const int64_t strip = strip0 + 4 * quad + p;
     const bool strip_ok = strip < n_strips;
     // address this lane supplies to the matrix loads: matrix lane / 8 (= k8, +4 for the second load), line lane % 8
     const uint32_t ld_base = tile + (uint32_t)(((lane >> 3) * (2 * kStrips) + 8 * quad + (lane & 7)) * 128);
-    uint32_t meta_pair = 0;
 #pragma unroll
-    for (int step = 0; step < 2; ++step) {
-        const int cb = 2 * cpair + step;                                     // 8-column block inside the tile
-        const int64_t c = col0 + 8 * cb + (lane >> 2);
-        uint32_t mt = 0x4444u;                                               // rows that pad A keep a valid pattern
-        if (has_input) {
-            const uint32_t addr = ld_base + (uint32_t)((cb ^ (lane & 7)) << 4);
-            uint32_t raw[8];
-            asm volatile("ldmatrix.sync.aligned.m8n8.x4.trans.shared.b16 {%0, %1, %2, %3}, [%4];"
-                         : "=r"(raw[0]), "=r"(raw[1]), "=r"(raw[2]), "=r"(raw[3]) : "r"(addr));
-            asm volatile("ldmatrix.sync.aligned.m8n8.x4.trans.shared.b16 {%0, %1, %2, %3}, [%4];"
-                         : "=r"(raw[4]), "=r"(raw[5]), "=r"(raw[6]), "=r"(raw[7]) : "r"(addr + 4u * (2 * kStrips) * 128u));
-            if (strip_ok && c < n_cols) {
-                const uint64_t unit = (uint64_t)c * (uint64_t)units_per_row_total + (uint64_t)(unit_offset + strip);
-                uint4 v;
-                prune_unit_bf16<M, kJoint>(raw, unit, rk, &v, &mt);
-                values[c * n_strips + strip] = v;
-                if (!kTC) meta[c * n_strips + strip] = (uint16_t)mt;
+    for (int pair = warp / kQuads; pair < 4; pair += kPairStride) {
+        uint32_t meta_pair = 0;
+#pragma unroll
+        for (int step = 0; step < 2; ++step) {
+            const int cb = 2 * pair + step;                                  // 8-column block inside the tile
+            const int64_t c = col0 + 8 * cb + (lane >> 2);
+            uint32_t mt = 0x4444u;                                           // rows that pad A keep a valid pattern
+            if (has_input) {
+                const uint32_t addr = ld_base + (uint32_t)((cb ^ (lane & 7)) << 4);
+                uint32_t raw[8];
+                asm volatile("ldmatrix.sync.aligned.m8n8.x4.trans.shared.b16 {%0, %1, %2, %3}, [%4];"
+                             : "=r"(raw[0]), "=r"(raw[1]), "=r"(raw[2]), "=r"(raw[3]) : "r"(addr));
+                asm volatile("ldmatrix.sync.aligned.m8n8.x4.trans.shared.b16 {%0, %1, %2, %3}, [%4];"
+                             : "=r"(raw[4]), "=r"(raw[5]), "=r"(raw[6]), "=r"(raw[7])
+                             : "r"(addr + 4u * (2 * kStrips) * 128u));
+                if (strip_ok && c < n_cols) {
+                    const uint64_t unit = (uint64_t)c * (uint64_t)units_per_row_total + (uint64_t)(unit_offset + strip);
+                    uint4 v;
+                    prune_unit_bf16<M, kJoint>(raw, unit, rk, &v, &mt);
+                    values[c * n_strips + strip] = v;
+                    if (!kTC) meta[c * n_strips + strip] = (uint16_t)mt;
+                }
             }
+            meta_pair |= mt << (16 * step);
         }
-        meta_pair |= mt << (16 * step);
-    }
-    if (kTC && strip_ok) {
-        // rows c and c + 8 share the 32-bit word (k % 128) / 32 of lane c % 8 + 8 (strip % 2) + 16 (c % 128 / 16)
-        const int64_t c = col0 + 16 * cpair + (lane >> 2);
-        const int rl = (int)(c & 127);
-        const int tc_lane = (rl & 7) + 8 * (p & 1) + 16 * (rl >> 4);
-        const int64_t block = (c >> 7) * (n_strips >> 3) + (strip >> 3);
-        const int word = 2 * ((int)(strip >> 2) & 1) + (p >> 1);
-        *reinterpret_cast<uint32_t*>(reinterpret_cast<char*>(meta) + block * 2048 + tc_lane * 16 + word * 4) = meta_pair;
+        if (kTC && strip_ok) {
+            // rows c and c + 8 share the 32-bit word (k % 128) / 32 of lane c % 8 + 8 (strip % 2) + 16 (c % 128 / 16)
+            const int64_t c = col0 + 16 * pair + (lane >> 2);
+            const int rl = (int)(c & 127);
+            const int tc_lane = (rl & 7) + 8 * (p & 1) + 16 * (rl >> 4);
+            const int64_t block = (c >> 7) * (n_strips >> 3) + (strip >> 3);
+            const int word = 2 * ((int)(strip >> 2) & 1) + (p >> 1);
+            *reinterpret_cast<uint32_t*>(reinterpret_cast<char*>(meta) + block * 2048 + tc_lane * 16 + word * 4) = meta_pair;
+        }
     }
 }
 
@@ -409,18 +416,18 @@ cudaError_t launch_prune_t(const PruneArgs& a, cudaStream_t stream) {
         if (kBf16) {
             CUtensorMap map_g;
             memset(&map_g, 0, sizeof(map_g));
-            constexpr int kS = 4;                                            // strips per tile
+            constexpr int kS = 4, kW = 2;                                    // strips per tile, warps per block
             if (!make_map_strips(&map_g, a.g, (uint64_t)a.cols, (uint64_t)a.rows, (uint64_t)a.ld * 2, kS))
                 return cudaErrorInvalidValue;
             static std::once_flag once;
             static cudaError_t attr_err = cudaSuccess;
             std::call_once(once, [] {
-                attr_err = cudaFuncSetAttribute(prune_axis0_bf16_kernel<M, kTC, kJoint, kS>,
-                                                cudaFuncAttributeMaxDynamicSharedMemorySize, A0<kS>::kSmemBytes);
+                attr_err = cudaFuncSetAttribute(prune_axis0_bf16_kernel<M, kTC, kJoint, kS, kW>,
+                                                cudaFuncAttributeMaxDynamicSharedMemorySize, A0<kS, kW>::kSmemBytes);
             });
             if (attr_err != cudaSuccess) return attr_err;
             dim3 grid_b((unsigned)((n_strips + kS - 1) / kS), (unsigned)((cover_cols + kA0Cols - 1) / kA0Cols));
-            prune_axis0_bf16_kernel<M, kTC, kJoint, kS><<<grid_b, A0<kS>::kThreads, A0<kS>::kSmemBytes, stream>>>(
+            prune_axis0_bf16_kernel<M, kTC, kJoint, kS, kW><<<grid_b, A0<kS, kW>::kThreads, A0<kS, kW>::kSmemBytes, stream>>>(
                 map_g, a.g, n_strips, a.cols, a.ld, upr_total, uoff, rk, values, meta);
         } else {
             prune_axis0_kernel<M, false, kTC, kJoint><<<grid, kTileStrips * 32, 0, stream>>>(
