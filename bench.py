@@ -366,6 +366,7 @@ def run_ours(args, cfg, n, m):
                                          "frac_of_hbm_peak": ogbs / peaks["hbm_gbs"], "steps": other[2]}
         if world == 1 and not args.no_extra:
             line["ffn_large"] = tensor_bound_case(n, m, peaks, joint[0])
+            line["mlp_stack"] = chain_case(n, m)
         if world == 1 and not args.no_cpu_baseline:
             sample_rows = min(T, 65536)
             gbs, threads, dt = oracle_sample(cfg, n, m, sample_rows, joint[0])
@@ -430,6 +431,61 @@ def tensor_bound_case(n, m, peaks, joint):
                          "peak_source": peaks["source"] + " dense bf16 burst x 2 (2:4 sparse)", "traffic": None}}
 
 
+def chain_case(n, m):
+    """The MLP-stack workload: backward + update chain of 12 blocks x (1024 -> 4096, activation, 4096 -> 1024) over
+    T = 32768 tokens, every neural gradient MVUE-pruned (prune along tokens -> sparse update product; independent
+    prune along the features -> sparse backward product with the f'(z) epilogue), timed as a whole next to the same
+    chain with dense bf16 matmuls.  Activations and f'(z) are seeded random tensors of the right shapes (the forward
+    pass is not part of the path)."""
+    import torch
+    from paper_2203_10991_b200 import binding, chain, workloads
+    cfg = workloads.CONFIGS["mlp_stack"]
+    T, d_ff, d = cfg["T"], cfg["out"], cfg["inp"]
+    dev = torch.device("cuda")
+    gen = torch.Generator(device=dev).manual_seed(cfg["seed"])
+    layers = []
+    for i in range(2 * cfg["layers"]):                      # top layer first: [d <- d_ff], [d_ff <- d], ...
+        out_f, in_f = (d, d_ff) if i % 2 == 0 else (d_ff, d)
+        layers.append({
+            "W": (torch.randn((out_f, in_f), generator=gen, device=dev) * in_f ** -0.5).to(torch.bfloat16),
+            "h": torch.randn((T, in_f), generator=gen, device=dev).to(torch.bfloat16),
+            "act_grad": None if i == 2 * cfg["layers"] - 1 else
+                        torch.rand((T, in_f), generator=gen, device=dev).to(torch.bfloat16)})
+    g_host = workloads.gradient((T, d), cfg["g_dist"], cfg["seed"], dtype="bf16")
+    g_top = torch.from_numpy(g_host.view(np.int16)).to(dev).view(torch.bfloat16)
+
+    def dense_chain():
+        g = g_top
+        for L in layers:
+            torch.matmul(g.t(), L["h"])
+            if L["act_grad"] is not None:
+                g = torch.matmul(g, L["W"]) * L["act_grad"]
+
+    def timed(fn, iters):
+        fn()
+        torch.cuda.synchronize()
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record()
+        for _ in range(iters):
+            fn()
+        e1.record()
+        torch.cuda.synchronize()
+        return e0.elapsed_time(e1) / iters
+
+    table_ms = timed(lambda: chain.backward_update(g_top, layers, n, m, base_seed=1), 5)
+    sys_ms = timed(lambda: chain.backward_update(g_top, layers, n, m, base_seed=1,
+                                                 joint=binding.MVUE_JOINT_SYSTEMATIC), 5) if m == 4 else None
+    dense_ms = timed(dense_chain, 5)
+    n_layers = len(layers)
+    flops = 2.0 * T * d * d_ff * (2 * n_layers - 1)         # update product per layer, backward for all but the bottom
+    return {"layers": n_layers, "T": T, "d": d, "d_ff": d_ff, "prune": f"{n}:{m}",
+            "launches_per_chain": 4 * n_layers - 2,
+            "ms": table_ms, "tflops_effective": flops / (table_ms * 1e-3) / 1e12,
+            "systematic_ms": sys_ms,
+            "systematic_tflops_effective": None if sys_ms is None else flops / (sys_ms * 1e-3) / 1e12,
+            "dense_torch_ms": dense_ms, "dense_torch_tflops": flops / (dense_ms * 1e-3) / 1e12}
+
+
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
@@ -441,7 +497,8 @@ def main():
     ap.add_argument("--joint", default="table", choices=["table", "systematic"],
                     help="2:4 law over pairs used by the step: App. A.2 pair table, or systematic sampling")
     ap.add_argument("--no-cpu-baseline", action="store_true")
-    ap.add_argument("--no-extra", action="store_true", help="skip the tensor-bound ffn_large case")
+    ap.add_argument("--no-extra", action="store_true",
+                    help="skip the riders: the other 2:4 law, the tensor-bound ffn_large case and the MLP-stack chain")
     args = ap.parse_args()
     from paper_2203_10991_b200 import workloads
     cfg = workloads.CONFIGS[args.workload]

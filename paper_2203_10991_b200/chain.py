@@ -22,18 +22,19 @@ def layer_seeds(base_seed: int, layer: int) -> tuple[int, int]:
            (base_seed * 0x9E3779B97F4A7C15 + 2 * layer + 1) & (2**64 - 1)
 
 
-def backward_update(g_top: torch.Tensor, layers, n: int = 2, m: int = 4, base_seed: int = 0):
+def backward_update(g_top: torch.Tensor, layers, n: int = 2, m: int = 4, base_seed: int = 0, joint: int | None = None):
     """layers: list (top layer first) of dicts {"W": [out x in] bf16, "h": [T x in] bf16,
     "act_grad": [T x in] bf16 or None (None for the bottom layer: no gradient is propagated further)}.
+    joint: the 2:4 law over pairs handed to mvue_prune_joint (None: mvue_prune, the App. A.2 table).
     Returns the list of dW (fp32), top layer first."""
     g = g_top
     grads = []
     for i, L in enumerate(layers):
         s_upd, s_bwd = layer_seeds(base_seed, i)
-        values, meta = binding.mvue_prune(g, n, m, 0, s_upd, layout=TC)
+        values, meta = binding.mvue_prune(g, n, m, 0, s_upd, layout=TC, joint=joint)
         grads.append(binding.mvue_sparse_update_gemm(values, meta, L["h"]))
         if L.get("act_grad") is not None:
-            values, meta = binding.mvue_prune(g, n, m, 1, s_bwd, layout=TC)
+            values, meta = binding.mvue_prune(g, n, m, 1, s_bwd, layout=TC, joint=joint)
             g = binding.mvue_sparse_backward_gemm(values, meta, L["W"], act_grad=L["act_grad"],
                                                   out_dtype=torch.bfloat16)
     return grads

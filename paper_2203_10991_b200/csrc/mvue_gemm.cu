@@ -123,9 +123,12 @@ struct GemmParams {
 
 // Epilogue of one thread: its accumulator row (32 columns at a time from tensor memory) goes to the
 // split-K workspace, or through the optional elementwise scale / accumulate / bf16 conversion to C.
+// kPre: the row's scale factors were loaded into registers (sc[c / 8] = columns c .. c + 7) while the main loop
+// ran, so the drain never waits on memory; the column loop is then unrolled so that sc[] stays in registers.
+template <bool kPre>
 __device__ __forceinline__ void epilogue_rows(const GemmParams& p, int split, int64_t row, int64_t n0,
-                                              uint32_t tmem_rows, bool have_acc) {
-#pragma unroll 1
+                                              uint32_t tmem_rows, bool have_acc, const uint4* sc_pre) {
+#pragma unroll(kPre ? BN / 32 : 1)
     for (int c = 0; c < BN; c += 32) {
         uint32_t v[32];
         if (have_acc) {
@@ -150,8 +153,9 @@ __device__ __forceinline__ void epilogue_rows(const GemmParams& p, int split, in
                     float f[8];
 #pragma unroll
                     for (int t = 0; t < 8; ++t) f[t] = __uint_as_float(v[e + t]);
-                    if (p.scale) {
-                        const uint4 sc = *reinterpret_cast<const uint4*>(p.scale + row * p.ldc + col0 + e);
+                    if (kPre || p.scale) {
+                        const uint4 sc = kPre ? sc_pre[(c + e) / 8]
+                                              : *reinterpret_cast<const uint4*>(p.scale + row * p.ldc + col0 + e);
                         const uint32_t sw[4] = {sc.x, sc.y, sc.z, sc.w};
 #pragma unroll
                         for (int t = 0; t < 4; ++t) {
@@ -264,6 +268,8 @@ __device__ __forceinline__ void tc_mma_sp_bf16_pair(uint32_t tmem_d, uint64_t a_
         ::"r"(tmem_d), "l"(a_desc), "l"(b_desc), "r"(tmem_meta), "r"(idesc), "r"(accumulate), "r"(zero) : "memory");
 }
 
+// kScale: the result is multiplied elementwise by p.scale and is not split along K.
+template <bool kScale>
 __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(kThreads, 1)
 sparse_gemm_pair_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ CUtensorMap map_b,
                         const __grid_constant__ CUtensorMap map_e, const GemmParams p) {
@@ -379,10 +385,20 @@ sparse_gemm_pair_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_
     } else if (warp >= 4) {
         // ------------------------------------------------------------ epilogue (both blocks, own rows)
         const int q = warp - 4;                                  // lanes 32 q .. 32 q + 31
+        const int64_t row = m0 + 32 * q + lane;
+        uint4 sc[kScale ? BN / 8 : 1];
+        if (kScale) {                                            // this row's scale factors, fetched under the main loop
+#pragma unroll
+            for (int e = 0; e < BN / 8; ++e) {
+                sc[e] = make_uint4(0u, 0u, 0u, 0u);
+                if (row < p.M && n0 + 8 * e < p.N)
+                    sc[e] = __ldg(reinterpret_cast<const uint4*>(p.scale + row * p.ldc + n0 + 8 * e));
+            }
+        }
         const bool acc_ok = n_steps > 0 ? mbar_wait(acc_bar, 0, abort_flag) : true;
         tc_fence_after();
-        const int64_t row = m0 + 32 * q + lane;
-        if (acc_ok) epilogue_rows(p, split, row, n0, tmem_base + ((uint32_t)(32 * q) << 16), n_steps > 0);
+        if (acc_ok)
+            epilogue_rows<kScale>(p, split, row, n0, tmem_base + ((uint32_t)(32 * q) << 16), n_steps > 0, sc);
     }
 
     tc_fence_before();
@@ -519,7 +535,8 @@ fused_update_kernel(const __grid_constant__ CUtensorMap map_b, const FusedParams
         const bool acc_ok = n_steps > 0 ? mbar_wait(acc_bar, 0, abort_flag) : true;
         tc_fence_after();
         const int64_t row = m0 + 32 * q + lane;
-        if (acc_ok) epilogue_rows(p, split, row, n0, tmem_base + ((uint32_t)(32 * q) << 16), n_steps > 0);
+        if (acc_ok)
+            epilogue_rows<false>(p, split, row, n0, tmem_base + ((uint32_t)(32 * q) << 16), n_steps > 0, nullptr);
     } else if (warp >= 8) {
         // ------------------------------------------------------------ prune warps
         const int strip_l = warp - 8;                               // 16-token strip of the stage
@@ -742,8 +759,11 @@ int launch_sparse_gemm(const SparseGemmArgs& a, cudaStream_t stream) {
     static std::once_flag once;
     static cudaError_t attr_err = cudaSuccess;
     std::call_once(once, [] {
-        attr_err = cudaFuncSetAttribute(sparse_gemm_pair_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
+        attr_err = cudaFuncSetAttribute(sparse_gemm_pair_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                         kSmemBytes);
+        if (attr_err == cudaSuccess)
+            attr_err = cudaFuncSetAttribute(sparse_gemm_pair_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                            kSmemBytes);
     });
     if (attr_err != cudaSuccess) { set_cuda_error(attr_err, "cudaFuncSetAttribute"); return MVUE_ERR_CUDA; }
 
@@ -758,7 +778,10 @@ int launch_sparse_gemm(const SparseGemmArgs& a, cudaStream_t stream) {
     p.c_is_bf16 = a.c_is_bf16; p.accumulate = a.accumulate; p.splits = splits;
     p.dev_status = a.dev_status;
     dim3 grid((unsigned)(2 * ((a.M + 2 * BM - 1) / (2 * BM)) * ((a.N + BN - 1) / BN)), 1u, (unsigned)splits);
-    sparse_gemm_pair_kernel<<<grid, kThreads, kSmemBytes, stream>>>(map_a, map_b, map_e, p);
+    if (p.scale != nullptr && splits == 1)
+        sparse_gemm_pair_kernel<true><<<grid, kThreads, kSmemBytes, stream>>>(map_a, map_b, map_e, p);
+    else
+        sparse_gemm_pair_kernel<false><<<grid, kThreads, kSmemBytes, stream>>>(map_a, map_b, map_e, p);
     cudaError_t e = cudaGetLastError();
     if (e == cudaSuccess && splits > 1) {
         const int64_t total = a.M * (a.N / 4);
