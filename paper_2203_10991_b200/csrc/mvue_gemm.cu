@@ -46,7 +46,8 @@ constexpr int kBBytes = (BN / 2 / 64) * kBBoxBytes;   // this block's 128 column
 constexpr int kEBytes = BM * 16;           // 2 KiB: 16 bytes per tensor-memory lane
 constexpr int kStageBytes = kABytes + kBBytes + kEBytes;
 constexpr int kSmemBytes = kStages * kStageBytes + 1024 /*alignment slack*/ + 256 /*barriers*/;
-constexpr int kThreads = 256;
+constexpr int kThreads = 352;            // pair kernel: producer, MMA, allocator and 8 epilogue warps
+constexpr int kEpiWarps = 8;
 constexpr int kBandTiles = 8;              // row tiles per band of the tile order
 constexpr uint32_t kTmemCols = 512;
 constexpr uint32_t kTmemECol = 256;        // metadata columns start after the accumulator
@@ -66,6 +67,25 @@ __device__ __forceinline__ bool mbar_try_wait(uint32_t bar, uint32_t parity) {
         "selp.u32 %0, 1, 0, p;\n\t}"
         : "=r"(ok) : "r"(bar), "r"(parity) : "memory");
     return ok != 0;
+}
+// The same test with acquire semantics at cluster scope: for a barrier that the peer block arrives on.
+__device__ __forceinline__ bool mbar_try_wait_cluster(uint32_t bar, uint32_t parity) {
+    uint32_t ok;
+    asm volatile(
+        "{\n\t.reg .pred p;\n\t"
+        "mbarrier.try_wait.parity.acquire.cluster.shared::cta.b64 p, [%1], %2;\n\t"
+        "selp.u32 %0, 1, 0, p;\n\t}"
+        : "=r"(ok) : "r"(bar), "r"(parity) : "memory");
+    return ok != 0;
+}
+__device__ __forceinline__ bool mbar_wait_cluster(uint32_t bar, uint32_t parity, volatile int* abort_flag) {
+    for (uint32_t spin = 0; spin < (1u << 22); ++spin) {
+        if (mbar_try_wait_cluster(bar, parity)) return true;
+        if (*abort_flag) return false;
+        if (spin > 64) __nanosleep(spin > 4096 ? 256 : 32);
+    }
+    *abort_flag = 1;
+    return false;
 }
 // Bounded wait.  Returns false (and raises the block's abort flag) when the bound expires
 // or another role has already given up.
@@ -118,6 +138,7 @@ struct GemmParams {
     int c_is_bf16;
     int accumulate;
     int splits;
+    int64_t n_work;           // tiles x splits (pair kernel)
     int* dev_status;
 };
 
@@ -268,8 +289,60 @@ __device__ __forceinline__ void tc_mma_sp_bf16_pair(uint32_t tmem_d, uint64_t a_
         ::"r"(tmem_d), "l"(a_desc), "l"(b_desc), "r"(tmem_meta), "r"(idesc), "r"(accumulate), "r"(zero) : "memory");
 }
 
-// kScale: the result is multiplied elementwise by p.scale and is not split along K.
-template <bool kScale>
+// One work item of the persistent pair kernel: an output tile (of one K split).
+struct WorkItem {
+    int64_t m_block, m0, n0;      // this block's 128-row block of A, its first row, the pair's first column
+    int split;
+    int64_t step_begin, n_steps;
+};
+
+// Work items are numbered split-major; inside a split the tiles go in bands of kBandTiles row tiles, row tile
+// fastest inside a band, so that the pairs running at the same time cover a compact block of the output and
+// share their A and B tiles in L2.
+__device__ __forceinline__ WorkItem decode_work(const GemmParams& p, int64_t w, uint32_t rank) {
+    const int64_t tiles_m = (p.M + 2 * BM - 1) / (2 * BM), tiles_n = (p.N + BN - 1) / BN;
+    const int64_t n_tiles = tiles_m * tiles_n;
+    WorkItem it;
+    it.split = (int)(w / n_tiles);
+    const int64_t pair_id = w - (int64_t)it.split * n_tiles;
+    const int64_t band = pair_id / (kBandTiles * tiles_n);
+    const int64_t band_h = tiles_m - band * kBandTiles < kBandTiles ? tiles_m - band * kBandTiles : kBandTiles;
+    const int64_t in_band = pair_id - band * kBandTiles * tiles_n;
+    const int64_t tile_m = band * kBandTiles + in_band % band_h, tile_n = in_band / band_h;
+    it.m_block = tile_m * 2 + rank;
+    it.m0 = it.m_block * BM;
+    it.n0 = tile_n * BN;
+    const int64_t total_steps = p.K / BK;
+    it.step_begin = (int64_t)it.split * p.k_steps_per_split;
+    int64_t step_end = it.step_begin + p.k_steps_per_split;
+    if (step_end > total_steps) step_end = total_steps;
+    it.n_steps = step_end > it.step_begin ? step_end - it.step_begin : 0;
+    return it;
+}
+
+// 8 values of one row to 32-byte-aligned memory in one store where the address allows, else two 16-byte stores.
+__device__ __forceinline__ void store8_b32(void* dst, const uint32_t* v) {
+    if ((reinterpret_cast<uintptr_t>(dst) & 31u) == 0) {
+        asm volatile("st.global.v8.b32 [%0], {%1, %2, %3, %4, %5, %6, %7, %8};"
+                     ::"l"(dst), "r"(v[0]), "r"(v[1]), "r"(v[2]), "r"(v[3]), "r"(v[4]), "r"(v[5]), "r"(v[6]), "r"(v[7])
+                     : "memory");
+    } else {
+        reinterpret_cast<uint4*>(dst)[0] = make_uint4(v[0], v[1], v[2], v[3]);
+        reinterpret_cast<uint4*>(dst)[1] = make_uint4(v[4], v[5], v[6], v[7]);
+    }
+}
+
+// Persistent kernel: every pair of thread blocks walks the work items pair, pair + #pairs, ...
+//   warp 0      TMA producer (both blocks); runs ahead into the next tile while the current one drains
+//   warp 1      metadata copy + MMA issue (leader block only)
+//   warp 2      tensor-memory allocation
+//   warps 3-10  epilogue: warp w drains lanes 32 (w % 4) .. of columns 128 ((w - 3) / 4) .. into registers,
+//               hands the accumulator back to the MMA warp at once, and only then converts and stores, so the
+//               stores of one tile overlap the main loop of the next
+// kMode fixes the output path at compile time so that the drained tile fits the register file:
+//   0: fp32 (C, C +=, or the split-K workspace)   1: bf16   2: bf16 times p.scale   3: fp32 times p.scale
+// The scale factors of a row are fetched into registers under the main loop.
+template <int kMode>
 __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(kThreads, 1)
 sparse_gemm_pair_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ CUtensorMap map_b,
                         const __grid_constant__ CUtensorMap map_e, const GemmParams p) {
@@ -279,29 +352,15 @@ sparse_gemm_pair_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_
     const uint32_t bar_base = smem_base + kStages * kStageBytes;
     auto full_bar = [&](int s) { return bar_base + 8u * s; };                 // used in the leader only
     auto empty_bar = [&](int s) { return bar_base + 8u * (kStages + s); };
-    const uint32_t acc_bar = bar_base + 8u * (2 * kStages);
-    uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(smem_gen + kStages * kStageBytes + 8 * (2 * kStages + 1));
+    const uint32_t acc_bar = bar_base + 8u * (2 * kStages);                   // accumulators complete (both blocks)
+    const uint32_t acc_free_bar = bar_base + 8u * (2 * kStages + 1);          // accumulators drained (leader only)
+    uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(smem_gen + kStages * kStageBytes + 8 * (2 * kStages + 2));
     volatile int* abort_flag = reinterpret_cast<volatile int*>(tmem_slot + 1);
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const uint32_t rank = cluster_ctarank();
-    // Tile order: bands of kBandTiles row tiles, row tile fastest inside a band, so that the pairs running
-    // at the same time cover a compact block of the output and share their A and B tiles in L2.
-    const int64_t tiles_m = (p.M + 2 * BM - 1) / (2 * BM), tiles_n = (p.N + BN - 1) / BN;
-    const int64_t pair_id = blockIdx.x >> 1;
-    const int64_t band = pair_id / (kBandTiles * tiles_n);
-    const int64_t band_h = tiles_m - band * kBandTiles < kBandTiles ? tiles_m - band * kBandTiles : kBandTiles;
-    const int64_t in_band = pair_id - band * kBandTiles * tiles_n;
-    const int64_t tile_m = band * kBandTiles + in_band % band_h, tile_n = in_band / band_h;
-    const int64_t m_block = tile_m * 2 + rank;                                      // 128-row block of A
-    const int64_t m0 = m_block * BM;
-    const int64_t n0 = tile_n * BN;                                                 // the pair's columns
-    const int split = blockIdx.z;
+    const int64_t n_pairs = gridDim.x >> 1, first = blockIdx.x >> 1;
     const int64_t total_steps = p.K / BK;
-    const int64_t step_begin = (int64_t)split * p.k_steps_per_split;
-    int64_t step_end = step_begin + p.k_steps_per_split;
-    if (step_end > total_steps) step_end = total_steps;
-    const int64_t n_steps = step_end > step_begin ? step_end - step_begin : 0;
 
     if (threadIdx.x == 0) {
         for (int s = 0; s < kStages; ++s) {
@@ -309,6 +368,7 @@ sparse_gemm_pair_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_
             mbar_init(empty_bar(s), 1);      // the leader's tcgen05.commit
         }
         mbar_init(acc_bar, 1);
+        mbar_init(acc_free_bar, 2 * kEpiWarps);   // one arrival per epilogue warp of both blocks
         *abort_flag = 0;
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     }
@@ -326,79 +386,184 @@ sparse_gemm_pair_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_
     if (warp == 0) {
         // ------------------------------------------------------------ TMA producer (both blocks)
         if (lane == 0) {
-            const bool rows_exist = m0 < p.M;            // a pair may hang over the last row block
-            for (int64_t i = 0; i < n_steps; ++i) {
-                const int s = (int)(i % kStages);
-                const uint32_t use = (uint32_t)(i / kStages);
-                if (use > 0 && !mbar_wait(empty_bar(s), (use - 1) & 1u, abort_flag)) break;
-                const uint32_t a_dst = smem_base + s * kStageBytes;
-                const uint32_t b_dst = a_dst + kABytes;
-                const uint32_t e_dst = b_dst + kBBytes;
-                const int64_t step = step_begin + i;
-                const int k = (int)(step * BK);
-                const uint32_t leader_full = map_to_cta(full_bar(s), 0);
-                // only the leader arrives, and locally: a cluster-scope release from the peer on every stage
-                // would wait out the copies already in flight and serialise the pipeline
-                if (rank == 0) mbar_expect_tx(full_bar(s), 2 * kStageBytes);
-                // rows past M read as zeros (out-of-range boxes are zero-filled); the metadata of a row
-                // block that does not exist is taken from block 0 -- any valid pattern is harmless there
-                tma_load_2d_pair(a_dst, &map_a, k / 2, (int)m0, leader_full);
+            uint32_t g = 0;                                  // stages filled so far, over all work items
+            bool ok = true;
+            for (int64_t w = first; w < p.n_work && ok; w += n_pairs) {
+                const WorkItem it = decode_work(p, w, rank);
+                const bool rows_exist = it.m0 < p.M;         // a pair may hang over the last row block
+                for (int64_t i = 0; i < it.n_steps; ++i, ++g) {
+                    const int s = (int)(g % kStages);
+                    const uint32_t use = g / kStages;
+                    if (use > 0 && !mbar_wait(empty_bar(s), (use - 1) & 1u, abort_flag)) { ok = false; break; }
+                    const uint32_t a_dst = smem_base + s * kStageBytes;
+                    const uint32_t b_dst = a_dst + kABytes;
+                    const uint32_t e_dst = b_dst + kBBytes;
+                    const int64_t step = it.step_begin + i;
+                    const int k = (int)(step * BK);
+                    const uint32_t leader_full = map_to_cta(full_bar(s), 0);
+                    // only the leader arrives, and locally: a cluster-scope release from the peer on every stage
+                    // would wait out the copies already in flight and serialise the pipeline
+                    if (rank == 0) mbar_expect_tx(full_bar(s), 2 * kStageBytes);
+                    // rows past M read as zeros (out-of-range boxes are zero-filled); the metadata of a row
+                    // block that does not exist is taken from block 0 -- any valid pattern is harmless there
+                    tma_load_2d_pair(a_dst, &map_a, k / 2, (int)it.m0, leader_full);
 #pragma unroll
-                for (int j = 0; j < BN / 2 / 64; ++j)
-                    tma_load_2d_pair(b_dst + j * kBBoxBytes, &map_b, (int)n0 + (int)rank * (BN / 2) + 64 * j, k,
-                                     leader_full);
-                const int64_t e_block = (rows_exist ? m_block : 0) * total_steps + step;
-                tma_load_2d_pair(e_dst, &map_e, 0, (int)(e_block * 8), leader_full);
+                    for (int j = 0; j < BN / 2 / 64; ++j)
+                        tma_load_2d_pair(b_dst + j * kBBoxBytes, &map_b, (int)it.n0 + (int)rank * (BN / 2) + 64 * j, k,
+                                         leader_full);
+                    const int64_t e_block = (rows_exist ? it.m_block : 0) * total_steps + step;
+                    tma_load_2d_pair(e_dst, &map_e, 0, (int)(e_block * 8), leader_full);
+                }
             }
         }
     } else if (warp == 1) {
         // ------------------------------------------------------------ MMA issuer (leader only)
         if (rank == 0 && lane == 0) {
+            uint32_t g = 0, tiles_done = 0;
             bool ok = true;
-            for (int64_t i = 0; i < n_steps && ok; ++i) {
-                const int s = (int)(i % kStages);
-                const uint32_t use = (uint32_t)(i / kStages);
-                ok = mbar_wait(full_bar(s), use & 1u, abort_flag);
-                if (!ok) break;
-                tc_fence_after();
-                const uint32_t a_addr = smem_base + s * kStageBytes;
-                const uint32_t b_addr = a_addr + kABytes;
-                const uint32_t e_addr = b_addr + kBBytes;
-                const uint32_t tmem_e = tmem_base + kTmemECol + 4u * s;
-                // metadata: 128 lanes x 16 bytes, rows contiguous (8-row core matrices 128 bytes apart)
-                tc_copy_128x128b_pair(tmem_e, make_smem_desc(e_addr, 16, 128, kSwizzleNone));
-#pragma unroll
-                for (int kb = 0; kb < BK / 32; ++kb) {
-                    // A: K-major, 128-byte swizzle, 8-row groups 1024 bytes apart; 32 bytes per K = 32 block
-                    const uint64_t a_desc = make_smem_desc(a_addr + kb * 32, 16, 1024, kSwizzle128B);
-                    // B: N-major, 128-byte swizzle; 64-column blocks kBBoxBytes apart (leading), 8-row
-                    //    groups 1024 bytes apart (stride); 32 k-rows per K = 32 block = 4096 bytes
-                    const uint64_t b_desc = make_smem_desc(b_addr + kb * 4096, kBBoxBytes, 1024, kSwizzle128B);
-                    // metadata of K block kb: column pair (kb & ~1) of the stage's four, selector kb & 1
-                    tc_mma_sp_bf16_pair(tmem_base, a_desc, b_desc, tmem_e + (uint32_t)(kb & ~1),
-                                        kInstrDesc2 | (uint32_t)(kb & 1), (i > 0 || kb > 0) ? 1u : 0u);
+            for (int64_t w = first; w < p.n_work && ok; w += n_pairs) {
+                const WorkItem it = decode_work(p, w, rank);
+                if (it.n_steps == 0) continue;
+                if (tiles_done > 0) {                        // the previous tile has left tensor memory
+                    ok = mbar_wait_cluster(acc_free_bar, (tiles_done - 1) & 1u, abort_flag);
+                    if (!ok) break;
+                    tc_fence_after();
                 }
-                tc_commit_pair(empty_bar(s));    // frees the stage in both blocks when the MMAs retire
-            }
-            tc_commit_pair(acc_bar);             // accumulators complete
-        }
-    } else if (warp >= 4) {
-        // ------------------------------------------------------------ epilogue (both blocks, own rows)
-        const int q = warp - 4;                                  // lanes 32 q .. 32 q + 31
-        const int64_t row = m0 + 32 * q + lane;
-        uint4 sc[kScale ? BN / 8 : 1];
-        if (kScale) {                                            // this row's scale factors, fetched under the main loop
+                for (int64_t i = 0; i < it.n_steps; ++i, ++g) {
+                    const int s = (int)(g % kStages);
+                    const uint32_t use = g / kStages;
+                    ok = mbar_wait(full_bar(s), use & 1u, abort_flag);
+                    if (!ok) break;
+                    tc_fence_after();
+                    const uint32_t a_addr = smem_base + s * kStageBytes;
+                    const uint32_t b_addr = a_addr + kABytes;
+                    const uint32_t e_addr = b_addr + kBBytes;
+                    const uint32_t tmem_e = tmem_base + kTmemECol + 4u * s;
+                    // 128 lanes x 16 bytes of metadata -> tensor-memory columns tmem_e .. tmem_e + 3 (both blocks)
+                    tc_copy_128x128b_pair(tmem_e, make_smem_desc(e_addr, 16, 128, kSwizzleNone));
 #pragma unroll
-            for (int e = 0; e < BN / 8; ++e) {
-                sc[e] = make_uint4(0u, 0u, 0u, 0u);
-                if (row < p.M && n0 + 8 * e < p.N)
-                    sc[e] = __ldg(reinterpret_cast<const uint4*>(p.scale + row * p.ldc + n0 + 8 * e));
+                    for (int kb = 0; kb < BK / 32; ++kb) {
+                        // A: K-major, 128-byte swizzle, 8-row groups 1024 bytes apart; 32 bytes per K = 32 block
+                        const uint64_t a_desc = make_smem_desc(a_addr + kb * 32, 16, 1024, kSwizzle128B);
+                        // B: N-major, 128-byte swizzle; 64-column blocks kBBoxBytes apart (leading), 8-row
+                        //    groups 1024 bytes apart (stride); 32 k-rows per K = 32 block = 4096 bytes
+                        const uint64_t b_desc = make_smem_desc(b_addr + kb * 4096, kBBoxBytes, 1024, kSwizzle128B);
+                        // metadata of K block kb: column pair (kb & ~1) of the stage's four, selector kb & 1
+                        tc_mma_sp_bf16_pair(tmem_base, a_desc, b_desc, tmem_e + (uint32_t)(kb & ~1),
+                                            kInstrDesc2 | (uint32_t)(kb & 1), (i > 0 || kb > 0) ? 1u : 0u);
+                    }
+                    tc_commit_pair(empty_bar(s));    // frees the stage in both blocks when the MMAs retire
+                }
+                if (!ok) break;
+                tc_commit_pair(acc_bar);             // accumulators complete
+                ++tiles_done;
             }
         }
-        const bool acc_ok = n_steps > 0 ? mbar_wait(acc_bar, 0, abort_flag) : true;
-        tc_fence_after();
-        if (acc_ok)
-            epilogue_rows<kScale>(p, split, row, n0, tmem_base + ((uint32_t)(32 * q) << 16), n_steps > 0, sc);
+    } else if (warp >= 3) {
+        // ------------------------------------------------------------ epilogue (both blocks, own rows)
+        const int q = warp & 3;                                  // tensor-memory lanes 32 q .. 32 q + 31 (a warp's quarter)
+        const int c_off = 128 * ((warp - 3) >> 2);               // this warp's half of the tile's columns
+        const uint32_t tmem_rows = tmem_base + ((uint32_t)(32 * q) << 16) + (uint32_t)c_off;
+        const uint32_t leader_free = map_to_cta(acc_free_bar, 0);
+        uint32_t tiles_done = 0;
+        for (int64_t w = first; w < p.n_work; w += n_pairs) {
+            const WorkItem it = decode_work(p, w, rank);
+            const int64_t row = it.m0 + 32 * q + lane;
+            const int64_t col0 = it.n0 + c_off;
+            const bool row_ok = row < p.M;
+            constexpr bool kScale = kMode >= 2, kToBf16 = kMode == 1 || kMode == 2;
+            uint4 sc[kScale ? 16 : 1];
+            if (kScale) {                                        // this row's scale factors, fetched under the main loop
+                const __nv_bfloat16* src = p.scale + row * p.ldc + col0;
+                const bool wide = (reinterpret_cast<uintptr_t>(src) & 31u) == 0;   // whole 32-byte sectors per load
+#pragma unroll
+                for (int e = 0; e < 16; e += 2) {
+                    sc[e] = sc[e + 1] = make_uint4(0u, 0u, 0u, 0u);
+                    if (row_ok && wide && col0 + 8 * e + 8 < p.N) {
+                        asm volatile("ld.global.nc.L1::no_allocate.v8.b32 {%0, %1, %2, %3, %4, %5, %6, %7}, [%8];"
+                                     : "=r"(sc[e].x), "=r"(sc[e].y), "=r"(sc[e].z), "=r"(sc[e].w), "=r"(sc[e + 1].x),
+                                       "=r"(sc[e + 1].y), "=r"(sc[e + 1].z), "=r"(sc[e + 1].w)
+                                     : "l"(src + 8 * e));
+                    } else if (row_ok) {
+                        if (col0 + 8 * e < p.N) sc[e] = __ldg(reinterpret_cast<const uint4*>(src + 8 * e));
+                        if (col0 + 8 * e + 8 < p.N) sc[e + 1] = __ldg(reinterpret_cast<const uint4*>(src + 8 * e + 8));
+                    }
+                }
+            }
+            uint32_t r[kToBf16 ? 64 : 128];                      // packed bf16 pairs, or fp32 bit patterns
+            if (it.n_steps > 0) {
+                if (!mbar_wait(acc_bar, tiles_done & 1u, abort_flag)) break;
+                tc_fence_after();
+#pragma unroll
+                for (int half = 0; half < 2; ++half) {           // 64 columns at a time
+                    uint32_t t0[32], t1[32];
+                    tmem_ld_32x32b_x32(tmem_rows + (uint32_t)(64 * half), t0);
+                    tmem_ld_32x32b_x32(tmem_rows + (uint32_t)(64 * half + 32), t1);
+                    tmem_ld_wait();
+#pragma unroll
+                    for (int e = 0; e < 64; e += 2) {
+                        float f0 = __uint_as_float(e < 32 ? t0[e] : t1[e - 32]);
+                        float f1 = __uint_as_float(e < 32 ? t0[e + 1] : t1[e - 31]);
+                        if (kScale) {
+                            const uint4 s4 = sc[(64 * half + e) / 8];
+                            const uint32_t sw = (e % 8) < 2 ? s4.x : ((e % 8) < 4 ? s4.y : ((e % 8) < 6 ? s4.z : s4.w));
+                            f0 *= __uint_as_float(sw << 16);
+                            f1 *= __uint_as_float(sw & 0xFFFF0000u);
+                        }
+                        if (kToBf16) {
+                            __nv_bfloat162 pr = __floats2bfloat162_rn(f0, f1);
+                            r[(64 * half + e) / 2] = *reinterpret_cast<uint32_t*>(&pr);
+                        } else {
+                            r[64 * half + e] = __float_as_uint(f0);
+                            r[64 * half + e + 1] = __float_as_uint(f1);
+                        }
+                    }
+                }
+                // the accumulator is in registers: give tensor memory back before touching global memory
+                tc_fence_before();
+                __syncwarp();
+                if (lane == 0)
+                    asm volatile("mbarrier.arrive.release.cluster.shared::cluster.b64 _, [%0];" ::"r"(leader_free) : "memory");
+                ++tiles_done;
+            } else {
+#pragma unroll
+                for (int e = 0; e < (kToBf16 ? 64 : 128); ++e) r[e] = 0u;
+            }
+            if (!row_ok) continue;
+            if (kToBf16) {
+                __nv_bfloat16* dst = reinterpret_cast<__nv_bfloat16*>(p.C) + row * p.ldc + col0;
+#pragma unroll
+                for (int e = 0; e < 128; e += 16) {
+                    if (col0 + e + 8 < p.N) store8_b32(dst + e, &r[e / 2]);
+                    else if (col0 + e < p.N)
+                        *reinterpret_cast<uint4*>(dst + e) = make_uint4(r[e / 2], r[e / 2 + 1], r[e / 2 + 2], r[e / 2 + 3]);
+                }
+            } else if (kMode == 0 && p.splits > 1) {
+                float* dst = p.partial + ((int64_t)it.split * p.M + row) * p.N + col0;
+#pragma unroll
+                for (int e = 0; e < 128; e += 8)
+                    if (col0 + e < p.N) store8_b32(dst + e, &r[e]);
+            } else {
+                float* dst = reinterpret_cast<float*>(p.C) + row * p.ldc + col0;
+#pragma unroll
+                for (int e = 0; e < 128; e += 8) {
+                    if (col0 + e >= p.N) break;
+                    if (kMode == 0 && p.accumulate) {
+                        const float4 c0 = *reinterpret_cast<const float4*>(dst + e);
+                        const float4 c1 = *reinterpret_cast<const float4*>(dst + e + 4);
+                        r[e] = __float_as_uint(__uint_as_float(r[e]) + c0.x);
+                        r[e + 1] = __float_as_uint(__uint_as_float(r[e + 1]) + c0.y);
+                        r[e + 2] = __float_as_uint(__uint_as_float(r[e + 2]) + c0.z);
+                        r[e + 3] = __float_as_uint(__uint_as_float(r[e + 3]) + c0.w);
+                        r[e + 4] = __float_as_uint(__uint_as_float(r[e + 4]) + c1.x);
+                        r[e + 5] = __float_as_uint(__uint_as_float(r[e + 5]) + c1.y);
+                        r[e + 6] = __float_as_uint(__uint_as_float(r[e + 6]) + c1.z);
+                        r[e + 7] = __float_as_uint(__uint_as_float(r[e + 7]) + c1.w);
+                    }
+                    store8_b32(dst + e, &r[e]);
+                }
+            }
+        }
     }
 
     tc_fence_before();
@@ -758,12 +923,24 @@ int launch_sparse_gemm(const SparseGemmArgs& a, cudaStream_t stream) {
     }
     static std::once_flag once;
     static cudaError_t attr_err = cudaSuccess;
+    static int max_pairs = 0;
     std::call_once(once, [] {
-        attr_err = cudaFuncSetAttribute(sparse_gemm_pair_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                        kSmemBytes);
-        if (attr_err == cudaSuccess)
-            attr_err = cudaFuncSetAttribute(sparse_gemm_pair_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                            kSmemBytes);
+        const void* kernels[4] = {reinterpret_cast<const void*>(sparse_gemm_pair_kernel<0>),
+                                  reinterpret_cast<const void*>(sparse_gemm_pair_kernel<1>),
+                                  reinterpret_cast<const void*>(sparse_gemm_pair_kernel<2>),
+                                  reinterpret_cast<const void*>(sparse_gemm_pair_kernel<3>)};
+        for (int i = 0; i < 4 && attr_err == cudaSuccess; ++i)
+            attr_err = cudaFuncSetAttribute(kernels[i], cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemBytes);
+        // pairs that can be resident at once (one block per SM): the size of the persistent grid
+        cudaLaunchConfig_t cfg = {};
+        cfg.gridDim = dim3(2, 1, 1);
+        cfg.blockDim = dim3(kThreads, 1, 1);
+        cfg.dynamicSmemBytes = kSmemBytes;
+        int n = 0;
+        if (attr_err == cudaSuccess &&
+            cudaOccupancyMaxActiveClusters(&n, sparse_gemm_pair_kernel<0>, &cfg) == cudaSuccess)
+            max_pairs = n;
+        (void)cudaGetLastError();
     });
     if (attr_err != cudaSuccess) { set_cuda_error(attr_err, "cudaFuncSetAttribute"); return MVUE_ERR_CUDA; }
 
@@ -777,11 +954,20 @@ int launch_sparse_gemm(const SparseGemmArgs& a, cudaStream_t stream) {
     p.scale = reinterpret_cast<const __nv_bfloat16*>(a.scale);
     p.c_is_bf16 = a.c_is_bf16; p.accumulate = a.accumulate; p.splits = splits;
     p.dev_status = a.dev_status;
-    dim3 grid((unsigned)(2 * ((a.M + 2 * BM - 1) / (2 * BM)) * ((a.N + BN - 1) / BN)), 1u, (unsigned)splits);
-    if (p.scale != nullptr && splits == 1)
-        sparse_gemm_pair_kernel<true><<<grid, kThreads, kSmemBytes, stream>>>(map_a, map_b, map_e, p);
+    p.n_work = ((a.M + 2 * BM - 1) / (2 * BM)) * ((a.N + BN - 1) / BN) * splits;
+    int64_t n_pairs = max_pairs > 0 ? max_pairs : a.sm_count / 2;
+    if (n_pairs > p.n_work) n_pairs = p.n_work;
+    if (n_pairs < 1) n_pairs = 1;
+    dim3 grid((unsigned)(2 * n_pairs), 1u, 1u);
+    const bool scaled = p.scale != nullptr && splits == 1, to_bf16 = p.c_is_bf16 && splits == 1;
+    if (scaled && to_bf16)
+        sparse_gemm_pair_kernel<2><<<grid, kThreads, kSmemBytes, stream>>>(map_a, map_b, map_e, p);
+    else if (scaled)
+        sparse_gemm_pair_kernel<3><<<grid, kThreads, kSmemBytes, stream>>>(map_a, map_b, map_e, p);
+    else if (to_bf16)
+        sparse_gemm_pair_kernel<1><<<grid, kThreads, kSmemBytes, stream>>>(map_a, map_b, map_e, p);
     else
-        sparse_gemm_pair_kernel<false><<<grid, kThreads, kSmemBytes, stream>>>(map_a, map_b, map_e, p);
+        sparse_gemm_pair_kernel<0><<<grid, kThreads, kSmemBytes, stream>>>(map_a, map_b, map_e, p);
     cudaError_t e = cudaGetLastError();
     if (e == cudaSuccess && splits > 1) {
         const int64_t total = a.M * (a.N / 4);
