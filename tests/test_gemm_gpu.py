@@ -139,6 +139,33 @@ def test_split_k_is_deterministic_and_equal_to_unsplit_sum():
     assert rel_fro(a.double().cpu().numpy(), want) <= TIGHT
 
 
+def test_more_tiles_than_resident_pairs():
+    # 8 x 12 = 96 output tiles for at most 74 resident pairs: every pair walks several tiles, the drained tile of
+    # one overlapping the main loop of the next.  fp32 out, fp32 accumulate, and the same shape again must match.
+    T, n_out, n_in = 512, 2048, 3072
+    g = workloads.gradient((T, n_out), "student_t", seed=21, dtype="bf16")
+    h = workloads.normal_bf16((T, n_in), seed=22)
+    vals, meta = binding.mvue_prune(to_dev(g), 2, 4, 0, seed=5, layout=TC)
+    assert binding.mvue_gemm_workspace_bytes(0, n_out, n_in, T) == 0
+    a = binding.mvue_sparse_update_gemm(vals, meta, to_dev(h))
+    b = binding.mvue_sparse_update_gemm(vals, meta, to_dev(h))
+    assert torch.equal(a, b)
+    acc = torch.full((n_out, n_in), -2.0, dtype=torch.float32, device="cuda")
+    binding.mvue_sparse_update_gemm(vals, meta, to_dev(h), out=acc, accumulate=True)
+    assert torch.allclose(acc, a - 2.0, rtol=1e-6, atol=1e-6)
+    v_ref, m_ref = oracle.prune(g, 2, 4, axis=0, seed=5, threads=oracle.host_threads())
+    want = oracle.gemm(oracle.unpack(v_ref, m_ref), h, threads=oracle.host_threads())
+    assert rel_fro(a.double().cpu().numpy(), want) <= TIGHT
+    # ragged edges in both directions with several rounds: 2056 x 3080 leaves 8-wide slivers of tiles
+    g2 = workloads.gradient((T, n_out + 8), "student_t", seed=23, dtype="bf16")
+    h2 = workloads.normal_bf16((T, n_in + 8), seed=24)
+    vals2, meta2 = binding.mvue_prune(to_dev(g2), 2, 4, 0, seed=6, layout=TC)
+    c = binding.mvue_sparse_update_gemm(vals2, meta2, to_dev(h2), out_dtype=torch.bfloat16)
+    v_ref, m_ref = oracle.prune(g2, 2, 4, axis=0, seed=6, threads=oracle.host_threads())
+    want2 = oracle.gemm(oracle.unpack(v_ref, m_ref), h2, threads=oracle.host_threads())
+    assert rel_fro(c.double().cpu().numpy(), want2) <= 4e-3
+
+
 def test_gemm_argument_checks():
     vals = torch.zeros((64, 64), dtype=torch.bfloat16, device="cuda")
     meta = torch.zeros((64, 16), dtype=torch.uint8, device="cuda")
