@@ -152,7 +152,10 @@ MVUE_API int mvue_unpack(const void* values, const void* meta, int layout, int64
  * accumulation on the sparse tensor cores.
  * workspace: mvue_gemm_workspace_bytes(0, out, in, T) bytes (may be 0, then
  * NULL is accepted), 16-byte aligned, contents scratch: small outputs with a long
- * reduction are split along K and summed in a second, deterministic pass.  dev_status: optional device int, receives
+ * reduction are split along K and summed in a second, deterministic pass (without
+ * that workspace: MVUE_ERR_WORKSPACE); large fp32 outputs whose last round of tiles
+ * would leave most of the GPU idle have those tiles split along K in the same way
+ * (with a smaller or NULL workspace they are simply computed whole).  dev_status: optional device int, receives
  * MVUE_ERR_DEVICE_TIMEOUT if a bounded pipeline wait expires (then dW is
  * unspecified); otherwise left untouched.
  * Preconditions: T a multiple of 64; out, in multiples of 8; pointers and

@@ -62,10 +62,12 @@ static int run_gemm(const void* values, const void* meta, int layout, int64_t M,
         return MVUE_ERR_ALIGN;
     DeviceInfo dev;
     if (int s = current_device_info(&dev)) return s;
-    const size_t need = gemm_workspace_bytes(M, N, K, dev.sm_count);
-    if (need > 0 && (!workspace || workspace_bytes < need || !aligned16(workspace))) return MVUE_ERR_WORKSPACE;
+    // the split of a long K needs its workspace; the K split of the last round's tiles is skipped without it
+    const size_t need = gemm_required_workspace_bytes(M, N, K, dev.sm_count);
+    if (need > 0 && (!workspace || workspace_bytes < need)) return MVUE_ERR_WORKSPACE;
+    if (workspace && !aligned16(workspace)) return MVUE_ERR_WORKSPACE;
     SparseGemmArgs a{values, meta, M, N, K, B, ldb, C, ldc, c_dtype == MVUE_BF16, accumulate, scale,
-                     workspace, dev_status, dev.sm_count};
+                     workspace, workspace ? workspace_bytes : 0, dev_status, dev.sm_count};
     return launch_sparse_gemm(a, reinterpret_cast<cudaStream_t>(stream));
 }
 
@@ -206,7 +208,7 @@ int mvue_fused_update_gemm(const void* g, int dtype, int64_t T, int64_t out, int
     if (need > 0 && (!workspace || workspace_bytes < need || !aligned16(workspace))) return MVUE_ERR_WORKSPACE;
     FusedArgs f{g, ldg, m, seed,
                 SparseGemmArgs{nullptr, nullptr, out, in, T, h, ldh, dW, lddW, dW_dtype == MVUE_BF16, accumulate,
-                               nullptr, workspace, dev_status, dev.sm_count}};
+                               nullptr, workspace, workspace ? workspace_bytes : 0, dev_status, dev.sm_count}};
     return launch_fused_update(f, reinterpret_cast<cudaStream_t>(stream));
 }
 
@@ -216,7 +218,7 @@ int mvue_sparse_update_gemm_noalloc(const void* values, const void* meta, int la
     if (out <= 0 || in <= 0 || T <= 0 || T % 128 != 0) return MVUE_ERR_SHAPE;
     DeviceInfo dev;
     if (int s = current_device_info(&dev)) return s;
-    const size_t need = gemm_workspace_bytes(out, in, T, dev.sm_count);
+    const size_t need = gemm_required_workspace_bytes(out, in, T, dev.sm_count);
     if (need > kStaticScratchBytes) return MVUE_ERR_WORKSPACE;     // beyond what the library carries
     void* scratch = nullptr;
     size_t scratch_bytes = 0;

@@ -138,7 +138,10 @@ struct GemmParams {
     int c_is_bf16;
     int accumulate;
     int splits;
-    int64_t n_work;           // tiles x splits (pair kernel)
+    int64_t n_work;           // work items of the pair kernel: tiles x splits, or n_main + tail_rem x tail_splits
+    int64_t n_main;           // work items below this number are whole tiles (or tiles of a K split)
+    int tail_rem, tail_splits;   // the last tail_rem tiles are cut into tail_splits parts along K (0, 1: not)
+    float* tail_partial;      // [tail_splits x tail_rem] tiles of 256 x 256 fp32
     int* dev_status;
 };
 
@@ -293,28 +296,53 @@ __device__ __forceinline__ void tc_mma_sp_bf16_pair(uint32_t tmem_d, uint64_t a_
 struct WorkItem {
     int64_t m_block, m0, n0;      // this block's 128-row block of A, its first row, the pair's first column
     int split;
+    int tail_slot;                // >= 0: part * tail_rem + tile of a tail tile cut along K; -1 otherwise
     int64_t step_begin, n_steps;
 };
 
-// Work items are numbered split-major; inside a split the tiles go in bands of kBandTiles row tiles, row tile
-// fastest inside a band, so that the pairs running at the same time cover a compact block of the output and
-// share their A and B tiles in L2.
-__device__ __forceinline__ WorkItem decode_work(const GemmParams& p, int64_t w, uint32_t rank) {
-    const int64_t tiles_m = (p.M + 2 * BM - 1) / (2 * BM), tiles_n = (p.N + BN - 1) / BN;
-    const int64_t n_tiles = tiles_m * tiles_n;
-    WorkItem it;
-    it.split = (int)(w / n_tiles);
-    const int64_t pair_id = w - (int64_t)it.split * n_tiles;
+// Tiles go in bands of kBandTiles row tiles, row tile fastest inside a band, so that the pairs running at the
+// same time cover a compact block of the output and share their A and B tiles in L2.
+__device__ __forceinline__ void tile_of(int64_t M, int64_t N, int64_t pair_id, int64_t* tile_m, int64_t* tile_n) {
+    const int64_t tiles_m = (M + 2 * BM - 1) / (2 * BM), tiles_n = (N + BN - 1) / BN;
     const int64_t band = pair_id / (kBandTiles * tiles_n);
     const int64_t band_h = tiles_m - band * kBandTiles < kBandTiles ? tiles_m - band * kBandTiles : kBandTiles;
     const int64_t in_band = pair_id - band * kBandTiles * tiles_n;
-    const int64_t tile_m = band * kBandTiles + in_band % band_h, tile_n = in_band / band_h;
+    *tile_m = band * kBandTiles + in_band % band_h;
+    *tile_n = in_band / band_h;
+}
+
+// Work items are numbered split-major (K splits of small outputs), or, for outputs of many tiles whose last round
+// would leave most pairs idle: first the n_main tiles of the full rounds, then the remaining tail_rem tiles cut
+// into tail_splits parts along K (part-major), whose fp32 partial tiles a second pass sums.
+__device__ __forceinline__ WorkItem decode_work(const GemmParams& p, int64_t w, uint32_t rank) {
+    const int64_t tiles_m = (p.M + 2 * BM - 1) / (2 * BM), tiles_n = (p.N + BN - 1) / BN;
+    const int64_t n_tiles = tiles_m * tiles_n;
+    const int64_t total_steps = p.K / BK;
+    WorkItem it;
+    int64_t pair_id, per_part;
+    int part;
+    if (w >= p.n_main) {                                  // a part of a tail tile
+        const int64_t j = w - p.n_main;
+        part = (int)(j / p.tail_rem);
+        const int tile = (int)(j - (int64_t)part * p.tail_rem);
+        pair_id = p.n_main + tile;
+        it.split = 0;
+        it.tail_slot = part * p.tail_rem + tile;
+        per_part = (total_steps + p.tail_splits - 1) / p.tail_splits;
+    } else {
+        it.split = (int)(w / n_tiles);
+        pair_id = w - (int64_t)it.split * n_tiles;
+        it.tail_slot = -1;
+        part = it.split;
+        per_part = p.k_steps_per_split;
+    }
+    int64_t tile_m, tile_n;
+    tile_of(p.M, p.N, pair_id, &tile_m, &tile_n);
     it.m_block = tile_m * 2 + rank;
     it.m0 = it.m_block * BM;
     it.n0 = tile_n * BN;
-    const int64_t total_steps = p.K / BK;
-    it.step_begin = (int64_t)it.split * p.k_steps_per_split;
-    int64_t step_end = it.step_begin + p.k_steps_per_split;
+    it.step_begin = (int64_t)part * per_part;
+    int64_t step_end = it.step_begin + per_part;
     if (step_end > total_steps) step_end = total_steps;
     it.n_steps = step_end > it.step_begin ? step_end - it.step_begin : 0;
     return it;
@@ -471,7 +499,9 @@ sparse_gemm_pair_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_
             const int64_t row = it.m0 + 32 * q + lane;
             const int64_t col0 = it.n0 + c_off;
             const bool row_ok = row < p.M;
-            constexpr bool kScale = kMode >= 2, kToBf16 = kMode == 1 || kMode == 2;
+            // bf16 x scale keeps the row's factors in registers; fp32 x scale has no room for them beside 128
+            // fp32 results and applies them after tensor memory has been handed back
+            constexpr bool kScale = kMode == 2, kLateScale = kMode == 3, kToBf16 = kMode == 1 || kMode == 2;
             uint4 sc[kScale ? 16 : 1];
             if (kScale) {                                        // this row's scale factors, fetched under the main loop
                 const __nv_bfloat16* src = p.scale + row * p.ldc + col0;
@@ -530,7 +560,11 @@ sparse_gemm_pair_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_
                 for (int e = 0; e < (kToBf16 ? 64 : 128); ++e) r[e] = 0u;
             }
             if (!row_ok) continue;
-            if (kToBf16) {
+            if (!kToBf16 && it.tail_slot >= 0) {             // a K part of a tail tile: unscaled fp32 partial tile
+                float* dst = p.tail_partial + (((int64_t)it.tail_slot * (2 * BM) + (int64_t)rank * BM + 32 * q + lane) * BN) + c_off;
+#pragma unroll
+                for (int e = 0; e < 128; e += 8) store8_b32(dst + e, &r[e]);
+            } else if (kToBf16) {
                 __nv_bfloat16* dst = reinterpret_cast<__nv_bfloat16*>(p.C) + row * p.ldc + col0;
 #pragma unroll
                 for (int e = 0; e < 128; e += 16) {
@@ -548,6 +582,16 @@ sparse_gemm_pair_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_
 #pragma unroll
                 for (int e = 0; e < 128; e += 8) {
                     if (col0 + e >= p.N) break;
+                    if (kLateScale) {
+                        const uint4 s4 = __ldg(reinterpret_cast<const uint4*>(p.scale + row * p.ldc + col0 + e));
+                        const uint32_t sw[4] = {s4.x, s4.y, s4.z, s4.w};
+#pragma unroll
+                        for (int t = 0; t < 4; ++t) {
+                            r[e + 2 * t] = __float_as_uint(__uint_as_float(r[e + 2 * t]) * __uint_as_float(sw[t] << 16));
+                            r[e + 2 * t + 1] =
+                                __float_as_uint(__uint_as_float(r[e + 2 * t + 1]) * __uint_as_float(sw[t] & 0xFFFF0000u));
+                        }
+                    }
                     if (kMode == 0 && p.accumulate) {
                         const float4 c0 = *reinterpret_cast<const float4*>(dst + e);
                         const float4 c1 = *reinterpret_cast<const float4*>(dst + e + 4);
@@ -799,6 +843,34 @@ splitk_reduce_kernel(const float* __restrict__ partial, int splits, int64_t M, i
     }
 }
 
+// Sums the K parts of the tail tiles (see decode_work) into C: one block per row of a tail tile.
+__global__ void __launch_bounds__(64)
+tail_reduce_kernel(const float* __restrict__ partial, int rem, int parts, int64_t n_main, int64_t M, int64_t N,
+                   float* __restrict__ C, int64_t ldc, const __nv_bfloat16* __restrict__ scale, int accumulate) {
+    const int tile = blockIdx.x / (2 * BM), lr = blockIdx.x % (2 * BM);
+    int64_t tile_m, tile_n;
+    tile_of(M, N, n_main + tile, &tile_m, &tile_n);
+    const int64_t row = tile_m * (2 * BM) + lr, col = tile_n * BN + 4 * threadIdx.x;
+    if (row >= M || col >= N) return;
+    float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
+    for (int part = 0; part < parts; ++part) {
+        const float4 v = *reinterpret_cast<const float4*>(
+            partial + (((int64_t)(part * rem + tile) * (2 * BM) + lr) * BN) + 4 * threadIdx.x);
+        acc.x += v.x; acc.y += v.y; acc.z += v.z; acc.w += v.w;
+    }
+    if (scale) {
+        const uint2 sc = *reinterpret_cast<const uint2*>(scale + row * ldc + col);
+        acc.x *= __uint_as_float(sc.x << 16); acc.y *= __uint_as_float(sc.x & 0xFFFF0000u);
+        acc.z *= __uint_as_float(sc.y << 16); acc.w *= __uint_as_float(sc.y & 0xFFFF0000u);
+    }
+    float* dst = C + row * ldc + col;
+    if (accumulate) {
+        const float4 o = *reinterpret_cast<const float4*>(dst);
+        acc.x += o.x; acc.y += o.y; acc.z += o.z; acc.w += o.w;
+    }
+    *reinterpret_cast<float4*>(dst) = acc;
+}
+
 // ---- host side ----------------------------------------------------------------
 }  // namespace
 
@@ -813,9 +885,77 @@ int gemm_split_count(int64_t M, int64_t N, int64_t K, int sm_count) {
     return (int)(splits < 1 ? 1 : splits);
 }
 
-size_t gemm_workspace_bytes(int64_t M, int64_t N, int64_t K, int sm_count) {
+size_t gemm_required_workspace_bytes(int64_t M, int64_t N, int64_t K, int sm_count) {
     const int splits = gemm_split_count(M, N, K, sm_count);
     return splits > 1 ? (size_t)splits * (size_t)M * (size_t)N * sizeof(float) : 0;
+}
+
+namespace {
+
+// The four instantiations of the pair kernel, their shared-memory attribute, and how many pairs fit the GPU at
+// once (one block per SM): the size of the persistent grid.  Looked up once.
+struct PairKernelSetup {
+    cudaError_t attr_err = cudaSuccess;
+    int max_pairs = 0;
+};
+const PairKernelSetup& pair_kernel_setup() {
+    static const PairKernelSetup st = [] {
+        PairKernelSetup r;
+        const void* kernels[4] = {reinterpret_cast<const void*>(sparse_gemm_pair_kernel<0>),
+                                  reinterpret_cast<const void*>(sparse_gemm_pair_kernel<1>),
+                                  reinterpret_cast<const void*>(sparse_gemm_pair_kernel<2>),
+                                  reinterpret_cast<const void*>(sparse_gemm_pair_kernel<3>)};
+        for (int i = 0; i < 4 && r.attr_err == cudaSuccess; ++i)
+            r.attr_err = cudaFuncSetAttribute(kernels[i], cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemBytes);
+        cudaLaunchConfig_t cfg = {};
+        cfg.gridDim = dim3(2, 1, 1);
+        cfg.blockDim = dim3(kThreads, 1, 1);
+        cfg.dynamicSmemBytes = kSmemBytes;
+        int n = 0;
+        if (r.attr_err == cudaSuccess &&
+            cudaOccupancyMaxActiveClusters(&n, sparse_gemm_pair_kernel<0>, &cfg) == cudaSuccess)
+            r.max_pairs = n;
+        (void)cudaGetLastError();
+        return r;
+    }();
+    return st;
+}
+int resident_pairs(int sm_count) {
+    const int n = pair_kernel_setup().max_pairs;
+    return n > 0 ? n : (sm_count / 2 > 0 ? sm_count / 2 : 1);
+}
+
+// When the output has more tiles than resident pairs and the last round would keep at most half of them busy,
+// the tiles of that round are cut along K into `parts` so that the round is short and full.
+struct TailPlan {
+    int rem = 0, parts = 0;
+    int64_t n_main = 0;       // tiles (times splits) handled whole
+};
+TailPlan tail_plan(int64_t M, int64_t N, int64_t K, int splits, int n_pairs) {
+    const int64_t n_tiles = ((M + 2 * BM - 1) / (2 * BM)) * ((N + BN - 1) / BN);
+    const int64_t steps = K / BK;
+    TailPlan t;
+    t.n_main = n_tiles * splits;
+    if (splits != 1 || n_tiles <= n_pairs) return t;
+    const int64_t rem = n_tiles % n_pairs;
+    if (rem == 0 || rem > n_pairs / 2 || steps < 16) return t;
+    int64_t parts = n_pairs / rem;
+    if (parts > steps / 8) parts = steps / 8;             // at least 8 stages (K = 1024) per part
+    if (parts > 16) parts = 16;
+    if (parts < 2) return t;
+    t.rem = (int)rem;
+    t.parts = (int)parts;
+    t.n_main = n_tiles - rem;
+    return t;
+}
+
+}  // namespace
+
+size_t gemm_workspace_bytes(int64_t M, int64_t N, int64_t K, int sm_count) {
+    const size_t required = gemm_required_workspace_bytes(M, N, K, sm_count);
+    if (required > 0) return required;
+    const TailPlan t = tail_plan(M, N, K, 1, resident_pairs(sm_count));
+    return (size_t)t.rem * (size_t)t.parts * (size_t)(2 * BM) * (size_t)BN * sizeof(float);
 }
 
 // ---- library-owned split-K scratch --------------------------------------------------
@@ -889,6 +1029,7 @@ int launch_fused_update(const FusedArgs& f, cudaStream_t stream) {
     p.C = a.C; p.ldc = a.ldc;
     p.scale = nullptr;
     p.c_is_bf16 = a.c_is_bf16; p.accumulate = a.accumulate; p.splits = splits;
+    p.n_work = p.n_main = 0; p.tail_rem = p.tail_splits = 0; p.tail_partial = nullptr;   // pair kernel only
     p.dev_status = a.dev_status;
     dim3 grid((unsigned)((a.N + BN - 1) / BN), (unsigned)((a.M + BM - 1) / BM), (unsigned)splits);
     if (f.m == 4)
@@ -921,28 +1062,8 @@ int launch_sparse_gemm(const SparseGemmArgs& a, cudaStream_t stream) {
         set_cuda_error(cudaErrorUnknown, "cuTensorMapEncodeTiled");
         return MVUE_ERR_CUDA;
     }
-    static std::once_flag once;
-    static cudaError_t attr_err = cudaSuccess;
-    static int max_pairs = 0;
-    std::call_once(once, [] {
-        const void* kernels[4] = {reinterpret_cast<const void*>(sparse_gemm_pair_kernel<0>),
-                                  reinterpret_cast<const void*>(sparse_gemm_pair_kernel<1>),
-                                  reinterpret_cast<const void*>(sparse_gemm_pair_kernel<2>),
-                                  reinterpret_cast<const void*>(sparse_gemm_pair_kernel<3>)};
-        for (int i = 0; i < 4 && attr_err == cudaSuccess; ++i)
-            attr_err = cudaFuncSetAttribute(kernels[i], cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemBytes);
-        // pairs that can be resident at once (one block per SM): the size of the persistent grid
-        cudaLaunchConfig_t cfg = {};
-        cfg.gridDim = dim3(2, 1, 1);
-        cfg.blockDim = dim3(kThreads, 1, 1);
-        cfg.dynamicSmemBytes = kSmemBytes;
-        int n = 0;
-        if (attr_err == cudaSuccess &&
-            cudaOccupancyMaxActiveClusters(&n, sparse_gemm_pair_kernel<0>, &cfg) == cudaSuccess)
-            max_pairs = n;
-        (void)cudaGetLastError();
-    });
-    if (attr_err != cudaSuccess) { set_cuda_error(attr_err, "cudaFuncSetAttribute"); return MVUE_ERR_CUDA; }
+    const PairKernelSetup& setup = pair_kernel_setup();
+    if (setup.attr_err != cudaSuccess) { set_cuda_error(setup.attr_err, "cudaFuncSetAttribute"); return MVUE_ERR_CUDA; }
 
     const int splits = gemm_split_count(a.M, a.N, a.K, a.sm_count);
     const int64_t steps = a.K / BK;
@@ -954,8 +1075,20 @@ int launch_sparse_gemm(const SparseGemmArgs& a, cudaStream_t stream) {
     p.scale = reinterpret_cast<const __nv_bfloat16*>(a.scale);
     p.c_is_bf16 = a.c_is_bf16; p.accumulate = a.accumulate; p.splits = splits;
     p.dev_status = a.dev_status;
-    p.n_work = ((a.M + 2 * BM - 1) / (2 * BM)) * ((a.N + BN - 1) / BN) * splits;
-    int64_t n_pairs = max_pairs > 0 ? max_pairs : a.sm_count / 2;
+    const int resident = resident_pairs(a.sm_count);
+    TailPlan tail = tail_plan(a.M, a.N, a.K, splits, resident);
+    const size_t tail_bytes = (size_t)tail.rem * (size_t)tail.parts * (size_t)(2 * BM) * (size_t)BN * sizeof(float);
+    // the tail split needs fp32 output and room for its partial tiles; without either the tiles simply stay whole
+    if (tail.parts < 2 || a.c_is_bf16 || a.workspace == nullptr || a.workspace_bytes < tail_bytes) {
+        tail = TailPlan();
+        tail.n_main = ((a.M + 2 * BM - 1) / (2 * BM)) * ((a.N + BN - 1) / BN) * splits;
+    }
+    p.n_main = tail.n_main;
+    p.tail_rem = tail.rem;
+    p.tail_splits = tail.parts;
+    p.tail_partial = reinterpret_cast<float*>(a.workspace);
+    p.n_work = tail.n_main + (int64_t)tail.rem * tail.parts;
+    int64_t n_pairs = resident;
     if (n_pairs > p.n_work) n_pairs = p.n_work;
     if (n_pairs < 1) n_pairs = 1;
     dim3 grid((unsigned)(2 * n_pairs), 1u, 1u);
@@ -969,6 +1102,12 @@ int launch_sparse_gemm(const SparseGemmArgs& a, cudaStream_t stream) {
     else
         sparse_gemm_pair_kernel<0><<<grid, kThreads, kSmemBytes, stream>>>(map_a, map_b, map_e, p);
     cudaError_t e = cudaGetLastError();
+    if (e == cudaSuccess && tail.parts > 1) {
+        tail_reduce_kernel<<<tail.rem * 2 * BM, BN / 4, 0, stream>>>(
+            p.tail_partial, tail.rem, tail.parts, tail.n_main, a.M, a.N, reinterpret_cast<float*>(a.C), a.ldc,
+            reinterpret_cast<const __nv_bfloat16*>(a.scale), a.accumulate);
+        e = cudaGetLastError();
+    }
     if (e == cudaSuccess && splits > 1) {
         const int64_t total = a.M * (a.N / 4);
         const int64_t want = (total + 255) / 256;

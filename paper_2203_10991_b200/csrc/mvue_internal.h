@@ -38,12 +38,14 @@ struct SparseGemmArgs {
     int accumulate;
     const void* scale;    // optional bf16 [M x N] (ld = ldc) multiplied into the result, or nullptr
     void* workspace;
+    size_t workspace_bytes;
     int* dev_status;
     int sm_count;
 };
 int launch_sparse_gemm(const SparseGemmArgs& a, cudaStream_t stream);     // returns an mvue_status
 int gemm_split_count(int64_t M, int64_t N, int64_t K, int sm_count);
-size_t gemm_workspace_bytes(int64_t M, int64_t N, int64_t K, int sm_count);
+size_t gemm_workspace_bytes(int64_t M, int64_t N, int64_t K, int sm_count);            // what lets every path run
+size_t gemm_required_workspace_bytes(int64_t M, int64_t N, int64_t K, int sm_count);   // the split along K alone
 
 struct FusedArgs {
     const void* g;        // dense bf16 gradient [T x out]

@@ -166,6 +166,40 @@ def test_more_tiles_than_resident_pairs():
     assert rel_fro(c.double().cpu().numpy(), want2) <= 4e-3
 
 
+def test_last_round_tiles_are_split_along_k():
+    # 10 x 8 = 80 tiles over at most 74 resident pairs: the 6 tiles of the last round are cut along K into parts
+    # (fp32 partial tiles in the workspace, summed by a second pass).  Rows from every row tile against the oracle;
+    # the same bits when repeated; accumulate; and the whole-tile path (no workspace) agrees to rounding.
+    T, n_out, n_in = 2048, 2560, 2048
+    g = workloads.gradient((T, n_out), "student_t", seed=31, dtype="bf16")
+    h = workloads.normal_bf16((T, n_in), seed=32)
+    vals, meta = binding.mvue_prune(to_dev(g), 2, 4, 0, seed=8, layout=TC)
+    need = binding.mvue_gemm_workspace_bytes(0, n_out, n_in, T)
+    assert need > 0                                        # the tail split asks for room
+    a = binding.mvue_sparse_update_gemm(vals, meta, to_dev(h))
+    b = binding.mvue_sparse_update_gemm(vals, meta, to_dev(h))
+    assert torch.equal(a, b)
+    acc = torch.full((n_out, n_in), 0.25, dtype=torch.float32, device="cuda")
+    binding.mvue_sparse_update_gemm(vals, meta, to_dev(h), out=acc, accumulate=True)
+    assert torch.allclose(acc, a + 0.25, rtol=1e-6, atol=1e-6)
+    # without a workspace the tiles stay whole (the raw entry point accepts NULL here)
+    whole = torch.empty_like(a)
+    L = binding.lib()
+    hd = to_dev(h)
+    rc = L.mvue_sparse_update_gemm(vals.data_ptr(), meta.data_ptr(), TC, n_out, T, hd.data_ptr(), n_in, n_in,
+                                   whole.data_ptr(), 0, n_in, 0, None, 0, None, None)
+    assert rc == 0
+    torch.cuda.synchronize()
+    assert torch.allclose(whole, a, rtol=1e-5, atol=1e-5)
+    v_ref, m_ref = oracle.prune(g, 2, 4, axis=0, seed=8, threads=oracle.host_threads())
+    rows = np.array(sorted({r for t in range(10) for r in (256 * t, 256 * t + 77, 256 * t + 130, 256 * t + 255)}))
+    A_rows = np.ascontiguousarray(oracle.unpack(np.ascontiguousarray(v_ref[rows]), np.ascontiguousarray(m_ref[rows])))
+    want = oracle.gemm(A_rows, h, threads=oracle.host_threads())
+    got = a[torch.from_numpy(rows).cuda()].double().cpu().numpy()
+    assert rel_fro(got, want) <= TIGHT
+    assert np.abs(got - want).max() <= 1e-4 * np.abs(want).max()
+
+
 def test_gemm_argument_checks():
     vals = torch.zeros((64, 64), dtype=torch.bfloat16, device="cuda")
     meta = torch.zeros((64, 16), dtype=torch.uint8, device="cuda")
