@@ -63,6 +63,14 @@ def lib() -> ctypes.CDLL:
         L.oracle_mvue_2of4.restype = None
         L.oracle_mvue_2of4_systematic.argtypes = L.oracle_mvue_2of4.argtypes
         L.oracle_mvue_2of4_systematic.restype = None
+        L.oracle_mvue_2of4_approx.argtypes = [ctypes.POINTER(ctypes.c_float), ctypes.c_uint32, ctypes.c_uint32,
+                                              ctypes.POINTER(ctypes.c_int), ctypes.POINTER(ctypes.c_float)]
+        L.oracle_mvue_2of4_approx.restype = None
+        L.oracle_block_word_pair.argtypes = [ctypes.c_uint64, ctypes.c_uint64, u32p]
+        L.oracle_block_word_pair.restype = None
+        L.oracle_sweep_approx24.argtypes = [ctypes.POINTER(ctypes.c_float), ctypes.POINTER(ctypes.c_uint64),
+                                            ctypes.POINTER(ctypes.c_uint64), ctypes.POINTER(ctypes.c_float)]
+        L.oracle_sweep_approx24.restype = None
         L.oracle_prune.argtypes = [ctypes.c_void_p, ctypes.c_int, ctypes.c_int64, ctypes.c_int64,
                                    ctypes.c_int64, ctypes.c_int, ctypes.c_int, ctypes.c_int,
                                    ctypes.c_uint64, ctypes.c_int64, ctypes.c_int64,
@@ -130,6 +138,7 @@ def mvue_1of2(a1: float, a2: float, word: int):
 
 
 JOINT_TABLE, JOINT_SYSTEMATIC = 0, 1      # 2:4 law over pairs: App. A.2 table / systematic sampling
+JOINT_APPROX = 2                          # approx-MVUE 2:4 of Sec. 4.4 (two sequential draws, two words per block)
 
 
 def mvue_2of4(a, word: int, joint: int = JOINT_TABLE):
@@ -141,6 +150,21 @@ def mvue_2of4(a, word: int, joint: int = JOINT_TABLE):
     return (int(idx[0]), int(idx[1])), (float(val[0]), float(val[1]))
 
 
+def mvue_2of4_approx(a, word1: int, word2: int):
+    """Sec. 4.4 on one block: ((idx0, idx1), (val0, val1)) with idx0 < idx1."""
+    arr = (ctypes.c_float * 4)(*[float(x) for x in a])
+    idx = (ctypes.c_int * 2)()
+    val = (ctypes.c_float * 2)()
+    lib().oracle_mvue_2of4_approx(arr, word1 & 0xFFFFFFFF, word2 & 0xFFFFFFFF, idx, val)
+    return (int(idx[0]), int(idx[1])), (float(val[0]), float(val[1]))
+
+
+def block_word_pair(seed: int, q: int):
+    out = (ctypes.c_uint32 * 2)()
+    lib().oracle_block_word_pair(seed & (2**64 - 1), q, out)
+    return int(out[0]), int(out[1])
+
+
 def packed_shapes(rows: int, cols: int, axis: int):
     mrows, k = (rows, cols) if axis == 1 else (cols, rows)
     return (mrows, k // 2), (mrows, k // 8)
@@ -149,7 +173,7 @@ def packed_shapes(rows: int, cols: int, axis: int):
 def prune(g: np.ndarray, n: int, m: int, axis: int, seed: int, *, k_total: int | None = None,
           k_offset: int = 0, threads: int = 1, joint: int = JOINT_TABLE):
     """MVUE n:m prune + pack of a 2-D array (float32, or uint16 holding bf16 bits).
-    joint: the 2:4 law over pairs (JOINT_TABLE: App. A.2; JOINT_SYSTEMATIC); ignored for 1:2.
+    joint: the 2:4 estimator (JOINT_TABLE: App. A.2; JOINT_SYSTEMATIC; JOINT_APPROX: Sec. 4.4); ignored for 1:2.
 
     Returns (values uint16 [Mrows, K/2], meta uint8 [Mrows, K/8]) in canonical form.
     """
@@ -223,3 +247,18 @@ def sweep_1of2(a1: float, a2: float):
     n = float(1 << 24)
     return (np.array([c for c in counts], dtype=np.float64) / n,
             np.array([s for s in sums]) / n, sq.value / n)
+
+
+def sweep_approx24(a):
+    """Sec. 4.4 sampler, one draw at a time over all 2^24 values of each uniform:
+    (P[first = i], P[second = j | first = i] (rows of never-drawn i are NaN), value of k when it survives)."""
+    arr = (ctypes.c_float * 4)(*[float(x) for x in a])
+    first = (ctypes.c_uint64 * 4)()
+    second = (ctypes.c_uint64 * 16)()
+    val = (ctypes.c_float * 4)()
+    lib().oracle_sweep_approx24(arr, first, second, val)
+    n = float(1 << 24)
+    f = np.array(list(first), dtype=np.float64) / n
+    sec = np.array(list(second), dtype=np.float64).reshape(4, 4) / n
+    sec[f == 0] = np.nan
+    return f, sec, np.array(list(val), dtype=np.float64)

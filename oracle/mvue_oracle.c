@@ -22,7 +22,9 @@
  * exhaustive sweep over every value of the 24-bit uniform; the second 2:4 law
  * (systematic sampling) against the same optimal marginals, mean and minimal
  * variance by the same sweep, and against its interval-overlap law; bf16 rounding
- * against a library cast; the product against a library fp64 matmul.
+ * against a library cast; the product against a library fp64 matmul; the
+ * approx-MVUE sampler of Sec. 4.4 against the sequential-draw probabilities and the
+ * inclusion-probability equation of that section by exhaustive sweeps of each draw.
  */
 #include <math.h>
 #include <stddef.h>
@@ -70,6 +72,19 @@ uint32_t oracle_block_word(uint64_t seed, uint64_t q)
     uint32_t out[4];
     oracle_philox4x32_10(ctr, key, out);
     return out[q & 3u];
+}
+
+/* The two words of block number q for the estimator that draws twice per block
+ * (Sec. 4.4): one generator call serves two consecutive blocks. */
+void oracle_block_word_pair(uint64_t seed, uint64_t q, uint32_t words[2])
+{
+    uint64_t call = q >> 1;
+    uint32_t ctr[4] = { (uint32_t)call, (uint32_t)(call >> 32), 0u, 0u };
+    uint32_t key[2] = { (uint32_t)seed, (uint32_t)(seed >> 32) };
+    uint32_t out[4];
+    oracle_philox4x32_10(ctr, key, out);
+    words[0] = out[2 * (q & 1u)];
+    words[1] = out[2 * (q & 1u) + 1];
 }
 
 /* eps in [0,1): the top 24 bits of the word, exactly representable. */
@@ -278,6 +293,91 @@ void oracle_mvue_2of4_systematic(const float a[4], uint32_t word, int idx[2], fl
 }
 
 /* ------------------------------------------------------------------------
+ * Approximately optimal 2:4 (Sec. 4.4, "approx-MVUE"): two sequential draws
+ * without replacement, each proportional to magnitude, and survivors divided by
+ * their exact inclusion probability (the equation of Sec. 4.4), so the estimator
+ * is unbiased; its variance is above the optimum of Sec. 4.2 by a factor the
+ * paper's scan bounds below two.
+ *
+ * Steps (m_k = |a_k|, block order, no sort):
+ * 1. First draw: element i with probability m_i / s, s = m_0+m_1+m_2+m_3, by the
+ *    threshold test of App. "Pruning Overhead" Part 1 walked over the running
+ *    sums c_1 = m_0, c_2 = c_1 + m_1, c_3 = c_2 + m_2, s = c_3 + m_3:
+ *        t_1 = n_1 (s 2^-24),   i = #{k in 1,2,3 : c_k <= t_1},
+ *    n_1 the top 24 bits of the block's first random word.
+ * 2. Second draw among the other three, in position order r_0 < r_1 < r_2, with
+ *    probability m_j / (s - m_i).  "s - m_i" is formed as the sum of the others,
+ *    R_i = (m_{r0} + m_{r1}) + m_{r2}, never as a difference:
+ *        d_1 = m_{r0}, d_2 = d_1 + m_{r1}, R_i = d_2 + m_{r2},
+ *        t_2 = n_2 (R_i 2^-24),   j = r_{#{k in 1,2 : d_k <= t_2}},
+ *    n_2 from the block's second random word.  i != j for every input.
+ * 3. Inclusion probability (Sec. 4.4): p_k = m_k/s + sum_{l != k} (m_l/s)(m_k/R_l)
+ *    = (m_k/s)(1 + T_k), T_k = sum_{l != k} vv_l, vv_l = m_l / R_l (Algorithm 1's vv;
+ *    its q - vv_k is T_k, summed here directly so nothing cancels).  The survivor
+ *    becomes a_k / p_k = sign(a_k) s / (1 + T_k): six divisions per block (the four
+ *    vv_l, then one per survivor).  Sums of three run in position order, (x + y) + z.
+ * Zero rules: an element of magnitude zero owns an empty interval in both walks.
+ * If R_i = 0 (at most one non-zero in the block) both survivors keep their own
+ * values (p = 1): the non-zero, if any, and a signed zero beside it; an all-zero
+ * block keeps positions 3 and 2.
+ *
+ * first / second: the positions drawn first and second; v_first / v_second
+ * their new values.
+ * ---------------------------------------------------------------------- */
+void oracle_mvue_2of4_approx_ordered(const float a[4], uint32_t word1, uint32_t word2,
+                                     int *first, int *second, float *v_first, float *v_second)
+{
+    float m[4], R[4], vv[4];
+    for (int k = 0; k < 4; ++k) m[k] = fabsf(a[k]);
+    /* first draw */
+    const float c1 = m[0];
+    const float c2 = c1 + m[1];
+    const float c3 = c2 + m[2];
+    const float s  = c3 + m[3];
+    const float t1 = (float)(word1 >> 8) * (s * 5.9604644775390625e-08f);
+    const int i = (c1 <= t1) + (c2 <= t1) + (c3 <= t1);
+    /* sums of the other three, in position order */
+    for (int k = 0; k < 4; ++k) {
+        int r[3], n = 0;
+        for (int l = 0; l < 4; ++l) if (l != k) r[n++] = l;
+        R[k] = (m[r[0]] + m[r[1]]) + m[r[2]];
+    }
+    /* second draw among the others */
+    int r[3], n = 0;
+    for (int l = 0; l < 4; ++l) if (l != i) r[n++] = l;
+    const float d1 = m[r[0]];
+    const float d2 = d1 + m[r[1]];
+    const float t2 = (float)(word2 >> 8) * (R[i] * 5.9604644775390625e-08f);
+    const int j = r[(d1 <= t2) + (d2 <= t2)];
+    /* survivors */
+    float vi, vj;
+    if (R[i] == 0.0f) {
+        vi = a[i]; vj = a[j];
+    } else {
+        for (int k = 0; k < 4; ++k) vv[k] = m[k] / R[k];
+        float T[2];
+        const int who[2] = { i, j };
+        for (int e = 0; e < 2; ++e) {
+            int o[3], c = 0;
+            for (int l = 0; l < 4; ++l) if (l != who[e]) o[c++] = l;
+            T[e] = (vv[o[0]] + vv[o[1]]) + vv[o[2]];
+        }
+        vi = copysignf(s / (1.0f + T[0]), a[i]);
+        vj = copysignf(s / (1.0f + T[1]), a[j]);
+    }
+    *first = i; *second = j; *v_first = vi; *v_second = vj;
+}
+
+/* The same with the survivors in ascending position: idx[0] < idx[1], val[] their new values. */
+void oracle_mvue_2of4_approx(const float a[4], uint32_t word1, uint32_t word2, int idx[2], float val[2])
+{
+    int i, j; float vi, vj;
+    oracle_mvue_2of4_approx_ordered(a, word1, word2, &i, &j, &vi, &vj);
+    if (i < j) { idx[0] = i; idx[1] = j; val[0] = vi; val[1] = vj; }
+    else       { idx[0] = j; idx[1] = i; val[0] = vj; val[1] = vi; }
+}
+
+/* ------------------------------------------------------------------------
  * Tensor-wide prune and pack.
  *
  * g is a row-major [rows x cols] matrix with leading dimension ld, fp32
@@ -297,8 +397,9 @@ void oracle_mvue_2of4_systematic(const float a[4], uint32_t word, int idx[2], fl
  *                        of four, low nibble = even group.
  * A 1:2 result is written as a valid 2:4 pattern: the pair (4j, 4j+1) gives
  * idx0 in {0,1}, the pair (4j+2, 4j+3) gives idx1 in {2,3}.
- * joint selects the 2:4 law over pairs: 0 = the pair table of App. A.2,
- * 1 = systematic sampling (above); 1:2 has a single law and ignores it.
+ * joint selects the 2:4 estimator: 0 = the pair table of App. A.2,
+ * 1 = systematic sampling, 2 = approx-MVUE of Sec. 4.4 (above; two random words
+ * per block); 1:2 has a single law and ignores it.
  * Returns 0, or -1 for an unsupported shape.
  * ---------------------------------------------------------------------- */
 static float load_elem(const void *g, int is_bf16, int64_t off)
@@ -315,6 +416,7 @@ int oracle_prune(const void *g, int is_bf16, int64_t rows, int64_t cols, int64_t
     const int64_t K     = axis == 1 ? cols : rows;
     if (!((n == 1 && m == 2) || (n == 2 && m == 4))) return -1;
     if (K % 8 != 0 || k_total % 8 != 0 || k_offset % 8 != 0 || k_offset + K > k_total) return -1;
+    if (joint < 0 || joint > 2) return -1;
     (void)threads;
 #pragma omp parallel for num_threads(threads) schedule(static)
     for (int64_t r = 0; r < Mrows; ++r) {
@@ -328,8 +430,13 @@ int oracle_prune(const void *g, int is_bf16, int64_t rows, int64_t cols, int64_t
             int idx[2]; float val[2];
             if (m == 4) {
                 uint64_t q = (uint64_t)r * (uint64_t)(k_total / 4) + (uint64_t)(k_offset / 4 + j);
-                if (joint == 0) oracle_mvue_2of4(a, oracle_block_word(seed, q), idx, val);
-                else            oracle_mvue_2of4_systematic(a, oracle_block_word(seed, q), idx, val);
+                if (joint == 0)      oracle_mvue_2of4(a, oracle_block_word(seed, q), idx, val);
+                else if (joint == 1) oracle_mvue_2of4_systematic(a, oracle_block_word(seed, q), idx, val);
+                else {
+                    uint32_t w[2];
+                    oracle_block_word_pair(seed, q, w);
+                    oracle_mvue_2of4_approx(a, w[0], w[1], idx, val);
+                }
             } else {
                 for (int half = 0; half < 2; ++half) {
                     uint64_t q = (uint64_t)r * (uint64_t)(k_total / 2)
@@ -442,5 +549,32 @@ void oracle_sweep_1of2(float a1, float a2, uint64_t counts[2], double sum_val[2]
         th[idx] = kept;
         sum_val[0] += th[0]; sum_val[1] += th[1];
         *sum_sq += (th[0] - (double)a1) * (th[0] - (double)a1) + (th[1] - (double)a2) * (th[1] - (double)a2);
+    }
+}
+
+/* Sweeps for the approx-MVUE sampler (Sec. 4.4), one draw at a time:
+ * first[i]      = how many of the 2^24 values of the first uniform draw element i first;
+ * second[i][j]  = with a first uniform that draws i (if none exists the row stays zero), how
+ *                 many of the 2^24 values of the second uniform draw j second;
+ * val[k]        = the value element k takes when it survives (it does not depend on the
+ *                 partner); NaN if k was never seen to survive. */
+void oracle_sweep_approx24(const float a[4], uint64_t first[4], uint64_t second[4][4], float val[4])
+{
+    uint32_t rep[4]; int have[4] = { 0, 0, 0, 0 };
+    for (int i = 0; i < 4; ++i) { first[i] = 0; val[i] = NAN; for (int j = 0; j < 4; ++j) second[i][j] = 0; }
+    for (uint32_t n = 0; n < (1u << 24); ++n) {
+        int i, j; float vi, vj;
+        oracle_mvue_2of4_approx_ordered(a, n << 8, 0u, &i, &j, &vi, &vj);
+        first[i] += 1;
+        if (!have[i]) { have[i] = 1; rep[i] = n << 8; }
+    }
+    for (int i = 0; i < 4; ++i) {
+        if (!have[i]) continue;
+        for (uint32_t n = 0; n < (1u << 24); ++n) {
+            int i2, j; float vi, vj;
+            oracle_mvue_2of4_approx_ordered(a, rep[i], n << 8, &i2, &j, &vi, &vj);
+            second[i][j] += 1;
+            val[i2] = vi; val[j] = vj;
+        }
     }
 }

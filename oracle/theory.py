@@ -121,6 +121,40 @@ def systematic_law24(a):
     return law
 
 
+# ------------------------------------------------- approx-MVUE 2:4 (Sec. 4.4) ---
+def approx24_ordered_law(a):
+    """Sec. 4.4: P[i drawn first, j drawn second] = (a_i / sum) (a_j / (sum - a_i)), as a 4x4
+    matrix (zero diagonal).  Needs at least two non-zeros."""
+    m = np.abs(np.asarray(a, dtype=np.float64))
+    total = m.sum()
+    law = np.zeros((4, 4))
+    for i in range(4):
+        for j in range(4):
+            if i != j and m[i] > 0 and m[j] > 0:
+                law[i, j] = m[i] / total * m[j] / (total - m[i])
+    return law
+
+
+def approx24_inclusion(a):
+    """Sec. 4.4, the numbered equation: p_i = |a_i|/sum + sum_{k != i} (|a_k|/sum)(|a_i| / sum_{j != k} |a_j|)."""
+    m = np.abs(np.asarray(a, dtype=np.float64))
+    total = m.sum()
+    p = np.zeros(4)
+    for i in range(4):
+        p[i] = m[i] / total + sum(m[k] / total * m[i] / (total - m[k]) for k in range(4) if k != i and m[k] > 0)
+    return p
+
+
+def approx24_variance(a) -> float:
+    """Block variance of approx-MVUE: Sec. 4.2's variance equation at the inclusion probabilities of Sec. 4.4."""
+    return block_variance(a, approx24_inclusion(a))
+
+
+def opt24_variance(a) -> float:
+    """Block variance of the optimal 2:4 estimator: the same equation at the optimal marginals."""
+    return block_variance(a, marginals24(a))
+
+
 # ------------------------------------------- 1:2 comparison estimators -------
 def estimator12(name: str, a1: float, a2: float):
     """Table 2's 1:2 pruners as a list of (probability, [theta_1, theta_2])."""
