@@ -154,7 +154,7 @@ def oracle_sample(cfg, n, m, sample_rows: int, joint: int = 0):
 def run_reference(args, cfg, n, m):
     if int(os.environ.get("RANK", "0")) != 0:
         return
-    joint = 1 if args.joint == "systematic" else 0
+    joint = {"table": 0, "systematic": 1, "approx": 2}[args.joint]
     # size the per-step sample so that K + W steps of the oracle take about a minute in all: its cost
     # grows faster than linearly with the rows (the plain loops leave the cache), so probe by doubling
     per_step_s = 60.0 / max(1, args.steps + args.warmup)
@@ -225,7 +225,8 @@ def run_ours(args, cfg, n, m):
     step_bytes = p_bytes + m_bytes
     gemm_flops = 2.0 * out * inp * T
 
-    joints = {"table": binding.MVUE_JOINT_TABLE, "systematic": binding.MVUE_JOINT_SYSTEMATIC}
+    joints = {"table": binding.MVUE_JOINT_TABLE, "systematic": binding.MVUE_JOINT_SYSTEMATIC,
+              "approx": binding.MVUE_JOINT_APPROX}
     joint = [joints[args.joint]]                        # a cell, so that the other law can be timed with the same step
 
     def step(i, ev=None):
@@ -269,22 +270,22 @@ def run_ours(args, cfg, n, m):
     ms_per_step = ms / args.steps
     value = world * step_bytes / (ms_per_step * 1e-3) / 1e9
 
-    # the same step with the other 2:4 law over pairs, for the per-kernel prune time only (the product that
+    # the same step with the other 2:4 estimators, for the per-kernel prune time only (the product that
     # follows keeps L2 cold for the next prune exactly as in the timed region above)
-    other = None
+    others = []
     if rank == 0 and world == 1 and m == 4 and not args.no_extra:
-        other_name = "systematic" if args.joint == "table" else "table"
-        joint[0] = joints[other_name]
-        k2 = max(3, min(args.steps, 200))
-        for i in range(3):
-            step(i)
-        evs2 = [[torch.cuda.Event(enable_timing=True) for _ in range(3)] for _ in range(k2)]
-        torch.cuda.synchronize()
-        for i in range(k2):
-            step(i, evs2[i])
-        torch.cuda.synchronize()
+        for other_name in [k for k in joints if k != args.joint]:
+            joint[0] = joints[other_name]
+            k2 = max(3, min(args.steps, 200))
+            for i in range(3):
+                step(i)
+            evs2 = [[torch.cuda.Event(enable_timing=True) for _ in range(3)] for _ in range(k2)]
+            torch.cuda.synchronize()
+            for i in range(k2):
+                step(i, evs2[i])
+            torch.cuda.synchronize()
+            others.append((other_name, float(np.mean([e[0].elapsed_time(e[1]) for e in evs2])), k2))
         joint[0] = joints[args.joint]
-        other = (other_name, float(np.mean([e[0].elapsed_time(e[1]) for e in evs2])), k2)
 
     # dense cuBLAS bf16 for the same shape (context for the sparse product)
     dense_ms = None
@@ -360,13 +361,16 @@ def run_ours(args, cfg, n, m):
                                "traffic": ncu_traffic("prune_axis0_bf16_kernel", args.workload)
                                if (n, m, args.joint) == (2, 4, "table") else None},
         }
-        if other is not None:
+        for other in others:
             ogbs = p_bytes / (other[1] * 1e-3) / 1e9
-            line["prune_other_joint"] = {"joint": other[0], "ms": other[1], "gbs": ogbs,
-                                         "frac_of_hbm_peak": ogbs / peaks["hbm_gbs"], "steps": other[2]}
+            key = "prune_other_joint" if other[0] in ("table", "systematic") else "prune_" + other[0]
+            line[key] = {"joint": other[0], "ms": other[1], "gbs": ogbs,
+                         "frac_of_hbm_peak": ogbs / peaks["hbm_gbs"], "steps": other[2]}
         if world == 1 and not args.no_extra:
             line["ffn_large"] = tensor_bound_case(n, m, peaks, joint[0])
             line["mlp_stack"] = chain_case(n, m)
+        if world == 1 and args.sweep:
+            line["prune_sweep"] = prune_sweep(peaks)
         if world == 1 and not args.no_cpu_baseline:
             sample_rows = min(T, 65536)
             gbs, threads, dt = oracle_sample(cfg, n, m, sample_rows, joint[0])
@@ -429,6 +433,71 @@ def tensor_bound_case(n, m, peaks, joint):
             "roofline": {"bound": "tensor", "kernel": "sparse_gemm_pair_kernel", "achieved": tf,
                          "peak": 2 * peaks["bf16_tflops"], "unit": "TFLOP/s", "frac": tf / (2 * peaks["bf16_tflops"]),
                          "peak_source": peaks["source"] + " dense bf16 burst x 2 (2:4 sparse)", "traffic": None}}
+
+
+def prune_sweep(peaks, max_log2: int = 32):
+    """Standalone prune+pack bandwidth over bf16 tensors of 2^20 .. 2^max_log2 bytes ([bytes / 8192 x 4096],
+    Student-t values), both pruned axes, 2:4 (pair table, systematic sampling) and 1:2.  Every point is a CUDA graph of
+    `reps` launches over rotating input copies that together exceed 2.5 x L2, replayed and timed with events, so the
+    small sizes are neither launch-bound on the host nor L2-warm."""
+    import torch
+    from paper_2203_10991_b200 import binding, workloads
+    dev = torch.device("cuda")
+    TC = binding.MVUE_LAYOUT_TC
+    l2 = 126e6
+    cols = 4096
+    # 256 MB of seeded values drawn on the host, tiled on the device up to the largest tensor
+    seed_rows = 1 << 15
+    base = workloads.gradient((seed_rows, cols), "student_t", 5, dtype="bf16")
+    base_dev = torch.from_numpy(base.view(np.int16)).to(dev).view(torch.bfloat16)
+    total_rows = 1 << (max_log2 - 13)
+    if total_rows > seed_rows:
+        base_dev = base_dev.repeat(total_rows // seed_rows, 1)
+    out_v = torch.empty(base_dev.numel() // 2, dtype=torch.bfloat16, device=dev)
+    out_m = torch.empty(base_dev.numel() // 8 + (1 << 16), dtype=torch.uint8, device=dev)
+    modes = [("2:4 table", 2, 4, binding.MVUE_JOINT_TABLE), ("2:4 systematic", 2, 4, binding.MVUE_JOINT_SYSTEMATIC),
+             ("1:2", 1, 2, binding.MVUE_JOINT_TABLE)]
+    points = []
+    side = torch.cuda.Stream()
+    for lg in range(20, max_log2 + 1):
+        nbytes = 1 << lg
+        rows = nbytes // (2 * cols)
+        copies = max(1, min(int(2.5 * l2 / nbytes) + 1, (base_dev.numel() * 2) // nbytes))
+        reps = max(4, min(64, copies))
+        views = [base_dev[i * rows:(i + 1) * rows] for i in range(copies)]
+        point = {"bytes": nbytes, "shape": [rows, cols], "copies": copies}
+        for axis in (0, 1):
+            mrows, k = (rows, cols) if axis == 1 else (cols, rows)
+            values = out_v[:mrows * k // 2].view(mrows, k // 2)
+            for name, n, m, joint in modes:
+                def burst():
+                    for i in range(reps):
+                        binding.mvue_prune(views[i % copies], n, m, axis, i, values=values, meta=out_m, layout=TC,
+                                           joint=joint)
+                side.wait_stream(torch.cuda.current_stream())
+                with torch.cuda.stream(side):
+                    burst()
+                torch.cuda.current_stream().wait_stream(side)
+                torch.cuda.synchronize()
+                graph = torch.cuda.CUDAGraph()
+                with torch.cuda.graph(graph):
+                    burst()
+                graph.replay()
+                torch.cuda.synchronize()
+                e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+                e0.record()
+                graph.replay()
+                e1.record()
+                torch.cuda.synchronize()
+                us = e0.elapsed_time(e1) * 1e3 / reps
+                gbs = prune_bytes(rows, cols, 2) / us / 1e3
+                point[f"axis{axis} {name}"] = {"us": round(us, 2), "gbs": round(gbs, 1),
+                                               "frac_of_hbm_peak": round(gbs / peaks["hbm_gbs"], 4)}
+                del graph
+        points.append(point)
+    return {"dtype": "bf16", "cols": cols, "dist": "student_t", "layout": "tensor-core metadata order",
+            "timing": "CUDA graph replay, inputs rotated over > 2.5 x L2 where the tensor is smaller than that",
+            "points": points}
 
 
 def chain_case(n, m):
@@ -517,9 +586,11 @@ def main():
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--workload", default="conv_im2col")
     ap.add_argument("--prune", default="2:4")
-    ap.add_argument("--joint", default="table", choices=["table", "systematic"],
+    ap.add_argument("--joint", default="table", choices=["table", "systematic", "approx"],
                     help="2:4 law over pairs used by the step: App. A.2 pair table, or systematic sampling")
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--sweep", action="store_true",
+                    help="add the standalone prune+pack bandwidth sweep over bf16 tensors of 1 MB .. 4 GB")
     ap.add_argument("--no-extra", action="store_true",
                     help="skip the riders: the other 2:4 law, the tensor-bound ffn_large case and the MLP-stack chain")
     args = ap.parse_args()

@@ -63,8 +63,23 @@ typedef enum { MVUE_F32 = 0, MVUE_BF16 = 1 } mvue_dtype;
  *   interval of length e_k = min(|a_k|, sum of the other three) of [0, D), D = sum e_k; the owners
  *   of t and t + D/2 survive, t = eps D/2 (eps: the top 23 bits of the block's random word);
  *   a survivor becomes sign(a_k) max(|a_k|, D/2).  About a fifth fewer instructions per block.
+ * MVUE_JOINT_APPROX:     not a law with the optimal marginals but the approximate estimator of
+ *   Sec. 4.4 ("approx-MVUE", the one the paper's 2:4 accuracy tables were run with): element i is
+ *   drawn with probability |a_i| / sum, then j among the other three with probability
+ *   |a_j| / (sum - |a_i|), in the block's own order; a survivor becomes a_k / p_k with p_k the
+ *   inclusion probability given by that section's equation, so E[theta(a)] = a still holds, with a
+ *   block variance the paper's scan bounds below twice the optimum.  It takes TWO random words per
+ *   block: block q reads words 2 (q & 1) and 2 (q & 1) + 1 of generator call q >> 1 (same key).
+ *   Arithmetic, binary32 in this order: m_k = |a_k|; c_1 = m_0, c_2 = c_1 + m_1, c_3 = c_2 + m_2,
+ *   s = c_3 + m_3; t_1 = n_1 (s 2^-24), i = #{c_k <= t_1}; R_k = the sum of the other three
+ *   magnitudes in position order, (x + y) + z; the second draw walks the others' running sums d_1,
+ *   d_2 with t_2 = n_2 (R_i 2^-24); vv_k = m_k / R_k; T_k = the sum of the other three vv in position
+ *   order; survivor k becomes sign(a_k) s / (1 + T_k) (IEEE divisions).  If R_i = 0 (at most one
+ *   non-zero) both survivors keep their own values.  Blocks whose non-zero magnitudes span more than
+ *   2^100, or sum to less than 2^-100, are outside the contract (valid pattern, unspecified values).
+ *   On this hardware the six divisions make it the slowest of the three, not the cheapest.
  * 1:2 has a single law (Sec. 4.1) and ignores the choice. */
-typedef enum { MVUE_JOINT_TABLE = 0, MVUE_JOINT_SYSTEMATIC = 1 } mvue_joint;
+typedef enum { MVUE_JOINT_TABLE = 0, MVUE_JOINT_SYSTEMATIC = 1, MVUE_JOINT_APPROX = 2 } mvue_joint;
 
 /* Packed operand layouts.
  * MVUE_LAYOUT_CANONICAL: for the sparse operand A[Mrows x K] (K = pruned axis)
@@ -131,7 +146,7 @@ MVUE_API int mvue_prune(const void* g, int dtype, int64_t rows, int64_t cols, in
                int axis, uint64_t seed, int64_t k_total, int64_t k_offset, void* values,
                void* meta, int layout, void* stream);
 
-/* mvue_prune with the 2:4 joint law chosen by the caller (an mvue_joint; mvue_prune itself uses
+/* mvue_prune with the 2:4 estimator chosen by the caller (an mvue_joint; mvue_prune itself uses
  * MVUE_JOINT_TABLE).  Everything else -- block numbering, random words, packed layouts, arguments,
  * preconditions, errors -- is as for mvue_prune; an unknown joint gives MVUE_ERR_JOINT. */
 MVUE_API int mvue_prune_joint(const void* g, int dtype, int64_t rows, int64_t cols, int64_t ld, int n, int m,

@@ -17,7 +17,7 @@ _lib = None
 MVUE_F32, MVUE_BF16 = 0, 1
 MVUE_LAYOUT_CANONICAL = 0
 MVUE_LAYOUT_TC = 1
-MVUE_JOINT_TABLE, MVUE_JOINT_SYSTEMATIC = 0, 1
+MVUE_JOINT_TABLE, MVUE_JOINT_SYSTEMATIC, MVUE_JOINT_APPROX = 0, 1, 2
 
 EXPORTS = ("mvue_version", "mvue_status_string", "mvue_last_cuda_error", "mvue_packed_sizes",
            "mvue_prune", "mvue_prune_joint", "mvue_unpack", "mvue_sparse_update_gemm", "mvue_sparse_backward_gemm",

@@ -92,7 +92,7 @@ const char* mvue_status_string(int status) {
         case MVUE_ERR_ARCH: return "device is not compute capability 10.x";
         case MVUE_ERR_CUDA: return "CUDA call failed (see mvue_last_cuda_error)";
         case MVUE_ERR_DEVICE_TIMEOUT: return "a bounded device-side wait expired";
-        case MVUE_ERR_JOINT: return "unknown joint law (only the App. A.2 table and systematic sampling)";
+        case MVUE_ERR_JOINT: return "unknown 2:4 estimator (App. A.2 table, systematic sampling or approx-MVUE)";
         default: return "unknown status";
     }
 }
@@ -126,7 +126,7 @@ int mvue_prune_joint(const void* g, int dtype, int64_t rows, int64_t cols, int64
                      int axis, uint64_t seed, int64_t k_total, int64_t k_offset, void* values,
                      void* meta, int layout, int joint, void* stream) {
     if (!g || !values || !meta) return MVUE_ERR_NULL;
-    if (joint != MVUE_JOINT_TABLE && joint != MVUE_JOINT_SYSTEMATIC) return MVUE_ERR_JOINT;
+    if (joint != MVUE_JOINT_TABLE && joint != MVUE_JOINT_SYSTEMATIC && joint != MVUE_JOINT_APPROX) return MVUE_ERR_JOINT;
     if (dtype != MVUE_F32 && dtype != MVUE_BF16) return MVUE_ERR_DTYPE;
     if (int s = mvue_packed_sizes(rows, cols, n, m, axis, layout, nullptr, nullptr)) return s;
     const int64_t K = axis == 1 ? cols : rows;

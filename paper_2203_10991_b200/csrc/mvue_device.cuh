@@ -314,15 +314,95 @@ __device__ __forceinline__ void mvue_2of4_sys_f32(uint32_t b0, uint32_t b1, uint
     *nibble = 14u - r.li - 4u * r.lj;
 }
 
+// ===========================================================================
+// Approximately optimal 2:4 (Sec. 4.4, "approx-MVUE"): two sequential draws without
+// replacement, each proportional to magnitude; a survivor is divided by its exact
+// inclusion probability p_k = (m_k / s)(1 + T_k), T_k = sum_{l != k} m_l / R_l, R_l = sum of
+// the magnitudes other than l (the equation of Sec. 4.4), i.e. becomes sign(a_k) s / (1 + T_k).
+// Block order, no sort; two random words per block.
+//   first draw:  c_1 = m_0, c_2 = c_1 + m_1, c_3 = c_2 + m_2, s = c_3 + m_3,
+//                t_1 = n_1 (s 2^-24), i = #{c_k <= t_1};
+//   second draw among the others in position order, d_1, d_2 their running sums,
+//                t_2 = n_2 (R_i 2^-24), j = the #{d_k <= t_2}-th of them;
+//   sums of three run in position order, (x + y) + z; the six divisions are IEEE.
+//   R_i = 0 (at most one non-zero): both survivors keep their own values.
+// Unlike the two exact laws this one cannot avoid division, so on this hardware it is the
+// most expensive of the three estimators, not the cheapest.
+// ===========================================================================
+__device__ __forceinline__ float sel4(uint32_t k, float x0, float x1, float x2, float x3) {
+    return k < 2u ? (k == 0u ? x0 : x1) : (k == 2u ? x2 : x3);
+}
+
+// b0..b3: the block as binary32 bit patterns.  out = the two survivors as bf16 (lower position in the
+// low half), nibble = idx0 | idx1 << 2.
+__device__ __forceinline__ void mvue_2of4_approx_f32(uint32_t b0, uint32_t b1, uint32_t b2, uint32_t b3,
+                                                     uint32_t word1, uint32_t word2, uint32_t* out,
+                                                     uint32_t* nibble) {
+    const float m0 = fabsf(__uint_as_float(b0)), m1 = fabsf(__uint_as_float(b1));
+    const float m2 = fabsf(__uint_as_float(b2)), m3 = fabsf(__uint_as_float(b3));
+    const float q01 = __fadd_rn(m0, m1), q12 = __fadd_rn(m1, m2), q02 = __fadd_rn(m0, m2);
+    const float R3 = __fadd_rn(q01, m2), R2 = __fadd_rn(q01, m3), R1 = __fadd_rn(q02, m3), R0 = __fadd_rn(q12, m3);
+    const float s = __fadd_rn(R3, m3);
+    const float t1 = __fmul_rn(top24(word1), __fmul_rn(s, 5.9604644775390625e-08f));
+    const uint32_t i = (m0 <= t1 ? 1u : 0u) + (q01 <= t1 ? 1u : 0u) + (R3 <= t1 ? 1u : 0u);
+    const float Ri = sel4(i, R0, R1, R2, R3);
+    const float d1 = i == 0u ? m1 : m0;
+    const float d2 = sel4(i, q12, q02, q01, q01);
+    const float t2 = __fmul_rn(top24(word2), __fmul_rn(Ri, 5.9604644775390625e-08f));
+    const uint32_t jj = (d1 <= t2 ? 1u : 0u) + (d2 <= t2 ? 1u : 0u);
+    const uint32_t j = jj + (jj >= i ? 1u : 0u);
+    // The IEEE division leaves its short path when an operand is zero, and zeros are everywhere in a
+    // ReLU-sparse gradient: divide stand-ins instead (0 / R is 0 whatever R; a quotient by R = 0 is only
+    // ever read when R_i = 0, where the survivors keep their own values), so that the warp stays together.
+    auto quot = [](float num, float den) {
+        const float q = __fdiv_rn(num == 0.0f ? 1.0f : num, den == 0.0f ? 1.0f : den);
+        return num == 0.0f ? 0.0f : q;
+    };
+    const float vv0 = quot(m0, R0), vv1 = quot(m1, R1), vv2 = quot(m2, R2), vv3 = quot(m3, R3);
+    const float u01 = __fadd_rn(vv0, vv1), u12 = __fadd_rn(vv1, vv2), u02 = __fadd_rn(vv0, vv2);
+    const uint32_t lo = min(i, j), hi = max(i, j);
+    // T_k = (sum of two) + (the last of the others)
+    const float Tlo = __fadd_rn(sel4(lo, u12, u02, u01, u01), lo == 3u ? vv2 : vv3);
+    const float Thi = __fadd_rn(sel4(hi, u12, u02, u01, u01), hi == 3u ? vv2 : vv3);
+    const bool own = Ri == 0.0f;
+    const float s_div = own ? 1.0f : s;                      // s may be 0 only when own
+    const float scaled_lo = __fdiv_rn(s_div, __fadd_rn(1.0f, Tlo)), scaled_hi = __fdiv_rn(s_div, __fadd_rn(1.0f, Thi));
+    const float mag_lo = own ? sel4(lo, m0, m1, m2, m3) : scaled_lo;
+    const float mag_hi = own ? sel4(hi, m0, m1, m2, m3) : scaled_hi;
+    const uint32_t blo = lo < 2u ? (lo == 0u ? b0 : b1) : (lo == 2u ? b2 : b3);
+    const uint32_t bhi = hi < 2u ? (hi == 0u ? b0 : b1) : (hi == 2u ? b2 : b3);
+    const float vlo = __uint_as_float(__float_as_uint(mag_lo) | (blo & 0x80000000u));
+    const float vhi = __uint_as_float(__float_as_uint(mag_hi) | (bhi & 0x80000000u));
+    *out = pack_bf16x2(vlo, vhi);
+    *nibble = lo | (hi << 2);
+}
+
+// bf16 source: x01 = a0 | a1 << 16, x23 = a2 | a3 << 16 (widened exactly).
+__device__ __forceinline__ void mvue_2of4_approx_bf16(uint32_t x01, uint32_t x23, uint32_t word1, uint32_t word2,
+                                                      uint32_t* out, uint32_t* nibble) {
+    mvue_2of4_approx_f32(x01 << 16, x01 & 0xFFFF0000u, x23 << 16, x23 & 0xFFFF0000u, word1, word2, out, nibble);
+}
+
 // One work unit of bf16 input: raw[8] = 16 elements along K, two per word.
-// kJoint selects the 2:4 law over pairs (0: App. A.2 table, 1: systematic sampling); 1:2 has one law.
+// kJoint selects the 2:4 estimator (0: App. A.2 table, 1: systematic sampling, 2: approx-MVUE of Sec. 4.4,
+// which takes two words per block: one generator call per two blocks); 1:2 has one law.
 template <int M, int kJoint = 0>
 __device__ __forceinline__ void prune_unit_bf16(const uint32_t (&raw)[8], uint64_t unit_index,
                                                 const RoundKeys& rk, uint4* out_values,
                                                 uint32_t* out_meta) {
     uint32_t v[4];                                   // 8 survivors, two bf16 per word
     uint32_t meta = 0;
-    if (M == 4) {
+    if (M == 4 && kJoint == 2) {
+        const uint4 wa = philox4x32_10(2 * unit_index, rk);
+        const uint4 wb = philox4x32_10(2 * unit_index + 1, rk);
+        const uint32_t words[8] = {wa.x, wa.y, wa.z, wa.w, wb.x, wb.y, wb.z, wb.w};
+#pragma unroll
+        for (int j = 0; j < 4; ++j) {
+            uint32_t nib;
+            mvue_2of4_approx_bf16(raw[2 * j], raw[2 * j + 1], words[2 * j], words[2 * j + 1], &v[j], &nib);
+            meta += nib << (4 * j);
+        }
+    } else if (M == 4) {
         const uint4 w = philox4x32_10(unit_index, rk);
         const uint32_t words[4] = {w.x, w.y, w.z, w.w};
 #pragma unroll
@@ -356,7 +436,19 @@ __device__ __forceinline__ void prune_unit_bf16_rows(const uint32_t (&w)[16], ui
                                                      const RoundKeys& rk, uint4* out_values, uint32_t* out_meta) {
     uint32_t v[4];
     uint32_t meta = 0;
-    if (M == 4) {
+    if (M == 4 && kJoint == 2) {
+        const uint4 ra = philox4x32_10(2 * unit_index, rk);
+        const uint4 rb = philox4x32_10(2 * unit_index + 1, rk);
+        const uint32_t words[8] = {ra.x, ra.y, ra.z, ra.w, rb.x, rb.y, rb.z, rb.w};
+#pragma unroll
+        for (int j = 0; j < 4; ++j) {
+            uint32_t nib;
+            auto widen = [](uint32_t x) { return kHigh ? (x & 0xFFFF0000u) : (x << 16); };
+            mvue_2of4_approx_f32(widen(w[4 * j]), widen(w[4 * j + 1]), widen(w[4 * j + 2]), widen(w[4 * j + 3]),
+                                 words[2 * j], words[2 * j + 1], &v[j], &nib);
+            meta += nib << (4 * j);
+        }
+    } else if (M == 4) {
         const uint4 r = philox4x32_10(unit_index, rk);
         const uint32_t words[4] = {r.x, r.y, r.z, r.w};
 #pragma unroll

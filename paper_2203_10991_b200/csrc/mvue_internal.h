@@ -19,7 +19,7 @@ struct PruneArgs {
     void* meta;
     int sm_count;
     bool tc_layout;      // metadata in tensor-core order instead of canonical rows
-    int joint;           // 2:4 law over pairs: 0 = App. A.2 table, 1 = systematic sampling
+    int joint;           // 2:4 estimator: 0 = App. A.2 table, 1 = systematic sampling, 2 = approx-MVUE (Sec. 4.4)
 };
 
 cudaError_t launch_prune(const PruneArgs& a, cudaStream_t stream);
