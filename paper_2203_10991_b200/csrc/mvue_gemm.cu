@@ -549,11 +549,13 @@ sparse_gemm_pair_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_
                         }
                     }
                 }
-                // the accumulator is in registers: give tensor memory back before touching global memory
+                // the accumulator is in registers (tcgen05.wait::ld has returned in every lane): give tensor
+                // memory back before touching global memory.  The arrival orders nothing but that, so it is
+                // relaxed: a release at cluster scope would first wait out the previous tile's global stores.
                 tc_fence_before();
                 __syncwarp();
                 if (lane == 0)
-                    asm volatile("mbarrier.arrive.release.cluster.shared::cluster.b64 _, [%0];" ::"r"(leader_free) : "memory");
+                    asm volatile("mbarrier.arrive.relaxed.cluster.shared::cluster.b64 _, [%0];" ::"r"(leader_free) : "memory");
                 ++tiles_done;
             } else {
 #pragma unroll
