@@ -360,6 +360,30 @@ __device__ __forceinline__ void store8_b32(void* dst, const uint32_t* v) {
     }
 }
 
+// 4 x 4 transpose of 16-word cells among the four lanes of a quad.  v[] is one row of 64 words seen as eight
+// 32-byte chunks; cell c = chunks c and c + 4 (words 8 c .. 8 c + 7 and 32 + 8 c .. 32 + 8 c + 7).  On entry a lane
+// holds the cells of its own row; on exit its cell c is cell (lane % 4) of the row of quad lane c, so that the four
+// lanes of a quad together hold whole 128-byte lines of each of the quad's four rows and a warp-wide 32-byte access
+// touches 8 lines instead of 32.  The transpose is its own inverse.
+__device__ __forceinline__ void quad_transpose(uint32_t (&v)[64], int lane) {
+#pragma unroll
+    for (int m = 1; m <= 2; m <<= 1) {
+        const bool up = (lane & m) != 0;
+#pragma unroll
+        for (int c = 0; c < 4; ++c) {
+            if (c & m) continue;
+#pragma unroll
+            for (int i = 0; i < 16; ++i) {
+                const int lo = (i < 8 ? 0 : 32) + 8 * c + (i & 7), hi = lo + 8 * m;   // cell c and cell c + m
+                const uint32_t send = up ? v[lo] : v[hi];
+                const uint32_t recv = __shfl_xor_sync(0xFFFFFFFFu, send, m);
+                if (up) v[lo] = recv;
+                else v[hi] = recv;
+            }
+        }
+    }
+}
+
 // Persistent kernel: every pair of thread blocks walks the work items pair, pair + #pairs, ...
 //   warp 0      TMA producer (both blocks); runs ahead into the next tile while the current one drains
 //   warp 1      metadata copy + MMA issue (leader block only)
@@ -502,27 +526,46 @@ sparse_gemm_pair_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_
             // bf16 x scale keeps the row's factors in registers; fp32 x scale has no room for them beside 128
             // fp32 results and applies them after tensor memory has been handed back
             constexpr bool kScale = kMode == 2, kLateScale = kMode == 3, kToBf16 = kMode == 1 || kMode == 2;
-            uint4 sc[kScale ? 16 : 1];
-            if (kScale) {                                        // this row's scale factors, fetched under the main loop
-                const __nv_bfloat16* src = p.scale + row * p.ldc + col0;
-                const bool wide = (reinterpret_cast<uintptr_t>(src) & 31u) == 0;   // whole 32-byte sectors per load
+            // bf16 outputs and their factors move in the quad-transposed arrangement (quad_transpose): lane
+            // 4 a + b reads / writes, for c = 0..3 and k = 0, 1, the 32-byte chunk b + 4 k of row 4 a + c of the warp's
+            // 32 rows, i.e. the quad covers whole 128-byte lines.
+            const int64_t row_q = it.m0 + 32 * q + 4 * (lane >> 2);      // first row of this lane's quad
+            const int64_t col_q = col0 + 16 * (lane & 3);                // this lane's chunk (k = 0) of those rows
+            uint32_t scw[kScale ? 64 : 1];
+            if constexpr (kScale) {                              // the factors, fetched under the main loop
 #pragma unroll
-                for (int e = 0; e < 16; e += 2) {
-                    sc[e] = sc[e + 1] = make_uint4(0u, 0u, 0u, 0u);
-                    if (row_ok && wide && col0 + 8 * e + 8 < p.N) {
-                        asm volatile("ld.global.nc.L1::no_allocate.v8.b32 {%0, %1, %2, %3, %4, %5, %6, %7}, [%8];"
-                                     : "=r"(sc[e].x), "=r"(sc[e].y), "=r"(sc[e].z), "=r"(sc[e].w), "=r"(sc[e + 1].x),
-                                       "=r"(sc[e + 1].y), "=r"(sc[e + 1].z), "=r"(sc[e + 1].w)
-                                     : "l"(src + 8 * e));
-                    } else if (row_ok) {
-                        if (col0 + 8 * e < p.N) sc[e] = __ldg(reinterpret_cast<const uint4*>(src + 8 * e));
-                        if (col0 + 8 * e + 8 < p.N) sc[e + 1] = __ldg(reinterpret_cast<const uint4*>(src + 8 * e + 8));
+                for (int c = 0; c < 4; ++c) {
+#pragma unroll
+                    for (int k = 0; k < 2; ++k) {
+                        uint32_t* d = &scw[32 * k + 8 * c];
+#pragma unroll
+                        for (int t = 0; t < 8; ++t) d[t] = 0u;
+                        const int64_t cc = col_q + 64 * k;
+                        if (row_q + c >= p.M) continue;
+                        const __nv_bfloat16* src = p.scale + (row_q + c) * p.ldc + cc;
+                        if (cc + 8 < p.N && (reinterpret_cast<uintptr_t>(src) & 31u) == 0) {   // one whole 32-byte sector
+                            asm volatile("ld.global.nc.L1::no_allocate.v8.b32 {%0, %1, %2, %3, %4, %5, %6, %7}, [%8];"
+                                         : "=r"(d[0]), "=r"(d[1]), "=r"(d[2]), "=r"(d[3]), "=r"(d[4]), "=r"(d[5]),
+                                           "=r"(d[6]), "=r"(d[7])
+                                         : "l"(src));
+                        } else {
+                            if (cc < p.N) {
+                                const uint4 v4 = __ldg(reinterpret_cast<const uint4*>(src));
+                                d[0] = v4.x; d[1] = v4.y; d[2] = v4.z; d[3] = v4.w;
+                            }
+                            if (cc + 8 < p.N) {
+                                const uint4 v4 = __ldg(reinterpret_cast<const uint4*>(src + 8));
+                                d[4] = v4.x; d[5] = v4.y; d[6] = v4.z; d[7] = v4.w;
+                            }
+                        }
                     }
                 }
+                quad_transpose(scw, lane);                       // back to one row per lane, as the drain multiplies
             }
             uint32_t r[kToBf16 ? 64 : 128];                      // packed bf16 pairs, or fp32 bit patterns
             if (it.n_steps > 0) {
-                if (!mbar_wait(acc_bar, tiles_done & 1u, abort_flag)) break;
+                // (warp-uniform: the lanes shuffle with each other further down)
+                if (!__all_sync(0xFFFFFFFFu, mbar_wait(acc_bar, tiles_done & 1u, abort_flag))) break;
                 tc_fence_after();
 #pragma unroll
                 for (int half = 0; half < 2; ++half) {           // 64 columns at a time
@@ -535,8 +578,7 @@ sparse_gemm_pair_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_
                         float f0 = __uint_as_float(e < 32 ? t0[e] : t1[e - 32]);
                         float f1 = __uint_as_float(e < 32 ? t0[e + 1] : t1[e - 31]);
                         if (kScale) {
-                            const uint4 s4 = sc[(64 * half + e) / 8];
-                            const uint32_t sw = (e % 8) < 2 ? s4.x : ((e % 8) < 4 ? s4.y : ((e % 8) < 6 ? s4.z : s4.w));
+                            const uint32_t sw = scw[(64 * half + e) / 2];
                             f0 *= __uint_as_float(sw << 16);
                             f1 *= __uint_as_float(sw & 0xFFFF0000u);
                         }
@@ -560,6 +602,22 @@ sparse_gemm_pair_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_
             } else {
 #pragma unroll
                 for (int e = 0; e < (kToBf16 ? 64 : 128); ++e) r[e] = 0u;
+            }
+            if constexpr (kToBf16) {
+                quad_transpose(r, lane);
+#pragma unroll
+                for (int c = 0; c < 4; ++c) {
+#pragma unroll
+                    for (int k = 0; k < 2; ++k) {
+                        const int64_t cc = col_q + 64 * k;
+                        if (row_q + c >= p.M) continue;
+                        __nv_bfloat16* dst = reinterpret_cast<__nv_bfloat16*>(p.C) + (row_q + c) * p.ldc + cc;
+                        const uint32_t* v = &r[32 * k + 8 * c];
+                        if (cc + 8 < p.N) store8_b32(dst, v);
+                        else if (cc < p.N) *reinterpret_cast<uint4*>(dst) = make_uint4(v[0], v[1], v[2], v[3]);
+                    }
+                }
+                continue;
             }
             if (!row_ok) continue;
             if (!kToBf16 && it.tail_slot >= 0) {             // a K part of a tail tile: unscaled fp32 partial tile
