@@ -54,3 +54,63 @@ def test_bench_workload_full_size(name, n, m, check_rows):
             w = oracle.gemm_entry(A_rows[i_r], h, j)
             scale = float(np.abs(A_rows[i_r]).sum()) * 3.0
             assert abs(got[r, j] - w) <= 1e-5 * scale + 1e-4 * abs(w), (r, j, got[r, j], w)
+
+
+def test_mlp_stack_block_full_size():
+    """One block of the MLP-stack workload at full size (T = 32768, d = 1024, d_ff = 4096): the two layers' four
+    prunes bit for bit over the whole tensors, and the two update and two backward products (f'(z) epilogue, bf16
+    out) on seeded samples computed entry by entry in fp64.  Each layer is checked on the gradient the GPU chain
+    actually propagated, so a mismatch names the step that made it."""
+    cfg = workloads.CONFIGS["mlp_stack"]
+    T, d_ff, d = cfg["T"], cfg["out"], cfg["inp"]
+    th = oracle.host_threads()
+    rng = np.random.Generator(np.random.PCG64(11))
+    g_np = workloads.gradient((T, d), cfg["g_dist"], cfg["seed"], dtype="bf16")
+    for layer, (n_out, n_in) in enumerate([(d, d_ff), (d_ff, d)]):
+        W = workloads.normal_bf16((n_out, n_in), seed=50 + layer, std=n_in ** -0.5)
+        h = workloads.normal_bf16((T, n_in), seed=60 + layer)
+        act = workloads.normal_bf16((T, n_in), seed=70 + layer)
+        g_dev, W_dev, h_dev, act_dev = to_dev(g_np), to_dev(W), to_dev(h), to_dev(act)
+        status = torch.zeros(1, dtype=torch.int32, device="cuda")
+        s_upd, s_bwd = 1000 + 2 * layer, 1001 + 2 * layer
+        v0, m0 = binding.mvue_prune(g_dev, 2, 4, 0, s_upd, layout=TC)
+        dW = binding.mvue_sparse_update_gemm(v0, m0, h_dev, dev_status=status)
+        v1, m1 = binding.mvue_prune(g_dev, 2, 4, 1, s_bwd, layout=TC)
+        dh = binding.mvue_sparse_backward_gemm(v1, m1, W_dev, act_grad=act_dev, out_dtype=torch.bfloat16,
+                                               dev_status=status)
+        torch.cuda.synchronize()
+        assert int(status.item()) == 0
+
+        # the four packed operands, whole
+        v0_ref, m0_ref = oracle.prune(g_np, 2, 4, axis=0, seed=s_upd, threads=th)
+        v1_ref, m1_ref = oracle.prune(g_np, 2, 4, axis=1, seed=s_bwd, threads=th)
+        assert np.array_equal(v0.view(torch.int16).cpu().numpy().view(np.uint16), v0_ref)
+        assert np.array_equal(m0.cpu().numpy().reshape(-1), layouts.canonical_to_tc(m0_ref))
+        assert np.array_equal(v1.view(torch.int16).cpu().numpy().view(np.uint16), v1_ref)
+        assert np.array_equal(m1.cpu().numpy().reshape(-1), layouts.canonical_to_tc(m1_ref))
+
+        # update product dW[n_out x n_in]: sampled entries
+        got = dW.double().cpu().numpy()
+        rows = sorted(set([0, n_out - 1] + [int(x) for x in rng.integers(0, n_out, 2)]))
+        A_rows = oracle.unpack(np.ascontiguousarray(v0_ref[rows]), np.ascontiguousarray(m0_ref[rows]))
+        for i_r, r in enumerate(rows):
+            for j in [0, n_in - 1] + [int(x) for x in rng.integers(0, n_in, 6)]:
+                w = oracle.gemm_entry(A_rows[i_r], h, j)
+                scale = float(np.abs(A_rows[i_r]).sum()) * 3.0
+                assert abs(got[r, j] - w) <= 1e-5 * scale + 1e-4 * abs(w), ("dW", layer, r, j, got[r, j], w)
+
+        # backward product dh[T x n_in] = (theta(g) W) * f'(z), stored as bf16: sampled entries (first and last tile
+        # rows and columns among them) within bf16 rounding of the fp64 value
+        dh_np = dh.view(torch.int16).cpu().numpy().view(np.uint16)
+        got_h = oracle.bf16_to_f32(dh_np).astype(np.float64)
+        t_rows = sorted(set([0, 127, 128, 255, 256, T - 1] + [int(x) for x in rng.integers(0, T, 10)]))
+        A_t = oracle.unpack(np.ascontiguousarray(v1_ref[t_rows]), np.ascontiguousarray(m1_ref[t_rows]))
+        act_f = oracle.bf16_to_f32(act).astype(np.float64)
+        for i_r, r in enumerate(t_rows):
+            for j in [0, 15, 16, 63, 64, 127, 128, 255, 256, n_in - 1] + [int(x) for x in rng.integers(0, n_in, 6)]:
+                w = oracle.gemm_entry(A_t[i_r], W, j) * act_f[r, j]
+                scale = float(np.abs(A_t[i_r]).sum()) * float(n_in ** -0.5) * 3.0 * abs(act_f[r, j])
+                assert abs(got_h[r, j] - w) <= 2.0 ** -8 * abs(w) + 1e-5 * scale, ("dh", layer, r, j, got_h[r, j], w)
+        g_np = np.ascontiguousarray(dh_np)                  # the next layer sees what the GPU stored
+        del g_dev, W_dev, h_dev, act_dev, v0, m0, v1, m1, dW, dh
+        torch.cuda.empty_cache()
