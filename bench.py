@@ -58,10 +58,14 @@ def gemm_bytes(M: int, N: int, K: int, c_bytes: int = 4) -> int:
 # each kernel (summaries under profiles/).  Each figure is tied to a digest of the sources the kernel is built
 # from: once those change the counters no longer describe the kernel and `traffic` is reported as null.
 NCU_TRAFFIC = {
-    "sparse_gemm_pair_kernel": (982700032 + 4155136, ("mvue_gemm.cu", "mvue_tma.h", "mvue_internal.h"),
-                                "679e6f23023c28dc"),
-    "prune_axis0_bf16_kernel": (103505152 + 26799104,
-                                ("mvue_prune.cu", "mvue_device.cuh", "mvue_tma.h", "mvue_internal.h"), "582b91dc0e5640ff"),
+    "sparse_gemm_pair_kernel": (982788096 + 3833856, ("mvue_gemm.cu", "mvue_tma.h", "mvue_internal.h"),
+                                "3c059758927216a7"),
+    "prune_axis0_bf16_kernel/table": (103706112 + 26853120,
+                                      ("mvue_prune.cu", "mvue_device.cuh", "mvue_tma.h", "mvue_internal.h"),
+                                      "7fb39c818c99b2dd"),
+    "prune_axis0_bf16_kernel/systematic": (103638784 + 25789696,
+                                           ("mvue_prune.cu", "mvue_device.cuh", "mvue_tma.h", "mvue_internal.h"),
+                                           "7fb39c818c99b2dd"),
 }
 
 
@@ -227,12 +231,13 @@ def run_ours(args, cfg, n, m):
 
     joints = {"table": binding.MVUE_JOINT_TABLE, "systematic": binding.MVUE_JOINT_SYSTEMATIC,
               "approx": binding.MVUE_JOINT_APPROX}
-    joint = [joints[args.joint]]                        # a cell, so that the other law can be timed with the same step
+    joint = [joints[args.joint]]                        # cells, so that the other estimators can be timed with the same step
+    nm = [(n, m)]
 
     def step(i, ev=None):
         if ev:
             ev[0].record()
-        binding.mvue_prune(g_dev, n, m, 0, i, values=values, meta=meta, layout=TC, joint=joint[0])
+        binding.mvue_prune(g_dev, nm[0][0], nm[0][1], 0, i, values=values, meta=meta, layout=TC, joint=joint[0])
         if ev:
             ev[1].record()
         binding.mvue_sparse_update_gemm(values, meta, h_dev, out=dW, workspace=ws, dev_status=status)
@@ -286,6 +291,17 @@ def run_ours(args, cfg, n, m):
             torch.cuda.synchronize()
             others.append((other_name, float(np.mean([e[0].elapsed_time(e[1]) for e in evs2])), k2))
         joint[0] = joints[args.joint]
+        # and MVUE 1:2 (emitted as a valid 2:4 pattern, so the same product consumes it)
+        nm[0] = (1, 2)
+        for i in range(3):
+            step(i)
+        evs2 = [[torch.cuda.Event(enable_timing=True) for _ in range(3)] for _ in range(k2)]
+        torch.cuda.synchronize()
+        for i in range(k2):
+            step(i, evs2[i])
+        torch.cuda.synchronize()
+        others.append(("1:2", float(np.mean([e[0].elapsed_time(e[1]) for e in evs2])), k2))
+        nm[0] = (n, m)
 
     # dense cuBLAS bf16 for the same shape (context for the sparse product)
     dense_ms = None
@@ -358,12 +374,13 @@ def run_ours(args, cfg, n, m):
             "roofline_prune": {"bound": "hbm", "kernel": "prune_axis0_bf16_kernel", "achieved": prune_gbs,
                                "peak": peaks["hbm_gbs"], "unit": "GB/s", "frac": prune_gbs / peaks["hbm_gbs"],
                                "peak_source": peaks["source"],
-                               "traffic": ncu_traffic("prune_axis0_bf16_kernel", args.workload)
-                               if (n, m, args.joint) == (2, 4, "table") else None},
+                               "traffic": ncu_traffic("prune_axis0_bf16_kernel/" + args.joint, args.workload)
+                               if (n, m) == (2, 4) else None},
         }
         for other in others:
             ogbs = p_bytes / (other[1] * 1e-3) / 1e9
-            key = "prune_other_joint" if other[0] in ("table", "systematic") else "prune_" + other[0]
+            key = {"table": "prune_other_joint", "systematic": "prune_other_joint", "1:2": "prune_1of2"}.get(
+                other[0], "prune_" + other[0])
             line[key] = {"joint": other[0], "ms": other[1], "gbs": ogbs,
                          "frac_of_hbm_peak": ogbs / peaks["hbm_gbs"], "steps": other[2]}
         if world == 1 and not args.no_extra:
@@ -411,6 +428,8 @@ def tensor_bound_case(n, m, peaks, joint):
     prune_ms = timed(lambda: binding.mvue_prune(g, n, m, 0, 1, values=values, meta=meta, layout=TC, joint=joint), 20)
     sys_ms = timed(lambda: binding.mvue_prune(g, n, m, 0, 1, values=values, meta=meta, layout=TC,
                                               joint=binding.MVUE_JOINT_SYSTEMATIC), 20)
+    table_ms = timed(lambda: binding.mvue_prune(g, n, m, 0, 1, values=values, meta=meta, layout=TC,
+                                                joint=binding.MVUE_JOINT_TABLE), 20)
     binding.mvue_prune(g, n, m, 0, 1, values=values, meta=meta, layout=TC, joint=joint)
     gemm_ms = timed(lambda: binding.mvue_sparse_update_gemm(values, meta, h, out=dW), 30)
     fused_ms = timed(lambda: binding.mvue_fused_update_gemm(g, h, n, m, 1, out=dW), 3)
@@ -423,6 +442,8 @@ def tensor_bound_case(n, m, peaks, joint):
             "prune_ms": prune_ms, "prune_gbs": pgbs, "prune_frac_of_hbm_peak": pgbs / peaks["hbm_gbs"],
             "prune_systematic_ms": sys_ms,
             "prune_systematic_frac_of_hbm_peak": prune_bytes(T, out, 2) / (sys_ms * 1e-3) / 1e9 / peaks["hbm_gbs"],
+            "prune_table_ms": table_ms,
+            "prune_table_frac_of_hbm_peak": prune_bytes(T, out, 2) / (table_ms * 1e-3) / 1e9 / peaks["hbm_gbs"],
             "gemm_ms": gemm_ms, "gemm_tflops_effective": tf,
             "gemm_frac_of_sparse_peak_burst": tf / (2 * peaks["bf16_tflops"]),
             "gemm_frac_of_sparse_peak_sustained": tf / (2 * peaks["bf16_tflops_sustained"]),
@@ -586,8 +607,9 @@ def main():
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--workload", default="conv_im2col")
     ap.add_argument("--prune", default="2:4")
-    ap.add_argument("--joint", default="table", choices=["table", "systematic", "approx"],
-                    help="2:4 law over pairs used by the step: App. A.2 pair table, or systematic sampling")
+    ap.add_argument("--joint", default="systematic", choices=["table", "systematic", "approx"],
+                    help="2:4 estimator used by the step: systematic sampling (the faster of the two exact MVUE laws), "
+                         "the App. A.2 pair table, or approx-MVUE (Sec. 4.4); the others are timed beside it")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--sweep", action="store_true",
                     help="add the standalone prune+pack bandwidth sweep over bf16 tensors of 1 MB .. 4 GB")
