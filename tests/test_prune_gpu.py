@@ -63,6 +63,50 @@ def test_linear_small_config(n, m):
     assert_parity(g, n, m, axis=1, seed=0)
 
 
+@pytest.mark.parametrize("n,m,joint", [(1, 2, None), (2, 4, binding.MVUE_JOINT_TABLE),
+                                       (2, 4, binding.MVUE_JOINT_SYSTEMATIC), (2, 4, binding.MVUE_JOINT_APPROX)])
+def test_linear_small_slice_is_unbiased_over_10k_seeds(n, m, joint):
+    # the 16 x 16 slice of the small linear-layer gradient, pruned by the CUDA kernel under 10000 seeds: the mean of
+    # the unpacked estimates must sit within six standard errors of the gradient, the standard error taken from the
+    # estimator's own survival probabilities (Sec. 4.1 / 4.2 / 4.4)
+    from oracle import theory
+    cfg = workloads.CONFIGS["linear_small"]
+    g = np.ascontiguousarray(
+        workloads.gradient((cfg["T"], cfg["out"]), cfg["g_dist"], cfg["seed"], dtype="f32")[:16, :16])
+    g_dev = to_dev(g)
+    n_seeds = 10000
+    acc = torch.zeros((16, 16), dtype=torch.float64, device=DEV)
+    values = torch.empty((16, 8), dtype=torch.bfloat16, device=DEV)
+    meta = torch.empty((16, 2), dtype=torch.uint8, device=DEV)
+    for seed in range(n_seeds):
+        binding.mvue_prune(g_dev, n, m, 0, seed, values=values, meta=meta, joint=joint)
+        acc += binding.mvue_unpack(values, meta).double()
+    mean = (acc / n_seeds).cpu().numpy()                                   # A = g^T: [16, 16]
+    A = g.T.astype(np.float64)
+    for r in range(16):
+        for j in range(4):
+            blk = A[r, 4 * j:4 * j + 4]
+            if m == 2:
+                p = np.zeros(4)
+                for h in range(2):
+                    s = abs(blk[2 * h]) + abs(blk[2 * h + 1])
+                    if s > 0:
+                        p[2 * h], p[2 * h + 1] = abs(blk[2 * h]) / s, abs(blk[2 * h + 1]) / s
+            elif np.count_nonzero(blk) < 2:
+                p = (blk != 0).astype(np.float64)
+            elif joint == binding.MVUE_JOINT_APPROX:
+                p = theory.approx24_inclusion(blk)
+            else:
+                p = theory.marginals24(blk)
+            for e in range(4):
+                a = blk[e]
+                if a == 0:
+                    assert mean[r, 4 * j + e] == 0
+                    continue
+                sd = np.sqrt(a * a * max(1 / p[e] - 1, 0.0) / n_seeds)
+                assert abs(mean[r, 4 * j + e] - a) <= 6 * sd + 2.0 ** -8 * abs(a), (r, j, e, mean[r, 4 * j + e], a)
+
+
 @pytest.mark.parametrize("n,m", MODES)
 @pytest.mark.parametrize("dtype", ["f32", "bf16"])
 def test_edge_values(n, m, dtype):
