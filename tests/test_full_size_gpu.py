@@ -114,3 +114,56 @@ def test_mlp_stack_block_full_size():
         g_np = np.ascontiguousarray(dh_np)                  # the next layer sees what the GPU stored
         del g_dev, W_dev, h_dev, act_dev, v0, m0, v1, m1, dW, dh
         torch.cuda.empty_cache()
+
+
+@pytest.mark.parametrize("axis", [0, 1])
+def test_prune_4gb_tensor_sampled(axis):
+    """The largest tensor of the bandwidth sweep, bf16 [524288 x 4096] = 4 GiB (element offsets reach 2^31, byte
+    offsets 2^32): seeded slices of the packed output against the oracle, which prunes any block on its own because
+    the random words are a function of the block number.  The tensor is 16 copies of a 256 MiB seeded base stacked
+    along the rows (as in the sweep), so a slice's input is known on the host without moving 4 GiB."""
+    rows, cols, base_rows = 1 << 19, 4096, 1 << 15
+    base = workloads.gradient((base_rows, cols), "student_t", 5, dtype="bf16")
+    g_dev = to_dev(base).repeat(rows // base_rows, 1)
+    assert g_dev.shape == (rows, cols) and g_dev.is_contiguous()
+    seed = 99
+    rng = np.random.Generator(np.random.PCG64(3))
+    for n, m in ((2, 4), (1, 2)):
+        values, meta = binding.mvue_prune(g_dev, n, m, axis, seed)            # canonical layout
+        torch.cuda.synchronize()
+        starts = sorted(set([0, rows - 128, rows // 2, rows // 2 + 128] +
+                            [int(x) * 128 for x in rng.integers(0, rows // 128, 6)]))
+        for lo in starts:
+            part = np.ascontiguousarray(base[np.arange(lo, lo + 128) % base_rows])
+            if axis == 1:      # A = g: rows lo .. lo+127 of A; block numbers depend on the global row
+                # the oracle's tensor call numbers blocks from row 0 of what it is given, so rows far down the
+                # tensor are checked through per-block calls with their global block numbers
+                v_gpu = values[lo:lo + 128].view(torch.int16).cpu().numpy().view(np.uint16)
+                m_gpu = meta[lo:lo + 128].cpu().numpy()
+                for r in (0, 1, 63, 127):
+                    for j in (0, 1, 511, 1023):
+                        blk = oracle.bf16_to_f32(part[r, 4 * j:4 * j + 4])
+                        nib = (int(m_gpu[r, j // 2]) >> (4 * (j % 2))) & 0xF
+                        got = oracle.bf16_to_f32(v_gpu[r, 2 * j:2 * j + 2])
+                        if m == 4:
+                            idx, val = oracle.mvue_2of4(blk, oracle.block_word(seed, (lo + r) * (cols // 4) + j))
+                        else:
+                            idx, val = [], []
+                            for half in range(2):
+                                i1, v1 = oracle.mvue_1of2(float(blk[2 * half]), float(blk[2 * half + 1]),
+                                                          oracle.block_word(seed, (lo + r) * (cols // 2) + 2 * j + half))
+                                idx.append(2 * half + i1)
+                                val.append(v1)
+                        assert nib == idx[0] | (idx[1] << 2), (lo, r, j)
+                        want = oracle.bf16_to_f32(oracle.bf16_rne(np.array(val, dtype=np.float32)))
+                        assert np.array_equal(got, want), (lo, r, j)
+            else:              # A = g^T: a K shard [lo, lo + 128) of every row of A
+                v_ref, m_ref = oracle.prune(part, n, m, axis=0, seed=seed, k_total=rows, k_offset=lo,
+                                            threads=oracle.host_threads())
+                v_gpu = values[:, lo // 2:lo // 2 + 64].contiguous().view(torch.int16).cpu().numpy().view(np.uint16)
+                m_gpu = meta[:, lo // 8:lo // 8 + 16].contiguous().cpu().numpy()
+                assert np.array_equal(v_gpu, v_ref), lo
+                assert np.array_equal(m_gpu, m_ref), lo
+        del values, meta
+    del g_dev
+    torch.cuda.empty_cache()
