@@ -203,8 +203,10 @@ MVUE_API int mvue_sparse_backward_gemm(const void* values, const void* meta, int
  * mvue_sparse_update_gemm with the same seed (up to fp32 summation order across K splits).
  * Every 128 x 256 output tile re-prunes its rows of g: the prune work grows with in / 256,
  * and the prune is bound by instruction issue, so for wide layers the separate calls are
- * faster; this entry point pays off only for in <= 256 or when memory for the packed
- * operand is not available.
+ * several times faster.  With in <= 256 (one column tile: nothing is pruned twice) it ties
+ * with mvue_prune + mvue_sparse_update_gemm and loses 10-30 % to mvue_prune_joint with
+ * systematic sampling + the product; its use is when memory for the packed operand is not
+ * available.
  * dtype must be MVUE_BF16 (else MVUE_ERR_DTYPE).  workspace: mvue_gemm_workspace_bytes(2, out,
  * in, T) bytes.  Other arguments, preconditions and errors as mvue_sparse_update_gemm. */
 MVUE_API int mvue_fused_update_gemm(const void* g, int dtype, int64_t T, int64_t out, int64_t ldg, int n,
