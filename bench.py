@@ -303,6 +303,24 @@ def run_ours(args, cfg, n, m):
         others.append(("1:2", float(np.mean([e[0].elapsed_time(e[1]) for e in evs2])), k2))
         nm[0] = (n, m)
 
+    # the step's prune timed alone (no product in between, so at the GPU's unthrottled clock), L2-cold: inputs
+    # rotated over copies of g that together exceed 2.5 x L2
+    alone_ms = None
+    if rank == 0 and world == 1 and not args.no_extra:
+        copies = max(2, int(2.5 * 126e6 / (T * out * elem)) + 1)
+        gs = [g_dev.clone() for _ in range(copies)]
+        for i in range(3):
+            binding.mvue_prune(gs[i % copies], n, m, 0, i, values=values, meta=meta, layout=TC, joint=joint[0])
+        torch.cuda.synchronize()
+        ka = max(3, min(args.steps, 100))
+        ev0.record()
+        for i in range(ka):
+            binding.mvue_prune(gs[i % copies], n, m, 0, i, values=values, meta=meta, layout=TC, joint=joint[0])
+        ev1.record()
+        torch.cuda.synchronize()
+        alone_ms = ev0.elapsed_time(ev1) / ka
+        del gs
+
     # dense cuBLAS bf16 for the same shape (context for the sparse product)
     dense_ms = None
     if rank == 0 and elem == 2:
@@ -377,6 +395,11 @@ def run_ours(args, cfg, n, m):
                                "traffic": ncu_traffic("prune_axis0_bf16_kernel/" + args.joint, args.workload)
                                if (n, m) == (2, 4) else None},
         }
+        if alone_ms is not None:
+            agbs = p_bytes / (alone_ms * 1e-3) / 1e9
+            line["prune_alone"] = {"joint": args.joint, "ms": alone_ms, "gbs": agbs,
+                                   "frac_of_hbm_peak": agbs / peaks["hbm_gbs"],
+                                   "note": "the step's prune launched back to back, L2-cold, without the product"}
         for other in others:
             ogbs = p_bytes / (other[1] * 1e-3) / 1e9
             key = {"table": "prune_other_joint", "systematic": "prune_other_joint", "1:2": "prune_1of2"}.get(
@@ -584,9 +607,13 @@ def chain_case(n, m):
     def run_sys():
         chain.backward_update(g_top, layers, n, m, base_seed=1, joint=binding.MVUE_JOINT_SYSTEMATIC)
 
+    def run_sys_overlap():
+        chain.backward_update(g_top, layers, n, m, base_seed=1, joint=binding.MVUE_JOINT_SYSTEMATIC, overlap=True)
+
     eager_ms = timed(run_table, 5)
     table_ms = timed(graphed(run_table), 10)
     sys_ms = timed(graphed(run_sys), 10) if m == 4 else None
+    overlap_ms = timed(graphed(run_sys_overlap), 10) if m == 4 else None
     dense_ms = timed(graphed(dense_chain), 10)
     n_layers = len(layers)
     flops = 2.0 * T * d * d_ff * (2 * n_layers - 1)         # update product per layer, backward for all but the bottom
@@ -596,6 +623,9 @@ def chain_case(n, m):
             "ms": table_ms, "tflops_effective": flops / (table_ms * 1e-3) / 1e12,
             "systematic_ms": sys_ms,
             "systematic_tflops_effective": None if sys_ms is None else flops / (sys_ms * 1e-3) / 1e12,
+            # the same chain with each update product on a second stream beside the next axis-1 prune
+            "systematic_two_stream_ms": overlap_ms,
+            "systematic_two_stream_tflops_effective": None if overlap_ms is None else flops / (overlap_ms * 1e-3) / 1e12,
             "dense_torch_ms": dense_ms, "dense_torch_tflops": flops / (dense_ms * 1e-3) / 1e12}
 
 

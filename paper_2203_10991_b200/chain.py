@@ -22,18 +22,40 @@ def layer_seeds(base_seed: int, layer: int) -> tuple[int, int]:
            (base_seed * 0x9E3779B97F4A7C15 + 2 * layer + 1) & (2**64 - 1)
 
 
-def backward_update(g_top: torch.Tensor, layers, n: int = 2, m: int = 4, base_seed: int = 0, joint: int | None = None):
+def backward_update(g_top: torch.Tensor, layers, n: int = 2, m: int = 4, base_seed: int = 0, joint: int | None = None,
+                    overlap: bool = False):
     """layers: list (top layer first) of dicts {"W": [out x in] bf16, "h": [T x in] bf16,
     "act_grad": [T x in] bf16 or None (None for the bottom layer: no gradient is propagated further)}.
     joint: the 2:4 law over pairs handed to mvue_prune_joint (None: mvue_prune, the App. A.2 table).
+    overlap: run each layer's update product on a second stream beside the prune that feeds its backward product.
+    The product issues on a few percent of an SM's instruction slots and the prune uses no tensor core; the update
+    product of a long token axis keeps a small register footprint, so blocks of the (shared-memory-free) prune along
+    the features fit on the same SMs.  Same calls, same seeds, same results; the streams join before each backward
+    product and before returning.
     Returns the list of dW (fp32), top layer first."""
     g = g_top
     grads = []
+    main = torch.cuda.current_stream()
+    side = torch.cuda.Stream(priority=-1) if overlap else None
     for i, L in enumerate(layers):
         s_upd, s_bwd = layer_seeds(base_seed, i)
         values, meta = binding.mvue_prune(g, n, m, 0, s_upd, layout=TC, joint=joint)
+        propagate = L.get("act_grad") is not None
+        if overlap and propagate:
+            dW = torch.empty((values.shape[0], L["h"].shape[1]), dtype=torch.float32, device=g.device)
+            ws_bytes = binding.mvue_gemm_workspace_bytes(0, dW.shape[0], dW.shape[1], g.shape[0])
+            ws = torch.empty(max(ws_bytes, 16), dtype=torch.uint8, device=g.device)
+            side.wait_stream(main)
+            with torch.cuda.stream(side):
+                binding.mvue_sparse_update_gemm(values, meta, L["h"], out=dW, workspace=ws)
+            values_b, meta_b = binding.mvue_prune(g, n, m, 1, s_bwd, layout=TC, joint=joint)
+            main.wait_stream(side)                       # (values, meta, ws stay referenced until here)
+            grads.append(dW)
+            g = binding.mvue_sparse_backward_gemm(values_b, meta_b, L["W"], act_grad=L["act_grad"],
+                                                  out_dtype=torch.bfloat16)
+            continue
         grads.append(binding.mvue_sparse_update_gemm(values, meta, L["h"]))
-        if L.get("act_grad") is not None:
+        if propagate:
             values, meta = binding.mvue_prune(g, n, m, 1, s_bwd, layout=TC, joint=joint)
             g = binding.mvue_sparse_backward_gemm(values, meta, L["W"], act_grad=L["act_grad"],
                                                   out_dtype=torch.bfloat16)

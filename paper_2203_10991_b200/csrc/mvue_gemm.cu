@@ -393,9 +393,10 @@ __device__ __forceinline__ void quad_transpose(uint32_t (&v)[64], int lane) {
 //               stores of one tile overlap the main loop of the next
 // kMode fixes the output path at compile time so that the drained tile fits the register file:
 //   0: fp32 (C, C +=, or the split-K workspace)   1: bf16   2: bf16 times p.scale   3: fp32 times p.scale
+//   4: as 0 with the small-footprint epilogue (64 registers per thread), for work items with long main loops
 // The scale factors of a row are fetched into registers under the main loop.
 template <int kMode>
-__global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(kThreads, 1)
+__global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(kMode == 4 ? 1024 : kThreads, 1)
 sparse_gemm_pair_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ CUtensorMap map_b,
                         const __grid_constant__ CUtensorMap map_e, const GemmParams p) {
     extern __shared__ uint8_t smem_raw[];
@@ -523,6 +524,69 @@ sparse_gemm_pair_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_
             const int64_t row = it.m0 + 32 * q + lane;
             const int64_t col0 = it.n0 + c_off;
             const bool row_ok = row < p.M;
+            if constexpr (kMode == 4) {
+                // fp32 output, small register footprint: 32 columns at a time from tensor memory straight to their
+                // destination, tensor memory handed back after the last store has been issued.  Next to a main loop
+                // of dozens of stages the longer hold is nothing, and at 64 registers per thread the block leaves
+                // two thirds of the SM's register file to other kernels' blocks.
+                const bool have_acc = it.n_steps > 0;
+                if (have_acc) {
+                    if (!__all_sync(0xFFFFFFFFu, mbar_wait(acc_bar, tiles_done & 1u, abort_flag))) break;
+                    tc_fence_after();
+                }
+                float* dst;
+                int64_t cols_here;                               // columns of this warp's 128 that exist
+                bool plain = false;                              // the final output (may accumulate), not a partial
+                if (it.tail_slot >= 0) {
+                    dst = p.tail_partial + (((int64_t)it.tail_slot * (2 * BM) + (int64_t)rank * BM + 32 * q + lane) * BN) + c_off;
+                    cols_here = 128;
+                } else if (p.splits > 1) {
+                    dst = p.partial + ((int64_t)it.split * p.M + row) * p.N + col0;
+                    cols_here = p.N - col0;
+                } else {
+                    dst = reinterpret_cast<float*>(p.C) + row * p.ldc + col0;
+                    cols_here = p.N - col0;
+                    plain = true;
+                }
+#pragma unroll 1
+                for (int c = 0; c < 128; c += 32) {
+                    uint32_t v[32];
+                    if (have_acc) {
+                        tmem_ld_32x32b_x32(tmem_rows + (uint32_t)c, v);
+                        tmem_ld_wait();
+                    } else {
+#pragma unroll
+                        for (int e = 0; e < 32; ++e) v[e] = 0u;
+                    }
+                    if (row_ok) {
+#pragma unroll
+                        for (int e = 0; e < 32; e += 8) {
+                            if (c + e >= cols_here) break;       // N is a multiple of 8
+                            if (plain && p.accumulate) {
+                                const float4 c0 = *reinterpret_cast<const float4*>(dst + c + e);
+                                const float4 c1 = *reinterpret_cast<const float4*>(dst + c + e + 4);
+                                v[e] = __float_as_uint(__uint_as_float(v[e]) + c0.x);
+                                v[e + 1] = __float_as_uint(__uint_as_float(v[e + 1]) + c0.y);
+                                v[e + 2] = __float_as_uint(__uint_as_float(v[e + 2]) + c0.z);
+                                v[e + 3] = __float_as_uint(__uint_as_float(v[e + 3]) + c0.w);
+                                v[e + 4] = __float_as_uint(__uint_as_float(v[e + 4]) + c1.x);
+                                v[e + 5] = __float_as_uint(__uint_as_float(v[e + 5]) + c1.y);
+                                v[e + 6] = __float_as_uint(__uint_as_float(v[e + 6]) + c1.z);
+                                v[e + 7] = __float_as_uint(__uint_as_float(v[e + 7]) + c1.w);
+                            }
+                            store8_b32(dst + c + e, &v[e]);
+                        }
+                    }
+                }
+                if (have_acc) {
+                    tc_fence_before();
+                    __syncwarp();
+                    if (lane == 0)
+                        asm volatile("mbarrier.arrive.relaxed.cluster.shared::cluster.b64 _, [%0];" ::"r"(leader_free) : "memory");
+                    ++tiles_done;
+                }
+                continue;
+            }
             // bf16 x scale keeps the row's factors in registers; fp32 x scale has no room for them beside 128
             // fp32 results and applies them after tensor memory has been handed back
             constexpr bool kScale = kMode == 2, kLateScale = kMode == 3, kToBf16 = kMode == 1 || kMode == 2;
@@ -961,11 +1025,12 @@ struct PairKernelSetup {
 const PairKernelSetup& pair_kernel_setup() {
     static const PairKernelSetup st = [] {
         PairKernelSetup r;
-        const void* kernels[4] = {reinterpret_cast<const void*>(sparse_gemm_pair_kernel<0>),
+        const void* kernels[5] = {reinterpret_cast<const void*>(sparse_gemm_pair_kernel<0>),
                                   reinterpret_cast<const void*>(sparse_gemm_pair_kernel<1>),
                                   reinterpret_cast<const void*>(sparse_gemm_pair_kernel<2>),
-                                  reinterpret_cast<const void*>(sparse_gemm_pair_kernel<3>)};
-        for (int i = 0; i < 4 && r.attr_err == cudaSuccess; ++i)
+                                  reinterpret_cast<const void*>(sparse_gemm_pair_kernel<3>),
+                                  reinterpret_cast<const void*>(sparse_gemm_pair_kernel<4>)};
+        for (int i = 0; i < 5 && r.attr_err == cudaSuccess; ++i)
             r.attr_err = cudaFuncSetAttribute(kernels[i], cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemBytes);
         cudaLaunchConfig_t cfg = {};
         cfg.gridDim = dim3(2, 1, 1);
@@ -1153,12 +1218,17 @@ int launch_sparse_gemm(const SparseGemmArgs& a, cudaStream_t stream) {
     if (n_pairs < 1) n_pairs = 1;
     dim3 grid((unsigned)(2 * n_pairs), 1u, 1u);
     const bool scaled = p.scale != nullptr && splits == 1, to_bf16 = p.c_is_bf16 && splits == 1;
+    // main loops of at least 32 stages (K = 4096) per work item: the small-footprint epilogue costs nothing there
+    const int64_t item_steps = tail.parts > 1 ? steps / tail.parts : p.k_steps_per_split;
+    const bool long_items = item_steps >= 32;
     if (scaled && to_bf16)
         sparse_gemm_pair_kernel<2><<<grid, kThreads, kSmemBytes, stream>>>(map_a, map_b, map_e, p);
     else if (scaled)
         sparse_gemm_pair_kernel<3><<<grid, kThreads, kSmemBytes, stream>>>(map_a, map_b, map_e, p);
     else if (to_bf16)
         sparse_gemm_pair_kernel<1><<<grid, kThreads, kSmemBytes, stream>>>(map_a, map_b, map_e, p);
+    else if (long_items)
+        sparse_gemm_pair_kernel<4><<<grid, kThreads, kSmemBytes, stream>>>(map_a, map_b, map_e, p);
     else
         sparse_gemm_pair_kernel<0><<<grid, kThreads, kSmemBytes, stream>>>(map_a, map_b, map_e, p);
     cudaError_t e = cudaGetLastError();

@@ -45,3 +45,22 @@ def test_three_layer_chain_matches_oracle_chain():
             v, mt = oracle.prune(g, 2, 4, axis=1, seed=s_bwd, threads=th)
             dh = oracle.gemm(oracle.unpack(v, mt), L["W"], L["act_grad"], threads=th)
             g = workloads.to_bf16_bits(dh.astype(np.float32))
+
+
+def test_overlapped_chain_gives_the_same_bits():
+    # the two-stream schedule (update product beside the prune that feeds the backward product) runs the same calls
+    # with the same seeds: every dW must be bit-identical to the one-stream chain's
+    T, dims = 1024, [256, 512, 256, 384]
+    layers = []
+    for i in range(3):
+        out_f, in_f = dims[3 - i], dims[2 - i]
+        layers.append({"W": to_dev(workloads.normal_bf16((out_f, in_f), seed=40 + i, std=in_f ** -0.5)),
+                       "h": to_dev(workloads.normal_bf16((T, in_f), seed=50 + i)),
+                       "act_grad": to_dev(workloads.normal_bf16((T, in_f), seed=60 + i)) if i < 2 else None})
+    g_top = to_dev(workloads.gradient((T, dims[3]), "student_t", seed=9, dtype="bf16"))
+    for joint in (None, 1):
+        a = chain.backward_update(g_top, layers, base_seed=5, joint=joint)
+        b = chain.backward_update(g_top, layers, base_seed=5, joint=joint, overlap=True)
+        torch.cuda.synchronize()
+        for x, y in zip(a, b):
+            assert torch.equal(x, y)
