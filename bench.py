@@ -458,6 +458,14 @@ def tensor_bound_case(n, m, peaks, joint):
     fused_ms = timed(lambda: binding.mvue_fused_update_gemm(g, h, n, m, 1, out=dW), 3)
     gT = g.t()
     dense_ms = timed(lambda: torch.matmul(gT, h), 30)
+    # what the sparse tensor cores retire when nothing is loaded (zeros in shared memory, so no power throttling
+    # either): the ceiling of any tiling, above what real operands can reach under the power cap
+    probe_status = torch.zeros(1, dtype=torch.int32, device="cuda")
+    probe_iters = 4096
+    _, probe_flops = binding.mvue_probe_sparse_mma(probe_iters, probe_status)
+    probe_ms = min(timed(lambda: binding.mvue_probe_sparse_mma(probe_iters, probe_status), 1) for _ in range(5))
+    assert int(probe_status.item()) == 0
+    issue_ceiling = probe_flops / (probe_ms * 1e-3) / 1e12
     flops = 2.0 * out * inp * T
     tf = flops / (gemm_ms * 1e-3) / 1e12
     pgbs = prune_bytes(T, out, 2) / (prune_ms * 1e-3) / 1e9
@@ -470,6 +478,8 @@ def tensor_bound_case(n, m, peaks, joint):
             "gemm_ms": gemm_ms, "gemm_tflops_effective": tf,
             "gemm_frac_of_sparse_peak_burst": tf / (2 * peaks["bf16_tflops"]),
             "gemm_frac_of_sparse_peak_sustained": tf / (2 * peaks["bf16_tflops_sustained"]),
+            "sparse_mma_issue_ceiling_tflops": issue_ceiling,
+            "gemm_frac_of_issue_ceiling": tf / issue_ceiling,
             "dense_cublas_ms": dense_ms, "dense_cublas_tflops": flops / (dense_ms * 1e-3) / 1e12,
             # three-way comparison: separate prune + sparse product vs the fused kernel vs dense cuBLAS
             "separate_ms": prune_ms + gemm_ms, "fused_ms": fused_ms,

@@ -247,6 +247,15 @@ MVUE_API int mvue_sparse_update_gemm_noalloc(const void* values, const void* met
                                              int64_t ldh, void* dW, int dW_dtype, int64_t lddW,
                                              int accumulate, int* dev_status, void* stream);
 
+/* Measurement aid (the paper has no counterpart): the rate at which this GPU retires the sparse tensor-core
+ * instruction of the products above when nothing has to be loaded.  One launch: every resident pair of thread blocks
+ * issues iters x 4 tcgen05.mma.sp (M = 256, N = 256, K = 32, bf16, fp32 accumulate) back to back on one
+ * shared-memory stage of zeros.  Time the launch with events on `stream`; *flops (HOST pointer, may be NULL) receives
+ * the dense-equivalent floating-point operations of the launch (2 M N K per instruction, as the products are
+ * counted), *pairs (HOST, may be NULL) the number of pairs.  1 <= iters <= 2^20, else MVUE_ERR_SHAPE.  dev_status as
+ * for the products (the one wait of the kernel is bounded).  Reads and writes no caller memory. */
+MVUE_API int mvue_probe_sparse_mma(int iters, int* pairs, double* flops, int* dev_status, void* stream);
+
 MVUE_API const char* mvue_status_string(int status);
 /* Text of the last CUDA error seen by the calling thread ("" if none). */
 MVUE_API const char* mvue_last_cuda_error(void);

@@ -21,7 +21,8 @@ MVUE_JOINT_TABLE, MVUE_JOINT_SYSTEMATIC, MVUE_JOINT_APPROX = 0, 1, 2
 
 EXPORTS = ("mvue_version", "mvue_status_string", "mvue_last_cuda_error", "mvue_packed_sizes",
            "mvue_prune", "mvue_prune_joint", "mvue_unpack", "mvue_sparse_update_gemm", "mvue_sparse_backward_gemm",
-           "mvue_gemm_workspace_bytes", "mvue_sparse_update_gemm_noalloc", "mvue_fused_update_gemm")
+           "mvue_gemm_workspace_bytes", "mvue_sparse_update_gemm_noalloc", "mvue_fused_update_gemm",
+           "mvue_probe_sparse_mma")
 
 
 class MvueError(RuntimeError):
@@ -59,6 +60,7 @@ def lib() -> ctypes.CDLL:
         L.mvue_fused_update_gemm.argtypes = [vp, ci, i64, i64, i64, ci, ci, u64, vp, i64, i64, vp, ci, i64, ci, vp,
                                              ctypes.c_size_t, vp, vp]
         L.mvue_sparse_update_gemm_noalloc.argtypes = [vp, vp, ci, i64, i64, vp, i64, i64, vp, ci, i64, ci, vp, vp]
+        L.mvue_probe_sparse_mma.argtypes = [ci, ctypes.POINTER(ctypes.c_int), ctypes.POINTER(ctypes.c_double), vp, vp]
         _lib = L
     return _lib
 
@@ -212,3 +214,13 @@ def mvue_fused_update_gemm(g: torch.Tensor, h: torch.Tensor, n: int, m: int, see
                                         None if dev_status is None else dev_status.data_ptr(), _stream_ptr()),
            "mvue_fused_update_gemm")
     return out
+
+
+def mvue_probe_sparse_mma(iters: int, dev_status: torch.Tensor | None = None):
+    """One launch of the sparse tensor-core issue-rate probe on the current stream.
+    Returns (pairs, dense-equivalent flops of the launch); time it with CUDA events."""
+    pairs, flops = ctypes.c_int(), ctypes.c_double()
+    _check(lib().mvue_probe_sparse_mma(iters, ctypes.byref(pairs), ctypes.byref(flops),
+                                       None if dev_status is None else dev_status.data_ptr(), _stream_ptr()),
+           "mvue_probe_sparse_mma")
+    return pairs.value, flops.value

@@ -212,6 +212,18 @@ int mvue_fused_update_gemm(const void* g, int dtype, int64_t T, int64_t out, int
     return launch_fused_update(f, reinterpret_cast<cudaStream_t>(stream));
 }
 
+int mvue_probe_sparse_mma(int iters, int* pairs, double* flops, int* dev_status, void* stream) {
+    if (iters <= 0 || iters > (1 << 20)) return MVUE_ERR_SHAPE;
+    DeviceInfo dev;
+    if (int s = current_device_info(&dev)) return s;
+    int n_pairs = 0;
+    if (int s = launch_sparse_mma_probe(iters, dev.sm_count, &n_pairs, dev_status, reinterpret_cast<cudaStream_t>(stream)))
+        return s;
+    if (pairs) *pairs = n_pairs;
+    if (flops) *flops = (double)n_pairs * (double)iters * 4.0 * 2.0 * 256.0 * 256.0 * 32.0;
+    return MVUE_OK;
+}
+
 int mvue_sparse_update_gemm_noalloc(const void* values, const void* meta, int layout, int64_t out, int64_t T,
                                     const void* h, int64_t in, int64_t ldh, void* dW, int dW_dtype,
                                     int64_t lddW, int accumulate, int* dev_status, void* stream) {

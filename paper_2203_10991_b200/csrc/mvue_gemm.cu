@@ -995,6 +995,71 @@ tail_reduce_kernel(const float* __restrict__ partial, int rem, int parts, int64_
     *reinterpret_cast<float4*>(dst) = acc;
 }
 
+// =============================================================================
+// Issue-rate probe: what the sparse tensor cores deliver when nothing has to be loaded.  Every pair fills ONE
+// pipeline stage with zeros and a valid metadata pattern and its leader issues `iters` x 4 of the very
+// tcgen05.mma.sp.cta_group::2 instructions of the product kernel (M = 256, N = 256, K = 32 each) on that stage, back to
+// back, one commit at the end.  The time of this launch is the ceiling any tiling of the product can approach.
+// =============================================================================
+__global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(128, 1)
+sparse_mma_issue_probe_kernel(int iters, int* dev_status) {
+    extern __shared__ uint8_t smem_raw[];
+    const uint32_t smem_base = (smem_u32(smem_raw) + 1023u) & ~1023u;
+    uint8_t* smem_gen = smem_raw + (smem_base - smem_u32(smem_raw));
+    const uint32_t done_bar = smem_base + kStageBytes;
+    uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(smem_gen + kStageBytes + 8);
+    volatile int* abort_flag = reinterpret_cast<volatile int*>(tmem_slot + 1);
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const uint32_t rank = cluster_ctarank();
+
+    for (int i = threadIdx.x; i < kStageBytes / 16; i += blockDim.x) {       // A and B zero, metadata "positions 0 and 1"
+        const uint32_t w = i * 16 >= kABytes + kBBytes ? 0x44444444u : 0u;
+        reinterpret_cast<uint4*>(smem_gen)[i] = make_uint4(w, w, w, w);
+    }
+    asm volatile("fence.proxy.async.shared::cta;" ::: "memory");             // the tensor cores read what the lanes wrote
+    if (threadIdx.x == 0) {
+        mbar_init(done_bar, 1);
+        *abort_flag = 0;
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    }
+    if (warp == 2) {
+        asm volatile("tcgen05.alloc.cta_group::2.sync.aligned.shared::cta.b32 [%0], %1;"
+                     ::"r"(smem_u32(tmem_slot)), "r"(kTmemCols) : "memory");
+        asm volatile("tcgen05.relinquish_alloc_permit.cta_group::2.sync.aligned;" ::: "memory");
+    }
+    tc_fence_before();
+    __syncthreads();
+    cluster_sync();
+    tc_fence_after();
+    const uint32_t tmem_base = *tmem_slot;
+
+    if (rank == 0 && warp == 1 && lane == 0) {
+        const uint32_t a_addr = smem_base, b_addr = a_addr + kABytes, e_addr = b_addr + kBBytes;
+        const uint32_t tmem_e = tmem_base + kTmemECol;
+        tc_copy_128x128b_pair(tmem_e, make_smem_desc(e_addr, 16, 128, kSwizzleNone));
+        for (int i = 0; i < iters; ++i) {
+#pragma unroll
+            for (int kb = 0; kb < BK / 32; ++kb) {
+                const uint64_t a_desc = make_smem_desc(a_addr + kb * 32, 16, 1024, kSwizzle128B);
+                const uint64_t b_desc = make_smem_desc(b_addr + kb * 4096, kBBoxBytes, 1024, kSwizzle128B);
+                tc_mma_sp_bf16_pair(tmem_base, a_desc, b_desc, tmem_e + (uint32_t)(kb & ~1), kInstrDesc2 | (uint32_t)(kb & 1),
+                                    (i > 0 || kb > 0) ? 1u : 0u);
+            }
+        }
+        tc_commit_pair(done_bar);                                            // both blocks' barriers, when the MMAs retire
+    }
+    const bool ok = mbar_wait(done_bar, 0u, abort_flag);                     // bounded
+    tc_fence_after();
+    __syncthreads();
+    if (!ok && threadIdx.x == 0 && dev_status) *dev_status = MVUE_ERR_DEVICE_TIMEOUT;
+    tc_fence_before();
+    cluster_sync();
+    if (warp == 2) {
+        tc_fence_after();
+        asm volatile("tcgen05.dealloc.cta_group::2.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"(kTmemCols) : "memory");
+    }
+}
+
 // ---- host side ----------------------------------------------------------------
 }  // namespace
 
@@ -1171,6 +1236,23 @@ int launch_fused_update(const FusedArgs& f, cudaStream_t stream) {
         e = cudaGetLastError();
     }
     if (e != cudaSuccess) { set_cuda_error(e, "fused update launch"); return MVUE_ERR_CUDA; }
+    return MVUE_OK;
+}
+
+int launch_sparse_mma_probe(int iters, int sm_count, int* pairs_out, int* dev_status, cudaStream_t stream) {
+    static std::once_flag once;
+    static cudaError_t attr_err = cudaSuccess;
+    std::call_once(once, [] {
+        attr_err = cudaFuncSetAttribute(sparse_mma_issue_probe_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                        kSmemBytes);
+    });
+    if (attr_err != cudaSuccess) { set_cuda_error(attr_err, "cudaFuncSetAttribute"); return MVUE_ERR_CUDA; }
+    const int pairs = resident_pairs(sm_count);
+    if (pairs_out) *pairs_out = pairs;
+    // the product kernel's shared-memory request, so that one block lands on each SM as it does there
+    sparse_mma_issue_probe_kernel<<<dim3((unsigned)(2 * pairs)), 128, kSmemBytes, stream>>>(iters, dev_status);
+    const cudaError_t e = cudaGetLastError();
+    if (e != cudaSuccess) { set_cuda_error(e, "sparse MMA probe launch"); return MVUE_ERR_CUDA; }
     return MVUE_OK;
 }
 

@@ -43,6 +43,7 @@ struct SparseGemmArgs {
     int sm_count;
 };
 int launch_sparse_gemm(const SparseGemmArgs& a, cudaStream_t stream);     // returns an mvue_status
+int launch_sparse_mma_probe(int iters, int sm_count, int* pairs_out, int* dev_status, cudaStream_t stream);   // mvue_status
 int gemm_split_count(int64_t M, int64_t N, int64_t K, int sm_count);
 size_t gemm_workspace_bytes(int64_t M, int64_t N, int64_t K, int sm_count);            // what lets every path run
 size_t gemm_required_workspace_bytes(int64_t M, int64_t N, int64_t K, int sm_count);   // the split along K alone
