@@ -303,8 +303,8 @@ def run_ours(args, cfg, n, m):
         others.append(("1:2", float(np.mean([e[0].elapsed_time(e[1]) for e in evs2])), k2))
         nm[0] = (n, m)
 
-    # the step's prune timed alone (no product in between, so at the GPU's unthrottled clock), L2-cold: inputs
-    # rotated over copies of g that together exceed 2.5 x L2
+    # the step's prune timed alone (no product in between), L2-cold: inputs rotated over copies of g that together
+    # exceed 2.5 x L2
     alone_ms = None
     if rank == 0 and world == 1 and not args.no_extra:
         copies = max(2, int(2.5 * 126e6 / (T * out * elem)) + 1)
