@@ -71,6 +71,11 @@ def lib() -> ctypes.CDLL:
         L.oracle_sweep_approx24.argtypes = [ctypes.POINTER(ctypes.c_float), ctypes.POINTER(ctypes.c_uint64),
                                             ctypes.POINTER(ctypes.c_uint64), ctypes.POINTER(ctypes.c_float)]
         L.oracle_sweep_approx24.restype = None
+        L.oracle_mvue_1of4.argtypes = [ctypes.POINTER(ctypes.c_float), ctypes.c_uint32, ctypes.POINTER(ctypes.c_float)]
+        L.oracle_mvue_1of4.restype = ctypes.c_int
+        L.oracle_sweep_1of4.argtypes = [ctypes.POINTER(ctypes.c_float), ctypes.POINTER(ctypes.c_uint64),
+                                        ctypes.POINTER(ctypes.c_double), ctypes.POINTER(ctypes.c_double)]
+        L.oracle_sweep_1of4.restype = None
         L.oracle_prune.argtypes = [ctypes.c_void_p, ctypes.c_int, ctypes.c_int64, ctypes.c_int64,
                                    ctypes.c_int64, ctypes.c_int, ctypes.c_int, ctypes.c_int,
                                    ctypes.c_uint64, ctypes.c_int64, ctypes.c_int64,
@@ -163,6 +168,25 @@ def block_word_pair(seed: int, q: int):
     out = (ctypes.c_uint32 * 2)()
     lib().oracle_block_word_pair(seed & (2**64 - 1), q, out)
     return int(out[0]), int(out[1])
+
+
+def mvue_1of4(a, word: int):
+    """MVUE 1:4 on one block: (surviving position, its new value)."""
+    arr = (ctypes.c_float * 4)(*[float(x) for x in a])
+    kept = ctypes.c_float()
+    i = lib().oracle_mvue_1of4(arr, word & 0xFFFFFFFF, ctypes.byref(kept))
+    return int(i), float(kept.value)
+
+
+def sweep_1of4(a):
+    """Frequencies of the four outcomes, mean of theta(a) and block variance over all 2^24 eps."""
+    arr = (ctypes.c_float * 4)(*[float(x) for x in a])
+    counts = (ctypes.c_uint64 * 4)()
+    sums = (ctypes.c_double * 4)()
+    sq = ctypes.c_double()
+    lib().oracle_sweep_1of4(arr, counts, sums, ctypes.byref(sq))
+    n = float(1 << 24)
+    return (np.array(list(counts), dtype=np.float64) / n, np.array(list(sums)) / n, sq.value / n)
 
 
 def packed_shapes(rows: int, cols: int, axis: int):

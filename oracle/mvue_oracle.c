@@ -378,6 +378,34 @@ void oracle_mvue_2of4_approx(const float a[4], uint32_t word1, uint32_t word2, i
 }
 
 /* ------------------------------------------------------------------------
+ * MVUE 1:4 (appendix "Additional sparsity results": like MVUE 1:2 for a block of
+ * four): one element survives, element i with probability |a_i| / S,
+ * S = |a_1|+|a_2|+|a_3|+|a_4|, and becomes sign(a_i) S.  This is Sec. 4.1's
+ * argument for a block of M: an unbiased estimator that keeps one element has
+ * theta_i = a_i / p_i, its variance sum_i a_i^2 / p_i - a_i^2 is least, under
+ * sum_i p_i = 1, at p_i proportional to |a_i|, where it equals S^2 - sum a_i^2.
+ * Draw: the threshold walk of App. "Pruning Overhead" Part 1 in the block's
+ * own order over c_1 = m_1, c_2 = c_1 + m_2, c_3 = c_2 + m_3, S = c_3 + m_4:
+ *     t = n (S 2^-24),   i = #{k in 1,2,3 : c_k <= t},
+ * n the top 24 bits of the block's random word (one word per block, as for 2:4).
+ * Zero rule: an element of magnitude zero owns an empty interval; an all-zero
+ * block keeps its last element (a signed zero).
+ * Returns the surviving position (0..3); *kept receives the new value.
+ * ---------------------------------------------------------------------- */
+int oracle_mvue_1of4(const float a[4], uint32_t word, float *kept)
+{
+    const float m0 = fabsf(a[0]), m1 = fabsf(a[1]), m2 = fabsf(a[2]), m3 = fabsf(a[3]);
+    const float c1 = m0;
+    const float c2 = c1 + m1;
+    const float c3 = c2 + m2;
+    const float S  = c3 + m3;
+    const float t  = (float)(word >> 8) * (S * 5.9604644775390625e-08f);
+    const int i = (c1 <= t) + (c2 <= t) + (c3 <= t);
+    *kept = copysignf(S, a[i]);
+    return i;
+}
+
+/* ------------------------------------------------------------------------
  * Tensor-wide prune and pack.
  *
  * g is a row-major [rows x cols] matrix with leading dimension ld, fp32
@@ -396,7 +424,9 @@ void oracle_mvue_2of4_approx(const float a[4], uint32_t word1, uint32_t word2, i
  *   meta  [Mrows x K/8]  bytes; each nibble = idx0 | idx1 << 2 for one group
  *                        of four, low nibble = even group.
  * A 1:2 result is written as a valid 2:4 pattern: the pair (4j, 4j+1) gives
- * idx0 in {0,1}, the pair (4j+2, 4j+3) gives idx1 in {2,3}.
+ * idx0 in {0,1}, the pair (4j+2, 4j+3) gives idx1 in {2,3}.  A 1:4 result
+ * (n = 1, m = 4) is written as the survivor beside a +0 partner: positions
+ * (i, 3) for i < 3, (2, 3) for i = 3.
  * joint selects the 2:4 estimator: 0 = the pair table of App. A.2,
  * 1 = systematic sampling, 2 = approx-MVUE of Sec. 4.4 (above; two random words
  * per block); 1:2 has a single law and ignores it.
@@ -414,7 +444,7 @@ int oracle_prune(const void *g, int is_bf16, int64_t rows, int64_t cols, int64_t
 {
     const int64_t Mrows = axis == 1 ? rows : cols;
     const int64_t K     = axis == 1 ? cols : rows;
-    if (!((n == 1 && m == 2) || (n == 2 && m == 4))) return -1;
+    if (!((n == 1 && m == 2) || (n == 2 && m == 4) || (n == 1 && m == 4))) return -1;
     if (K % 8 != 0 || k_total % 8 != 0 || k_offset % 8 != 0 || k_offset + K > k_total) return -1;
     if (joint < 0 || joint > 2) return -1;
     (void)threads;
@@ -428,7 +458,14 @@ int oracle_prune(const void *g, int is_bf16, int64_t rows, int64_t cols, int64_t
                 a[e] = load_elem(g, is_bf16, off);
             }
             int idx[2]; float val[2];
-            if (m == 4) {
+            if (m == 4 && n == 1) {
+                /* one survivor, stored in the 2:4 container beside a +0: positions (i, 3), or (2, 3) when i = 3 */
+                uint64_t q = (uint64_t)r * (uint64_t)(k_total / 4) + (uint64_t)(k_offset / 4 + j);
+                float kept;
+                int i = oracle_mvue_1of4(a, oracle_block_word(seed, q), &kept);
+                if (i < 3) { idx[0] = i; idx[1] = 3; val[0] = kept; val[1] = 0.0f; }
+                else       { idx[0] = 2; idx[1] = 3; val[0] = 0.0f; val[1] = kept; }
+            } else if (m == 4) {
                 uint64_t q = (uint64_t)r * (uint64_t)(k_total / 4) + (uint64_t)(k_offset / 4 + j);
                 if (joint == 0)      oracle_mvue_2of4(a, oracle_block_word(seed, q), idx, val);
                 else if (joint == 1) oracle_mvue_2of4_systematic(a, oracle_block_word(seed, q), idx, val);
@@ -575,6 +612,22 @@ void oracle_sweep_approx24(const float a[4], uint64_t first[4], uint64_t second[
             oracle_mvue_2of4_approx_ordered(a, rep[i], n << 8, &i2, &j, &vi, &vj);
             second[i][j] += 1;
             val[i2] = vi; val[j] = vj;
+        }
+    }
+}
+
+void oracle_sweep_1of4(const float a[4], uint64_t counts[4], double sum_val[4], double *sum_sq)
+{
+    for (int i = 0; i < 4; ++i) { counts[i] = 0; sum_val[i] = 0.0; }
+    *sum_sq = 0.0;
+    for (uint32_t n = 0; n < (1u << 24); ++n) {
+        float kept;
+        int i = oracle_mvue_1of4(a, n << 8, &kept);
+        counts[i] += 1;
+        sum_val[i] += kept;
+        for (int k = 0; k < 4; ++k) {
+            double d = (k == i ? (double)kept : 0.0) - (double)a[k];
+            *sum_sq += d * d;
         }
     }
 }

@@ -32,6 +32,22 @@ def var12_opt(a1: float, a2: float) -> float:
     return 2.0 * abs(a1) * abs(a2)
 
 
+# ---------------------------------------------------------------- 1:M -------
+def var1m_opt(a) -> float:
+    """Sec. 4.1's argument for a block of M with one survivor: theta_i = a_i / p_i w.p. p_i, sum p_i = 1; the
+    variance sum a_i^2 / p_i - a_i^2 is least at p_i = |a_i| / S, where it is S^2 - sum a_i^2."""
+    m = np.abs(np.asarray(a, dtype=np.float64))
+    return float(m.sum() ** 2 - np.sum(m ** 2))
+
+
+def var1m_of_p(a, p) -> float:
+    """Variance of the keep-one unbiased estimator with survival probabilities p (p_i > 0 wherever a_i != 0)."""
+    m = np.abs(np.asarray(a, dtype=np.float64))
+    p = np.asarray(p, dtype=np.float64)
+    nz = m > 0
+    return float(np.sum(m[nz] ** 2 / p[nz] - m[nz] ** 2))
+
+
 # ---------------------------------------------------------------- 2:4 -------
 def block_variance(a, p) -> float:
     """Sec. 4.2: Var_B = sum_i a_i^2 / p_i - a_i^2 for theta_i = a_i / p_i w.p. p_i."""
