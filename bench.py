@@ -301,6 +301,16 @@ def run_ours(args, cfg, n, m):
             step(i, evs2[i])
         torch.cuda.synchronize()
         others.append(("1:2", float(np.mean([e[0].elapsed_time(e[1]) for e in evs2])), k2))
+        # and MVUE 1:4 (one survivor beside a zero in the 2:4 container)
+        nm[0] = (1, 4)
+        for i in range(3):
+            step(i)
+        evs2 = [[torch.cuda.Event(enable_timing=True) for _ in range(3)] for _ in range(k2)]
+        torch.cuda.synchronize()
+        for i in range(k2):
+            step(i, evs2[i])
+        torch.cuda.synchronize()
+        others.append(("1:4", float(np.mean([e[0].elapsed_time(e[1]) for e in evs2])), k2))
         nm[0] = (n, m)
 
     # the step's prune timed alone (no product in between), L2-cold: inputs rotated over copies of g that together
@@ -402,7 +412,7 @@ def run_ours(args, cfg, n, m):
                                    "note": "the step's prune launched back to back, L2-cold, without the product"}
         for other in others:
             ogbs = p_bytes / (other[1] * 1e-3) / 1e9
-            key = {"table": "prune_other_joint", "systematic": "prune_other_joint", "1:2": "prune_1of2"}.get(
+            key = {"table": "prune_other_joint", "systematic": "prune_other_joint", "1:2": "prune_1of2", "1:4": "prune_1of4"}.get(
                 other[0], "prune_" + other[0])
             line[key] = {"joint": other[0], "ms": other[1], "gbs": ogbs,
                          "frac_of_hbm_peak": ogbs / peaks["hbm_gbs"], "steps": other[2]}

@@ -40,7 +40,7 @@ extern "C" {
 typedef enum {
     MVUE_OK = 0,
     MVUE_ERR_NULL = -1,           /* a required pointer is NULL */
-    MVUE_ERR_NM = -2,             /* only (N,M) = (1,2) and (2,4) exist */
+    MVUE_ERR_NM = -2,             /* only (N,M) = (1,2), (2,4) and (1,4) exist (the fused product: the first two) */
     MVUE_ERR_SHAPE = -3,          /* non-positive / non-multiple extents, ld < cols, bad axis or K shard */
     MVUE_ERR_ALIGN = -4,          /* base pointer or leading dimension not 16-byte aligned */
     MVUE_ERR_DTYPE = -5,
@@ -117,6 +117,13 @@ MVUE_API int mvue_packed_sizes(int64_t rows, int64_t cols, int n, int m, int axi
  *          the joint law over pairs of App. A.2 (three cases on the sorted
  *          magnitudes), drawn by walking the cumulative pair table in the order
  *          13, 14, 23, 24, 34.
+ *   (1,4): the paper's "MVUE 1:4" (appendix "Additional sparsity results": like MVUE 1:2 for a
+ *          block of four; Sec. 4.1's argument with one survivor of M): element i survives with
+ *          probability |a_i| / S, S the sum of the block's magnitudes, and becomes sign(a_i) S;
+ *          running sums in the block's own order, i = #{c_k <= eps S}.  One random word per
+ *          block, numbered as for (2,4).  The survivor is stored in the 2:4 container beside a
+ *          +0 partner -- positions (i, 3), or (2, 3) when i = 3 -- so the products below consume
+ *          it unchanged (at the 2:4 rate: no tensor core runs 1:4).
  * The draw is the threshold test eps < p of App. "Pruning Overhead" (Part 1)
  * with eps = (w >> 8) * 2^-24, w the 32-bit word of block number q:
  *   w = Philox4x32-10(counter = (lo32(q>>2), hi32(q>>2), 0, 0),

@@ -42,7 +42,7 @@ int current_device_info(DeviceInfo* info) {
 static bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
 
 static int check_nm(int n, int m) {
-    return ((n == 1 && m == 2) || (n == 2 && m == 4)) ? MVUE_OK : MVUE_ERR_NM;
+    return ((n == 1 && m == 2) || (n == 2 && m == 4) || (n == 1 && m == 4)) ? MVUE_OK : MVUE_ERR_NM;
 }
 
 static int run_gemm(const void* values, const void* meta, int layout, int64_t M, int64_t N, int64_t K,
@@ -139,7 +139,7 @@ int mvue_prune_joint(const void* g, int dtype, int64_t rows, int64_t cols, int64
     DeviceInfo dev;
     if (int s = current_device_info(&dev)) return s;
     PruneArgs a{g, dtype == MVUE_BF16, rows, cols, ld, m, axis, seed, k_total, k_offset, values, meta, dev.sm_count,
-                layout == MVUE_LAYOUT_TC, joint};
+                layout == MVUE_LAYOUT_TC, (n == 1 && m == 4) ? 3 : joint};     // one survivor of four has a single law
     cudaError_t e = launch_prune(a, reinterpret_cast<cudaStream_t>(stream));
     if (e != cudaSuccess) { set_cuda_error(e, "mvue_prune launch"); return MVUE_ERR_CUDA; }
     return MVUE_OK;
@@ -192,6 +192,7 @@ int mvue_fused_update_gemm(const void* g, int dtype, int64_t T, int64_t out, int
                            int* dev_status, void* stream) {
     if (!g || !h || !dW) return MVUE_ERR_NULL;
     if (int s = check_nm(n, m)) return s;
+    if (n == 1 && m == 4) return MVUE_ERR_NM;                      // the fused path prunes to 1:2 and 2:4 only
     if (dtype != MVUE_BF16) return MVUE_ERR_DTYPE;                 // the fused path takes bf16 gradients only
     if (dW_dtype != MVUE_F32 && dW_dtype != MVUE_BF16) return MVUE_ERR_DTYPE;
     if (accumulate && dW_dtype != MVUE_F32) return MVUE_ERR_DTYPE;

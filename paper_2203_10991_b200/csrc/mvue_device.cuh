@@ -383,16 +383,46 @@ __device__ __forceinline__ void mvue_2of4_approx_bf16(uint32_t x01, uint32_t x23
     mvue_2of4_approx_f32(x01 << 16, x01 & 0xFFFF0000u, x23 << 16, x23 & 0xFFFF0000u, word1, word2, out, nibble);
 }
 
+// ===========================================================================
+// MVUE 1:4 (the paper's "MVUE 1:4 is similar to MVUE 1:2, but for a bigger block"): element i of the block
+// survives with probability |a_i| / S, S the sum of the four magnitudes, and becomes sign(a_i) S.
+//   c_1 = m_0, c_2 = c_1 + m_1, c_3 = c_2 + m_2, S = c_3 + m_3;  t = n (S 2^-24);  i = #{c_k <= t}.
+// The survivor is stored in the 2:4 container beside a +0: positions (i, 3), or (2, 3) when i = 3.
+// ===========================================================================
+__device__ __forceinline__ void mvue_1of4_f32(uint32_t b0, uint32_t b1, uint32_t b2, uint32_t b3, uint32_t word,
+                                              uint32_t* out, uint32_t* nibble) {
+    const float m0 = fabsf(__uint_as_float(b0)), m1 = fabsf(__uint_as_float(b1));
+    const float m2 = fabsf(__uint_as_float(b2)), m3 = fabsf(__uint_as_float(b3));
+    const float c2 = __fadd_rn(m0, m1), c3 = __fadd_rn(c2, m2), S = __fadd_rn(c3, m3);
+    const float t = __fmul_rn(top24(word), __fmul_rn(S, 5.9604644775390625e-08f));
+    const uint32_t i = (m0 <= t ? 1u : 0u) + (c2 <= t ? 1u : 0u) + (c3 <= t ? 1u : 0u);
+    const uint32_t bi = i < 2u ? (i == 0u ? b0 : b1) : (i == 2u ? b2 : b3);
+    const float v = __uint_as_float(__float_as_uint(S) | (bi & 0x80000000u));
+    const uint32_t h = pack_bf16x2(v, 0.0f);                 // survivor in the low half, +0 in the high half
+    *out = i < 3u ? h : h << 16;
+    *nibble = i < 3u ? (i | 12u) : 14u;
+}
+
 // One work unit of bf16 input: raw[8] = 16 elements along K, two per word.
 // kJoint selects the 2:4 estimator (0: App. A.2 table, 1: systematic sampling, 2: approx-MVUE of Sec. 4.4,
-// which takes two words per block: one generator call per two blocks); 1:2 has one law.
+// which takes two words per block: one generator call per two blocks) or, with 3, MVUE 1:4; 1:2 has one law.
 template <int M, int kJoint = 0>
 __device__ __forceinline__ void prune_unit_bf16(const uint32_t (&raw)[8], uint64_t unit_index,
                                                 const RoundKeys& rk, uint4* out_values,
                                                 uint32_t* out_meta) {
     uint32_t v[4];                                   // 8 survivors, two bf16 per word
     uint32_t meta = 0;
-    if (M == 4 && kJoint == 2) {
+    if (M == 4 && kJoint == 3) {                      // MVUE 1:4: one word per block, as for 2:4
+        const uint4 w = philox4x32_10(unit_index, rk);
+        const uint32_t words[4] = {w.x, w.y, w.z, w.w};
+#pragma unroll
+        for (int j = 0; j < 4; ++j) {
+            uint32_t nib;
+            mvue_1of4_f32(raw[2 * j] << 16, raw[2 * j] & 0xFFFF0000u, raw[2 * j + 1] << 16, raw[2 * j + 1] & 0xFFFF0000u,
+                          words[j], &v[j], &nib);
+            meta += nib << (4 * j);
+        }
+    } else if (M == 4 && kJoint == 2) {
         const uint4 wa = philox4x32_10(2 * unit_index, rk);
         const uint4 wb = philox4x32_10(2 * unit_index + 1, rk);
         const uint32_t words[8] = {wa.x, wa.y, wa.z, wa.w, wb.x, wb.y, wb.z, wb.w};
@@ -436,7 +466,18 @@ __device__ __forceinline__ void prune_unit_bf16_rows(const uint32_t (&w)[16], ui
                                                      const RoundKeys& rk, uint4* out_values, uint32_t* out_meta) {
     uint32_t v[4];
     uint32_t meta = 0;
-    if (M == 4 && kJoint == 2) {
+    if (M == 4 && kJoint == 3) {
+        const uint4 r = philox4x32_10(unit_index, rk);
+        const uint32_t words[4] = {r.x, r.y, r.z, r.w};
+#pragma unroll
+        for (int j = 0; j < 4; ++j) {
+            uint32_t nib;
+            auto widen = [](uint32_t x) { return kHigh ? (x & 0xFFFF0000u) : (x << 16); };
+            mvue_1of4_f32(widen(w[4 * j]), widen(w[4 * j + 1]), widen(w[4 * j + 2]), widen(w[4 * j + 3]), words[j],
+                          &v[j], &nib);
+            meta += nib << (4 * j);
+        }
+    } else if (M == 4 && kJoint == 2) {
         const uint4 ra = philox4x32_10(2 * unit_index, rk);
         const uint4 rb = philox4x32_10(2 * unit_index + 1, rk);
         const uint32_t words[8] = {ra.x, ra.y, ra.z, ra.w, rb.x, rb.y, rb.z, rb.w};

@@ -11,7 +11,7 @@ struct PruneArgs {
     const void* g;
     bool is_bf16;
     int64_t rows, cols, ld;
-    int m;               // 2 or 4 (n is implied: 1 or 2)
+    int m;               // 2 or 4 (n is implied: 1 or 2; one survivor of four is joint = 3)
     int axis;            // 0 or 1
     uint64_t seed;
     int64_t k_total, k_offset;
@@ -19,7 +19,7 @@ struct PruneArgs {
     void* meta;
     int sm_count;
     bool tc_layout;      // metadata in tensor-core order instead of canonical rows
-    int joint;           // 2:4 estimator: 0 = App. A.2 table, 1 = systematic sampling, 2 = approx-MVUE (Sec. 4.4)
+    int joint;           // 2:4 estimator: 0 = App. A.2 table, 1 = systematic sampling, 2 = approx-MVUE (Sec. 4.4); 3 = MVUE 1:4
 };
 
 cudaError_t launch_prune(const PruneArgs& a, cudaStream_t stream);

@@ -42,7 +42,16 @@ __device__ __forceinline__ void prune_unit_f32(const uint32_t (&b)[16], uint64_t
                                                uint32_t* out_meta) {
     uint32_t v[4];
     uint32_t meta = 0;
-    if (M == 4 && kJoint == 2) {
+    if (M == 4 && kJoint == 3) {
+        const uint4 w = philox4x32_10(unit_index, rk);
+        const uint32_t words[4] = {w.x, w.y, w.z, w.w};
+#pragma unroll
+        for (int j = 0; j < 4; ++j) {
+            uint32_t nib;
+            mvue_1of4_f32(b[4 * j], b[4 * j + 1], b[4 * j + 2], b[4 * j + 3], words[j], &v[j], &nib);
+            meta |= nib << (4 * j);
+        }
+    } else if (M == 4 && kJoint == 2) {
         const uint4 wa = philox4x32_10(2 * unit_index, rk);
         const uint4 wb = philox4x32_10(2 * unit_index + 1, rk);
         const uint32_t words[8] = {wa.x, wa.y, wa.z, wa.w, wb.x, wb.y, wb.z, wb.w};
@@ -459,6 +468,7 @@ cudaError_t launch_prune_m(const PruneArgs& a, cudaStream_t stream) {
 
 cudaError_t launch_prune(const PruneArgs& a, cudaStream_t stream) {
     if (a.m == 2) return launch_prune_m<2, 0>(a, stream);
+    if (a.joint == 3) return launch_prune_m<4, 3>(a, stream);          // MVUE 1:4
     if (a.joint == 2) return launch_prune_m<4, 2>(a, stream);
     return a.joint == 1 ? launch_prune_m<4, 1>(a, stream) : launch_prune_m<4, 0>(a, stream);
 }

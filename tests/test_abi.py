@@ -47,7 +47,8 @@ def test_packed_sizes_and_host_side_checks(L):
     from paper_2203_10991_b200 import binding
     assert binding.mvue_packed_sizes(512, 256, 1, 2, 0) == (256 * 256 * 2, 256 * 64)
     assert binding.mvue_packed_sizes(512, 256, 2, 4, 1) == (512 * 128 * 2, 512 * 32)
-    for n, m in [(1, 4), (4, 8), (2, 2), (0, 0)]:
+    assert binding.mvue_packed_sizes(512, 256, 1, 4, 1) == (512 * 128 * 2, 512 * 32)    # 1:4 sits in the 2:4 container
+    for n, m in [(3, 4), (4, 8), (2, 2), (0, 0)]:
         with pytest.raises(binding.MvueError) as e:
             binding.mvue_packed_sizes(512, 256, n, m, 0)
         assert e.value.status == -2

@@ -62,7 +62,7 @@ def test_one_hot_probes_fix_every_layout():
 
 @pytest.mark.parametrize("T,n_out,n_in", [(128, 8, 8), (512, 256, 256), (640, 136, 264), (2048, 384, 520),
                                           (8192, 768, 3072), (16384, 256, 2304)])
-@pytest.mark.parametrize("n,m", [(2, 4), (1, 2)])
+@pytest.mark.parametrize("n,m", [(2, 4), (1, 2), (1, 4)])
 def test_update_gemm_matches_oracle(T, n_out, n_in, n, m):
     g = workloads.gradient((T, n_out), "student_t", seed=T + n_out, dtype="bf16")
     h = workloads.normal_bf16((T, n_in), seed=7)

@@ -35,7 +35,7 @@ def assert_parity(g_np, n, m, axis, seed, **kw):
     assert bad_v.size == 0, f"{bad_v.size} packed values differ, first at {bad_v[:4]}"
 
 
-MODES = [(1, 2), (2, 4)]
+MODES = [(1, 2), (2, 4), (1, 4)]
 # shapes span several thread blocks and leave ragged tails in both grid dimensions
 SHAPES = [(16, 16), (48, 80), (528, 264), (1040, 1000), (4096, 1024)]
 
@@ -64,7 +64,8 @@ def test_linear_small_config(n, m):
 
 
 @pytest.mark.parametrize("n,m,joint", [(1, 2, None), (2, 4, binding.MVUE_JOINT_TABLE),
-                                       (2, 4, binding.MVUE_JOINT_SYSTEMATIC), (2, 4, binding.MVUE_JOINT_APPROX)])
+                                       (2, 4, binding.MVUE_JOINT_SYSTEMATIC), (2, 4, binding.MVUE_JOINT_APPROX),
+                                       (1, 4, None)])
 def test_linear_small_slice_is_unbiased_over_10k_seeds(n, m, joint):
     # the 16 x 16 slice of the small linear-layer gradient, pruned by the CUDA kernel under 10000 seeds: the mean of
     # the unpacked estimates must sit within six standard errors of the gradient, the standard error taken from the
@@ -92,6 +93,8 @@ def test_linear_small_slice_is_unbiased_over_10k_seeds(n, m, joint):
                     s = abs(blk[2 * h]) + abs(blk[2 * h + 1])
                     if s > 0:
                         p[2 * h], p[2 * h + 1] = abs(blk[2 * h]) / s, abs(blk[2 * h + 1]) / s
+            elif n == 1:                                                    # MVUE 1:4: p_i = |a_i| / S
+                p = np.abs(blk) / max(np.abs(blk).sum(), 1e-300)
             elif np.count_nonzero(blk) < 2:
                 p = (blk != 0).astype(np.float64)
             elif joint == binding.MVUE_JOINT_APPROX:
@@ -170,7 +173,7 @@ def test_same_seed_same_bits_and_seed_matters():
 
 def test_bad_arguments_launch_nothing():
     g = to_dev(workloads.gradient((64, 64), "student_t", seed=1, dtype="bf16"))
-    for n, m, axis, status in [(1, 4, 1, -2), (2, 4, 3, -3)]:
+    for n, m, axis, status in [(3, 4, 1, -2), (2, 4, 3, -3)]:
         with pytest.raises(binding.MvueError) as e:
             binding.mvue_prune(g, n, m, axis, 0)
         assert e.value.status == status
