@@ -96,44 +96,80 @@ __device__ __forceinline__ void prune_unit_f32(const uint32_t (&b)[16], uint64_t
 // index needs a division.
 constexpr int kA1Units = 16;                          // units per block along K
 
+// 32 bytes in one load where the address allows (whole sectors, nothing kept in L1), else two 16-byte loads.
+__device__ __forceinline__ void ldg256(const char* p, uint32_t (&v)[8]) {
+    if ((reinterpret_cast<uintptr_t>(p) & 31u) == 0) {
+        asm volatile("ld.global.nc.L1::no_allocate.v8.b32 {%0, %1, %2, %3, %4, %5, %6, %7}, [%8];"
+                     : "=r"(v[0]), "=r"(v[1]), "=r"(v[2]), "=r"(v[3]), "=r"(v[4]), "=r"(v[5]), "=r"(v[6]), "=r"(v[7])
+                     : "l"(p));
+    } else {
+        const uint4 a = ldg128(p), b = ldg128(p + 16);
+        v[0] = a.x; v[1] = a.y; v[2] = a.z; v[3] = a.w; v[4] = b.x; v[5] = b.y; v[6] = b.z; v[7] = b.w;
+    }
+}
+
 template <int M, bool kBf16, bool kTC, int kJoint>
 __global__ void __launch_bounds__(8 * kA1Units, kBf16 ? 12 : 8)
 prune_axis1_kernel(const void* __restrict__ g, int64_t n_rows, int units_per_row, int64_t ld,
                    int64_t units_per_row_total, int64_t unit_offset, RoundKeys rk,
                    uint4* __restrict__ values, uint16_t* __restrict__ meta) {
-    constexpr int LW = kBf16 ? 2 : 4;                 // 16-byte loads per unit
     const int j = threadIdx.x & 7;
     const int c = blockIdx.y * kA1Units + (threadIdx.x >> 3);
     if (c >= units_per_row) return;
     const int64_t r0 = (int64_t)blockIdx.x * 16 + j;
     uint32_t meta_pair = 0;
+    if (kBf16) {
+        // The short selections (1:2, 1:4) are bound by bytes in flight: both rows' units are requested before either
+        // is pruned (64 bytes per thread).  The 2:4 selections are bound by instruction issue at 40 registers and
+        // keep the second row's load behind the first row's arithmetic.
+        constexpr bool kBothFirst = M == 2 || kJoint == 3;
+        uint32_t raw[2][8];
+        if (kBothFirst) {
 #pragma unroll
-    for (int h = 0; h < 2; ++h) {
-        const int64_t r = r0 + 8 * h;
-        uint32_t mt = 0x4444u;                        // rows that pad A to a multiple of 128 keep a valid pattern
-        if (r < n_rows) {
-            const char* p = reinterpret_cast<const char*>(g) + (r * ld + (int64_t)c * 16) * (kBf16 ? 2 : 4);
-            uint4 in[LW];
+            for (int h = 0; h < 2; ++h) {
+                const int64_t r = r0 + 8 * h;
+                if (r < n_rows) {
+                    ldg256(reinterpret_cast<const char*>(g) + (r * ld + (int64_t)c * 16) * 2, raw[h]);
+                } else {
 #pragma unroll
-            for (int i = 0; i < LW; ++i) in[i] = ldg128(p + 16 * i);
-            const uint64_t unit = (uint64_t)r * (uint64_t)units_per_row_total + (uint64_t)(unit_offset + c);
-            uint4 v;
-            if (kBf16) {
-                const uint32_t raw[8] = {in[0].x, in[0].y, in[0].z, in[0].w, in[1].x, in[1].y, in[1].z, in[1].w};
-                prune_unit_bf16<M, kJoint>(raw, unit, rk, &v, &mt);
-            } else {
-                uint32_t b[16];
-#pragma unroll
-                for (int i = 0; i < 4; ++i) {
-                    b[4 * i] = (&in[i].x)[0]; b[4 * i + 1] = (&in[i].x)[1];
-                    b[4 * i + 2] = (&in[i].x)[2]; b[4 * i + 3] = (&in[i].x)[3];
+                    for (int i = 0; i < 8; ++i) raw[h][i] = 0u;
                 }
-                prune_unit_f32<M, kJoint>(b, unit, rk, &v, &mt);
             }
-            values[r * units_per_row + c] = v;
-            if (!kTC) meta[r * units_per_row + c] = (uint16_t)mt;
         }
-        meta_pair |= mt << (16 * h);
+#pragma unroll
+        for (int h = 0; h < 2; ++h) {
+            const int64_t r = r0 + 8 * h;
+            uint32_t mt = 0x4444u;                    // rows that pad A to a multiple of 128 keep a valid pattern
+            if (r < n_rows) {
+                if (!kBothFirst) ldg256(reinterpret_cast<const char*>(g) + (r * ld + (int64_t)c * 16) * 2, raw[h]);
+                const uint64_t unit = (uint64_t)r * (uint64_t)units_per_row_total + (uint64_t)(unit_offset + c);
+                uint4 v;
+                prune_unit_bf16<M, kJoint>(raw[h], unit, rk, &v, &mt);
+                values[r * units_per_row + c] = v;
+                if (!kTC) meta[r * units_per_row + c] = (uint16_t)mt;
+            }
+            meta_pair |= mt << (16 * h);
+        }
+    } else {
+#pragma unroll
+        for (int h = 0; h < 2; ++h) {
+            const int64_t r = r0 + 8 * h;
+            uint32_t mt = 0x4444u;
+            if (r < n_rows) {
+                const char* p = reinterpret_cast<const char*>(g) + (r * ld + (int64_t)c * 16) * 4;
+                uint32_t lo[8], hi[8];
+                ldg256(p, lo);
+                ldg256(p + 32, hi);
+                const uint32_t b[16] = {lo[0], lo[1], lo[2], lo[3], lo[4], lo[5], lo[6], lo[7],
+                                        hi[0], hi[1], hi[2], hi[3], hi[4], hi[5], hi[6], hi[7]};
+                const uint64_t unit = (uint64_t)r * (uint64_t)units_per_row_total + (uint64_t)(unit_offset + c);
+                uint4 v;
+                prune_unit_f32<M, kJoint>(b, unit, rk, &v, &mt);
+                values[r * units_per_row + c] = v;
+                if (!kTC) meta[r * units_per_row + c] = (uint16_t)mt;
+            }
+            meta_pair |= mt << (16 * h);
+        }
     }
     if (kTC)   // (r0, c) is the low half of its word; r0 % 16 < 8
         *reinterpret_cast<uint32_t*>(reinterpret_cast<char*>(meta) + tc_meta_offset(r0, c, units_per_row >> 3)) = meta_pair;
