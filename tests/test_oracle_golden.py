@@ -11,7 +11,7 @@ from paper_2203_10991_b200 import workloads
 def test_frozen_packed_output():
     rows = [l for l in (Path(__file__).parent / "golden" / "prune_small.txt").read_text().splitlines()
             if l and not l.startswith("#")]
-    assert len(rows) == 12
+    assert len(rows) == 20
     for row in rows:
         head, vhex, mhex = [s.strip() for s in row.split("|")]
         dist, n, m, axis, joint = head.split()
