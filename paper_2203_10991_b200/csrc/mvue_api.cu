@@ -77,13 +77,13 @@ using namespace mvue;
 
 extern "C" {
 
-int mvue_version(void) { return 100; }
+int mvue_version(void) { return 110; }   // 1.1: MVUE 1:4, approx-MVUE 2:4, the issue-rate probe
 
 const char* mvue_status_string(int status) {
     switch (status) {
         case MVUE_OK: return "ok";
         case MVUE_ERR_NULL: return "null pointer";
-        case MVUE_ERR_NM: return "unsupported N:M (only 1:2 and 2:4)";
+        case MVUE_ERR_NM: return "unsupported N:M (only 1:2, 2:4 and 1:4; the fused product: 1:2 and 2:4)";
         case MVUE_ERR_SHAPE: return "bad shape, axis, leading dimension or K shard";
         case MVUE_ERR_ALIGN: return "pointer or leading dimension not 16-byte aligned";
         case MVUE_ERR_DTYPE: return "unsupported dtype";
