@@ -501,7 +501,7 @@ def tensor_bound_case(n, m, peaks, joint):
 
 def prune_sweep(peaks, max_log2: int = 32):
     """Standalone prune+pack bandwidth over bf16 tensors of 2^20 .. 2^max_log2 bytes ([bytes / 8192 x 4096],
-    Student-t values), both pruned axes, 2:4 (pair table, systematic sampling) and 1:2.  Every point is a CUDA graph of
+    Student-t values), both pruned axes, 2:4 (pair table, systematic sampling), 1:2 and 1:4.  Every point is a CUDA graph of
     `reps` launches over rotating input copies that together exceed 2.5 x L2, replayed and timed with events, so the
     small sizes are neither launch-bound on the host nor L2-warm."""
     import torch
@@ -520,7 +520,7 @@ def prune_sweep(peaks, max_log2: int = 32):
     out_v = torch.empty(base_dev.numel() // 2, dtype=torch.bfloat16, device=dev)
     out_m = torch.empty(base_dev.numel() // 8 + (1 << 16), dtype=torch.uint8, device=dev)
     modes = [("2:4 table", 2, 4, binding.MVUE_JOINT_TABLE), ("2:4 systematic", 2, 4, binding.MVUE_JOINT_SYSTEMATIC),
-             ("1:2", 1, 2, binding.MVUE_JOINT_TABLE)]
+             ("1:2", 1, 2, binding.MVUE_JOINT_TABLE), ("1:4", 1, 4, binding.MVUE_JOINT_TABLE)]
     points = []
     side = torch.cuda.Stream()
     for lg in range(20, max_log2 + 1):
