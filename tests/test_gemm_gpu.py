@@ -240,3 +240,35 @@ def test_issue_rate_probe_runs_and_counts_its_work():
         with pytest.raises(binding.MvueError) as e:
             binding.mvue_probe_sparse_mma(bad)
         assert e.value.status == -3
+
+
+def test_long_reduction_ragged_output_with_and_without_the_tail_split():
+    # K = 16384 (128 stages per tile): the small-footprint fp32 epilogue.  9 x 10 = 90 ragged tiles (2056 x 2312: 8-wide
+    # slivers in both directions) over at most 74 resident pairs: with the workspace the last round's tiles are cut
+    # along K (partial tiles written by the same epilogue), without it they stay whole; accumulate; sampled rows of
+    # every row tile, the sliver included, against the oracle.
+    T, n_out, n_in = 16384, 2056, 2312
+    g = workloads.gradient((T, n_out), "student_t", seed=41, dtype="bf16")
+    h = workloads.normal_bf16((T, n_in), seed=42)
+    gd, hd = to_dev(g), to_dev(h)
+    vals, meta = binding.mvue_prune(gd, 2, 4, 0, seed=9, layout=TC)
+    st = torch.zeros(1, dtype=torch.int32, device="cuda")
+    a = binding.mvue_sparse_update_gemm(vals, meta, hd, dev_status=st)            # workspace from the binding
+    whole = torch.empty_like(a)
+    rc = binding.lib().mvue_sparse_update_gemm(vals.data_ptr(), meta.data_ptr(), TC, n_out, T, hd.data_ptr(), n_in, n_in,
+                                               whole.data_ptr(), 0, n_in, 0, None, 0, st.data_ptr(), None)
+    assert rc == 0
+    acc = torch.full((n_out, n_in), 1.5, dtype=torch.float32, device="cuda")
+    binding.mvue_sparse_update_gemm(vals, meta, hd, out=acc, accumulate=True)
+    torch.cuda.synchronize()
+    assert int(st.item()) == 0
+    # the K parts are summed in another order than the whole tile: fp32 rounding of sums of ~0.3-sized entries
+    assert float((whole - a).abs().max()) <= 1e-5 and rel_fro(whole.double().cpu().numpy(), a.double().cpu().numpy()) <= 1e-6
+    assert torch.allclose(acc, a + 1.5, rtol=1e-6, atol=1e-6)
+    v_ref, m_ref = oracle.prune(g, 2, 4, axis=0, seed=9, threads=oracle.host_threads())
+    rows = np.array(sorted({min(r, n_out - 1) for t in range(9) for r in (256 * t, 256 * t + 131, 256 * t + 255)}))
+    A_rows = np.ascontiguousarray(oracle.unpack(np.ascontiguousarray(v_ref[rows]), np.ascontiguousarray(m_ref[rows])))
+    want = oracle.gemm(A_rows, h, threads=oracle.host_threads())
+    for out in (a, whole):
+        got = out[torch.from_numpy(rows).cuda()].double().cpu().numpy()
+        assert rel_fro(got, want) <= TIGHT
