@@ -10,7 +10,8 @@
  * General rules for every call
  *  - All tensor pointers are DEVICE pointers unless an argument says "host".
  *    The caller owns every buffer; the library never allocates or frees device
- *    memory and keeps no device state.
+ *    memory and keeps no device state -- with one exception, the fixed scratch
+ *    array of mvue_sparse_update_gemm_noalloc (described at its declaration).
  *  - `stream` is a cudaStream_t passed as void* (NULL = the legacy default
  *    stream).  Calls enqueue work on that stream and return without waiting.
  *  - The return value is an mvue_status.  Argument errors are detected on the
@@ -131,9 +132,14 @@ MVUE_API int mvue_packed_sizes(int64_t rows, int64_t cols, int n, int m, int axi
  *   q = r * (k_total / M) + (k_offset / M + j) for block j of row r of A.
  * All selection arithmetic is IEEE binary32 in a fixed order without fused
  * multiply-add; survivors are rounded once to bf16 (nearest even).  Zeros: an
- * element of magnitude zero survives only when fewer than N non-zeros exist,
- * with value +0, in the lowest free position.  A (1,2) result is emitted as a
- * valid 2:4 pattern (pair 0 -> position 0/1, pair 1 -> position 2/3).
+ * element of magnitude zero owns a zero-width interval of every threshold walk,
+ * so it survives only when fewer than N non-zeros exist, as a signed zero (its
+ * own sign bit).  Which zero then fills the pattern: (2,4) with the pair table
+ * keeps the top ranks of the (magnitude, position) order -- a lone non-zero
+ * beside position 3, or beside position 2 if it is itself at 3; an all-zero block
+ * keeps positions 2 and 3; (1,2) keeps a_1 whenever a_2 = 0; (1,4) keeps the last
+ * element of an all-zero block.  A (1,2) result is emitted as a valid 2:4 pattern
+ * (pair 0 -> position 0/1, pair 1 -> position 2/3).
  * The same (g, n, m, axis, seed, k_total, k_offset) always gives the same bits.
  *
  * Arguments.
@@ -180,7 +186,7 @@ MVUE_API int mvue_unpack(const void* values, const void* meta, int layout, int64
  * (with a smaller or NULL workspace they are simply computed whole).  dev_status: optional device int, receives
  * MVUE_ERR_DEVICE_TIMEOUT if a bounded pipeline wait expires (then dW is
  * unspecified); otherwise left untouched.
- * Preconditions: T a multiple of 64; out, in multiples of 8; pointers and
+ * Preconditions: T a multiple of 128; out, in multiples of 8; pointers and
  * leading dimensions (in bytes) 16-byte aligned; act_grad needs a bf16 or
  * MVUE_F32 output without accumulate. */
 MVUE_API int mvue_sparse_update_gemm(const void* values, const void* meta, int layout, int64_t out,
@@ -236,12 +242,22 @@ MVUE_API int mvue_gemm_workspace_bytes(int which, int64_t M, int64_t N, int64_t 
  * supply the split-K workspace that mvue_sparse_update_gemm asks for on small outputs
  * with a long reduction.
  *
- * Same result and same arguments as mvue_sparse_update_gemm, minus the workspace: the
- * scratch is a fixed 8 MiB (MVUE_NOALLOC_SCRATCH_BYTES) array inside the library's device
- * image.  Every GPU on which the library is loaded holds those bytes until the process
- * exits.  The call itself allocates nothing, on the host side or the device side.
- *  - A problem whose mvue_gemm_workspace_bytes(0, out, in, T) exceeds the array is refused
- *    with MVUE_ERR_WORKSPACE; nothing is launched.
+ * Same arguments as mvue_sparse_update_gemm, minus the workspace, and the same product (equal
+ * up to the order of the fp32 sums over K, see below): the scratch is a fixed 8 MiB
+ * (MVUE_NOALLOC_SCRATCH_BYTES) array inside the library's device image.  Every GPU on which
+ * the library is loaded holds those bytes until the process exits.  The call itself allocates
+ * nothing, on the host side or the device side.
+ *  - Arguments are checked first, as for mvue_sparse_update_gemm, before anything else happens.
+ *  - Only the split of a long reduction over a small output NEEDS scratch.  A problem whose
+ *    split needs more than the array (the K-split part of mvue_gemm_workspace_bytes(0, out, in,
+ *    T), which is all of it whenever the split applies) is refused with MVUE_ERR_WORKSPACE;
+ *    nothing is launched.
+ *  - Large fp32 outputs use scratch only optionally, to cut the tiles of a mostly idle last
+ *    round along K: that happens here when those partial tiles fit the array, and otherwise the
+ *    tiles are computed whole, exactly as mvue_sparse_update_gemm does when it is given no
+ *    workspace.  So the array may be in use (and the race described below applies) for every
+ *    shape, and the result can differ from mvue_sparse_update_gemm with a full workspace in
+ *    the last bits of those tiles (a different summation order over K).
  *  - The first call on each device looks up the array's device address (that device must
  *    be current, as for every call).  Make that first call outside any stream capture.
  *  - All calls on a device share the one array, and it keeps whatever the last call left.
@@ -262,6 +278,15 @@ MVUE_API int mvue_sparse_update_gemm_noalloc(const void* values, const void* met
  * counted), *pairs (HOST, may be NULL) the number of pairs.  1 <= iters <= 2^20, else MVUE_ERR_SHAPE.  dev_status as
  * for the products (the one wait of the kernel is bounded).  Reads and writes no caller memory. */
 MVUE_API int mvue_probe_sparse_mma(int iters, int* pairs, double* flops, int* dev_status, void* stream);
+
+/* Self-test of the bounded-wait exit that every pipeline wait of the products shares (the paper has no counterpart).
+ * One launch of the probe's blocks with nothing issued: no copy, no tensor-core instruction and no caller memory is in
+ * flight, and nobody ever arrives on the barrier each block waits for, so that wait gives up after `polls` polls
+ * (1 <= polls <= 65536, else MVUE_ERR_SHAPE; a few thousand polls take well under a millisecond).  Every block then
+ * leaves the ordinary way: MVUE_ERR_DEVICE_TIMEOUT is written to *dev_status (device int, required), the pair of
+ * blocks meets at its cluster barrier and tensor memory is handed back.  Nothing traps or faults; the context stays
+ * usable and the next product call must be correct.  Returns MVUE_OK when the launch was enqueued. */
+MVUE_API int mvue_selftest_wait_timeout(int polls, int* dev_status, void* stream);
 
 MVUE_API const char* mvue_status_string(int status);
 /* Text of the last CUDA error seen by the calling thread ("" if none). */

@@ -62,6 +62,12 @@ def lib() -> ctypes.CDLL:
                                        ctypes.POINTER(ctypes.c_int), ctypes.POINTER(ctypes.c_float)]
         L.oracle_mvue_2of4.restype = None
         L.oracle_mvue_2of4_systematic.argtypes = L.oracle_mvue_2of4.argtypes
+        L.oracle_mvue_2of4_cases.argtypes = [ctypes.POINTER(ctypes.c_float), ctypes.c_uint32,
+                                             ctypes.POINTER(ctypes.c_int), ctypes.POINTER(ctypes.c_double)]
+        L.oracle_mvue_2of4_cases.restype = ctypes.c_int
+        L.oracle_sweep_2of4_cases.argtypes = [ctypes.POINTER(ctypes.c_float), ctypes.c_int, ctypes.POINTER(ctypes.c_uint64),
+                                              ctypes.POINTER(ctypes.c_double)]
+        L.oracle_sweep_2of4_cases.restype = ctypes.c_int
         L.oracle_mvue_2of4_systematic.restype = None
         L.oracle_mvue_2of4_approx.argtypes = [ctypes.POINTER(ctypes.c_float), ctypes.c_uint32, ctypes.c_uint32,
                                               ctypes.POINTER(ctypes.c_int), ctypes.POINTER(ctypes.c_float)]
@@ -153,6 +159,29 @@ def mvue_2of4(a, word: int, joint: int = JOINT_TABLE):
     fn = lib().oracle_mvue_2of4 if joint == JOINT_TABLE else lib().oracle_mvue_2of4_systematic
     fn(arr, word & 0xFFFFFFFF, idx, val)
     return (int(idx[0]), int(idx[1])), (float(val[0]), float(val[1]))
+
+
+def mvue_2of4_cases(a, word: int):
+    """App. A.2 case by case in binary64: (case number, (idx0, idx1), (val0, val1)); case -1 (nothing else
+    computed) for a block with fewer than two non-zeros, which the appendix does not cover."""
+    arr = (ctypes.c_float * 4)(*[float(x) for x in a])
+    idx = (ctypes.c_int * 2)()
+    val = (ctypes.c_double * 2)()
+    which = lib().oracle_mvue_2of4_cases(arr, word & 0xFFFFFFFF, idx, val)
+    if which < 0:
+        return -1, None, None
+    return int(which), (int(idx[0]), int(idx[1])), (float(val[0]), float(val[1]))
+
+
+def sweep_2of4_cases(a, mistake: int = 0):
+    """All 2^24 eps through the case-by-case statement of App. A.2 and through mvue_2of4:
+    (case number, draws on which the kept pairs differ, largest relative difference of the kept values).
+    mistake = 1, 2, 3 plants an error in that case's formulas of the case-by-case statement (power check)."""
+    arr = (ctypes.c_float * 4)(*[float(x) for x in a])
+    diff = ctypes.c_uint64()
+    rel = ctypes.c_double()
+    which = lib().oracle_sweep_2of4_cases(arr, int(mistake), ctypes.byref(diff), ctypes.byref(rel))
+    return int(which), int(diff.value), float(rel.value)
 
 
 def mvue_2of4_approx(a, word1: int, word2: int):

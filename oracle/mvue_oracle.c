@@ -19,7 +19,10 @@
  * Parity pins (see tests): Philox against two independent implementations;
  * the 1:2 sampler against the closed form of Sec. 4.1; the 2:4 sampler against
  * the pair table of App. A.2 and the optimal marginals of Sec. 4.2 by an
- * exhaustive sweep over every value of the 24-bit uniform; the second 2:4 law
+ * exhaustive sweep over every value of the 24-bit uniform, and draw by draw
+ * against oracle_mvue_2of4_cases, the appendix written out case by case in
+ * binary64 (same pair on all but a handful of the 2^24 draws, same kept values
+ * to binary32 rounding); the second 2:4 law
  * (systematic sampling) against the same optimal marginals, mean and minimal
  * variance by the same sweep, and against its interval-overlap law; bf16 rounding
  * against a library cast; the product against a library fp64 matmul; the
@@ -212,6 +215,137 @@ void oracle_mvue_2of4(const float a[4], uint32_t word, int idx[2], float val[2])
     const float vb = copysignf(s4 > quarter_D ? s4 : quarter_D, a[pos[kb]]);
     if (pos[ka] < pos[kb]) { idx[0] = pos[ka]; idx[1] = pos[kb]; val[0] = va; val[1] = vb; }
     else                   { idx[0] = pos[kb]; idx[1] = pos[ka]; val[0] = vb; val[1] = va; }
+}
+
+/* ------------------------------------------------------------------------
+ * MVUE 2:4 exactly as App. A.2 prints it, case by case, in binary64.
+ *
+ * This is the reference statement of the appendix and nothing else: sort the
+ * magnitudes (ties by position), decide which of the three cases holds, form
+ * that case's own six pair probabilities p_12 .. p_34 over that case's own
+ * denominator with divisions, and draw the pair by the threshold test
+ * eps < (cumulative p) of App. "Pruning Overhead" Part 1, walking the pairs in
+ * the order the appendix lists them (12, 13, 14, 23, 24, 34), eps = n / 2^24.
+ * A survivor becomes a_i / p_i (Sec. 4.2) with p_i the sum of the p_ij that
+ * contain i.  No algebra is shared between the cases and nothing is rearranged
+ * to avoid a division.
+ *
+ * oracle_mvue_2of4 above is the binary32, division-free evaluation that the GPU
+ * must reproduce bit for bit; this function is what pins it to the appendix
+ * (tests/test_oracle_mvue24.py sweeps every eps through both).  The two may
+ * differ only where binary32 rounding moves a threshold: a handful of the 2^24
+ * draws per block, and the last place of a kept value.
+ *
+ * The appendix assumes a_4 > a_3 > a_2 > a_1 > 0.  Ties and zeros among three
+ * or more non-zeros are covered by its formulas as they stand (a zero gets
+ * zero-width intervals).  With fewer than two non-zero elements every
+ * denominator vanishes (0/0): the function then returns -1 and computes
+ * nothing -- that situation is ruled by the zero rule stated above, not by the
+ * appendix.  Returns the case number (1, 2 or 3) otherwise.
+ * idx[0] < idx[1]: surviving original positions; val[]: their new values
+ * (binary64).
+ * ---------------------------------------------------------------------- */
+int oracle_mvue_2of4_cases_planted(const float a[4], uint32_t word, int idx[2], double val[2], int mistake);
+
+int oracle_mvue_2of4_cases(const float a[4], uint32_t word, int idx[2], double val[2])
+{
+    return oracle_mvue_2of4_cases_planted(a, word, idx, val, 0);
+}
+
+/* The same with one deliberate mistake planted (mistake = 1, 2, 3: in that case's formulas), so that the tests
+ * can show that the comparison with the binary32 sampler would notice it.  mistake = 0 is the appendix. */
+int oracle_mvue_2of4_cases_planted(const float a[4], uint32_t word, int idx[2], double val[2], int mistake)
+{
+    double s[4];
+    int    pos[4];
+    for (int i = 0; i < 4; ++i) {                           /* stable insertion sort by magnitude */
+        double m = fabs((double)a[i]);
+        int j = i;
+        while (j > 0 && m < s[j - 1]) { s[j] = s[j - 1]; pos[j] = pos[j - 1]; --j; }
+        s[j] = m; pos[j] = i;
+    }
+    const double a1 = s[0], a2 = s[1], a3 = s[2], a4 = s[3];
+    if (a3 == 0.0) return -1;                               /* fewer than two non-zeros: 0/0 in every case */
+    const double eps = (double)(word >> 8) / 16777216.0;    /* n / 2^24 */
+    double p12, p13, p14, p23, p24, p34;
+    int which;
+    if (a4 >= a1 + a2 + a3) {
+        /* case 3: a_4 is kept with probability 1, and one of a_1, a_2, a_3 with
+         * probability a_i / (a_1 + a_2 + a_3) */
+        which = 3;
+        const double rest = a1 + a2 + a3;
+        p12 = 0.0; p13 = 0.0; p23 = 0.0;
+        p14 = a1 / rest;
+        p24 = a2 / rest;
+        p34 = a3 / rest;
+        if (mistake == 3) { p14 = p24 = p34 = 1.0 / 3.0; }        /* planted: partner drawn uniformly */
+    } else if (a4 <= 2.0 * a1 + a3) {
+        /* case 1 */
+        which = 1;
+        const double sum = a1 + a2 + a3 + a4;
+        p12 = 0.0;
+        p13 = (2.0 * a1 + a3 - a4) / (2.0 * sum);
+        p14 = (2.0 * a1 - a3 + a4) / (2.0 * sum);
+        p23 = (2.0 * a2 + a3 - a4) / (2.0 * sum);
+        p24 = (2.0 * a2 - a3 + a4) / (2.0 * sum);
+        p34 = (-a1 - a2 + a3 + a4) / sum;
+        if (mistake == 1) { double t = p13; p13 = p14; p14 = t; }  /* planted: a_3 and a_4 swapped in the first row */
+    } else {
+        /* case 2: 2 a_1 + a_3 <= a_4 <= a_1 + a_2 + a_3 */
+        which = 2;
+        const double sum = a1 + a2 + a3 + a4;
+        p12 = 0.0;
+        p13 = 0.0;
+        p14 = (mistake == 2 ? 1.0 : 2.0) * a1 / sum;               /* planted: the factor two dropped */
+        p23 = (a1 + a2 + a3 - a4) / sum;
+        p24 = (-a1 + a2 - a3 + a4) / sum;
+        p34 = (-a1 - a2 + a3 + a4) / sum;
+    }
+    /* threshold walk in the appendix's order */
+    int ra, rb;                                             /* sorted ranks (0..3) of the survivors */
+    double c = p12;
+    if (eps < c) { ra = 0; rb = 1; }
+    else if (eps < (c += p13)) { ra = 0; rb = 2; }
+    else if (eps < (c += p14)) { ra = 0; rb = 3; }
+    else if (eps < (c += p23)) { ra = 1; rb = 2; }
+    else if (eps < (c += p24)) { ra = 1; rb = 3; }
+    else { ra = 2; rb = 3; }
+    /* survival probabilities of the four ranks: sums over the pairs that hold them */
+    const double p[4] = { p12 + p13 + p14, p12 + p23 + p24, p13 + p23 + p34, p14 + p24 + p34 };
+    const double va = copysign(s[ra] / p[ra], (double)a[pos[ra]]);
+    const double vb = copysign(s[rb] / p[rb], (double)a[pos[rb]]);
+    if (pos[ra] < pos[rb]) { idx[0] = pos[ra]; idx[1] = pos[rb]; val[0] = va; val[1] = vb; }
+    else                   { idx[0] = pos[rb]; idx[1] = pos[ra]; val[0] = vb; val[1] = va; }
+    return which;
+}
+
+/* Every eps through both statements of App. A.2 (the case-by-case binary64 one and
+ * the binary32 one above): *pair_diff = the number of the 2^24 draws on which they
+ * keep different pairs; *max_rel = the largest relative difference between their
+ * kept values over the draws on which they keep the same pair (mistake: see
+ * oracle_mvue_2of4_cases_planted; 0 for the appendix as printed).  Returns the case
+ * number, or -1 (and touches nothing) for a block with fewer than two non-zeros. */
+int oracle_sweep_2of4_cases(const float a[4], int mistake, uint64_t *pair_diff, double *max_rel)
+{
+    uint64_t diff = 0;
+    double worst = 0.0;
+    int which = -1;
+    for (uint32_t n = 0; n < (1u << 24); ++n) {
+        int ia[2], ib[2]; double va[2]; float vb[2];
+        which = oracle_mvue_2of4_cases_planted(a, n << 8, ia, va, mistake);
+        if (which < 0) return -1;
+        oracle_mvue_2of4(a, n << 8, ib, vb);
+        if (ia[0] != ib[0] || ia[1] != ib[1]) { diff += 1; continue; }
+        for (int e = 0; e < 2; ++e) {
+            double d = fabs(va[e] - (double)vb[e]);
+            double ref = fabs(va[e]);
+            double rel = ref > 0.0 ? d / ref : d;
+            if (rel > worst) worst = rel;
+        }
+    }
+    *pair_diff = diff;
+    *max_rel = worst;
+    return which;
 }
 
 /* ------------------------------------------------------------------------

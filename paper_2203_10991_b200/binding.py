@@ -22,7 +22,7 @@ MVUE_JOINT_TABLE, MVUE_JOINT_SYSTEMATIC, MVUE_JOINT_APPROX = 0, 1, 2
 EXPORTS = ("mvue_version", "mvue_status_string", "mvue_last_cuda_error", "mvue_packed_sizes",
            "mvue_prune", "mvue_prune_joint", "mvue_unpack", "mvue_sparse_update_gemm", "mvue_sparse_backward_gemm",
            "mvue_gemm_workspace_bytes", "mvue_sparse_update_gemm_noalloc", "mvue_fused_update_gemm",
-           "mvue_probe_sparse_mma")
+           "mvue_probe_sparse_mma", "mvue_selftest_wait_timeout")
 
 
 class MvueError(RuntimeError):
@@ -61,6 +61,7 @@ def lib() -> ctypes.CDLL:
                                              ctypes.c_size_t, vp, vp]
         L.mvue_sparse_update_gemm_noalloc.argtypes = [vp, vp, ci, i64, i64, vp, i64, i64, vp, ci, i64, ci, vp, vp]
         L.mvue_probe_sparse_mma.argtypes = [ci, ctypes.POINTER(ctypes.c_int), ctypes.POINTER(ctypes.c_double), vp, vp]
+        L.mvue_selftest_wait_timeout.argtypes = [ci, vp, vp]
         _lib = L
     return _lib
 
@@ -224,3 +225,9 @@ def mvue_probe_sparse_mma(iters: int, dev_status: torch.Tensor | None = None):
                                        None if dev_status is None else dev_status.data_ptr(), _stream_ptr()),
            "mvue_probe_sparse_mma")
     return pairs.value, flops.value
+
+
+def mvue_selftest_wait_timeout(polls: int, dev_status: torch.Tensor) -> None:
+    """One launch whose only wait nobody answers: it expires after `polls` polls and the blocks leave through the
+    ordinary exit, writing MVUE_ERR_DEVICE_TIMEOUT (-10) to dev_status (int32 CUDA tensor)."""
+    _check(lib().mvue_selftest_wait_timeout(polls, dev_status.data_ptr(), _stream_ptr()), "mvue_selftest_wait_timeout")

@@ -45,9 +45,10 @@ static int check_nm(int n, int m) {
     return ((n == 1 && m == 2) || (n == 2 && m == 4) || (n == 1 && m == 4)) ? MVUE_OK : MVUE_ERR_NM;
 }
 
-static int run_gemm(const void* values, const void* meta, int layout, int64_t M, int64_t N, int64_t K,
-                    const void* B, int64_t ldb, const void* scale, void* C, int c_dtype, int64_t ldc,
-                    int accumulate, void* workspace, size_t workspace_bytes, int* dev_status, void* stream) {
+// Host-side checks shared by the product entry points; fills *dev for the current device.
+static int check_gemm(const void* values, const void* meta, int layout, int64_t M, int64_t N, int64_t K,
+                      const void* B, int64_t ldb, const void* scale, void* C, int c_dtype, int64_t ldc,
+                      int accumulate, DeviceInfo* dev) {
     if (!values || !meta || !B || !C) return MVUE_ERR_NULL;
     if (layout != MVUE_LAYOUT_TC) return MVUE_ERR_LAYOUT;
     if (c_dtype != MVUE_F32 && c_dtype != MVUE_BF16) return MVUE_ERR_DTYPE;
@@ -60,8 +61,14 @@ static int run_gemm(const void* values, const void* meta, int layout, int64_t M,
     if (!aligned16(values) || !aligned16(meta) || !aligned16(B) || !aligned16(C) || (ldb * 2) % 16 != 0 ||
         (ldc * c_esz) % 16 != 0 || (scale && (!aligned16(scale) || (ldc * 2) % 16 != 0)))
         return MVUE_ERR_ALIGN;
+    return current_device_info(dev);
+}
+
+static int run_gemm(const void* values, const void* meta, int layout, int64_t M, int64_t N, int64_t K,
+                    const void* B, int64_t ldb, const void* scale, void* C, int c_dtype, int64_t ldc,
+                    int accumulate, void* workspace, size_t workspace_bytes, int* dev_status, void* stream) {
     DeviceInfo dev;
-    if (int s = current_device_info(&dev)) return s;
+    if (int s = check_gemm(values, meta, layout, M, N, K, B, ldb, scale, C, c_dtype, ldc, accumulate, &dev)) return s;
     // the split of a long K needs its workspace; the K split of the last round's tiles is skipped without it
     const size_t need = gemm_required_workspace_bytes(M, N, K, dev.sm_count);
     if (need > 0 && (!workspace || workspace_bytes < need)) return MVUE_ERR_WORKSPACE;
@@ -77,7 +84,7 @@ using namespace mvue;
 
 extern "C" {
 
-int mvue_version(void) { return 110; }   // 1.1: MVUE 1:4, approx-MVUE 2:4, the issue-rate probe
+int mvue_version(void) { return 120; }   // 1.2: per-device set-up, the bounded-wait self-test
 
 const char* mvue_status_string(int status) {
     switch (status) {
@@ -218,19 +225,29 @@ int mvue_probe_sparse_mma(int iters, int* pairs, double* flops, int* dev_status,
     DeviceInfo dev;
     if (int s = current_device_info(&dev)) return s;
     int n_pairs = 0;
-    if (int s = launch_sparse_mma_probe(iters, dev.sm_count, &n_pairs, dev_status, reinterpret_cast<cudaStream_t>(stream)))
+    if (int s = launch_sparse_mma_probe(iters, 0u, dev.sm_count, &n_pairs, dev_status, reinterpret_cast<cudaStream_t>(stream)))
         return s;
     if (pairs) *pairs = n_pairs;
     if (flops) *flops = (double)n_pairs * (double)iters * 4.0 * 2.0 * 256.0 * 256.0 * 32.0;
     return MVUE_OK;
 }
 
+int mvue_selftest_wait_timeout(int polls, int* dev_status, void* stream) {
+    if (!dev_status) return MVUE_ERR_NULL;
+    if (polls <= 0 || polls > (1 << 16)) return MVUE_ERR_SHAPE;
+    DeviceInfo dev;
+    if (int s = current_device_info(&dev)) return s;
+    return launch_sparse_mma_probe(0, (uint32_t)polls, dev.sm_count, nullptr, dev_status,
+                                   reinterpret_cast<cudaStream_t>(stream));
+}
+
 int mvue_sparse_update_gemm_noalloc(const void* values, const void* meta, int layout, int64_t out, int64_t T,
                                     const void* h, int64_t in, int64_t ldh, void* dW, int dW_dtype,
                                     int64_t lddW, int accumulate, int* dev_status, void* stream) {
-    if (out <= 0 || in <= 0 || T <= 0 || T % 128 != 0) return MVUE_ERR_SHAPE;
+    // every argument is checked before the scratch array's address is looked up (a CUDA call on first use)
     DeviceInfo dev;
-    if (int s = current_device_info(&dev)) return s;
+    if (int s = check_gemm(values, meta, layout, out, in, T, h, ldh, nullptr, dW, dW_dtype, lddW, accumulate, &dev))
+        return s;
     const size_t need = gemm_required_workspace_bytes(out, in, T, dev.sm_count);
     if (need > kStaticScratchBytes) return MVUE_ERR_WORKSPACE;     // beyond what the library carries
     void* scratch = nullptr;

@@ -384,7 +384,7 @@ __device__ __forceinline__ void mvue_2of4_approx_bf16(uint32_t x01, uint32_t x23
 }
 
 // ===========================================================================
-// MVUE 1:4 (the paper's "MVUE 1:4 is similar to MVUE 1:2, but for a bigger block"): element i of the block
+// MVUE 1:4 (appendix "Additional sparsity results"; Sec. 4.1's argument with one survivor of four): element i of the block
 // survives with probability |a_i| / S, S the sum of the four magnitudes, and becomes sign(a_i) S.
 //   c_1 = m_0, c_2 = c_1 + m_1, c_3 = c_2 + m_2, S = c_3 + m_3;  t = n (S 2^-24);  i = #{c_k <= t}.
 // The survivor is stored in the 2:4 container beside a +0: positions (i, 3), or (2, 3) when i = 3.

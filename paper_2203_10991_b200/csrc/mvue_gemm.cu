@@ -89,8 +89,9 @@ __device__ __forceinline__ bool mbar_wait_cluster(uint32_t bar, uint32_t parity,
 }
 // Bounded wait.  Returns false (and raises the block's abort flag) when the bound expires
 // or another role has already given up.
-__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile int* abort_flag) {
-    for (uint32_t spin = 0; spin < kSpinLimit; ++spin) {
+__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile int* abort_flag,
+                                          uint32_t limit = kSpinLimit) {
+    for (uint32_t spin = 0; spin < limit; ++spin) {
         if (mbar_try_wait(bar, parity)) return true;
         if (*abort_flag) return false;
         if (spin > 64) __nanosleep(spin > 4096 ? 256 : 32);
@@ -1002,7 +1003,7 @@ tail_reduce_kernel(const float* __restrict__ partial, int rem, int parts, int64_
 // back, one commit at the end.  The time of this launch is the ceiling any tiling of the product can approach.
 // =============================================================================
 __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(128, 1)
-sparse_mma_issue_probe_kernel(int iters, int* dev_status) {
+sparse_mma_issue_probe_kernel(int iters, uint32_t spin_limit, int* dev_status) {
     extern __shared__ uint8_t smem_raw[];
     const uint32_t smem_base = (smem_u32(smem_raw) + 1023u) & ~1023u;
     uint8_t* smem_gen = smem_raw + (smem_base - smem_u32(smem_raw));
@@ -1033,7 +1034,9 @@ sparse_mma_issue_probe_kernel(int iters, int* dev_status) {
     tc_fence_after();
     const uint32_t tmem_base = *tmem_slot;
 
-    if (rank == 0 && warp == 1 && lane == 0) {
+    // iters = 0 issues nothing and commits nothing: nobody ever arrives on done_bar, so the wait below runs out after
+    // spin_limit polls and both blocks leave through the ordinary exit (the self-test of the bounded-wait path)
+    if (iters > 0 && rank == 0 && warp == 1 && lane == 0) {
         const uint32_t a_addr = smem_base, b_addr = a_addr + kABytes, e_addr = b_addr + kBBytes;
         const uint32_t tmem_e = tmem_base + kTmemECol;
         tc_copy_128x128b_pair(tmem_e, make_smem_desc(e_addr, 16, 128, kSwizzleNone));
@@ -1048,7 +1051,7 @@ sparse_mma_issue_probe_kernel(int iters, int* dev_status) {
         }
         tc_commit_pair(done_bar);                                            // both blocks' barriers, when the MMAs retire
     }
-    const bool ok = mbar_wait(done_bar, 0u, abort_flag);                     // bounded
+    const bool ok = mbar_wait(done_bar, 0u, abort_flag, spin_limit);         // bounded
     tc_fence_after();
     __syncthreads();
     if (!ok && threadIdx.x == 0 && dev_status) *dev_status = MVUE_ERR_DEVICE_TIMEOUT;
@@ -1081,37 +1084,42 @@ size_t gemm_required_workspace_bytes(int64_t M, int64_t N, int64_t K, int sm_cou
 
 namespace {
 
-// The four instantiations of the pair kernel, their shared-memory attribute, and how many pairs fit the GPU at
-// once (one block per SM): the size of the persistent grid.  Looked up once.
+// The instantiations of the pair kernel, their shared-memory attribute, and how many pairs fit the GPU at
+// once (one block per SM): the size of the persistent grid.  Looked up once per device.
 struct PairKernelSetup {
-    cudaError_t attr_err = cudaSuccess;
-    int max_pairs = 0;
+    PerDeviceOnce once;
+    int max_pairs[kMaxDevices] = {};
 };
-const PairKernelSetup& pair_kernel_setup() {
-    static const PairKernelSetup st = [] {
-        PairKernelSetup r;
+PairKernelSetup& pair_setup() {
+    static PairKernelSetup st;
+    return st;
+}
+cudaError_t pair_kernel_setup() {
+    PairKernelSetup& st = pair_setup();
+    return once_per_device(st.once, [&st](int dev) {
         const void* kernels[5] = {reinterpret_cast<const void*>(sparse_gemm_pair_kernel<0>),
                                   reinterpret_cast<const void*>(sparse_gemm_pair_kernel<1>),
                                   reinterpret_cast<const void*>(sparse_gemm_pair_kernel<2>),
                                   reinterpret_cast<const void*>(sparse_gemm_pair_kernel<3>),
                                   reinterpret_cast<const void*>(sparse_gemm_pair_kernel<4>)};
-        for (int i = 0; i < 5 && r.attr_err == cudaSuccess; ++i)
-            r.attr_err = cudaFuncSetAttribute(kernels[i], cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemBytes);
+        cudaError_t err = cudaSuccess;
+        for (int i = 0; i < 5 && err == cudaSuccess; ++i)
+            err = cudaFuncSetAttribute(kernels[i], cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemBytes);
         cudaLaunchConfig_t cfg = {};
         cfg.gridDim = dim3(2, 1, 1);
         cfg.blockDim = dim3(kThreads, 1, 1);
         cfg.dynamicSmemBytes = kSmemBytes;
         int n = 0;
-        if (r.attr_err == cudaSuccess &&
-            cudaOccupancyMaxActiveClusters(&n, sparse_gemm_pair_kernel<0>, &cfg) == cudaSuccess)
-            r.max_pairs = n;
+        if (err == cudaSuccess && cudaOccupancyMaxActiveClusters(&n, sparse_gemm_pair_kernel<0>, &cfg) == cudaSuccess)
+            st.max_pairs[dev] = n;
         (void)cudaGetLastError();
-        return r;
-    }();
-    return st;
+        return err;
+    });
 }
 int resident_pairs(int sm_count) {
-    const int n = pair_kernel_setup().max_pairs;
+    int dev = 0, n = 0;
+    if (pair_kernel_setup() == cudaSuccess && cudaGetDevice(&dev) == cudaSuccess && dev >= 0 && dev < kMaxDevices)
+        n = pair_setup().max_pairs[dev];
     return n > 0 ? n : (sm_count / 2 > 0 ? sm_count / 2 : 1);
 }
 
@@ -1156,11 +1164,11 @@ __device__ __align__(256) static unsigned char g_static_scratch[kStaticScratchBy
 
 int static_scratch(void** ptr, size_t* bytes) {
     static std::mutex mu;
-    static void* addr[64] = {};
+    static void* addr[kMaxDevices] = {};
     int dev = 0;
     cudaError_t e = cudaGetDevice(&dev);
     if (e != cudaSuccess) { set_cuda_error(e, "cudaGetDevice"); return MVUE_ERR_CUDA; }
-    if (dev < 0 || dev >= 64) return MVUE_ERR_ARCH;
+    if (dev < 0 || dev >= kMaxDevices) return MVUE_ERR_ARCH;
     std::lock_guard<std::mutex> lock(mu);
     if (!addr[dev]) {
         void* q = nullptr;
@@ -1196,13 +1204,12 @@ int launch_fused_update(const FusedArgs& f, cudaStream_t stream) {
         set_cuda_error(cudaErrorUnknown, "cuTensorMapEncodeTiled");
         return MVUE_ERR_CUDA;
     }
-    static std::once_flag once;
-    static cudaError_t attr_err = cudaSuccess;
-    std::call_once(once, [] {
-        attr_err = cudaFuncSetAttribute(fused_update_kernel<4>, cudaFuncAttributeMaxDynamicSharedMemorySize, kFSmemBytes);
-        if (attr_err == cudaSuccess)
-            attr_err = cudaFuncSetAttribute(fused_update_kernel<2>, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                            kFSmemBytes);
+    static PerDeviceOnce once;
+    const cudaError_t attr_err = once_per_device(once, [](int) {
+        cudaError_t err = cudaFuncSetAttribute(fused_update_kernel<4>, cudaFuncAttributeMaxDynamicSharedMemorySize, kFSmemBytes);
+        if (err == cudaSuccess)
+            err = cudaFuncSetAttribute(fused_update_kernel<2>, cudaFuncAttributeMaxDynamicSharedMemorySize, kFSmemBytes);
+        return err;
     });
     if (attr_err != cudaSuccess) { set_cuda_error(attr_err, "cudaFuncSetAttribute"); return MVUE_ERR_CUDA; }
 
@@ -1239,18 +1246,18 @@ int launch_fused_update(const FusedArgs& f, cudaStream_t stream) {
     return MVUE_OK;
 }
 
-int launch_sparse_mma_probe(int iters, int sm_count, int* pairs_out, int* dev_status, cudaStream_t stream) {
-    static std::once_flag once;
-    static cudaError_t attr_err = cudaSuccess;
-    std::call_once(once, [] {
-        attr_err = cudaFuncSetAttribute(sparse_mma_issue_probe_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                        kSmemBytes);
+int launch_sparse_mma_probe(int iters, uint32_t spin_limit, int sm_count, int* pairs_out, int* dev_status,
+                            cudaStream_t stream) {
+    static PerDeviceOnce once;
+    const cudaError_t attr_err = once_per_device(once, [](int) {
+        return cudaFuncSetAttribute(sparse_mma_issue_probe_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemBytes);
     });
     if (attr_err != cudaSuccess) { set_cuda_error(attr_err, "cudaFuncSetAttribute"); return MVUE_ERR_CUDA; }
     const int pairs = resident_pairs(sm_count);
     if (pairs_out) *pairs_out = pairs;
     // the product kernel's shared-memory request, so that one block lands on each SM as it does there
-    sparse_mma_issue_probe_kernel<<<dim3((unsigned)(2 * pairs)), 128, kSmemBytes, stream>>>(iters, dev_status);
+    sparse_mma_issue_probe_kernel<<<dim3((unsigned)(2 * pairs)), 128, kSmemBytes, stream>>>(
+        iters, spin_limit == 0 ? kSpinLimit : spin_limit, dev_status);
     const cudaError_t e = cudaGetLastError();
     if (e != cudaSuccess) { set_cuda_error(e, "sparse MMA probe launch"); return MVUE_ERR_CUDA; }
     return MVUE_OK;
@@ -1269,8 +1276,8 @@ int launch_sparse_gemm(const SparseGemmArgs& a, cudaStream_t stream) {
         set_cuda_error(cudaErrorUnknown, "cuTensorMapEncodeTiled");
         return MVUE_ERR_CUDA;
     }
-    const PairKernelSetup& setup = pair_kernel_setup();
-    if (setup.attr_err != cudaSuccess) { set_cuda_error(setup.attr_err, "cudaFuncSetAttribute"); return MVUE_ERR_CUDA; }
+    const cudaError_t setup_err = pair_kernel_setup();
+    if (setup_err != cudaSuccess) { set_cuda_error(setup_err, "cudaFuncSetAttribute"); return MVUE_ERR_CUDA; }
 
     const int splits = gemm_split_count(a.M, a.N, a.K, a.sm_count);
     const int64_t steps = a.K / BK;

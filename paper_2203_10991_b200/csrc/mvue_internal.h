@@ -4,6 +4,7 @@
 
 #include <cstddef>
 #include <cstdint>
+#include <mutex>
 
 namespace mvue {
 
@@ -43,7 +44,9 @@ struct SparseGemmArgs {
     int sm_count;
 };
 int launch_sparse_gemm(const SparseGemmArgs& a, cudaStream_t stream);     // returns an mvue_status
-int launch_sparse_mma_probe(int iters, int sm_count, int* pairs_out, int* dev_status, cudaStream_t stream);   // mvue_status
+// iters = 0: nothing is issued and the kernel's one wait expires after spin_limit polls (0: the default bound)
+int launch_sparse_mma_probe(int iters, uint32_t spin_limit, int sm_count, int* pairs_out, int* dev_status,
+                            cudaStream_t stream);                           // mvue_status
 int gemm_split_count(int64_t M, int64_t N, int64_t K, int sm_count);
 size_t gemm_workspace_bytes(int64_t M, int64_t N, int64_t K, int sm_count);            // what lets every path run
 size_t gemm_required_workspace_bytes(int64_t M, int64_t N, int64_t K, int sm_count);   // the split along K alone
@@ -69,5 +72,27 @@ struct DeviceInfo {
 };
 int current_device_info(DeviceInfo* info);   // returns an mvue_status
 void set_cuda_error(cudaError_t e, const char* where);
+
+// Function attributes (the dynamic shared-memory limit) and occupancy figures belong to a device, not to the
+// process: a set-up step guarded by this runs once on every device that a call arrives on, with that device current.
+constexpr int kMaxDevices = 64;
+struct PerDeviceOnce {
+    std::mutex mu;
+    bool done[kMaxDevices] = {};
+    cudaError_t err[kMaxDevices] = {};
+};
+template <typename F>
+cudaError_t once_per_device(PerDeviceOnce& st, F&& setup) {
+    int dev = 0;
+    const cudaError_t e = cudaGetDevice(&dev);
+    if (e != cudaSuccess) return e;
+    if (dev < 0 || dev >= kMaxDevices) return cudaErrorInvalidDevice;
+    std::lock_guard<std::mutex> lock(st.mu);
+    if (!st.done[dev]) {
+        st.err[dev] = setup(dev);
+        st.done[dev] = true;
+    }
+    return st.err[dev];
+}
 
 }  // namespace mvue

@@ -475,11 +475,10 @@ cudaError_t launch_prune_t(const PruneArgs& a, cudaStream_t stream) {
             constexpr int kS = 4, kW = 2;                                    // strips per tile, warps per block
             if (!make_map_strips(&map_g, a.g, (uint64_t)a.cols, (uint64_t)a.rows, (uint64_t)a.ld * 2, kS))
                 return cudaErrorInvalidValue;
-            static std::once_flag once;
-            static cudaError_t attr_err = cudaSuccess;
-            std::call_once(once, [] {
-                attr_err = cudaFuncSetAttribute(prune_axis0_bf16_kernel<M, kTC, kJoint, kS, kW>,
-                                                cudaFuncAttributeMaxDynamicSharedMemorySize, A0<kS, kW>::kSmemBytes);
+            static PerDeviceOnce once;
+            const cudaError_t attr_err = once_per_device(once, [](int) {
+                return cudaFuncSetAttribute(prune_axis0_bf16_kernel<M, kTC, kJoint, kS, kW>,
+                                            cudaFuncAttributeMaxDynamicSharedMemorySize, A0<kS, kW>::kSmemBytes);
             });
             if (attr_err != cudaSuccess) return attr_err;
             dim3 grid_b((unsigned)((n_strips + kS - 1) / kS), (unsigned)((cover_cols + kA0Cols - 1) / kA0Cols));

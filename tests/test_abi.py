@@ -68,6 +68,17 @@ def test_packed_sizes_and_host_side_checks(L):
     assert L.mvue_prune(ctypes.c_void_p(4100), 1, 16, 16, 16, 2, 4, 1, 0, 16, 0, fake, fake, 0, None) == -4
     assert L.mvue_prune(fake, 1, 16, 16, 20, 2, 4, 1, 0, 16, 0, fake, fake, 0, None) == -4     # ld * 2 % 16
     assert L.mvue_unpack(None, fake, 0, 16, 16, fake, None) == -1
+    # the allocation-free update product checks its arguments like the regular one, before any CUDA call
+    na = L.mvue_sparse_update_gemm_noalloc
+    assert na(None, fake, 1, 256, 512, fake, 256, 256, fake, 0, 256, 0, None, None) == -1
+    assert na(fake, fake, 0, 256, 512, fake, 256, 256, fake, 0, 256, 0, None, None) == -6          # canonical layout
+    assert na(fake, fake, 1, 256, 500, fake, 256, 256, fake, 0, 256, 0, None, None) == -3          # T % 128
+    assert na(fake, fake, 1, 256, 512, ctypes.c_void_p(4100), 256, 256, fake, 0, 256, 0, None, None) == -4
+    assert na(fake, fake, 1, 256, 512, fake, 256, 256, fake, 1, 256, 1, None, None) == -5          # bf16 += is not offered
+    # the bounded-wait self-test: a status word is required, the poll count is bounded
+    assert L.mvue_selftest_wait_timeout(100, None, None) == -1
+    assert L.mvue_selftest_wait_timeout(0, fake, None) == -3
+    assert L.mvue_selftest_wait_timeout(1 << 20, fake, None) == -3
 
 
 def test_no_silent_cpu_path(L):

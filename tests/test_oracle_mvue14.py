@@ -1,5 +1,5 @@
-"""Pins for the oracle's MVUE 1:4 sampler: the keep-one estimator of Sec. 4.1 on a block of four (the paper's
-"MVUE 1:4 is similar to MVUE 1:2, but for a bigger block")."""
+"""Pins for the oracle's MVUE 1:4 sampler: the keep-one estimator of Sec. 4.1 on a block of four (the MVUE 1:4 of
+the appendix "Additional sparsity results")."""
 import itertools
 import math
 

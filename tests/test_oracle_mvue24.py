@@ -209,3 +209,54 @@ def test_case3_keeps_the_dominant_element_for_every_eps():
         with_top = sum(f for (pair, f) in zip(oracle.PAIRS, freq) if top in pair)
         assert with_top == 1.0
         assert mean[top] == np.float32(block[top])
+
+
+# ------------------------------------------- the appendix, case by case -------
+# oracle.mvue_2of4_cases is App. A.2 as printed (three branches, each with its own numerators and denominator,
+# divisions, binary64); oracle.mvue_2of4 is the binary32, division-free evaluation that the GPU reproduces.
+CASE_BLOCKS = [b for b in ADVERSARIAL if np.count_nonzero(b) >= 2] + [list(b) for b in random_blocks(10)]
+PAIR_SLIPS_PER_BLOCK = 4          # draws (of 2^24) on which binary32 rounding of a threshold may move the pair (seen: <= 2)
+
+
+@pytest.mark.parametrize("block", CASE_BLOCKS)
+def test_binary32_sampler_equals_the_case_by_case_appendix(block):
+    a32 = np.array(block, dtype=np.float32)
+    if np.count_nonzero(a32) < 2:
+        pytest.skip("fewer than two non-zeros: outside the appendix (zero rule)")
+    which, slips, rel = oracle.sweep_2of4_cases(a32)
+    m = np.sort(np.abs(a32.astype(np.float64)))
+    want_case = 3 if m[3] >= m[0] + m[1] + m[2] else (1 if m[3] <= 2 * m[0] + m[2] else 2)
+    assert which == want_case
+    # same pair on every draw but a handful, same kept values to binary32 rounding on all of them
+    assert slips <= PAIR_SLIPS_PER_BLOCK
+    assert rel <= 2.0 ** -22           # three binary32 additions against exact binary64 (seen: 2^-24.2)
+
+
+def test_case_by_case_appendix_on_single_draws():
+    # [1,2,3,4] is case 1 with denominators 2 * 10: p_13 = 1/20, p_14 = 3/20, p_23 = 3/20, p_24 = 5/20, p_34 = 8/20
+    def pick(eps):
+        return oracle.mvue_2of4_cases([1, 2, 3, 4], int(eps * 2**24) << 8)
+    assert pick(0.02)[:2] == (1, (0, 2)) and pick(0.10)[:2] == (1, (0, 3)) and pick(0.30)[:2] == (1, (1, 2))
+    assert pick(0.50)[:2] == (1, (1, 3)) and pick(0.70)[:2] == (1, (2, 3))
+    assert np.allclose(pick(0.30)[2], (5.0, 5.0), rtol=1e-15)                 # a_i / p_i = sum / 2
+    # case 2, [1,2,3,5.5] (sum 11.5): p_14 = 2/11.5, p_23 = 0.5/11.5, p_24 = 3.5/11.5, p_34 = 5.5/11.5
+    which, idx, val = oracle.mvue_2of4_cases([1, 2, 3, 5.5], int(0.1 * 2**24) << 8)
+    assert (which, idx) == (2, (0, 3)) and np.allclose(val, (5.75, 5.75), rtol=1e-15)
+    assert oracle.mvue_2of4_cases([1, 2, 3, 5.5], int(0.2 * 2**24) << 8)[1] == (1, 2)
+    # case 3, [1,-1,-10,1]: the dominant element keeps its value, the partner becomes sign * 3
+    which, idx, val = oracle.mvue_2of4_cases([1, -1, -10, 1], int(0.5 * 2**24) << 8)
+    assert which == 3 and idx == (1, 2) and np.allclose(val, (-3.0, -10.0), rtol=1e-15)
+    # fewer than two non-zeros: the appendix has nothing to say (0/0)
+    assert oracle.mvue_2of4_cases([0, 2, 0, 0], 0)[0] == -1
+    assert oracle.mvue_2of4_cases([0, 0, 0, 0], 0)[0] == -1
+
+
+def test_the_comparison_with_the_appendix_has_power():
+    # one mistake planted in each case of the case-by-case statement: the sweep then disagrees with the binary32
+    # sampler on a macroscopic share of the draws, not on a handful
+    for mistake, block in ((1, [1, 2, 3, 4]), (2, [1, 2, 3, 5.5]), (3, [1, 2, 3, 10])):
+        a32 = np.array(block, dtype=np.float32)
+        which, slips, _ = oracle.sweep_2of4_cases(a32, mistake)
+        assert which == mistake
+        assert slips > 2 ** 24 // 50
+        assert oracle.sweep_2of4_cases(a32)[1] <= PAIR_SLIPS_PER_BLOCK
