@@ -301,6 +301,74 @@ __device__ __forceinline__ void mvue_2of4_sys_bf16(uint32_t x01, uint32_t x23, u
     *nibble = 14u - r.li - 4u * r.lj;                                         // i | j << 2
 }
 
+// Two blocks at a time on packed binary32 pairs: add.rn.f32x2 / sub.rn.f32x2 round each half exactly as the scalar
+// instruction does, so the result is that of mvue_2of4_sys_bf16 on each block, bit for bit, in about three quarters of
+// the issue slots (the kernel is bound by instruction issue, not by the arithmetic pipes).  Every multiplication
+// stays scalar: a packed multiply that feeds a packed add or subtract gets contracted into a fused multiply-add --
+// one rounding instead of two -- which moves a threshold by one unit in the last place on a few draws in 2^23.
+__device__ __forceinline__ uint64_t pack_f32x2(float lo, float hi) {
+    uint64_t r;
+    asm("mov.b64 %0, {%1, %2};" : "=l"(r) : "f"(lo), "f"(hi));
+    return r;
+}
+__device__ __forceinline__ void unpack_f32x2(uint64_t v, float& lo, float& hi) {
+    asm("mov.b64 {%0, %1}, %2;" : "=f"(lo), "=f"(hi) : "l"(v));
+}
+__device__ __forceinline__ uint64_t add_f32x2(uint64_t a, uint64_t b) {
+    uint64_t r;
+    asm("add.rn.f32x2 %0, %1, %2;" : "=l"(r) : "l"(a), "l"(b));
+    return r;
+}
+__device__ __forceinline__ uint64_t sub_f32x2(uint64_t a, uint64_t b) {
+    uint64_t r;
+    asm("sub.rn.f32x2 %0, %1, %2;" : "=l"(r) : "l"(a), "l"(b));
+    return r;
+}
+
+// Blocks A = (xa01, xa23; word wa) and B = (xb01, xb23; word wb), each as in mvue_2of4_sys_bf16.
+__device__ __forceinline__ void mvue_2of4_sys_bf16_x2(uint32_t xa01, uint32_t xa23, uint32_t xb01, uint32_t xb23,
+                                                      uint32_t wa, uint32_t wb, uint32_t* out_a, uint32_t* out_b,
+                                                      uint32_t* nibble_a, uint32_t* nibble_b) {
+    // magnitudes: both sign bits of a word cleared at once, then widened
+    const uint32_t ya01 = xa01 & 0x7FFF7FFFu, ya23 = xa23 & 0x7FFF7FFFu, yb01 = xb01 & 0x7FFF7FFFu, yb23 = xb23 & 0x7FFF7FFFu;
+    const float a0 = __uint_as_float(ya01 << 16), a1 = __uint_as_float(ya01 & 0xFFFF0000u);
+    const float a2 = __uint_as_float(ya23 << 16), a3 = __uint_as_float(ya23 & 0xFFFF0000u);
+    const float b0 = __uint_as_float(yb01 << 16), b1 = __uint_as_float(yb01 & 0xFFFF0000u);
+    const float b2 = __uint_as_float(yb23 << 16), b3 = __uint_as_float(yb23 & 0xFFFF0000u);
+    const uint64_t m0 = pack_f32x2(a0, b0), m1 = pack_f32x2(a1, b1), m2 = pack_f32x2(a2, b2), m3 = pack_f32x2(a3, b3);
+    const float tiny1 = __uint_as_float(1u);                                  // 2^-149
+    const uint64_t tiny = pack_f32x2(tiny1, tiny1);
+    const uint64_t q01 = add_f32x2(add_f32x2(m0, m1), tiny), q23 = add_f32x2(add_f32x2(m2, m3), tiny);
+    const uint64_t R0 = add_f32x2(m1, q23), R1 = add_f32x2(m0, q23), R2 = add_f32x2(q01, m3), R3 = add_f32x2(q01, m2);
+    float r0a, r0b, r1a, r1b, r2a, r2b, r3a, r3b;
+    unpack_f32x2(R0, r0a, r0b); unpack_f32x2(R1, r1a, r1b); unpack_f32x2(R2, r2a, r2b); unpack_f32x2(R3, r3a, r3b);
+    const uint64_t c1 = pack_f32x2(fminf(a0, r0a), fminf(b0, r0b)), e1 = pack_f32x2(fminf(a1, r1a), fminf(b1, r1b));
+    const uint64_t e2 = pack_f32x2(fminf(a2, r2a), fminf(b2, r2b)), e3 = pack_f32x2(fminf(a3, r3a), fminf(b3, r3b));
+    const uint64_t c2 = add_f32x2(c1, e1), c3 = add_f32x2(c2, e2), D = add_f32x2(c3, e3);
+    float Da, Db;
+    unpack_f32x2(D, Da, Db);
+    const float Ha = __fmul_rn(0.5f, Da), Hb = __fmul_rn(0.5f, Db);
+    const float t2a = __fmul_rn(__uint_as_float(__umulhi(wa, 1u << 23) + 0x4B000000u), __fmul_rn(Da, 5.9604644775390625e-08f));
+    const float t2b = __fmul_rn(__uint_as_float(__umulhi(wb, 1u << 23) + 0x4B000000u), __fmul_rn(Db, 5.9604644775390625e-08f));
+    const uint64_t t2 = pack_f32x2(t2a, t2b), t = sub_f32x2(t2, pack_f32x2(Ha, Hb));
+    float d1a, d1b, d2a, d2b, d3a, d3b, d4a, d4b;                             // x < c is the sign bit of x - c
+    unpack_f32x2(sub_f32x2(t, c1), d1a, d1b); unpack_f32x2(sub_f32x2(t, c2), d2a, d2b);
+    unpack_f32x2(sub_f32x2(t2, c2), d3a, d3b); unpack_f32x2(sub_f32x2(t2, c3), d4a, d4b);
+    auto sign = [](float x) { return __umulhi(__float_as_uint(x), 2u); };
+    {
+        const uint32_t li = sign(d1a) + sign(d2a), lj = min(sign(d3a) + sign(d4a), li);
+        const uint32_t raw = __byte_perm(xa01, xa23, 0x7654u - 0x22u * li - 0x2200u * lj);
+        *out_a = __vmaxs2(raw, pack_bf16x2(Ha, Ha) | (raw & 0x80008000u));
+        *nibble_a = 14u - li - 4u * lj;
+    }
+    {
+        const uint32_t li = sign(d1b) + sign(d2b), lj = min(sign(d3b) + sign(d4b), li);
+        const uint32_t raw = __byte_perm(xb01, xb23, 0x7654u - 0x22u * li - 0x2200u * lj);
+        *out_b = __vmaxs2(raw, pack_bf16x2(Hb, Hb) | (raw & 0x80008000u));
+        *nibble_b = 14u - li - 4u * lj;
+    }
+}
+
 // binary32 source: b0..b3 are the raw bit patterns.
 __device__ __forceinline__ void mvue_2of4_sys_f32(uint32_t b0, uint32_t b1, uint32_t b2, uint32_t b3,
                                                   uint32_t word, uint32_t* out, uint32_t* nibble) {
@@ -432,17 +500,20 @@ __device__ __forceinline__ void prune_unit_bf16(const uint32_t (&raw)[8], uint64
             mvue_2of4_approx_bf16(raw[2 * j], raw[2 * j + 1], words[2 * j], words[2 * j + 1], &v[j], &nib);
             meta += nib << (4 * j);
         }
+    } else if (M == 4 && kJoint == 1) {                // systematic sampling: the unit's four blocks two at a time
+        const uint4 w = philox4x32_10(unit_index, rk);
+        uint32_t nib[4];
+        mvue_2of4_sys_bf16_x2(raw[0], raw[1], raw[2], raw[3], w.x, w.y, &v[0], &v[1], &nib[0], &nib[1]);
+        mvue_2of4_sys_bf16_x2(raw[4], raw[5], raw[6], raw[7], w.z, w.w, &v[2], &v[3], &nib[2], &nib[3]);
+        meta = nib[0] + (nib[1] << 4) + (nib[2] << 8) + (nib[3] << 12);
     } else if (M == 4) {
         const uint4 w = philox4x32_10(unit_index, rk);
         const uint32_t words[4] = {w.x, w.y, w.z, w.w};
 #pragma unroll
         for (int j = 0; j < 4; ++j) {
             uint32_t nib;
-            if (kJoint == 0)
-                mvue_2of4_bf16<false, true, false, true>(raw[2 * j], raw[2 * j], raw[2 * j + 1], raw[2 * j + 1],
-                                                         words[j], &v[j], &nib);
-            else
-                mvue_2of4_sys_bf16(raw[2 * j], raw[2 * j + 1], words[j], &v[j], &nib);
+            mvue_2of4_bf16<false, true, false, true>(raw[2 * j], raw[2 * j], raw[2 * j + 1], raw[2 * j + 1],
+                                                     words[j], &v[j], &nib);
             meta += nib << (4 * j);
         }
     } else {

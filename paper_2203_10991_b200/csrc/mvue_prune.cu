@@ -415,6 +415,101 @@ prune_axis0_bf16_kernel(const __grid_constant__ CUtensorMap map_g, const void* _
     }
 }
 
+// ---- axis 0, bf16, whole tiles ------------------------------------------------
+// For tensors made of whole tiles of 128 rows x 64 columns (every packed operand in tensor-core order is: K is a multiple
+// of 128 there).  One TMA box copy through the 5-D view of make_map_strip_pairs; four warps, warp w owns the 16 columns
+// 16 w .. 16 w + 15 of the tile, lane l the columns 16 w + l / 4 and + 8 and, of each, the two consecutive strips
+// 2 (l % 4) and 2 (l % 4) + 1 of the tile's eight: four units per lane, the two strips of a column leave as ONE 32-byte
+// store of survivors, and rows c and c + 8 of A share their metadata words as in the kernel above.  Against that kernel:
+// half as many blocks, barriers and copies per byte, no bounds checks, and the addressing of a unit pair shared.
+constexpr int kWTRows = 128, kWTCols = 64, kWTBytes = kWTRows * kWTCols * 2, kWTWarps = 4;
+
+template <int kDummy>
+__device__ __noinline__ void fill_whole_tile_bf16(const char* g, int64_t ld, int64_t row0, int64_t col0, unsigned char* tile) {
+    for (int i = threadIdx.x; i < kWTRows * 8; i += 32 * kWTWarps) {         // 16-byte chunks; line = 16 k8 + 8 h + 2 pair + k2
+        const int line = i >> 3, chunk = i & 7;
+        const int k8 = line >> 4, h = (line >> 3) & 1, pair = (line >> 1) & 3, k2 = line & 1;
+        const int64_t r = row0 + 32 * pair + 16 * h + 2 * k8 + k2, c = col0 + 8 * chunk;
+        *reinterpret_cast<uint4*>(tile + line * 128 + ((chunk ^ (line & 7)) << 4)) = ldg128(g + (r * ld + c) * 2);
+    }
+}
+
+template <int M, bool kTC, int kJoint>
+__global__ void __launch_bounds__(32 * kWTWarps, 12)
+prune_axis0_bf16_whole_tiles_kernel(const __grid_constant__ CUtensorMap map_g, const void* __restrict__ g, int64_t n_strips,
+                                    int64_t ld, int64_t units_per_row_total, int64_t unit_offset, RoundKeys rk,
+                                    uint4* __restrict__ values, uint16_t* __restrict__ meta) {
+    __shared__ __align__(1024) unsigned char s_tile[kWTBytes];                // the 128-byte swizzle needs 1 KiB alignment
+    __shared__ __align__(8) uint64_t s_bar;
+    const uint32_t tile = smem_addr(s_tile), bar = smem_addr(&s_bar);
+    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+    const int64_t strip0 = (int64_t)blockIdx.x * 8;
+    const int64_t col0 = (int64_t)blockIdx.y * kWTCols;
+
+    if (tid == 0) {
+        asm volatile("mbarrier.init.shared::cta.b64 [%0], 1;" ::"r"(bar));
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+        asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "r"(kWTBytes) : "memory");
+        asm volatile(
+            "cp.async.bulk.tensor.5d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3, %4, %5, %6}], [%7];"
+            ::"r"(tile), "l"(&map_g), "r"((int)col0), "r"(0), "r"((int)(strip0 >> 1)), "r"(0), "r"(0), "r"(bar) : "memory");
+    }
+    __syncthreads();
+    bool landed = false;
+    for (uint32_t spin = 0; spin < (1u << 20) && !landed; ++spin) {           // bounded wait
+        uint32_t ok;
+        asm volatile("{\n\t.reg .pred p;\n\tmbarrier.try_wait.parity.shared::cta.b64 p, [%1], 0;\n\t"
+                     "selp.u32 %0, 1, 0, p;\n\t}" : "=r"(ok) : "r"(bar) : "memory");
+        landed = ok != 0;
+    }
+    if (__syncthreads_or(!landed)) {                                         // the copy never landed: plain loads instead
+        fill_whole_tile_bf16<0>(reinterpret_cast<const char*>(g), ld, strip0 * 16, col0, s_tile);
+        __syncthreads();
+    }
+
+    const int p = lane & 3, cq = lane >> 2;
+    // address this lane supplies to the matrix loads: matrix lane / 8 = k8 (+ 4 for the second load), line
+    // 16 k8 + 8 h + lane % 8, 16-byte chunk (column block) ^ (lane % 8)
+    const uint32_t ld_base = tile + (uint32_t)((16 * (lane >> 3) + (lane & 7)) * 128 + ((lane & 7) << 4));
+    const int64_t strip = strip0 + 2 * p;                                    // this lane's first strip (even)
+    uint32_t meta_h[2] = {0u, 0u};                                           // strip parity h: rows c (low half) and c + 8 (high)
+#pragma unroll
+    for (int step = 0; step < 2; ++step) {
+        const int cb = 2 * warp + step;                                      // 8-column block inside the tile
+        const int64_t c = col0 + 8 * cb + cq;
+        const uint64_t unit = (uint64_t)c * (uint64_t)units_per_row_total + (uint64_t)(unit_offset + strip);
+        uint32_t raw[2][8];
+#pragma unroll
+        for (int h = 0; h < 2; ++h) {
+            const uint32_t addr = (ld_base ^ (uint32_t)(cb << 4)) + (uint32_t)(h * 8 * 128);
+            asm volatile("ldmatrix.sync.aligned.m8n8.x4.trans.shared.b16 {%0, %1, %2, %3}, [%4];"
+                         : "=r"(raw[h][0]), "=r"(raw[h][1]), "=r"(raw[h][2]), "=r"(raw[h][3]) : "r"(addr));
+            asm volatile("ldmatrix.sync.aligned.m8n8.x4.trans.shared.b16 {%0, %1, %2, %3}, [%4];"
+                         : "=r"(raw[h][4]), "=r"(raw[h][5]), "=r"(raw[h][6]), "=r"(raw[h][7]) : "r"(addr + 64u * 128u));
+        }
+        uint4 v[2];
+        uint32_t mt[2];
+#pragma unroll
+        for (int h = 0; h < 2; ++h) prune_unit_bf16<M, kJoint>(raw[h], unit + h, rk, &v[h], &mt[h]);
+        uint4* dst = values + c * n_strips + strip;                          // 32-byte aligned: n_strips and strip are even
+        asm volatile("st.global.v8.b32 [%0], {%1, %2, %3, %4, %5, %6, %7, %8};"
+                     ::"l"(dst), "r"(v[0].x), "r"(v[0].y), "r"(v[0].z), "r"(v[0].w), "r"(v[1].x), "r"(v[1].y),
+                       "r"(v[1].z), "r"(v[1].w) : "memory");
+        if (!kTC) *reinterpret_cast<uint32_t*>(meta + c * n_strips + strip) = mt[0] | (mt[1] << 16);
+        meta_h[0] |= mt[0] << (16 * step);
+        meta_h[1] |= mt[1] << (16 * step);
+    }
+    if (kTC) {
+        // rows c and c + 8 share the 32-bit word (k % 128) / 32 = p of lane c % 8 + 8 h + 16 (c % 128 / 16)
+        const int64_t c = col0 + 16 * warp + cq;
+        const int rl = (int)(c & 127);
+        const int64_t block = (c >> 7) * (n_strips >> 3) + (strip0 >> 3);
+        char* base = reinterpret_cast<char*>(meta) + block * 2048 + ((rl & 7) + 16 * (rl >> 4)) * 16 + p * 4;
+        *reinterpret_cast<uint32_t*>(base) = meta_h[0];
+        *reinterpret_cast<uint32_t*>(base + 128) = meta_h[1];
+    }
+}
+
 // ---- unpack ---------------------------------------------------------------
 // One thread expands one unit: a 16-bit metadata word (four groups) and its 8 survivors
 // become 16 dense elements (32 bytes).
@@ -469,7 +564,17 @@ cudaError_t launch_prune_t(const PruneArgs& a, cudaStream_t stream) {
         const int64_t cover_cols = kTC ? ((a.cols + 127) / 128) * 128 : a.cols;
         dim3 grid((unsigned)((n_strips + kTileStrips - 1) / kTileStrips),
                   (unsigned)((cover_cols + kTileCols - 1) / kTileCols));
-        if (kBf16) {
+        // whole tiles of 128 rows x 64 columns (and no padding rows of A to cover): the kernel without bounds checks
+        if (kBf16 && a.rows % kWTRows == 0 && a.cols % kWTCols == 0 && cover_cols == a.cols &&
+            reinterpret_cast<uintptr_t>(a.values) % 32 == 0) {
+            CUtensorMap map_g;
+            memset(&map_g, 0, sizeof(map_g));
+            if (!make_map_strip_pairs(&map_g, a.g, (uint64_t)a.cols, (uint64_t)a.rows, (uint64_t)a.ld * 2))
+                return cudaErrorInvalidValue;
+            dim3 grid_w((unsigned)(a.rows / kWTRows), (unsigned)(a.cols / kWTCols));
+            prune_axis0_bf16_whole_tiles_kernel<M, kTC, kJoint><<<grid_w, 32 * kWTWarps, 0, stream>>>(
+                map_g, a.g, n_strips, a.ld, upr_total, uoff, rk, values, meta);
+        } else if (kBf16) {
             CUtensorMap map_g;
             memset(&map_g, 0, sizeof(map_g));
             constexpr int kS = 4, kW = 2;                                    // strips per tile, warps per block

@@ -40,8 +40,9 @@ def assert_parity(g_np, axis, seed, joint=SYS, **kw):
     assert bad_v.size == 0, f"{bad_v.size} packed values differ, first at {bad_v[:4]}"
 
 
-# shapes span several thread blocks and leave ragged tails in both grid dimensions
-SHAPES = [(16, 16), (48, 80), (528, 264), (1040, 1000), (4096, 1024)]
+# shapes span several thread blocks and leave ragged tails in both grid dimensions; the last three are made of whole
+# 128 x 64 tiles, which the bf16 prune down the rows handles with a kernel of its own
+SHAPES = [(16, 16), (48, 80), (528, 264), (1040, 1000), (4096, 1024), (256, 192), (1152, 320)]
 
 
 @pytest.mark.parametrize("joint", JOINTS)
