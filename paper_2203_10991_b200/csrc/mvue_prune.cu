@@ -438,13 +438,15 @@ template <int M, bool kTC, int kJoint>
 __global__ void __launch_bounds__(32 * kWTWarps, 12)
 prune_axis0_bf16_whole_tiles_kernel(const __grid_constant__ CUtensorMap map_g, const void* __restrict__ g, int64_t n_strips,
                                     int64_t ld, int64_t units_per_row_total, int64_t unit_offset, RoundKeys rk,
-                                    uint4* __restrict__ values, uint16_t* __restrict__ meta) {
+                                    uint4* __restrict__ values, uint16_t* __restrict__ meta, int col_tiles_fastest) {
     __shared__ __align__(1024) unsigned char s_tile[kWTBytes];                // the 128-byte swizzle needs 1 KiB alignment
     __shared__ __align__(8) uint64_t s_bar;
     const uint32_t tile = smem_addr(s_tile), bar = smem_addr(&s_bar);
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
-    const int64_t strip0 = (int64_t)blockIdx.x * 8;
-    const int64_t col0 = (int64_t)blockIdx.y * kWTCols;
+    // a narrow g (a few column tiles) is walked column tile fastest: the blocks that run together then read whole rows
+    // of g between them instead of one 128-byte piece of every row
+    const int64_t strip0 = (int64_t)(col_tiles_fastest ? blockIdx.y : blockIdx.x) * 8;
+    const int64_t col0 = (int64_t)(col_tiles_fastest ? blockIdx.x : blockIdx.y) * kWTCols;
 
     if (tid == 0) {
         asm volatile("mbarrier.init.shared::cta.b64 [%0], 1;" ::"r"(bar));
@@ -571,9 +573,11 @@ cudaError_t launch_prune_t(const PruneArgs& a, cudaStream_t stream) {
             memset(&map_g, 0, sizeof(map_g));
             if (!make_map_strip_pairs(&map_g, a.g, (uint64_t)a.cols, (uint64_t)a.rows, (uint64_t)a.ld * 2))
                 return cudaErrorInvalidValue;
-            dim3 grid_w((unsigned)(a.rows / kWTRows), (unsigned)(a.cols / kWTCols));
+            const unsigned row_tiles = (unsigned)(a.rows / kWTRows), col_tiles = (unsigned)(a.cols / kWTCols);
+            const bool col_fast = col_tiles <= 8 && row_tiles <= 65535u;    // (the second grid dimension is 16 bits wide)
+            const dim3 grid_w = col_fast ? dim3(col_tiles, row_tiles) : dim3(row_tiles, col_tiles);
             prune_axis0_bf16_whole_tiles_kernel<M, kTC, kJoint><<<grid_w, 32 * kWTWarps, 0, stream>>>(
-                map_g, a.g, n_strips, a.ld, upr_total, uoff, rk, values, meta);
+                map_g, a.g, n_strips, a.ld, upr_total, uoff, rk, values, meta, col_fast ? 1 : 0);
         } else if (kBf16) {
             CUtensorMap map_g;
             memset(&map_g, 0, sizeof(map_g));
