@@ -87,6 +87,12 @@ def lib() -> ctypes.CDLL:
                                    ctypes.c_uint64, ctypes.c_int64, ctypes.c_int64,
                                    ctypes.c_void_p, ctypes.c_void_p, ctypes.c_int, ctypes.c_int]
         L.oracle_prune.restype = ctypes.c_int
+        L.oracle_prune_rounded.argtypes = L.oracle_prune.argtypes + [ctypes.c_int]
+        L.oracle_prune_rounded.restype = ctypes.c_int
+        L.oracle_bf16_sr.argtypes = [ctypes.c_float, ctypes.c_uint16]
+        L.oracle_bf16_sr.restype = ctypes.c_uint16
+        L.oracle_rounding_bits.argtypes = [ctypes.c_uint64, ctypes.c_uint64, ctypes.c_int]
+        L.oracle_rounding_bits.restype = ctypes.c_uint16
         L.oracle_unpack.argtypes = [ctypes.c_void_p, ctypes.c_void_p, ctypes.c_int64, ctypes.c_int64,
                                     ctypes.c_void_p]
         L.oracle_unpack.restype = None
@@ -223,10 +229,20 @@ def packed_shapes(rows: int, cols: int, axis: int):
     return (mrows, k // 2), (mrows, k // 8)
 
 
+def bf16_sr(x: float, r: int) -> int:
+    """Stochastic rounding of a binary32 value to bf16 bits with the 16 random bits r."""
+    return int(lib().oracle_bf16_sr(float(x), r & 0xFFFF))
+
+
+def rounding_bits(seed: int, unit: int, slot: int) -> int:
+    return int(lib().oracle_rounding_bits(seed & (2**64 - 1), unit, slot))
+
+
 def prune(g: np.ndarray, n: int, m: int, axis: int, seed: int, *, k_total: int | None = None,
-          k_offset: int = 0, threads: int = 1, joint: int = JOINT_TABLE):
+          k_offset: int = 0, threads: int = 1, joint: int = JOINT_TABLE, stochastic_rounding: bool = False):
     """MVUE n:m prune + pack of a 2-D array (float32, or uint16 holding bf16 bits).
     joint: the 2:4 estimator (JOINT_TABLE: App. A.2; JOINT_SYSTEMATIC; JOINT_APPROX: Sec. 4.4); ignored for 1:2.
+    stochastic_rounding: survivors are rounded to bf16 stochastically (unbiased storage) instead of to nearest.
 
     Returns (values uint16 [Mrows, K/2], meta uint8 [Mrows, K/8]) in canonical form.
     """
@@ -237,9 +253,10 @@ def prune(g: np.ndarray, n: int, m: int, axis: int, seed: int, *, k_total: int |
     k = cols if axis == 1 else rows
     values = np.zeros(vshape, dtype=np.uint16)
     meta = np.zeros(mshape, dtype=np.uint8)
-    rc = lib().oracle_prune(g.ctypes.data, int(g.dtype == np.uint16), rows, cols, cols, n, m, axis,
-                            seed & (2**64 - 1), k if k_total is None else k_total, k_offset,
-                            values.ctypes.data, meta.ctypes.data, max(1, threads), int(joint))
+    rc = lib().oracle_prune_rounded(g.ctypes.data, int(g.dtype == np.uint16), rows, cols, cols, n, m, axis,
+                                    seed & (2**64 - 1), k if k_total is None else k_total, k_offset,
+                                    values.ctypes.data, meta.ctypes.data, max(1, threads), int(joint),
+                                    int(bool(stochastic_rounding)))
     if rc != 0:
         raise ValueError("oracle_prune: unsupported N:M or shape")
     return values, meta

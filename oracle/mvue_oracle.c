@@ -118,6 +118,46 @@ float oracle_bf16_to_f32(uint16_t h)
 }
 
 /* ------------------------------------------------------------------------
+ * Stochastic rounding of a survivor to bf16 (Sec. 3 recalls that the neural
+ * gradients want an unbiased quantiser "such as stochastic rounding"; App.
+ * "Pruning Overhead" Part 1 names stochastic rounding as the sampling
+ * primitive).  With round-to-nearest the stored survivor is a_i / p_i only up
+ * to the bf16 grid, so E[stored] = a_i (1 + delta), |delta| <= 2^-9; rounding
+ * stochastically makes the stored value itself unbiased:
+ *     x lies between two neighbouring bf16 numbers lo <= x < hi (same sign);
+ *     store hi with probability (x - lo) / (hi - lo), else lo.
+ * On the bit pattern: the low 16 bits f of x are the numerator of that
+ * probability over 2^16, and adding r, a uniform 16-bit integer, carries into
+ * the upper half exactly when f + r >= 2^16, i.e. for f of the 2^16 values of r:
+ *     stored = (bits(x) + r) >> 16.
+ * A value already on the bf16 grid (f = 0) never moves; a carry out of the
+ * mantissa lands on the next power of two, which is the correct neighbour.
+ * Inputs are finite and below 2^127 in magnitude.
+ * ---------------------------------------------------------------------- */
+uint16_t oracle_bf16_sr(float x, uint16_t r)
+{
+    uint32_t bits;
+    memcpy(&bits, &x, 4);
+    return (uint16_t)((bits + (uint32_t)r) >> 16);
+}
+
+/* The 16 random bits that round survivor slot e (0..7) of unit number u (a unit
+ * is 16 consecutive elements along K: four blocks of four, or eight pairs; its
+ * eight survivors in packed order are the slots).  They come from a generator
+ * call of their own, counter (lo32(u), hi32(u), 1, 0) under the same key -- the
+ * selection draws all have third counter word 0 -- slot e taking the low (e even)
+ * or high (e odd) half of word e / 2. */
+uint16_t oracle_rounding_bits(uint64_t seed, uint64_t u, int e)
+{
+    uint32_t ctr[4] = { (uint32_t)u, (uint32_t)(u >> 32), 1u, 0u };
+    uint32_t key[2] = { (uint32_t)seed, (uint32_t)(seed >> 32) };
+    uint32_t out[4];
+    oracle_philox4x32_10(ctr, key, out);
+    uint32_t w = out[e >> 1];
+    return (uint16_t)((e & 1) ? (w >> 16) : (w & 0xFFFFu));
+}
+
+/* ------------------------------------------------------------------------
  * MVUE 1:2 (Sec. 4.1, the estimator that closes that section; derivation in
  * App. A.1): keep a_1 with probability |a_1| / (|a_1| + |a_2|), else a_2; the
  * survivor becomes sign(a_i) (|a_1| + |a_2|).  The draw is the threshold test
@@ -572,15 +612,32 @@ static float load_elem(const void *g, int is_bf16, int64_t off)
     return ((const float *)g)[off];
 }
 
+int oracle_prune_rounded(const void *g, int is_bf16, int64_t rows, int64_t cols, int64_t ld,
+                         int n, int m, int axis, uint64_t seed, int64_t k_total, int64_t k_offset,
+                         uint16_t *values, uint8_t *meta, int threads, int joint, int stochastic_rounding);
+
 int oracle_prune(const void *g, int is_bf16, int64_t rows, int64_t cols, int64_t ld,
                  int n, int m, int axis, uint64_t seed, int64_t k_total, int64_t k_offset,
                  uint16_t *values, uint8_t *meta, int threads, int joint)
+{
+    return oracle_prune_rounded(g, is_bf16, rows, cols, ld, n, m, axis, seed, k_total, k_offset, values, meta,
+                                threads, joint, 0);
+}
+
+/* The same with the rounding of the survivors chosen: stochastic_rounding = 0 rounds to the nearest bf16 (ties to
+ * even), 1 rounds stochastically (oracle_bf16_sr) with the bits of oracle_rounding_bits: the survivor stored at
+ * values[r][8 t + e] is slot e of unit number r (k_total / 16) + k_offset / 16 + t.  Needs K, k_total, k_offset
+ * multiples of 16 then. */
+int oracle_prune_rounded(const void *g, int is_bf16, int64_t rows, int64_t cols, int64_t ld,
+                         int n, int m, int axis, uint64_t seed, int64_t k_total, int64_t k_offset,
+                         uint16_t *values, uint8_t *meta, int threads, int joint, int stochastic_rounding)
 {
     const int64_t Mrows = axis == 1 ? rows : cols;
     const int64_t K     = axis == 1 ? cols : rows;
     if (!((n == 1 && m == 2) || (n == 2 && m == 4) || (n == 1 && m == 4))) return -1;
     if (K % 8 != 0 || k_total % 8 != 0 || k_offset % 8 != 0 || k_offset + K > k_total) return -1;
     if (joint < 0 || joint > 2) return -1;
+    if (stochastic_rounding && (K % 16 != 0 || k_total % 16 != 0 || k_offset % 16 != 0)) return -1;
     (void)threads;
 #pragma omp parallel for num_threads(threads) schedule(static)
     for (int64_t r = 0; r < Mrows; ++r) {
@@ -616,8 +673,15 @@ int oracle_prune(const void *g, int is_bf16, int64_t rows, int64_t cols, int64_t
                                                             oracle_block_word(seed, q), &val[half]);
                 }
             }
-            values[r * (K / 2) + 2 * j]     = oracle_bf16_rne(val[0]);
-            values[r * (K / 2) + 2 * j + 1] = oracle_bf16_rne(val[1]);
+            if (stochastic_rounding) {
+                uint64_t u = (uint64_t)r * (uint64_t)(k_total / 16) + (uint64_t)(k_offset / 16 + j / 4);
+                int slot = 2 * (int)(j % 4);
+                values[r * (K / 2) + 2 * j]     = oracle_bf16_sr(val[0], oracle_rounding_bits(seed, u, slot));
+                values[r * (K / 2) + 2 * j + 1] = oracle_bf16_sr(val[1], oracle_rounding_bits(seed, u, slot + 1));
+            } else {
+                values[r * (K / 2) + 2 * j]     = oracle_bf16_rne(val[0]);
+                values[r * (K / 2) + 2 * j + 1] = oracle_bf16_rne(val[1]);
+            }
             uint8_t nib = (uint8_t)(idx[0] | (idx[1] << 2));
             uint8_t *byte = &meta[r * (K / 8) + j / 2];
             if (j % 2 == 0) *byte = (uint8_t)((*byte & 0xF0u) | nib);
