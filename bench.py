@@ -346,12 +346,13 @@ def run_ours(args, cfg, n, m):
               "approx": binding.MVUE_JOINT_APPROX}
     joint = [joints[args.joint]]                        # cells, so that the other estimators can be timed with the same step
     nm = [(n, m)]
+    opts = [binding.MVUE_OPT_NONE]
 
     def step(i, ev=None):
         if ev:
             ev[0].record()
         binding.mvue_prune(g_dev, nm[0][0], nm[0][1], 0, i, k_total=k_total, k_offset=k_offset, values=values,
-                           meta=meta, layout=TC, joint=joint[0])
+                           meta=meta, layout=TC, joint=joint[0], options=opts[0])
         if ev:
             ev[1].record()
         binding.mvue_sparse_update_gemm(values, meta, h_dev, out=dW, workspace=ws, dev_status=status)
@@ -418,15 +419,17 @@ def run_ours(args, cfg, n, m):
     others = []
     if extras and m == 4:
         k2 = max(20, min(args.steps, 200))
-        variants = [(name, (2, 4), jid) for name, jid in joints.items() if name != args.joint]
-        variants += [("1:2", (1, 2), joints[args.joint]), ("1:4", (1, 4), joints[args.joint])]
-        for name, nm_v, jid in variants:
-            joint[0], nm[0] = jid, nm_v
+        variants = [(name, (2, 4), jid, 0) for name, jid in joints.items() if name != args.joint]
+        variants += [("1:2", (1, 2), joints[args.joint], 0), ("1:4", (1, 4), joints[args.joint], 0),
+                     # the step's law with the survivors rounded to bf16 stochastically (unbiased storage)
+                     ("stochastic_rounding", (2, 4), joints[args.joint], binding.MVUE_OPT_STOCHASTIC_ROUNDING)]
+        for name, nm_v, jid, opt in variants:
+            joint[0], nm[0], opts[0] = jid, nm_v, opt
             for i in range(3):
                 step(i)
             pt, _ = step_kernel_times(k2)
             others.append((name, float(np.mean(pt)), float(np.min(pt)), k2))
-        joint[0], nm[0] = joints[args.joint], (n, m)
+        joint[0], nm[0], opts[0] = joints[args.joint], (n, m), binding.MVUE_OPT_NONE
 
     # the step's prune timed alone (no product in between), L2-cold: inputs rotated over copies of g that together
     # exceed 2.5 x L2
@@ -660,6 +663,8 @@ def tensor_bound_case(tm: Timer, n, m, peaks, joint, issue_cold):
     sys_ms = tm.loop(prune_with((2, 4), binding.MVUE_JOINT_SYSTEMATIC), 20)
     table_ms = tm.loop(prune_with((2, 4), binding.MVUE_JOINT_TABLE), 20)
     one_two_ms = tm.loop(prune_with((1, 2), joint), 20)
+    sr_ms = tm.loop(lambda: binding.mvue_prune(g, n, m, 0, 1, values=values, meta=meta, layout=TC, joint=joint,
+                                               options=binding.MVUE_OPT_STOCHASTIC_ROUNDING), 20)
     prune_with((n, m), joint)()
     gemm_ms = tm.loop(lambda: binding.mvue_sparse_update_gemm(values, meta, h, out=dW, workspace=ws), 30)
     fused_ms = tm.loop(lambda: binding.mvue_fused_update_gemm(g, h, n, m, 1, out=dW), 3)
@@ -674,6 +679,8 @@ def tensor_bound_case(tm: Timer, n, m, peaks, joint, issue_cold):
             "prune_systematic_ms": sys_ms, "prune_systematic_frac_of_hbm_peak": pb / (sys_ms * 1e-3) / 1e9 / peaks["hbm_gbs"],
             "prune_table_ms": table_ms, "prune_table_frac_of_hbm_peak": pb / (table_ms * 1e-3) / 1e9 / peaks["hbm_gbs"],
             "prune_1of2_ms": one_two_ms, "prune_1of2_frac_of_hbm_peak": pb / (one_two_ms * 1e-3) / 1e9 / peaks["hbm_gbs"],
+            "prune_stochastic_rounding_ms": sr_ms,
+            "prune_stochastic_rounding_frac_of_hbm_peak": pb / (sr_ms * 1e-3) / 1e9 / peaks["hbm_gbs"],
             "gemm_ms": gemm_ms, "gemm_tflops_effective": tf,
             "sparse_issue_rate_cold_tflops": issue_cold, "sparse_issue_rate_after_products_tflops": issue_warm,
             "gemm_frac_of_issue_rate_after_products": tf / issue_warm,

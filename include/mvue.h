@@ -50,7 +50,8 @@ typedef enum {
     MVUE_ERR_ARCH = -8,           /* current device is not sm_100 */
     MVUE_ERR_CUDA = -9,           /* a CUDA runtime/driver call failed; text in mvue_last_cuda_error() */
     MVUE_ERR_DEVICE_TIMEOUT = -10,/* only ever written to a device status word: a bounded wait expired */
-    MVUE_ERR_JOINT = -11          /* unknown mvue_joint */
+    MVUE_ERR_JOINT = -11,         /* unknown mvue_joint */
+    MVUE_ERR_OPTION = -12         /* unknown bit in the options of mvue_prune_opts */
 } mvue_status;
 
 typedef enum { MVUE_F32 = 0, MVUE_BF16 = 1 } mvue_dtype;
@@ -165,6 +166,25 @@ MVUE_API int mvue_prune(const void* g, int dtype, int64_t rows, int64_t cols, in
 MVUE_API int mvue_prune_joint(const void* g, int dtype, int64_t rows, int64_t cols, int64_t ld, int n, int m,
                      int axis, uint64_t seed, int64_t k_total, int64_t k_offset, void* values,
                      void* meta, int layout, int joint, void* stream);
+
+/* mvue_prune_joint with options (a bitwise OR of mvue_prune_option; an unknown bit gives MVUE_ERR_OPTION).
+ *
+ * MVUE_OPT_STOCHASTIC_ROUNDING: the survivors are rounded to bf16 stochastically instead of to the nearest bf16
+ *   (Sec. 3: the neural gradients want an unbiased quantiser such as stochastic rounding; App. "Pruning Overhead",
+ *   Part 1, names stochastic rounding as the sampling primitive).  Round-to-nearest stores a_i / p_i only up to the
+ *   bf16 grid, E[stored] = a_i (1 + delta) with |delta| <= 2^-9; with this option the stored value itself is unbiased:
+ *   a binary32 survivor x between the neighbouring bf16 numbers lo <= |x| < hi is stored as hi with probability
+ *   (|x| - lo) / (hi - lo), else lo -- on the bit pattern, stored = (bits(x) + r) >> 16 with r a uniform 16-bit
+ *   integer.  Masks and metadata are those of the same call without the option; survivors already on the bf16 grid
+ *   (every survivor that keeps its own bf16 value) never move.  The bits r: unit u = r_A (k_total / 16) + k_offset / 16
+ *   + t (16 consecutive k of row r_A of A) makes one more generator call, Philox4x32-10 with counter
+ *   (lo32(u), hi32(u), 1, 0) under the same key (the selection draws all have third counter word 0); the survivor stored
+ *   at values[r_A][8 t + e] takes the low (e even) or high (e odd) half of word e / 2.  About 15 more instructions per
+ *   block of four. */
+typedef enum { MVUE_OPT_NONE = 0, MVUE_OPT_STOCHASTIC_ROUNDING = 1 } mvue_prune_option;
+MVUE_API int mvue_prune_opts(const void* g, int dtype, int64_t rows, int64_t cols, int64_t ld, int n, int m,
+                    int axis, uint64_t seed, int64_t k_total, int64_t k_offset, void* values,
+                    void* meta, int layout, int joint, unsigned options, void* stream);
 
 /* Expand a packed operand back to dense bf16 A[Mrows x K] (row-major, ld = K).
  * A checking aid: the inverse of the pack step, no arithmetic. */

@@ -18,9 +18,10 @@ MVUE_F32, MVUE_BF16 = 0, 1
 MVUE_LAYOUT_CANONICAL = 0
 MVUE_LAYOUT_TC = 1
 MVUE_JOINT_TABLE, MVUE_JOINT_SYSTEMATIC, MVUE_JOINT_APPROX = 0, 1, 2
+MVUE_OPT_NONE, MVUE_OPT_STOCHASTIC_ROUNDING = 0, 1
 
 EXPORTS = ("mvue_version", "mvue_status_string", "mvue_last_cuda_error", "mvue_packed_sizes",
-           "mvue_prune", "mvue_prune_joint", "mvue_unpack", "mvue_sparse_update_gemm", "mvue_sparse_backward_gemm",
+           "mvue_prune", "mvue_prune_joint", "mvue_prune_opts", "mvue_unpack", "mvue_sparse_update_gemm", "mvue_sparse_backward_gemm",
            "mvue_gemm_workspace_bytes", "mvue_sparse_update_gemm_noalloc", "mvue_fused_update_gemm",
            "mvue_probe_sparse_mma", "mvue_selftest_wait_timeout")
 
@@ -51,6 +52,7 @@ def lib() -> ctypes.CDLL:
         L.mvue_packed_sizes.argtypes = [i64, i64, ci, ci, ci, ci, szp, szp]
         L.mvue_prune.argtypes = [vp, ci, i64, i64, i64, ci, ci, ci, u64, i64, i64, vp, vp, ci, vp]
         L.mvue_prune_joint.argtypes = [vp, ci, i64, i64, i64, ci, ci, ci, u64, i64, i64, vp, vp, ci, ci, vp]
+        L.mvue_prune_opts.argtypes = [vp, ci, i64, i64, i64, ci, ci, ci, u64, i64, i64, vp, vp, ci, ci, ctypes.c_uint, vp]
         L.mvue_unpack.argtypes = [vp, vp, ci, i64, i64, vp, vp]
         L.mvue_sparse_update_gemm.argtypes = [vp, vp, ci, i64, i64, vp, i64, i64, vp, ci, i64, ci, vp,
                                               ctypes.c_size_t, vp, vp]
@@ -92,10 +94,11 @@ def mvue_packed_sizes(rows: int, cols: int, n: int, m: int, axis: int, layout: i
 
 def mvue_prune(g: torch.Tensor, n: int, m: int, axis: int, seed: int, *, k_total: int | None = None,
                k_offset: int = 0, values: torch.Tensor | None = None, meta: torch.Tensor | None = None,
-               layout: int = MVUE_LAYOUT_CANONICAL, joint: int | None = None):
+               layout: int = MVUE_LAYOUT_CANONICAL, joint: int | None = None, options: int = MVUE_OPT_NONE):
     """MVUE n:m prune + pack of a 2-D CUDA tensor g (fp32 or bf16, unit column stride).
 
     joint: None calls mvue_prune (App. A.2 pair table); an mvue_joint value calls mvue_prune_joint.
+    options: non-zero calls mvue_prune_opts (MVUE_OPT_STOCHASTIC_ROUNDING: unbiased bf16 storage of the survivors).
     Returns (values bf16 [Mrows, K/2], meta uint8 [Mrows, K/8]).
     """
     assert g.is_cuda and g.dim() == 2 and g.stride(1) == 1
@@ -105,7 +108,13 @@ def mvue_prune(g: torch.Tensor, n: int, m: int, axis: int, seed: int, *, k_total
         _, meta_bytes = mvue_packed_sizes(rows, cols, n, m, axis, layout)   # validates before allocating
         values = torch.empty((mrows, k // 2), dtype=torch.bfloat16, device=g.device)
         meta = torch.empty((meta_bytes // (k // 8), k // 8), dtype=torch.uint8, device=g.device)
-    if joint is None:
+    if options:
+        _check(lib().mvue_prune_opts(g.data_ptr(), _dtype_code(g), rows, cols, g.stride(0), n, m, axis,
+                                     seed & (2**64 - 1), k if k_total is None else k_total, k_offset,
+                                     values.data_ptr(), meta.data_ptr(), layout,
+                                     MVUE_JOINT_TABLE if joint is None else int(joint), int(options), _stream_ptr()),
+               "mvue_prune_opts")
+    elif joint is None:
         _check(lib().mvue_prune(g.data_ptr(), _dtype_code(g), rows, cols, g.stride(0), n, m, axis,
                                 seed & (2**64 - 1), k if k_total is None else k_total, k_offset,
                                 values.data_ptr(), meta.data_ptr(), layout, _stream_ptr()), "mvue_prune")

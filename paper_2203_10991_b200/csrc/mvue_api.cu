@@ -84,7 +84,7 @@ using namespace mvue;
 
 extern "C" {
 
-int mvue_version(void) { return 120; }   // 1.2: per-device set-up, the bounded-wait self-test
+int mvue_version(void) { return 130; }   // 1.3: stochastic rounding of survivors, per-device set-up, the bounded-wait self-test
 
 const char* mvue_status_string(int status) {
     switch (status) {
@@ -100,6 +100,7 @@ const char* mvue_status_string(int status) {
         case MVUE_ERR_CUDA: return "CUDA call failed (see mvue_last_cuda_error)";
         case MVUE_ERR_DEVICE_TIMEOUT: return "a bounded device-side wait expired";
         case MVUE_ERR_JOINT: return "unknown 2:4 estimator (App. A.2 table, systematic sampling or approx-MVUE)";
+        case MVUE_ERR_OPTION: return "unknown prune option bit";
         default: return "unknown status";
     }
 }
@@ -132,7 +133,15 @@ int mvue_prune(const void* g, int dtype, int64_t rows, int64_t cols, int64_t ld,
 int mvue_prune_joint(const void* g, int dtype, int64_t rows, int64_t cols, int64_t ld, int n, int m,
                      int axis, uint64_t seed, int64_t k_total, int64_t k_offset, void* values,
                      void* meta, int layout, int joint, void* stream) {
+    return mvue_prune_opts(g, dtype, rows, cols, ld, n, m, axis, seed, k_total, k_offset, values, meta, layout, joint,
+                           MVUE_OPT_NONE, stream);
+}
+
+int mvue_prune_opts(const void* g, int dtype, int64_t rows, int64_t cols, int64_t ld, int n, int m,
+                    int axis, uint64_t seed, int64_t k_total, int64_t k_offset, void* values,
+                    void* meta, int layout, int joint, unsigned options, void* stream) {
     if (!g || !values || !meta) return MVUE_ERR_NULL;
+    if (options & ~(unsigned)MVUE_OPT_STOCHASTIC_ROUNDING) return MVUE_ERR_OPTION;
     if (joint != MVUE_JOINT_TABLE && joint != MVUE_JOINT_SYSTEMATIC && joint != MVUE_JOINT_APPROX) return MVUE_ERR_JOINT;
     if (dtype != MVUE_F32 && dtype != MVUE_BF16) return MVUE_ERR_DTYPE;
     if (int s = mvue_packed_sizes(rows, cols, n, m, axis, layout, nullptr, nullptr)) return s;
@@ -146,7 +155,8 @@ int mvue_prune_joint(const void* g, int dtype, int64_t rows, int64_t cols, int64
     DeviceInfo dev;
     if (int s = current_device_info(&dev)) return s;
     PruneArgs a{g, dtype == MVUE_BF16, rows, cols, ld, m, axis, seed, k_total, k_offset, values, meta, dev.sm_count,
-                layout == MVUE_LAYOUT_TC, (n == 1 && m == 4) ? 3 : joint};     // one survivor of four has a single law
+                layout == MVUE_LAYOUT_TC, (n == 1 && m == 4) ? 3 : joint,      // one survivor of four has a single law
+                (options & MVUE_OPT_STOCHASTIC_ROUNDING) != 0};
     cudaError_t e = launch_prune(a, reinterpret_cast<cudaStream_t>(stream));
     if (e != cudaSuccess) { set_cuda_error(e, "mvue_prune launch"); return MVUE_ERR_CUDA; }
     return MVUE_OK;

@@ -38,9 +38,10 @@ __host__ inline RoundKeys make_round_keys(uint64_t seed) {
     return rk;
 }
 
-// Words of generator call number `call` (counter = (lo, hi, 0, 0)).
-__device__ __forceinline__ uint4 philox4x32_10(uint64_t call, const RoundKeys& rk) {
-    uint32_t c0 = (uint32_t)call, c1 = (uint32_t)(call >> 32), c2 = 0u, c3 = 0u;
+// Words of generator call number `call` (counter = (lo, hi, stream, 0); the selection draws use stream 0, the
+// rounding bits of the survivors stream 1).
+__device__ __forceinline__ uint4 philox4x32_10(uint64_t call, const RoundKeys& rk, uint32_t stream = 0u) {
+    uint32_t c0 = (uint32_t)call, c1 = (uint32_t)(call >> 32), c2 = stream, c3 = 0u;
 #pragma unroll
     for (int r = 0; r < 10; ++r) {
         const uint64_t p0 = (uint64_t)0xD2511F53u * (uint64_t)c0;
@@ -66,6 +67,16 @@ __device__ __forceinline__ uint32_t pack_bf16x2(float lo, float hi) {
     return *reinterpret_cast<uint32_t*>(&p);
 }
 
+// Two binary32 survivors -> one word of two bf16 (lo first): to nearest even, or (kSR) stochastically -- the low 16 bits
+// of a survivor are the probability, over 2^16, of its upper bf16 neighbour, and adding the slot's 16 random bits
+// (rnd = bits of the low slot | bits of the high slot << 16) carries into the upper half exactly that often:
+// stored = (bits + r) >> 16, whose expectation over r is the survivor itself.
+template <bool kSR>
+__device__ __forceinline__ uint32_t pack_out(float lo, float hi, uint32_t rnd) {
+    if (!kSR) return pack_bf16x2(lo, hi);
+    return __byte_perm(__float_as_uint(lo) + (rnd & 0xFFFFu), __float_as_uint(hi) + (rnd >> 16), 0x7632u);
+}
+
 // ===========================================================================
 // MVUE 1:2 (Sec. 4.1): keep a_1 iff eps (|a_1|+|a_2|) < |a_1| (or a_2 = 0); the
 // survivor becomes sign(a_i)(|a_1|+|a_2|).
@@ -85,8 +96,9 @@ __device__ __forceinline__ bool mvue_1of2(float f0, float f1, uint32_t word, flo
 // Two adjacent bf16 pairs (one group of four): x0 = a0 | a1 << 16, x1 = a2 | a3 << 16.
 // Outputs the group's two survivors as bf16 (pair 0 in the low half) and its nibble
 // (pair 0 -> position 0/1, pair 1 -> position 2/3).
+template <bool kSR = false>
 __device__ __forceinline__ void mvue_1of2x2_bf16(uint32_t x0, uint32_t x1, uint32_t word0,
-                                                 uint32_t word1, uint32_t* out, uint32_t* nibble) {
+                                                 uint32_t word1, uint32_t* out, uint32_t* nibble, uint32_t rnd = 0u) {
     const float a0 = __uint_as_float(x0 << 16), a1 = __uint_as_float(x0 & 0xFFFF0000u);
     const float b0 = __uint_as_float(x1 << 16), b1 = __uint_as_float(x1 & 0xFFFF0000u);
     const float SA = __fadd_rn(fabsf(a0), fabsf(a1));
@@ -98,7 +110,7 @@ __device__ __forceinline__ void mvue_1of2x2_bf16(uint32_t x0, uint32_t x1, uint3
     // byte 1 <- high byte of the survivor of pair 0, byte 3 <- high byte of the survivor of pair 1
     const uint32_t sel = (keepA ? 0x0010u : 0x0030u) | (keepB ? 0x5000u : 0x7000u);
     const uint32_t signs = __byte_perm(x0, x1, sel) & 0x80008000u;
-    *out = pack_bf16x2(SA, SB) | signs;
+    *out = pack_out<kSR>(SA, SB, rnd) | signs;
     *nibble = (keepA ? 0u : 1u) | (keepB ? 8u : 12u);
 }
 
@@ -187,9 +199,9 @@ __device__ __forceinline__ Pick24<KeyT> pick_2of4(KeyT k1, KeyT k2, KeyT k3, Key
 // `nibble` = idx0 | idx1 << 2.
 // The four elements are the halves (kH* = false: low, true: high) of the words w0..w3: adjacent pairs of two
 // words when K is contiguous (w0 = w1, w2 = w3), or the same half of four row words when K runs down the rows.
-template <bool kH0, bool kH1, bool kH2, bool kH3>
+template <bool kH0, bool kH1, bool kH2, bool kH3, bool kSR = false>
 __device__ __forceinline__ void mvue_2of4_bf16(uint32_t w0, uint32_t w1, uint32_t w2, uint32_t w3, uint32_t word,
-                                               uint32_t* out, uint32_t* nibble) {
+                                               uint32_t* out, uint32_t* nibble, uint32_t rnd = 0u) {
     const float f0 = __uint_as_float(__byte_perm(w0, 0x00u, kH0 ? 0x3243 : 0x1041));
     const float f1 = __uint_as_float(__byte_perm(w1, 0x40u, kH1 ? 0x3243 : 0x1041));
     const float f2 = __uint_as_float(__byte_perm(w2, 0x80u, kH2 ? 0x3243 : 0x1041));
@@ -206,9 +218,10 @@ __device__ __forceinline__ void mvue_2of4_bf16(uint32_t w0, uint32_t w1, uint32_
 
     const uint32_t ua = __float_as_uint(r.key_a), ub = __float_as_uint(r.key_b);
     const uint32_t signs = __byte_perm(ua, ub, 0x4000) & 0x80008000u;   // byte 1 <- a's sign byte, byte 3 <- b's
-    const uint32_t ab = pack_bf16x2(r.va, r.vb) | signs;                // a low, b high
     const uint32_t pa = ua << 16, pb = ub << 16;                        // position in the top two bits
     const bool swap = pa > pb;
+    // (the rounding bits belong to the slots: when a ends up in the high slot it takes the high slot's bits)
+    const uint32_t ab = pack_out<kSR>(r.va, r.vb, kSR ? __byte_perm(rnd, 0u, swap ? 0x1032u : 0x3210u) : 0u) | signs;   // a low, b high
     *out = __byte_perm(ab, 0u, swap ? 0x1032u : 0x3210u);
     // (p >> 30) and (p >> 28) as high products: bits 29..28 of p are zero, so p >> 28 = position << 2
     const uint32_t nib_ab = __umulhi(pa, 4u) + __umulhi(pb, 16u);
@@ -218,8 +231,9 @@ __device__ __forceinline__ void mvue_2of4_bf16(uint32_t w0, uint32_t w1, uint32_
 
 // ---- binary32 source ---------------------------------------------------------
 // 64-bit keys (magnitude bits << 2 | position); b0..b3 are the raw bit patterns.
+template <bool kSR = false>
 __device__ __forceinline__ void mvue_2of4_f32(uint32_t b0, uint32_t b1, uint32_t b2, uint32_t b3,
-                                              uint32_t word, uint32_t* out, uint32_t* nibble) {
+                                              uint32_t word, uint32_t* out, uint32_t* nibble, uint32_t rnd = 0u) {
     auto make = [](uint32_t b, uint32_t p) { return ((uint64_t)(b & 0x7FFFFFFFu) << 2) | p; };
     auto cswap = [](uint64_t& a, uint64_t& b) {
         const uint64_t lo = a < b ? a : b, hi = a < b ? b : a;
@@ -236,7 +250,7 @@ __device__ __forceinline__ void mvue_2of4_f32(uint32_t b0, uint32_t b1, uint32_t
     const float va = __uint_as_float(__float_as_uint(r.va) | sa);
     const float vb = __uint_as_float(__float_as_uint(r.vb) | sb);
     const bool swap = ia > ib;
-    *out = swap ? pack_bf16x2(vb, va) : pack_bf16x2(va, vb);
+    *out = pack_out<kSR>(swap ? vb : va, swap ? va : vb, rnd);
     *nibble = swap ? (ib | (ia << 2)) : (ia | (ib << 2));
 }
 
@@ -289,14 +303,17 @@ __device__ __forceinline__ Pick24Sys pick_2of4_sys(float m0, float m1, float m2,
 // permute (selector bytes 2i, 2i+1, 2j, 2j+1); bf16 rounding is monotone, so the rounded max(|a|, H)
 // is the larger of the element's own bits and the rounded H, taken on both halves at once as
 // signed 16-bit integers (with equal sign bits the larger magnitude is the larger integer).
+template <bool kSR = false>
 __device__ __forceinline__ void mvue_2of4_sys_bf16(uint32_t x01, uint32_t x23, uint32_t word, uint32_t* out,
-                                                   uint32_t* nibble) {
+                                                   uint32_t* nibble, uint32_t rnd = 0u) {
     const Pick24Sys r = pick_2of4_sys<false>(fabsf(__uint_as_float(x01 << 16)), fabsf(__uint_as_float(x01 & 0xFFFF0000u)),
                                              fabsf(__uint_as_float(x23 << 16)), fabsf(__uint_as_float(x23 & 0xFFFF0000u)),
                                              word);
     const uint32_t sel = 0x7654u - 0x22u * r.li - 0x2200u * r.lj;
     const uint32_t raw = __byte_perm(x01, x23, sel);
-    const uint32_t hs = pack_bf16x2(r.H, r.H) | (raw & 0x80008000u);
+    // (a survivor below H takes H rounded for its own slot; one at or above H is a bf16 number no smaller than either
+    // neighbour of H, so the maximum still picks it)
+    const uint32_t hs = pack_out<kSR>(r.H, r.H, rnd) | (raw & 0x80008000u);
     *out = __vmaxs2(raw, hs);
     *nibble = 14u - r.li - 4u * r.lj;                                         // i | j << 2
 }
@@ -326,9 +343,11 @@ __device__ __forceinline__ uint64_t sub_f32x2(uint64_t a, uint64_t b) {
 }
 
 // Blocks A = (xa01, xa23; word wa) and B = (xb01, xb23; word wb), each as in mvue_2of4_sys_bf16.
+template <bool kSR = false>
 __device__ __forceinline__ void mvue_2of4_sys_bf16_x2(uint32_t xa01, uint32_t xa23, uint32_t xb01, uint32_t xb23,
                                                       uint32_t wa, uint32_t wb, uint32_t* out_a, uint32_t* out_b,
-                                                      uint32_t* nibble_a, uint32_t* nibble_b) {
+                                                      uint32_t* nibble_a, uint32_t* nibble_b, uint32_t rnd_a = 0u,
+                                                      uint32_t rnd_b = 0u) {
     // magnitudes: both sign bits of a word cleared at once, then widened
     const uint32_t ya01 = xa01 & 0x7FFF7FFFu, ya23 = xa23 & 0x7FFF7FFFu, yb01 = xb01 & 0x7FFF7FFFu, yb23 = xb23 & 0x7FFF7FFFu;
     const float a0 = __uint_as_float(ya01 << 16), a1 = __uint_as_float(ya01 & 0xFFFF0000u);
@@ -358,27 +377,28 @@ __device__ __forceinline__ void mvue_2of4_sys_bf16_x2(uint32_t xa01, uint32_t xa
     {
         const uint32_t li = sign(d1a) + sign(d2a), lj = min(sign(d3a) + sign(d4a), li);
         const uint32_t raw = __byte_perm(xa01, xa23, 0x7654u - 0x22u * li - 0x2200u * lj);
-        *out_a = __vmaxs2(raw, pack_bf16x2(Ha, Ha) | (raw & 0x80008000u));
+        *out_a = __vmaxs2(raw, pack_out<kSR>(Ha, Ha, rnd_a) | (raw & 0x80008000u));
         *nibble_a = 14u - li - 4u * lj;
     }
     {
         const uint32_t li = sign(d1b) + sign(d2b), lj = min(sign(d3b) + sign(d4b), li);
         const uint32_t raw = __byte_perm(xb01, xb23, 0x7654u - 0x22u * li - 0x2200u * lj);
-        *out_b = __vmaxs2(raw, pack_bf16x2(Hb, Hb) | (raw & 0x80008000u));
+        *out_b = __vmaxs2(raw, pack_out<kSR>(Hb, Hb, rnd_b) | (raw & 0x80008000u));
         *nibble_b = 14u - li - 4u * lj;
     }
 }
 
 // binary32 source: b0..b3 are the raw bit patterns.
+template <bool kSR = false>
 __device__ __forceinline__ void mvue_2of4_sys_f32(uint32_t b0, uint32_t b1, uint32_t b2, uint32_t b3,
-                                                  uint32_t word, uint32_t* out, uint32_t* nibble) {
+                                                  uint32_t word, uint32_t* out, uint32_t* nibble, uint32_t rnd = 0u) {
     const Pick24Sys r = pick_2of4_sys<true>(fabsf(__uint_as_float(b0)), fabsf(__uint_as_float(b1)),
                                             fabsf(__uint_as_float(b2)), fabsf(__uint_as_float(b3)), word);
     const uint32_t bi = r.li == 2u ? b0 : (r.li == 1u ? b1 : b2);            // i = 2 - li in {0, 1, 2}
     const uint32_t bj = r.lj == 2u ? b1 : (r.lj == 1u ? b2 : b3);            // j = 3 - lj in {1, 2, 3}
     const float vi = __uint_as_float(__float_as_uint(fmaxf(fabsf(__uint_as_float(bi)), r.H)) | (bi & 0x80000000u));
     const float vj = __uint_as_float(__float_as_uint(fmaxf(fabsf(__uint_as_float(bj)), r.H)) | (bj & 0x80000000u));
-    *out = pack_bf16x2(vi, vj);
+    *out = pack_out<kSR>(vi, vj, rnd);
     *nibble = 14u - r.li - 4u * r.lj;
 }
 
@@ -403,9 +423,10 @@ __device__ __forceinline__ float sel4(uint32_t k, float x0, float x1, float x2, 
 
 // b0..b3: the block as binary32 bit patterns.  out = the two survivors as bf16 (lower position in the
 // low half), nibble = idx0 | idx1 << 2.
+template <bool kSR = false>
 __device__ __forceinline__ void mvue_2of4_approx_f32(uint32_t b0, uint32_t b1, uint32_t b2, uint32_t b3,
                                                      uint32_t word1, uint32_t word2, uint32_t* out,
-                                                     uint32_t* nibble) {
+                                                     uint32_t* nibble, uint32_t rnd = 0u) {
     const float m0 = fabsf(__uint_as_float(b0)), m1 = fabsf(__uint_as_float(b1));
     const float m2 = fabsf(__uint_as_float(b2)), m3 = fabsf(__uint_as_float(b3));
     const float q01 = __fadd_rn(m0, m1), q12 = __fadd_rn(m1, m2), q02 = __fadd_rn(m0, m2);
@@ -441,14 +462,15 @@ __device__ __forceinline__ void mvue_2of4_approx_f32(uint32_t b0, uint32_t b1, u
     const uint32_t bhi = hi < 2u ? (hi == 0u ? b0 : b1) : (hi == 2u ? b2 : b3);
     const float vlo = __uint_as_float(__float_as_uint(mag_lo) | (blo & 0x80000000u));
     const float vhi = __uint_as_float(__float_as_uint(mag_hi) | (bhi & 0x80000000u));
-    *out = pack_bf16x2(vlo, vhi);
+    *out = pack_out<kSR>(vlo, vhi, rnd);
     *nibble = lo | (hi << 2);
 }
 
 // bf16 source: x01 = a0 | a1 << 16, x23 = a2 | a3 << 16 (widened exactly).
+template <bool kSR = false>
 __device__ __forceinline__ void mvue_2of4_approx_bf16(uint32_t x01, uint32_t x23, uint32_t word1, uint32_t word2,
-                                                      uint32_t* out, uint32_t* nibble) {
-    mvue_2of4_approx_f32(x01 << 16, x01 & 0xFFFF0000u, x23 << 16, x23 & 0xFFFF0000u, word1, word2, out, nibble);
+                                                      uint32_t* out, uint32_t* nibble, uint32_t rnd = 0u) {
+    mvue_2of4_approx_f32<kSR>(x01 << 16, x01 & 0xFFFF0000u, x23 << 16, x23 & 0xFFFF0000u, word1, word2, out, nibble, rnd);
 }
 
 // ===========================================================================
@@ -457,8 +479,9 @@ __device__ __forceinline__ void mvue_2of4_approx_bf16(uint32_t x01, uint32_t x23
 //   c_1 = m_0, c_2 = c_1 + m_1, c_3 = c_2 + m_2, S = c_3 + m_3;  t = n (S 2^-24);  i = #{c_k <= t}.
 // The survivor is stored in the 2:4 container beside a +0: positions (i, 3), or (2, 3) when i = 3.
 // ===========================================================================
+template <bool kSR = false>
 __device__ __forceinline__ void mvue_1of4_f32(uint32_t b0, uint32_t b1, uint32_t b2, uint32_t b3, uint32_t word,
-                                              uint32_t* out, uint32_t* nibble) {
+                                              uint32_t* out, uint32_t* nibble, uint32_t rnd = 0u) {
     const float m0 = fabsf(__uint_as_float(b0)), m1 = fabsf(__uint_as_float(b1));
     const float m2 = fabsf(__uint_as_float(b2)), m3 = fabsf(__uint_as_float(b3));
     const float c2 = __fadd_rn(m0, m1), c3 = __fadd_rn(c2, m2), S = __fadd_rn(c3, m3);
@@ -466,28 +489,39 @@ __device__ __forceinline__ void mvue_1of4_f32(uint32_t b0, uint32_t b1, uint32_t
     const uint32_t i = (m0 <= t ? 1u : 0u) + (c2 <= t ? 1u : 0u) + (c3 <= t ? 1u : 0u);
     const uint32_t bi = i < 2u ? (i == 0u ? b0 : b1) : (i == 2u ? b2 : b3);
     const float v = __uint_as_float(__float_as_uint(S) | (bi & 0x80000000u));
-    const uint32_t h = pack_bf16x2(v, 0.0f);                 // survivor in the low half, +0 in the high half
-    *out = i < 3u ? h : h << 16;
+    if (kSR) {                                               // the survivor takes the rounding bits of the slot it lands in
+        *out = pack_out<true>(i < 3u ? v : 0.0f, i < 3u ? 0.0f : v, rnd);
+    } else {
+        const uint32_t h = pack_bf16x2(v, 0.0f);             // survivor in the low half, +0 in the high half
+        *out = i < 3u ? h : h << 16;
+    }
     *nibble = i < 3u ? (i | 12u) : 14u;
 }
 
 // One work unit of bf16 input: raw[8] = 16 elements along K, two per word.
 // kJoint selects the 2:4 estimator (0: App. A.2 table, 1: systematic sampling, 2: approx-MVUE of Sec. 4.4,
 // which takes two words per block: one generator call per two blocks) or, with 3, MVUE 1:4; 1:2 has one law.
-template <int M, int kJoint = 0>
+// kSR: survivors are rounded to bf16 stochastically; the unit's eight slots draw their 16 bits each from one more
+// generator call, numbered by the unit itself on stream 1 (group j's two slots: word j).
+template <int M, int kJoint = 0, bool kSR = false>
 __device__ __forceinline__ void prune_unit_bf16(const uint32_t (&raw)[8], uint64_t unit_index,
                                                 const RoundKeys& rk, uint4* out_values,
                                                 uint32_t* out_meta) {
     uint32_t v[4];                                   // 8 survivors, two bf16 per word
     uint32_t meta = 0;
+    uint32_t rnd[4] = {0u, 0u, 0u, 0u};
+    if (kSR) {
+        const uint4 r = philox4x32_10(unit_index, rk, 1u);
+        rnd[0] = r.x; rnd[1] = r.y; rnd[2] = r.z; rnd[3] = r.w;
+    }
     if (M == 4 && kJoint == 3) {                      // MVUE 1:4: one word per block, as for 2:4
         const uint4 w = philox4x32_10(unit_index, rk);
         const uint32_t words[4] = {w.x, w.y, w.z, w.w};
 #pragma unroll
         for (int j = 0; j < 4; ++j) {
             uint32_t nib;
-            mvue_1of4_f32(raw[2 * j] << 16, raw[2 * j] & 0xFFFF0000u, raw[2 * j + 1] << 16, raw[2 * j + 1] & 0xFFFF0000u,
-                          words[j], &v[j], &nib);
+            mvue_1of4_f32<kSR>(raw[2 * j] << 16, raw[2 * j] & 0xFFFF0000u, raw[2 * j + 1] << 16, raw[2 * j + 1] & 0xFFFF0000u,
+                               words[j], &v[j], &nib, rnd[j]);
             meta += nib << (4 * j);
         }
     } else if (M == 4 && kJoint == 2) {
@@ -497,14 +531,14 @@ __device__ __forceinline__ void prune_unit_bf16(const uint32_t (&raw)[8], uint64
 #pragma unroll
         for (int j = 0; j < 4; ++j) {
             uint32_t nib;
-            mvue_2of4_approx_bf16(raw[2 * j], raw[2 * j + 1], words[2 * j], words[2 * j + 1], &v[j], &nib);
+            mvue_2of4_approx_bf16<kSR>(raw[2 * j], raw[2 * j + 1], words[2 * j], words[2 * j + 1], &v[j], &nib, rnd[j]);
             meta += nib << (4 * j);
         }
     } else if (M == 4 && kJoint == 1) {                // systematic sampling: the unit's four blocks two at a time
         const uint4 w = philox4x32_10(unit_index, rk);
         uint32_t nib[4];
-        mvue_2of4_sys_bf16_x2(raw[0], raw[1], raw[2], raw[3], w.x, w.y, &v[0], &v[1], &nib[0], &nib[1]);
-        mvue_2of4_sys_bf16_x2(raw[4], raw[5], raw[6], raw[7], w.z, w.w, &v[2], &v[3], &nib[2], &nib[3]);
+        mvue_2of4_sys_bf16_x2<kSR>(raw[0], raw[1], raw[2], raw[3], w.x, w.y, &v[0], &v[1], &nib[0], &nib[1], rnd[0], rnd[1]);
+        mvue_2of4_sys_bf16_x2<kSR>(raw[4], raw[5], raw[6], raw[7], w.z, w.w, &v[2], &v[3], &nib[2], &nib[3], rnd[2], rnd[3]);
         meta = nib[0] + (nib[1] << 4) + (nib[2] << 8) + (nib[3] << 12);
     } else if (M == 4) {
         const uint4 w = philox4x32_10(unit_index, rk);
@@ -512,8 +546,8 @@ __device__ __forceinline__ void prune_unit_bf16(const uint32_t (&raw)[8], uint64
 #pragma unroll
         for (int j = 0; j < 4; ++j) {
             uint32_t nib;
-            mvue_2of4_bf16<false, true, false, true>(raw[2 * j], raw[2 * j], raw[2 * j + 1], raw[2 * j + 1],
-                                                     words[j], &v[j], &nib);
+            mvue_2of4_bf16<false, true, false, true, kSR>(raw[2 * j], raw[2 * j], raw[2 * j + 1], raw[2 * j + 1],
+                                                          words[j], &v[j], &nib, rnd[j]);
             meta += nib << (4 * j);
         }
     } else {
@@ -523,7 +557,7 @@ __device__ __forceinline__ void prune_unit_bf16(const uint32_t (&raw)[8], uint64
 #pragma unroll
         for (int j = 0; j < 4; ++j) {
             uint32_t nib;
-            mvue_1of2x2_bf16(raw[2 * j], raw[2 * j + 1], words[2 * j], words[2 * j + 1], &v[j], &nib);
+            mvue_1of2x2_bf16<kSR>(raw[2 * j], raw[2 * j + 1], words[2 * j], words[2 * j + 1], &v[j], &nib, rnd[j]);
             meta += nib << (4 * j);
         }
     }
