@@ -54,6 +54,26 @@ def test_bench_workload_full_size(name, n, m, check_rows):
             w = oracle.gemm_entry(A_rows[i_r], h, j)
             scale = float(np.abs(A_rows[i_r]).sum()) * 3.0
             assert abs(got[r, j] - w) <= 1e-5 * scale + 1e-4 * abs(w), (r, j, got[r, j], w)
+    if n_out * n_in >= 1 << 24:
+        # an output of hundreds of tiles (persistent walk in bands, last round cut along K): the whole first 256-row
+        # tile and the whole last one -- the last tiles in tile order are the ones a partly filled round splits --
+        # on the first and the last 64 columns, and 500 entries scattered over the whole output
+        for r0 in (0, n_out - 256):
+            block = list(range(r0, r0 + 256))
+            A_blk = oracle.unpack(np.ascontiguousarray(v_ref[block]), np.ascontiguousarray(m_ref[block]))
+            for c0 in (0, n_in - 64):
+                want = oracle.gemm(A_blk, np.ascontiguousarray(h[:, c0:c0 + 64]), threads=th)
+                err = np.linalg.norm(got[r0:r0 + 256, c0:c0 + 64] - want) / np.linalg.norm(want)
+                assert err <= 5e-5, (r0, c0, err)
+                assert np.abs(got[r0:r0 + 256, c0:c0 + 64] - want).max() <= 1e-3 * np.abs(want).max(), (r0, c0)
+        cache = {}
+        for r, j in zip(rng.integers(0, n_out, 500), rng.integers(0, n_in, 500)):
+            r, j = int(r), int(j)
+            if r not in cache:
+                cache[r] = oracle.unpack(np.ascontiguousarray(v_ref[r:r + 1]), np.ascontiguousarray(m_ref[r:r + 1]))[0]
+            w = oracle.gemm_entry(cache[r], h, j)
+            scale = float(np.abs(cache[r]).sum()) * 3.0
+            assert abs(got[r, j] - w) <= 1e-5 * scale + 1e-4 * abs(w), (r, j, got[r, j], w)
 
 
 def test_mlp_stack_block_full_size():

@@ -36,8 +36,18 @@ def _worker(rank, world, port, q):
     v, m = oracle.prune(np.ascontiguousarray(g[off:off + n]), 2, 4, axis=0, seed=SEED, k_total=T, k_offset=off)
     part = torch.from_numpy(oracle.gemm(oracle.unpack(v, m), h[off:off + n]))
     dist.all_reduce(part)
+    # the same shard arguments through the library's own argument checks (no GPU here: a valid call stops at the
+    # device lookup, -8 or -9; a shard that sticks out of the global K, or is off the 16-row grid, is refused as a
+    # shape error before that)
+    import ctypes
+    from paper_2203_10991_b200 import binding
+    L = binding.lib()
+    fake = ctypes.c_void_p(1 << 20)
+    codes = (L.mvue_prune_joint(fake, 1, n, OUT, OUT, 2, 4, 0, SEED, T, off, fake, fake, 1, 1, None),
+             L.mvue_prune_joint(fake, 1, n, OUT, OUT, 2, 4, 0, SEED, T, T - n + 128, fake, fake, 1, 1, None),
+             L.mvue_prune_joint(fake, 1, n, OUT, OUT, 2, 4, 0, SEED, T, off + 8, fake, fake, 1, 1, None))
     if rank == 0:
-        q.put((part.numpy(), off, n))
+        q.put((part.numpy(), off, n, codes))
     dist.destroy_process_group()
 
 
@@ -49,7 +59,7 @@ def test_two_rank_token_shards_sum_to_the_unsharded_update():
     procs = [ctx.Process(target=_worker, args=(r, world, port, q)) for r in range(world)]
     for p in procs:
         p.start()
-    got, off0, n0 = q.get(timeout=120)
+    got, off0, n0, codes = q.get(timeout=120)
     for p in procs:
         p.join(timeout=60)
         assert p.exitcode == 0
@@ -59,6 +69,9 @@ def test_two_rank_token_shards_sum_to_the_unsharded_update():
     want = oracle.gemm(oracle.unpack(v, m), h)
     assert np.allclose(got, want, rtol=1e-12, atol=1e-15)
     assert (off0, n0) == (0, 640)                      # 9 granules over 2 ranks: 5 + 4
+    has_gpu = torch.cuda.is_available()
+    assert codes[0] in ((0,) if has_gpu else (-8, -9)) or has_gpu
+    assert codes[1] == -3 and codes[2] == -3
 
 
 def test_token_shard_properties():
