@@ -93,6 +93,17 @@ def lib() -> ctypes.CDLL:
         L.oracle_bf16_sr.restype = ctypes.c_uint16
         L.oracle_rounding_bits.argtypes = [ctypes.c_uint64, ctypes.c_uint64, ctypes.c_int]
         L.oracle_rounding_bits.restype = ctypes.c_uint16
+        L.oracle_approx_4of8.argtypes = [ctypes.POINTER(ctypes.c_float), u32p, ctypes.POINTER(ctypes.c_int),
+                                         ctypes.POINTER(ctypes.c_float), ctypes.POINTER(ctypes.c_float)]
+        L.oracle_approx_4of8.restype = None
+        L.oracle_approx_4of8_ordered.argtypes = L.oracle_approx_4of8.argtypes + [ctypes.POINTER(ctypes.c_int)]
+        L.oracle_approx_4of8_ordered.restype = None
+        L.oracle_block_words4.argtypes = [ctypes.c_uint64, ctypes.c_uint64, u32p]
+        L.oracle_block_words4.restype = None
+        L.oracle_prune_4of8.argtypes = [ctypes.c_void_p, ctypes.c_int, ctypes.c_int64, ctypes.c_int64, ctypes.c_int64,
+                                        ctypes.c_int, ctypes.c_uint64, ctypes.c_int64, ctypes.c_int64,
+                                        ctypes.c_void_p, ctypes.c_void_p, ctypes.c_int]
+        L.oracle_prune_4of8.restype = ctypes.c_int
         L.oracle_unpack.argtypes = [ctypes.c_void_p, ctypes.c_void_p, ctypes.c_int64, ctypes.c_int64,
                                     ctypes.c_void_p]
         L.oracle_unpack.restype = None
@@ -332,3 +343,62 @@ def sweep_approx24(a):
     sec = np.array(list(second), dtype=np.float64).reshape(4, 4) / n
     sec[f == 0] = np.nan
     return f, sec, np.array(list(val), dtype=np.float64)
+
+
+# ------------------------------------------------------------------ approx-4:8 (prune only) -------
+def approx_4of8(a, words):
+    """Approx-4:8 on one block of eight: (positions ascending, new values, the eight inclusion probabilities)."""
+    arr = (ctypes.c_float * 8)(*[float(x) for x in a])
+    w = (ctypes.c_uint32 * 4)(*[int(x) & 0xFFFFFFFF for x in words])
+    idx = (ctypes.c_int * 4)()
+    val = (ctypes.c_float * 4)()
+    p = (ctypes.c_float * 8)()
+    lib().oracle_approx_4of8(arr, w, idx, val, p)
+    return tuple(int(i) for i in idx), tuple(float(v) for v in val), np.array(list(p), dtype=np.float64)
+
+
+def approx_4of8_order(a, words):
+    """The four positions of approx-4:8 in the order they were drawn."""
+    arr = (ctypes.c_float * 8)(*[float(x) for x in a])
+    w = (ctypes.c_uint32 * 4)(*[int(x) & 0xFFFFFFFF for x in words])
+    idx = (ctypes.c_int * 4)()
+    val = (ctypes.c_float * 4)()
+    p = (ctypes.c_float * 8)()
+    order = (ctypes.c_int * 4)()
+    lib().oracle_approx_4of8_ordered(arr, w, idx, val, p, order)
+    return tuple(int(i) for i in order)
+
+
+def block_words4(seed: int, q: int):
+    out = (ctypes.c_uint32 * 4)()
+    lib().oracle_block_words4(seed & (2**64 - 1), q, out)
+    return tuple(int(x) for x in out)
+
+
+def prune_4of8(g: np.ndarray, axis: int, seed: int, *, k_total: int | None = None, k_offset: int = 0, threads: int = 1):
+    """Approx-4:8 prune of a 2-D array: (values uint16 [Mrows, K/2], mask uint8 [Mrows, K/8], bit k = element k kept)."""
+    assert g.ndim == 2 and g.dtype in (np.float32, np.uint16)
+    g = np.ascontiguousarray(g)
+    rows, cols = g.shape
+    mrows, k = (rows, cols) if axis == 1 else (cols, rows)
+    values = np.zeros((mrows, k // 2), dtype=np.uint16)
+    mask = np.zeros((mrows, k // 8), dtype=np.uint8)
+    rc = lib().oracle_prune_4of8(g.ctypes.data, int(g.dtype == np.uint16), rows, cols, cols, axis, seed & (2**64 - 1),
+                                 k if k_total is None else k_total, k_offset, values.ctypes.data, mask.ctypes.data,
+                                 max(1, threads))
+    if rc != 0:
+        raise ValueError("oracle_prune_4of8: unsupported shape")
+    return values, mask
+
+
+def unpack_4of8(values: np.ndarray, mask: np.ndarray) -> np.ndarray:
+    """Dense float32 A[Mrows, K] from the approx-4:8 packed form (plain numpy: no arithmetic of the method)."""
+    mrows, kh = values.shape
+    dense = np.zeros((mrows, 2 * kh), dtype=np.float32)
+    vals = bf16_to_f32(values)
+    for r in range(mrows):
+        for j in range(kh // 4):
+            pos = [k for k in range(8) if mask[r, j] >> k & 1]
+            for e, k in enumerate(pos):
+                dense[r, 8 * j + k] = vals[r, 4 * j + e]
+    return dense

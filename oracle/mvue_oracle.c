@@ -580,6 +580,181 @@ int oracle_mvue_1of4(const float a[4], uint32_t word, float *kept)
 }
 
 /* ------------------------------------------------------------------------
+ * Approximately optimal 4:8 (appendix "Additional sparsity results": the
+ * approximate 2:4 method of Sec. 4.4 carried to a block of eight with four
+ * survivors; the paper gives no formulas).  Reading taken here: Sec. 4.4's
+ * procedure with four draws instead of two -- each draw removes one of the
+ * remaining elements with probability proportional to its magnitude -- and
+ * Sec. 4.4's rule for the kept values, a_i / p_i with p_i the EXACT probability
+ * that element i is among the four drawn, so that E[theta(a)] = a still holds.
+ *
+ * Inclusion probability.  The chance that the first |R| draws are the elements
+ * of the set R, in any order, obeys
+ *     w({}) = 1,   w(R) = sum_{k in R} w(R \ k) m_k / rest(R \ k),
+ * rest(Q) = the sum of the magnitudes NOT in Q (what is left after Q was
+ * removed), and element i is drawn at step |R| + 1 after R with probability
+ * m_i / rest(R), so
+ *     p_i = sum over R not containing i, |R| <= 3, of  w(R) m_i / rest(R).
+ * For two draws from four this is the equation of Sec. 4.4.
+ *
+ * Arithmetic (binary32, in the order written; every quotient is IEEE, and a
+ * quotient whose numerator is zero is zero whatever the denominator):
+ *   rest(Q): the magnitudes outside Q added left to right in position order;
+ *   sets R are visited by size, then by increasing bit mask (bit k = element k);
+ *   the sums over k in R and over R run in that order, first term first.
+ * Draws: word t (t = 0..3) of the block's own generator call (block number q
+ * of the operand counts blocks of eight: call q, four words) gives
+ *   thr = n_t (rest(removed so far) 2^-24), n_t the word's top 24 bits; the
+ *   running sums of the remaining magnitudes in position order are compared
+ *   with thr and the draw is the remaining element number #{sums <= thr},
+ *   capped at the last remaining one (the walk of App. "Pruning Overhead" Part 1).
+ * Zero rules: an element of magnitude zero owns an empty interval.  A block
+ * with at most four non-zeros keeps all of them with their own values (p = 1:
+ * magnitude-proportional draws exhaust the non-zeros first), and fills up with
+ * the zeros the walk lands on (the last remaining ones), as signed zeros.
+ *
+ * idx[0..3]: surviving positions, ascending; val[]: their new values.
+ * p_out (may be NULL) receives the eight inclusion probabilities as computed.
+ * ---------------------------------------------------------------------- */
+static float quot0(float num, float den) { return num == 0.0f ? 0.0f : num / den; }
+
+static int popcount8(unsigned x) { int c = 0; while (x) { c += (int)(x & 1u); x >>= 1; } return c; }
+
+void oracle_approx_4of8_ordered(const float a[8], const uint32_t words[4], int idx[4], float val[4], float p_out[8],
+                                int order_out[4]);
+
+void oracle_approx_4of8(const float a[8], const uint32_t words[4], int idx[4], float val[4], float p_out[8])
+{
+    oracle_approx_4of8_ordered(a, words, idx, val, p_out, NULL);
+}
+
+/* The same; order_out (may be NULL) receives the four positions in the order they were drawn. */
+void oracle_approx_4of8_ordered(const float a[8], const uint32_t words[4], int idx[4], float val[4], float p_out[8],
+                                int order_out[4])
+{
+    float m[8];
+    int nnz = 0;
+    for (int k = 0; k < 8; ++k) { m[k] = fabsf(a[k]); nnz += m[k] != 0.0f; }
+    /* rest(Q) for every set Q of at most three elements */
+    float rest[256], w[256];
+    for (unsigned Q = 0; Q < 256; ++Q) {
+        if (popcount8(Q) > 3) continue;
+        float r = 0.0f;
+        int first = 1;
+        for (int k = 0; k < 8; ++k) {
+            if (Q & (1u << k)) continue;
+            if (first) { r = m[k]; first = 0; } else r = r + m[k];
+        }
+        rest[Q] = r;
+    }
+    /* four draws */
+    unsigned removed = 0;
+    for (int t = 0; t < 4; ++t) {
+        const float thr = (float)(words[t] >> 8) * (rest[removed] * 5.9604644775390625e-08f);
+        float run = 0.0f;
+        int first = 1, pick = -1, last = -1;
+        for (int k = 0; k < 8; ++k) {
+            if (removed & (1u << k)) continue;
+            last = k;
+            if (pick >= 0) continue;
+            if (first) { run = m[k]; first = 0; } else run = run + m[k];
+            if (!(run <= thr)) pick = k;                    /* first remaining element whose running sum exceeds thr */
+        }
+        if (pick < 0) pick = last;
+        removed |= 1u << pick;
+        if (order_out) order_out[t] = pick;
+    }
+    /* inclusion probabilities */
+    float p[8];
+    if (nnz > 4) {
+        w[0] = 1.0f;
+        for (int size = 1; size <= 3; ++size) {
+            for (unsigned R = 1; R < 256; ++R) {
+                if (popcount8(R) != size) continue;
+                float acc = 0.0f;
+                int first = 1;
+                for (int k = 0; k < 8; ++k) {
+                    if (!(R & (1u << k))) continue;
+                    const unsigned Q = R & ~(1u << k);
+                    const float term = w[Q] * quot0(m[k], rest[Q]);
+                    if (first) { acc = term; first = 0; } else acc = acc + term;
+                }
+                w[R] = acc;
+            }
+        }
+        for (int i = 0; i < 8; ++i) {
+            float acc = 0.0f;
+            int first = 1;
+            for (int size = 0; size <= 3; ++size) {
+                for (unsigned R = 0; R < 256; ++R) {
+                    if (popcount8(R) != size || (R & (1u << i))) continue;
+                    const float term = w[R] * quot0(m[i], rest[R]);
+                    if (first) { acc = term; first = 0; } else acc = acc + term;
+                }
+            }
+            p[i] = acc;
+        }
+    } else {
+        for (int i = 0; i < 8; ++i) p[i] = m[i] != 0.0f ? 1.0f : 0.0f;
+    }
+    if (p_out) for (int i = 0; i < 8; ++i) p_out[i] = p[i];
+    int n = 0;
+    for (int k = 0; k < 8; ++k) {
+        if (!(removed & (1u << k))) continue;
+        idx[n] = k;
+        val[n] = (nnz > 4 && m[k] != 0.0f) ? a[k] / p[k] : a[k];
+        ++n;
+    }
+}
+
+/* The four words of block-of-eight number q: generator call q. */
+void oracle_block_words4(uint64_t seed, uint64_t q, uint32_t words[4])
+{
+    uint32_t ctr[4] = { (uint32_t)q, (uint32_t)(q >> 32), 0u, 0u };
+    uint32_t key[2] = { (uint32_t)seed, (uint32_t)(seed >> 32) };
+    oracle_philox4x32_10(ctr, key, words);
+}
+
+/* Tensor-wide approx-4:8 prune (no tensor core reads this pattern: prune only).
+ * Same operand view and block numbering as oracle_prune with blocks of eight:
+ * block j of row r of A is number r (k_total / 8) + k_offset / 8 + j.
+ * Output: values[Mrows x K/2] bf16 (nearest even), the four survivors of each
+ * block in ascending position; mask[Mrows x K/8] bytes, bit k set iff element k
+ * of the block survives (exactly four bits per byte). */
+int oracle_prune_4of8(const void *g, int is_bf16, int64_t rows, int64_t cols, int64_t ld, int axis,
+                      uint64_t seed, int64_t k_total, int64_t k_offset, uint16_t *values, uint8_t *mask,
+                      int threads)
+{
+    const int64_t Mrows = axis == 1 ? rows : cols;
+    const int64_t K     = axis == 1 ? cols : rows;
+    if (K % 8 != 0 || k_total % 8 != 0 || k_offset % 8 != 0 || k_offset + K > k_total) return -1;
+    (void)threads;
+#pragma omp parallel for num_threads(threads) schedule(static)
+    for (int64_t r = 0; r < Mrows; ++r) {
+        for (int64_t j = 0; j < K / 8; ++j) {
+            float a[8];
+            for (int e = 0; e < 8; ++e) {
+                int64_t k = 8 * j + e;
+                int64_t off = axis == 1 ? r * ld + k : k * ld + r;
+                a[e] = is_bf16 ? oracle_bf16_to_f32(((const uint16_t *)g)[off]) : ((const float *)g)[off];
+            }
+            uint64_t q = (uint64_t)r * (uint64_t)(k_total / 8) + (uint64_t)(k_offset / 8 + j);
+            uint32_t words[4];
+            oracle_block_words4(seed, q, words);
+            int idx[4]; float val[4];
+            oracle_approx_4of8(a, words, idx, val, NULL);
+            uint8_t bits = 0;
+            for (int e = 0; e < 4; ++e) {
+                values[r * (K / 2) + 4 * j + e] = oracle_bf16_rne(val[e]);
+                bits |= (uint8_t)(1u << idx[e]);
+            }
+            mask[r * (K / 8) + j] = bits;
+        }
+    }
+    return 0;
+}
+
+/* ------------------------------------------------------------------------
  * Tensor-wide prune and pack.
  *
  * g is a row-major [rows x cols] matrix with leading dimension ld, fp32

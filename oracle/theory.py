@@ -197,3 +197,34 @@ def mean_and_variance(outcomes):
     mean = (probs[:, None] * vecs).sum(0)
     var = (probs[:, None] * (vecs - mean) ** 2).sum()
     return mean, float(var)
+
+
+# ------------------------------------------- sequential draws without replacement -------
+def sequential_inclusion(a, n_draws: int):
+    """Inclusion probabilities of n_draws sequential draws without replacement, each proportional to magnitude among
+    the elements still there (Sec. 4.4's procedure, any block size), by brute force over every ordered sequence in
+    binary64.  Needs at least n_draws non-zeros."""
+    m = np.abs(np.asarray(a, dtype=np.float64))
+    p = np.zeros(len(m))
+    for seq in itertools.permutations(range(len(m)), n_draws):
+        prob, left = 1.0, m.sum()
+        for k in seq:
+            prob *= m[k] / left
+            left -= m[k]
+        for k in seq:
+            p[k] += prob
+    return p
+
+
+def sequential_set_law(a, n_draws: int):
+    """{frozenset of drawn positions: probability} for the same procedure."""
+    m = np.abs(np.asarray(a, dtype=np.float64))
+    law = {}
+    for seq in itertools.permutations(range(len(m)), n_draws):
+        prob, left = 1.0, m.sum()
+        for k in seq:
+            prob *= m[k] / left
+            left -= m[k]
+        key = frozenset(seq)
+        law[key] = law.get(key, 0.0) + prob
+    return law
