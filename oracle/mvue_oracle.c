@@ -597,9 +597,12 @@ int oracle_mvue_1of4(const float a[4], uint32_t word, float *kept)
  *     p_i = sum over R not containing i, |R| <= 3, of  w(R) m_i / rest(R).
  * For two draws from four this is the equation of Sec. 4.4.
  *
- * Arithmetic (binary32, in the order written; every quotient is IEEE, and a
- * quotient whose numerator is zero is zero whatever the denominator):
+ * Arithmetic (binary32, in the order written; one IEEE division per set):
  *   rest(Q): the magnitudes outside Q added left to right in position order;
+ *   inv(Q) = 1 / rest(Q), or 0 when rest(Q) = 0 (then nothing is left to draw);
+ *   u(Q) = w(Q) inv(Q), so that m_k / rest(Q) times w(Q) is formed as u(Q) m_k:
+ *     u({}) = inv({}),  w(R) = sum_{k in R} u(R \ k) m_k,  u(R) = w(R) inv(R),
+ *     p_i = sum_{R not containing i, |R| <= 3} u(R) m_i;
  *   sets R are visited by size, then by increasing bit mask (bit k = element k);
  *   the sums over k in R and over R run in that order, first term first.
  * Draws: word t (t = 0..3) of the block's own generator call (block number q
@@ -613,11 +616,14 @@ int oracle_mvue_1of4(const float a[4], uint32_t word, float *kept)
  * magnitude-proportional draws exhaust the non-zeros first), and fills up with
  * the zeros the walk lands on (the last remaining ones), as signed zeros.
  *
+ * Contract: the non-zero magnitudes of a block lie within a factor 2^60 of each
+ * other and sum to between 2^-100 and 2^100 (reciprocals and their products
+ * then stay normal numbers); outside it the pattern is still a valid one, the
+ * values are unspecified.
+ *
  * idx[0..3]: surviving positions, ascending; val[]: their new values.
  * p_out (may be NULL) receives the eight inclusion probabilities as computed.
  * ---------------------------------------------------------------------- */
-static float quot0(float num, float den) { return num == 0.0f ? 0.0f : num / den; }
-
 static int popcount8(unsigned x) { int c = 0; while (x) { c += (int)(x & 1u); x >>= 1; } return c; }
 
 void oracle_approx_4of8_ordered(const float a[8], const uint32_t words[4], int idx[4], float val[4], float p_out[8],
@@ -635,8 +641,8 @@ void oracle_approx_4of8_ordered(const float a[8], const uint32_t words[4], int i
     float m[8];
     int nnz = 0;
     for (int k = 0; k < 8; ++k) { m[k] = fabsf(a[k]); nnz += m[k] != 0.0f; }
-    /* rest(Q) for every set Q of at most three elements */
-    float rest[256], w[256];
+    /* rest(Q) and its reciprocal for every set Q of at most three elements */
+    float rest[256], inv[256], u[256];
     for (unsigned Q = 0; Q < 256; ++Q) {
         if (popcount8(Q) > 3) continue;
         float r = 0.0f;
@@ -646,6 +652,7 @@ void oracle_approx_4of8_ordered(const float a[8], const uint32_t words[4], int i
             if (first) { r = m[k]; first = 0; } else r = r + m[k];
         }
         rest[Q] = r;
+        inv[Q] = r == 0.0f ? 0.0f : 1.0f / r;
     }
     /* four draws */
     unsigned removed = 0;
@@ -667,7 +674,7 @@ void oracle_approx_4of8_ordered(const float a[8], const uint32_t words[4], int i
     /* inclusion probabilities */
     float p[8];
     if (nnz > 4) {
-        w[0] = 1.0f;
+        u[0] = inv[0];
         for (int size = 1; size <= 3; ++size) {
             for (unsigned R = 1; R < 256; ++R) {
                 if (popcount8(R) != size) continue;
@@ -675,11 +682,10 @@ void oracle_approx_4of8_ordered(const float a[8], const uint32_t words[4], int i
                 int first = 1;
                 for (int k = 0; k < 8; ++k) {
                     if (!(R & (1u << k))) continue;
-                    const unsigned Q = R & ~(1u << k);
-                    const float term = w[Q] * quot0(m[k], rest[Q]);
+                    const float term = u[R & ~(1u << k)] * m[k];
                     if (first) { acc = term; first = 0; } else acc = acc + term;
                 }
-                w[R] = acc;
+                u[R] = acc * inv[R];
             }
         }
         for (int i = 0; i < 8; ++i) {
@@ -688,7 +694,7 @@ void oracle_approx_4of8_ordered(const float a[8], const uint32_t words[4], int i
             for (int size = 0; size <= 3; ++size) {
                 for (unsigned R = 0; R < 256; ++R) {
                     if (popcount8(R) != size || (R & (1u << i))) continue;
-                    const float term = w[R] * quot0(m[i], rest[R]);
+                    const float term = u[R] * m[i];
                     if (first) { acc = term; first = 0; } else acc = acc + term;
                 }
             }

@@ -96,8 +96,12 @@ def test_zero_rules_and_validity():
         words = tuple(int(x) for x in RNG.integers(0, 2**32, 4))
         idx, val, _ = oracle.approx_4of8(a, words)
         assert list(idx) == sorted(set(idx)) and len(idx) == 4 and all(0 <= i < 8 for i in idx)
-        assert all(np.isfinite(v) for v in val)
-        assert all(np.sign(v) == np.sign(a[i]) or v == 0 for i, v in zip(idx, val))
+        # values are specified only inside the contract (non-zero magnitudes within 2^60 of each other, sums between
+        # 2^-100 and 2^100: the reciprocals and their products then stay normal numbers); the pattern is always valid
+        nz = np.abs(a[a != 0]).astype(np.float64)
+        if nz.size == 0 or (nz.max() / nz.min() <= 2.0 ** 60 and 2.0 ** -100 <= nz.sum() <= 2.0 ** 100):
+            assert all(np.isfinite(v) for v in val)
+            assert all(np.sign(v) == np.sign(a[i]) or v == 0 for i, v in zip(idx, val))
 
 
 def test_tensor_prune_numbering_shards_axes_and_monte_carlo():
