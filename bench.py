@@ -665,6 +665,7 @@ def tensor_bound_case(tm: Timer, n, m, peaks, joint, issue_cold):
     one_two_ms = tm.loop(prune_with((1, 2), joint), 20)
     sr_ms = tm.loop(lambda: binding.mvue_prune(g, n, m, 0, 1, values=values, meta=meta, layout=TC, joint=joint,
                                                options=binding.MVUE_OPT_STOCHASTIC_ROUNDING), 20)
+    four_eight_ms = tm.loop(lambda: binding.mvue_prune_4of8(g, 0, 1), 3, warm=1)     # approx-4:8, prune only
     prune_with((n, m), joint)()
     gemm_ms = tm.loop(lambda: binding.mvue_sparse_update_gemm(values, meta, h, out=dW, workspace=ws), 30)
     fused_ms = tm.loop(lambda: binding.mvue_fused_update_gemm(g, h, n, m, 1, out=dW), 3)
@@ -679,6 +680,8 @@ def tensor_bound_case(tm: Timer, n, m, peaks, joint, issue_cold):
             "prune_systematic_ms": sys_ms, "prune_systematic_frac_of_hbm_peak": pb / (sys_ms * 1e-3) / 1e9 / peaks["hbm_gbs"],
             "prune_table_ms": table_ms, "prune_table_frac_of_hbm_peak": pb / (table_ms * 1e-3) / 1e9 / peaks["hbm_gbs"],
             "prune_1of2_ms": one_two_ms, "prune_1of2_frac_of_hbm_peak": pb / (one_two_ms * 1e-3) / 1e9 / peaks["hbm_gbs"],
+            "prune_approx_4of8_ms": four_eight_ms,
+            "prune_approx_4of8_frac_of_hbm_peak": pb / (four_eight_ms * 1e-3) / 1e9 / peaks["hbm_gbs"],
             "prune_stochastic_rounding_ms": sr_ms,
             "prune_stochastic_rounding_frac_of_hbm_peak": pb / (sr_ms * 1e-3) / 1e9 / peaks["hbm_gbs"],
             "gemm_ms": gemm_ms, "gemm_tflops_effective": tf,

@@ -186,6 +186,27 @@ MVUE_API int mvue_prune_opts(const void* g, int dtype, int64_t rows, int64_t col
                     int axis, uint64_t seed, int64_t k_total, int64_t k_offset, void* values,
                     void* meta, int layout, int joint, unsigned options, void* stream);
 
+/* Approx-4:8 prune (appendix "Additional sparsity results": the approximate 2:4 method of Sec. 4.4 carried to four
+ * survivors of eight; the paper prints no formulas).  Prune only: no tensor core reads a 4:8 pattern, so there is no
+ * product that consumes this output.
+ * What it computes, per block of eight elements contiguous along K (operand view, axis, k_total, k_offset as for
+ * mvue_prune; block j of row r of A is number q = r (k_total / 8) + k_offset / 8 + j): four sequential draws, each
+ * removing one of the remaining elements with probability proportional to its magnitude (threshold walk in position
+ * order with eps = the top 24 bits of word t of Philox4x32-10(counter (lo32(q), hi32(q), 0, 0), key = seed), t = 0..3);
+ * a survivor becomes a_i / p_i with p_i the exact probability that i is among the four drawn, so E[theta(a)] = a:
+ *   rest(Q) = the magnitudes outside the set Q added left to right, inv(Q) = 1 / rest(Q) (0 if rest(Q) = 0),
+ *   u({}) = inv({}), w(R) = sum_{k in R} u(R \ k) |a_k|, u(R) = w(R) inv(R),
+ *   p_i = sum over R not containing i, |R| <= 3, of u(R) |a_i|
+ * (binary32, sets by size then by increasing bit mask, sums first term first; for two draws of four this is the
+ * inclusion probability printed in Sec. 4.4).  A block with at most four non-zeros keeps them all with their own
+ * values.  Values are specified for blocks whose non-zero magnitudes lie within 2^60 of each other and sum to between
+ * 2^-100 and 2^100; the pattern is valid for every input.
+ * Output: values bf16 [Mrows x K/2] (nearest even), the four survivors of each block in ascending position;
+ *         mask  bytes [Mrows x K/8], bit k of a byte set iff element k of that block survives.
+ * Preconditions: K, k_total, k_offset multiples of 8; g and ld * sizeof(element) 16-byte aligned, values 8-byte. */
+MVUE_API int mvue_prune_4of8(const void* g, int dtype, int64_t rows, int64_t cols, int64_t ld, int axis, uint64_t seed,
+                    int64_t k_total, int64_t k_offset, void* values, void* mask, void* stream);
+
 /* Expand a packed operand back to dense bf16 A[Mrows x K] (row-major, ld = K).
  * A checking aid: the inverse of the pack step, no arithmetic. */
 MVUE_API int mvue_unpack(const void* values, const void* meta, int layout, int64_t mrows, int64_t K,

@@ -21,7 +21,7 @@ MVUE_JOINT_TABLE, MVUE_JOINT_SYSTEMATIC, MVUE_JOINT_APPROX = 0, 1, 2
 MVUE_OPT_NONE, MVUE_OPT_STOCHASTIC_ROUNDING = 0, 1
 
 EXPORTS = ("mvue_version", "mvue_status_string", "mvue_last_cuda_error", "mvue_packed_sizes",
-           "mvue_prune", "mvue_prune_joint", "mvue_prune_opts", "mvue_unpack", "mvue_sparse_update_gemm", "mvue_sparse_backward_gemm",
+           "mvue_prune", "mvue_prune_joint", "mvue_prune_opts", "mvue_prune_4of8", "mvue_unpack", "mvue_sparse_update_gemm", "mvue_sparse_backward_gemm",
            "mvue_gemm_workspace_bytes", "mvue_sparse_update_gemm_noalloc", "mvue_fused_update_gemm",
            "mvue_probe_sparse_mma", "mvue_selftest_wait_timeout")
 
@@ -53,6 +53,7 @@ def lib() -> ctypes.CDLL:
         L.mvue_prune.argtypes = [vp, ci, i64, i64, i64, ci, ci, ci, u64, i64, i64, vp, vp, ci, vp]
         L.mvue_prune_joint.argtypes = [vp, ci, i64, i64, i64, ci, ci, ci, u64, i64, i64, vp, vp, ci, ci, vp]
         L.mvue_prune_opts.argtypes = [vp, ci, i64, i64, i64, ci, ci, ci, u64, i64, i64, vp, vp, ci, ci, ctypes.c_uint, vp]
+        L.mvue_prune_4of8.argtypes = [vp, ci, i64, i64, i64, ci, u64, i64, i64, vp, vp, vp]
         L.mvue_unpack.argtypes = [vp, vp, ci, i64, i64, vp, vp]
         L.mvue_sparse_update_gemm.argtypes = [vp, vp, ci, i64, i64, vp, i64, i64, vp, ci, i64, ci, vp,
                                               ctypes.c_size_t, vp, vp]
@@ -124,6 +125,19 @@ def mvue_prune(g: torch.Tensor, n: int, m: int, axis: int, seed: int, *, k_total
                                       values.data_ptr(), meta.data_ptr(), layout, int(joint), _stream_ptr()),
                "mvue_prune_joint")
     return values, meta
+
+
+def mvue_prune_4of8(g: torch.Tensor, axis: int, seed: int, *, k_total: int | None = None, k_offset: int = 0):
+    """Approx-4:8 prune (prune only) of a 2-D CUDA tensor: (values bf16 [Mrows, K/2], mask uint8 [Mrows, K/8])."""
+    assert g.is_cuda and g.dim() == 2 and g.stride(1) == 1
+    rows, cols = g.shape
+    mrows, k = (rows, cols) if axis == 1 else (cols, rows)
+    values = torch.empty((mrows, k // 2), dtype=torch.bfloat16, device=g.device)
+    mask = torch.empty((mrows, k // 8), dtype=torch.uint8, device=g.device)
+    _check(lib().mvue_prune_4of8(g.data_ptr(), _dtype_code(g), rows, cols, g.stride(0), axis, seed & (2**64 - 1),
+                                 k if k_total is None else k_total, k_offset, values.data_ptr(), mask.data_ptr(),
+                                 _stream_ptr()), "mvue_prune_4of8")
+    return values, mask
 
 
 def mvue_unpack(values: torch.Tensor, meta: torch.Tensor, layout: int = MVUE_LAYOUT_CANONICAL) -> torch.Tensor:

@@ -162,6 +162,25 @@ int mvue_prune_opts(const void* g, int dtype, int64_t rows, int64_t cols, int64_
     return MVUE_OK;
 }
 
+int mvue_prune_4of8(const void* g, int dtype, int64_t rows, int64_t cols, int64_t ld, int axis, uint64_t seed,
+                    int64_t k_total, int64_t k_offset, void* values, void* mask, void* stream) {
+    if (!g || !values || !mask) return MVUE_ERR_NULL;
+    if (dtype != MVUE_F32 && dtype != MVUE_BF16) return MVUE_ERR_DTYPE;
+    if (axis != 0 && axis != 1) return MVUE_ERR_SHAPE;
+    if (rows <= 0 || cols <= 0 || ld < cols) return MVUE_ERR_SHAPE;
+    const int64_t K = axis == 1 ? cols : rows;
+    if (K % 8 != 0 || k_total % 8 != 0 || k_offset % 8 != 0 || k_offset < 0 || k_offset + K > k_total) return MVUE_ERR_SHAPE;
+    const int64_t esz = dtype == MVUE_BF16 ? 2 : 4;
+    if (!aligned16(g) || (reinterpret_cast<uintptr_t>(values) & 7u) != 0 || (ld * esz) % 16 != 0) return MVUE_ERR_ALIGN;
+    DeviceInfo dev;
+    if (int s = current_device_info(&dev)) return s;
+    PruneArgs a{g, dtype == MVUE_BF16, rows, cols, ld, 8, axis, seed, k_total, k_offset, values, mask, dev.sm_count,
+                false, 0};
+    cudaError_t e = launch_prune_4of8(a, reinterpret_cast<cudaStream_t>(stream));
+    if (e != cudaSuccess) { set_cuda_error(e, "mvue_prune_4of8 launch"); return MVUE_ERR_CUDA; }
+    return MVUE_OK;
+}
+
 int mvue_unpack(const void* values, const void* meta, int layout, int64_t mrows, int64_t K,
                 void* dense_bf16, void* stream) {
     if (!values || !meta || !dense_bf16) return MVUE_ERR_NULL;

@@ -498,6 +498,129 @@ __device__ __forceinline__ void mvue_1of4_f32(uint32_t b0, uint32_t b1, uint32_t
     *nibble = i < 3u ? (i | 12u) : 14u;
 }
 
+// ===========================================================================
+// Approx-4:8 (appendix "Additional sparsity results": Sec. 4.4's procedure with four survivors of eight).  Four
+// sequential draws, each proportional to magnitude among the elements still there; a survivor is divided by its exact
+// inclusion probability p_i = sum over the sets R (|R| <= 3, i not in R) of u(R) m_i, with
+//   rest(Q) = the magnitudes outside Q added left to right,  inv(Q) = 1 / rest(Q) (0 if rest is 0),
+//   u({}) = inv({}),  w(R) = sum_{k in R} u(R \ k) m_k,  u(R) = w(R) inv(R),
+// sets visited by size, then by increasing bit mask, sums first term first.  A block with at most four non-zeros keeps
+// them all with their own values.  No tensor core reads this pattern: prune only.
+// b[8]: the block as binary32 bit patterns; words: the block's own generator call.  Returns the mask (bit k = element k
+// survives); out[0..1] = the four survivors as bf16, ascending position.
+// ===========================================================================
+__host__ __device__ constexpr int popcount8_c(unsigned x) {
+    return (int)((x & 1u) + ((x >> 1) & 1u) + ((x >> 2) & 1u) + ((x >> 3) & 1u) + ((x >> 4) & 1u) + ((x >> 5) & 1u) +
+                 ((x >> 6) & 1u) + ((x >> 7) & 1u));
+}
+
+__device__ __forceinline__ uint32_t approx_4of8(const uint32_t (&b)[8], uint4 words, uint32_t (&out)[2]) {
+    float m[8];
+    int nnz = 0;
+#pragma unroll
+    for (int k = 0; k < 8; ++k) {
+        m[k] = fabsf(__uint_as_float(b[k]));
+        nnz += m[k] != 0.0f ? 1 : 0;
+    }
+    auto rest_of = [&](unsigned Q) {                       // left to right over the elements outside Q
+        float r = 0.0f;
+        bool first = true;
+#pragma unroll
+        for (int k = 0; k < 8; ++k) {
+            if (Q & (1u << k)) continue;
+            r = first ? m[k] : __fadd_rn(r, m[k]);
+            first = false;
+        }
+        return r;
+    };
+    // four draws
+    const uint32_t w4[4] = {words.x, words.y, words.z, words.w};
+    unsigned removed = 0;
+#pragma unroll
+    for (int t = 0; t < 4; ++t) {
+        float left = 0.0f;
+        bool first = true;
+#pragma unroll
+        for (int k = 0; k < 8; ++k) {
+            if (removed & (1u << k)) continue;
+            left = first ? m[k] : __fadd_rn(left, m[k]);
+            first = false;
+        }
+        const float thr = __fmul_rn(top24(w4[t]), __fmul_rn(left, 5.9604644775390625e-08f));
+        float run = 0.0f;
+        first = true;
+        int pick = -1, last = -1;
+#pragma unroll
+        for (int k = 0; k < 8; ++k) {
+            if (removed & (1u << k)) continue;
+            last = k;
+            if (pick >= 0) continue;
+            run = first ? m[k] : __fadd_rn(run, m[k]);
+            first = false;
+            if (!(run <= thr)) pick = k;
+        }
+        if (pick < 0) pick = last;
+        removed |= 1u << pick;
+    }
+    float p[8];
+#pragma unroll
+    for (int i = 0; i < 8; ++i) p[i] = 1.0f;
+    if (nnz > 4) {
+        float u[256];                                       // only the 93 sets of at most three elements are ever touched
+#pragma unroll
+        for (int size = 0; size <= 3; ++size) {
+#pragma unroll
+            for (unsigned R = 0; R < 256; ++R) {
+                if (popcount8_c(R) != size) continue;
+                const float r = rest_of(R);
+                const float inv = r == 0.0f ? 0.0f : __fdiv_rn(1.0f, r);
+                float acc = 1.0f;                           // w({}) = 1
+                bool first = true;
+#pragma unroll
+                for (int k = 0; k < 8; ++k) {
+                    if (!(R & (1u << k))) continue;
+                    const float term = __fmul_rn(u[R & ~(1u << k)], m[k]);
+                    acc = first ? term : __fadd_rn(acc, term);
+                    first = false;
+                }
+                u[R] = size == 0 ? inv : __fmul_rn(acc, inv);
+            }
+        }
+#pragma unroll
+        for (int i = 0; i < 8; ++i) {
+            float acc = 0.0f;
+            bool first = true;
+#pragma unroll
+            for (int size = 0; size <= 3; ++size) {
+#pragma unroll
+                for (unsigned R = 0; R < 256; ++R) {
+                    if (popcount8_c(R) != size || (R & (1u << i))) continue;
+                    const float term = __fmul_rn(u[R], m[i]);
+                    acc = first ? term : __fadd_rn(acc, term);
+                    first = false;
+                }
+            }
+            p[i] = acc;
+        }
+    }
+    // survivors in ascending position
+    float v[4] = {0.0f, 0.0f, 0.0f, 0.0f};
+    int n = 0;
+#pragma unroll
+    for (int k = 0; k < 8; ++k) {
+        if (!(removed & (1u << k))) continue;
+        const float a = __uint_as_float(b[k]);
+        const float val = (nnz > 4 && m[k] != 0.0f) ? __fdiv_rn(a, p[k]) : a;
+#pragma unroll
+        for (int e = 0; e < 4; ++e)
+            if (e == n) v[e] = val;
+        ++n;
+    }
+    out[0] = pack_bf16x2(v[0], v[1]);
+    out[1] = pack_bf16x2(v[2], v[3]);
+    return removed;
+}
+
 // One work unit of bf16 input: raw[8] = 16 elements along K, two per word.
 // kJoint selects the 2:4 estimator (0: App. A.2 table, 1: systematic sampling, 2: approx-MVUE of Sec. 4.4,
 // which takes two words per block: one generator call per two blocks) or, with 3, MVUE 1:4; 1:2 has one law.

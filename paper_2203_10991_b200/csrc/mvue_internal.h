@@ -25,6 +25,7 @@ struct PruneArgs {
 };
 
 cudaError_t launch_prune(const PruneArgs& a, cudaStream_t stream);
+cudaError_t launch_prune_4of8(const PruneArgs& a, cudaStream_t stream);   // approx-4:8, prune only (meta = mask bytes)
 cudaError_t launch_unpack(const void* values, const void* meta, bool tc_layout, int64_t mrows, int64_t K,
                           void* dense, int sm_count, cudaStream_t stream);
 

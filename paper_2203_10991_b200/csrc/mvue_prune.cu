@@ -517,6 +517,48 @@ prune_axis0_bf16_whole_tiles_kernel(const __grid_constant__ CUtensorMap map_g, c
     }
 }
 
+// ---- approx-4:8 (prune only) ---------------------------------------------------
+// One thread per block of eight.  Row r of A and block j along K; threads run along K for axis 1 (8 contiguous
+// elements per thread) and along the rows of A for axis 0 (8 rows of g, neighbouring threads on neighbouring columns),
+// so that the loads of a warp coalesce either way.  The arithmetic (93 reciprocals and a few hundred multiply-adds per
+// block) is what bounds this kernel, not memory.
+template <bool kBf16>
+__global__ void __launch_bounds__(128)
+prune_4of8_kernel(const void* __restrict__ g, int64_t mrows, int64_t kblocks, int64_t ld, int axis,
+                  int64_t kblocks_total, int64_t kblock_offset, RoundKeys rk, uint2* __restrict__ values,
+                  uint8_t* __restrict__ mask) {
+    const int64_t n = mrows * kblocks;
+    for (int64_t i = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; i < n; i += (int64_t)gridDim.x * blockDim.x) {
+        const int64_t r = axis == 1 ? i / kblocks : i % mrows;
+        const int64_t j = axis == 1 ? i % kblocks : i / mrows;
+        uint32_t b[8];
+        if (axis == 1) {
+            if (kBf16) {
+                const uint4 x = ldg128(reinterpret_cast<const char*>(g) + (r * ld + 8 * j) * 2);
+                const uint32_t w[4] = {x.x, x.y, x.z, x.w};
+#pragma unroll
+                for (int e = 0; e < 4; ++e) { b[2 * e] = w[e] << 16; b[2 * e + 1] = w[e] & 0xFFFF0000u; }
+            } else {
+                const uint4 x = ldg128(reinterpret_cast<const char*>(g) + (r * ld + 8 * j) * 4);
+                const uint4 y = ldg128(reinterpret_cast<const char*>(g) + (r * ld + 8 * j) * 4 + 16);
+                b[0] = x.x; b[1] = x.y; b[2] = x.z; b[3] = x.w; b[4] = y.x; b[5] = y.y; b[6] = y.z; b[7] = y.w;
+            }
+        } else {
+#pragma unroll
+            for (int e = 0; e < 8; ++e) {
+                const int64_t off = (8 * j + e) * ld + r;
+                b[e] = kBf16 ? (uint32_t)__ldg(reinterpret_cast<const uint16_t*>(g) + off) << 16
+                             : __ldg(reinterpret_cast<const uint32_t*>(g) + off);
+            }
+        }
+        const uint64_t q = (uint64_t)r * (uint64_t)kblocks_total + (uint64_t)(kblock_offset + j);
+        uint32_t out[2];
+        const uint32_t bits = approx_4of8(b, philox4x32_10(q, rk), out);
+        values[r * kblocks + j] = make_uint2(out[0], out[1]);
+        mask[r * kblocks + j] = (uint8_t)bits;
+    }
+}
+
 // ---- unpack ---------------------------------------------------------------
 // One thread expands one unit: a 16-bit metadata word (four groups) and its 8 survivors
 // become 16 dense elements (32 bytes).
@@ -627,6 +669,21 @@ cudaError_t launch_prune(const PruneArgs& a, cudaStream_t stream) {
     if (a.joint == 3) return launch_prune_m<4, 3>(a, stream);          // MVUE 1:4
     if (a.joint == 2) return launch_prune_m<4, 2>(a, stream);
     return a.joint == 1 ? launch_prune_m<4, 1>(a, stream) : launch_prune_m<4, 0>(a, stream);
+}
+
+cudaError_t launch_prune_4of8(const PruneArgs& a, cudaStream_t stream) {
+    const int64_t mrows = a.axis == 1 ? a.rows : a.cols, K = a.axis == 1 ? a.cols : a.rows;
+    const int64_t n = mrows * (K / 8);
+    const int64_t want = (n + 127) / 128;
+    const int grid = (int)(want < (int64_t)a.sm_count * 16 ? want : (int64_t)a.sm_count * 16);
+    const RoundKeys rk = make_round_keys(a.seed);
+    if (a.is_bf16)
+        prune_4of8_kernel<true><<<grid, 128, 0, stream>>>(a.g, mrows, K / 8, a.ld, a.axis, a.k_total / 8, a.k_offset / 8, rk,
+                                                         reinterpret_cast<uint2*>(a.values), reinterpret_cast<uint8_t*>(a.meta));
+    else
+        prune_4of8_kernel<false><<<grid, 128, 0, stream>>>(a.g, mrows, K / 8, a.ld, a.axis, a.k_total / 8, a.k_offset / 8, rk,
+                                                          reinterpret_cast<uint2*>(a.values), reinterpret_cast<uint8_t*>(a.meta));
+    return cudaGetLastError();
 }
 
 cudaError_t launch_unpack(const void* values, const void* meta, bool tc_layout, int64_t mrows, int64_t K,
