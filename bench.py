@@ -739,6 +739,16 @@ def gemm_shapes_case(tm: Timer, peaks, issue_cold):
             dmean, _ = tm.each(lambda: torch.matmul(A_dense, B), 10)
             dfmean, _ = tm.each(lambda: torch.matmul(A_dense, B) * fz, 10)
             row["dense_us"], row["dense_act_grad_us"] = 1e3 * dmean, 1e3 * dfmean
+            if N % 128 == 0:
+                # the same product pruning its own output along N in the epilogue, against the product followed by
+                # the separate prune of its output
+                emean, _ = tm.each(lambda: binding.mvue_sparse_backward_gemm_pruned(
+                    v, mt, B, fz, 5, next_joint=binding.MVUE_JOINT_SYSTEMATIC, workspace=ws), 10)
+                pv, pm = binding.mvue_prune(C, 2, 4, 1, 5, layout=TC, joint=binding.MVUE_JOINT_SYSTEMATIC)
+                pmean, _ = tm.each(lambda: binding.mvue_prune(C, 2, 4, 1, 5, values=pv, meta=pm, layout=TC,
+                                                              joint=binding.MVUE_JOINT_SYSTEMATIC), 10)
+                row["act_grad_epilogue_prune_us"] = 1e3 * emean
+                row["separate_prune_of_output_us"] = 1e3 * pmean
         rows.append(row)
         del g, v, mt, B, C
         torch.cuda.empty_cache()
@@ -879,10 +889,16 @@ def chain_case(n, m):
     def run_sys_overlap():
         chain.backward_update(g_top, layers, n, m, base_seed=1, joint=binding.MVUE_JOINT_SYSTEMATIC, overlap=True)
 
+    def run_sys_epilogue():
+        # backward products with a long reduction axis (out = 4096) prune their own output for the layer below
+        chain.backward_update(g_top, layers, n, m, base_seed=1, joint=binding.MVUE_JOINT_SYSTEMATIC, overlap=True,
+                              prune_in_epilogue_min_k=4096)
+
     eager_ms = timed(run_table, 5)
     table_ms = timed(graphed(run_table), 10)
     sys_ms = timed(graphed(run_sys), 10) if m == 4 else None
     overlap_ms = timed(graphed(run_sys_overlap), 10) if m == 4 else None
+    epilogue_ms = timed(graphed(run_sys_epilogue), 10) if m == 4 else None
     dense_ms = timed(graphed(dense_chain), 10)
     n_layers = len(layers)
     flops = 2.0 * T * d * d_ff * (2 * n_layers - 1)         # update product per layer, backward for all but the bottom
@@ -895,6 +911,9 @@ def chain_case(n, m):
             # the same chain with each update product on a second stream beside the next axis-1 prune
             "systematic_two_stream_ms": overlap_ms,
             "systematic_two_stream_tflops_effective": None if overlap_ms is None else flops / (overlap_ms * 1e-3) / 1e12,
+            # and with the long-K backward products pruning their own output in the epilogue (one prune launch less
+            # per block of two layers)
+            "systematic_two_stream_epilogue_prune_ms": epilogue_ms,
             "dense_torch_ms": dense_ms, "dense_torch_tflops": flops / (dense_ms * 1e-3) / 1e12}
 
 

@@ -22,6 +22,7 @@ MVUE_OPT_NONE, MVUE_OPT_STOCHASTIC_ROUNDING = 0, 1
 
 EXPORTS = ("mvue_version", "mvue_status_string", "mvue_last_cuda_error", "mvue_packed_sizes",
            "mvue_prune", "mvue_prune_joint", "mvue_prune_opts", "mvue_prune_4of8", "mvue_unpack", "mvue_sparse_update_gemm", "mvue_sparse_backward_gemm",
+           "mvue_sparse_backward_gemm_pruned",
            "mvue_gemm_workspace_bytes", "mvue_sparse_update_gemm_noalloc", "mvue_fused_update_gemm",
            "mvue_probe_sparse_mma", "mvue_selftest_wait_timeout")
 
@@ -59,6 +60,8 @@ def lib() -> ctypes.CDLL:
                                               ctypes.c_size_t, vp, vp]
         L.mvue_sparse_backward_gemm.argtypes = [vp, vp, ci, i64, i64, vp, i64, i64, vp, vp, ci, i64, vp,
                                                 ctypes.c_size_t, vp, vp]
+        L.mvue_sparse_backward_gemm_pruned.argtypes = [vp, vp, ci, i64, i64, vp, i64, i64, vp, vp, i64, u64, ci, vp, vp,
+                                                       vp, ctypes.c_size_t, vp, vp]
         L.mvue_gemm_workspace_bytes.argtypes = [ci, i64, i64, i64, szp]
         L.mvue_fused_update_gemm.argtypes = [vp, ci, i64, i64, i64, ci, ci, u64, vp, i64, i64, vp, ci, i64, ci, vp,
                                              ctypes.c_size_t, vp, vp]
@@ -203,6 +206,31 @@ def mvue_sparse_backward_gemm(values: torch.Tensor, meta: torch.Tensor, W: torch
                                            None if dev_status is None else dev_status.data_ptr(), _stream_ptr()),
            "mvue_sparse_backward_gemm")
     return out
+
+
+def mvue_sparse_backward_gemm_pruned(values: torch.Tensor, meta: torch.Tensor, W: torch.Tensor, act_grad: torch.Tensor,
+                                     next_seed: int, *, next_joint: int = MVUE_JOINT_TABLE,
+                                     workspace: torch.Tensor | None = None, dev_status: torch.Tensor | None = None,
+                                     layout: int = MVUE_LAYOUT_TC):
+    """dh = (theta(g) . W) * act_grad (bf16) and, from the same launch, dh pruned 2:4 along its columns in tensor-core
+    order (what mvue_prune(dh, 2, 4, axis=1, next_seed, layout=MVUE_LAYOUT_TC, joint=next_joint) gives).
+    Returns (dh, next_values, next_meta)."""
+    T, half_o = values.shape
+    n_out, n_in = W.shape
+    assert W.dtype == torch.bfloat16 and W.stride(1) == 1 and 2 * half_o == n_out
+    out = torch.empty((T, n_in), dtype=torch.bfloat16, device=W.device)
+    assert act_grad.dtype == torch.bfloat16 and act_grad.shape == out.shape and act_grad.stride(0) == out.stride(0)
+    _, meta_bytes = mvue_packed_sizes(T, n_in, 2, 4, 1, MVUE_LAYOUT_TC)
+    next_values = torch.empty((T, n_in // 2), dtype=torch.bfloat16, device=W.device)
+    next_meta = torch.empty((meta_bytes // (n_in // 8), n_in // 8), dtype=torch.uint8, device=W.device)
+    ws, ws_bytes = _workspace(1, T, n_in, n_out, W.device, workspace)
+    _check(lib().mvue_sparse_backward_gemm_pruned(values.data_ptr(), meta.data_ptr(), layout, T, n_out, W.data_ptr(), n_in,
+                                                  W.stride(0), act_grad.data_ptr(), out.data_ptr(), out.stride(0),
+                                                  next_seed & (2**64 - 1), int(next_joint), next_values.data_ptr(),
+                                                  next_meta.data_ptr(), None if ws is None else ws.data_ptr(), ws_bytes,
+                                                  None if dev_status is None else dev_status.data_ptr(), _stream_ptr()),
+           "mvue_sparse_backward_gemm_pruned")
+    return out, next_values, next_meta
 
 
 def mvue_sparse_update_gemm_noalloc(values: torch.Tensor, meta: torch.Tensor, h: torch.Tensor, out: torch.Tensor, *,

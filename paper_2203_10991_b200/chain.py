@@ -23,7 +23,7 @@ def layer_seeds(base_seed: int, layer: int) -> tuple[int, int]:
 
 
 def backward_update(g_top: torch.Tensor, layers, n: int = 2, m: int = 4, base_seed: int = 0, joint: int | None = None,
-                    overlap: bool = False):
+                    overlap: bool = False, prune_in_epilogue_min_k: int | None = None):
     """layers: list (top layer first) of dicts {"W": [out x in] bf16, "h": [T x in] bf16,
     "act_grad": [T x in] bf16 or None (None for the bottom layer: no gradient is propagated further)}.
     joint: the 2:4 law over pairs handed to mvue_prune_joint (None: mvue_prune, the App. A.2 table).
@@ -32,9 +32,33 @@ def backward_update(g_top: torch.Tensor, layers, n: int = 2, m: int = 4, base_se
     product of a long token axis keeps a small register footprint, so blocks of the (shared-memory-free) prune along
     the features fit on the same SMs.  Same calls, same seeds, same results; the streams join before each backward
     product and before returning.
+    prune_in_epilogue_min_k: when set (2:4 only), a backward product whose reduction axis (the layer's out) is at least
+    this long also prunes its own output along the features in its epilogue (mvue_sparse_backward_gemm_pruned), with
+    the seed the layer below would have used, so that layer's prune along the features is not launched.  Same bits.
     Returns the list of dW (fp32), top layer first."""
     g = g_top
     grads = []
+    ready = None                                          # (values, meta) of the current g along the features, if already made
+    fuse_joint = binding.MVUE_JOINT_TABLE if joint is None else joint
+
+    def backward(i, L, values_b, meta_b):
+        nonlocal ready
+        below = layers[i + 1] if i + 1 < len(layers) else None
+        if (prune_in_epilogue_min_k is not None and (n, m) == (2, 4) and L["W"].shape[0] >= prune_in_epilogue_min_k
+                and below is not None and below.get("act_grad") is not None and L["W"].shape[1] % 128 == 0
+                and fuse_joint in (binding.MVUE_JOINT_TABLE, binding.MVUE_JOINT_SYSTEMATIC)):
+            g_next, nv, nm = binding.mvue_sparse_backward_gemm_pruned(values_b, meta_b, L["W"], L["act_grad"],
+                                                                      layer_seeds(base_seed, i + 1)[1], next_joint=fuse_joint)
+            ready = (nv, nm)
+            return g_next
+        ready = None
+        return binding.mvue_sparse_backward_gemm(values_b, meta_b, L["W"], act_grad=L["act_grad"], out_dtype=torch.bfloat16)
+
+    def prune_features(g, s_bwd):
+        if ready is not None:
+            return ready
+        return binding.mvue_prune(g, n, m, 1, s_bwd, layout=TC, joint=joint)
+
     main = torch.cuda.current_stream()
     side = torch.cuda.Stream(priority=-1) if overlap else None
     for i, L in enumerate(layers):
@@ -48,15 +72,13 @@ def backward_update(g_top: torch.Tensor, layers, n: int = 2, m: int = 4, base_se
             side.wait_stream(main)
             with torch.cuda.stream(side):
                 binding.mvue_sparse_update_gemm(values, meta, L["h"], out=dW, workspace=ws)
-            values_b, meta_b = binding.mvue_prune(g, n, m, 1, s_bwd, layout=TC, joint=joint)
+            values_b, meta_b = prune_features(g, s_bwd)
             main.wait_stream(side)                       # (values, meta, ws stay referenced until here)
             grads.append(dW)
-            g = binding.mvue_sparse_backward_gemm(values_b, meta_b, L["W"], act_grad=L["act_grad"],
-                                                  out_dtype=torch.bfloat16)
+            g = backward(i, L, values_b, meta_b)
             continue
         grads.append(binding.mvue_sparse_update_gemm(values, meta, L["h"]))
         if propagate:
-            values, meta = binding.mvue_prune(g, n, m, 1, s_bwd, layout=TC, joint=joint)
-            g = binding.mvue_sparse_backward_gemm(values, meta, L["W"], act_grad=L["act_grad"],
-                                                  out_dtype=torch.bfloat16)
+            values, meta = prune_features(g, s_bwd)
+            g = backward(i, L, values, meta)
     return grads

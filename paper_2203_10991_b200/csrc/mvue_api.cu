@@ -222,6 +222,38 @@ int mvue_sparse_backward_gemm(const void* values, const void* meta, int layout, 
                     workspace_bytes, dev_status, stream);
 }
 
+int mvue_sparse_backward_gemm_pruned(const void* values, const void* meta, int layout, int64_t T, int64_t out,
+                                     const void* W, int64_t in, int64_t ldW, const void* act_grad, void* dh,
+                                     int64_t lddh, uint64_t next_seed, int next_joint, void* next_values,
+                                     void* next_meta, void* workspace, size_t workspace_bytes, int* dev_status,
+                                     void* stream) {
+    if (!act_grad || !next_values || !next_meta) return MVUE_ERR_NULL;
+    if (next_joint != MVUE_JOINT_TABLE && next_joint != MVUE_JOINT_SYSTEMATIC) return MVUE_ERR_JOINT;
+    if (in % 128 != 0) return MVUE_ERR_SHAPE;                      // K of the next product, tensor-core order
+    if (!aligned16(next_values) || !aligned16(next_meta)) return MVUE_ERR_ALIGN;
+    DeviceInfo dev;
+    if (int s = check_gemm(values, meta, layout, T, in, out, W, ldW, act_grad, dh, MVUE_BF16, lddh, 0, &dev)) return s;
+    const size_t need = gemm_required_workspace_bytes(T, in, out, dev.sm_count);
+    if (need > 0 && (!workspace || workspace_bytes < need)) return MVUE_ERR_WORKSPACE;
+    if (workspace && !aligned16(workspace)) return MVUE_ERR_WORKSPACE;
+    SparseGemmArgs a{values, meta, T, in, out, W, ldW, dh, lddh, 1, 0, act_grad, workspace,
+                     workspace ? workspace_bytes : 0, dev_status, dev.sm_count};
+    if (need == 0 && T % 128 == 0) {                                // one launch: the prune rides in the epilogue
+        a.next_values = next_values;
+        a.next_meta = next_meta;
+        a.next_seed = next_seed;
+        a.next_joint = next_joint;
+        return launch_sparse_gemm(a, reinterpret_cast<cudaStream_t>(stream));
+    }
+    // a product split along K (its tiles are partial sums) or with a ragged last row block: the two steps one after the other
+    if (int s = launch_sparse_gemm(a, reinterpret_cast<cudaStream_t>(stream))) return s;
+    if (T % 8 != 0) return MVUE_ERR_SHAPE;
+    PruneArgs pa{dh, true, T, in, lddh, 4, 1, next_seed, in, 0, next_values, next_meta, dev.sm_count, true, next_joint};
+    cudaError_t e = launch_prune(pa, reinterpret_cast<cudaStream_t>(stream));
+    if (e != cudaSuccess) { set_cuda_error(e, "mvue_sparse_backward_gemm_pruned prune launch"); return MVUE_ERR_CUDA; }
+    return MVUE_OK;
+}
+
 int mvue_fused_update_gemm(const void* g, int dtype, int64_t T, int64_t out, int64_t ldg, int n, int m,
                            uint64_t seed, const void* h, int64_t in, int64_t ldh, void* dW, int dW_dtype,
                            int64_t lddW, int accumulate, void* workspace, size_t workspace_bytes,

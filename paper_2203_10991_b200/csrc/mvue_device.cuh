@@ -621,6 +621,16 @@ __device__ __forceinline__ uint32_t approx_4of8(const uint32_t (&b)[8], uint4 wo
     return removed;
 }
 
+// Byte offset of the 16-bit metadata word of (row r of A, strip = k / 16) in the tensor-core order:
+// blocks of 128 rows x 128 k (2 KiB, row-block major), inside a block 128 lanes of 16 bytes with
+// lane = r % 8 + 8 * (strip % 2) + 16 * (r % 128 / 16), word = strip % 8 / 2, half-word = r / 8 % 2.
+// This is the arrangement tcgen05.cp.128x128b moves verbatim into tensor memory for four MMAs.
+__device__ __forceinline__ int64_t tc_meta_offset(int64_t r, int64_t strip, int64_t kblocks) {
+    const int rl = (int)(r & 127), st = (int)(strip & 7);
+    const int lane = (rl & 7) + 8 * (st & 1) + 16 * (rl >> 4);
+    return ((r >> 7) * kblocks + (strip >> 3)) * 2048 + lane * 16 + (st >> 1) * 4 + ((rl >> 3) & 1) * 2;
+}
+
 // One work unit of bf16 input: raw[8] = 16 elements along K, two per word.
 // kJoint selects the 2:4 estimator (0: App. A.2 table, 1: systematic sampling, 2: approx-MVUE of Sec. 4.4,
 // which takes two words per block: one generator call per two blocks) or, with 3, MVUE 1:4; 1:2 has one law.

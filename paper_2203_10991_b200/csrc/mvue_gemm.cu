@@ -144,6 +144,11 @@ struct GemmParams {
     int tail_rem, tail_splits;   // the last tail_rem tiles are cut into tail_splits parts along K (0, 1: not)
     float* tail_partial;      // [tail_splits x tail_rem] tiles of 256 x 256 fp32
     int* dev_status;
+    // modes 5 / 6: the bf16 output tile is also pruned along its own columns (MVUE 2:4, the next product's reduction
+    // axis) and packed, as mvue_prune(output, axis 1, next_seed, tensor-core order) would
+    uint4* next_values;       // [M x N/2] bf16 survivors of the pruned output
+    uint8_t* next_meta;       // its metadata in tensor-core order
+    RoundKeys next_rk;
 };
 
 // Epilogue of one thread: its accumulator row (32 columns at a time from tensor memory) goes to the
@@ -395,6 +400,10 @@ __device__ __forceinline__ void quad_transpose(uint32_t (&v)[64], int lane) {
 // kMode fixes the output path at compile time so that the drained tile fits the register file:
 //   0: fp32 (C, C +=, or the split-K workspace)   1: bf16   2: bf16 times p.scale   3: fp32 times p.scale
 //   4: as 0 with the small-footprint epilogue (64 registers per thread), for work items with long main loops
+//   5, 6: as 2, and the drained bf16 tile -- one row per lane, 128 consecutive columns: eight prune units in the form a
+//         unit has when K is contiguous -- is pruned in registers (5: systematic sampling, 6: App. A.2 table) and its
+//         survivors and metadata stored before the dense tile goes out: the output of the backward product (Sec. 1,
+//         backward equation) leaves already pruned along the next backward product's reduction axis
 // The scale factors of a row are fetched into registers under the main loop.
 template <int kMode>
 __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(kMode == 4 ? 1024 : kThreads, 1)
@@ -590,7 +599,8 @@ sparse_gemm_pair_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_
             }
             // bf16 x scale keeps the row's factors in registers; fp32 x scale has no room for them beside 128
             // fp32 results and applies them after tensor memory has been handed back
-            constexpr bool kScale = kMode == 2, kLateScale = kMode == 3, kToBf16 = kMode == 1 || kMode == 2;
+            constexpr bool kPrune = kMode == 5 || kMode == 6;
+            constexpr bool kScale = kMode == 2 || kPrune, kLateScale = kMode == 3, kToBf16 = kMode == 1 || kScale;
             // bf16 outputs and their factors move in the quad-transposed arrangement (quad_transpose): lane
             // 4 a + b reads / writes, for c = 0..3 and k = 0, 1, the 32-byte chunk b + 4 k of row 4 a + c of the warp's
             // 32 rows, i.e. the quad covers whole 128-byte lines.
@@ -667,6 +677,24 @@ sparse_gemm_pair_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_
             } else {
 #pragma unroll
                 for (int e = 0; e < (kToBf16 ? 64 : 128); ++e) r[e] = 0u;
+            }
+            if constexpr (kPrune) {
+                // r[8 t .. 8 t + 7] = columns col0 + 16 t .. + 15 of this lane's row as bf16 pairs: prune unit t of the row
+                if (row_ok && col0 < p.N) {                              // (N is a multiple of 128: all eight units exist)
+                    const int64_t upr = p.N >> 4, strip0 = col0 >> 4;
+                    uint4* vdst = p.next_values + row * upr + strip0;
+#pragma unroll
+                    for (int t = 0; t < 8; ++t) {
+                        uint32_t raw[8];
+#pragma unroll
+                        for (int e = 0; e < 8; ++e) raw[e] = r[8 * t + e];
+                        uint4 v;
+                        uint32_t mt;
+                        prune_unit_bf16<4, kMode == 5 ? 1 : 0>(raw, (uint64_t)(row * upr + strip0 + t), p.next_rk, &v, &mt);
+                        vdst[t] = v;
+                        *reinterpret_cast<uint16_t*>(p.next_meta + tc_meta_offset(row, strip0 + t, p.N >> 7)) = (uint16_t)mt;
+                    }
+                }
             }
             if constexpr (kToBf16) {
                 quad_transpose(r, lane);
@@ -1097,13 +1125,15 @@ PairKernelSetup& pair_setup() {
 cudaError_t pair_kernel_setup() {
     PairKernelSetup& st = pair_setup();
     return once_per_device(st.once, [&st](int dev) {
-        const void* kernels[5] = {reinterpret_cast<const void*>(sparse_gemm_pair_kernel<0>),
+        const void* kernels[7] = {reinterpret_cast<const void*>(sparse_gemm_pair_kernel<0>),
                                   reinterpret_cast<const void*>(sparse_gemm_pair_kernel<1>),
                                   reinterpret_cast<const void*>(sparse_gemm_pair_kernel<2>),
                                   reinterpret_cast<const void*>(sparse_gemm_pair_kernel<3>),
-                                  reinterpret_cast<const void*>(sparse_gemm_pair_kernel<4>)};
+                                  reinterpret_cast<const void*>(sparse_gemm_pair_kernel<4>),
+                                  reinterpret_cast<const void*>(sparse_gemm_pair_kernel<5>),
+                                  reinterpret_cast<const void*>(sparse_gemm_pair_kernel<6>)};
         cudaError_t err = cudaSuccess;
-        for (int i = 0; i < 5 && err == cudaSuccess; ++i)
+        for (int i = 0; i < 7 && err == cudaSuccess; ++i)
             err = cudaFuncSetAttribute(kernels[i], cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemBytes);
         cudaLaunchConfig_t cfg = {};
         cfg.gridDim = dim3(2, 1, 1);
@@ -1227,6 +1257,7 @@ int launch_fused_update(const FusedArgs& f, cudaStream_t stream) {
     p.scale = nullptr;
     p.c_is_bf16 = a.c_is_bf16; p.accumulate = a.accumulate; p.splits = splits;
     p.n_work = p.n_main = 0; p.tail_rem = p.tail_splits = 0; p.tail_partial = nullptr;   // pair kernel only
+    p.next_values = nullptr; p.next_meta = nullptr; p.next_rk = fp.rk;
     p.dev_status = a.dev_status;
     dim3 grid((unsigned)((a.N + BN - 1) / BN), (unsigned)((a.M + BM - 1) / BM), (unsigned)splits);
     if (f.m == 4)
@@ -1289,6 +1320,9 @@ int launch_sparse_gemm(const SparseGemmArgs& a, cudaStream_t stream) {
     p.scale = reinterpret_cast<const __nv_bfloat16*>(a.scale);
     p.c_is_bf16 = a.c_is_bf16; p.accumulate = a.accumulate; p.splits = splits;
     p.dev_status = a.dev_status;
+    p.next_values = reinterpret_cast<uint4*>(a.next_values);
+    p.next_meta = reinterpret_cast<uint8_t*>(a.next_meta);
+    p.next_rk = make_round_keys(a.next_seed);
     const int resident = resident_pairs(a.sm_count);
     TailPlan tail = tail_plan(a.M, a.N, a.K, splits, resident);
     const size_t tail_bytes = (size_t)tail.rem * (size_t)tail.parts * (size_t)(2 * BM) * (size_t)BN * sizeof(float);
@@ -1310,7 +1344,13 @@ int launch_sparse_gemm(const SparseGemmArgs& a, cudaStream_t stream) {
     // main loops of at least 32 stages (K = 4096) per work item: the small-footprint epilogue costs nothing there
     const int64_t item_steps = tail.parts > 1 ? steps / tail.parts : p.k_steps_per_split;
     const bool long_items = item_steps >= 32;
-    if (scaled && to_bf16)
+    if (a.next_values != nullptr) {
+        if (!(scaled && to_bf16)) return MVUE_ERR_SHAPE;         // (the caller routes split products elsewhere)
+        if (a.next_joint == 1)
+            sparse_gemm_pair_kernel<5><<<grid, kThreads, kSmemBytes, stream>>>(map_a, map_b, map_e, p);
+        else
+            sparse_gemm_pair_kernel<6><<<grid, kThreads, kSmemBytes, stream>>>(map_a, map_b, map_e, p);
+    } else if (scaled && to_bf16)
         sparse_gemm_pair_kernel<2><<<grid, kThreads, kSmemBytes, stream>>>(map_a, map_b, map_e, p);
     else if (scaled)
         sparse_gemm_pair_kernel<3><<<grid, kThreads, kSmemBytes, stream>>>(map_a, map_b, map_e, p);

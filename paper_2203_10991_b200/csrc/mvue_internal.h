@@ -44,6 +44,11 @@ struct SparseGemmArgs {
     size_t workspace_bytes;
     int* dev_status;
     int sm_count;
+    // optional: the bf16 output pruned along its columns in the epilogue (needs scale, bf16 output, no K split)
+    void* next_values = nullptr;
+    void* next_meta = nullptr;
+    uint64_t next_seed = 0;
+    int next_joint = 0;   // 0 = App. A.2 table, 1 = systematic sampling
 };
 int launch_sparse_gemm(const SparseGemmArgs& a, cudaStream_t stream);     // returns an mvue_status
 // iters = 0: nothing is issued and the kernel's one wait expires after spin_limit polls (0: the default bound)

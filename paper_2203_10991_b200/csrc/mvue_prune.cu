@@ -21,16 +21,6 @@
 namespace mvue {
 namespace {
 
-// Byte offset of the 16-bit metadata word of (row r of A, strip = k / 16) in the tensor-core order:
-// blocks of 128 rows x 128 k (2 KiB, row-block major), inside a block 128 lanes of 16 bytes with
-// lane = r % 8 + 8 * (strip % 2) + 16 * (r % 128 / 16), word = strip % 8 / 2, half-word = r / 8 % 2.
-// This is the arrangement tcgen05.cp.128x128b moves verbatim into tensor memory for four MMAs.
-__device__ __forceinline__ int64_t tc_meta_offset(int64_t r, int64_t strip, int64_t kblocks) {
-    const int rl = (int)(r & 127), st = (int)(strip & 7);
-    const int lane = (rl & 7) + 8 * (st & 1) + 16 * (rl >> 4);
-    return ((r >> 7) * kblocks + (strip >> 3)) * 2048 + lane * 16 + (st >> 1) * 4 + ((rl >> 3) & 1) * 2;
-}
-
 __device__ __forceinline__ uint4 ldg128(const void* p) {
     return __ldg(reinterpret_cast<const uint4*>(p));
 }

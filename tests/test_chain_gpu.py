@@ -64,3 +64,24 @@ def test_overlapped_chain_gives_the_same_bits():
         torch.cuda.synchronize()
         for x, y in zip(a, b):
             assert torch.equal(x, y)
+
+
+def test_chain_with_the_prune_in_the_backward_epilogue_gives_the_same_bits():
+    # the backward products prune their own output for the layer below (same seeds, same block numbers): every dW of
+    # the chain must be bit-identical to the chain that launches those prunes separately -- alone and with the
+    # two-stream schedule; T and the layer widths make both the one-launch route and the two-step route occur
+    T, dims = 2048, [256, 2048, 512, 1024]
+    layers = []
+    for i in range(3):
+        out_f, in_f = dims[3 - i], dims[2 - i]
+        layers.append({"W": to_dev(workloads.normal_bf16((out_f, in_f), seed=70 + i, std=in_f ** -0.5)),
+                       "h": to_dev(workloads.normal_bf16((T, in_f), seed=80 + i)),
+                       "act_grad": to_dev(workloads.normal_bf16((T, in_f), seed=90 + i)) if i < 2 else None})
+    g_top = to_dev(workloads.gradient((T, dims[3]), "student_t", seed=13, dtype="bf16"))
+    for joint in (None, 1):
+        a = chain.backward_update(g_top, layers, base_seed=7, joint=joint)
+        b = chain.backward_update(g_top, layers, base_seed=7, joint=joint, prune_in_epilogue_min_k=256)
+        c = chain.backward_update(g_top, layers, base_seed=7, joint=joint, prune_in_epilogue_min_k=256, overlap=True)
+        torch.cuda.synchronize()
+        for x, y, z in zip(a, b, c):
+            assert torch.equal(x, y) and torch.equal(x, z)
