@@ -89,6 +89,12 @@ def lib() -> ctypes.CDLL:
         L.oracle_prune.restype = ctypes.c_int
         L.oracle_prune_rounded.argtypes = L.oracle_prune.argtypes + [ctypes.c_int]
         L.oracle_prune_rounded.restype = ctypes.c_int
+        L.oracle_prune_opts.argtypes = L.oracle_prune.argtypes + [ctypes.c_int, ctypes.c_int]
+        L.oracle_prune_opts.restype = ctypes.c_int
+        L.oracle_block_word16.argtypes = [ctypes.c_uint64, ctypes.c_uint64]
+        L.oracle_block_word16.restype = ctypes.c_uint32
+        L.oracle_block_word_pair16.argtypes = [ctypes.c_uint64, ctypes.c_uint64, u32p]
+        L.oracle_block_word_pair16.restype = None
         L.oracle_bf16_sr.argtypes = [ctypes.c_float, ctypes.c_uint16]
         L.oracle_bf16_sr.restype = ctypes.c_uint16
         L.oracle_rounding_bits.argtypes = [ctypes.c_uint64, ctypes.c_uint64, ctypes.c_int]
@@ -141,6 +147,17 @@ def philox4x32_10(ctr, key):
 
 def block_word(seed: int, q: int) -> int:
     return int(lib().oracle_block_word(seed & (2**64 - 1), q))
+
+
+def block_word16(seed: int, q: int) -> int:
+    """The word of block q when blocks draw sixteen bits each: those bits in the top half, zero below."""
+    return int(lib().oracle_block_word16(seed & (2**64 - 1), q))
+
+
+def block_word_pair16(seed: int, q: int):
+    out = (ctypes.c_uint32 * 2)()
+    lib().oracle_block_word_pair16(seed & (2**64 - 1), q, out)
+    return int(out[0]), int(out[1])
 
 
 def uniform24(word: int) -> float:
@@ -250,10 +267,12 @@ def rounding_bits(seed: int, unit: int, slot: int) -> int:
 
 
 def prune(g: np.ndarray, n: int, m: int, axis: int, seed: int, *, k_total: int | None = None,
-          k_offset: int = 0, threads: int = 1, joint: int = JOINT_TABLE, stochastic_rounding: bool = False):
+          k_offset: int = 0, threads: int = 1, joint: int = JOINT_TABLE, stochastic_rounding: bool = False,
+          eps16: bool = False):
     """MVUE n:m prune + pack of a 2-D array (float32, or uint16 holding bf16 bits).
     joint: the 2:4 estimator (JOINT_TABLE: App. A.2; JOINT_SYSTEMATIC; JOINT_APPROX: Sec. 4.4); ignored for 1:2.
     stochastic_rounding: survivors are rounded to bf16 stochastically (unbiased storage) instead of to nearest.
+    eps16: sixteen random bits per block (one generator call per eight blocks) instead of thirty-two.
 
     Returns (values uint16 [Mrows, K/2], meta uint8 [Mrows, K/8]) in canonical form.
     """
@@ -264,10 +283,10 @@ def prune(g: np.ndarray, n: int, m: int, axis: int, seed: int, *, k_total: int |
     k = cols if axis == 1 else rows
     values = np.zeros(vshape, dtype=np.uint16)
     meta = np.zeros(mshape, dtype=np.uint8)
-    rc = lib().oracle_prune_rounded(g.ctypes.data, int(g.dtype == np.uint16), rows, cols, cols, n, m, axis,
-                                    seed & (2**64 - 1), k if k_total is None else k_total, k_offset,
-                                    values.ctypes.data, meta.ctypes.data, max(1, threads), int(joint),
-                                    int(bool(stochastic_rounding)))
+    rc = lib().oracle_prune_opts(g.ctypes.data, int(g.dtype == np.uint16), rows, cols, cols, n, m, axis,
+                                 seed & (2**64 - 1), k if k_total is None else k_total, k_offset,
+                                 values.ctypes.data, meta.ctypes.data, max(1, threads), int(joint),
+                                 int(bool(stochastic_rounding)), int(bool(eps16)))
     if rc != 0:
         raise ValueError("oracle_prune: unsupported N:M or shape")
     return values, meta

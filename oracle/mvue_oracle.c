@@ -90,6 +90,39 @@ void oracle_block_word_pair(uint64_t seed, uint64_t q, uint32_t words[2])
     words[1] = out[2 * (q & 1u) + 1];
 }
 
+/* Sixteen random bits per block instead of thirty-two: one generator call then serves eight consecutive blocks
+ * (sixteen elements of 1:2, thirty-two of 2:4 / 1:4).  Block number q takes the low (q even) or high (q odd) half
+ * of word (q >> 1) & 3 of generator call q >> 3, and the sampler is handed those sixteen bits in the TOP half of a
+ * 32-bit word whose low half is zero -- so the block samplers themselves are unchanged, only eps has a resolution of
+ * 2^-16 (2^-15 for systematic sampling, which reads one bit less) instead of 2^-24 / 2^-23.  The paper asks only for
+ * i.i.d. eps ~ U[0,1] (App. "Pruning Overhead", Part 1); every mask probability moves by at most that resolution,
+ * still two hundred times finer than the bf16 grid the survivors are stored on. */
+uint32_t oracle_block_word16(uint64_t seed, uint64_t q)
+{
+    uint64_t call = q >> 3;
+    uint32_t ctr[4] = { (uint32_t)call, (uint32_t)(call >> 32), 0u, 0u };
+    uint32_t key[2] = { (uint32_t)seed, (uint32_t)(seed >> 32) };
+    uint32_t out[4];
+    oracle_philox4x32_10(ctr, key, out);
+    uint32_t w = out[(q >> 1) & 3u];
+    return (q & 1u) ? (w & 0xFFFF0000u) : (w << 16);
+}
+
+/* The same economy for the estimator that draws twice per block (Sec. 4.4): block q takes word q & 3 of generator
+ * call q >> 2 (one call serves four blocks instead of two), its low half for the first draw, its high half for the
+ * second, each in the top half of a word. */
+void oracle_block_word_pair16(uint64_t seed, uint64_t q, uint32_t words[2])
+{
+    uint64_t call = q >> 2;
+    uint32_t ctr[4] = { (uint32_t)call, (uint32_t)(call >> 32), 0u, 0u };
+    uint32_t key[2] = { (uint32_t)seed, (uint32_t)(seed >> 32) };
+    uint32_t out[4];
+    oracle_philox4x32_10(ctr, key, out);
+    uint32_t w = out[q & 3u];
+    words[0] = w << 16;
+    words[1] = w & 0xFFFF0000u;
+}
+
 /* eps in [0,1): the top 24 bits of the word, exactly representable. */
 float oracle_uniform24(uint32_t word)
 {
@@ -793,9 +826,17 @@ static float load_elem(const void *g, int is_bf16, int64_t off)
     return ((const float *)g)[off];
 }
 
+int oracle_prune_opts(const void *g, int is_bf16, int64_t rows, int64_t cols, int64_t ld,
+                      int n, int m, int axis, uint64_t seed, int64_t k_total, int64_t k_offset,
+                      uint16_t *values, uint8_t *meta, int threads, int joint, int stochastic_rounding, int eps16);
+
 int oracle_prune_rounded(const void *g, int is_bf16, int64_t rows, int64_t cols, int64_t ld,
                          int n, int m, int axis, uint64_t seed, int64_t k_total, int64_t k_offset,
-                         uint16_t *values, uint8_t *meta, int threads, int joint, int stochastic_rounding);
+                         uint16_t *values, uint8_t *meta, int threads, int joint, int stochastic_rounding)
+{
+    return oracle_prune_opts(g, is_bf16, rows, cols, ld, n, m, axis, seed, k_total, k_offset, values, meta, threads,
+                             joint, stochastic_rounding, 0);
+}
 
 int oracle_prune(const void *g, int is_bf16, int64_t rows, int64_t cols, int64_t ld,
                  int n, int m, int axis, uint64_t seed, int64_t k_total, int64_t k_offset,
@@ -809,9 +850,10 @@ int oracle_prune(const void *g, int is_bf16, int64_t rows, int64_t cols, int64_t
  * even), 1 rounds stochastically (oracle_bf16_sr) with the bits of oracle_rounding_bits: the survivor stored at
  * values[r][8 t + e] is slot e of unit number r (k_total / 16) + k_offset / 16 + t.  Needs K, k_total, k_offset
  * multiples of 16 then. */
-int oracle_prune_rounded(const void *g, int is_bf16, int64_t rows, int64_t cols, int64_t ld,
-                         int n, int m, int axis, uint64_t seed, int64_t k_total, int64_t k_offset,
-                         uint16_t *values, uint8_t *meta, int threads, int joint, int stochastic_rounding)
+/* eps16 = 1: the blocks draw sixteen random bits each (oracle_block_word16 / oracle_block_word_pair16). */
+int oracle_prune_opts(const void *g, int is_bf16, int64_t rows, int64_t cols, int64_t ld,
+                      int n, int m, int axis, uint64_t seed, int64_t k_total, int64_t k_offset,
+                      uint16_t *values, uint8_t *meta, int threads, int joint, int stochastic_rounding, int eps16)
 {
     const int64_t Mrows = axis == 1 ? rows : cols;
     const int64_t K     = axis == 1 ? cols : rows;
@@ -834,16 +876,18 @@ int oracle_prune_rounded(const void *g, int is_bf16, int64_t rows, int64_t cols,
                 /* one survivor, stored in the 2:4 container beside a +0: positions (i, 3), or (2, 3) when i = 3 */
                 uint64_t q = (uint64_t)r * (uint64_t)(k_total / 4) + (uint64_t)(k_offset / 4 + j);
                 float kept;
-                int i = oracle_mvue_1of4(a, oracle_block_word(seed, q), &kept);
+                int i = oracle_mvue_1of4(a, eps16 ? oracle_block_word16(seed, q) : oracle_block_word(seed, q), &kept);
                 if (i < 3) { idx[0] = i; idx[1] = 3; val[0] = kept; val[1] = 0.0f; }
                 else       { idx[0] = 2; idx[1] = 3; val[0] = 0.0f; val[1] = kept; }
             } else if (m == 4) {
                 uint64_t q = (uint64_t)r * (uint64_t)(k_total / 4) + (uint64_t)(k_offset / 4 + j);
-                if (joint == 0)      oracle_mvue_2of4(a, oracle_block_word(seed, q), idx, val);
-                else if (joint == 1) oracle_mvue_2of4_systematic(a, oracle_block_word(seed, q), idx, val);
+                const uint32_t word = joint == 2 ? 0u : eps16 ? oracle_block_word16(seed, q) : oracle_block_word(seed, q);
+                if (joint == 0)      oracle_mvue_2of4(a, word, idx, val);
+                else if (joint == 1) oracle_mvue_2of4_systematic(a, word, idx, val);
                 else {
                     uint32_t w[2];
-                    oracle_block_word_pair(seed, q, w);
+                    if (eps16) oracle_block_word_pair16(seed, q, w);
+                    else       oracle_block_word_pair(seed, q, w);
                     oracle_mvue_2of4_approx(a, w[0], w[1], idx, val);
                 }
             } else {
@@ -851,7 +895,8 @@ int oracle_prune_rounded(const void *g, int is_bf16, int64_t rows, int64_t cols,
                     uint64_t q = (uint64_t)r * (uint64_t)(k_total / 2)
                                + (uint64_t)(k_offset / 2 + 2 * j + half);
                     idx[half] = 2 * half + oracle_mvue_1of2(a[2 * half], a[2 * half + 1],
-                                                            oracle_block_word(seed, q), &val[half]);
+                                                            eps16 ? oracle_block_word16(seed, q)
+                                                                  : oracle_block_word(seed, q), &val[half]);
                 }
             }
             if (stochastic_rounding) {
