@@ -180,8 +180,15 @@ MVUE_API int mvue_prune_joint(const void* g, int dtype, int64_t rows, int64_t co
  *   + t (16 consecutive k of row r_A of A) makes one more generator call, Philox4x32-10 with counter
  *   (lo32(u), hi32(u), 1, 0) under the same key (the selection draws all have third counter word 0); the survivor stored
  *   at values[r_A][8 t + e] takes the low (e even) or high (e odd) half of word e / 2.  About 15 more instructions per
- *   block of four. */
-typedef enum { MVUE_OPT_NONE = 0, MVUE_OPT_STOCHASTIC_ROUNDING = 1 } mvue_prune_option;
+ *   block of four.
+ * MVUE_OPT_EPS16: sixteen random bits per block instead of thirty-two, so that one generator call serves eight
+ *   blocks (App. "Pruning Overhead", Part 1, asks only for i.i.d. eps ~ U[0,1]; the generator is a fifth of the
+ *   instructions of the prune).  Block q takes the low (q even) or high (q odd) half of word (q >> 1) & 3 of call
+ *   q >> 3; approx-MVUE, which draws twice per block, takes word q & 3 of call q >> 2, low half first.  The sixteen
+ *   bits are used as the top half of a word whose low half is zero, so every formula above stands with eps on a grid
+ *   of 2^-16 (2^-15 for systematic sampling): each mask probability moves by at most that, two hundred times below
+ *   the bf16 grid of the survivors.  Masks differ from those of the same call without the option. */
+typedef enum { MVUE_OPT_NONE = 0, MVUE_OPT_STOCHASTIC_ROUNDING = 1, MVUE_OPT_EPS16 = 2 } mvue_prune_option;
 MVUE_API int mvue_prune_opts(const void* g, int dtype, int64_t rows, int64_t cols, int64_t ld, int n, int m,
                     int axis, uint64_t seed, int64_t k_total, int64_t k_offset, void* values,
                     void* meta, int layout, int joint, unsigned options, void* stream);

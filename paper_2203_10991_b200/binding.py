@@ -18,7 +18,7 @@ MVUE_F32, MVUE_BF16 = 0, 1
 MVUE_LAYOUT_CANONICAL = 0
 MVUE_LAYOUT_TC = 1
 MVUE_JOINT_TABLE, MVUE_JOINT_SYSTEMATIC, MVUE_JOINT_APPROX = 0, 1, 2
-MVUE_OPT_NONE, MVUE_OPT_STOCHASTIC_ROUNDING = 0, 1
+MVUE_OPT_NONE, MVUE_OPT_STOCHASTIC_ROUNDING, MVUE_OPT_EPS16 = 0, 1, 2
 
 EXPORTS = ("mvue_version", "mvue_status_string", "mvue_last_cuda_error", "mvue_packed_sizes",
            "mvue_prune", "mvue_prune_joint", "mvue_prune_opts", "mvue_prune_4of8", "mvue_unpack", "mvue_sparse_update_gemm", "mvue_sparse_backward_gemm",

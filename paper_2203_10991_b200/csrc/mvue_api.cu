@@ -141,7 +141,7 @@ int mvue_prune_opts(const void* g, int dtype, int64_t rows, int64_t cols, int64_
                     int axis, uint64_t seed, int64_t k_total, int64_t k_offset, void* values,
                     void* meta, int layout, int joint, unsigned options, void* stream) {
     if (!g || !values || !meta) return MVUE_ERR_NULL;
-    if (options & ~(unsigned)MVUE_OPT_STOCHASTIC_ROUNDING) return MVUE_ERR_OPTION;
+    if (options & ~(unsigned)(MVUE_OPT_STOCHASTIC_ROUNDING | MVUE_OPT_EPS16)) return MVUE_ERR_OPTION;
     if (joint != MVUE_JOINT_TABLE && joint != MVUE_JOINT_SYSTEMATIC && joint != MVUE_JOINT_APPROX) return MVUE_ERR_JOINT;
     if (dtype != MVUE_F32 && dtype != MVUE_BF16) return MVUE_ERR_DTYPE;
     if (int s = mvue_packed_sizes(rows, cols, n, m, axis, layout, nullptr, nullptr)) return s;
@@ -156,7 +156,7 @@ int mvue_prune_opts(const void* g, int dtype, int64_t rows, int64_t cols, int64_
     if (int s = current_device_info(&dev)) return s;
     PruneArgs a{g, dtype == MVUE_BF16, rows, cols, ld, m, axis, seed, k_total, k_offset, values, meta, dev.sm_count,
                 layout == MVUE_LAYOUT_TC, (n == 1 && m == 4) ? 3 : joint,      // one survivor of four has a single law
-                (options & MVUE_OPT_STOCHASTIC_ROUNDING) != 0};
+                (options & MVUE_OPT_STOCHASTIC_ROUNDING) != 0, (options & MVUE_OPT_EPS16) != 0};
     cudaError_t e = launch_prune(a, reinterpret_cast<cudaStream_t>(stream));
     if (e != cudaSuccess) { set_cuda_error(e, "mvue_prune launch"); return MVUE_ERR_CUDA; }
     return MVUE_OK;

@@ -634,12 +634,52 @@ __device__ __forceinline__ int64_t tc_meta_offset(int64_t r, int64_t strip, int6
 // One work unit of bf16 input: raw[8] = 16 elements along K, two per word.
 // kJoint selects the 2:4 estimator (0: App. A.2 table, 1: systematic sampling, 2: approx-MVUE of Sec. 4.4,
 // which takes two words per block: one generator call per two blocks) or, with 3, MVUE 1:4; 1:2 has one law.
+// The random words of unit number `unit` (16 consecutive elements along K).  kWords = 4: one word per block of four
+// (2:4 with the pair table or systematic sampling, 1:4); kWords = 8: two per block (approx-MVUE) or one per pair (1:2).
+// 32 bits per word: generator call `unit` (kWords = 4) or calls 2 unit, 2 unit + 1 (kWords = 8).
+// kEps16: sixteen bits per word, handed over in the top half of a word whose low half is zero, so that one call serves
+// eight words: call unit / 2, its first or second pair of words (kWords = 4), or call `unit` (kWords = 8).
+template <int kWords, bool kEps16>
+__device__ __forceinline__ void unit_words(uint64_t unit, const RoundKeys& rk, uint32_t (&w)[kWords]) {
+    if (kWords == 4 && !kEps16) {
+        const uint4 r = philox4x32_10(unit, rk);
+        w[0] = r.x; w[1] = r.y; w[2] = r.z; w[3] = r.w;
+    } else if (kWords == 4) {
+        const uint4 r = philox4x32_10(unit >> 1, rk);
+        const bool second = (unit & 1u) != 0;
+        const uint32_t a = second ? r.z : r.x, b = second ? r.w : r.y;
+        w[0] = a << 16; w[1] = a & 0xFFFF0000u; w[2] = b << 16; w[3] = b & 0xFFFF0000u;
+    } else if (!kEps16) {
+        const uint4 ra = philox4x32_10(2 * unit, rk), rb = philox4x32_10(2 * unit + 1, rk);
+        w[0] = ra.x; w[1] = ra.y; w[2] = ra.z; w[3] = ra.w;
+        w[kWords - 4] = rb.x; w[kWords - 3] = rb.y; w[kWords - 2] = rb.z; w[kWords - 1] = rb.w;
+    } else {
+        const uint4 r = philox4x32_10(unit, rk);
+        const uint32_t x[4] = {r.x, r.y, r.z, r.w};
+#pragma unroll
+        for (int i = 0; i < 4; ++i) {
+            w[2 * i % kWords] = x[i] << 16;
+            w[(2 * i + 1) % kWords] = x[i] & 0xFFFF0000u;
+        }
+    }
+}
+// The words of the two consecutive units `unit` (even) and `unit + 1` at sixteen bits per word from their one shared call.
+__device__ __forceinline__ void unit_pair_words16(uint64_t unit, const RoundKeys& rk, uint32_t (&w0)[4], uint32_t (&w1)[4]) {
+    const uint4 r = philox4x32_10(unit >> 1, rk);
+    w0[0] = r.x << 16; w0[1] = r.x & 0xFFFF0000u; w0[2] = r.y << 16; w0[3] = r.y & 0xFFFF0000u;
+    w1[0] = r.z << 16; w1[1] = r.z & 0xFFFF0000u; w1[2] = r.w << 16; w1[3] = r.w & 0xFFFF0000u;
+}
+
+template <int M, int kJoint>
+struct UnitWords { static constexpr int kCount = (M == 2 || kJoint == 2) ? 8 : 4; };
+
+// One work unit with its random words given (UnitWords<M, kJoint>::kCount of them).
 // kSR: survivors are rounded to bf16 stochastically; the unit's eight slots draw their 16 bits each from one more
 // generator call, numbered by the unit itself on stream 1 (group j's two slots: word j).
-template <int M, int kJoint = 0, bool kSR = false>
-__device__ __forceinline__ void prune_unit_bf16(const uint32_t (&raw)[8], uint64_t unit_index,
-                                                const RoundKeys& rk, uint4* out_values,
-                                                uint32_t* out_meta) {
+template <int M, int kJoint, bool kSR>
+__device__ __forceinline__ void prune_unit_bf16_w(const uint32_t (&raw)[8], const uint32_t (&words)[UnitWords<M, kJoint>::kCount],
+                                                  uint64_t unit_index, const RoundKeys& rk, uint4* out_values,
+                                                  uint32_t* out_meta) {
     uint32_t v[4];                                   // 8 survivors, two bf16 per word
     uint32_t meta = 0;
     uint32_t rnd[4] = {0u, 0u, 0u, 0u};
@@ -648,8 +688,6 @@ __device__ __forceinline__ void prune_unit_bf16(const uint32_t (&raw)[8], uint64
         rnd[0] = r.x; rnd[1] = r.y; rnd[2] = r.z; rnd[3] = r.w;
     }
     if (M == 4 && kJoint == 3) {                      // MVUE 1:4: one word per block, as for 2:4
-        const uint4 w = philox4x32_10(unit_index, rk);
-        const uint32_t words[4] = {w.x, w.y, w.z, w.w};
 #pragma unroll
         for (int j = 0; j < 4; ++j) {
             uint32_t nib;
@@ -658,24 +696,21 @@ __device__ __forceinline__ void prune_unit_bf16(const uint32_t (&raw)[8], uint64
             meta += nib << (4 * j);
         }
     } else if (M == 4 && kJoint == 2) {
-        const uint4 wa = philox4x32_10(2 * unit_index, rk);
-        const uint4 wb = philox4x32_10(2 * unit_index + 1, rk);
-        const uint32_t words[8] = {wa.x, wa.y, wa.z, wa.w, wb.x, wb.y, wb.z, wb.w};
 #pragma unroll
         for (int j = 0; j < 4; ++j) {
             uint32_t nib;
-            mvue_2of4_approx_bf16<kSR>(raw[2 * j], raw[2 * j + 1], words[2 * j], words[2 * j + 1], &v[j], &nib, rnd[j]);
+            mvue_2of4_approx_bf16<kSR>(raw[2 * j], raw[2 * j + 1], words[(2 * j) % UnitWords<M, kJoint>::kCount],
+                                       words[(2 * j + 1) % UnitWords<M, kJoint>::kCount], &v[j], &nib, rnd[j]);
             meta += nib << (4 * j);
         }
     } else if (M == 4 && kJoint == 1) {                // systematic sampling: the unit's four blocks two at a time
-        const uint4 w = philox4x32_10(unit_index, rk);
         uint32_t nib[4];
-        mvue_2of4_sys_bf16_x2<kSR>(raw[0], raw[1], raw[2], raw[3], w.x, w.y, &v[0], &v[1], &nib[0], &nib[1], rnd[0], rnd[1]);
-        mvue_2of4_sys_bf16_x2<kSR>(raw[4], raw[5], raw[6], raw[7], w.z, w.w, &v[2], &v[3], &nib[2], &nib[3], rnd[2], rnd[3]);
+        mvue_2of4_sys_bf16_x2<kSR>(raw[0], raw[1], raw[2], raw[3], words[0], words[1], &v[0], &v[1], &nib[0], &nib[1],
+                                   rnd[0], rnd[1]);
+        mvue_2of4_sys_bf16_x2<kSR>(raw[4], raw[5], raw[6], raw[7], words[2], words[3], &v[2], &v[3], &nib[2], &nib[3],
+                                   rnd[2], rnd[3]);
         meta = nib[0] + (nib[1] << 4) + (nib[2] << 8) + (nib[3] << 12);
     } else if (M == 4) {
-        const uint4 w = philox4x32_10(unit_index, rk);
-        const uint32_t words[4] = {w.x, w.y, w.z, w.w};
 #pragma unroll
         for (int j = 0; j < 4; ++j) {
             uint32_t nib;
@@ -684,18 +719,25 @@ __device__ __forceinline__ void prune_unit_bf16(const uint32_t (&raw)[8], uint64
             meta += nib << (4 * j);
         }
     } else {
-        const uint4 wa = philox4x32_10(2 * unit_index, rk);
-        const uint4 wb = philox4x32_10(2 * unit_index + 1, rk);
-        const uint32_t words[8] = {wa.x, wa.y, wa.z, wa.w, wb.x, wb.y, wb.z, wb.w};
 #pragma unroll
         for (int j = 0; j < 4; ++j) {
             uint32_t nib;
-            mvue_1of2x2_bf16<kSR>(raw[2 * j], raw[2 * j + 1], words[2 * j], words[2 * j + 1], &v[j], &nib, rnd[j]);
+            mvue_1of2x2_bf16<kSR>(raw[2 * j], raw[2 * j + 1], words[(2 * j) % UnitWords<M, kJoint>::kCount],
+                                  words[(2 * j + 1) % UnitWords<M, kJoint>::kCount], &v[j], &nib, rnd[j]);
             meta += nib << (4 * j);
         }
     }
     *out_values = make_uint4(v[0], v[1], v[2], v[3]);
     *out_meta = meta;
+}
+
+template <int M, int kJoint = 0, bool kSR = false, bool kEps16 = false>
+__device__ __forceinline__ void prune_unit_bf16(const uint32_t (&raw)[8], uint64_t unit_index,
+                                                const RoundKeys& rk, uint4* out_values,
+                                                uint32_t* out_meta) {
+    uint32_t words[UnitWords<M, kJoint>::kCount];
+    unit_words<UnitWords<M, kJoint>::kCount, kEps16>(unit_index, rk, words);
+    prune_unit_bf16_w<M, kJoint, kSR>(raw, words, unit_index, rk, out_values, out_meta);
 }
 
 // One work unit whose 16 elements are the half kHigh of 16 row words (K runs down the rows of g).

@@ -22,6 +22,7 @@ struct PruneArgs {
     bool tc_layout;      // metadata in tensor-core order instead of canonical rows
     int joint;           // 2:4 estimator: 0 = App. A.2 table, 1 = systematic sampling, 2 = approx-MVUE (Sec. 4.4); 3 = MVUE 1:4
     bool stochastic_rounding = false;   // survivors rounded to bf16 stochastically (unbiased storage) instead of to nearest
+    bool eps16 = false;                 // sixteen random bits per block: one generator call per eight blocks
 };
 
 cudaError_t launch_prune(const PruneArgs& a, cudaStream_t stream);

@@ -26,10 +26,11 @@ __device__ __forceinline__ uint4 ldg128(const void* p) {
 }
 
 // One work unit of binary32 input: b[16] = bit patterns of 16 elements along K.
-template <int M, int kJoint = 0, bool kSR = false>
+template <int M, int kJoint = 0, bool kSR = false, bool kEps16 = false>
 __device__ __forceinline__ void prune_unit_f32(const uint32_t (&b)[16], uint64_t unit_index,
                                                const RoundKeys& rk, uint4* out_values,
                                                uint32_t* out_meta) {
+    constexpr int kW = UnitWords<M, kJoint>::kCount;
     uint32_t v[4];
     uint32_t meta = 0;
     uint32_t rnd[4] = {0u, 0u, 0u, 0u};              // stochastic rounding: 16 bits per survivor slot, stream 1 of the unit
@@ -37,48 +38,28 @@ __device__ __forceinline__ void prune_unit_f32(const uint32_t (&b)[16], uint64_t
         const uint4 r = philox4x32_10(unit_index, rk, 1u);
         rnd[0] = r.x; rnd[1] = r.y; rnd[2] = r.z; rnd[3] = r.w;
     }
-    if (M == 4 && kJoint == 3) {
-        const uint4 w = philox4x32_10(unit_index, rk);
-        const uint32_t words[4] = {w.x, w.y, w.z, w.w};
+    uint32_t words[kW];
+    unit_words<kW, kEps16>(unit_index, rk, words);
 #pragma unroll
-        for (int j = 0; j < 4; ++j) {
-            uint32_t nib;
+    for (int j = 0; j < 4; ++j) {
+        uint32_t nib;
+        if (M == 4 && kJoint == 3) {
             mvue_1of4_f32<kSR>(b[4 * j], b[4 * j + 1], b[4 * j + 2], b[4 * j + 3], words[j], &v[j], &nib, rnd[j]);
-            meta |= nib << (4 * j);
-        }
-    } else if (M == 4 && kJoint == 2) {
-        const uint4 wa = philox4x32_10(2 * unit_index, rk);
-        const uint4 wb = philox4x32_10(2 * unit_index + 1, rk);
-        const uint32_t words[8] = {wa.x, wa.y, wa.z, wa.w, wb.x, wb.y, wb.z, wb.w};
-#pragma unroll
-        for (int j = 0; j < 4; ++j) {
-            uint32_t nib;
-            mvue_2of4_approx_f32<kSR>(b[4 * j], b[4 * j + 1], b[4 * j + 2], b[4 * j + 3], words[2 * j], words[2 * j + 1],
-                                      &v[j], &nib, rnd[j]);
-            meta |= nib << (4 * j);
-        }
-    } else if (M == 4) {
-        const uint4 w = philox4x32_10(unit_index, rk);
-        const uint32_t words[4] = {w.x, w.y, w.z, w.w};
-#pragma unroll
-        for (int j = 0; j < 4; ++j) {
-            uint32_t nib;
-            if (kJoint == 0) mvue_2of4_f32<kSR>(b[4 * j], b[4 * j + 1], b[4 * j + 2], b[4 * j + 3], words[j], &v[j], &nib, rnd[j]);
-            else             mvue_2of4_sys_f32<kSR>(b[4 * j], b[4 * j + 1], b[4 * j + 2], b[4 * j + 3], words[j], &v[j], &nib, rnd[j]);
-            meta |= nib << (4 * j);
-        }
-    } else {
-        const uint4 wa = philox4x32_10(2 * unit_index, rk);
-        const uint4 wb = philox4x32_10(2 * unit_index + 1, rk);
-        const uint32_t words[8] = {wa.x, wa.y, wa.z, wa.w, wb.x, wb.y, wb.z, wb.w};
-#pragma unroll
-        for (int j = 0; j < 4; ++j) {
+        } else if (M == 4 && kJoint == 2) {
+            mvue_2of4_approx_f32<kSR>(b[4 * j], b[4 * j + 1], b[4 * j + 2], b[4 * j + 3], words[(2 * j) % kW],
+                                      words[(2 * j + 1) % kW], &v[j], &nib, rnd[j]);
+        } else if (M == 4 && kJoint == 1) {
+            mvue_2of4_sys_f32<kSR>(b[4 * j], b[4 * j + 1], b[4 * j + 2], b[4 * j + 3], words[j], &v[j], &nib, rnd[j]);
+        } else if (M == 4) {
+            mvue_2of4_f32<kSR>(b[4 * j], b[4 * j + 1], b[4 * j + 2], b[4 * j + 3], words[j], &v[j], &nib, rnd[j]);
+        } else {
             float v0, v1;
-            const bool k0 = mvue_1of2(__uint_as_float(b[4 * j]), __uint_as_float(b[4 * j + 1]), words[2 * j], &v0);
-            const bool k1 = mvue_1of2(__uint_as_float(b[4 * j + 2]), __uint_as_float(b[4 * j + 3]), words[2 * j + 1], &v1);
+            const bool k0 = mvue_1of2(__uint_as_float(b[4 * j]), __uint_as_float(b[4 * j + 1]), words[(2 * j) % kW], &v0);
+            const bool k1 = mvue_1of2(__uint_as_float(b[4 * j + 2]), __uint_as_float(b[4 * j + 3]), words[(2 * j + 1) % kW], &v1);
             v[j] = pack_out<kSR>(v0, v1, rnd[j]);
-            meta |= (k0 ? 0u : (1u << (4 * j))) | (k1 ? (8u << (4 * j)) : (12u << (4 * j)));
+            nib = (k0 ? 0u : 1u) | (k1 ? 8u : 12u);
         }
+        meta |= nib << (4 * j);
     }
     *out_values = make_uint4(v[0], v[1], v[2], v[3]);
     *out_meta = meta;
@@ -103,7 +84,7 @@ __device__ __forceinline__ void ldg256(const char* p, uint32_t (&v)[8]) {
     }
 }
 
-template <int M, bool kBf16, bool kTC, int kJoint, bool kSR>
+template <int M, bool kBf16, bool kTC, int kJoint, bool kSR, bool kEps16>
 __global__ void __launch_bounds__(8 * kA1Units, kBf16 ? 12 : 8)
 prune_axis1_kernel(const void* __restrict__ g, int64_t n_rows, int units_per_row, int64_t ld,
                    int64_t units_per_row_total, int64_t unit_offset, RoundKeys rk,
@@ -139,7 +120,7 @@ prune_axis1_kernel(const void* __restrict__ g, int64_t n_rows, int units_per_row
                 if (!kBothFirst) ldg256(reinterpret_cast<const char*>(g) + (r * ld + (int64_t)c * 16) * 2, raw[h]);
                 const uint64_t unit = (uint64_t)r * (uint64_t)units_per_row_total + (uint64_t)(unit_offset + c);
                 uint4 v;
-                prune_unit_bf16<M, kJoint, kSR>(raw[h], unit, rk, &v, &mt);
+                prune_unit_bf16<M, kJoint, kSR, kEps16>(raw[h], unit, rk, &v, &mt);
                 values[r * units_per_row + c] = v;
                 if (!kTC) meta[r * units_per_row + c] = (uint16_t)mt;
             }
@@ -159,7 +140,7 @@ prune_axis1_kernel(const void* __restrict__ g, int64_t n_rows, int units_per_row
                                         hi[0], hi[1], hi[2], hi[3], hi[4], hi[5], hi[6], hi[7]};
                 const uint64_t unit = (uint64_t)r * (uint64_t)units_per_row_total + (uint64_t)(unit_offset + c);
                 uint4 v;
-                prune_unit_f32<M, kJoint, kSR>(b, unit, rk, &v, &mt);
+                prune_unit_f32<M, kJoint, kSR, kEps16>(b, unit, rk, &v, &mt);
                 values[r * units_per_row + c] = v;
                 if (!kTC) meta[r * units_per_row + c] = (uint16_t)mt;
             }
@@ -187,7 +168,7 @@ __device__ __forceinline__ uint32_t smem_addr(const void* p) {
 }
 
 // (Used for binary32 input; bf16 input takes prune_axis0_bf16_kernel below.)
-template <int M, bool kBf16, bool kTC, int kJoint, bool kSR>
+template <int M, bool kBf16, bool kTC, int kJoint, bool kSR, bool kEps16>
 __global__ void __launch_bounds__(kTileStrips * 32, kBf16 ? 3 : 2)
 prune_axis0_kernel(const void* __restrict__ g, int64_t n_strips, int64_t n_cols, int64_t ld,
                    int64_t units_per_row_total, int64_t unit_offset, RoundKeys rk,
@@ -239,7 +220,7 @@ prune_axis0_kernel(const void* __restrict__ g, int64_t n_strips, int64_t n_cols,
                 uint32_t b[16];
 #pragma unroll
                 for (int i = 0; i < 16; ++i) b[i] = w[i][kBf16 ? 0 : e];
-                prune_unit_f32<M, kJoint, kSR>(b, unit, rk, &v, &mt);
+                prune_unit_f32<M, kJoint, kSR, kEps16>(b, unit, rk, &v, &mt);
             }
             s_val[col_l * kTileStrips + (strip_l ^ (lane & 15))] = v;
             if (kTC) {
@@ -324,7 +305,7 @@ __device__ __noinline__ void fill_tile_bf16(const char* g, int64_t ld, int64_t n
     }
 }
 
-template <int M, bool kTC, int kJoint, bool kSR, int kStrips, int kWarps>
+template <int M, bool kTC, int kJoint, bool kSR, bool kEps16, int kStrips, int kWarps>
 __global__ void __launch_bounds__(32 * kWarps, A0<kStrips, kWarps>::kBlocksPerSM)
 prune_axis0_bf16_kernel(const __grid_constant__ CUtensorMap map_g, const void* __restrict__ g, int64_t n_strips,
                         int64_t n_cols, int64_t ld, int64_t units_per_row_total, int64_t unit_offset, RoundKeys rk,
@@ -391,7 +372,7 @@ prune_axis0_bf16_kernel(const __grid_constant__ CUtensorMap map_g, const void* _
                 if (strip_ok && c < n_cols) {
                     const uint64_t unit = (uint64_t)c * (uint64_t)units_per_row_total + (uint64_t)(unit_offset + strip);
                     uint4 v;
-                    prune_unit_bf16<M, kJoint, kSR>(raw, unit, rk, &v, &mt);
+                    prune_unit_bf16<M, kJoint, kSR, kEps16>(raw, unit, rk, &v, &mt);
                     values[c * n_strips + strip] = v;
                     if (!kTC) meta[c * n_strips + strip] = (uint16_t)mt;
                 }
@@ -429,7 +410,7 @@ __device__ __noinline__ void fill_whole_tile_bf16(const char* g, int64_t ld, int
     }
 }
 
-template <int M, bool kTC, int kJoint, bool kSR>
+template <int M, bool kTC, int kJoint, bool kSR, bool kEps16>
 __global__ void __launch_bounds__(32 * kWTWarps, 12)
 prune_axis0_bf16_whole_tiles_kernel(const __grid_constant__ CUtensorMap map_g, const void* __restrict__ g, int64_t n_strips,
                                     int64_t ld, int64_t units_per_row_total, int64_t unit_offset, RoundKeys rk,
@@ -486,8 +467,17 @@ prune_axis0_bf16_whole_tiles_kernel(const __grid_constant__ CUtensorMap map_g, c
         }
         uint4 v[2];
         uint32_t mt[2];
+        if (kEps16 && UnitWords<M, kJoint>::kCount == 4) {    // the lane's two units share one generator call (unit is even)
+            uint32_t w0[4], w1[4];
+            unit_pair_words16(unit, rk, w0, w1);
+            prune_unit_bf16_w<M, kJoint, kSR>(raw[0], reinterpret_cast<const uint32_t (&)[UnitWords<M, kJoint>::kCount]>(w0),
+                                              unit, rk, &v[0], &mt[0]);
+            prune_unit_bf16_w<M, kJoint, kSR>(raw[1], reinterpret_cast<const uint32_t (&)[UnitWords<M, kJoint>::kCount]>(w1),
+                                              unit + 1, rk, &v[1], &mt[1]);
+        } else {
 #pragma unroll
-        for (int h = 0; h < 2; ++h) prune_unit_bf16<M, kJoint, kSR>(raw[h], unit + h, rk, &v[h], &mt[h]);
+            for (int h = 0; h < 2; ++h) prune_unit_bf16<M, kJoint, kSR, kEps16>(raw[h], unit + h, rk, &v[h], &mt[h]);
+        }
         uint4* dst = values + c * n_strips + strip;                          // 32-byte aligned: n_strips and strip are even
         asm volatile("st.global.v8.b32 [%0], {%1, %2, %3, %4, %5, %6, %7, %8};"
                      ::"l"(dst), "r"(v[0].x), "r"(v[0].y), "r"(v[0].z), "r"(v[0].w), "r"(v[1].x), "r"(v[1].y),
@@ -584,7 +574,7 @@ unpack_kernel(const uint4* __restrict__ values, const uint16_t* __restrict__ met
     }
 }
 
-template <int M, bool kBf16, bool kTC, int kJoint, bool kSR>
+template <int M, bool kBf16, bool kTC, int kJoint, bool kSR, bool kEps16>
 cudaError_t launch_prune_t(const PruneArgs& a, cudaStream_t stream) {
     const RoundKeys rk = make_round_keys(a.seed);
     const int64_t upr_total = a.k_total / 16, uoff = a.k_offset / 16;
@@ -595,7 +585,7 @@ cudaError_t launch_prune_t(const PruneArgs& a, cudaStream_t stream) {
         // in tensor-core order the rows of A are padded to 128: the blocks past the last row write only metadata
         const int64_t cover_rows = kTC ? ((a.rows + 127) / 128) * 128 : a.rows;
         dim3 grid((unsigned)((cover_rows + 15) / 16), (unsigned)((upr + kA1Units - 1) / kA1Units));
-        prune_axis1_kernel<M, kBf16, kTC, kJoint, kSR><<<grid, 8 * kA1Units, 0, stream>>>(
+        prune_axis1_kernel<M, kBf16, kTC, kJoint, kSR, kEps16><<<grid, 8 * kA1Units, 0, stream>>>(
             a.g, a.rows, (int)upr, a.ld, upr_total, uoff, rk, values, meta);
     } else {
         const int64_t n_strips = a.rows / 16;
@@ -604,7 +594,9 @@ cudaError_t launch_prune_t(const PruneArgs& a, cudaStream_t stream) {
         dim3 grid((unsigned)((n_strips + kTileStrips - 1) / kTileStrips),
                   (unsigned)((cover_cols + kTileCols - 1) / kTileCols));
         // whole tiles of 128 rows x 64 columns (and no padding rows of A to cover): the kernel without bounds checks
-        if (kBf16 && a.rows % kWTRows == 0 && a.cols % kWTCols == 0 && cover_cols == a.cols &&
+        // (with sixteen bits per block a lane's two units share a generator call: they must be units 2 i, 2 i + 1)
+        const bool pairs_aligned = !kEps16 || UnitWords<M, kJoint>::kCount != 4 || (uoff % 2 == 0 && upr_total % 2 == 0);
+        if (kBf16 && a.rows % kWTRows == 0 && a.cols % kWTCols == 0 && cover_cols == a.cols && pairs_aligned &&
             reinterpret_cast<uintptr_t>(a.values) % 32 == 0) {
             CUtensorMap map_g;
             memset(&map_g, 0, sizeof(map_g));
@@ -613,7 +605,7 @@ cudaError_t launch_prune_t(const PruneArgs& a, cudaStream_t stream) {
             const unsigned row_tiles = (unsigned)(a.rows / kWTRows), col_tiles = (unsigned)(a.cols / kWTCols);
             const bool col_fast = col_tiles <= 8 && row_tiles <= 65535u;    // (the second grid dimension is 16 bits wide)
             const dim3 grid_w = col_fast ? dim3(col_tiles, row_tiles) : dim3(row_tiles, col_tiles);
-            prune_axis0_bf16_whole_tiles_kernel<M, kTC, kJoint, kSR><<<grid_w, 32 * kWTWarps, 0, stream>>>(
+            prune_axis0_bf16_whole_tiles_kernel<M, kTC, kJoint, kSR, kEps16><<<grid_w, 32 * kWTWarps, 0, stream>>>(
                 map_g, a.g, n_strips, a.ld, upr_total, uoff, rk, values, meta, col_fast ? 1 : 0);
         } else if (kBf16) {
             CUtensorMap map_g;
@@ -623,33 +615,37 @@ cudaError_t launch_prune_t(const PruneArgs& a, cudaStream_t stream) {
                 return cudaErrorInvalidValue;
             static PerDeviceOnce once;
             const cudaError_t attr_err = once_per_device(once, [](int) {
-                return cudaFuncSetAttribute(prune_axis0_bf16_kernel<M, kTC, kJoint, kSR, kS, kW>,
+                return cudaFuncSetAttribute(prune_axis0_bf16_kernel<M, kTC, kJoint, kSR, kEps16, kS, kW>,
                                             cudaFuncAttributeMaxDynamicSharedMemorySize, A0<kS, kW>::kSmemBytes);
             });
             if (attr_err != cudaSuccess) return attr_err;
             dim3 grid_b((unsigned)((n_strips + kS - 1) / kS), (unsigned)((cover_cols + kA0Cols - 1) / kA0Cols));
-            prune_axis0_bf16_kernel<M, kTC, kJoint, kSR, kS, kW><<<grid_b, A0<kS, kW>::kThreads, A0<kS, kW>::kSmemBytes, stream>>>(
+            prune_axis0_bf16_kernel<M, kTC, kJoint, kSR, kEps16, kS, kW><<<grid_b, A0<kS, kW>::kThreads, A0<kS, kW>::kSmemBytes, stream>>>(
                 map_g, a.g, n_strips, a.cols, a.ld, upr_total, uoff, rk, values, meta);
         } else {
-            prune_axis0_kernel<M, false, kTC, kJoint, kSR><<<grid, kTileStrips * 32, 0, stream>>>(
+            prune_axis0_kernel<M, false, kTC, kJoint, kSR, kEps16><<<grid, kTileStrips * 32, 0, stream>>>(
                 a.g, n_strips, a.cols, a.ld, upr_total, uoff, rk, values, meta);
         }
     }
     return cudaGetLastError();
 }
 
-template <int M, int kJoint, bool kSR>
+template <int M, int kJoint, bool kSR, bool kEps16>
 cudaError_t launch_prune_r(const PruneArgs& a, cudaStream_t stream) {
     if (a.tc_layout)
-        return a.is_bf16 ? launch_prune_t<M, true, true, kJoint, kSR>(a, stream)
-                         : launch_prune_t<M, false, true, kJoint, kSR>(a, stream);
-    return a.is_bf16 ? launch_prune_t<M, true, false, kJoint, kSR>(a, stream)
-                     : launch_prune_t<M, false, false, kJoint, kSR>(a, stream);
+        return a.is_bf16 ? launch_prune_t<M, true, true, kJoint, kSR, kEps16>(a, stream)
+                         : launch_prune_t<M, false, true, kJoint, kSR, kEps16>(a, stream);
+    return a.is_bf16 ? launch_prune_t<M, true, false, kJoint, kSR, kEps16>(a, stream)
+                     : launch_prune_t<M, false, false, kJoint, kSR, kEps16>(a, stream);
 }
 
 template <int M, int kJoint>
 cudaError_t launch_prune_m(const PruneArgs& a, cudaStream_t stream) {
-    return a.stochastic_rounding ? launch_prune_r<M, kJoint, true>(a, stream) : launch_prune_r<M, kJoint, false>(a, stream);
+    if (a.eps16)
+        return a.stochastic_rounding ? launch_prune_r<M, kJoint, true, true>(a, stream)
+                                     : launch_prune_r<M, kJoint, false, true>(a, stream);
+    return a.stochastic_rounding ? launch_prune_r<M, kJoint, true, false>(a, stream)
+                                 : launch_prune_r<M, kJoint, false, false>(a, stream);
 }
 
 }  // namespace
