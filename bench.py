@@ -152,7 +152,7 @@ class ClockSampler:
 
 
 # --------------------------------------------------------------------------- CPU oracle arm
-def oracle_sample(cfg, n, m, sample_rows: int, joint: int = 0, prune_repeats: int = 1):
+def oracle_sample(cfg, n, m, sample_rows: int, joint: int = 0, prune_repeats: int = 1, eps16: bool = False):
     """One pass of the oracle, as it stands, over the first `sample_rows` token rows: prune+pack (repeated
     `prune_repeats` times so that the timed work is seconds, not milliseconds), unpack, and the fp64 plain-loop update
     product.  Returns (GB/s of the prune+pack's algorithmic bytes, GB/s of one whole pass, threads, seconds of one
@@ -164,7 +164,8 @@ def oracle_sample(cfg, n, m, sample_rows: int, joint: int = 0, prune_repeats: in
     threads = oracle.host_threads()
     t0 = time.perf_counter()
     for rep in range(prune_repeats):
-        values, meta = oracle.prune(g, n, m, axis=0, seed=rep, k_total=cfg["T"], k_offset=0, threads=threads, joint=joint)
+        values, meta = oracle.prune(g, n, m, axis=0, seed=rep, k_total=cfg["T"], k_offset=0, threads=threads, joint=joint,
+                                    eps16=eps16)
     t1 = time.perf_counter()
     oracle.gemm(oracle.unpack(values, meta), h, threads=threads)
     t2 = time.perf_counter()
@@ -183,15 +184,15 @@ def run_reference(args, cfg, n, m):
     per_step_s = 60.0 / max(1, args.steps + args.warmup)
     sample_rows = 512
     while sample_rows * 2 <= cfg["T"]:
-        dt_probe = oracle_sample(cfg, n, m, sample_rows, joint)[3]
+        dt_probe = oracle_sample(cfg, n, m, sample_rows, joint, eps16=args.eps16)[3]
         if dt_probe > per_step_s / 3:
             break
         sample_rows *= 2
     for _ in range(args.warmup):
-        oracle_sample(cfg, n, m, sample_rows, joint)
+        oracle_sample(cfg, n, m, sample_rows, joint, eps16=args.eps16)
     vals, steps_gbs, t_all, threads = [], [], 0.0, 1
     for _ in range(args.steps):
-        p_gbs, s_gbs, threads, dt, _ = oracle_sample(cfg, n, m, sample_rows, joint, prune_repeats=20)
+        p_gbs, s_gbs, threads, dt, _ = oracle_sample(cfg, n, m, sample_rows, joint, prune_repeats=20, eps16=args.eps16)
         vals.append(p_gbs)
         steps_gbs.append(s_gbs)
         t_all += dt
@@ -202,8 +203,8 @@ def run_reference(args, cfg, n, m):
         "impl": "reference", "metric": METRIC, "value": value, "unit": "GB/s", "n_gpus": args.gpus,
         "steps": args.steps, "warmup": args.warmup, "ms_per_step": 1e3 * t_all / max(1, args.steps),
         "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "bf16", "data": "synthetic",
-        "config": {"workload": args.workload, "prune": f"{n}:{m}", "joint": args.joint, "axis": 0,
-                   "sample_rows": sample_rows},
+        "config": {"workload": args.workload, "prune": f"{n}:{m}", "joint": args.joint,
+                   "random_bits_per_block": 16 if args.eps16 else 32, "axis": 0, "sample_rows": sample_rows},
         "step_gbs": float(np.mean(steps_gbs)),
         "cpu_baseline": {"value": value, "unit": "GB/s", "cores": threads, "kind": "oracle", "sample": sample},
         "e2e": {"value": value, "unit": "GB/s", "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
@@ -346,7 +347,8 @@ def run_ours(args, cfg, n, m):
               "approx": binding.MVUE_JOINT_APPROX}
     joint = [joints[args.joint]]                        # cells, so that the other estimators can be timed with the same step
     nm = [(n, m)]
-    opts = [binding.MVUE_OPT_NONE]
+    base_opt = binding.MVUE_OPT_EPS16 if args.eps16 else binding.MVUE_OPT_NONE
+    opts = [base_opt]
 
     def step(i, ev=None):
         if ev:
@@ -419,17 +421,19 @@ def run_ours(args, cfg, n, m):
     others = []
     if extras and m == 4:
         k2 = max(20, min(args.steps, 200))
-        variants = [(name, (2, 4), jid, 0) for name, jid in joints.items() if name != args.joint]
-        variants += [("1:2", (1, 2), joints[args.joint], 0), ("1:4", (1, 4), joints[args.joint], 0),
+        variants = [(name, (2, 4), jid, base_opt) for name, jid in joints.items() if name != args.joint]
+        variants += [("1:2", (1, 2), joints[args.joint], base_opt), ("1:4", (1, 4), joints[args.joint], base_opt),
                      # the step's law with the survivors rounded to bf16 stochastically (unbiased storage)
-                     ("stochastic_rounding", (2, 4), joints[args.joint], binding.MVUE_OPT_STOCHASTIC_ROUNDING)]
+                     ("stochastic_rounding", (2, 4), joints[args.joint], base_opt | binding.MVUE_OPT_STOCHASTIC_ROUNDING),
+                     # and with the other width of the random stream (32 bits per block if the step draws 16, and back)
+                     ("eps32" if args.eps16 else "eps16", (2, 4), joints[args.joint], base_opt ^ binding.MVUE_OPT_EPS16)]
         for name, nm_v, jid, opt in variants:
             joint[0], nm[0], opts[0] = jid, nm_v, opt
             for i in range(3):
                 step(i)
             pt, _ = step_kernel_times(k2)
             others.append((name, float(np.mean(pt)), float(np.min(pt)), k2))
-        joint[0], nm[0], opts[0] = joints[args.joint], (n, m), binding.MVUE_OPT_NONE
+        joint[0], nm[0], opts[0] = joints[args.joint], (n, m), base_opt
 
     # the step's prune timed alone (no product in between), L2-cold: inputs rotated over copies of g that together
     # exceed 2.5 x L2
@@ -440,7 +444,8 @@ def run_ours(args, cfg, n, m):
         it = [0]
 
         def prune_rot():
-            binding.mvue_prune(gs[it[0] % copies], n, m, 0, it[0], values=values, meta=meta, layout=TC, joint=joint[0])
+            binding.mvue_prune(gs[it[0] % copies], n, m, 0, it[0], values=values, meta=meta, layout=TC, joint=joint[0],
+                               options=base_opt)
             it[0] += 1
         alone_loop = tm.loop(prune_rot, max(20, min(args.steps, 100)))
         alone_mean, alone_best = tm.each(prune_rot, 20, flush=False)
@@ -492,7 +497,8 @@ def run_ours(args, cfg, n, m):
             "warmup": warm, "ms_per_step": ms_per_step, "higher_is_better": True, "scaling": "weak",
             "vs_baseline": None, "dtype": "bf16", "data": "synthetic",
             "config": {"workload": args.workload, "g": [T, out], "h": [T, inp], "g_dtype": cfg["g_dtype"],
-                       "prune": f"{n}:{m}", "joint": args.joint, "axis": 0, "dW_dtype": "f32",
+                       "prune": f"{n}:{m}", "joint": args.joint, "random_bits_per_block": 16 if args.eps16 else 32,
+                       "axis": 0, "dW_dtype": "f32",
                        "value_is": "prune+pack kernel GB/s (algorithmic bytes: g read, survivors + metadata written) "
                                    "measured inside the step, mean over the timed steps",
                        "k_total": k_total, "k_offset_of_rank0": 0,
@@ -536,16 +542,16 @@ def run_ours(args, cfg, n, m):
             line["sparse_issue_rate_cold_tflops"] = issue_cold
             line["linear_small"] = linear_small_case(tm, peaks)
             line["ffn_768"] = ffn_768_case(tm, peaks, issue_cold, joint[0])
-            line["ffn_large"] = tensor_bound_case(tm, n, m, peaks, joint[0], issue_cold)
+            line["ffn_large"] = tensor_bound_case(tm, n, m, peaks, joint[0], issue_cold, base_opt)
             line["mlp_stack"] = chain_case(n, m)
             line["prune_sweep"] = prune_sweep(peaks, sizes_log2=(26, 29, 32) if not args.sweep else range(20, 33),
-                                              step_joint=joint[0])
+                                              step_joint=joint[0], options=base_opt)
         if solo and args.gemm_shapes:
             line["gemm_shapes"] = gemm_shapes_case(tm, peaks, issue_cold)
         if solo and not args.no_cpu_baseline:
             sample_rows = min(T, 65536)
             reps = 200
-            p_gbs, s_gbs, threads, dt, dt_prune = oracle_sample(cfg, n, m, sample_rows, joint[0], prune_repeats=reps)
+            p_gbs, s_gbs, threads, dt, dt_prune = oracle_sample(cfg, n, m, sample_rows, joint[0], prune_repeats=reps, eps16=args.eps16)
             line["cpu_baseline"] = {"value": p_gbs, "unit": "GB/s", "cores": threads, "kind": "oracle",
                                     "step_gbs": s_gbs,
                                     "sample": f"first {sample_rows} of {T} token rows: MVUE {n}:{m} prune+pack, {reps} passes "
@@ -641,7 +647,7 @@ def ffn_768_case(tm: Timer, peaks, issue_cold, joint):
     return res
 
 
-def tensor_bound_case(tm: Timer, n, m, peaks, joint, issue_cold):
+def tensor_bound_case(tm: Timer, n, m, peaks, joint, issue_cold, base_opt=0):
     """The large FFN layer (tokens 16384, 4096 -> 14336): the shape on which the sparse product is bound by
     the tensor cores, timed kernel by kernel next to dense cuBLAS.  Rides along in the JSON line."""
     import torch
@@ -656,15 +662,16 @@ def tensor_bound_case(tm: Timer, n, m, peaks, joint, issue_cold):
     ws = torch.empty(max(16, binding.mvue_gemm_workspace_bytes(0, out, inp, T)), dtype=torch.uint8, device="cuda")
     pb = prune_bytes(T, out, 2)
 
-    def prune_with(nm, j):
-        return lambda: binding.mvue_prune(g, nm[0], nm[1], 0, 1, values=values, meta=meta, layout=TC, joint=j)
+    def prune_with(nm, j, opt=base_opt):
+        return lambda: binding.mvue_prune(g, nm[0], nm[1], 0, 1, values=values, meta=meta, layout=TC, joint=j, options=opt)
 
     prune_ms = tm.loop(prune_with((n, m), joint), 20)
     sys_ms = tm.loop(prune_with((2, 4), binding.MVUE_JOINT_SYSTEMATIC), 20)
     table_ms = tm.loop(prune_with((2, 4), binding.MVUE_JOINT_TABLE), 20)
     one_two_ms = tm.loop(prune_with((1, 2), joint), 20)
-    sr_ms = tm.loop(lambda: binding.mvue_prune(g, n, m, 0, 1, values=values, meta=meta, layout=TC, joint=joint,
-                                               options=binding.MVUE_OPT_STOCHASTIC_ROUNDING), 20)
+    sr_ms = tm.loop(prune_with((n, m), joint, base_opt | binding.MVUE_OPT_STOCHASTIC_ROUNDING), 20)
+    sys32_ms = tm.loop(prune_with((2, 4), binding.MVUE_JOINT_SYSTEMATIC, binding.MVUE_OPT_NONE), 20)
+    table32_ms = tm.loop(prune_with((2, 4), binding.MVUE_JOINT_TABLE, binding.MVUE_OPT_NONE), 20)
     four_eight_ms = tm.loop(lambda: binding.mvue_prune_4of8(g, 0, 1), 3, warm=1)     # approx-4:8, prune only
     prune_with((n, m), joint)()
     gemm_ms = tm.loop(lambda: binding.mvue_sparse_update_gemm(values, meta, h, out=dW, workspace=ws), 30)
@@ -680,6 +687,11 @@ def tensor_bound_case(tm: Timer, n, m, peaks, joint, issue_cold):
             "prune_systematic_ms": sys_ms, "prune_systematic_frac_of_hbm_peak": pb / (sys_ms * 1e-3) / 1e9 / peaks["hbm_gbs"],
             "prune_table_ms": table_ms, "prune_table_frac_of_hbm_peak": pb / (table_ms * 1e-3) / 1e9 / peaks["hbm_gbs"],
             "prune_1of2_ms": one_two_ms, "prune_1of2_frac_of_hbm_peak": pb / (one_two_ms * 1e-3) / 1e9 / peaks["hbm_gbs"],
+            "random_bits_per_block": 16 if base_opt & binding.MVUE_OPT_EPS16 else 32,
+            "prune_systematic_32bit_ms": sys32_ms,
+            "prune_systematic_32bit_frac_of_hbm_peak": pb / (sys32_ms * 1e-3) / 1e9 / peaks["hbm_gbs"],
+            "prune_table_32bit_ms": table32_ms,
+            "prune_table_32bit_frac_of_hbm_peak": pb / (table32_ms * 1e-3) / 1e9 / peaks["hbm_gbs"],
             "prune_approx_4of8_ms": four_eight_ms,
             "prune_approx_4of8_frac_of_hbm_peak": pb / (four_eight_ms * 1e-3) / 1e9 / peaks["hbm_gbs"],
             "prune_stochastic_rounding_ms": sr_ms,
@@ -755,7 +767,7 @@ def gemm_shapes_case(tm: Timer, peaks, issue_cold):
     return {"timing": "per call, L2 flushed before each; mean / best of 10", "rows": rows}
 
 
-def prune_sweep(peaks, sizes_log2=range(20, 33), step_joint=1):
+def prune_sweep(peaks, sizes_log2=range(20, 33), step_joint=1, options=0):
     """Standalone prune+pack bandwidth over bf16 tensors of 2^k bytes ([bytes / 8192 x 4096], Student-t values), both
     pruned axes, 2:4 (pair table, systematic sampling), 1:2 and 1:4.  Every point is a CUDA graph of `reps` launches
     over rotating input copies that together exceed 2.5 x L2, replayed and timed with events, so the small sizes are
@@ -796,7 +808,7 @@ def prune_sweep(peaks, sizes_log2=range(20, 33), step_joint=1):
                 def burst():
                     for i in range(reps):
                         binding.mvue_prune(views[i % copies], n, m, axis, i, values=values, meta=out_m, layout=TC,
-                                           joint=joint)
+                                           joint=joint, options=options)
                 side.wait_stream(torch.cuda.current_stream())
                 with torch.cuda.stream(side):
                     burst()
@@ -819,6 +831,7 @@ def prune_sweep(peaks, sizes_log2=range(20, 33), step_joint=1):
                 del graph
         points.append(point)
     return {"dtype": "bf16", "cols": cols, "dist": "student_t", "layout": "tensor-core metadata order",
+            "random_bits_per_block": 16 if options & 2 else 32,
             "timing": "CUDA graph replay, inputs rotated over > 2.5 x L2 where the tensor is smaller than that",
             "points": points}
 
@@ -889,6 +902,10 @@ def chain_case(n, m):
     def run_sys_overlap():
         chain.backward_update(g_top, layers, n, m, base_seed=1, joint=binding.MVUE_JOINT_SYSTEMATIC, overlap=True)
 
+    def run_sys16_overlap():
+        chain.backward_update(g_top, layers, n, m, base_seed=1, joint=binding.MVUE_JOINT_SYSTEMATIC, overlap=True,
+                              options=binding.MVUE_OPT_EPS16)
+
     def run_sys_epilogue():
         # backward products with a long reduction axis (out = 4096) prune their own output for the layer below
         chain.backward_update(g_top, layers, n, m, base_seed=1, joint=binding.MVUE_JOINT_SYSTEMATIC, overlap=True,
@@ -899,6 +916,7 @@ def chain_case(n, m):
     sys_ms = timed(graphed(run_sys), 10) if m == 4 else None
     overlap_ms = timed(graphed(run_sys_overlap), 10) if m == 4 else None
     epilogue_ms = timed(graphed(run_sys_epilogue), 10) if m == 4 else None
+    sys16_ms = timed(graphed(run_sys16_overlap), 10) if m == 4 else None
     dense_ms = timed(graphed(dense_chain), 10)
     n_layers = len(layers)
     flops = 2.0 * T * d * d_ff * (2 * n_layers - 1)         # update product per layer, backward for all but the bottom
@@ -914,6 +932,9 @@ def chain_case(n, m):
             # and with the long-K backward products pruning their own output in the epilogue (one prune launch less
             # per block of two layers)
             "systematic_two_stream_epilogue_prune_ms": epilogue_ms,
+            # the two-stream chain with sixteen random bits per block (one generator call per eight blocks)
+            "systematic_16bit_two_stream_ms": sys16_ms,
+            "systematic_16bit_two_stream_tflops_effective": None if sys16_ms is None else flops / (sys16_ms * 1e-3) / 1e12,
             "dense_torch_ms": dense_ms, "dense_torch_tflops": flops / (dense_ms * 1e-3) / 1e12}
 
 
@@ -942,6 +963,9 @@ def main():
     ap.add_argument("--joint", default="systematic", choices=["table", "systematic", "approx"],
                     help="2:4 estimator used by the step: systematic sampling (the faster of the two exact MVUE laws), "
                          "the App. A.2 pair table, or approx-MVUE (Sec. 4.4); the others are timed beside it")
+    ap.add_argument("--eps32", dest="eps16", action="store_false",
+                    help="32 random bits per block (one generator call per four blocks) in the step instead of 16 "
+                         "(MVUE_OPT_EPS16: one call per eight blocks); the other width is timed beside it")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--sweep", action="store_true",
                     help="the whole standalone prune+pack sweep over bf16 tensors of 1 MB .. 4 GB (default: three sizes)")

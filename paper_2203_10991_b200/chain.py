@@ -23,7 +23,7 @@ def layer_seeds(base_seed: int, layer: int) -> tuple[int, int]:
 
 
 def backward_update(g_top: torch.Tensor, layers, n: int = 2, m: int = 4, base_seed: int = 0, joint: int | None = None,
-                    overlap: bool = False, prune_in_epilogue_min_k: int | None = None):
+                    overlap: bool = False, prune_in_epilogue_min_k: int | None = None, options: int = 0):
     """layers: list (top layer first) of dicts {"W": [out x in] bf16, "h": [T x in] bf16,
     "act_grad": [T x in] bf16 or None (None for the bottom layer: no gradient is propagated further)}.
     joint: the 2:4 law over pairs handed to mvue_prune_joint (None: mvue_prune, the App. A.2 table).
@@ -32,7 +32,8 @@ def backward_update(g_top: torch.Tensor, layers, n: int = 2, m: int = 4, base_se
     product of a long token axis keeps a small register footprint, so blocks of the (shared-memory-free) prune along
     the features fit on the same SMs.  Same calls, same seeds, same results; the streams join before each backward
     product and before returning.
-    prune_in_epilogue_min_k: when set (2:4 only), a backward product whose reduction axis (the layer's out) is at least
+    options: mvue_prune_option bits handed to every prune (stochastic rounding, sixteen random bits per block).
+    prune_in_epilogue_min_k: when set (2:4 only, options 0), a backward product whose reduction axis (the layer's out) is at least
     this long also prunes its own output along the features in its epilogue (mvue_sparse_backward_gemm_pruned), with
     the seed the layer below would have used, so that layer's prune along the features is not launched.  Same bits.
     Returns the list of dW (fp32), top layer first."""
@@ -44,7 +45,7 @@ def backward_update(g_top: torch.Tensor, layers, n: int = 2, m: int = 4, base_se
     def backward(i, L, values_b, meta_b):
         nonlocal ready
         below = layers[i + 1] if i + 1 < len(layers) else None
-        if (prune_in_epilogue_min_k is not None and (n, m) == (2, 4) and L["W"].shape[0] >= prune_in_epilogue_min_k
+        if (prune_in_epilogue_min_k is not None and options == 0 and (n, m) == (2, 4) and L["W"].shape[0] >= prune_in_epilogue_min_k
                 and below is not None and below.get("act_grad") is not None and L["W"].shape[1] % 128 == 0
                 and fuse_joint in (binding.MVUE_JOINT_TABLE, binding.MVUE_JOINT_SYSTEMATIC)):
             g_next, nv, nm = binding.mvue_sparse_backward_gemm_pruned(values_b, meta_b, L["W"], L["act_grad"],
@@ -57,13 +58,13 @@ def backward_update(g_top: torch.Tensor, layers, n: int = 2, m: int = 4, base_se
     def prune_features(g, s_bwd):
         if ready is not None:
             return ready
-        return binding.mvue_prune(g, n, m, 1, s_bwd, layout=TC, joint=joint)
+        return binding.mvue_prune(g, n, m, 1, s_bwd, layout=TC, joint=joint, options=options)
 
     main = torch.cuda.current_stream()
     side = torch.cuda.Stream(priority=-1) if overlap else None
     for i, L in enumerate(layers):
         s_upd, s_bwd = layer_seeds(base_seed, i)
-        values, meta = binding.mvue_prune(g, n, m, 0, s_upd, layout=TC, joint=joint)
+        values, meta = binding.mvue_prune(g, n, m, 0, s_upd, layout=TC, joint=joint, options=options)
         propagate = L.get("act_grad") is not None
         if overlap and propagate:
             dW = torch.empty((values.shape[0], L["h"].shape[1]), dtype=torch.float32, device=g.device)
