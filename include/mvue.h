@@ -280,22 +280,26 @@ MVUE_API int mvue_sparse_backward_gemm_pruned(const void* values, const void* me
 /* Prune fused into the update product (Sec. 4.1 / 4.2 + App. A.2 applied to g along the
  * token axis, then the update equation of Sec. 1) in ONE kernel:
  *   dW[out x in] (+)= theta(g)^T h,   g bf16 [T x out] (ld ldg), h bf16 [T x in]
- * g is read from memory once and the packed operand is never written.  The random words
- * are those of mvue_prune(g, n, m, axis 0, seed), so the result equals mvue_prune followed by
- * mvue_sparse_update_gemm with the same seed (up to fp32 summation order across K splits).
- * Every 128 x 256 output tile re-prunes its rows of g: the prune work grows with in / 256,
- * and the prune is bound by instruction issue, so for wide layers the separate calls are
- * several times faster.  With in <= 256 (one column tile: nothing is pruned twice) it ties
- * with mvue_prune + mvue_sparse_update_gemm and loses 10-30 % to mvue_prune_joint with
- * systematic sampling + the product; its use is when memory for the packed operand is not
- * available.
- * dtype must be MVUE_BF16 (else MVUE_ERR_DTYPE).  workspace: mvue_gemm_workspace_bytes(2, out,
+ * The packed operand is never written to memory.  The random words are those of mvue_prune(g, n, m, axis 0, seed)
+ * (mvue_prune_joint with `joint` for the _joint form: MVUE_JOINT_TABLE or MVUE_JOINT_SYSTEMATIC), so the result equals
+ * that prune followed by mvue_sparse_update_gemm with the same seed (up to fp32 summation order across K splits).
+ * One thread block per 128 x 256 output tile; up to four blocks whose tiles are neighbours along `in` form a cluster
+ * and share every pruned stage through each other's shared memory, so a row tile of g is read and pruned once per 1024
+ * output columns (when in / 256 is a multiple of 4; once per 512 / 256 columns when it is only even / odd).  The prune
+ * then hides under the tensor-core time of wide layers; on narrow layers (in <= 256) the prune is the whole cost and the
+ * kernel ties with the separate calls.  Its use is when memory for the packed operand is not available.
+ * dtype must be MVUE_BF16 (else MVUE_ERR_DTYPE); (n, m) = (1,2) or (2,4).  workspace: mvue_gemm_workspace_bytes(2, out,
  * in, T) bytes.  Other arguments, preconditions and errors as mvue_sparse_update_gemm. */
 MVUE_API int mvue_fused_update_gemm(const void* g, int dtype, int64_t T, int64_t out, int64_t ldg, int n,
                                     int m, uint64_t seed, const void* h, int64_t in, int64_t ldh,
                                     void* dW, int dW_dtype, int64_t lddW, int accumulate,
                                     void* workspace, size_t workspace_bytes, int* dev_status,
                                     void* stream);
+MVUE_API int mvue_fused_update_gemm_joint(const void* g, int dtype, int64_t T, int64_t out, int64_t ldg, int n,
+                                          int m, int joint, uint64_t seed, const void* h, int64_t in, int64_t ldh,
+                                          void* dW, int dW_dtype, int64_t lddW, int accumulate,
+                                          void* workspace, size_t workspace_bytes, int* dev_status,
+                                          void* stream);
 
 /* Scratch bytes the product C[M x N] = A[M x K] . B[K x N] needs
  * (which: 0 update, 1 backward, 2 fused update).  bytes is a HOST pointer. */

@@ -23,7 +23,7 @@ MVUE_OPT_NONE, MVUE_OPT_STOCHASTIC_ROUNDING, MVUE_OPT_EPS16 = 0, 1, 2
 EXPORTS = ("mvue_version", "mvue_status_string", "mvue_last_cuda_error", "mvue_packed_sizes",
            "mvue_prune", "mvue_prune_joint", "mvue_prune_opts", "mvue_prune_4of8", "mvue_unpack", "mvue_sparse_update_gemm", "mvue_sparse_backward_gemm",
            "mvue_sparse_backward_gemm_pruned",
-           "mvue_gemm_workspace_bytes", "mvue_sparse_update_gemm_noalloc", "mvue_fused_update_gemm",
+           "mvue_gemm_workspace_bytes", "mvue_sparse_update_gemm_noalloc", "mvue_fused_update_gemm", "mvue_fused_update_gemm_joint",
            "mvue_probe_sparse_mma", "mvue_selftest_wait_timeout")
 
 
@@ -65,6 +65,8 @@ def lib() -> ctypes.CDLL:
         L.mvue_gemm_workspace_bytes.argtypes = [ci, i64, i64, i64, szp]
         L.mvue_fused_update_gemm.argtypes = [vp, ci, i64, i64, i64, ci, ci, u64, vp, i64, i64, vp, ci, i64, ci, vp,
                                              ctypes.c_size_t, vp, vp]
+        L.mvue_fused_update_gemm_joint.argtypes = [vp, ci, i64, i64, i64, ci, ci, ci, u64, vp, i64, i64, vp, ci, i64, ci, vp,
+                                                   ctypes.c_size_t, vp, vp]
         L.mvue_sparse_update_gemm_noalloc.argtypes = [vp, vp, ci, i64, i64, vp, i64, i64, vp, ci, i64, ci, vp, vp]
         L.mvue_probe_sparse_mma.argtypes = [ci, ctypes.POINTER(ctypes.c_int), ctypes.POINTER(ctypes.c_double), vp, vp]
         L.mvue_selftest_wait_timeout.argtypes = [ci, vp, vp]
@@ -252,15 +254,17 @@ def mvue_sparse_update_gemm_noalloc(values: torch.Tensor, meta: torch.Tensor, h:
 def mvue_fused_update_gemm(g: torch.Tensor, h: torch.Tensor, n: int, m: int, seed: int, *,
                            out: torch.Tensor | None = None, out_dtype=torch.float32, accumulate: bool = False,
                            workspace: torch.Tensor | None = None,
-                           dev_status: torch.Tensor | None = None) -> torch.Tensor:
-    """dW[out, in] (+)= theta(g)^T . h in one kernel: g bf16 [T, out] is pruned along the tokens on the fly."""
+                           dev_status: torch.Tensor | None = None, joint: int = MVUE_JOINT_TABLE) -> torch.Tensor:
+    """dW[out, in] (+)= theta(g)^T . h in one kernel: g bf16 [T, out] is pruned along the tokens on the fly
+    (joint: the 2:4 law, MVUE_JOINT_TABLE or MVUE_JOINT_SYSTEMATIC)."""
     T, n_out = g.shape
     T2, n_in = h.shape
     assert T == T2 and g.stride(1) == 1 and h.stride(1) == 1
     if out is None:
         out = torch.empty((n_out, n_in), dtype=out_dtype, device=h.device)
     ws, ws_bytes = _workspace(2, n_out, n_in, T, h.device, workspace)
-    _check(lib().mvue_fused_update_gemm(g.data_ptr(), _dtype_code(g), T, n_out, g.stride(0), n, m, seed & (2**64 - 1),
+    _check(lib().mvue_fused_update_gemm_joint(g.data_ptr(), _dtype_code(g), T, n_out, g.stride(0), n, m, int(joint),
+                                              seed & (2**64 - 1),
                                         h.data_ptr(), n_in, h.stride(0), out.data_ptr(), _dtype_code(out),
                                         out.stride(0), int(accumulate), None if ws is None else ws.data_ptr(), ws_bytes,
                                         None if dev_status is None else dev_status.data_ptr(), _stream_ptr()),

@@ -258,7 +258,16 @@ int mvue_fused_update_gemm(const void* g, int dtype, int64_t T, int64_t out, int
                            uint64_t seed, const void* h, int64_t in, int64_t ldh, void* dW, int dW_dtype,
                            int64_t lddW, int accumulate, void* workspace, size_t workspace_bytes,
                            int* dev_status, void* stream) {
+    return mvue_fused_update_gemm_joint(g, dtype, T, out, ldg, n, m, MVUE_JOINT_TABLE, seed, h, in, ldh, dW, dW_dtype, lddW,
+                                        accumulate, workspace, workspace_bytes, dev_status, stream);
+}
+
+int mvue_fused_update_gemm_joint(const void* g, int dtype, int64_t T, int64_t out, int64_t ldg, int n, int m, int joint,
+                                 uint64_t seed, const void* h, int64_t in, int64_t ldh, void* dW, int dW_dtype,
+                                 int64_t lddW, int accumulate, void* workspace, size_t workspace_bytes,
+                                 int* dev_status, void* stream) {
     if (!g || !h || !dW) return MVUE_ERR_NULL;
+    if (joint != MVUE_JOINT_TABLE && joint != MVUE_JOINT_SYSTEMATIC) return MVUE_ERR_JOINT;
     if (int s = check_nm(n, m)) return s;
     if (n == 1 && m == 4) return MVUE_ERR_NM;                      // the fused path prunes to 1:2 and 2:4 only
     if (dtype != MVUE_BF16) return MVUE_ERR_DTYPE;                 // the fused path takes bf16 gradients only
@@ -277,7 +286,8 @@ int mvue_fused_update_gemm(const void* g, int dtype, int64_t T, int64_t out, int
     if (need > 0 && (!workspace || workspace_bytes < need || !aligned16(workspace))) return MVUE_ERR_WORKSPACE;
     FusedArgs f{g, ldg, m, seed,
                 SparseGemmArgs{nullptr, nullptr, out, in, T, h, ldh, dW, lddW, dW_dtype == MVUE_BF16, accumulate,
-                               nullptr, workspace, workspace ? workspace_bytes : 0, dev_status, dev.sm_count}};
+                               nullptr, workspace, workspace ? workspace_bytes : 0, dev_status, dev.sm_count},
+                joint};
     return launch_fused_update(f, reinterpret_cast<cudaStream_t>(stream));
 }
 

@@ -780,20 +780,24 @@ sparse_gemm_pair_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_
 }
 
 // =============================================================================
-// Prune fused into the update product: dW[out x in] = theta(g)^T h with g read once and the
+// Prune fused into the update product: dW[out x in] = theta(g)^T h with g read once per cluster and the
 // packed operand never written to memory.  One thread block per 128 x 256 output tile
-// (tcgen05.mma.sp.cta_group::1, M = 128), two stages of K = 128:
-//   warp 0      TMA producer of the B tile only (four 64-column boxes of h)
-//   warp 1      tcgen05.cp of the stage's metadata, four MMAs, commit
+// (tcgen05.mma.sp.cta_group::1, M = 128), two stages of K = 128; C = 1, 2 or 4 blocks whose tiles are neighbours
+// along `in` form a cluster and SHARE the pruned stage: every block prunes 1 / C of the stage's 1024 units (a unit =
+// one row of A x 16 tokens) and writes each result -- 16 bytes of survivors at their 128-byte-swizzled place in the
+// A tile, 2 bytes of metadata at their tensor-core lane / word -- into the shared memory of all C blocks
+// (st.shared::cluster), so a row tile of g is pruned in / (256 C) times instead of in / 256 times.
+//   warp 0      TMA producer of the block's own B tile (four 64-column boxes of h)
+//   warp 1      tcgen05.cp of the stage's metadata, four MMAs, commit -- arriving on the "empty" barrier of ALL
+//               blocks of the cluster: a stage is rewritten only when every block has consumed it
 //   warp 2      tensor-memory allocation
 //   warps 4-7   epilogue
-//   warps 8-15  prune: warp w owns the 16-token strip w of the stage, lane l the four columns
-//               4l..4l+3 of g (= rows of A); each (column, strip) is one prune unit and yields 8
-//               survivors -- one 16-byte chunk of the A tile, written at its 128-byte-swizzled
-//               place -- and one 16-bit metadata word, written at its tensor-core lane / word.
-// The random words are those of mvue_prune for the same seed (block number over the whole
-// operand), so the result equals mvue_prune followed by mvue_sparse_update_gemm.
-// Every block that shares a row tile re-prunes it: the prune work grows with in / 256.
+//   warps 8-15  prune: warp w of block r owns strip (8 / C) r + w / C of the stage and the rows
+//               (128 / C) (w % C) + lane + 32 i, i < 4 / C; a lane reads its column of g for the strip's 16 tokens
+//               (a warp reads 64 contiguous bytes per token), prunes the unit with the same unit function and the
+//               same global block numbers as mvue_prune, stores to every block, fences the writes for the
+//               tensor cores' asynchronous reads and arrives on every block's "full" barrier (1 + 8 C arrivals).
+// No block leaves before all have (cluster barrier): peers write into its shared memory until the last stage.
 // =============================================================================
 constexpr int kFStages = 2;
 constexpr int kFBBytes = (BN / 64) * kBBoxBytes;                 // 64 KiB: all 256 columns
@@ -805,13 +809,33 @@ constexpr uint32_t kInstrDesc1 = (1u << 2) | (1u << 4) | (1u << 7) | (1u << 10) 
                                  ((uint32_t)(BN >> 3) << 17) | ((uint32_t)(BM >> 4) << 24);
 
 struct FusedParams {
-    const uint32_t* g;        // bf16 [T x out], two elements per word
-    int64_t ldg_words;        // leading dimension of g in 32-bit words
+    const uint16_t* g;        // bf16 [T x out]
+    int64_t ldg;              // leading dimension of g in elements
     RoundKeys rk;
     GemmParams gemm;          // M = out, N = in, K = T
 };
 
-template <int NM>
+__device__ __forceinline__ uint32_t cluster_nctarank() {
+    uint32_t r;
+    asm volatile("mov.u32 %0, %%cluster_nctarank;" : "=r"(r));
+    return r;
+}
+__device__ __forceinline__ void st_cluster_v4(uint32_t addr, uint4 v) {
+    asm volatile("st.shared::cluster.v4.b32 [%0], {%1, %2, %3, %4};" ::"r"(addr), "r"(v.x), "r"(v.y), "r"(v.z), "r"(v.w) : "memory");
+}
+__device__ __forceinline__ void st_cluster_u16(uint32_t addr, uint16_t v) {
+    asm volatile("st.shared::cluster.b16 [%0], %1;" ::"r"(addr), "h"(v) : "memory");
+}
+__device__ __forceinline__ void mbar_arrive_cluster(uint32_t remote_bar) {
+    asm volatile("mbarrier.arrive.release.cluster.shared::cluster.b64 _, [%0];" ::"r"(remote_bar) : "memory");
+}
+__device__ __forceinline__ void tc_commit_cluster(uint32_t bar, uint16_t mask) {   // arrives on `bar` in every block of the mask
+    asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.multicast::cluster.b64 [%0], %1;"
+                 ::"r"(bar), "h"(mask) : "memory");
+}
+
+// NM: 2 (1:2) or 4 (2:4); kJoint: the 2:4 law (0 App. A.2 table, 1 systematic sampling).
+template <int NM, int kJoint, int kC>
 __global__ void __launch_bounds__(kFThreads, 1)
 fused_update_kernel(const __grid_constant__ CUtensorMap map_b, const FusedParams fp) {
     const GemmParams& p = fp.gemm;
@@ -826,6 +850,8 @@ fused_update_kernel(const __grid_constant__ CUtensorMap map_b, const FusedParams
     volatile int* abort_flag = reinterpret_cast<volatile int*>(tmem_slot + 1);
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    constexpr uint32_t C = kC;                                               // blocks of a cluster differ in blockIdx.x only
+    const uint32_t rank = cluster_ctarank();
     const int64_t m0 = (int64_t)blockIdx.y * BM;
     const int64_t n0 = (int64_t)blockIdx.x * BN;
     const int split = blockIdx.z;
@@ -837,8 +863,8 @@ fused_update_kernel(const __grid_constant__ CUtensorMap map_b, const FusedParams
 
     if (threadIdx.x == 0) {
         for (int s = 0; s < kFStages; ++s) {
-            mbar_init(full_bar(s), 1 + kFPruneWarps);   // B bytes + one arrival per prune warp
-            mbar_init(empty_bar(s), 1);
+            mbar_init(full_bar(s), 1 + kFPruneWarps * C);   // B bytes + one arrival per prune warp of every block
+            mbar_init(empty_bar(s), C);                     // every block's MMA warp has consumed the stage
         }
         mbar_init(acc_bar, 1);
         *abort_flag = 0;
@@ -850,6 +876,7 @@ fused_update_kernel(const __grid_constant__ CUtensorMap map_b, const FusedParams
     }
     tc_fence_before();
     __syncthreads();
+    cluster_sync();                          // the peers' barriers exist before anyone signals them
     tc_fence_after();
     const uint32_t tmem_base = *tmem_slot;
 
@@ -858,7 +885,7 @@ fused_update_kernel(const __grid_constant__ CUtensorMap map_b, const FusedParams
             for (int64_t i = 0; i < n_steps; ++i) {
                 const int s = (int)(i % kFStages);
                 const uint32_t use = (uint32_t)(i / kFStages);
-                if (use > 0 && !mbar_wait(empty_bar(s), (use - 1) & 1u, abort_flag)) break;
+                if (use > 0 && !mbar_wait_cluster(empty_bar(s), (use - 1) & 1u, abort_flag)) break;
                 const uint32_t b_dst = smem_base + s * kFStageBytes + kABytes;
                 const int k = (int)((step_begin + i) * BK);
                 mbar_expect_tx(full_bar(s), kFBBytes);
@@ -870,10 +897,11 @@ fused_update_kernel(const __grid_constant__ CUtensorMap map_b, const FusedParams
     } else if (warp == 1) {
         if (lane == 0) {
             bool ok = true;
+            const uint16_t all = (uint16_t)((1u << C) - 1u);
             for (int64_t i = 0; i < n_steps && ok; ++i) {
                 const int s = (int)(i % kFStages);
                 const uint32_t use = (uint32_t)(i / kFStages);
-                ok = mbar_wait(full_bar(s), use & 1u, abort_flag);
+                ok = mbar_wait_cluster(full_bar(s), use & 1u, abort_flag);
                 if (!ok) break;
                 tc_fence_after();
                 const uint32_t a_addr = smem_base + s * kFStageBytes;
@@ -888,7 +916,7 @@ fused_update_kernel(const __grid_constant__ CUtensorMap map_b, const FusedParams
                     tc_mma_sp_bf16(tmem_base, a_desc, b_desc, tmem_e + (uint32_t)(kb & ~1),
                                    kInstrDesc1 | (uint32_t)(kb & 1), (i > 0 || kb > 0) ? 1u : 0u);
                 }
-                tc_commit(empty_bar(s));
+                tc_commit_cluster(empty_bar(s), all);
             }
             tc_commit(acc_bar);
         }
@@ -897,51 +925,80 @@ fused_update_kernel(const __grid_constant__ CUtensorMap map_b, const FusedParams
         const bool acc_ok = n_steps > 0 ? mbar_wait(acc_bar, 0, abort_flag) : true;
         tc_fence_after();
         const int64_t row = m0 + 32 * q + lane;
-        if (acc_ok)
+        if (acc_ok && n0 < p.N)
             epilogue_rows<false>(p, split, row, n0, tmem_base + ((uint32_t)(32 * q) << 16), n_steps > 0, nullptr);
     } else if (warp >= 8) {
         // ------------------------------------------------------------ prune warps
-        const int strip_l = warp - 8;                               // 16-token strip of the stage
-        const int64_t col = m0 + 4 * lane;                          // first of this lane's four columns of g
-        const bool cols_exist = col < p.M;                          // out is a multiple of 8: all four or none
+        const int pw = warp - 8;
+        constexpr int kStripsOwn = 8 / kC, kUnits = 4 / kC;         // strips of a stage per block, units per lane
+        const int strip_l = kStripsOwn * (int)rank + pw / kC;       // 16-token strip of the stage
+        const int row_base = (128 / kC) * (pw % kC) + lane;         // first of this lane's rows of the A tile
         const int64_t units_per_row = p.K / 16;
+        // the lane's columns of g for one stage: 16 tokens each; the next stage's are requested before this one is pruned
+        auto load_stage = [&](int64_t i, uint32_t (&dst)[kUnits][16]) {
+            const int64_t k0 = (step_begin + i) * BK + 16 * strip_l;
+#pragma unroll
+            for (int u = 0; u < kUnits; ++u) {
+                const int64_t col = m0 + row_base + 32 * u;                 // row of A = column of g
+                const uint16_t* src = fp.g + k0 * fp.ldg + col;
+#pragma unroll
+                for (int r = 0; r < 16; ++r) dst[u][r] = col < p.M ? (uint32_t)__ldg(src + r * fp.ldg) : 0u;
+            }
+        };
+        constexpr bool kPrefetch = kUnits <= 2;                      // (four units per lane leave no registers for a second set)
+        uint32_t cur[kUnits][16], nxt[kPrefetch ? kUnits : 1][16];
+        if (kPrefetch && n_steps > 0) load_stage(0, cur);
         bool ok = true;
         for (int64_t i = 0; i < n_steps && ok; ++i) {
             const int s = (int)(i % kFStages);
             const uint32_t use = (uint32_t)(i / kFStages);
             const int64_t k0 = (step_begin + i) * BK + 16 * strip_l;        // first token of the strip
-            uint2 w[16];
-            if (cols_exist) {
-                const uint32_t* src = fp.g + k0 * fp.ldg_words + (col >> 1);
-#pragma unroll
-                for (int r = 0; r < 16; ++r) w[r] = __ldg(reinterpret_cast<const uint2*>(src + r * fp.ldg_words));
+            if constexpr (kPrefetch) {
+                if (i + 1 < n_steps) load_stage(i + 1, nxt);
+            } else {
+                load_stage(i, cur);
             }
-            if (use > 0) ok = mbar_wait(empty_bar(s), (use - 1) & 1u, abort_flag);
+            if (use > 0) ok = mbar_wait_cluster(empty_bar(s), (use - 1) & 1u, abort_flag);
             if (!ok) break;
-            uint8_t* a_tile = smem_gen + s * kFStageBytes;
-            uint8_t* e_tile = a_tile + kABytes + kFBBytes;
+            const uint32_t a_tile = smem_base + s * kFStageBytes;
+            const uint32_t e_tile = a_tile + kABytes + kFBBytes;
 #pragma unroll
-            for (int e = 0; e < 4; ++e) {
-                const int m_l = 4 * lane + e;                              // row of the A tile
+            for (int u = 0; u < kUnits; ++u) {
+                const int m_l = row_base + 32 * u;                          // row of the A tile
+                const int64_t col = m0 + m_l;
                 uint4 v = make_uint4(0u, 0u, 0u, 0u);
                 uint32_t mt = 0x4444u;
-                if (cols_exist) {
-                    uint32_t rw[16];
+                if (col < p.M) {
+                    uint32_t raw[8];                                         // the unit as it is when K is contiguous
 #pragma unroll
-                    for (int r = 0; r < 16; ++r) rw[r] = (e < 2) ? w[r].x : w[r].y;
-                    const uint64_t unit = (uint64_t)(col + e) * (uint64_t)units_per_row + (uint64_t)(k0 >> 4);
-                    if (e & 1) prune_unit_bf16_rows<NM, true>(rw, unit, fp.rk, &v, &mt);
-                    else       prune_unit_bf16_rows<NM, false>(rw, unit, fp.rk, &v, &mt);
+                    for (int e = 0; e < 8; ++e) raw[e] = cur[u][2 * e] | (cur[u][2 * e + 1] << 16);
+                    const uint64_t unit = (uint64_t)col * (uint64_t)units_per_row + (uint64_t)(k0 >> 4);
+                    prune_unit_bf16<NM, kJoint>(raw, unit, fp.rk, &v, &mt);
                 }
-                // A tile: row m_l is 128 bytes; the strip's 8 survivors are chunk strip_l, swizzled by the row
-                *reinterpret_cast<uint4*>(a_tile + m_l * 128 + ((strip_l ^ (m_l & 7)) << 4)) = v;
-                // metadata: lane / word / half-word of the tensor-core order
+                // A tile: row m_l is 128 bytes; the strip's 8 survivors are chunk strip_l, swizzled by the row;
+                // metadata: lane / word / half-word of the tensor-core order.  Same place in every block of the cluster.
+                const uint32_t a_off = a_tile + (uint32_t)(m_l * 128 + ((strip_l ^ (m_l & 7)) << 4));
                 const int tc_lane = (m_l & 7) + 8 * (strip_l & 1) + 16 * (m_l >> 4);
-                *reinterpret_cast<uint16_t*>(e_tile + tc_lane * 16 + (strip_l >> 1) * 4 + ((m_l >> 3) & 1) * 2) = (uint16_t)mt;
+                const uint32_t e_off = e_tile + (uint32_t)(tc_lane * 16 + (strip_l >> 1) * 4 + ((m_l >> 3) & 1) * 2);
+#pragma unroll
+                for (uint32_t d = 0; d < C; ++d) {
+                    st_cluster_v4(map_to_cta(a_off, d), v);
+                    st_cluster_u16(map_to_cta(e_off, d), (uint16_t)mt);
+                }
             }
-            asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+            asm volatile("fence.proxy.async.shared::cluster;" ::: "memory");
             __syncwarp();
-            if (lane == 0) mbar_arrive(full_bar(s));
+            if (lane == 0) {
+#pragma unroll
+                for (uint32_t d = 0; d < C; ++d) mbar_arrive_cluster(map_to_cta(full_bar(s), d));
+            }
+            if constexpr (kPrefetch) {
+#pragma unroll
+                for (int u = 0; u < kUnits; ++u) {
+#pragma unroll
+                    for (int r = 0; r < 16; ++r) cur[u][r] = nxt[u][r];
+                }
+            }
         }
     }
 
@@ -956,6 +1013,7 @@ fused_update_kernel(const __grid_constant__ CUtensorMap map_b, const FusedParams
         }
         __syncthreads();
     }
+    cluster_sync();                          // no block leaves while a peer may still write to it or signal it
     if (warp == 2) {
         tc_fence_after();
         tmem_dealloc(tmem_base, kTmemCols);
@@ -1226,6 +1284,35 @@ size_t fused_workspace_bytes(int64_t M, int64_t N, int64_t K, int sm_count) {
     return splits > 1 ? (size_t)splits * (size_t)M * (size_t)N * sizeof(float) : 0;
 }
 
+template <int NM, int kJoint, int kC>
+cudaError_t launch_fused_c(const CUtensorMap& map_b, const FusedParams& fp, dim3 grid, cudaStream_t stream) {
+    constexpr unsigned cluster = kC;
+    static PerDeviceOnce once;
+    const cudaError_t attr_err = once_per_device(once, [](int) {
+        return cudaFuncSetAttribute(fused_update_kernel<NM, kJoint, kC>, cudaFuncAttributeMaxDynamicSharedMemorySize, kFSmemBytes);
+    });
+    if (attr_err != cudaSuccess) return attr_err;
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = grid;
+    cfg.blockDim = dim3(kFThreads, 1, 1);
+    cfg.dynamicSmemBytes = kFSmemBytes;
+    cfg.stream = stream;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeClusterDimension;
+    attr[0].val.clusterDim.x = cluster;
+    attr[0].val.clusterDim.y = 1;
+    attr[0].val.clusterDim.z = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = 1;
+    return cudaLaunchKernelEx(&cfg, fused_update_kernel<NM, kJoint, kC>, map_b, fp);
+}
+template <int NM, int kJoint>
+cudaError_t launch_fused_t(const CUtensorMap& map_b, const FusedParams& fp, dim3 grid, unsigned cluster, cudaStream_t stream) {
+    if (cluster == 4) return launch_fused_c<NM, kJoint, 4>(map_b, fp, grid, stream);
+    if (cluster == 2) return launch_fused_c<NM, kJoint, 2>(map_b, fp, grid, stream);
+    return launch_fused_c<NM, kJoint, 1>(map_b, fp, grid, stream);
+}
+
 int launch_fused_update(const FusedArgs& f, cudaStream_t stream) {
     const SparseGemmArgs& a = f.gemm;
     CUtensorMap map_b;
@@ -1234,20 +1321,11 @@ int launch_fused_update(const FusedArgs& f, cudaStream_t stream) {
         set_cuda_error(cudaErrorUnknown, "cuTensorMapEncodeTiled");
         return MVUE_ERR_CUDA;
     }
-    static PerDeviceOnce once;
-    const cudaError_t attr_err = once_per_device(once, [](int) {
-        cudaError_t err = cudaFuncSetAttribute(fused_update_kernel<4>, cudaFuncAttributeMaxDynamicSharedMemorySize, kFSmemBytes);
-        if (err == cudaSuccess)
-            err = cudaFuncSetAttribute(fused_update_kernel<2>, cudaFuncAttributeMaxDynamicSharedMemorySize, kFSmemBytes);
-        return err;
-    });
-    if (attr_err != cudaSuccess) { set_cuda_error(attr_err, "cudaFuncSetAttribute"); return MVUE_ERR_CUDA; }
-
     const int splits = fused_split_count(a.M, a.N, a.K, a.sm_count);
     const int64_t steps = a.K / BK;
     FusedParams fp;
-    fp.g = reinterpret_cast<const uint32_t*>(f.g);
-    fp.ldg_words = f.ldg / 2;
+    fp.g = reinterpret_cast<const uint16_t*>(f.g);
+    fp.ldg = f.ldg;
     fp.rk = make_round_keys(f.seed);
     GemmParams& p = fp.gemm;
     p.M = a.M; p.N = a.N; p.K = a.K;
@@ -1259,12 +1337,15 @@ int launch_fused_update(const FusedArgs& f, cudaStream_t stream) {
     p.n_work = p.n_main = 0; p.tail_rem = p.tail_splits = 0; p.tail_partial = nullptr;   // pair kernel only
     p.next_values = nullptr; p.next_meta = nullptr; p.next_rk = fp.rk;
     p.dev_status = a.dev_status;
-    dim3 grid((unsigned)((a.N + BN - 1) / BN), (unsigned)((a.M + BM - 1) / BM), (unsigned)splits);
-    if (f.m == 4)
-        fused_update_kernel<4><<<grid, kFThreads, kFSmemBytes, stream>>>(map_b, fp);
-    else
-        fused_update_kernel<2><<<grid, kFThreads, kFSmemBytes, stream>>>(map_b, fp);
-    cudaError_t e = cudaGetLastError();
+    // blocks whose tiles are neighbours along N share the pruned stage: clusters of 4, 2 or 1 along the first grid axis
+    const unsigned tiles_n = (unsigned)((a.N + BN - 1) / BN);
+    const unsigned cluster = tiles_n % 4 == 0 ? 4u : (tiles_n % 2 == 0 ? 2u : 1u);
+    dim3 grid(tiles_n, (unsigned)((a.M + BM - 1) / BM), (unsigned)splits);
+    cudaError_t e;
+    if (f.m == 2)          e = launch_fused_t<2, 0>(map_b, fp, grid, cluster, stream);
+    else if (f.joint == 1) e = launch_fused_t<4, 1>(map_b, fp, grid, cluster, stream);
+    else                   e = launch_fused_t<4, 0>(map_b, fp, grid, cluster, stream);
+    if (e == cudaSuccess) e = cudaGetLastError();
     if (e == cudaSuccess && splits > 1) {
         const int64_t total = a.M * (a.N / 4);
         const int64_t want = (total + 255) / 256;

@@ -65,6 +65,7 @@ struct FusedArgs {
     int m;                // 2 or 4
     uint64_t seed;
     SparseGemmArgs gemm;  // M = out, N = in, K = T; values / meta unused
+    int joint = 0;        // the 2:4 law: 0 = App. A.2 table, 1 = systematic sampling
 };
 int launch_fused_update(const FusedArgs& f, cudaStream_t stream);         // returns an mvue_status
 size_t fused_workspace_bytes(int64_t M, int64_t N, int64_t K, int sm_count);
