@@ -151,6 +151,68 @@ prune_axis1_kernel(const void* __restrict__ g, int64_t n_rows, int units_per_row
         *reinterpret_cast<uint32_t*>(reinterpret_cast<char*>(meta) + tc_meta_offset(r0, c, units_per_row >> 3)) = meta_pair;
 }
 
+// ---- axis 1, bf16, whole blocks ---------------------------------------------------
+// For tensors whose rows are a multiple of 16 and whose K is a multiple of 512 elements, 32-byte aligned (the packed
+// operands of the backward products).  A thread block owns 16 rows of A by 32 units; thread = (row % 8, unit pair)
+// handles the two consecutive units 2 c, 2 c + 1 of rows r and r + 8: 64 contiguous bytes per row (both rows requested
+// before either is pruned), a 32-byte store of survivors per row, two whole metadata words in tensor-core order.  No
+// bounds checks, half the addressing per unit, and with sixteen bits per block the two units of a row share one
+// generator call.  A warp reads 8 rows x 256 contiguous bytes.
+constexpr int kA1PairsPerBlock = 16;
+
+__device__ __forceinline__ void ldg256_aligned(const char* p, uint32_t (&v)[8]) {
+    asm volatile("ld.global.nc.L1::no_allocate.v8.b32 {%0, %1, %2, %3, %4, %5, %6, %7}, [%8];"
+                 : "=r"(v[0]), "=r"(v[1]), "=r"(v[2]), "=r"(v[3]), "=r"(v[4]), "=r"(v[5]), "=r"(v[6]), "=r"(v[7])
+                 : "l"(p));
+}
+
+template <int M, bool kTC, int kJoint, bool kSR, bool kEps16>
+__global__ void __launch_bounds__(8 * kA1PairsPerBlock, 6)
+prune_axis1_bf16_pairs_kernel(const void* __restrict__ g, int units_per_row, int64_t ld, int64_t units_per_row_total,
+                              int64_t unit_offset, RoundKeys rk, uint4* __restrict__ values, uint16_t* __restrict__ meta) {
+    const int j = threadIdx.x & 7;
+    const int c = 2 * (blockIdx.y * kA1PairsPerBlock + (threadIdx.x >> 3));   // first unit of the pair
+    const int64_t r0 = (int64_t)blockIdx.x * 16 + j;
+    uint32_t raw[2][2][8];                                                    // [row h][unit][8 words]
+#pragma unroll
+    for (int h = 0; h < 2; ++h) {
+        const char* p = reinterpret_cast<const char*>(g) + ((r0 + 8 * h) * ld + (int64_t)c * 16) * 2;
+        ldg256_aligned(p, raw[h][0]);
+        ldg256_aligned(p + 32, raw[h][1]);
+    }
+    uint32_t meta_pair[2] = {0u, 0u};                                         // unit 2 c and 2 c + 1: rows r (low), r + 8 (high)
+#pragma unroll
+    for (int h = 0; h < 2; ++h) {
+        const int64_t r = r0 + 8 * h;
+        const uint64_t unit = (uint64_t)r * (uint64_t)units_per_row_total + (uint64_t)(unit_offset + c);
+        uint4 v[2];
+        uint32_t mt[2];
+        if (kEps16 && UnitWords<M, kJoint>::kCount == 4) {                    // unit is even: the two units share one call
+            uint32_t w0[4], w1[4];
+            unit_pair_words16(unit, rk, w0, w1);
+            prune_unit_bf16_w<M, kJoint, kSR>(raw[h][0], reinterpret_cast<const uint32_t (&)[UnitWords<M, kJoint>::kCount]>(w0),
+                                              unit, rk, &v[0], &mt[0]);
+            prune_unit_bf16_w<M, kJoint, kSR>(raw[h][1], reinterpret_cast<const uint32_t (&)[UnitWords<M, kJoint>::kCount]>(w1),
+                                              unit + 1, rk, &v[1], &mt[1]);
+        } else {
+#pragma unroll
+            for (int e = 0; e < 2; ++e) prune_unit_bf16<M, kJoint, kSR, kEps16>(raw[h][e], unit + e, rk, &v[e], &mt[e]);
+        }
+        uint4* dst = values + r * units_per_row + c;
+        asm volatile("st.global.v8.b32 [%0], {%1, %2, %3, %4, %5, %6, %7, %8};"
+                     ::"l"(dst), "r"(v[0].x), "r"(v[0].y), "r"(v[0].z), "r"(v[0].w), "r"(v[1].x), "r"(v[1].y),
+                       "r"(v[1].z), "r"(v[1].w) : "memory");
+        if (!kTC) *reinterpret_cast<uint32_t*>(meta + r * units_per_row + c) = mt[0] | (mt[1] << 16);
+        meta_pair[0] |= mt[0] << (16 * h);
+        meta_pair[1] |= mt[1] << (16 * h);
+    }
+    if (kTC) {
+        char* base = reinterpret_cast<char*>(meta);
+        *reinterpret_cast<uint32_t*>(base + tc_meta_offset(r0, c, units_per_row >> 3)) = meta_pair[0];
+        *reinterpret_cast<uint32_t*>(base + tc_meta_offset(r0, c + 1, units_per_row >> 3)) = meta_pair[1];
+    }
+}
+
 // ---- axis 0 ---------------------------------------------------------------
 // g is [K x C] row-major; A = g^T.  A thread block owns a tile of 256 rows (16
 // strips of 16, one warp per strip) by 64 columns (two per lane).  Each lane reads
@@ -584,9 +646,21 @@ cudaError_t launch_prune_t(const PruneArgs& a, cudaStream_t stream) {
         const int64_t upr = a.cols / 16;
         // in tensor-core order the rows of A are padded to 128: the blocks past the last row write only metadata
         const int64_t cover_rows = kTC ? ((a.rows + 127) / 128) * 128 : a.rows;
-        dim3 grid((unsigned)((cover_rows + 15) / 16), (unsigned)((upr + kA1Units - 1) / kA1Units));
-        prune_axis1_kernel<M, kBf16, kTC, kJoint, kSR, kEps16><<<grid, 8 * kA1Units, 0, stream>>>(
-            a.g, a.rows, (int)upr, a.ld, upr_total, uoff, rk, values, meta);
+        // whole blocks of 16 rows x 32 units, 32-byte aligned rows and outputs, no padding rows of A to cover, and (for
+        // sixteen bits per block) unit pairs that start on even unit numbers: the kernel without bounds checks
+        const bool whole = kBf16 && a.rows % 16 == 0 && upr % (2 * kA1PairsPerBlock) == 0 && cover_rows == a.rows &&
+                           (a.ld * 2) % 32 == 0 && reinterpret_cast<uintptr_t>(a.g) % 32 == 0 &&
+                           reinterpret_cast<uintptr_t>(a.values) % 32 == 0 &&
+                           (!kEps16 || UnitWords<M, kJoint>::kCount != 4 || (uoff % 2 == 0 && upr_total % 2 == 0));
+        if (whole) {
+            dim3 grid_p((unsigned)(a.rows / 16), (unsigned)(upr / (2 * kA1PairsPerBlock)));
+            prune_axis1_bf16_pairs_kernel<M, kTC, kJoint, kSR, kEps16><<<grid_p, 8 * kA1PairsPerBlock, 0, stream>>>(
+                a.g, (int)upr, a.ld, upr_total, uoff, rk, values, meta);
+        } else {
+            dim3 grid((unsigned)((cover_rows + 15) / 16), (unsigned)((upr + kA1Units - 1) / kA1Units));
+            prune_axis1_kernel<M, kBf16, kTC, kJoint, kSR, kEps16><<<grid, 8 * kA1Units, 0, stream>>>(
+                a.g, a.rows, (int)upr, a.ld, upr_total, uoff, rk, values, meta);
+        }
     } else {
         const int64_t n_strips = a.rows / 16;
         // in tensor-core order the rows of A are padded to 128: cover the padding with (load-free) tiles

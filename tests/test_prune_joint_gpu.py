@@ -41,8 +41,9 @@ def assert_parity(g_np, axis, seed, joint=SYS, **kw):
 
 
 # shapes span several thread blocks and leave ragged tails in both grid dimensions; the last three are made of whole
-# 128 x 64 tiles, which the bf16 prune down the rows handles with a kernel of its own
-SHAPES = [(16, 16), (48, 80), (528, 264), (1040, 1000), (4096, 1024), (256, 192), (1152, 320)]
+# 128 x 64 tiles, which the bf16 prune down the rows handles with a kernel of its own; (4096, 1024) and (176, 1536) are
+# whole blocks of 16 rows x 512 columns, which the bf16 prune along the rows handles with a kernel of its own
+SHAPES = [(16, 16), (48, 80), (528, 264), (1040, 1000), (4096, 1024), (256, 192), (1152, 320), (176, 1536)]
 
 
 @pytest.mark.parametrize("joint", JOINTS)
