@@ -109,6 +109,34 @@ def test_backward_gemm_matches_oracle(T, n_out, n_in, with_act, out_dtype):
     assert err <= (TIGHT if out_dtype == torch.float32 else 4e-3), err
 
 
+@pytest.mark.parametrize("T,n_out,n_in", [(8192 + 72, 1024, 4104), (4096, 2048, 520), (20000, 128, 1280)])
+@pytest.mark.parametrize("with_act", [False, True])
+def test_short_k_bf16_products_with_many_tiles(T, n_out, n_in, with_act):
+    # bf16 outputs over a short reduction axis: every pair of blocks walks through several tiles back to back (the
+    # hand-over of the accumulator between tiles is most of what such a product waits for), the last row and column tiles
+    # are ragged, and the same product written as fp32 must round to the same bf16 numbers
+    g = workloads.gradient((T, n_out), "student_t", seed=31, dtype="bf16")
+    W = workloads.normal_bf16((n_out, n_in), seed=32, std=n_out ** -0.5)
+    act = workloads.normal_bf16((T, n_in), seed=33) if with_act else None
+    act_dev = None if act is None else to_dev(act)
+    vals, meta = binding.mvue_prune(to_dev(g), 2, 4, 1, seed=34, layout=TC, joint=binding.MVUE_JOINT_SYSTEMATIC)
+    status = torch.zeros(1, dtype=torch.int32, device="cuda")
+    dh = binding.mvue_sparse_backward_gemm(vals, meta, to_dev(W), act_grad=act_dev, out_dtype=torch.bfloat16,
+                                           dev_status=status)
+    ref32 = binding.mvue_sparse_backward_gemm(vals, meta, to_dev(W), act_grad=act_dev, out_dtype=torch.float32,
+                                              dev_status=status)
+    torch.cuda.synchronize()
+    assert int(status.item()) == 0
+    assert torch.equal(dh.view(torch.int16), ref32.to(torch.bfloat16).view(torch.int16))
+    v_ref, m_ref = oracle.prune(g, 2, 4, axis=1, seed=34, threads=oracle.host_threads(), joint=oracle.JOINT_SYSTEMATIC)
+    rows = np.array(sorted({0, 127, 128, 255, 256, T - 1, T - 9} | set(
+        np.random.Generator(np.random.PCG64(2)).integers(0, T, 40).tolist())))
+    A = oracle.unpack(np.ascontiguousarray(v_ref[rows]), np.ascontiguousarray(m_ref[rows]))
+    want = oracle.gemm(A, W, None if act is None else np.ascontiguousarray(act[rows]), threads=oracle.host_threads())
+    err = rel_fro(dh.double().cpu().numpy()[rows], want)
+    assert err <= 4e-3, err
+
+
 def test_accumulate_and_preallocated_output():
     T, n_out, n_in = 1024, 256, 512
     g = workloads.gradient((T, n_out), "relu_lognormal", seed=1, dtype="bf16")
