@@ -63,14 +63,15 @@ def gemm_bytes(M: int, N: int, K: int, c_bytes: int = 4, scale: bool = False) ->
 # each kernel (summaries under profiles/).  Each figure is tied to a digest of the sources the kernel is built
 # from: once those change the counters no longer describe the kernel and `traffic` is reported as null.
 NCU_TRAFFIC = {
-    "sparse_gemm_pair_kernel": (983140864 + 5710080, ("mvue_gemm.cu", "mvue_tma.h", "mvue_internal.h"),
-                                "af3ecf5baf4a736b"),
-    "prune_axis0_bf16_kernel/table": (103502080 + 26827520,
-                                      ("mvue_prune.cu", "mvue_device.cuh", "mvue_tma.h", "mvue_internal.h"),
-                                      "383e6715b6c6e3ef"),
-    "prune_axis0_bf16_kernel/systematic": (103674368 + 26032128,
-                                           ("mvue_prune.cu", "mvue_device.cuh", "mvue_tma.h", "mvue_internal.h"),
-                                           "383e6715b6c6e3ef"),
+    "sparse_gemm_pair_kernel": (982858496 + 4140032, ("mvue_gemm.cu", "mvue_tma.h", "mvue_internal.h"),
+                                "dafb315d5888dc93"),
+    "prune_axis0_bf16_whole_tiles_kernel/table/16": (102795776 + 24107008,
+                                                     ("mvue_prune.cu", "mvue_device.cuh", "mvue_tma.h", "mvue_internal.h"),
+                                                     "e1a5a7e46ae8379f"),
+    "prune_axis0_bf16_whole_tiles_kernel/systematic/16": (102780672 + 22041856,
+                                                          ("mvue_prune.cu", "mvue_device.cuh", "mvue_tma.h",
+                                                           "mvue_internal.h"),
+                                                          "e1a5a7e46ae8379f"),
 }
 
 
@@ -522,8 +523,8 @@ def run_ours(args, cfg, n, m):
             # 200704 rows, ~240 flop/B) it is bound by streaming h from HBM, not by the tensor cores
             "roofline": hbm_roofline("sparse_gemm_pair_kernel", m_bytes, gemm_ms, peaks,
                                      ncu_traffic("sparse_gemm_pair_kernel", args.workload) if (n, m) == (2, 4) else None),
-            "roofline_prune": hbm_roofline("prune_axis0_bf16_kernel", p_bytes, prune_ms, peaks,
-                                           ncu_traffic("prune_axis0_bf16_kernel/" + args.joint, args.workload)
+            "roofline_prune": hbm_roofline("prune_axis0_bf16_whole_tiles_kernel", p_bytes, prune_ms, peaks,
+                                           ncu_traffic(f"prune_axis0_bf16_whole_tiles_kernel/{args.joint}/{16 if args.eps16 else 32}", args.workload)
                                            if (n, m) == (2, 4) else None),
         }
         if sustained is not None:
@@ -615,7 +616,7 @@ def ffn_768_case(tm: Timer, peaks, issue_cold, joint):
         du_mean, du_best = tm.each(lambda: torch.matmul(gT, h), 20)
         flops = 2.0 * n_out * n_in * T
         entry["prune_axis0_us"] = 1e3 * p_mean
-        entry["prune_axis0_roofline"] = hbm_roofline("prune_axis0_bf16_kernel", prune_bytes(T, n_out, 2), p_mean, peaks)
+        entry["prune_axis0_roofline"] = hbm_roofline("prune_axis0_bf16_whole_tiles_kernel", prune_bytes(T, n_out, 2), p_mean, peaks)
         entry["update_us"] = 1e3 * u_mean
         entry["update_us_best"] = 1e3 * u_best
         entry["update_roofline"] = tensor_roofline("sparse_gemm_pair_kernel", flops, u_mean, peaks, issue_cold)
@@ -683,7 +684,7 @@ def tensor_bound_case(tm: Timer, n, m, peaks, joint, issue_cold, base_opt=0):
     tf = flops / (gemm_ms * 1e-3) / 1e12
     return {"g": [T, out], "h": [T, inp], "prune": f"{n}:{m}",
             "timing": "back-to-back loop (inputs 470 MB / 134 MB per call, larger than L2)",
-            "prune_ms": prune_ms, "roofline_prune": hbm_roofline("prune_axis0_bf16_kernel", pb, prune_ms, peaks),
+            "prune_ms": prune_ms, "roofline_prune": hbm_roofline("prune_axis0_bf16_whole_tiles_kernel", pb, prune_ms, peaks),
             "prune_systematic_ms": sys_ms, "prune_systematic_frac_of_hbm_peak": pb / (sys_ms * 1e-3) / 1e9 / peaks["hbm_gbs"],
             "prune_table_ms": table_ms, "prune_table_frac_of_hbm_peak": pb / (table_ms * 1e-3) / 1e9 / peaks["hbm_gbs"],
             "prune_1of2_ms": one_two_ms, "prune_1of2_frac_of_hbm_peak": pb / (one_two_ms * 1e-3) / 1e9 / peaks["hbm_gbs"],
