@@ -166,8 +166,13 @@ __device__ __forceinline__ void ldg256_aligned(const char* p, uint32_t (&v)[8]) 
                  : "l"(p));
 }
 
+// Resident blocks per SM: eight (64 registers) where the arithmetic is short enough to fit them without spills that
+// cost more than the extra warps bring; six for the App. A.2 table and for 1:2 with its two generator calls per unit.
+template <int M, int kJoint, bool kEps16>
+constexpr int a1_pairs_min_blocks() { return ((M == 4 && kJoint == 0) || (M == 2 && !kEps16)) ? 6 : 8; }
+
 template <int M, bool kTC, int kJoint, bool kSR, bool kEps16>
-__global__ void __launch_bounds__(8 * kA1PairsPerBlock, 6)
+__global__ void __launch_bounds__(8 * kA1PairsPerBlock, a1_pairs_min_blocks<M, kJoint, kEps16>())
 prune_axis1_bf16_pairs_kernel(const void* __restrict__ g, int units_per_row, int64_t ld, int64_t units_per_row_total,
                               int64_t unit_offset, RoundKeys rk, uint4* __restrict__ values, uint16_t* __restrict__ meta) {
     const int j = threadIdx.x & 7;
