@@ -153,7 +153,9 @@ prune_axis1_kernel(const void* __restrict__ g, int64_t n_rows, int units_per_row
 
 // ---- axis 1, bf16, whole blocks ---------------------------------------------------
 // For tensors whose rows are a multiple of 16 and whose K is a multiple of 512 elements, 32-byte aligned (the packed
-// operands of the backward products).  A thread block owns 16 rows of A by 32 units; thread = (row % 8, unit pair)
+// operands of the backward products); a narrower K of 32, 64, 128 or 256 elements is taken too, the block then owning
+// 16, 8, 4 or 2 groups of 16 rows (`pair_shift` = log2 of the unit pairs of a row that one block covers, 4 for wide K).
+// A thread block owns 16 rows of A by 32 units; thread = (row % 8, unit pair)
 // handles the two consecutive units 2 c, 2 c + 1 of rows r and r + 8: 64 contiguous bytes per row (both rows requested
 // before either is pruned), a 32-byte store of survivors per row, two whole metadata words in tensor-core order.  No
 // bounds checks, half the addressing per unit, and with sixteen bits per block the two units of a row share one
@@ -174,10 +176,11 @@ constexpr int a1_pairs_min_blocks() { return ((M == 4 && kJoint == 0) || (M == 2
 template <int M, bool kTC, int kJoint, bool kSR, bool kEps16>
 __global__ void __launch_bounds__(8 * kA1PairsPerBlock, a1_pairs_min_blocks<M, kJoint, kEps16>())
 prune_axis1_bf16_pairs_kernel(const void* __restrict__ g, int units_per_row, int64_t ld, int64_t units_per_row_total,
-                              int64_t unit_offset, RoundKeys rk, uint4* __restrict__ values, uint16_t* __restrict__ meta) {
-    const int j = threadIdx.x & 7;
-    const int c = 2 * (blockIdx.y * kA1PairsPerBlock + (threadIdx.x >> 3));   // first unit of the pair
-    const int64_t r0 = (int64_t)blockIdx.x * 16 + j;
+                              int64_t unit_offset, RoundKeys rk, uint4* __restrict__ values, uint16_t* __restrict__ meta,
+                              int pair_shift) {
+    const int j = threadIdx.x & 7, q = threadIdx.x >> 3;
+    const int c = 2 * (blockIdx.y * kA1PairsPerBlock + (q & ((1 << pair_shift) - 1)));   // first unit of the pair
+    const int64_t r0 = ((((int64_t)blockIdx.x) << (4 - pair_shift)) + (q >> pair_shift)) * 16 + j;
     uint32_t raw[2][2][8];                                                    // [row h][unit][8 words]
 #pragma unroll
     for (int h = 0; h < 2; ++h) {
@@ -653,14 +656,17 @@ cudaError_t launch_prune_t(const PruneArgs& a, cudaStream_t stream) {
         const int64_t cover_rows = kTC ? ((a.rows + 127) / 128) * 128 : a.rows;
         // whole blocks of 16 rows x 32 units, 32-byte aligned rows and outputs, no padding rows of A to cover, and (for
         // sixteen bits per block) unit pairs that start on even unit numbers: the kernel without bounds checks
-        const bool whole = kBf16 && a.rows % 16 == 0 && upr % (2 * kA1PairsPerBlock) == 0 && cover_rows == a.rows &&
+        int pair_shift = 4;                                  // unit pairs of a row per block = 2^pair_shift
+        if (upr == 2 || upr == 4 || upr == 8 || upr == 16) pair_shift = upr == 2 ? 0 : upr == 4 ? 1 : upr == 8 ? 2 : 3;
+        const int64_t rows_per_block = 16 << (4 - pair_shift);
+        const bool whole = kBf16 && a.rows % rows_per_block == 0 && upr % (2 << pair_shift) == 0 && cover_rows == a.rows &&
                            (a.ld * 2) % 32 == 0 && reinterpret_cast<uintptr_t>(a.g) % 32 == 0 &&
                            reinterpret_cast<uintptr_t>(a.values) % 32 == 0 &&
                            (!kEps16 || UnitWords<M, kJoint>::kCount != 4 || (uoff % 2 == 0 && upr_total % 2 == 0));
         if (whole) {
-            dim3 grid_p((unsigned)(a.rows / 16), (unsigned)(upr / (2 * kA1PairsPerBlock)));
+            dim3 grid_p((unsigned)(a.rows / rows_per_block), (unsigned)(upr / (2 << pair_shift)));
             prune_axis1_bf16_pairs_kernel<M, kTC, kJoint, kSR, kEps16><<<grid_p, 8 * kA1PairsPerBlock, 0, stream>>>(
-                a.g, (int)upr, a.ld, upr_total, uoff, rk, values, meta);
+                a.g, (int)upr, a.ld, upr_total, uoff, rk, values, meta, pair_shift);
         } else {
             dim3 grid((unsigned)((cover_rows + 15) / 16), (unsigned)((upr + kA1Units - 1) / kA1Units));
             prune_axis1_kernel<M, kBf16, kTC, kJoint, kSR, kEps16><<<grid, 8 * kA1Units, 0, stream>>>(

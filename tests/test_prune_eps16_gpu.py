@@ -27,7 +27,7 @@ def gpu(g_np, n, m, joint, axis, seed, options=E16, **kw):
     return values.view(torch.int16).cpu().numpy().view(np.uint16), meta.cpu().numpy()
 
 
-SHAPES = [(48, 80), (528, 264), (256, 192), (1152, 320), (176, 1536)]        # ragged; whole 128 x 64 tiles (a kernel of its own down the rows)
+SHAPES = [(48, 80), (528, 264), (256, 192), (1152, 320), (176, 1536), (512, 256), (384, 64)]        # ragged; whole 128 x 64 tiles (a kernel of its own down the rows)
 
 
 @pytest.mark.parametrize("n,m,joint", ESTIMATORS)

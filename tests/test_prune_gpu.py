@@ -39,7 +39,8 @@ MODES = [(1, 2), (2, 4), (1, 4)]
 # shapes span several thread blocks and leave ragged tails in both grid dimensions; the last three are made of whole
 # 128 x 64 tiles, which the bf16 prune down the rows handles with a kernel of its own; (4096, 1024) and (176, 1536) are
 # whole blocks of 16 rows x 512 columns, which the bf16 prune along the rows handles with a kernel of its own
-SHAPES = [(16, 16), (48, 80), (528, 264), (1040, 1000), (4096, 1024), (256, 192), (1152, 320), (176, 1536)]
+SHAPES = [(16, 16), (48, 80), (528, 264), (1040, 1000), (4096, 1024), (256, 192), (1152, 320), (176, 1536),
+          (512, 256), (256, 32), (384, 64), (192, 128)]      # narrow K along the rows: several row groups per block
 
 
 @pytest.mark.parametrize("n,m", MODES)

@@ -28,7 +28,7 @@ def gpu(g_np, n, m, joint, axis, seed, **kw):
 
 
 # ragged shapes (general kernels) and shapes of whole 128 x 64 tiles (the bf16 kernel of its own down the rows)
-SHAPES = [(48, 80), (528, 264), (256, 192), (1152, 320), (176, 1536)]
+SHAPES = [(48, 80), (528, 264), (256, 192), (1152, 320), (176, 1536), (512, 256), (384, 64)]
 
 
 @pytest.mark.parametrize("n,m,joint", ESTIMATORS)
