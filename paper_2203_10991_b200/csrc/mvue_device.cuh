@@ -388,6 +388,35 @@ __device__ __forceinline__ void mvue_2of4_sys_bf16_x2(uint32_t xa01, uint32_t xa
     }
 }
 
+// ---- App. A.2 pair table, bf16 source with K contiguous, gathered output ------------------------------------------
+// The same law and the same bits as mvue_2of4_bf16 (x01 = a0 | a1 << 16, x23 = a2 | a3 << 16), with the output stage
+// of the systematic law:
+//   sort key = the bf16 in the upper half, the position in the two lowest bits (the sign comes back with the gather);
+//   every survivor's new magnitude is max(|a|, D/4): D/4 for a survivor with p < 1 (then D/4 >= |a|, also after the
+//   roundings of pick_2of4: the sums only add non-negative terms, and in the uncapped case D/2 = fl(2 S3 - (S3 - a_4))
+//   cannot round below 2 a_4), |a| itself for the capped dominant element;
+//   so the two survivors are gathered in position order by one byte permute and raised to bf16(D/4) with one signed
+//   16-bit maximum per half.
+template <bool kSR = false>
+__device__ __forceinline__ void mvue_2of4_bf16_gather(uint32_t x01, uint32_t x23, uint32_t word, uint32_t* out,
+                                                      uint32_t* nibble, uint32_t rnd = 0u) {
+    const float f0 = __uint_as_float(__byte_perm(x01, 0u, 0x1054)), f1 = __uint_as_float(__byte_perm(x01, 1u, 0x3254));
+    const float f2 = __uint_as_float(__byte_perm(x23, 2u, 0x1054)), f3 = __uint_as_float(__byte_perm(x23, 3u, 0x3254));
+    const float lo01 = fminf(fabsf(f0), fabsf(f1)), hi01 = fmaxf(fabsf(f0), fabsf(f1));
+    const float lo23 = fminf(fabsf(f2), fabsf(f3)), hi23 = fmaxf(fabsf(f2), fabsf(f3));
+    const float k1 = fminf(lo01, lo23), mid_a = fmaxf(lo01, lo23);
+    const float mid_b = fminf(hi01, hi23), k4 = fmaxf(hi01, hi23);
+    const float k2 = fminf(mid_a, mid_b), k3 = fmaxf(mid_a, mid_b);
+    const Pick24<float> r = pick_2of4(
+        k1, k2, k3, k4, word,
+        [](float k) { return __uint_as_float(__float_as_uint(k) & 0xFFFF0000u); });
+    const uint32_t pa = __float_as_uint(r.key_a) & 3u, pb = __float_as_uint(r.key_b) & 3u;
+    const uint32_t i = min(pa, pb), j = max(pa, pb);
+    const uint32_t raw = __byte_perm(x01, x23, 0x1010u + 0x22u * i + 0x2200u * j);
+    *out = __vmaxs2(raw, pack_out<kSR>(r.va, r.va, rnd) | (raw & 0x80008000u));
+    *nibble = i + 4u * j;
+}
+
 // binary32 source: b0..b3 are the raw bit patterns.
 template <bool kSR = false>
 __device__ __forceinline__ void mvue_2of4_sys_f32(uint32_t b0, uint32_t b1, uint32_t b2, uint32_t b3,
@@ -714,8 +743,7 @@ __device__ __forceinline__ void prune_unit_bf16_w(const uint32_t (&raw)[8], cons
 #pragma unroll
         for (int j = 0; j < 4; ++j) {
             uint32_t nib;
-            mvue_2of4_bf16<false, true, false, true, kSR>(raw[2 * j], raw[2 * j], raw[2 * j + 1], raw[2 * j + 1],
-                                                          words[j], &v[j], &nib, rnd[j]);
+            mvue_2of4_bf16_gather<kSR>(raw[2 * j], raw[2 * j + 1], words[j], &v[j], &nib, rnd[j]);
             meta += nib << (4 * j);
         }
     } else {
