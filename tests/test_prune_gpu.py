@@ -40,7 +40,8 @@ MODES = [(1, 2), (2, 4), (1, 4)]
 # 128 x 64 tiles, which the bf16 prune down the rows handles with a kernel of its own; (4096, 1024) and (176, 1536) are
 # whole blocks of 16 rows x 512 columns, which the bf16 prune along the rows handles with a kernel of its own
 SHAPES = [(16, 16), (48, 80), (528, 264), (1040, 1000), (4096, 1024), (256, 192), (1152, 320), (176, 1536),
-          (512, 256), (256, 32), (384, 64), (192, 128)]      # narrow K along the rows: several row groups per block
+          (512, 256), (256, 32), (384, 64), (192, 128),      # narrow K along the rows: several row groups per block
+          (256, 768), (128, 640), (256, 576), (384, 1536)]   # down the rows: 12, 10, 9, 24 column tiles (tile walk orders)
 
 
 @pytest.mark.parametrize("n,m", MODES)
@@ -212,7 +213,8 @@ def test_full_size_configs_sampled(name, n, m):
 
 @pytest.mark.parametrize("n,m", MODES)
 @pytest.mark.parametrize("axis", [0, 1])
-@pytest.mark.parametrize("shape", [(128, 128), (384, 200), (1024, 136), (2048, 1000), (4096, 1024)])
+@pytest.mark.parametrize("shape", [(128, 128), (384, 200), (1024, 136), (2048, 1000), (4096, 1024), (256, 768), (128, 640),
+                                   (256, 1152)])
 @pytest.mark.parametrize("dtype", ["bf16", "f32"])
 def test_tensor_core_metadata_order(n, m, axis, shape, dtype):
     """layout = MVUE_LAYOUT_TC: same survivors, metadata bit-identical to the oracle's once carried into
