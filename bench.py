@@ -986,7 +986,7 @@ def main():
         return
     if args.gpus > 1 and "WORLD_SIZE" not in os.environ:
         sys.exit(spawn_ranks(args))
-    args.steps = 1000 if args.steps is None else args.steps
+    args.steps = 200 if args.steps is None else args.steps
     run_ours(args, cfg, n, m)
 
 
