@@ -260,3 +260,38 @@ def test_the_comparison_with_the_appendix_has_power():
         assert which == mistake
         assert slips > 2 ** 24 // 50
         assert oracle.sweep_2of4_cases(a32)[1] <= PAIR_SLIPS_PER_BLOCK
+
+
+@pytest.mark.parametrize("joint", [oracle.JOINT_TABLE, oracle.JOINT_SYSTEMATIC])
+@pytest.mark.parametrize("dist,seed", [("student_t", 3), ("relu_lognormal", 4), ("tile", 5)])
+def test_survivors_are_their_own_value_or_one_common_raised_value(joint, dist, seed):
+    """Sec. 4.2: a survivor becomes a_i / p_i, which is one common magnitude (half the clipped sum) for every survivor
+    with p_i < 1 and the element itself when p_i = 1.  So in every bf16 block, with H = the smaller of the two stored
+    magnitudes, each survivor stores max(|a_i|, H), with its own sign: no stored value is below its element, and two
+    survivors that were both raised store the same magnitude.  (The CUDA kernels gather the survivors by position and
+    raise them with one maximum against the rounded common value; this is the property that makes that exact.)"""
+    from paper_2203_10991_b200 import workloads as gen
+    rows, K = 256, 512
+    if dist == "tile":      # adversarial blocks: ties, zeros, dominant elements, neighbours in bf16, tiny and huge scales
+        pats = np.array([[1, 1, 1, 1], [0, 0, 0, 3], [0, 2, 0, 0], [1, 2, 3, 7], [1, 2, 3, 6], [1, 2, 3, 5.96875],
+                         [1, 1.0078125, 1, 1.0078125], [0, 0, 5, 5], [1e-38, 2e-38, 3e-38, 1e-37],
+                         [3e38, 1e38, 2e38, 3e38], [0, 0, 0, 0], [1, -1, 1, -1], [-4, 1, 0.5, 0.25],
+                         [2 ** -126, 2 ** -127, 2 ** -130, 2 ** -133], [7, 0, 0, 7], [1, 255, 256, 257]], dtype=np.float32)
+        g32 = np.tile(pats.reshape(-1), rows * K // pats.size + 1)[:rows * K].reshape(rows, K)
+        g = oracle.bf16_rne(g32[:1]).repeat(rows, axis=0)                     # every pattern is a bf16 number already
+    else:
+        g = gen.gradient((rows, K), dist, seed, dtype="bf16")
+    values, meta = oracle.prune(g, 2, 4, axis=1, seed=seed, joint=joint)
+    a = (g & 0x7FFF).astype(np.int64).reshape(rows, K // 4, 4)              # magnitudes as ordered integers
+    nib = np.stack([meta & 15, meta >> 4], axis=-1).reshape(rows, K // 4)   # block j: low nibble first
+    i0, i1 = nib & 3, nib >> 2
+    assert (i0 < i1).all()
+    v = values.reshape(rows, K // 4, 2)
+    own = np.stack([np.take_along_axis(a, i0[..., None], 2)[..., 0], np.take_along_axis(a, i1[..., None], 2)[..., 0]], -1)
+    sign_in = np.stack([np.take_along_axis(g.reshape(rows, K // 4, 4), i0[..., None], 2)[..., 0],
+                        np.take_along_axis(g.reshape(rows, K // 4, 4), i1[..., None], 2)[..., 0]], -1) & 0x8000
+    out = (v & 0x7FFF).astype(np.int64)
+    assert ((v & 0x8000) == sign_in).all()
+    H = out.min(axis=-1, keepdims=True)
+    assert (out == np.maximum(own, H)).all()
+    assert (out != own).any() and (out == own).any()                        # both kinds occur in the sample
