@@ -914,12 +914,17 @@ def chain_case(n, m):
         chain.backward_update(g_top, layers, n, m, base_seed=1, joint=binding.MVUE_JOINT_SYSTEMATIC, overlap=True,
                               prune_in_epilogue_min_k=4096)
 
+    def run_sys16_epilogue():
+        chain.backward_update(g_top, layers, n, m, base_seed=1, joint=binding.MVUE_JOINT_SYSTEMATIC, overlap=True,
+                              prune_in_epilogue_min_k=4096, options=binding.MVUE_OPT_EPS16)
+
     eager_ms = timed(run_table, 5)
     table_ms = timed(graphed(run_table), 10)
     sys_ms = timed(graphed(run_sys), 10) if m == 4 else None
     overlap_ms = timed(graphed(run_sys_overlap), 10) if m == 4 else None
     epilogue_ms = timed(graphed(run_sys_epilogue), 10) if m == 4 else None
     sys16_ms = timed(graphed(run_sys16_overlap), 10) if m == 4 else None
+    sys16_epilogue_ms = timed(graphed(run_sys16_epilogue), 10) if m == 4 else None
     dense_ms = timed(graphed(dense_chain), 10)
     n_layers = len(layers)
     flops = 2.0 * T * d * d_ff * (2 * n_layers - 1)         # update product per layer, backward for all but the bottom
@@ -938,6 +943,7 @@ def chain_case(n, m):
             # the two-stream chain with sixteen random bits per block (one generator call per eight blocks)
             "systematic_16bit_two_stream_ms": sys16_ms,
             "systematic_16bit_two_stream_tflops_effective": None if sys16_ms is None else flops / (sys16_ms * 1e-3) / 1e12,
+            "systematic_16bit_two_stream_epilogue_prune_ms": sys16_epilogue_ms,
             "dense_torch_ms": dense_ms, "dense_torch_tflops": flops / (dense_ms * 1e-3) / 1e12}
 
 

@@ -259,23 +259,26 @@ MVUE_API int mvue_sparse_backward_gemm(const void* values, const void* meta, int
 /* The backward product that hands its result on already pruned (Sec. 1, backward equation: the g_l it produces is
  * the gradient the next layer down prunes again for its own backward product):
  *   dh[T x in] = (theta(g)[T x out] . W[out x in]) * act_grad[T x in]            (bf16, as mvue_sparse_backward_gemm)
- *   (next_values, next_meta) = mvue_prune_joint(dh, 2:4, axis 1, next_seed, k_total = in, k_offset = 0,
- *                                               MVUE_LAYOUT_TC, next_joint)
+ *   (next_values, next_meta) = mvue_prune_opts(dh, 2:4, axis 1, next_seed, k_total = in, k_offset = 0,
+ *                                              MVUE_LAYOUT_TC, next_joint, next_options)
  * in ONE launch: in the epilogue a thread holds one row of the output tile, 128 consecutive columns as bf16 -- eight
  * prune units in the form they have when K is contiguous -- and prunes them in registers before the dense tile is
  * stored, so dh is not read back for this prune.  The packed output is bit-identical to the separate call on the
  * stored dh.  dh itself is still written (the update product's prune, down the token axis, needs it).
- * next_joint: MVUE_JOINT_TABLE or MVUE_JOINT_SYSTEMATIC.  act_grad is required; in must be a multiple of 128.
- * When the product has to be split along K (small outputs, see mvue_gemm_workspace_bytes) or T is not a multiple of
- * 128, the entry point runs the two steps one after the other instead -- same results.  The epilogue costs ~2000
+ * next_joint: MVUE_JOINT_TABLE or MVUE_JOINT_SYSTEMATIC; next_options: mvue_prune_option bits (another bit:
+ * MVUE_ERR_OPTION).  act_grad is required; in must be a multiple of 128.
+ * When the product has to be split along K (small outputs, see mvue_gemm_workspace_bytes), T is not a multiple of
+ * 128, or MVUE_OPT_STOCHASTIC_ROUNDING is asked for, the entry point runs the two steps one after the other instead
+ * -- same results.  The epilogue costs ~2000
  * instructions per thread and tile: it hides under main loops of K = out >= 4096 and slows products with a short K,
  * where the separate calls are the better choice.  Other arguments, workspace, dev_status and errors as
  * mvue_sparse_backward_gemm. */
 MVUE_API int mvue_sparse_backward_gemm_pruned(const void* values, const void* meta, int layout, int64_t T,
                                               int64_t out, const void* W, int64_t in, int64_t ldW,
                                               const void* act_grad, void* dh, int64_t lddh, uint64_t next_seed,
-                                              int next_joint, void* next_values, void* next_meta, void* workspace,
-                                              size_t workspace_bytes, int* dev_status, void* stream);
+                                              int next_joint, unsigned next_options, void* next_values,
+                                              void* next_meta, void* workspace, size_t workspace_bytes,
+                                              int* dev_status, void* stream);
 
 /* Prune fused into the update product (Sec. 4.1 / 4.2 + App. A.2 applied to g along the
  * token axis, then the update equation of Sec. 1) in ONE kernel:

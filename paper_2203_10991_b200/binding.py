@@ -60,8 +60,8 @@ def lib() -> ctypes.CDLL:
                                               ctypes.c_size_t, vp, vp]
         L.mvue_sparse_backward_gemm.argtypes = [vp, vp, ci, i64, i64, vp, i64, i64, vp, vp, ci, i64, vp,
                                                 ctypes.c_size_t, vp, vp]
-        L.mvue_sparse_backward_gemm_pruned.argtypes = [vp, vp, ci, i64, i64, vp, i64, i64, vp, vp, i64, u64, ci, vp, vp,
-                                                       vp, ctypes.c_size_t, vp, vp]
+        L.mvue_sparse_backward_gemm_pruned.argtypes = [vp, vp, ci, i64, i64, vp, i64, i64, vp, vp, i64, u64, ci,
+                                                       ctypes.c_uint, vp, vp, vp, ctypes.c_size_t, vp, vp]
         L.mvue_gemm_workspace_bytes.argtypes = [ci, i64, i64, i64, szp]
         L.mvue_fused_update_gemm.argtypes = [vp, ci, i64, i64, i64, ci, ci, u64, vp, i64, i64, vp, ci, i64, ci, vp,
                                              ctypes.c_size_t, vp, vp]
@@ -211,11 +211,12 @@ def mvue_sparse_backward_gemm(values: torch.Tensor, meta: torch.Tensor, W: torch
 
 
 def mvue_sparse_backward_gemm_pruned(values: torch.Tensor, meta: torch.Tensor, W: torch.Tensor, act_grad: torch.Tensor,
-                                     next_seed: int, *, next_joint: int = MVUE_JOINT_TABLE,
+                                     next_seed: int, *, next_joint: int = MVUE_JOINT_TABLE, next_options: int = MVUE_OPT_NONE,
                                      workspace: torch.Tensor | None = None, dev_status: torch.Tensor | None = None,
                                      layout: int = MVUE_LAYOUT_TC):
     """dh = (theta(g) . W) * act_grad (bf16) and, from the same launch, dh pruned 2:4 along its columns in tensor-core
-    order (what mvue_prune(dh, 2, 4, axis=1, next_seed, layout=MVUE_LAYOUT_TC, joint=next_joint) gives).
+    order (what mvue_prune(dh, 2, 4, axis=1, next_seed, layout=MVUE_LAYOUT_TC, joint=next_joint,
+    options=next_options) gives).
     Returns (dh, next_values, next_meta)."""
     T, half_o = values.shape
     n_out, n_in = W.shape
@@ -228,7 +229,7 @@ def mvue_sparse_backward_gemm_pruned(values: torch.Tensor, meta: torch.Tensor, W
     ws, ws_bytes = _workspace(1, T, n_in, n_out, W.device, workspace)
     _check(lib().mvue_sparse_backward_gemm_pruned(values.data_ptr(), meta.data_ptr(), layout, T, n_out, W.data_ptr(), n_in,
                                                   W.stride(0), act_grad.data_ptr(), out.data_ptr(), out.stride(0),
-                                                  next_seed & (2**64 - 1), int(next_joint), next_values.data_ptr(),
+                                                  next_seed & (2**64 - 1), int(next_joint), int(next_options), next_values.data_ptr(),
                                                   next_meta.data_ptr(), None if ws is None else ws.data_ptr(), ws_bytes,
                                                   None if dev_status is None else dev_status.data_ptr(), _stream_ptr()),
            "mvue_sparse_backward_gemm_pruned")

@@ -33,7 +33,7 @@ def backward_update(g_top: torch.Tensor, layers, n: int = 2, m: int = 4, base_se
     the features fit on the same SMs.  Same calls, same seeds, same results; the streams join before each backward
     product and before returning.
     options: mvue_prune_option bits handed to every prune (stochastic rounding, sixteen random bits per block).
-    prune_in_epilogue_min_k: when set (2:4 only, options 0), a backward product whose reduction axis (the layer's out) is at least
+    prune_in_epilogue_min_k: when set (2:4 only), a backward product whose reduction axis (the layer's out) is at least
     this long also prunes its own output along the features in its epilogue (mvue_sparse_backward_gemm_pruned), with
     the seed the layer below would have used, so that layer's prune along the features is not launched.  Same bits.
     Returns the list of dW (fp32), top layer first."""
@@ -45,11 +45,12 @@ def backward_update(g_top: torch.Tensor, layers, n: int = 2, m: int = 4, base_se
     def backward(i, L, values_b, meta_b):
         nonlocal ready
         below = layers[i + 1] if i + 1 < len(layers) else None
-        if (prune_in_epilogue_min_k is not None and options == 0 and (n, m) == (2, 4) and L["W"].shape[0] >= prune_in_epilogue_min_k
+        if (prune_in_epilogue_min_k is not None and (n, m) == (2, 4) and L["W"].shape[0] >= prune_in_epilogue_min_k
                 and below is not None and below.get("act_grad") is not None and L["W"].shape[1] % 128 == 0
                 and fuse_joint in (binding.MVUE_JOINT_TABLE, binding.MVUE_JOINT_SYSTEMATIC)):
             g_next, nv, nm = binding.mvue_sparse_backward_gemm_pruned(values_b, meta_b, L["W"], L["act_grad"],
-                                                                      layer_seeds(base_seed, i + 1)[1], next_joint=fuse_joint)
+                                                                      layer_seeds(base_seed, i + 1)[1], next_joint=fuse_joint,
+                                                                      next_options=options)
             ready = (nv, nm)
             return g_next
         ready = None

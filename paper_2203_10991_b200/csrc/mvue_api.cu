@@ -84,7 +84,7 @@ using namespace mvue;
 
 extern "C" {
 
-int mvue_version(void) { return 130; }   // 1.3: stochastic rounding of survivors, per-device set-up, the bounded-wait self-test
+int mvue_version(void) { return 140; }   // 1.4: prune options on the backward product that prunes its own output
 
 const char* mvue_status_string(int status) {
     switch (status) {
@@ -224,11 +224,13 @@ int mvue_sparse_backward_gemm(const void* values, const void* meta, int layout, 
 
 int mvue_sparse_backward_gemm_pruned(const void* values, const void* meta, int layout, int64_t T, int64_t out,
                                      const void* W, int64_t in, int64_t ldW, const void* act_grad, void* dh,
-                                     int64_t lddh, uint64_t next_seed, int next_joint, void* next_values,
-                                     void* next_meta, void* workspace, size_t workspace_bytes, int* dev_status,
-                                     void* stream) {
+                                     int64_t lddh, uint64_t next_seed, int next_joint, unsigned next_options,
+                                     void* next_values, void* next_meta, void* workspace, size_t workspace_bytes,
+                                     int* dev_status, void* stream) {
     if (!act_grad || !next_values || !next_meta) return MVUE_ERR_NULL;
     if (next_joint != MVUE_JOINT_TABLE && next_joint != MVUE_JOINT_SYSTEMATIC) return MVUE_ERR_JOINT;
+    if (next_options & ~(unsigned)(MVUE_OPT_STOCHASTIC_ROUNDING | MVUE_OPT_EPS16)) return MVUE_ERR_OPTION;
+    const bool next_sr = (next_options & MVUE_OPT_STOCHASTIC_ROUNDING) != 0, next_eps16 = (next_options & MVUE_OPT_EPS16) != 0;
     if (in % 128 != 0) return MVUE_ERR_SHAPE;                      // K of the next product, tensor-core order
     if (!aligned16(next_values) || !aligned16(next_meta)) return MVUE_ERR_ALIGN;
     DeviceInfo dev;
@@ -238,17 +240,21 @@ int mvue_sparse_backward_gemm_pruned(const void* values, const void* meta, int l
     if (workspace && !aligned16(workspace)) return MVUE_ERR_WORKSPACE;
     SparseGemmArgs a{values, meta, T, in, out, W, ldW, dh, lddh, 1, 0, act_grad, workspace,
                      workspace ? workspace_bytes : 0, dev_status, dev.sm_count};
-    if (need == 0 && T % 128 == 0) {                                // one launch: the prune rides in the epilogue
+    if (need == 0 && T % 128 == 0 && !next_sr) {                    // one launch: the prune rides in the epilogue
         a.next_values = next_values;
         a.next_meta = next_meta;
         a.next_seed = next_seed;
         a.next_joint = next_joint;
+        a.next_eps16 = next_eps16;
         return launch_sparse_gemm(a, reinterpret_cast<cudaStream_t>(stream));
     }
-    // a product split along K (its tiles are partial sums) or with a ragged last row block: the two steps one after the other
+    // a product split along K (its tiles are partial sums), a ragged last row block, or stochastic rounding (its extra
+    // generator call per unit has no room in the epilogue's registers): the two steps one after the other
     if (int s = launch_sparse_gemm(a, reinterpret_cast<cudaStream_t>(stream))) return s;
     if (T % 8 != 0) return MVUE_ERR_SHAPE;
     PruneArgs pa{dh, true, T, in, lddh, 4, 1, next_seed, in, 0, next_values, next_meta, dev.sm_count, true, next_joint};
+    pa.stochastic_rounding = next_sr;
+    pa.eps16 = next_eps16;
     cudaError_t e = launch_prune(pa, reinterpret_cast<cudaStream_t>(stream));
     if (e != cudaSuccess) { set_cuda_error(e, "mvue_sparse_backward_gemm_pruned prune launch"); return MVUE_ERR_CUDA; }
     return MVUE_OK;

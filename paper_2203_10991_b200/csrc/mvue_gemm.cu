@@ -401,6 +401,7 @@ __device__ __forceinline__ void quad_transpose(uint32_t (&v)[64], int lane) {
 //         unit has when K is contiguous -- is pruned in registers (5: systematic sampling, 6: App. A.2 table) and its
 //         survivors and metadata stored before the dense tile goes out: the output of the backward product (Sec. 1,
 //         backward equation) leaves already pruned along the next backward product's reduction axis
+//   7, 8: as 5, 6 with sixteen random bits per block (two units share one generator call)
 // The scale factors of a row are fetched into registers under the main loop.
 template <int kMode>
 __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(kMode == 4 ? 1024 : kThreads, 1)
@@ -596,7 +597,9 @@ sparse_gemm_pair_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_
             }
             // bf16 x scale keeps the row's factors in registers; fp32 x scale has no room for them beside 128
             // fp32 results and applies them after tensor memory has been handed back
-            constexpr bool kPrune = kMode == 5 || kMode == 6;
+            constexpr bool kPrune = kMode >= 5 && kMode <= 8;             // 5, 7: systematic sampling; 6, 8: App. A.2 table
+            constexpr int kPruneJoint = (kMode == 5 || kMode == 7) ? 1 : 0;
+            constexpr bool kPruneEps16 = kMode >= 7;                       // 7, 8: sixteen random bits per block
             constexpr bool kScale = kMode == 2 || kPrune, kLateScale = kMode == 3, kToBf16 = kMode == 1 || kScale;
             // bf16 outputs and their factors move in the quad-transposed arrangement (quad_transpose): lane
             // 4 a + b reads / writes, for c = 0..3 and k = 0, 1, the 32-byte chunk b + 4 k of row 4 a + c of the warp's
@@ -681,15 +684,26 @@ sparse_gemm_pair_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_
                     const int64_t upr = p.N >> 4, strip0 = col0 >> 4;
                     uint4* vdst = p.next_values + row * upr + strip0;
 #pragma unroll
-                    for (int t = 0; t < 8; ++t) {
-                        uint32_t raw[8];
+                    for (int t = 0; t < 8; t += 2) {                     // units 2i, 2i + 1 (strip0 + t is even)
+                        uint32_t raw0[8], raw1[8];
 #pragma unroll
-                        for (int e = 0; e < 8; ++e) raw[e] = r[8 * t + e];
-                        uint4 v;
-                        uint32_t mt;
-                        prune_unit_bf16<4, kMode == 5 ? 1 : 0>(raw, (uint64_t)(row * upr + strip0 + t), p.next_rk, &v, &mt);
-                        vdst[t] = v;
-                        *reinterpret_cast<uint16_t*>(p.next_meta + tc_meta_offset(row, strip0 + t, p.N >> 7)) = (uint16_t)mt;
+                        for (int e = 0; e < 8; ++e) { raw0[e] = r[8 * t + e]; raw1[e] = r[8 * t + 8 + e]; }
+                        const uint64_t unit = (uint64_t)(row * upr + strip0 + t);
+                        uint4 v0, v1;
+                        uint32_t mt0, mt1;
+                        if constexpr (kPruneEps16) {                      // the two units share one generator call
+                            uint32_t w0[4], w1[4];
+                            unit_pair_words16(unit, p.next_rk, w0, w1);
+                            prune_unit_bf16_w<4, kPruneJoint, false>(raw0, w0, unit, p.next_rk, &v0, &mt0);
+                            prune_unit_bf16_w<4, kPruneJoint, false>(raw1, w1, unit + 1, p.next_rk, &v1, &mt1);
+                        } else {
+                            prune_unit_bf16<4, kPruneJoint>(raw0, unit, p.next_rk, &v0, &mt0);
+                            prune_unit_bf16<4, kPruneJoint>(raw1, unit + 1, p.next_rk, &v1, &mt1);
+                        }
+                        vdst[t] = v0;
+                        vdst[t + 1] = v1;
+                        *reinterpret_cast<uint16_t*>(p.next_meta + tc_meta_offset(row, strip0 + t, p.N >> 7)) = (uint16_t)mt0;
+                        *reinterpret_cast<uint16_t*>(p.next_meta + tc_meta_offset(row, strip0 + t + 1, p.N >> 7)) = (uint16_t)mt1;
                     }
                 }
             }
@@ -1175,15 +1189,17 @@ PairKernelSetup& pair_setup() {
 cudaError_t pair_kernel_setup() {
     PairKernelSetup& st = pair_setup();
     return once_per_device(st.once, [&st](int dev) {
-        const void* kernels[7] = {reinterpret_cast<const void*>(sparse_gemm_pair_kernel<0>),
+        const void* kernels[9] = {reinterpret_cast<const void*>(sparse_gemm_pair_kernel<0>),
                                   reinterpret_cast<const void*>(sparse_gemm_pair_kernel<1>),
                                   reinterpret_cast<const void*>(sparse_gemm_pair_kernel<2>),
                                   reinterpret_cast<const void*>(sparse_gemm_pair_kernel<3>),
                                   reinterpret_cast<const void*>(sparse_gemm_pair_kernel<4>),
                                   reinterpret_cast<const void*>(sparse_gemm_pair_kernel<5>),
-                                  reinterpret_cast<const void*>(sparse_gemm_pair_kernel<6>)};
+                                  reinterpret_cast<const void*>(sparse_gemm_pair_kernel<6>),
+                                  reinterpret_cast<const void*>(sparse_gemm_pair_kernel<7>),
+                                  reinterpret_cast<const void*>(sparse_gemm_pair_kernel<8>)};
         cudaError_t err = cudaSuccess;
-        for (int i = 0; i < 7 && err == cudaSuccess; ++i)
+        for (int i = 0; i < 9 && err == cudaSuccess; ++i)
             err = cudaFuncSetAttribute(kernels[i], cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemBytes);
         cudaLaunchConfig_t cfg = {};
         cfg.gridDim = dim3(2, 1, 1);
@@ -1419,8 +1435,12 @@ int launch_sparse_gemm(const SparseGemmArgs& a, cudaStream_t stream) {
     const bool long_items = item_steps >= 32;
     if (a.next_values != nullptr) {
         if (!(scaled && to_bf16)) return MVUE_ERR_SHAPE;         // (the caller routes split products elsewhere)
-        if (a.next_joint == 1)
+        if (a.next_joint == 1 && a.next_eps16)
+            sparse_gemm_pair_kernel<7><<<grid, kThreads, kSmemBytes, stream>>>(map_a, map_b, map_e, p);
+        else if (a.next_joint == 1)
             sparse_gemm_pair_kernel<5><<<grid, kThreads, kSmemBytes, stream>>>(map_a, map_b, map_e, p);
+        else if (a.next_eps16)
+            sparse_gemm_pair_kernel<8><<<grid, kThreads, kSmemBytes, stream>>>(map_a, map_b, map_e, p);
         else
             sparse_gemm_pair_kernel<6><<<grid, kThreads, kSmemBytes, stream>>>(map_a, map_b, map_e, p);
     } else if (scaled && to_bf16)

@@ -50,6 +50,7 @@ struct SparseGemmArgs {
     void* next_meta = nullptr;
     uint64_t next_seed = 0;
     int next_joint = 0;   // 0 = App. A.2 table, 1 = systematic sampling
+    bool next_eps16 = false;   // sixteen random bits per block for that prune
 };
 int launch_sparse_gemm(const SparseGemmArgs& a, cudaStream_t stream);     // returns an mvue_status
 // iters = 0: nothing is issued and the kernel's one wait expires after spin_limit polls (0: the default bound)
