@@ -16,6 +16,12 @@
 
 namespace mvue {
 
+// First statement of every kernel launched with launch_dependent(): returns once the grids this launch depends on have
+// completed and their stores are visible (at once when the kernel was launched the ordinary way).
+__device__ __forceinline__ void grid_dependency_wait() {
+    asm volatile("griddepcontrol.wait;" ::: "memory");
+}
+
 // ---------------------------------------------------------------------------
 // Philox4x32 with ten rounds (Salmon et al., SC'11).  The ten round keys depend
 // on the seed only, so the host expands them once and passes them by value; in

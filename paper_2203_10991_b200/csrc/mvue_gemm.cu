@@ -407,6 +407,7 @@ template <int kMode>
 __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(kMode == 4 ? 1024 : kThreads, 1)
 sparse_gemm_pair_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ CUtensorMap map_b,
                         const __grid_constant__ CUtensorMap map_e, const GemmParams p) {
+    grid_dependency_wait();
     extern __shared__ uint8_t smem_raw[];
     const uint32_t smem_base = (smem_u32(smem_raw) + 1023u) & ~1023u;
     uint8_t* smem_gen = smem_raw + (smem_base - smem_u32(smem_raw));
@@ -1033,6 +1034,7 @@ splitk_reduce_kernel(const float* __restrict__ partial, int splits, int64_t M, i
                      const __nv_bfloat16* __restrict__ scale, int c_is_bf16, int accumulate) {
     const int64_t n4 = N / 4;
     const int64_t total = M * n4;
+    grid_dependency_wait();
     for (int64_t i = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; i < total; i += (int64_t)gridDim.x * blockDim.x) {
         const int64_t r = i / n4, c = (i - r * n4) * 4;
         float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
@@ -1064,6 +1066,7 @@ splitk_reduce_kernel(const float* __restrict__ partial, int splits, int64_t M, i
 __global__ void __launch_bounds__(64)
 tail_reduce_kernel(const float* __restrict__ partial, int rem, int parts, int64_t n_main, int64_t M, int64_t N,
                    float* __restrict__ C, int64_t ldc, const __nv_bfloat16* __restrict__ scale, int accumulate) {
+    grid_dependency_wait();
     const int tile = blockIdx.x / (2 * BM), lr = blockIdx.x % (2 * BM);
     int64_t tile_m, tile_n;
     tile_of(M, N, n_main + tile, &tile_m, &tile_n);
@@ -1433,40 +1436,30 @@ int launch_sparse_gemm(const SparseGemmArgs& a, cudaStream_t stream) {
     // main loops of at least 32 stages (K = 4096) per work item: the small-footprint epilogue costs nothing there
     const int64_t item_steps = tail.parts > 1 ? steps / tail.parts : p.k_steps_per_split;
     const bool long_items = item_steps >= 32;
+    using PairKernel = void (*)(CUtensorMap, CUtensorMap, CUtensorMap, GemmParams);
+    PairKernel kernel;
     if (a.next_values != nullptr) {
         if (!(scaled && to_bf16)) return MVUE_ERR_SHAPE;         // (the caller routes split products elsewhere)
-        if (a.next_joint == 1 && a.next_eps16)
-            sparse_gemm_pair_kernel<7><<<grid, kThreads, kSmemBytes, stream>>>(map_a, map_b, map_e, p);
-        else if (a.next_joint == 1)
-            sparse_gemm_pair_kernel<5><<<grid, kThreads, kSmemBytes, stream>>>(map_a, map_b, map_e, p);
-        else if (a.next_eps16)
-            sparse_gemm_pair_kernel<8><<<grid, kThreads, kSmemBytes, stream>>>(map_a, map_b, map_e, p);
-        else
-            sparse_gemm_pair_kernel<6><<<grid, kThreads, kSmemBytes, stream>>>(map_a, map_b, map_e, p);
-    } else if (scaled && to_bf16)
-        sparse_gemm_pair_kernel<2><<<grid, kThreads, kSmemBytes, stream>>>(map_a, map_b, map_e, p);
-    else if (scaled)
-        sparse_gemm_pair_kernel<3><<<grid, kThreads, kSmemBytes, stream>>>(map_a, map_b, map_e, p);
-    else if (to_bf16)
-        sparse_gemm_pair_kernel<1><<<grid, kThreads, kSmemBytes, stream>>>(map_a, map_b, map_e, p);
-    else if (long_items)
-        sparse_gemm_pair_kernel<4><<<grid, kThreads, kSmemBytes, stream>>>(map_a, map_b, map_e, p);
-    else
-        sparse_gemm_pair_kernel<0><<<grid, kThreads, kSmemBytes, stream>>>(map_a, map_b, map_e, p);
-    cudaError_t e = cudaGetLastError();
+        kernel = a.next_joint == 1 ? (a.next_eps16 ? sparse_gemm_pair_kernel<7> : sparse_gemm_pair_kernel<5>)
+                                   : (a.next_eps16 ? sparse_gemm_pair_kernel<8> : sparse_gemm_pair_kernel<6>);
+    } else {
+        kernel = scaled && to_bf16 ? sparse_gemm_pair_kernel<2>
+               : scaled            ? sparse_gemm_pair_kernel<3>
+               : to_bf16           ? sparse_gemm_pair_kernel<1>
+               : long_items        ? sparse_gemm_pair_kernel<4> : sparse_gemm_pair_kernel<0>;
+    }
+    cudaError_t e = launch_dependent(kernel, grid, dim3(kThreads), kSmemBytes, stream, map_a, map_b, map_e, p);
     if (e == cudaSuccess && tail.parts > 1) {
-        tail_reduce_kernel<<<tail.rem * 2 * BM, BN / 4, 0, stream>>>(
-            p.tail_partial, tail.rem, tail.parts, tail.n_main, a.M, a.N, reinterpret_cast<float*>(a.C), a.ldc,
-            reinterpret_cast<const __nv_bfloat16*>(a.scale), a.accumulate);
-        e = cudaGetLastError();
+        e = launch_dependent(tail_reduce_kernel, dim3((unsigned)(tail.rem * 2 * BM)), dim3(BN / 4), 0, stream,
+                             p.tail_partial, tail.rem, tail.parts, tail.n_main, a.M, a.N, reinterpret_cast<float*>(a.C),
+                             a.ldc, reinterpret_cast<const __nv_bfloat16*>(a.scale), a.accumulate);
     }
     if (e == cudaSuccess && splits > 1) {
         const int64_t total = a.M * (a.N / 4);
         const int64_t want = (total + 255) / 256;
         const int blocks = (int)(want < (int64_t)a.sm_count * 8 ? want : (int64_t)a.sm_count * 8);
-        splitk_reduce_kernel<<<blocks, 256, 0, stream>>>(p.partial, splits, a.M, a.N, a.C, a.ldc, p.scale,
-                                                         a.c_is_bf16, a.accumulate);
-        e = cudaGetLastError();
+        e = launch_dependent(splitk_reduce_kernel, dim3((unsigned)blocks), dim3(256), 0, stream, p.partial, splits, a.M,
+                             a.N, a.C, a.ldc, p.scale, a.c_is_bf16, a.accumulate);
     }
     if (e != cudaSuccess) { set_cuda_error(e, "sparse GEMM launch"); return MVUE_ERR_CUDA; }
     return MVUE_OK;

@@ -89,6 +89,7 @@ __global__ void __launch_bounds__(8 * kA1Units, kBf16 ? 12 : 8)
 prune_axis1_kernel(const void* __restrict__ g, int64_t n_rows, int units_per_row, int64_t ld,
                    int64_t units_per_row_total, int64_t unit_offset, RoundKeys rk,
                    uint4* __restrict__ values, uint16_t* __restrict__ meta) {
+    grid_dependency_wait();
     const int j = threadIdx.x & 7;
     const int c = blockIdx.y * kA1Units + (threadIdx.x >> 3);
     if (c >= units_per_row) return;
@@ -178,6 +179,7 @@ __global__ void __launch_bounds__(8 * kA1PairsPerBlock, a1_pairs_min_blocks<M, k
 prune_axis1_bf16_pairs_kernel(const void* __restrict__ g, int units_per_row, int64_t ld, int64_t units_per_row_total,
                               int64_t unit_offset, RoundKeys rk, uint4* __restrict__ values, uint16_t* __restrict__ meta,
                               int pair_shift) {
+    grid_dependency_wait();
     const int j = threadIdx.x & 7, q = threadIdx.x >> 3;
     const int c = 2 * (blockIdx.y * kA1PairsPerBlock + (q & ((1 << pair_shift) - 1)));   // first unit of the pair
     const int64_t r0 = ((((int64_t)blockIdx.x) << (4 - pair_shift)) + (q >> pair_shift)) * 16 + j;
@@ -243,6 +245,7 @@ __global__ void __launch_bounds__(kTileStrips * 32, kBf16 ? 3 : 2)
 prune_axis0_kernel(const void* __restrict__ g, int64_t n_strips, int64_t n_cols, int64_t ld,
                    int64_t units_per_row_total, int64_t unit_offset, RoundKeys rk,
                    uint4* __restrict__ values, uint16_t* __restrict__ meta) {
+    grid_dependency_wait();
     constexpr int ES = kBf16 ? 2 : 4;
     constexpr int NT = kTileStrips * 32;
     __shared__ uint4 s_val[kTileCols * kTileStrips];
@@ -380,6 +383,7 @@ __global__ void __launch_bounds__(32 * kWarps, A0<kStrips, kWarps>::kBlocksPerSM
 prune_axis0_bf16_kernel(const __grid_constant__ CUtensorMap map_g, const void* __restrict__ g, int64_t n_strips,
                         int64_t n_cols, int64_t ld, int64_t units_per_row_total, int64_t unit_offset, RoundKeys rk,
                         uint4* __restrict__ values, uint16_t* __restrict__ meta) {
+    grid_dependency_wait();
     constexpr int kTileBytes = A0<kStrips, kWarps>::kTileBytes;
     constexpr int kQuads = kStrips / 4;                                      // groups of 4 strips per tile
     constexpr int kPairStride = kWarps / kQuads;                             // warps that share a group of 4 strips
@@ -485,6 +489,7 @@ __global__ void __launch_bounds__(32 * kWTWarps, 12)
 prune_axis0_bf16_whole_tiles_kernel(const __grid_constant__ CUtensorMap map_g, const void* __restrict__ g, int64_t n_strips,
                                     int64_t ld, int64_t units_per_row_total, int64_t unit_offset, RoundKeys rk,
                                     uint4* __restrict__ values, uint16_t* __restrict__ meta, int walk) {
+    grid_dependency_wait();
     __shared__ __align__(1024) unsigned char s_tile[kWTBytes];                // the 128-byte swizzle needs 1 KiB alignment
     __shared__ __align__(8) uint64_t s_bar;
     const uint32_t tile = smem_addr(s_tile), bar = smem_addr(&s_bar);
@@ -670,12 +675,13 @@ cudaError_t launch_prune_t(const PruneArgs& a, cudaStream_t stream) {
                            (!kEps16 || UnitWords<M, kJoint>::kCount != 4 || (uoff % 2 == 0 && upr_total % 2 == 0));
         if (whole) {
             dim3 grid_p((unsigned)(a.rows / rows_per_block), (unsigned)(upr / (2 << pair_shift)));
-            prune_axis1_bf16_pairs_kernel<M, kTC, kJoint, kSR, kEps16><<<grid_p, 8 * kA1PairsPerBlock, 0, stream>>>(
-                a.g, (int)upr, a.ld, upr_total, uoff, rk, values, meta, pair_shift);
+            launch_dependent(prune_axis1_bf16_pairs_kernel<M, kTC, kJoint, kSR, kEps16>, dim3(grid_p),
+                             dim3(8 * kA1PairsPerBlock), 0, stream, a.g, (int)upr, a.ld, upr_total, uoff, rk, values,
+                             meta, pair_shift);
         } else {
             dim3 grid((unsigned)((cover_rows + 15) / 16), (unsigned)((upr + kA1Units - 1) / kA1Units));
-            prune_axis1_kernel<M, kBf16, kTC, kJoint, kSR, kEps16><<<grid, 8 * kA1Units, 0, stream>>>(
-                a.g, a.rows, (int)upr, a.ld, upr_total, uoff, rk, values, meta);
+            launch_dependent(prune_axis1_kernel<M, kBf16, kTC, kJoint, kSR, kEps16>, dim3(grid), dim3(8 * kA1Units),
+                             0, stream, a.g, a.rows, (int)upr, a.ld, upr_total, uoff, rk, values, meta);
         }
     } else {
         const int64_t n_strips = a.rows / 16;
@@ -697,8 +703,9 @@ cudaError_t launch_prune_t(const PruneArgs& a, cudaStream_t stream) {
             // otherwise groups of 8, 4 or 2 column tiles (whichever divides their number), or row tiles fastest
             const int shift = row_tiles > (1u << 27) ? 0 : col_tiles % 8 == 0 ? 3 : col_tiles % 4 == 0 ? 2 : col_tiles % 2 == 0 ? 1 : 0;
             const dim3 grid_w = col_fast ? dim3(col_tiles, row_tiles) : dim3(row_tiles << shift, col_tiles >> shift);
-            prune_axis0_bf16_whole_tiles_kernel<M, kTC, kJoint, kSR, kEps16><<<grid_w, 32 * kWTWarps, 0, stream>>>(
-                map_g, a.g, n_strips, a.ld, upr_total, uoff, rk, values, meta, col_fast ? -1 : shift);
+            launch_dependent(prune_axis0_bf16_whole_tiles_kernel<M, kTC, kJoint, kSR, kEps16>, dim3(grid_w),
+                             dim3(32 * kWTWarps), 0, stream, map_g, a.g, n_strips, a.ld, upr_total, uoff, rk, values,
+                             meta, col_fast ? -1 : shift);
         } else if (kBf16) {
             CUtensorMap map_g;
             memset(&map_g, 0, sizeof(map_g));
@@ -712,11 +719,13 @@ cudaError_t launch_prune_t(const PruneArgs& a, cudaStream_t stream) {
             });
             if (attr_err != cudaSuccess) return attr_err;
             dim3 grid_b((unsigned)((n_strips + kS - 1) / kS), (unsigned)((cover_cols + kA0Cols - 1) / kA0Cols));
-            prune_axis0_bf16_kernel<M, kTC, kJoint, kSR, kEps16, kS, kW><<<grid_b, A0<kS, kW>::kThreads, A0<kS, kW>::kSmemBytes, stream>>>(
-                map_g, a.g, n_strips, a.cols, a.ld, upr_total, uoff, rk, values, meta);
+            launch_dependent(prune_axis0_bf16_kernel<M, kTC, kJoint, kSR, kEps16, kS, kW>, dim3(grid_b),
+                             dim3(A0<kS, kW>::kThreads), A0<kS, kW>::kSmemBytes, stream, map_g, a.g, n_strips, a.cols,
+                             a.ld, upr_total, uoff, rk, values, meta);
         } else {
-            prune_axis0_kernel<M, false, kTC, kJoint, kSR, kEps16><<<grid, kTileStrips * 32, 0, stream>>>(
-                a.g, n_strips, a.cols, a.ld, upr_total, uoff, rk, values, meta);
+            launch_dependent(prune_axis0_kernel<M, false, kTC, kJoint, kSR, kEps16>, dim3(grid),
+                             dim3(kTileStrips * 32), 0, stream, a.g, n_strips, a.cols, a.ld, upr_total, uoff, rk,
+                             values, meta);
         }
     }
     return cudaGetLastError();
