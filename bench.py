@@ -63,15 +63,15 @@ def gemm_bytes(M: int, N: int, K: int, c_bytes: int = 4, scale: bool = False) ->
 # each kernel (summaries under profiles/).  Each figure is tied to a digest of the sources the kernel is built
 # from: once those change the counters no longer describe the kernel and `traffic` is reported as null.
 NCU_TRAFFIC = {
-    "sparse_gemm_pair_kernel": (982863872 + 4129280, ("mvue_gemm.cu", "mvue_tma.h", "mvue_internal.h"),
-                                "66cf1d62b301a64c"),
-    "prune_axis0_bf16_whole_tiles_kernel/table/16": (102786560 + 26039040,
+    "sparse_gemm_pair_kernel": (982859520 + 4034048, ("mvue_gemm.cu", "mvue_tma.h", "mvue_internal.h"),
+                                "14864604f8e1a0f7"),
+    "prune_axis0_bf16_whole_tiles_kernel/table/16": (102822144 + 27183872,
                                                      ("mvue_prune.cu", "mvue_device.cuh", "mvue_tma.h", "mvue_internal.h"),
-                                                     "68447606fbe058ee"),
-    "prune_axis0_bf16_whole_tiles_kernel/systematic/16": (102778880 + 21218048,
+                                                     "03ff148a36b1cb8b"),
+    "prune_axis0_bf16_whole_tiles_kernel/systematic/16": (102779136 + 20355328,
                                                           ("mvue_prune.cu", "mvue_device.cuh", "mvue_tma.h",
                                                            "mvue_internal.h"),
-                                                          "68447606fbe058ee"),
+                                                          "03ff148a36b1cb8b"),
 }
 
 
