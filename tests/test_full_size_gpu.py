@@ -187,3 +187,43 @@ def test_prune_4gb_tensor_sampled(axis):
         del values, meta
     del g_dev
     torch.cuda.empty_cache()
+
+
+@pytest.mark.parametrize("axis", [0, 1])
+def test_prune_4gb_tensor_sampled_in_the_sweeps_configuration(axis):
+    """The same 4 GiB tensor as the bandwidth sweep launches it: systematic sampling, sixteen random bits per block,
+    metadata in tensor-core order (down the rows this is the whole-tile kernel walking groups of eight column tiles;
+    along the rows the whole-block kernel).  Seeded slices against the oracle: K shards of 128 rows down the rows,
+    single rows with their global block numbers along the rows."""
+    rows, cols, base_rows = 1 << 19, 4096, 1 << 15
+    base = workloads.gradient((base_rows, cols), "student_t", 5, dtype="bf16")
+    g_dev = to_dev(base).repeat(rows // base_rows, 1)
+    seed, joint = 1234, binding.MVUE_JOINT_SYSTEMATIC
+    values, meta = binding.mvue_prune(g_dev, 2, 4, axis, seed, layout=TC, joint=joint, options=binding.MVUE_OPT_EPS16)
+    torch.cuda.synchronize()
+    meta_flat = meta.reshape(-1)
+    rng = np.random.Generator(np.random.PCG64(8))
+    starts = sorted(set([0, rows - 128, rows // 2 - 128, rows // 2] + [int(x) * 128 for x in rng.integers(0, rows // 128, 6)]))
+    th = oracle.host_threads()
+    for lo in starts:
+        part = np.ascontiguousarray(base[np.arange(lo, lo + 128) % base_rows])
+        if axis == 0:          # A = g^T [cols x rows]: the K block lo / 128 of every row block of A
+            v_ref, m_ref = oracle.prune(part, 2, 4, axis=0, seed=seed, k_total=rows, k_offset=lo, joint=joint, eps16=True,
+                                        threads=th)
+            v_gpu = values.view(cols, rows // 2)[:, lo // 2:lo // 2 + 64].contiguous().view(torch.int16).cpu().numpy()
+            assert np.array_equal(v_gpu.view(np.uint16), v_ref), lo
+            kblocks, kb = rows // 128, lo // 128
+            blocks = torch.stack([meta_flat[(rb * kblocks + kb) * 2048:(rb * kblocks + kb + 1) * 2048]
+                                  for rb in range(cols // 128)]).cpu().numpy()
+            assert np.array_equal(layouts.tc_to_canonical(blocks, cols, 128), m_ref), lo
+        else:                  # A = g: the row block lo / 128 with all its K blocks is contiguous in tensor-core order
+            kblocks, rb = cols // 128, lo // 128
+            m_gpu = layouts.tc_to_canonical(meta_flat[rb * kblocks * 2048:(rb + 1) * kblocks * 2048].cpu().numpy(), 128, cols)
+            v_gpu = values.view(rows, cols // 2)[lo:lo + 128].view(torch.int16).cpu().numpy().view(np.uint16)
+            for r in (0, 7, 8, 64, 127):
+                v1, m1 = oracle.prune(np.ascontiguousarray(part[r:r + 1]), 2, 4, axis=1, seed=seed, joint=joint, eps16=True,
+                                      k_total=cols * (lo + r + 1), k_offset=cols * (lo + r))
+                assert np.array_equal(v_gpu[r], v1[0]), (lo, r)
+                assert np.array_equal(m_gpu[r], m1[0]), (lo, r)
+    del values, meta, g_dev
+    torch.cuda.empty_cache()
