@@ -227,3 +227,19 @@ def test_prune_4gb_tensor_sampled_in_the_sweeps_configuration(axis):
                 assert np.array_equal(m_gpu[r], m1[0]), (lo, r)
     del values, meta, g_dev
     torch.cuda.empty_cache()
+
+
+@pytest.mark.parametrize("name", ["conv_im2col", "ffn_large"])
+@pytest.mark.parametrize("axis", [0, 1])
+def test_bench_step_prune_full_size(name, axis):
+    """The prune exactly as `bench.py`'s step and riders launch it (systematic sampling, sixteen random bits per block,
+    tensor-core order), both orientations, on the whole tensor: every survivor and every metadata byte."""
+    cfg = workloads.CONFIGS[name]
+    T, n_out = cfg["T"], cfg["out"]
+    g = workloads.gradient((T, n_out), cfg["g_dist"], cfg["seed"], dtype="bf16")
+    seed, joint = 77, binding.MVUE_JOINT_SYSTEMATIC
+    values, meta = binding.mvue_prune(to_dev(g), 2, 4, axis, seed, layout=TC, joint=joint, options=binding.MVUE_OPT_EPS16)
+    torch.cuda.synchronize()
+    v_ref, m_ref = oracle.prune(g, 2, 4, axis=axis, seed=seed, joint=joint, eps16=True, threads=oracle.host_threads())
+    assert np.array_equal(values.view(torch.int16).cpu().numpy().view(np.uint16).reshape(v_ref.shape), v_ref)
+    assert np.array_equal(meta.cpu().numpy().reshape(-1), layouts.canonical_to_tc(m_ref))
