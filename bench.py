@@ -67,11 +67,11 @@ NCU_TRAFFIC = {
                                 "14864604f8e1a0f7"),
     "prune_axis0_bf16_whole_tiles_kernel/table/16": (102822144 + 27183872,
                                                      ("mvue_prune.cu", "mvue_device.cuh", "mvue_tma.h", "mvue_internal.h"),
-                                                     "03ff148a36b1cb8b"),
+                                                     "65483dfb9e3e781a"),
     "prune_axis0_bf16_whole_tiles_kernel/systematic/16": (102779136 + 20355328,
                                                           ("mvue_prune.cu", "mvue_device.cuh", "mvue_tma.h",
                                                            "mvue_internal.h"),
-                                                          "03ff148a36b1cb8b"),
+                                                          "65483dfb9e3e781a"),
 }
 
 

@@ -701,7 +701,8 @@ cudaError_t launch_prune_t(const PruneArgs& a, cudaStream_t stream) {
             const unsigned row_tiles = (unsigned)(a.rows / kWTRows), col_tiles = (unsigned)(a.cols / kWTCols);
             const bool col_fast = col_tiles <= 8 && row_tiles <= 65535u;    // (the second grid dimension is 16 bits wide)
             // otherwise groups of 8, 4 or 2 column tiles (whichever divides their number), or row tiles fastest
-            const int shift = row_tiles > (1u << 27) ? 0 : col_tiles % 8 == 0 ? 3 : col_tiles % 4 == 0 ? 2 : col_tiles % 2 == 0 ? 1 : 0;
+            const int shift = row_tiles > (1u << 27) ? 0
+                            : col_tiles % 8 == 0 ? 3 : col_tiles % 4 == 0 ? 2 : col_tiles % 2 == 0 ? 1 : 0;
             const dim3 grid_w = col_fast ? dim3(col_tiles, row_tiles) : dim3(row_tiles << shift, col_tiles >> shift);
             launch_dependent(prune_axis0_bf16_whole_tiles_kernel<M, kTC, kJoint, kSR, kEps16>, dim3(grid_w),
                              dim3(32 * kWTWarps), 0, stream, map_g, a.g, n_strips, a.ld, upr_total, uoff, rk, values,
