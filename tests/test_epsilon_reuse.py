@@ -1,5 +1,6 @@
 """Re-use of the random samples across iterations (App. "Pruning Overhead", Part 1): what re-using a seed changes and
-what it leaves alone, on the oracle.  The numbers of the full study (oracle/epsilon_reuse_study.py) are in the design doc."""
+what it leaves alone, on the oracle.  The full study is oracle/epsilon_reuse_study.py (run it to print its table);
+these tests assert its two statements on a short run."""
 import numpy as np
 
 from oracle import epsilon_reuse_study as study
